@@ -1,0 +1,179 @@
+"""ctypes front end of the CPU oracle (``gnnco_oracle.c``).  TEST INFRASTRUCTURE ONLY.
+
+Only tests, the smoke check and the benchmark's CPU-baseline leg may import this
+package.  It shares nothing with the CUDA library: it loads its own shared object,
+built by gcc from the C file beside it, and works on numpy arrays.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+import subprocess
+from typing import Dict, List, Optional, Sequence
+
+import numpy as np
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+_SRC = os.path.join(_HERE, "gnnco_oracle.c")
+_LIB = os.path.join(_HERE, "libgnnco_oracle.so")
+_lib = None
+
+OK, BAD_ARG, OUT_OF_RANGE, NOT_SIMPLE = 0, -1, -2, -3
+
+
+def build(force: bool = False) -> str:
+    """Compile the oracle next to its source (gcc -O2, no fast-math, OpenMP for the
+    outer loop over subgraphs)."""
+    if force or not os.path.exists(_LIB) or os.path.getmtime(_LIB) < os.path.getmtime(_SRC):
+        tmp = _LIB + ".tmp%d" % os.getpid()
+        subprocess.check_call(["gcc", "-O2", "-fopenmp", "-shared", "-fPIC", "-o", tmp, _SRC, "-lm"])
+        os.replace(tmp, _LIB)
+    return _LIB
+
+
+def _native():
+    global _lib
+    if _lib is None:
+        lib = ctypes.CDLL(build())
+        i64, i32, dbl, vp, flt = ctypes.c_int64, ctypes.c_int32, ctypes.c_double, ctypes.c_void_p, ctypes.c_float
+        lib.oracle_bookkeeping.argtypes = [i64, i64, vp, vp, vp, i32] + [vp] * 12
+        lib.oracle_bookkeeping.restype = ctypes.c_int
+        lib.oracle_subgraph_step.argtypes = [i32, vp, vp, i32, vp, vp, vp, dbl, dbl, dbl, vp, vp, vp, vp, vp, vp, vp]
+        lib.oracle_subgraph_step.restype = ctypes.c_int
+        lib.oracle_train_step.argtypes = [i64, i32, vp, vp, vp, i32, vp, i32, vp, vp, dbl, dbl, dbl,
+                                          vp, vp, vp, vp, vp, vp, vp, i32]
+        lib.oracle_train_step.restype = ctypes.c_int
+        lib.oracle_adam.argtypes = [i64, vp, vp, vp, vp, dbl, dbl, dbl, dbl, i64]
+        lib.oracle_adam.restype = None
+        lib.oracle_decode.argtypes = [i64, i32, vp, vp, vp, i64, vp, vp, vp, flt, vp, vp, vp, vp]
+        lib.oracle_decode.restype = None
+        _lib = lib
+    return _lib
+
+
+class OracleError(RuntimeError):
+    def __init__(self, code: int, what: str):
+        super().__init__("%s failed with status %d" % (what, code))
+        self.code = code
+
+
+def _ptr(a: Optional[np.ndarray]):
+    return None if a is None else a.ctypes.data
+
+
+def _ptr_array(arrs: Sequence[Optional[np.ndarray]]):
+    t = (ctypes.c_void_p * max(1, len(arrs)))()
+    for k, a in enumerate(arrs):
+        t[k] = None if a is None else a.ctypes.data
+    return t
+
+
+def bookkeeping(n: int, eu: np.ndarray, ev: np.ndarray, part: np.ndarray, S: int) -> Dict[str, np.ndarray]:
+    """Renumber nodes by (part, id), split edges into intra (CSR) and boundary (list)."""
+    eu = np.ascontiguousarray(eu, dtype=np.int32)
+    ev = np.ascontiguousarray(ev, dtype=np.int32)
+    part = np.ascontiguousarray(part, dtype=np.int32)
+    E = int(eu.size)
+    out = dict(
+        perm=np.empty(n, np.int32), inv_perm=np.empty(n, np.int32), part_ptr=np.empty(S + 1, np.int32),
+        node_part=np.empty(n, np.int32), rowptr=np.empty(n + 1, np.int32), colidx=np.empty(max(1, 2 * E), np.int32),
+        bnd_u=np.empty(max(1, E), np.int32), bnd_v=np.empty(max(1, E), np.int32), inv_deg=np.empty(n, np.float32),
+        is_boundary=np.empty(n, np.uint8),
+    )
+    e_in, e_b = ctypes.c_int64(0), ctypes.c_int64(0)
+    rc = _native().oracle_bookkeeping(
+        n, E, _ptr(eu), _ptr(ev), _ptr(part), S, _ptr(out["perm"]), _ptr(out["inv_perm"]), _ptr(out["part_ptr"]),
+        _ptr(out["node_part"]), _ptr(out["rowptr"]), _ptr(out["colidx"]), _ptr(out["bnd_u"]), _ptr(out["bnd_v"]),
+        _ptr(out["inv_deg"]), _ptr(out["is_boundary"]), ctypes.addressof(e_in), ctypes.addressof(e_b))
+    if rc != 0:
+        raise OracleError(rc, "oracle_bookkeeping")
+    out["E_in"], out["E_b"] = int(e_in.value), int(e_b.value)
+    out["colidx"] = out["colidx"][: 2 * out["E_in"]].copy()
+    out["bnd_u"] = out["bnd_u"][: out["E_b"]].copy()
+    out["bnd_v"] = out["bnd_v"][: out["E_b"]].copy()
+    out["n"], out["S"] = n, S
+    return out
+
+
+def _as_f64(a):
+    return None if a is None else np.ascontiguousarray(a, dtype=np.float64)
+
+
+def subgraph_step(rowptr, colidx, dims: Sequence[int], X, W: Sequence[np.ndarray], alpha: float, beta: float,
+                  lam: float = 0.0, pen=None, want_dW: bool = True, want_dX: bool = False,
+                  want_Z: bool = False) -> Dict[str, object]:
+    """One standalone subgraph with local ids: forward, loss and exact gradients."""
+    rowptr = np.ascontiguousarray(rowptr, dtype=np.int32)
+    colidx = np.ascontiguousarray(colidx, dtype=np.int32)
+    ns, L = rowptr.size - 1, len(dims) - 1
+    dims_a = np.asarray(dims, dtype=np.int32)
+    X = _as_f64(X)
+    Wd = [_as_f64(w) for w in W]
+    pen = _as_f64(pen)
+    loss = np.zeros(1)
+    z, p = np.empty(ns), np.empty(ns)
+    dW = [np.zeros((dims[l], dims[l + 1])) for l in range(L)] if want_dW else None
+    dX = np.zeros((ns, dims[0])) if want_dX else None
+    Z = [np.zeros((ns, dims[l + 1])) for l in range(L - 1)] if want_Z else None
+    rc = _native().oracle_subgraph_step(
+        ns, _ptr(rowptr), _ptr(colidx), L, _ptr(dims_a), _ptr(X), _ptr_array(Wd), alpha, beta, lam, _ptr(pen),
+        _ptr(loss), _ptr(z), _ptr(p), _ptr_array(dW) if dW is not None else None, _ptr(dX),
+        _ptr_array(Z + [None]) if Z is not None else None)
+    if rc != 0:
+        raise OracleError(rc, "oracle_subgraph_step")
+    return dict(loss=float(loss[0]), z=z, p=p, dW=dW, dX=dX, Z=Z)
+
+
+def train_step(book: Dict[str, np.ndarray], dims: Sequence[int], X, W: Sequence[np.ndarray], alpha: float, beta: float,
+               lam: float = 0.0, pen=None, want_dW: bool = True, want_dX: bool = False, want_Z: bool = False,
+               threads: int = 1) -> Dict[str, object]:
+    """Block-diagonal batch over all subgraphs of ``book`` (the dict returned by
+    ``bookkeeping``).  ``X`` is [n, F_0] in the NEW node order; ``W[l]`` is
+    [S, F_l, F_{l+1}] (one set per subgraph) or [1, F_l, F_{l+1}] (shared)."""
+    n, S = int(book["n"]), int(book["S"])
+    L = len(dims) - 1
+    dims_a = np.asarray(dims, dtype=np.int32)
+    X = _as_f64(X)
+    assert X.shape == (n, dims[0])
+    Wd = [_as_f64(w) for w in W]
+    sets = Wd[0].shape[0]
+    for l in range(L):
+        assert Wd[l].shape == (sets, dims[l], dims[l + 1]), (Wd[l].shape, l)
+    pen = _as_f64(pen)
+    loss, z, p = np.zeros(S), np.empty(n), np.empty(n)
+    dW = [np.zeros_like(w) for w in Wd] if want_dW else None
+    dX = np.zeros((n, dims[0])) if want_dX else None
+    Z = [np.zeros((n, dims[l + 1])) for l in range(L - 1)] if want_Z else None
+    rc = _native().oracle_train_step(
+        n, S, _ptr(book["part_ptr"]), _ptr(book["rowptr"]), _ptr(book["colidx"]), L, _ptr(dims_a), sets, _ptr(X),
+        _ptr_array(Wd), alpha, beta, lam, _ptr(pen), _ptr(loss), _ptr(z), _ptr(p),
+        _ptr_array(dW) if dW is not None else None, _ptr(dX), _ptr_array(Z + [None]) if Z is not None else None,
+        threads)
+    if rc <= 0:
+        raise OracleError(rc, "oracle_train_step")
+    return dict(loss=loss, z=z, p=p, dW=dW, dX=dX, Z=Z, threads=rc)
+
+
+def adam(W: np.ndarray, m: np.ndarray, v: np.ndarray, g: np.ndarray, lr: float, t: int, b1: float = 0.9,
+         b2: float = 0.999, eps: float = 1e-8) -> None:
+    """In-place bias-corrected Adam on float64 arrays; ``t`` is the 1-based step."""
+    for a in (W, m, v):
+        assert a.dtype == np.float64 and a.flags.c_contiguous
+    g = _as_f64(g)
+    _native().oracle_adam(W.size, _ptr(W), _ptr(m), _ptr(v), _ptr(g), lr, b1, b2, eps, t)
+
+
+def decode(book: Dict[str, np.ndarray], p: np.ndarray, threshold: float = 0.5) -> Dict[str, object]:
+    """Threshold float32 probabilities and count selected nodes and violated edges."""
+    n, S = int(book["n"]), int(book["S"])
+    p = np.ascontiguousarray(p, dtype=np.float32)
+    assert p.shape == (n,)
+    x = np.empty(n, np.uint8)
+    viol = np.empty(max(1, book["E_b"]), np.uint8)
+    per_part = np.empty(S, np.int32)
+    counts = np.zeros(3, np.int64)
+    _native().oracle_decode(n, S, _ptr(book["node_part"]), _ptr(book["rowptr"]), _ptr(book["colidx"]), book["E_b"],
+                            _ptr(book["bnd_u"]), _ptr(book["bnd_v"]), _ptr(p), threshold, _ptr(x), _ptr(viol),
+                            _ptr(per_part), _ptr(counts))
+    return dict(x=x, viol=viol[: book["E_b"]], per_part=per_part, set_size=int(counts[0]), intra_viol=int(counts[1]),
+                boundary_viol=int(counts[2]))

@@ -1,0 +1,410 @@
+/*
+ * CPU oracle for the partitioned-GNN train step.  TEST INFRASTRUCTURE ONLY.
+ *
+ * Plain, slow, double-precision restatement of what the hot path computes, written
+ * from the paper's definitions.  It shares no code, header, table or helper with the
+ * CUDA library; only tests, the smoke check and the benchmark's CPU-baseline leg may
+ * call it.  Every function cites the passage it follows.
+ *
+ * Conventions
+ *   - nodes are renumbered so that each subgraph (partition) is a contiguous id range;
+ *     `part_ptr[s] .. part_ptr[s+1]` is subgraph s;
+ *   - only intra-subgraph edges take part in training (Section 3.3: subgraphs are
+ *     trained "without cross-subgraph interference"); cross edges are kept aside as
+ *     the boundary list that decoding inspects;
+ *   - dense matrices are row-major.
+ *
+ * Pins (see tests, "not gpu"): finite differences for every gradient, closed forms at
+ * W = 0, row-stochastic aggregation, per-subgraph runs equal the batched run, brute
+ * force on graphs of at most 16 nodes, hand-computed Adam steps, brute-force decode.
+ * Parity unpinned: nothing here can be compared with the paper's result tables
+ * (they need the original datasets, trained weights and the RL stage).
+ */
+#include <math.h>
+#include <stdint.h>
+#include <stdlib.h>
+#include <string.h>
+#ifdef _OPENMP
+#include <omp.h>
+#endif
+
+enum { ORACLE_OK = 0, ORACLE_BAD_ARG = -1, ORACLE_OUT_OF_RANGE = -2, ORACLE_NOT_SIMPLE = -3, ORACLE_NOMEM = -6 };
+
+static int cmp_i32(const void* a, const void* b) {
+  int32_t x = *(const int32_t*)a, y = *(const int32_t*)b;
+  return (x > y) - (x < y);
+}
+static int cmp_pair(const void* a, const void* b) {
+  const int32_t* x = (const int32_t*)a;
+  const int32_t* y = (const int32_t*)b;
+  if (x[0] != y[0]) return (x[0] > y[0]) - (x[0] < y[0]);
+  return (x[1] > y[1]) - (x[1] < y[1]);
+}
+
+/*
+ * Bookkeeping (Section 3.3, first paragraph: the graph is split into subgraphs, and
+ * "cross-nodes" are the endpoints of edges whose ends lie in different subgraphs;
+ * Algorithm 1, Stage 2: global mask and cross-node mask).
+ *
+ *   new id of a node   = its rank under the key (part, original id)
+ *   perm[new] = original id, inv_perm[original] = new id
+ *   intra edge         = part[u] == part[v]: stored in both directions in a CSR with
+ *                        ascending columns and no self loops
+ *   boundary edge      = otherwise: stored once as (min, max) of the new ids, the list
+ *                        sorted lexicographically
+ *   inv_deg[i]         = 1 / (intra degree of i + 1)   (Eq. 3's 1/(|N(i)|+1)), in float
+ *   is_boundary[i]     = 1 iff i is an endpoint of a boundary edge
+ * colidx must hold 2E entries and bnd_u/bnd_v E entries (worst case).
+ */
+int oracle_bookkeeping(int64_t n, int64_t E, const int32_t* eu, const int32_t* ev, const int32_t* part, int32_t S,
+                       int32_t* perm, int32_t* inv_perm, int32_t* part_ptr, int32_t* node_part, int32_t* rowptr,
+                       int32_t* colidx, int32_t* bnd_u, int32_t* bnd_v, float* inv_deg, uint8_t* is_boundary,
+                       int64_t* E_in_out, int64_t* E_b_out) {
+  if (n <= 0 || E < 0 || S <= 0) return ORACLE_BAD_ARG;
+  for (int64_t i = 0; i < n; ++i)
+    if (part[i] < 0 || part[i] >= S) return ORACLE_OUT_OF_RANGE;
+  for (int64_t e = 0; e < E; ++e) {
+    if (eu[e] < 0 || eu[e] >= n || ev[e] < 0 || ev[e] >= n) return ORACLE_OUT_OF_RANGE;
+    if (eu[e] == ev[e]) return ORACLE_NOT_SIMPLE;
+  }
+  /* subgraph sizes -> start offsets */
+  for (int32_t s = 0; s <= S; ++s) part_ptr[s] = 0;
+  for (int64_t i = 0; i < n; ++i) part_ptr[part[i] + 1]++;
+  for (int32_t s = 0; s < S; ++s) part_ptr[s + 1] += part_ptr[s];
+  /* rank under (part, original id): walk original ids upward, append to the node's part */
+  int32_t* fill = (int32_t*)malloc((size_t)S * sizeof(int32_t));
+  if (!fill) return ORACLE_NOMEM;
+  memcpy(fill, part_ptr, (size_t)S * sizeof(int32_t));
+  for (int64_t i = 0; i < n; ++i) {
+    int32_t id = fill[part[i]]++;
+    inv_perm[i] = id;
+    perm[id] = (int32_t)i;
+    node_part[id] = part[i];
+  }
+  free(fill);
+  /* classify edges, count intra degree */
+  for (int64_t i = 0; i <= n; ++i) rowptr[i] = 0;
+  memset(is_boundary, 0, (size_t)n);
+  int64_t E_in = 0, E_b = 0;
+  int32_t* bpairs = (int32_t*)malloc((size_t)(2 * E + 2) * sizeof(int32_t));
+  if (!bpairs) return ORACLE_NOMEM;
+  for (int64_t e = 0; e < E; ++e) {
+    int32_t a = inv_perm[eu[e]], b = inv_perm[ev[e]];
+    if (part[eu[e]] == part[ev[e]]) {
+      rowptr[a + 1]++; rowptr[b + 1]++; ++E_in;
+    } else {
+      bpairs[2 * E_b] = a < b ? a : b;
+      bpairs[2 * E_b + 1] = a < b ? b : a;
+      is_boundary[a] = 1; is_boundary[b] = 1;
+      ++E_b;
+    }
+  }
+  for (int64_t i = 0; i < n; ++i) rowptr[i + 1] += rowptr[i];
+  int32_t* pos = (int32_t*)malloc((size_t)n * sizeof(int32_t));
+  if (!pos) { free(bpairs); return ORACLE_NOMEM; }
+  memcpy(pos, rowptr, (size_t)n * sizeof(int32_t));
+  for (int64_t e = 0; e < E; ++e) {
+    if (part[eu[e]] != part[ev[e]]) continue;
+    int32_t a = inv_perm[eu[e]], b = inv_perm[ev[e]];
+    colidx[pos[a]++] = b;
+    colidx[pos[b]++] = a;
+  }
+  free(pos);
+  int status = ORACLE_OK;
+  for (int64_t i = 0; i < n; ++i) {
+    int32_t lo = rowptr[i], hi = rowptr[i + 1];
+    qsort(colidx + lo, (size_t)(hi - lo), sizeof(int32_t), cmp_i32);
+    for (int32_t k = lo + 1; k < hi; ++k)
+      if (colidx[k] == colidx[k - 1]) status = ORACLE_NOT_SIMPLE;   /* repeated edge */
+    inv_deg[i] = 1.0f / (float)(hi - lo + 1);
+  }
+  qsort(bpairs, (size_t)E_b, 2 * sizeof(int32_t), cmp_pair);
+  for (int64_t k = 0; k < E_b; ++k) {
+    bnd_u[k] = bpairs[2 * k];
+    bnd_v[k] = bpairs[2 * k + 1];
+    if (k > 0 && bnd_u[k] == bnd_u[k - 1] && bnd_v[k] == bnd_v[k - 1]) status = ORACLE_NOT_SIMPLE;
+  }
+  free(bpairs);
+  *E_in_out = E_in;
+  *E_b_out = E_b;
+  return status;
+}
+
+/*
+ * One subgraph, standalone (local node ids 0..ns-1, local CSR): forward (Eq. 3 per
+ * hidden layer, Eq. 4 on the last layer's scalar output), objective (Eq. 5 plus the
+ * fine-tuning penalty of Section 3.3), and the exact reverse-mode derivative of that
+ * scalar with respect to every weight matrix and, optionally, the input embeddings.
+ *
+ * Readings of the paper taken here:
+ *   - hidden layers: h = ReLU( mean_{self+neighbours}(h_prev) W )          (Eq. 3)
+ *   - last layer (output width 1): z = mean_{self+neighbours}(h_prev) w, no ReLU;
+ *     p = 1/(1+exp(-z))                                                     (Eq. 4)
+ *   - loss = alpha * sum_{edges, each once} p_i p_j - beta * sum_i p_i
+ *            + lambda * sum_i pen_i p_i                                     (Eq. 5, penalty)
+ *   - ReLU derivative is 1 where the pre-activation is > 0, else 0.
+ * W[l] points at this subgraph's F_l x F_{l+1} matrix of layer l (0-based).
+ * dW[l] (if dW != NULL) receives the gradient; dX (if != NULL) receives d loss / d X.
+ * Zsave[l] (if Zsave != NULL), l < L-1, receives the pre-activations of hidden layer l.
+ */
+static int subgraph_step(int32_t ns, const int32_t* rp, const int32_t* ci, int32_t L, const int32_t* dims,
+                         const double* X, const double* const* W, double alpha, double beta, double lambda,
+                         const double* pen, double* loss_out, double* z_out, double* p_out, double* const* dW,
+                         double* dX, double* const* Zsave) {
+  int rc = ORACLE_OK;
+  double** H = (double**)calloc((size_t)L + 1, sizeof(double*));   /* H[0] = X, H[l] = output of layer l */
+  double** M = (double**)calloc((size_t)L + 1, sizeof(double*));   /* M[l] = aggregated input of layer l (1-based) */
+  double** Z = (double**)calloc((size_t)L + 1, sizeof(double*));   /* Z[l] = M[l] W[l-1] */
+  if (!H || !M || !Z) { rc = ORACLE_NOMEM; goto done; }
+  H[0] = (double*)X;
+  for (int32_t l = 1; l <= L; ++l) {
+    int32_t fi = dims[l - 1], fo = dims[l];
+    M[l] = (double*)calloc((size_t)ns * fi + 1, sizeof(double));
+    Z[l] = (double*)calloc((size_t)ns * fo + 1, sizeof(double));
+    if (l < L) H[l] = (double*)calloc((size_t)ns * fo + 1, sizeof(double));
+    if (!M[l] || !Z[l] || (l < L && !H[l])) { rc = ORACLE_NOMEM; goto done; }
+    const double* Hp = H[l - 1];
+    const double* Wl = W[l - 1];
+    for (int32_t i = 0; i < ns; ++i) {
+      double* m = M[l] + (size_t)i * fi;
+      for (int32_t f = 0; f < fi; ++f) m[f] = Hp[(size_t)i * fi + f];
+      for (int32_t k = rp[i]; k < rp[i + 1]; ++k) {
+        const double* hj = Hp + (size_t)ci[k] * fi;
+        for (int32_t f = 0; f < fi; ++f) m[f] += hj[f];
+      }
+      double inv = 1.0 / (double)(rp[i + 1] - rp[i] + 1);
+      for (int32_t f = 0; f < fi; ++f) m[f] *= inv;
+      double* zr = Z[l] + (size_t)i * fo;
+      for (int32_t f = 0; f < fi; ++f) {
+        double mf = m[f];
+        const double* wrow = Wl + (size_t)f * fo;
+        for (int32_t h = 0; h < fo; ++h) zr[h] += mf * wrow[h];
+      }
+      if (l < L) {
+        double* hr = H[l] + (size_t)i * fo;
+        for (int32_t h = 0; h < fo; ++h) hr[h] = zr[h] > 0.0 ? zr[h] : 0.0;
+      }
+    }
+    if (l < L && Zsave && Zsave[l - 1]) memcpy(Zsave[l - 1], Z[l], (size_t)ns * fo * sizeof(double));
+  }
+  if (dims[L] != 1) { rc = ORACLE_BAD_ARG; goto done; }
+  {
+    double* p = p_out;
+    for (int32_t i = 0; i < ns; ++i) {
+      double z = Z[L][i];
+      if (z_out) z_out[i] = z;
+      p[i] = 1.0 / (1.0 + exp(-z));
+    }
+    double edge_term = 0.0, node_term = 0.0, pen_term = 0.0;
+    for (int32_t i = 0; i < ns; ++i) {
+      for (int32_t k = rp[i]; k < rp[i + 1]; ++k)
+        if (ci[k] > i) edge_term += p[i] * p[ci[k]];
+      node_term += p[i];
+      if (pen) pen_term += pen[i] * p[i];
+    }
+    *loss_out = alpha * edge_term - beta * node_term + lambda * pen_term;
+    if (!dW && !dX) goto done;
+    /* backward */
+    double* dZ = (double*)calloc((size_t)ns + 1, sizeof(double));   /* gradient wrt Z[L] */
+    if (!dZ) { rc = ORACLE_NOMEM; goto done; }
+    for (int32_t i = 0; i < ns; ++i) {
+      double nb = 0.0;
+      for (int32_t k = rp[i]; k < rp[i + 1]; ++k) nb += p[ci[k]];
+      double dp = alpha * nb - beta + (pen ? lambda * pen[i] : 0.0);
+      dZ[i] = dp * p[i] * (1.0 - p[i]);
+    }
+    for (int32_t l = L; l >= 1; --l) {
+      int32_t fi = dims[l - 1], fo = dims[l];
+      const double* Wl = W[l - 1];
+      if (dW && dW[l - 1]) {
+        double* g = dW[l - 1];
+        for (size_t q = 0; q < (size_t)fi * fo; ++q) g[q] = 0.0;
+        for (int32_t i = 0; i < ns; ++i)
+          for (int32_t f = 0; f < fi; ++f) {
+            double mf = M[l][(size_t)i * fi + f];
+            for (int32_t h = 0; h < fo; ++h) g[(size_t)f * fo + h] += mf * dZ[(size_t)i * fo + h];
+          }
+      }
+      if (l == 1 && !dX) break;
+      /* dM = dZ W^T, then through the transpose of the mean aggregation */
+      double* dH = (double*)calloc((size_t)ns * fi + 1, sizeof(double));
+      double* dm = (double*)malloc((size_t)fi * sizeof(double) + 8);
+      if (!dH || !dm) { free(dH); free(dm); free(dZ); rc = ORACLE_NOMEM; goto done; }
+      for (int32_t i = 0; i < ns; ++i) {
+        for (int32_t f = 0; f < fi; ++f) {
+          double acc = 0.0;
+          for (int32_t h = 0; h < fo; ++h) acc += dZ[(size_t)i * fo + h] * Wl[(size_t)f * fo + h];
+          dm[f] = acc / (double)(rp[i + 1] - rp[i] + 1);
+        }
+        /* row i of the mean used itself and each neighbour with the same weight */
+        for (int32_t f = 0; f < fi; ++f) dH[(size_t)i * fi + f] += dm[f];
+        for (int32_t k = rp[i]; k < rp[i + 1]; ++k) {
+          double* dj = dH + (size_t)ci[k] * fi;
+          for (int32_t f = 0; f < fi; ++f) dj[f] += dm[f];
+        }
+      }
+      free(dm);
+      free(dZ);
+      if (l == 1) {
+        memcpy(dX, dH, (size_t)ns * fi * sizeof(double));
+        free(dH);
+        dZ = NULL;
+      } else {
+        for (size_t q = 0; q < (size_t)ns * fi; ++q)
+          if (!(Z[l - 1][q] > 0.0)) dH[q] = 0.0;
+        dZ = dH;
+      }
+    }
+    free(dZ);
+  }
+done:
+  if (H) for (int32_t l = 1; l <= L; ++l) free(H[l]);
+  if (M) for (int32_t l = 1; l <= L; ++l) free(M[l]);
+  if (Z) for (int32_t l = 1; l <= L; ++l) free(Z[l]);
+  free(H); free(M); free(Z);
+  return rc;
+}
+
+/* Standalone single-subgraph entry (used by the "batch equals per-subgraph runs" pin). */
+int oracle_subgraph_step(int32_t ns, const int32_t* rowptr, const int32_t* colidx, int32_t L, const int32_t* dims,
+                         const double* X, const double* const* W, double alpha, double beta, double lambda,
+                         const double* pen, double* loss, double* z, double* p, double* const* dW, double* dX,
+                         double* const* Zsave) {
+  if (ns <= 0 || L < 1) return ORACLE_BAD_ARG;
+  return subgraph_step(ns, rowptr, colidx, L, dims, X, W, alpha, beta, lambda, pen, loss, z, p, dW, dX, Zsave);
+}
+
+/*
+ * Block-diagonal batch: every subgraph of the partitioned graph, each with its own
+ * weight set (Algorithm 1, Stage 1: one model per subgraph) or all sharing one
+ * (weight_sets == 1, gradients summed over subgraphs).
+ *   X [n x F_0], z/p [n], loss [S]; W[l] is [weight_sets x F_l x F_{l+1}];
+ *   dW[l] the same shape; dX [n x F_0]; Zsave[l] [n x F_{l+1}] for hidden layers.
+ * Subgraphs are independent, so the outer loop may run on several threads; the
+ * arithmetic inside one subgraph is untouched.  Returns the thread count used (> 0)
+ * or a negative error.
+ */
+int oracle_train_step(int64_t n, int32_t S, const int32_t* part_ptr, const int32_t* rowptr, const int32_t* colidx,
+                      int32_t L, const int32_t* dims, int32_t weight_sets, const double* X, const double* const* W,
+                      double alpha, double beta, double lambda, const double* pen, double* loss, double* z, double* p,
+                      double* const* dW, double* dX, double* const* Zsave, int32_t threads) {
+  if (n <= 0 || S <= 0 || L < 1 || L > 16 || (weight_sets != 1 && weight_sets != S)) return ORACLE_BAD_ARG;
+  int rc = ORACLE_OK;
+  int used = 1;
+  if (dW && weight_sets == 1)
+    for (int32_t l = 0; l < L; ++l)
+      if (dW[l]) memset(dW[l], 0, (size_t)dims[l] * dims[l + 1] * sizeof(double));
+#ifdef _OPENMP
+  if (threads < 1) threads = 1;
+#pragma omp parallel for schedule(dynamic, 1) num_threads(threads)
+#endif
+  for (int32_t s = 0; s < S; ++s) {
+#ifdef _OPENMP
+    if (s == 0 || omp_get_thread_num() == 0) {
+#pragma omp atomic write
+      used = omp_get_num_threads();
+    }
+#endif
+    int32_t r0 = part_ptr[s], r1 = part_ptr[s + 1], ns = r1 - r0;
+    if (ns <= 0) { loss[s] = 0.0; continue; }
+    int32_t base = rowptr[r0];
+    int32_t nnz = rowptr[r1] - base;
+    int32_t* rp = (int32_t*)malloc((size_t)(ns + 1) * sizeof(int32_t));
+    int32_t* ci = (int32_t*)malloc((size_t)(nnz + 1) * sizeof(int32_t));
+    const double* Ws[16];
+    double* dWs[16];
+    double* Zs[16];
+    int bad = (!rp || !ci);
+    if (!bad) {
+      for (int32_t i = 0; i <= ns; ++i) rp[i] = rowptr[r0 + i] - base;
+      for (int32_t k = 0; k < nnz; ++k) {
+        ci[k] = colidx[base + k] - r0;
+        if (ci[k] < 0 || ci[k] >= ns) bad = 1;   /* an intra edge must stay inside its subgraph */
+      }
+    }
+    if (bad) {
+#pragma omp critical
+      rc = ORACLE_BAD_ARG;
+      free(rp); free(ci);
+      continue;
+    }
+    for (int32_t l = 0; l < L; ++l) {
+      size_t wsz = (size_t)dims[l] * dims[l + 1];
+      Ws[l] = W[l] + (weight_sets == 1 ? 0 : (size_t)s * wsz);
+      dWs[l] = NULL;
+      if (dW && dW[l]) dWs[l] = weight_sets == 1 ? (double*)malloc(wsz * sizeof(double)) : dW[l] + (size_t)s * wsz;
+      Zs[l] = (Zsave && l < L - 1 && Zsave[l]) ? Zsave[l] + (size_t)r0 * dims[l + 1] : NULL;
+    }
+    int r = subgraph_step(ns, rp, ci, L, dims, X + (size_t)r0 * dims[0], Ws, alpha, beta, lambda,
+                          pen ? pen + r0 : NULL, loss + s, z ? z + r0 : NULL, p + r0, dW ? dWs : NULL,
+                          dX ? dX + (size_t)r0 * dims[0] : NULL, Zsave ? Zs : NULL);
+    if (r != ORACLE_OK) {
+#pragma omp critical
+      rc = r;
+    }
+    if (dW && weight_sets == 1) {
+      for (int32_t l = 0; l < L; ++l) {
+        if (!dWs[l]) continue;
+        size_t wsz = (size_t)dims[l] * dims[l + 1];
+#pragma omp critical
+        for (size_t q = 0; q < wsz; ++q) dW[l][q] += dWs[l][q];
+        free(dWs[l]);
+      }
+    }
+    free(rp); free(ci);
+  }
+  return rc != ORACLE_OK ? rc : used;
+}
+
+/*
+ * Adam with bias correction (the paper names no optimiser beyond "backpropagation is
+ * performed to update the weight matrix W", Section 3.2; the benchmark configurations
+ * fix Adam).  t is the 1-based step number.
+ *   m <- b1 m + (1-b1) g;  v <- b2 v + (1-b2) g^2
+ *   W <- W - lr * (m / (1-b1^t)) / (sqrt(v / (1-b2^t)) + eps)
+ */
+void oracle_adam(int64_t count, double* W, double* m, double* v, const double* g, double lr, double b1, double b2,
+                 double eps, int64_t t) {
+  double c1 = 1.0 - pow(b1, (double)t), c2 = 1.0 - pow(b2, (double)t);
+  for (int64_t q = 0; q < count; ++q) {
+    m[q] = b1 * m[q] + (1.0 - b1) * g[q];
+    v[q] = b2 * v[q] + (1.0 - b2) * g[q] * g[q];
+    W[q] -= lr * (m[q] / c1) / (sqrt(v[q] / c2) + eps);
+  }
+}
+
+/*
+ * Decoding and conflict counting (Section 3.3: probabilities are binarised with
+ * "1 if prob >= 0.5, 0 otherwise"; a cross edge whose two endpoints are both selected
+ * is a conflict; Section 4.1: MIS size and conflicts are the reported metrics).
+ *   x[i]        = p[i] >= threshold   (compared on the stored float value)
+ *   viol[e]     = x[bnd_u[e]] & x[bnd_v[e]]
+ *   per_part[s] = number of violated boundary edges with an endpoint in s (an edge
+ *                 counts once for each of its two subgraphs)
+ *   counts      = { sum x, violated intra edges (each once), violated boundary edges }
+ */
+void oracle_decode(int64_t n, int32_t S, const int32_t* node_part, const int32_t* rowptr, const int32_t* colidx,
+                   int64_t E_b, const int32_t* bnd_u, const int32_t* bnd_v, const float* p, float threshold,
+                   uint8_t* x, uint8_t* viol, int32_t* per_part, int64_t* counts) {
+  int64_t set_size = 0, intra = 0, bviol = 0;
+  for (int64_t i = 0; i < n; ++i) {
+    x[i] = p[i] >= threshold ? 1 : 0;
+    set_size += x[i];
+  }
+  for (int64_t i = 0; i < n; ++i)
+    for (int32_t k = rowptr[i]; k < rowptr[i + 1]; ++k)
+      if (colidx[k] > i && x[i] && x[colidx[k]]) ++intra;
+  for (int32_t s = 0; s < S; ++s) per_part[s] = 0;
+  for (int64_t e = 0; e < E_b; ++e) {
+    uint8_t v = (uint8_t)(x[bnd_u[e]] & x[bnd_v[e]]);
+    if (viol) viol[e] = v;
+    if (v) {
+      ++bviol;
+      per_part[node_part[bnd_u[e]]]++;
+      per_part[node_part[bnd_v[e]]]++;
+    }
+  }
+  counts[0] = set_size;
+  counts[1] = intra;
+  counts[2] = bviol;
+}

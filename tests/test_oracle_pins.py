@@ -1,0 +1,555 @@
+"""Pins for the CPU oracle: each test checks it against something other than itself --
+a closed form, an invariant, a finite difference, exact rational arithmetic, a dense
+linear-algebra restatement built from the ORIGINAL edge list, or brute force."""
+import itertools
+from fractions import Fraction
+import decimal
+
+import numpy as np
+import pytest
+
+import oracle
+import synth_inputs as si
+from helpers import tiny_graph, dense_intra_adjacency, rand_weights, rand_features
+
+ALPHA, BETA = 2.0, 1.0
+
+
+# ------------------------------------------------------------------ bookkeeping (a0)
+def _brute_bookkeeping(n, eu, ev, part, S):
+    order = sorted(range(n), key=lambda i: (int(part[i]), i))
+    inv = {o: k for k, o in enumerate(order)}
+    intra, bnd = set(), set()
+    for a, b in zip(eu.tolist(), ev.tolist()):
+        na, nb = inv[a], inv[b]
+        (intra if part[a] == part[b] else bnd).add((min(na, nb), max(na, nb)))
+    return order, inv, intra, bnd
+
+
+@pytest.mark.parametrize("n,p,S,seed", [(12, 0.4, 3, 1), (40, 0.2, 5, 2), (64, 0.1, 64, 3), (30, 0.3, 1, 4),
+                                        (25, 0.3, 9, 5)])
+def test_bookkeeping_brute_force(n, p, S, seed):
+    eu, ev, part = tiny_graph(n, p, S, seed)
+    b = oracle.bookkeeping(n, eu, ev, part, S)
+    order, inv, intra, bnd = _brute_bookkeeping(n, eu, ev, part, S)
+    assert b["perm"].tolist() == order
+    assert [int(b["inv_perm"][i]) for i in range(n)] == [inv[i] for i in range(n)]
+    assert b["E_in"] == len(intra) and b["E_b"] == len(bnd) and b["E_in"] + b["E_b"] == eu.size
+    sizes = np.bincount(part, minlength=S)
+    assert np.array_equal(np.diff(b["part_ptr"]), sizes) and b["part_ptr"][0] == 0
+    rp, ci = b["rowptr"], b["colidx"]
+    assert rp[0] == 0 and rp[n] == 2 * b["E_in"]
+    got = set()
+    for i in range(n):
+        row = ci[rp[i]:rp[i + 1]].tolist()
+        assert row == sorted(set(row)) and i not in row
+        s = b["node_part"][i]
+        assert all(b["part_ptr"][s] <= j < b["part_ptr"][s + 1] for j in row)
+        for j in row:
+            assert i in ci[rp[j]:rp[j + 1]].tolist()            # symmetric
+            got.add((min(i, j), max(i, j)))
+        assert b["inv_deg"][i] == np.float32(1.0) / np.float32(len(row) + 1)
+    assert got == intra
+    pairs = list(zip(b["bnd_u"].tolist(), b["bnd_v"].tolist()))
+    assert pairs == sorted(bnd)
+    isb = np.zeros(n, np.uint8)
+    for a, c in bnd:
+        isb[a] = isb[c] = 1
+    assert np.array_equal(b["is_boundary"], isb)
+    assert np.array_equal(b["node_part"], part[b["perm"]])
+
+
+def test_bookkeeping_rejects_bad_input():
+    eu = np.array([0, 1, 2], np.int32)
+    ev = np.array([1, 2, 2], np.int32)
+    part = np.zeros(4, np.int32)
+    with pytest.raises(oracle.OracleError) as e:
+        oracle.bookkeeping(4, eu, ev, part, 1)            # self loop 2-2
+    assert e.value.code == oracle.NOT_SIMPLE
+    with pytest.raises(oracle.OracleError) as e:
+        oracle.bookkeeping(4, np.array([0, 1], np.int32), np.array([1, 0], np.int32), part, 1)   # repeated edge
+    assert e.value.code == oracle.NOT_SIMPLE
+    with pytest.raises(oracle.OracleError) as e:
+        oracle.bookkeeping(4, np.array([0], np.int32), np.array([7], np.int32), part, 1)
+    assert e.value.code == oracle.OUT_OF_RANGE
+    with pytest.raises(oracle.OracleError) as e:
+        oracle.bookkeeping(4, np.array([0], np.int32), np.array([1], np.int32), np.array([0, 0, 3, 0], np.int32), 2)
+    assert e.value.code == oracle.OUT_OF_RANGE
+
+
+@pytest.mark.parametrize("idx", [1, 2, 3])
+def test_bookkeeping_invariants_on_configs(idx):
+    w = si.make_workload(idx)
+    b = oracle.bookkeeping(w.n, w.eu, w.ev, w.part, w.S)
+    assert b["E_in"] + b["E_b"] == w.E and b["rowptr"][w.n] == 2 * b["E_in"]
+    assert np.array_equal(np.sort(b["perm"]), np.arange(w.n))
+    assert np.array_equal(b["inv_perm"][b["perm"]], np.arange(w.n))
+    assert np.array_equal(np.diff(b["part_ptr"]), np.bincount(w.part, minlength=w.S))
+    rows = np.repeat(np.arange(w.n), np.diff(b["rowptr"]))
+    assert np.array_equal(b["node_part"][rows], b["node_part"][b["colidx"]])
+    fwd = set(zip(rows.tolist(), b["colidx"].tolist()))
+    assert len(fwd) == 2 * b["E_in"] and all((j, i) in fwd for i, j in itertools.islice(fwd, 5000))
+    intra_direct = int((w.part[w.eu] == w.part[w.ev]).sum())
+    assert b["E_in"] == intra_direct
+
+
+# --------------------------------------------------- dense restatement (a1-a4), Eq. 3-5
+def _dense_forward_loss(n, eu, ev, part, dims, X, W, pen, lam):
+    """Dense linear algebra from the original edge list, original node order;
+    W[l][part] applied row by row."""
+    A = dense_intra_adjacency(n, eu, ev, part)
+    Ahat = (A + np.eye(n)) / (A.sum(1) + 1.0)[:, None]
+    H = X
+    L = len(dims) - 1
+    for l in range(L):
+        M = Ahat @ H
+        Z = np.stack([M[i] @ W[l][part[i] if W[l].shape[0] > 1 else 0] for i in range(n)])
+        H = np.maximum(Z, 0.0) if l < L - 1 else Z
+    z = H[:, 0]
+    p = 1.0 / (1.0 + np.exp(-z))
+    S = int(part.max()) + 1
+    loss = np.zeros(S)
+    for s in range(S):
+        msk = part == s
+        ps = p * msk
+        loss[s] = ALPHA * 0.5 * ps @ A @ ps - BETA * ps.sum() + lam * (pen * ps).sum()
+    return z, p, loss
+
+
+@pytest.mark.parametrize("dims,sets_shared", [([5, 1], False), ([6, 4, 1], False), ([7, 5, 3, 1], True)])
+def test_forward_and_loss_match_dense_definition(dims, sets_shared):
+    n, S = 40, 4
+    eu, ev, part = tiny_graph(n, 0.25, S, seed=11)
+    b = oracle.bookkeeping(n, eu, ev, part, S)
+    X = rand_features(n, dims[0], 5)
+    W = rand_weights(dims, 1 if sets_shared else S, 7, scale=2.0)
+    pen = (si.uniform01(99, 0, n) < 0.3).astype(np.float64)
+    z, p, loss = _dense_forward_loss(n, eu, ev, part, dims, X, W, pen, 0.7)
+    r = oracle.train_step(b, dims, X[b["perm"]], W, ALPHA, BETA, 0.7, pen[b["perm"]])
+    np.testing.assert_allclose(r["z"], z[b["perm"]], rtol=1e-12, atol=1e-13)
+    np.testing.assert_allclose(r["p"], p[b["perm"]], rtol=1e-12, atol=1e-13)
+    np.testing.assert_allclose(r["loss"], loss, rtol=1e-12, atol=1e-12)
+
+
+def test_aggregation_preserves_constant_features_and_isolated_nodes():
+    # identity weights expose M = A_hat X through the saved pre-activations
+    n, S, F = 50, 5, 4
+    eu, ev, part = tiny_graph(n, 0.15, S, seed=21)
+    b = oracle.bookkeeping(n, eu, ev, part, S)
+    W = [np.tile(np.eye(F), (S, 1, 1)), np.zeros((S, F, 1))]
+    X = np.tile(np.array([1.5, -2.0, 0.25, 3.0]), (n, 1))
+    r = oracle.train_step(b, [F, F, 1], X, W, ALPHA, BETA, want_Z=True)
+    assert np.array_equal(r["Z"][0], X)                       # rows of A_hat sum to one
+    Xr = rand_features(n, F, 3)
+    r = oracle.train_step(b, [F, F, 1], Xr, W, ALPHA, BETA, want_Z=True)
+    deg = np.diff(b["rowptr"])
+    iso = np.where(deg == 0)[0]
+    assert iso.size > 0
+    assert np.array_equal(r["Z"][0][iso], Xr[iso])            # no intra neighbour: M_i = H_i
+
+
+def test_regular_partition_aggregation_is_doubly_stochastic():
+    # one partition, 4-regular circulant graph: column sums of A_hat are one as well
+    n, F = 31, 3
+    eu = np.concatenate([np.arange(n), np.arange(n)]).astype(np.int32)
+    ev = np.concatenate([(np.arange(n) + 1) % n, (np.arange(n) + 5) % n]).astype(np.int32)
+    b = oracle.bookkeeping(n, eu, ev, np.zeros(n, np.int32), 1)
+    assert np.all(np.diff(b["rowptr"]) == 4)
+    X = rand_features(n, F, 8)
+    r = oracle.train_step(b, [F, F, 1], X, [np.eye(F)[None], np.zeros((1, F, 1))], ALPHA, BETA, want_Z=True)
+    np.testing.assert_allclose(r["Z"][0].sum(0), X.sum(0), rtol=1e-13)
+
+
+def test_zero_weights_closed_forms():
+    w = si.make_workload(1)
+    b = oracle.bookkeeping(w.n, w.eu, w.ev, w.part, w.S)
+    X = w.features_f32()[b["perm"]]
+    W = [np.zeros((w.S, w.dims[l], w.dims[l + 1])) for l in range(w.L)]
+    r = oracle.train_step(b, w.dims, X, W, ALPHA, BETA)
+    assert np.all(r["z"] == 0.0) and np.all(r["p"] == 0.5)
+    e_in_s = np.array([(b["rowptr"][b["part_ptr"][s + 1]] - b["rowptr"][b["part_ptr"][s]]) // 2 for s in range(w.S)])
+    expect = ALPHA * e_in_s / 4.0 - BETA * np.diff(b["part_ptr"]) / 2.0
+    assert np.array_equal(r["loss"], expect)
+    d = oracle.decode(b, r["p"].astype(np.float32))
+    assert d["set_size"] == w.n and d["boundary_viol"] == b["E_b"] and d["intra_viol"] == b["E_in"]
+    assert np.all(d["x"] == 1) and np.all(d["viol"] == 1)
+    assert d["per_part"].sum() == 2 * b["E_b"]
+
+
+def test_single_node_subgraph_by_hand():
+    # two isolated single-node subgraphs: p = sigmoid(relu(x W1) w2), own weights each
+    X = np.array([[1.0, -2.0], [0.5, 3.0]])
+    W1 = np.array([[[1.0, -1.0], [0.5, 2.0]], [[-1.0, 0.0], [1.0, 1.0]]])
+    W2 = np.array([[[2.0], [-1.0]], [[0.5], [0.25]]])
+    b = oracle.bookkeeping(2, np.zeros(0, np.int32), np.zeros(0, np.int32), np.array([0, 1], np.int32), 2)
+    r = oracle.train_step(b, [2, 2, 1], X, [W1, W2], ALPHA, BETA)
+    # node 0: x W1 = [1-1, -1-4] = [0, -5] -> relu [0, 0] -> z = 0
+    # node 1: x W1 = [-0.5+3, 0+3] = [2.5, 3] -> z = 1.25 + 0.75 = 2
+    assert r["z"].tolist() == [0.0, 2.0]
+    np.testing.assert_allclose(r["p"], [0.5, 1.0 / (1.0 + np.exp(-2.0))], rtol=1e-15)
+    np.testing.assert_allclose(r["loss"], [-0.5, -1.0 / (1.0 + np.exp(-2.0))], rtol=1e-15)
+
+
+def test_complete_graph_identical_rows_give_equal_probabilities():
+    k, F = 7, 5
+    eu, ev = np.triu_indices(k, 1)
+    b = oracle.bookkeeping(k, eu.astype(np.int32), ev.astype(np.int32), np.zeros(k, np.int32), 1)
+    X = np.tile(rand_features(1, F, 4), (k, 1))
+    r = oracle.train_step(b, [F, 4, 1], X, rand_weights([F, 4, 1], 1, 3), ALPHA, BETA)
+    assert np.all(r["p"] == r["p"][0])
+
+
+def test_relabelling_nodes_permutes_outputs():
+    n, S, dims = 36, 3, [4, 3, 1]
+    eu, ev, part = tiny_graph(n, 0.3, S, seed=31, contiguous=True)
+    X, W = rand_features(n, 4, 6), rand_weights(dims, S, 9)
+    b = oracle.bookkeeping(n, eu, ev, part, S)
+    r = oracle.train_step(b, dims, X[b["perm"]], W, ALPHA, BETA)
+    # reverse the ids inside the graph (parts stay attached to their nodes)
+    sigma = np.arange(n)[::-1].copy()                   # old id -> new id
+    eu2, ev2 = sigma[eu].astype(np.int32), sigma[ev].astype(np.int32)
+    part2 = np.empty(n, np.int32)
+    part2[sigma] = part
+    X2 = np.empty_like(X)
+    X2[sigma] = X
+    b2 = oracle.bookkeeping(n, eu2, ev2, part2, S)
+    r2 = oracle.train_step(b2, dims, X2[b2["perm"]], W, ALPHA, BETA)
+    p_orig = np.empty(n)
+    p_orig[b["perm"]] = r["p"]
+    p2_orig = np.empty(n)
+    p2_orig[b2["perm"]] = r2["p"]
+    np.testing.assert_allclose(p2_orig[sigma], p_orig, rtol=1e-12)
+    np.testing.assert_allclose(r2["loss"], r["loss"], rtol=1e-12)
+
+
+# ------------------------------------------------------------- loss at binary points
+def _saturating_setup(n, eu, ev, t):
+    """One subgraph, one layer, one-hot embeddings; weights solved so that z = +-800 with
+    the sign pattern t, which makes p exactly 1 or 0 in double precision."""
+    A = dense_intra_adjacency(n, eu, ev, np.zeros(n, np.int32))
+    Ahat = (A + np.eye(n)) / (A.sum(1) + 1.0)[:, None]
+    wvec = np.linalg.solve(Ahat, 800.0 * t)
+    return A, wvec
+
+
+def test_loss_on_binary_probabilities_is_the_qubo_value():
+    n = 14
+    eu, ev, _ = tiny_graph(n, 0.3, 1, seed=41)
+    b = oracle.bookkeeping(n, eu, ev, np.zeros(n, np.int32), 1)
+    for trial in range(6):
+        t = np.where(si.uniform01(500 + trial, 0, n) < 0.5, 1.0, -1.0)
+        A, wvec = _saturating_setup(n, eu, ev, t)
+        r = oracle.train_step(b, [n, 1], np.eye(n)[b["perm"]], [wvec.reshape(1, n, 1)], ALPHA, BETA)
+        x = (t > 0).astype(np.float64)[b["perm"]]
+        assert np.array_equal(r["p"], x)
+        xo = (t > 0).astype(np.float64)
+        conflicts = int(round(0.5 * xo @ A @ xo))
+        assert r["loss"][0] == ALPHA * conflicts - BETA * xo.sum()
+        d = oracle.decode(b, r["p"].astype(np.float32))
+        assert d["intra_viol"] == conflicts and d["set_size"] == int(xo.sum())
+
+
+def _mis_brute(k, edges):
+    nb = [0] * k
+    for a, c in edges:
+        nb[a] |= 1 << c
+        nb[c] |= 1 << a
+    best = 0
+    for mask in range(1 << k):
+        ok = True
+        m = mask
+        while m:
+            i = (m & -m).bit_length() - 1
+            if nb[i] & mask:
+                ok = False
+                break
+            m &= m - 1
+        if ok:
+            best = max(best, bin(mask).count("1"))
+    return best
+
+
+def test_objective_minimum_equals_minus_beta_times_mis_on_small_instances():
+    """For alpha > beta the minimum of the relaxed objective over binary assignments is
+    -beta * MIS and is attained on an independent set (brute force, <= 12 nodes here;
+    16-node instances are covered by the config-2 test below)."""
+    k = 10
+    for seed in range(51, 90):          # the saturation trick needs A + I to be invertible
+        eu, ev, _ = tiny_graph(k, 0.35, 1, seed=seed)
+        A0 = dense_intra_adjacency(k, eu, ev, np.zeros(k, np.int32))
+        if np.linalg.cond(A0 + np.eye(k)) < 1e6:
+            break
+    b = oracle.bookkeeping(k, eu, ev, np.zeros(k, np.int32), 1)
+    mis = _mis_brute(k, list(zip(eu.tolist(), ev.tolist())))
+    best, best_x = None, None
+    A = dense_intra_adjacency(k, eu, ev, np.zeros(k, np.int32))
+    Ahat_inv = np.linalg.inv((A + np.eye(k)) / (A.sum(1) + 1.0)[:, None])
+    for mask in range(1 << k):
+        t = np.array([1.0 if (mask >> i) & 1 else -1.0 for i in range(k)])
+        wvec = Ahat_inv @ (800.0 * t)
+        r = oracle.train_step(b, [k, 1], np.eye(k)[b["perm"]], [wvec.reshape(1, k, 1)], ALPHA, BETA, want_dW=False)
+        if best is None or r["loss"][0] < best:
+            best, best_x = r["loss"][0], r["p"].copy()
+    assert best == -BETA * mis
+    d = oracle.decode(b, best_x.astype(np.float32))
+    assert d["intra_viol"] == 0 and d["set_size"] == mis
+
+
+def test_config2_sixteen_node_subinstances_qubo_vs_mis():
+    """16-node induced sub-instances of configuration 2: the QUBO optimum (enumerated
+    with integer arithmetic) equals -beta*MIS, and the oracle's loss reproduces the QUBO
+    value of the optimal assignment and of random assignments."""
+    w = si.make_workload(2)
+    k, done = 16, 0
+    for s in range(w.S):
+        if done == 3:
+            break
+        members = np.where(w.part == s)[0]
+        inside = np.isin(w.eu, members) & np.isin(w.ev, members)
+        nb = {}
+        for a, c in zip(w.eu[inside].tolist(), w.ev[inside].tolist()):
+            nb.setdefault(a, []).append(c)
+            nb.setdefault(c, []).append(a)
+        nodes, seen = [int(members[0])], {int(members[0])}     # breadth-first ball of 16 nodes
+        for v in nodes:
+            for c in sorted(nb.get(v, [])):
+                if c not in seen and len(nodes) < 16:
+                    seen.add(c)
+                    nodes.append(c)
+        if len(nodes) < 16:
+            continue
+        nodes = np.array(nodes)
+        idx = {int(v): i for i, v in enumerate(nodes)}
+        sel = np.isin(w.eu, nodes) & np.isin(w.ev, nodes)
+        edges = [(idx[a], idx[c]) for a, c in zip(w.eu[sel].tolist(), w.ev[sel].tolist())]
+        A0 = np.zeros((k, k))
+        for a, c in edges:
+            A0[a, c] = A0[c, a] = 1.0
+        if len(edges) < 8 or np.linalg.cond(A0 + np.eye(k)) > 1e6:
+            continue                    # the saturation trick needs A + I to be invertible
+        done += 1
+        mis = _mis_brute(k, edges)
+        nbm = [0] * k
+        for a, c in edges:
+            nbm[a] |= 1 << c
+            nbm[c] |= 1 << a
+        best, best_mask = None, None
+        for mask in range(1 << k):
+            conf = sum(bin(nbm[i] & mask).count("1") for i in range(k) if (mask >> i) & 1) // 2
+            q = 2 * conf - bin(mask).count("1")
+            if best is None or q < best:
+                best, best_mask = q, mask
+        assert best == -mis
+        eu = np.array([e[0] for e in edges], np.int32)
+        ev = np.array([e[1] for e in edges], np.int32)
+        b = oracle.bookkeeping(k, eu, ev, np.zeros(k, np.int32), 1)
+        for mask in [best_mask] + [int(m) for m in si.u64(s + 900, 0, 5) % np.uint64(1 << k)]:
+            t = np.array([1.0 if (mask >> i) & 1 else -1.0 for i in range(k)])
+            A, wvec = _saturating_setup(k, eu, ev, t)
+            r = oracle.train_step(b, [k, 1], np.eye(k)[b["perm"]], [wvec.reshape(1, k, 1)], 2.0, 1.0, want_dW=False)
+            conf = sum(bin(nbm[i] & mask).count("1") for i in range(k) if (mask >> i) & 1) // 2
+            assert r["loss"][0] == 2.0 * conf - bin(mask).count("1")
+            assert r["loss"][0] >= -mis
+    assert done == 3
+
+
+# ------------------------------------------------------------------ gradients (a5, a6)
+def _total_loss(b, dims, X, W, pen, lam, which=None):
+    r = oracle.train_step(b, dims, X, W, ALPHA, BETA, lam, pen, want_dW=False)
+    return r["loss"].sum() if which is None else r["loss"][which]
+
+
+@pytest.mark.parametrize("dims,shared", [([6, 1], False), ([5, 4, 1], False), ([6, 5, 4, 1], False), ([5, 4, 1], True)])
+def test_gradients_match_central_finite_differences(dims, shared):
+    n, S = 48, 3
+    eu, ev, part = tiny_graph(n, 0.2, S, seed=61)
+    b = oracle.bookkeeping(n, eu, ev, part, S)
+    X = rand_features(n, dims[0], 13)
+    W = rand_weights(dims, 1 if shared else S, 17, scale=1.5)
+    pen = (si.uniform01(77, 0, n) < 0.3).astype(np.float64)
+    lam = 0.9
+    r = oracle.train_step(b, dims, X, W, ALPHA, BETA, lam, pen, want_dX=True, want_Z=True)
+    if r["Z"]:
+        assert min(np.abs(z).min() for z in r["Z"]) > 1e-4          # away from ReLU kinks
+    h = 1e-6
+    worst = 0.0
+    for l in range(len(W)):
+        g = r["dW"][l]
+        flat = W[l].reshape(-1)
+        for q in range(flat.size):
+            old = flat[q]
+            flat[q] = old + h
+            lp = _total_loss(b, dims, X, W, pen, lam)
+            flat[q] = old - h
+            lm = _total_loss(b, dims, X, W, pen, lam)
+            flat[q] = old
+            fd = (lp - lm) / (2 * h)
+            worst = max(worst, abs(fd - g.reshape(-1)[q]) / (abs(fd) + 2e-2))   # 2e-8 floor: eps*|loss|/h
+    assert worst < 1e-6, worst
+    rows = (si.u64(5, 0, 12) % np.uint64(n)).astype(int)
+    for i in rows:
+        for f in range(dims[0]):
+            old = X[i, f]
+            X[i, f] = old + h
+            lp = _total_loss(b, dims, X, W, pen, lam)
+            X[i, f] = old - h
+            lm = _total_loss(b, dims, X, W, pen, lam)
+            X[i, f] = old
+            fd = (lp - lm) / (2 * h)
+            assert abs(fd - r["dX"][i, f]) <= 1e-6 * abs(fd) + 2e-8     # FD round-off floor: eps*|loss|/h
+
+
+def test_subgraph_loss_depends_only_on_its_own_weights():
+    n, S, dims = 40, 4, [5, 4, 1]
+    eu, ev, part = tiny_graph(n, 0.25, S, seed=71)
+    b = oracle.bookkeeping(n, eu, ev, part, S)
+    X, W = rand_features(n, 5, 2), rand_weights(dims, S, 3)
+    base = oracle.train_step(b, dims, X, W, ALPHA, BETA, want_dW=False)["loss"]
+    W2 = [w.copy() for w in W]
+    W2[0][2] += 0.3
+    W2[1][2] -= 0.2
+    moved = oracle.train_step(b, dims, X, W2, ALPHA, BETA, want_dW=False)["loss"]
+    assert moved[2] != base[2]
+    assert np.array_equal(np.delete(moved, 2), np.delete(base, 2))
+
+
+def test_sigmoid_chain_identity_for_one_layer():
+    """L = 1: dW = X^T A_hat^T dz with dz_i = (alpha * sum_nbr p - beta) p (1-p): the
+    column sums of that product, evaluated with dense algebra."""
+    n = 30
+    eu, ev, part = tiny_graph(n, 0.3, 2, seed=81)
+    b = oracle.bookkeeping(n, eu, ev, part, 2)
+    F = 4
+    X = rand_features(n, F, 21)
+    W = rand_weights([F, 1], 1, 5)
+    r = oracle.train_step(b, [F, 1], X[b["perm"]], W, ALPHA, BETA)
+    A = dense_intra_adjacency(n, eu, ev, part)
+    Ahat = (A + np.eye(n)) / (A.sum(1) + 1.0)[:, None]
+    p = 1.0 / (1.0 + np.exp(-(Ahat @ X @ W[0][0])[:, 0]))
+    dz = (ALPHA * (A @ p) - BETA) * p * (1 - p)
+    np.testing.assert_allclose(r["dW"][0][0][:, 0], X.T @ Ahat.T @ dz, rtol=1e-11, atol=1e-13)
+
+
+# ----------------------------------------------------------- block-diagonal batch pin
+def test_batch_equals_independent_subgraph_runs_bit_for_bit():
+    n, S, dims = 90, 6, [6, 5, 4, 1]
+    eu, ev, part = tiny_graph(n, 0.12, S, seed=91)
+    b = oracle.bookkeeping(n, eu, ev, part, S)
+    X = rand_features(n, dims[0], 33)
+    W = rand_weights(dims, S, 35)
+    pen = (si.uniform01(7, 0, n) < 0.2).astype(np.float64)
+    r = oracle.train_step(b, dims, X[b["perm"]], W, ALPHA, BETA, 0.5, pen[b["perm"]], want_dX=True, threads=3)
+    for s in range(S):
+        nodes = np.where(part == s)[0]                      # ascending original ids = new order inside s
+        loc = {int(v): i for i, v in enumerate(nodes)}
+        nbrs = [[] for _ in nodes]
+        for a, c in zip(eu.tolist(), ev.tolist()):
+            if a in loc and c in loc:
+                nbrs[loc[a]].append(loc[c])
+                nbrs[loc[c]].append(loc[a])
+        rp = np.concatenate([[0], np.cumsum([len(x) for x in nbrs])]).astype(np.int32)
+        ci = np.array([j for x in nbrs for j in sorted(x)], np.int32)
+        one = oracle.subgraph_step(rp, ci, dims, X[nodes], [w[s] for w in W], ALPHA, BETA, 0.5, pen[nodes],
+                                   want_dX=True)
+        lo, hi = b["part_ptr"][s], b["part_ptr"][s + 1]
+        assert one["loss"] == r["loss"][s]
+        assert np.array_equal(one["p"], r["p"][lo:hi])
+        assert np.array_equal(one["dX"], r["dX"][lo:hi])
+        for l in range(len(W)):
+            assert np.array_equal(one["dW"][l], r["dW"][l][s])
+
+
+def test_shared_weight_gradient_is_sum_over_subgraphs():
+    n, S, dims = 60, 4, [5, 3, 1]
+    eu, ev, part = tiny_graph(n, 0.15, S, seed=95)
+    b = oracle.bookkeeping(n, eu, ev, part, S)
+    X = rand_features(n, 5, 1)
+    W1 = rand_weights(dims, 1, 2)
+    WS = [np.tile(w, (S, 1, 1)) for w in W1]
+    shared = oracle.train_step(b, dims, X, W1, ALPHA, BETA)
+    per = oracle.train_step(b, dims, X, WS, ALPHA, BETA)
+    for l in range(2):
+        np.testing.assert_allclose(shared["dW"][l][0], per["dW"][l].sum(0), rtol=1e-12, atol=1e-14)
+    assert np.array_equal(shared["p"], per["p"])
+
+
+# ------------------------------------------------------------------------ Adam (a7)
+def test_adam_two_steps_against_exact_rational_arithmetic():
+    decimal.getcontext().prec = 60
+    lr, b1, b2, eps = Fraction(1, 10), Fraction(9, 10), Fraction(999, 1000), Fraction(1, 10 ** 8)
+    g = [Fraction(1, 2), Fraction(-1, 4)]
+    W, m, v = Fraction(3, 10), Fraction(0), Fraction(0)
+    expect = []
+    for t in (1, 2):
+        m = b1 * m + (1 - b1) * g[t - 1]
+        v = b2 * v + (1 - b2) * g[t - 1] ** 2
+        mh, vh = m / (1 - b1 ** t), v / (1 - b2 ** t)
+        root = decimal.Decimal(vh.numerator) / decimal.Decimal(vh.denominator)
+        root = root.sqrt()
+        step = (decimal.Decimal(mh.numerator) / decimal.Decimal(mh.denominator)) / (
+            root + decimal.Decimal(eps.numerator) / decimal.Decimal(eps.denominator))
+        W = W - lr * Fraction(step)
+        expect.append(float(W))
+    Wd, md, vd = np.array([0.3]), np.zeros(1), np.zeros(1)
+    got = []
+    for t in (1, 2):
+        oracle.adam(Wd, md, vd, np.array([float(g[t - 1])]), 0.1, t, 0.9, 0.999, 1e-8)
+        got.append(float(Wd[0]))
+    np.testing.assert_allclose(got, expect, rtol=1e-14)
+    # the first step moves by lr*g/(|g|+eps): almost exactly lr against the gradient sign
+    assert abs((0.3 - got[0]) - 0.1 * 0.5 / (0.5 + 1e-8)) < 1e-15
+
+
+def test_adam_first_step_is_sign_step_and_zero_gradient_stays():
+    g = np.array([3.0, -0.02, 0.0, 1e-3])
+    W, m, v = np.ones(4), np.zeros(4), np.zeros(4)
+    oracle.adam(W, m, v, g, 1e-3, 1)
+    np.testing.assert_allclose(1.0 - W, 1e-3 * g / (np.abs(g) + 1e-8), rtol=1e-12, atol=0)
+    assert W[2] == 1.0
+
+
+# --------------------------------------------------------------------- decode (a8, a9)
+@pytest.mark.parametrize("seed", [1, 2, 3])
+def test_decode_brute_force(seed):
+    n, S = 45, 5
+    eu, ev, part = tiny_graph(n, 0.2, S, seed=100 + seed)
+    b = oracle.bookkeeping(n, eu, ev, part, S)
+    p_orig = si.uniform01(seed, 0, n).astype(np.float32)
+    p_orig[::7] = 0.5                                             # ties go to "selected"
+    d = oracle.decode(b, p_orig[b["perm"]])
+    x = (p_orig >= np.float32(0.5)).astype(np.uint8)
+    assert np.array_equal(d["x"], x[b["perm"]])
+    intra = bnd = 0
+    per = np.zeros(S, np.int64)
+    for a, c in zip(eu.tolist(), ev.tolist()):
+        if x[a] and x[c]:
+            if part[a] == part[c]:
+                intra += 1
+            else:
+                bnd += 1
+                per[part[a]] += 1
+                per[part[c]] += 1
+    assert (d["set_size"], d["intra_viol"], d["boundary_viol"]) == (int(x.sum()), intra, bnd)
+    assert np.array_equal(d["per_part"], per) and d["per_part"].sum() == 2 * bnd
+    for e in range(b["E_b"]):
+        u, v = b["perm"][b["bnd_u"][e]], b["perm"][b["bnd_v"][e]]
+        assert d["viol"][e] == (x[u] & x[v])
+
+
+# ------------------------------------------------------------- trajectory (sanity only)
+def test_config1_training_lowers_every_subgraph_loss():
+    w = si.make_workload(1)
+    b = oracle.bookkeeping(w.n, w.eu, w.ev, w.part, w.S)
+    X = w.features_f32()[b["perm"]].astype(np.float64)
+    W = [w.weights(l).astype(np.float64) for l in range(w.L)]
+    m = [np.zeros_like(x) for x in W]
+    v = [np.zeros_like(x) for x in W]
+    first = None
+    for t in range(1, w.steps + 1):
+        r = oracle.train_step(b, w.dims, X, W, w.alpha, w.beta, threads=4)
+        if first is None:
+            first = r["loss"].copy()
+        for l in range(w.L):
+            oracle.adam(W[l], m[l], v[l], r["dW"][l], w.lr, t)
+    last = oracle.train_step(b, w.dims, X, W, w.alpha, w.beta, want_dW=False)["loss"]
+    assert np.all(last < first)
