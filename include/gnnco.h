@@ -1,0 +1,214 @@
+/*
+ * gnnco -- partitioned-GNN training step for combinatorial optimisation on one GPU.
+ *
+ * C ABI of the CUDA library.  The calls follow the problem statement of the method
+ * (Algorithm 1: inputs "graph G, subgraph set {G_i}, QUBO Q", output "bitstring x"):
+ *
+ *   gnnco_partition_load   graph + partition  -> block-diagonal batch of subgraphs
+ *                          (Section 3.3, first paragraph; Algorithm 1, Stage 2 masks)
+ *   gnnco_train_step       one full-batch GCN training step over every subgraph
+ *                          (Section 3.2, Eqs. 3-5; penalty term of Section 3.3;
+ *                          Algorithm 1, Stage 1)
+ *   gnnco_decode_boundary  threshold the probabilities and count conflicts on
+ *                          cross-subgraph edges (Section 3.3; Algorithm 1, Stage 2 and
+ *                          the first line of Stage 3)
+ *
+ * General rules
+ *   - Every function returns a gnnco_status (0 = success, negative = error); nothing
+ *     throws, aborts or traps the device.
+ *   - All buffers are CALLER-OWNED.  The library allocates no device memory; sizes of
+ *     work areas come from the *_workspace_bytes queries.  Work areas must be 256-byte
+ *     aligned.
+ *   - Unless a parameter says "host", pointers are DEVICE pointers of the current
+ *     CUDA device.  `stream` is a cudaStream_t passed as void*.
+ *   - Per-node arrays (X, p, x, pen, dX, z) are in the library's NEW node order, in
+ *     which every subgraph is a contiguous id range; `perm` (new -> original) and
+ *     `inv_perm` (original -> new) from gnnco_graph_info map back to the caller's ids.
+ *   - Dense matrices are row-major.
+ */
+#ifndef GNNCO_H_
+#define GNNCO_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define GNNCO_MAX_LAYERS 8
+
+typedef enum {
+  GNNCO_OK = 0,
+  GNNCO_INVALID_ARGUMENT = -1,    /* null pointer, bad size, bad enum, misaligned work area */
+  GNNCO_OUT_OF_RANGE = -2,        /* node id or partition id outside its range */
+  GNNCO_NOT_SIMPLE_GRAPH = -3,    /* self loop or repeated edge */
+  GNNCO_UNSUPPORTED = -4,         /* dtype / width combination not implemented */
+  GNNCO_WORKSPACE_TOO_SMALL = -5,
+  GNNCO_CUDA_ERROR = -6,
+  GNNCO_INTERNAL = -7
+} gnnco_status;
+
+typedef enum { GNNCO_F32 = 0, GNNCO_BF16 = 1 } gnnco_dtype;
+
+/* flags of gnnco_train_step */
+#define GNNCO_WANT_DX 1u        /* also compute d loss / d X (runs the transposed aggregation of layer 1) */
+#define GNNCO_FORWARD_ONLY 2u   /* stop after loss and p (Algorithm 1, Stage 2: "run forward to get p_i") */
+
+typedef struct gnnco_handle gnnco_handle;
+
+/* Input graph: undirected, unweighted, simple.  Edge e joins edge_u[e] and edge_v[e]
+ * (each edge listed once, either orientation); part[i] in [0, S) is node i's subgraph. */
+typedef struct {
+  int64_t n;                /* nodes, 1 <= n < 2^31 */
+  int64_t E;                /* undirected edges, 0 <= E, 2E < 2^31 */
+  int32_t S;                /* subgraphs, 1 <= S <= n */
+  const int32_t* edge_u;    /* [E] */
+  const int32_t* edge_v;    /* [E] */
+  const int32_t* part;      /* [n] */
+} gnnco_graph_desc;
+
+/* Read-only view of what gnnco_partition_load built (pointers live in the caller's
+ * persistent work area and stay valid until gnnco_destroy). */
+typedef struct {
+  int64_t n;
+  int32_t S;
+  int64_t E_in;                 /* intra-subgraph edges */
+  int64_t E_b;                  /* boundary (cross-subgraph) edges */
+  int32_t max_row;              /* largest intra degree */
+  const int32_t* perm;          /* [n]   new id -> original id */
+  const int32_t* inv_perm;      /* [n]   original id -> new id */
+  const int32_t* part_ptr;      /* [S+1] subgraph s owns new ids part_ptr[s] .. part_ptr[s+1]-1 */
+  const int32_t* node_part;     /* [n]   subgraph of each new id */
+  const int32_t* rowptr;        /* [n+1] CSR of intra edges, both directions, no self loops */
+  const int32_t* colidx;        /* [2*E_in] ascending inside a row */
+  const int32_t* bnd_u;         /* [E_b] boundary edges in new ids, bnd_u < bnd_v, sorted by (u, v) */
+  const int32_t* bnd_v;         /* [E_b] */
+  const float* inv_deg;         /* [n]   1 / (intra degree + 1), Eq. 3's normaliser */
+  const uint8_t* is_boundary;   /* [n]   1 iff the node touches a boundary edge ("cross-node") */
+} gnnco_graph_view;
+
+/* GCN of L layers, widths dims[0] -> dims[1] -> ... -> dims[L] with dims[L] == 1
+ * (Eq. 3 per layer, ReLU on hidden layers; Eq. 4 on the last layer's scalar).
+ * W[l] is layer l's weight, [weight_sets x dims[l] x dims[l+1]] float32; weight_sets is
+ * S (one model per subgraph, Algorithm 1 Stage 1) or 1 (one shared model).
+ * feat_dtype is the storage type of X and of the activations the library keeps;
+ * accumulation is always float32.  With GNNCO_BF16 the weights are rounded to bf16
+ * for the matrix products while W itself (the master copy Adam updates) stays float32. */
+typedef struct {
+  int32_t L;
+  int32_t dims[GNNCO_MAX_LAYERS + 1];
+  int32_t feat_dtype;            /* gnnco_dtype */
+  int32_t weight_sets;
+  float* W[GNNCO_MAX_LAYERS];
+} gnnco_model_desc;
+
+/* Eq. 5 with the fine-tuning penalty of Section 3.3:
+ *   loss_s = alpha * sum_{intra edges (i,j) of s} p_i p_j - beta * sum_{i in s} p_i
+ *            + lambda * sum_{i in s} pen[i] * p_i
+ * pen may be NULL (no penalty). */
+typedef struct {
+  float alpha, beta, lambda;
+  const float* pen;              /* [n] or NULL */
+} gnnco_objective;
+
+/* Adam state (bias-corrected; eps outside the square root).  `step` is the 1-based
+ * number of THIS update; the caller increments it between calls.  m[l], v[l] have the
+ * shape of W[l]. */
+typedef struct {
+  float lr, beta1, beta2, eps;
+  int64_t step;
+  float* m[GNNCO_MAX_LAYERS];
+  float* v[GNNCO_MAX_LAYERS];
+} gnnco_adam_state;
+
+/* Outputs of a training step.  loss and p are required; the rest may be NULL. */
+typedef struct {
+  float* loss;                   /* [S]  per-subgraph objective */
+  float* p;                      /* [n]  selection probabilities (Eq. 4) */
+  float* z;                      /* [n]  pre-sigmoid values, or NULL */
+  float* dW[GNNCO_MAX_LAYERS];   /* gradient of sum_s loss_s wrt W[l], shape of W[l], or NULL */
+  void* dX;                      /* [n x dims[0]] in feat_dtype; written only with GNNCO_WANT_DX */
+} gnnco_train_out;
+
+typedef struct {
+  int64_t set_size;              /* number of selected nodes */
+  int64_t intra_viol;            /* intra edges with both ends selected */
+  int64_t boundary_viol;         /* boundary edges with both ends selected */
+} gnnco_counts;
+
+const char* gnnco_status_string(int32_t status);
+
+/* Sizes (bytes) of the two work areas of gnnco_partition_load for a graph of n nodes,
+ * E edges and S subgraphs: `persistent` must outlive the handle, `scratch` may be
+ * released when gnnco_partition_load returns. */
+int32_t gnnco_partition_workspace_bytes(int64_t n, int64_t E, int32_t S, size_t* persistent, size_t* scratch);
+
+/* Build the block-diagonal batch (Section 3.3: split into subgraphs; cross edges set
+ * aside).  New ids rank nodes by (part, original id); intra edges become a symmetric
+ * CSR; boundary edges a sorted list.  All integer results are exactly defined (no
+ * ordering freedom).  Runs on `stream` and synchronises it (sizes and the validation
+ * result must reach the host).  On success *out receives a handle (host object, freed by
+ * gnnco_destroy).  Errors: GNNCO_OUT_OF_RANGE, GNNCO_NOT_SIMPLE_GRAPH,
+ * GNNCO_WORKSPACE_TOO_SMALL, GNNCO_INVALID_ARGUMENT, GNNCO_CUDA_ERROR. */
+int32_t gnnco_partition_load(const gnnco_graph_desc* g, void* persistent_ws, size_t persistent_bytes,
+                             void* scratch_ws, size_t scratch_bytes, void* stream, gnnco_handle** out);
+
+int32_t gnnco_graph_info(const gnnco_handle* h, gnnco_graph_view* out);
+
+/* dst[i] = src[index[i]] for i < rows, rows of row_bytes bytes each (row_bytes a
+ * multiple of 4).  With index = perm it brings a per-node array from the caller's
+ * original order into the new order (Algorithm 1, Stage 2 uses the inverse to "map
+ * local probs to global mask"): pass inv_perm to go back. */
+int32_t gnnco_gather_rows(const gnnco_handle* h, const void* src, void* dst, const int32_t* index, int64_t rows,
+                          int64_t row_bytes, void* stream);
+
+/* Work-area size of gnnco_train_step for this graph and model. */
+int32_t gnnco_train_workspace_bytes(const gnnco_handle* h, const gnnco_model_desc* m, uint32_t flags, size_t* bytes);
+
+/* One training step over all subgraphs at once (Section 3.2):
+ *   forward   per hidden layer  H' = ReLU( mean_{self + intra neighbours}(H) W_s )   (Eq. 3)
+ *             last layer        z = mean_{self + intra neighbours}(H) w_s,  p = sigmoid(z)   (Eq. 4)
+ *   objective loss_s as in gnnco_objective                                           (Eq. 5)
+ *   backward  exact gradient of sum_s loss_s wrt every W (and X with GNNCO_WANT_DX)
+ *   update    Adam on every W (skipped when opt == NULL or with GNNCO_FORWARD_ONLY)
+ * X is [n x dims[0]] in feat_dtype, new node order, and is not modified.  Asynchronous
+ * on `stream`; per-subgraph results are deterministic (no floating-point atomics). */
+int32_t gnnco_train_step(gnnco_handle* h, const gnnco_model_desc* m, const void* X, const gnnco_objective* obj,
+                         gnnco_adam_state* opt, const gnnco_train_out* out, uint32_t flags, void* ws,
+                         size_t ws_bytes, void* stream);
+
+/* Same step with HOST buffers for the per-step data: X_host [n x dims[0]] (feat_dtype,
+ * new order; pinned memory recommended), pen_host [n] or NULL, loss_host [S], p_host [n].
+ * Weights, Adam moments and the work area stay on the device.  Copies run on `stream`,
+ * which is synchronised before returning.  ws must hold
+ * gnnco_train_host_workspace_bytes bytes. */
+int32_t gnnco_train_host_workspace_bytes(const gnnco_handle* h, const gnnco_model_desc* m, uint32_t flags,
+                                         size_t* bytes);
+int32_t gnnco_train_step_host(gnnco_handle* h, const gnnco_model_desc* m, const void* X_host, float alpha,
+                              float beta, float lambda, const float* pen_host, gnnco_adam_state* opt,
+                              float* loss_host, float* p_host, uint32_t flags, void* ws, size_t ws_bytes,
+                              void* stream);
+
+/* Decode (Section 3.3): x[i] = (p[i] >= threshold) on the stored float32 value; a
+ * boundary edge is violated when both ends are selected.
+ *   x        [n] uint8, required          viol     [E_b] uint8 or NULL
+ *   per_part [S] int32 or NULL: violated boundary edges touching subgraph s (an edge
+ *            counts for both of its subgraphs, so the entries sum to 2*boundary_viol)
+ *   counts   device gnnco_counts, required
+ * Integer results are exact.  Asynchronous on `stream`; needs no work area. */
+int32_t gnnco_decode_boundary(const gnnco_handle* h, const float* p, float threshold, uint8_t* x, uint8_t* viol,
+                              int32_t* per_part, gnnco_counts* counts, void* stream);
+
+/* Host read of the device-side status word (synchronises `stream`). */
+int32_t gnnco_async_status(const gnnco_handle* h, void* stream, int32_t* status);
+
+/* Number of kernels this handle has launched so far (for launch accounting). */
+int64_t gnnco_launch_count(const gnnco_handle* h);
+
+int32_t gnnco_destroy(gnnco_handle* h);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* GNNCO_H_ */

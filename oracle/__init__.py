@@ -38,10 +38,10 @@ def _native():
         i64, i32, dbl, vp, flt = ctypes.c_int64, ctypes.c_int32, ctypes.c_double, ctypes.c_void_p, ctypes.c_float
         lib.oracle_bookkeeping.argtypes = [i64, i64, vp, vp, vp, i32] + [vp] * 12
         lib.oracle_bookkeeping.restype = ctypes.c_int
-        lib.oracle_subgraph_step.argtypes = [i32, vp, vp, i32, vp, vp, vp, dbl, dbl, dbl, vp, vp, vp, vp, vp, vp, vp]
+        lib.oracle_subgraph_step.argtypes = [i32, vp, vp, i32, vp, vp, vp, dbl, dbl, dbl, vp, vp, vp, vp, vp, vp, vp, i32]
         lib.oracle_subgraph_step.restype = ctypes.c_int
         lib.oracle_train_step.argtypes = [i64, i32, vp, vp, vp, i32, vp, i32, vp, vp, dbl, dbl, dbl,
-                                          vp, vp, vp, vp, vp, vp, vp, i32]
+                                          vp, vp, vp, vp, vp, vp, vp, i32, i32]
         lib.oracle_train_step.restype = ctypes.c_int
         lib.oracle_adam.argtypes = [i64, vp, vp, vp, vp, dbl, dbl, dbl, dbl, i64]
         lib.oracle_adam.restype = None
@@ -101,8 +101,9 @@ def _as_f64(a):
 
 def subgraph_step(rowptr, colidx, dims: Sequence[int], X, W: Sequence[np.ndarray], alpha: float, beta: float,
                   lam: float = 0.0, pen=None, want_dW: bool = True, want_dX: bool = False,
-                  want_Z: bool = False) -> Dict[str, object]:
-    """One standalone subgraph with local ids: forward, loss and exact gradients."""
+                  want_Z: bool = False, store_bf16: bool = False) -> Dict[str, object]:
+    """One standalone subgraph with local ids: forward, loss and exact gradients.
+    ``store_bf16`` rounds the stored hidden tensors (M_l, H_l) to bfloat16."""
     rowptr = np.ascontiguousarray(rowptr, dtype=np.int32)
     colidx = np.ascontiguousarray(colidx, dtype=np.int32)
     ns, L = rowptr.size - 1, len(dims) - 1
@@ -118,7 +119,7 @@ def subgraph_step(rowptr, colidx, dims: Sequence[int], X, W: Sequence[np.ndarray
     rc = _native().oracle_subgraph_step(
         ns, _ptr(rowptr), _ptr(colidx), L, _ptr(dims_a), _ptr(X), _ptr_array(Wd), alpha, beta, lam, _ptr(pen),
         _ptr(loss), _ptr(z), _ptr(p), _ptr_array(dW) if dW is not None else None, _ptr(dX),
-        _ptr_array(Z + [None]) if Z is not None else None)
+        _ptr_array(Z + [None]) if Z is not None else None, int(store_bf16))
     if rc != 0:
         raise OracleError(rc, "oracle_subgraph_step")
     return dict(loss=float(loss[0]), z=z, p=p, dW=dW, dX=dX, Z=Z)
@@ -126,7 +127,7 @@ def subgraph_step(rowptr, colidx, dims: Sequence[int], X, W: Sequence[np.ndarray
 
 def train_step(book: Dict[str, np.ndarray], dims: Sequence[int], X, W: Sequence[np.ndarray], alpha: float, beta: float,
                lam: float = 0.0, pen=None, want_dW: bool = True, want_dX: bool = False, want_Z: bool = False,
-               threads: int = 1) -> Dict[str, object]:
+               threads: int = 1, store_bf16: bool = False) -> Dict[str, object]:
     """Block-diagonal batch over all subgraphs of ``book`` (the dict returned by
     ``bookkeeping``).  ``X`` is [n, F_0] in the NEW node order; ``W[l]`` is
     [S, F_l, F_{l+1}] (one set per subgraph) or [1, F_l, F_{l+1}] (shared)."""
@@ -148,7 +149,7 @@ def train_step(book: Dict[str, np.ndarray], dims: Sequence[int], X, W: Sequence[
         n, S, _ptr(book["part_ptr"]), _ptr(book["rowptr"]), _ptr(book["colidx"]), L, _ptr(dims_a), sets, _ptr(X),
         _ptr_array(Wd), alpha, beta, lam, _ptr(pen), _ptr(loss), _ptr(z), _ptr(p),
         _ptr_array(dW) if dW is not None else None, _ptr(dX), _ptr_array(Z + [None]) if Z is not None else None,
-        threads)
+        threads, int(store_bf16))
     if rc <= 0:
         raise OracleError(rc, "oracle_train_step")
     return dict(loss=loss, z=z, p=p, dW=dW, dX=dX, Z=Z, threads=rc)

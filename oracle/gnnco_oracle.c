@@ -41,6 +41,19 @@ static int cmp_pair(const void* a, const void* b) {
   return (x[1] > y[1]) - (x[1] < y[1]);
 }
 
+/* Round a double to the nearest-even bfloat16 value (via float), returned as double.
+ * Used only where a workload fixes bfloat16 STORAGE of activations. */
+static double round_bf16(double x) {
+  float f = (float)x;
+  uint32_t u;
+  memcpy(&u, &f, 4);
+  if ((u & 0x7F800000u) == 0x7F800000u) return (double)f;      /* inf / nan unchanged */
+  u += 0x7FFFu + ((u >> 16) & 1u);
+  u &= 0xFFFF0000u;
+  memcpy(&f, &u, 4);
+  return (double)f;
+}
+
 /*
  * Bookkeeping (Section 3.3, first paragraph: the graph is split into subgraphs, and
  * "cross-nodes" are the endpoints of edges whose ends lie in different subgraphs;
@@ -146,11 +159,18 @@ int oracle_bookkeeping(int64_t n, int64_t E, const int32_t* eu, const int32_t* e
  * W[l] points at this subgraph's F_l x F_{l+1} matrix of layer l (0-based).
  * dW[l] (if dW != NULL) receives the gradient; dX (if != NULL) receives d loss / d X.
  * Zsave[l] (if Zsave != NULL), l < L-1, receives the pre-activations of hidden layer l.
+ *
+ * store_bf16 != 0 models a workload whose activations are STORED in bfloat16 while all
+ * sums are carried at higher precision (the "bf16 embeddings, fp32 accumulation"
+ * benchmark configuration): the aggregated input M_l and the activation H_l of every
+ * hidden layer are rounded to the nearest bfloat16 before they are used again.  The
+ * ReLU mask is a 0/1 decision taken from floating point, so it must be taken on values
+ * of the same precision on both sides of a comparison.  Everything else stays double.
  */
 static int subgraph_step(int32_t ns, const int32_t* rp, const int32_t* ci, int32_t L, const int32_t* dims,
                          const double* X, const double* const* W, double alpha, double beta, double lambda,
                          const double* pen, double* loss_out, double* z_out, double* p_out, double* const* dW,
-                         double* dX, double* const* Zsave) {
+                         double* dX, double* const* Zsave, int store_bf16) {
   int rc = ORACLE_OK;
   double** H = (double**)calloc((size_t)L + 1, sizeof(double*));   /* H[0] = X, H[l] = output of layer l */
   double** M = (double**)calloc((size_t)L + 1, sizeof(double*));   /* M[l] = aggregated input of layer l (1-based) */
@@ -174,6 +194,8 @@ static int subgraph_step(int32_t ns, const int32_t* rp, const int32_t* ci, int32
       }
       double inv = 1.0 / (double)(rp[i + 1] - rp[i] + 1);
       for (int32_t f = 0; f < fi; ++f) m[f] *= inv;
+      if (store_bf16 && l < L)
+        for (int32_t f = 0; f < fi; ++f) m[f] = round_bf16(m[f]);     /* aggregated tensor is stored */
       double* zr = Z[l] + (size_t)i * fo;
       for (int32_t f = 0; f < fi; ++f) {
         double mf = m[f];
@@ -183,6 +205,8 @@ static int subgraph_step(int32_t ns, const int32_t* rp, const int32_t* ci, int32
       if (l < L) {
         double* hr = H[l] + (size_t)i * fo;
         for (int32_t h = 0; h < fo; ++h) hr[h] = zr[h] > 0.0 ? zr[h] : 0.0;
+        if (store_bf16)
+          for (int32_t h = 0; h < fo; ++h) hr[h] = round_bf16(hr[h]);   /* activation is stored */
       }
     }
     if (l < L && Zsave && Zsave[l - 1]) memcpy(Zsave[l - 1], Z[l], (size_t)ns * fo * sizeof(double));
@@ -269,9 +293,10 @@ done:
 int oracle_subgraph_step(int32_t ns, const int32_t* rowptr, const int32_t* colidx, int32_t L, const int32_t* dims,
                          const double* X, const double* const* W, double alpha, double beta, double lambda,
                          const double* pen, double* loss, double* z, double* p, double* const* dW, double* dX,
-                         double* const* Zsave) {
+                         double* const* Zsave, int32_t store_bf16) {
   if (ns <= 0 || L < 1) return ORACLE_BAD_ARG;
-  return subgraph_step(ns, rowptr, colidx, L, dims, X, W, alpha, beta, lambda, pen, loss, z, p, dW, dX, Zsave);
+  return subgraph_step(ns, rowptr, colidx, L, dims, X, W, alpha, beta, lambda, pen, loss, z, p, dW, dX, Zsave,
+                       store_bf16);
 }
 
 /*
@@ -287,7 +312,7 @@ int oracle_subgraph_step(int32_t ns, const int32_t* rowptr, const int32_t* colid
 int oracle_train_step(int64_t n, int32_t S, const int32_t* part_ptr, const int32_t* rowptr, const int32_t* colidx,
                       int32_t L, const int32_t* dims, int32_t weight_sets, const double* X, const double* const* W,
                       double alpha, double beta, double lambda, const double* pen, double* loss, double* z, double* p,
-                      double* const* dW, double* dX, double* const* Zsave, int32_t threads) {
+                      double* const* dW, double* dX, double* const* Zsave, int32_t threads, int32_t store_bf16) {
   if (n <= 0 || S <= 0 || L < 1 || L > 16 || (weight_sets != 1 && weight_sets != S)) return ORACLE_BAD_ARG;
   int rc = ORACLE_OK;
   int used = 1;
@@ -337,7 +362,7 @@ int oracle_train_step(int64_t n, int32_t S, const int32_t* part_ptr, const int32
     }
     int r = subgraph_step(ns, rp, ci, L, dims, X + (size_t)r0 * dims[0], Ws, alpha, beta, lambda,
                           pen ? pen + r0 : NULL, loss + s, z ? z + r0 : NULL, p + r0, dW ? dWs : NULL,
-                          dX ? dX + (size_t)r0 * dims[0] : NULL, Zsave ? Zs : NULL);
+                          dX ? dX + (size_t)r0 * dims[0] : NULL, Zsave ? Zs : NULL, store_bf16);
     if (r != ORACLE_OK) {
 #pragma omp critical
       rc = r;

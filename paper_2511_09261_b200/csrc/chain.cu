@@ -1,0 +1,141 @@
+// The width-1 tail of the training step: output-layer aggregation and sigmoid (Eq. 4),
+// the relaxed objective with its per-subgraph reduction (Eq. 5 plus the fine-tuning
+// penalty of Section 3.3), and the gradient that enters the backward pass.
+//
+//   z_i  = inv_deg_i * (u_i + sum_{j in N(i)} u_j),   p_i = 1 / (1 + exp(-z_i))
+//   q_i  = sum_{j in N(i)} p_j
+//   loss_s = sum_{i in s} ( alpha/2 * p_i q_i + c_i p_i ),  c_i = -beta + lambda * pen_i
+//   dz_i = (alpha q_i + c_i) p_i (1 - p_i),  t_i = inv_deg_i dz_i
+//   g_i  = t_i + sum_{j in N(i)} t_j            ( = (A_hat^T dz)_i, adjacency symmetric )
+//
+// All three passes are one thread per row; a row longer than 32 entries is instead summed
+// by its whole warp, so a hub cannot stall its warp for thousands of dependent loads.
+#include "internal.cuh"
+
+namespace {
+
+constexpr int kLongRow = 32;
+
+// Sum of val[col] over the CSR row [r0, r1) of each lane's own row.
+__device__ __forceinline__ float row_sum(const float* __restrict__ val, const int32_t* __restrict__ colidx, int32_t r0,
+                                         int32_t r1, bool active) {
+  const int lane = threadIdx.x & 31;
+  const bool is_long = active && (r1 - r0 > kLongRow);
+  float sum = 0.0f;
+  if (active && !is_long)
+    for (int32_t k = r0; k < r1; ++k) sum += __ldg(val + __ldg(colidx + k));
+  uint32_t todo = __ballot_sync(0xffffffffu, is_long);
+  while (todo) {
+    const int src = __ffs(todo) - 1;
+    todo &= todo - 1;
+    const int32_t a = __shfl_sync(0xffffffffu, r0, src), b = __shfl_sync(0xffffffffu, r1, src);
+    float part = 0.0f;
+    for (int32_t k = a + lane; k < b; k += 32) part += __ldg(val + __ldg(colidx + k));
+#pragma unroll
+    for (int d = 16; d > 0; d >>= 1) part += __shfl_xor_sync(0xffffffffu, part, d);
+    if (lane == src) sum = part;
+  }
+  return sum;
+}
+
+__global__ void __launch_bounds__(256) output_forward(const float* __restrict__ u, const int32_t* __restrict__ rowptr,
+                                                      const int32_t* __restrict__ colidx,
+                                                      const float* __restrict__ inv_deg, float* __restrict__ z_out,
+                                                      float* __restrict__ p_out, int64_t n) {
+  const int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+  const bool active = i < n;
+  int32_t r0 = 0, r1 = 0;
+  if (active) { r0 = rowptr[i]; r1 = rowptr[i + 1]; }
+  float s = row_sum(u, colidx, r0, r1, active);
+  if (!active) return;
+  const float z = inv_deg[i] * (u[i] + s);
+  if (z_out) z_out[i] = z;
+  p_out[i] = 1.0f / (1.0f + expf(-z));
+}
+
+// One block per work item (at most kItemRows consecutive rows of one subgraph).
+__global__ void __launch_bounds__(256) objective_items(const float* __restrict__ p, const float* __restrict__ pen,
+                                                       const int32_t* __restrict__ rowptr,
+                                                       const int32_t* __restrict__ colidx,
+                                                       const float* __restrict__ inv_deg,
+                                                       const int32_t* __restrict__ item_row0,
+                                                       const int32_t* __restrict__ item_row1, float alpha, float beta,
+                                                       float lambda, float* __restrict__ item_loss,
+                                                       float* __restrict__ t_out) {
+  __shared__ float warp_part[8];
+  const int32_t a = item_row0[blockIdx.x], b = item_row1[blockIdx.x];
+  float local = 0.0f;
+  for (int32_t base = a; base < b; base += 256) {      // uniform trip count across the block
+    const int32_t i = base + threadIdx.x;
+    const bool active = i < b;
+    int32_t r0 = 0, r1 = 0;
+    if (active) { r0 = rowptr[i]; r1 = rowptr[i + 1]; }
+    const float q = row_sum(p, colidx, r0, r1, active);
+    if (active) {
+      const float pi = p[i];
+      const float c = -beta + (pen ? lambda * pen[i] : 0.0f);
+      local += 0.5f * alpha * pi * q + c * pi;
+      if (t_out) t_out[i] = inv_deg[i] * ((alpha * q + c) * pi * (1.0f - pi));
+    }
+  }
+  // fixed-shape tree: lanes, then warps in order
+#pragma unroll
+  for (int d = 16; d > 0; d >>= 1) local += __shfl_xor_sync(0xffffffffu, local, d);
+  if ((threadIdx.x & 31) == 0) warp_part[threadIdx.x >> 5] = local;
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    float tot = 0.0f;
+#pragma unroll
+    for (int w = 0; w < 8; ++w) tot += warp_part[w];
+    item_loss[blockIdx.x] = tot;
+  }
+}
+
+__global__ void sum_items_per_subgraph(const float* __restrict__ item_loss, const int32_t* __restrict__ part_item_ptr,
+                                       float* __restrict__ loss, int32_t S) {
+  const int32_t s = blockIdx.x * blockDim.x + threadIdx.x;
+  if (s >= S) return;
+  float tot = 0.0f;
+  for (int32_t k = part_item_ptr[s]; k < part_item_ptr[s + 1]; ++k) tot += item_loss[k];
+  loss[s] = tot;
+}
+
+__global__ void __launch_bounds__(256) output_backward(const float* __restrict__ t, const int32_t* __restrict__ rowptr,
+                                                       const int32_t* __restrict__ colidx, float* __restrict__ g,
+                                                       int64_t n) {
+  const int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+  const bool active = i < n;
+  int32_t r0 = 0, r1 = 0;
+  if (active) { r0 = rowptr[i]; r1 = rowptr[i + 1]; }
+  float s = row_sum(t, colidx, r0, r1, active);
+  if (active) g[i] = t[i] + s;
+}
+
+}  // namespace
+
+int32_t launch_output_forward(gnnco_handle* h, const float* u, float* z, float* p, cudaStream_t st) {
+  unsigned grid = (unsigned)((h->n + 255) / 256);
+  output_forward<<<grid, 256, 0, st>>>(u, h->rowptr, h->colidx, h->inv_deg, z, p, h->n);
+  h->launches += 1;
+  GNNCO_LAUNCH_CHECK();
+  return GNNCO_OK;
+}
+
+int32_t launch_objective(gnnco_handle* h, const float* p, const float* pen, float alpha, float beta, float lambda,
+                         float* item_loss, float* loss, float* t, cudaStream_t st) {
+  if (h->n_items > 0)
+    objective_items<<<h->n_items, 256, 0, st>>>(p, pen, h->rowptr, h->colidx, h->inv_deg, h->item_row0, h->item_row1,
+                                                alpha, beta, lambda, item_loss, t);
+  sum_items_per_subgraph<<<(h->S + 255) / 256, 256, 0, st>>>(item_loss, h->part_item_ptr, loss, h->S);
+  h->launches += 2;
+  GNNCO_LAUNCH_CHECK();
+  return GNNCO_OK;
+}
+
+int32_t launch_output_backward(gnnco_handle* h, const float* t, float* g, cudaStream_t st) {
+  unsigned grid = (unsigned)((h->n + 255) / 256);
+  output_backward<<<grid, 256, 0, st>>>(t, h->rowptr, h->colidx, g, h->n);
+  h->launches += 1;
+  GNNCO_LAUNCH_CHECK();
+  return GNNCO_OK;
+}

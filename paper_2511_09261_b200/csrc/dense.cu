@@ -1,0 +1,326 @@
+// Dense per-subgraph weight transform (Eq. 3's "... W"), its two gradients, and the
+// element-wise kernels around it, on the FMA pipes.  Works for every width and both
+// feature types; rows of a tile always belong to one subgraph, so one tile uses one
+// weight set.
+//
+//   transform      Y = act( A W_s ) or A W_s^T, optional per-row scale (folds D^-1 into
+//                  the tensor that feeds the transposed aggregation)
+//   weight_grad    dW_s = A_s^T G_s        (one block per output tile, fixed row order)
+//   gemv / weight_grad_vec / rank1_masked  the same three roles for the last layer,
+//                  whose output width is 1 (Eq. 4)
+//   adam           bias-corrected Adam on the float32 master weights
+#include "internal.cuh"
+
+namespace {
+
+__device__ __forceinline__ float ld(const float* p) { return __ldg(p); }
+__device__ __forceinline__ float ld(const __nv_bfloat16* p) {
+  return __uint_as_float((uint32_t)__ldg(reinterpret_cast<const unsigned short*>(p)) << 16);
+}
+__device__ __forceinline__ void st(float* p, float x) { *p = x; }
+__device__ __forceinline__ void st(__nv_bfloat16* p, float x) { *p = __float2bfloat16_rn(x); }
+
+constexpr int BM = 128, BN = 64, BK = 16;
+
+template <typename TA, typename TW, bool TRANSB>
+__global__ void __launch_bounds__(256) transform_fma(const TA* __restrict__ A, const TW* __restrict__ W,
+                                                     int64_t w_stride, TA* __restrict__ Y, int K, int N, int relu,
+                                                     const float* __restrict__ row_scale,
+                                                     const int32_t* __restrict__ tile_row0,
+                                                     const int32_t* __restrict__ tile_rows,
+                                                     const int32_t* __restrict__ node_part) {
+  __shared__ __align__(16) float As[BK][BM + 4];
+  __shared__ __align__(16) float Bs[BK][BN + 4];
+  const int tid = threadIdx.x, tx = tid & 15, ty = tid >> 4;
+  const int64_t row0 = tile_row0[blockIdx.x];
+  const int rows = tile_rows[blockIdx.x];
+  const int n0 = blockIdx.y * BN;
+  const TW* Ws = W + (int64_t)node_part[row0] * w_stride;
+  float acc[8][4];
+#pragma unroll
+  for (int i = 0; i < 8; ++i)
+#pragma unroll
+    for (int j = 0; j < 4; ++j) acc[i][j] = 0.0f;
+  for (int k0 = 0; k0 < K; k0 += BK) {
+#pragma unroll
+    for (int r = 0; r < (BM * BK) / 256; ++r) {
+      int idx = tid + r * 256;
+      int row = idx / BK, kk = idx % BK;
+      float v = 0.0f;
+      if (row < rows && k0 + kk < K) v = ld(A + (row0 + row) * K + k0 + kk);
+      As[kk][row] = v;
+    }
+#pragma unroll
+    for (int r = 0; r < (BN * BK) / 256; ++r) {
+      int idx = tid + r * 256;
+      float v = 0.0f;
+      if (TRANSB) {
+        int nn = idx / BK, kk = idx % BK;
+        if (n0 + nn < N && k0 + kk < K) v = ld(Ws + (int64_t)(n0 + nn) * K + k0 + kk);
+        Bs[kk][nn] = v;
+      } else {
+        int kk = idx / BN, nn = idx % BN;
+        if (n0 + nn < N && k0 + kk < K) v = ld(Ws + (int64_t)(k0 + kk) * N + n0 + nn);
+        Bs[kk][nn] = v;
+      }
+    }
+    __syncthreads();
+#pragma unroll
+    for (int kk = 0; kk < BK; ++kk) {
+      float a[8], b[4];
+      const float4 a0 = *reinterpret_cast<const float4*>(&As[kk][ty * 8]);
+      const float4 a1 = *reinterpret_cast<const float4*>(&As[kk][ty * 8 + 4]);
+      const float4 b0 = *reinterpret_cast<const float4*>(&Bs[kk][tx * 4]);
+      a[0] = a0.x; a[1] = a0.y; a[2] = a0.z; a[3] = a0.w; a[4] = a1.x; a[5] = a1.y; a[6] = a1.z; a[7] = a1.w;
+      b[0] = b0.x; b[1] = b0.y; b[2] = b0.z; b[3] = b0.w;
+#pragma unroll
+      for (int i = 0; i < 8; ++i)
+#pragma unroll
+        for (int j = 0; j < 4; ++j) acc[i][j] = fmaf(a[i], b[j], acc[i][j]);
+    }
+    __syncthreads();
+  }
+#pragma unroll
+  for (int i = 0; i < 8; ++i) {
+    const int row = ty * 8 + i;
+    if (row >= rows) continue;
+    const float s = row_scale ? row_scale[row0 + row] : 1.0f;
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+      const int col = n0 + tx * 4 + j;
+      if (col >= N) continue;
+      float v = acc[i][j] * s;
+      if (relu) v = v > 0.0f ? v : 0.0f;
+      st(Y + (row0 + row) * N + col, v);
+    }
+  }
+}
+
+// dW[s] tile (64 x 64) = sum over the rows of subgraph s of A[i, k]^T G[i, n]
+template <typename TA>
+__global__ void __launch_bounds__(256) weight_grad_fma(const TA* __restrict__ A, const TA* __restrict__ G,
+                                                       float* __restrict__ dW, int K, int N,
+                                                       const int32_t* __restrict__ part_ptr) {
+  __shared__ __align__(16) float As[16][64 + 4];
+  __shared__ __align__(16) float Gs[16][64 + 4];
+  const int tid = threadIdx.x, tx = tid & 15, ty = tid >> 4;
+  const int s = blockIdx.x, k0 = blockIdx.y * 64, n0 = blockIdx.z * 64;
+  const int64_t ra = part_ptr[s], rb = part_ptr[s + 1];
+  float acc[4][4];
+#pragma unroll
+  for (int i = 0; i < 4; ++i)
+#pragma unroll
+    for (int j = 0; j < 4; ++j) acc[i][j] = 0.0f;
+  for (int64_t r0 = ra; r0 < rb; r0 += 16) {
+#pragma unroll
+    for (int r = 0; r < 4; ++r) {
+      int idx = tid + r * 256;
+      int rr = idx / 64, cc = idx % 64;
+      bool in = r0 + rr < rb;
+      As[rr][cc] = (in && k0 + cc < K) ? ld(A + (r0 + rr) * K + k0 + cc) : 0.0f;
+      Gs[rr][cc] = (in && n0 + cc < N) ? ld(G + (r0 + rr) * N + n0 + cc) : 0.0f;
+    }
+    __syncthreads();
+#pragma unroll
+    for (int rr = 0; rr < 16; ++rr) {
+      const float4 a = *reinterpret_cast<const float4*>(&As[rr][ty * 4]);
+      const float4 g = *reinterpret_cast<const float4*>(&Gs[rr][tx * 4]);
+      const float av[4] = {a.x, a.y, a.z, a.w}, gv[4] = {g.x, g.y, g.z, g.w};
+#pragma unroll
+      for (int i = 0; i < 4; ++i)
+#pragma unroll
+        for (int j = 0; j < 4; ++j) acc[i][j] = fmaf(av[i], gv[j], acc[i][j]);
+    }
+    __syncthreads();
+  }
+  float* out = dW + (int64_t)s * K * N;
+#pragma unroll
+  for (int i = 0; i < 4; ++i)
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+      int k = k0 + ty * 4 + i, n = n0 + tx * 4 + j;
+      if (k < K && n < N) out[(int64_t)k * N + n] = acc[i][j];
+    }
+}
+
+template <typename TA, typename TW>
+__global__ void __launch_bounds__(256) gemv_rows(const TA* __restrict__ H, const TW* __restrict__ w, int64_t w_stride,
+                                                 const int32_t* __restrict__ node_part, float* __restrict__ u,
+                                                 int64_t n, int F) {
+  const int lane = threadIdx.x & 31;
+  const int64_t row = (int64_t)blockIdx.x * 8 + (threadIdx.x >> 5);
+  if (row >= n) return;
+  const TW* ws = w + (int64_t)node_part[row] * w_stride;
+  float acc = 0.0f;
+  for (int f = lane; f < F; f += 32) acc = fmaf(ld(H + row * F + f), ld(ws + f), acc);
+#pragma unroll
+  for (int d = 16; d > 0; d >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, d);
+  if (lane == 0) u[row] = acc;
+}
+
+template <typename TA>
+__global__ void __launch_bounds__(256) weight_grad_vec_kernel(const TA* __restrict__ H, const float* __restrict__ g,
+                                                              float* __restrict__ dw, int F,
+                                                              const int32_t* __restrict__ part_ptr) {
+  const int s = blockIdx.x;
+  const int f = blockIdx.y * 256 + threadIdx.x;
+  if (f >= F) return;
+  const int64_t ra = part_ptr[s], rb = part_ptr[s + 1];
+  float acc = 0.0f;
+  for (int64_t i = ra; i < rb; ++i) acc = fmaf(ld(H + i * F + f), __ldg(g + i), acc);
+  dw[(int64_t)s * F + f] = acc;
+}
+
+template <typename TA, typename TW>
+__global__ void __launch_bounds__(256) rank1_masked_kernel(const float* __restrict__ g, const TW* __restrict__ w,
+                                                           int64_t w_stride, const int32_t* __restrict__ node_part,
+                                                           const TA* __restrict__ H, TA* __restrict__ dZ, int64_t n,
+                                                           int F) {
+  const int64_t t = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+  if (t >= n * F) return;
+  const int64_t i = t / F;
+  const int f = (int)(t - i * F);
+  const float hv = H ? ld(H + t) : 1.0f;
+  const float v = hv > 0.0f ? __ldg(g + i) * ld(w + (int64_t)node_part[i] * w_stride + f) : 0.0f;
+  st(dZ + t, v);
+}
+
+__global__ void sum_over_sets_kernel(const float* __restrict__ in, float* __restrict__ out, int64_t count,
+                                     int32_t sets) {
+  const int64_t q = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+  if (q >= count) return;
+  float acc = 0.0f;
+  for (int32_t s = 0; s < sets; ++s) acc += in[(int64_t)s * count + q];
+  out[q] = acc;
+}
+
+__global__ void cast_bf16_kernel(const float* __restrict__ in, __nv_bfloat16* __restrict__ out, int64_t count) {
+  const int64_t q = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+  if (q < count) out[q] = __float2bfloat16_rn(in[q]);
+}
+
+__global__ void adam_kernel(float* __restrict__ W, float* __restrict__ m, float* __restrict__ v,
+                            const float* __restrict__ g, int64_t count, float lr, float b1, float b2, float eps,
+                            float inv_c1, float inv_c2) {
+  const int64_t q = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+  if (q >= count) return;
+  const float gq = g[q];
+  const float mq = b1 * m[q] + (1.0f - b1) * gq;
+  const float vq = b2 * v[q] + (1.0f - b2) * gq * gq;
+  m[q] = mq;
+  v[q] = vq;
+  W[q] -= lr * (mq * inv_c1) / (sqrtf(vq * inv_c2) + eps);
+}
+
+inline unsigned blocks_for(int64_t work, int threads) { return (unsigned)((work + threads - 1) / threads); }
+
+}  // namespace
+
+int32_t launch_transform(gnnco_handle* h, int dtype, const void* A, const void* W, int64_t w_stride, void* Y, int K,
+                         int N, bool transB, bool relu, const float* row_scale, cudaStream_t stream) {
+  if (h->n_tiles == 0) return GNNCO_OK;
+  dim3 grid(h->n_tiles, (N + BN - 1) / BN);
+  if (grid.y > 65535) return GNNCO_UNSUPPORTED;
+#define GNNCO_TRANSFORM(TA, TW, TB)                                                                            \
+  transform_fma<TA, TW, TB><<<grid, 256, 0, stream>>>((const TA*)A, (const TW*)W, w_stride, (TA*)Y, K, N, relu, \
+                                                      row_scale, h->tile_row0, h->tile_rows, h->node_part)
+  if (dtype == GNNCO_F32) {
+    if (transB) GNNCO_TRANSFORM(float, float, true);
+    else GNNCO_TRANSFORM(float, float, false);
+  } else if (dtype == GNNCO_BF16) {
+    if (transB) GNNCO_TRANSFORM(__nv_bfloat16, __nv_bfloat16, true);
+    else GNNCO_TRANSFORM(__nv_bfloat16, __nv_bfloat16, false);
+  } else {
+    return GNNCO_UNSUPPORTED;
+  }
+#undef GNNCO_TRANSFORM
+  h->launches += 1;
+  GNNCO_LAUNCH_CHECK();
+  return GNNCO_OK;
+}
+
+int32_t launch_gemv(gnnco_handle* h, int dtype, const void* H, const void* w, int64_t w_stride, float* u, int F,
+                    cudaStream_t stream) {
+  unsigned grid = blocks_for(h->n, 8);
+  if (dtype == GNNCO_F32)
+    gemv_rows<float, float><<<grid, 256, 0, stream>>>((const float*)H, (const float*)w, w_stride, h->node_part, u,
+                                                      h->n, F);
+  else if (dtype == GNNCO_BF16)
+    gemv_rows<__nv_bfloat16, __nv_bfloat16><<<grid, 256, 0, stream>>>(
+        (const __nv_bfloat16*)H, (const __nv_bfloat16*)w, w_stride, h->node_part, u, h->n, F);
+  else
+    return GNNCO_UNSUPPORTED;
+  h->launches += 1;
+  GNNCO_LAUNCH_CHECK();
+  return GNNCO_OK;
+}
+
+int32_t launch_weight_grad(gnnco_handle* h, int dtype, const void* A, const void* G, float* dW, int K, int N,
+                           cudaStream_t stream) {
+  dim3 grid(h->S, (K + 63) / 64, (N + 63) / 64);
+  if (grid.y > 65535 || grid.z > 65535) return GNNCO_UNSUPPORTED;
+  if (dtype == GNNCO_F32)
+    weight_grad_fma<float><<<grid, 256, 0, stream>>>((const float*)A, (const float*)G, dW, K, N, h->part_ptr);
+  else if (dtype == GNNCO_BF16)
+    weight_grad_fma<__nv_bfloat16><<<grid, 256, 0, stream>>>((const __nv_bfloat16*)A, (const __nv_bfloat16*)G, dW, K,
+                                                             N, h->part_ptr);
+  else
+    return GNNCO_UNSUPPORTED;
+  h->launches += 1;
+  GNNCO_LAUNCH_CHECK();
+  return GNNCO_OK;
+}
+
+int32_t launch_weight_grad_vec(gnnco_handle* h, int dtype, const void* H, const float* g, float* dw, int F,
+                               cudaStream_t stream) {
+  dim3 grid(h->S, (F + 255) / 256);
+  if (grid.y > 65535) return GNNCO_UNSUPPORTED;
+  if (dtype == GNNCO_F32)
+    weight_grad_vec_kernel<float><<<grid, 256, 0, stream>>>((const float*)H, g, dw, F, h->part_ptr);
+  else if (dtype == GNNCO_BF16)
+    weight_grad_vec_kernel<__nv_bfloat16><<<grid, 256, 0, stream>>>((const __nv_bfloat16*)H, g, dw, F, h->part_ptr);
+  else
+    return GNNCO_UNSUPPORTED;
+  h->launches += 1;
+  GNNCO_LAUNCH_CHECK();
+  return GNNCO_OK;
+}
+
+int32_t launch_rank1_masked(gnnco_handle* h, int dtype, const float* g, const void* w, int64_t w_stride, const void* H,
+                            void* dZ, int F, cudaStream_t stream) {
+  unsigned grid = blocks_for(h->n * F, 256);
+  if (dtype == GNNCO_F32)
+    rank1_masked_kernel<float, float><<<grid, 256, 0, stream>>>(g, (const float*)w, w_stride, h->node_part,
+                                                                (const float*)H, (float*)dZ, h->n, F);
+  else if (dtype == GNNCO_BF16)
+    rank1_masked_kernel<__nv_bfloat16, __nv_bfloat16><<<grid, 256, 0, stream>>>(
+        g, (const __nv_bfloat16*)w, w_stride, h->node_part, (const __nv_bfloat16*)H, (__nv_bfloat16*)dZ, h->n, F);
+  else
+    return GNNCO_UNSUPPORTED;
+  h->launches += 1;
+  GNNCO_LAUNCH_CHECK();
+  return GNNCO_OK;
+}
+
+int32_t launch_sum_over_sets(gnnco_handle* h, const float* in, float* out, int64_t count, int32_t sets,
+                             cudaStream_t stream) {
+  sum_over_sets_kernel<<<blocks_for(count, 256), 256, 0, stream>>>(in, out, count, sets);
+  h->launches += 1;
+  GNNCO_LAUNCH_CHECK();
+  return GNNCO_OK;
+}
+
+int32_t launch_cast_bf16(gnnco_handle* h, const float* in, __nv_bfloat16* out, int64_t count, cudaStream_t stream) {
+  cast_bf16_kernel<<<blocks_for(count, 256), 256, 0, stream>>>(in, out, count);
+  h->launches += 1;
+  GNNCO_LAUNCH_CHECK();
+  return GNNCO_OK;
+}
+
+int32_t launch_adam(gnnco_handle* h, float* W, float* m, float* v, const float* g, int64_t count, float lr, float b1,
+                    float b2, float eps, float c1, float c2, cudaStream_t stream) {
+  adam_kernel<<<blocks_for(count, 256), 256, 0, stream>>>(W, m, v, g, count, lr, b1, b2, eps, 1.0f / c1, 1.0f / c2);
+  h->launches += 1;
+  GNNCO_LAUNCH_CHECK();
+  return GNNCO_OK;
+}

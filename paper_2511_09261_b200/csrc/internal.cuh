@@ -1,0 +1,98 @@
+// Internal declarations shared by the translation units of libgnnco.
+#pragma once
+
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include <vector>
+
+#include "gnnco.h"
+
+#define GNNCO_CUDA_TRY(expr)                      \
+  do {                                            \
+    cudaError_t e__ = (expr);                     \
+    if (e__ != cudaSuccess) return GNNCO_CUDA_ERROR; \
+  } while (0)
+
+#define GNNCO_LAUNCH_CHECK()                                   \
+  do {                                                         \
+    if (cudaPeekAtLastError() != cudaSuccess) { cudaGetLastError(); return GNNCO_CUDA_ERROR; } \
+  } while (0)
+
+constexpr int kGemmTileRows = 128;   // rows of one dense-transform tile (never straddles a subgraph)
+constexpr int kItemRows = 1024;      // rows of one objective work item (never straddles a subgraph)
+
+struct gnnco_handle {
+  int64_t n = 0, E = 0, E_in = 0, E_b = 0;
+  int32_t S = 0, max_row = 0;
+  int device = 0;
+  // device arrays inside the caller's persistent work area
+  int32_t *perm = nullptr, *inv_perm = nullptr, *part_ptr = nullptr, *node_part = nullptr;
+  int32_t *rowptr = nullptr, *colidx = nullptr, *bnd_u = nullptr, *bnd_v = nullptr;
+  float* inv_deg = nullptr;
+  uint8_t* is_boundary = nullptr;
+  int32_t *tile_row0 = nullptr, *tile_rows = nullptr;      // dense-transform tiles
+  int32_t *item_row0 = nullptr, *item_row1 = nullptr;      // objective work items
+  int32_t* part_item_ptr = nullptr;                        // [S+1] items of each subgraph
+  int32_t* status = nullptr;                               // device status word + counters
+  int32_t n_tiles = 0, n_items = 0;
+  std::vector<int32_t> h_part_ptr;
+  int64_t launches = 0;
+};
+
+static inline size_t align_up(size_t x, size_t a = 256) { return (x + a - 1) / a * a; }
+
+// A bump allocator over a caller-provided work area.
+struct Carver {
+  char* base;
+  size_t off = 0, cap;
+  Carver(void* p, size_t bytes) : base(static_cast<char*>(p)), cap(bytes) {}
+  template <typename T>
+  T* take(size_t count) {
+    size_t bytes = align_up(count * sizeof(T));
+    T* r = reinterpret_cast<T*>(base + off);
+    off += bytes;
+    return r;
+  }
+  bool ok() const { return off <= cap; }
+};
+
+// ---- partition.cu
+int32_t partition_scratch_bytes(int64_t n, int64_t E, int32_t S, size_t* bytes);
+
+// ---- spmm.cu : out[i] = scale[i] * (in[i] + sum_{j in row i} in[j]), optionally zeroed where mask[i,f] <= 0
+int32_t launch_aggregate(gnnco_handle* h, int dtype, const void* in, void* out, int F, const float* row_scale,
+                         const void* relu_mask, cudaStream_t st);
+
+// ---- dense.cu
+// Y[tile rows x N] = act( A[rows x K] * B_s ), B_s = W[s] (K x N) or, with transB, W[s]^T where W[s] is (N x K).
+int32_t launch_transform(gnnco_handle* h, int dtype, const void* A, const void* W, int64_t w_stride, void* Y, int K,
+                         int N, bool transB, bool relu, const float* row_scale, cudaStream_t st);
+// u[i] = H[i,:] . w_s
+int32_t launch_gemv(gnnco_handle* h, int dtype, const void* H, const void* w, int64_t w_stride, float* u, int F,
+                    cudaStream_t st);
+// dW[s] (K x N) = sum_{i in s} A[i,:]^T G[i,:]
+int32_t launch_weight_grad(gnnco_handle* h, int dtype, const void* A, const void* G, float* dW, int K, int N,
+                           cudaStream_t st);
+// dw[s][f] = sum_{i in s} H[i,f] g[i]
+int32_t launch_weight_grad_vec(gnnco_handle* h, int dtype, const void* H, const float* g, float* dw, int F,
+                               cudaStream_t st);
+// dZ[i,f] = g[i] * w_s[f] where H[i,f] > 0, else 0 (H == nullptr: no mask)
+int32_t launch_rank1_masked(gnnco_handle* h, int dtype, const float* g, const void* w, int64_t w_stride, const void* H,
+                            void* dZ, int F, cudaStream_t st);
+// out[q] = sum_s in[s][q]
+int32_t launch_sum_over_sets(gnnco_handle* h, const float* in, float* out, int64_t count, int32_t sets, cudaStream_t st);
+int32_t launch_cast_bf16(gnnco_handle* h, const float* in, __nv_bfloat16* out, int64_t count, cudaStream_t st);
+int32_t launch_adam(gnnco_handle* h, float* W, float* m, float* v, const float* g, int64_t count, float lr, float b1,
+                    float b2, float eps, float c1, float c2, cudaStream_t st);
+
+// ---- chain.cu : the width-1 part of the step
+int32_t launch_output_forward(gnnco_handle* h, const float* u, float* z, float* p, cudaStream_t st);
+int32_t launch_objective(gnnco_handle* h, const float* p, const float* pen, float alpha, float beta, float lambda,
+                         float* item_loss, float* loss, float* t, cudaStream_t st);
+int32_t launch_output_backward(gnnco_handle* h, const float* t, float* g, cudaStream_t st);
+
+// ---- decode.cu
+int32_t launch_decode(gnnco_handle* h, const float* p, float thr, uint8_t* x, uint8_t* viol, int32_t* per_part,
+                      gnnco_counts* counts, cudaStream_t st);

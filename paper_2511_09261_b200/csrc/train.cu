@@ -1,0 +1,265 @@
+// gnnco_train_step: host-side plan of one full-batch training step over the
+// block-diagonal batch (Section 3.2, Eqs. 3-5; Algorithm 1, Stage 1).  Only kernel
+// launches happen here; every arithmetic step runs on the device.
+//
+// Forward, hidden layer l (1-based, widths d_{l-1} -> d_l):
+//     M_l = A_hat H_{l-1}            aggregate   (spmm.cu)
+//     H_l = ReLU(M_l W_l)            transform   (dense.cu)
+// Output layer:  u = H_{L-1} w_L ;  z = A_hat u ;  p = sigmoid(z)      (chain.cu)
+// Objective:     q = A p, per-subgraph loss, t = D^-1 dz ;  g = (A+I) t = A_hat^T dz
+// Backward:      dw_L = H_{L-1}^T g ;  dZ_{L-1} = (g w_L^T) * [H_{L-1} > 0]
+//     for l = L-1 .. 1:  dM_l = D^-1 (dZ_l W_l^T) ;  dW_l = M_l^T dZ_l ;  Adam on W_l
+//                        dZ_{l-1} = ((A+I) dM_l) * [H_{l-1} > 0]      (dX when l = 1)
+// The transposed aggregation reuses the forward CSR because the intra adjacency is
+// symmetric: A_hat^T G = (A+I)(D^-1 G).
+#include <math.h>
+
+#include "internal.cuh"
+
+namespace {
+
+struct TrainLayout {
+  void* M[GNNCO_MAX_LAYERS];          // M[l], l = 1..L-1: aggregated input of hidden layer l
+  void* H[GNNCO_MAX_LAYERS];          // H[l], l = 1..L-1: activation of hidden layer l
+  void* Ga;                           // gradient ping-pong buffers, n x max width
+  void* Gb;
+  float *u, *t, *g, *item_loss;
+  float* dW_scratch;                  // one layer's gradient (all sets), when the caller wants none
+  float* dW_sets;                     // per-subgraph partials when the model shares one weight set
+  __nv_bfloat16* W_lp[GNNCO_MAX_LAYERS];   // bf16 copies of the weights (bf16 features only)
+  // host-variant staging
+  void* X_stage;
+  float *pen_stage, *loss_stage, *p_stage;
+  size_t bytes;
+};
+
+size_t elem_size(int dtype) { return dtype == GNNCO_BF16 ? 2 : 4; }
+
+int32_t check_model(const gnnco_handle* h, const gnnco_model_desc* m, bool need_ptrs) {
+  if (!h || !m) return GNNCO_INVALID_ARGUMENT;
+  if (m->L < 1 || m->L > GNNCO_MAX_LAYERS) return GNNCO_INVALID_ARGUMENT;
+  if (m->feat_dtype != GNNCO_F32 && m->feat_dtype != GNNCO_BF16) return GNNCO_UNSUPPORTED;
+  if (m->weight_sets != 1 && m->weight_sets != h->S) return GNNCO_INVALID_ARGUMENT;
+  for (int l = 0; l <= m->L; ++l)
+    if (m->dims[l] < 1 || m->dims[l] > 65536) return GNNCO_INVALID_ARGUMENT;
+  if (m->dims[m->L] != 1) return GNNCO_INVALID_ARGUMENT;
+  if (m->feat_dtype == GNNCO_BF16)
+    for (int l = 0; l < m->L; ++l)
+      if (m->dims[l] % 2) return GNNCO_UNSUPPORTED;     // bf16 rows must stay 4-byte aligned
+  if (need_ptrs)
+    for (int l = 0; l < m->L; ++l)
+      if (!m->W[l]) return GNNCO_INVALID_ARGUMENT;
+  return GNNCO_OK;
+}
+
+TrainLayout carve_train(const gnnco_handle* h, const gnnco_model_desc* m, uint32_t flags, void* base, bool host) {
+  TrainLayout T{};
+  Carver c(base, ~(size_t)0);
+  const size_t es = elem_size(m->feat_dtype);
+  const size_t n = (size_t)h->n;
+  const int L = m->L;
+  int maxw = 1;
+  size_t max_wcount = 0;
+  for (int l = 0; l < L; ++l) {
+    if (m->dims[l] > maxw) maxw = m->dims[l];
+    size_t wc = (size_t)m->dims[l] * m->dims[l + 1];
+    if (wc > max_wcount) max_wcount = wc;
+  }
+  for (int l = 1; l < L; ++l) {
+    T.M[l] = c.take<char>(n * m->dims[l - 1] * es);
+    T.H[l] = c.take<char>(n * m->dims[l] * es);
+  }
+  T.u = c.take<float>(n);
+  T.t = c.take<float>(n);
+  T.g = c.take<float>(n);
+  T.item_loss = c.take<float>((size_t)h->n_items + 1);
+  if (!(flags & GNNCO_FORWARD_ONLY)) {
+    T.Ga = c.take<char>(n * maxw * es);
+    T.Gb = c.take<char>(n * maxw * es);
+    T.dW_scratch = c.take<float>(max_wcount * m->weight_sets);
+    if (m->weight_sets == 1) T.dW_sets = c.take<float>(max_wcount * (size_t)h->S);
+  }
+  if (m->feat_dtype == GNNCO_BF16)
+    for (int l = 0; l < L; ++l)
+      T.W_lp[l] = c.take<__nv_bfloat16>((size_t)m->dims[l] * m->dims[l + 1] * m->weight_sets);
+  if (host) {
+    T.X_stage = c.take<char>(n * m->dims[0] * es);
+    T.pen_stage = c.take<float>(n);
+    T.loss_stage = c.take<float>((size_t)h->S);
+    T.p_stage = c.take<float>(n);
+  }
+  T.bytes = c.off;
+  return T;
+}
+
+int32_t run_step(gnnco_handle* h, const gnnco_model_desc* m, const void* X, const gnnco_objective* obj,
+                 gnnco_adam_state* opt, const gnnco_train_out* out, uint32_t flags, const TrainLayout& T,
+                 cudaStream_t st) {
+  const int L = m->L, dt = m->feat_dtype;
+  const bool bf16 = dt == GNNCO_BF16;
+  const int32_t sets = m->weight_sets;
+  int32_t rc;
+#define GNNCO_TRY(call) do { rc = (call); if (rc != GNNCO_OK) return rc; } while (0)
+  // weights as the matrix products see them
+  const void* Wc[GNNCO_MAX_LAYERS];
+  int64_t wstride[GNNCO_MAX_LAYERS];
+  for (int l = 0; l < L; ++l) {
+    const int64_t wc = (int64_t)m->dims[l] * m->dims[l + 1];
+    wstride[l] = sets == 1 ? 0 : wc;
+    if (bf16) {
+      GNNCO_TRY(launch_cast_bf16(h, m->W[l], T.W_lp[l], wc * sets, st));
+      Wc[l] = T.W_lp[l];
+    } else {
+      Wc[l] = m->W[l];
+    }
+  }
+  // ---- forward
+  const void* Hprev = X;
+  for (int l = 1; l < L; ++l) {
+    GNNCO_TRY(launch_aggregate(h, dt, Hprev, T.M[l], m->dims[l - 1], h->inv_deg, nullptr, st));
+    GNNCO_TRY(launch_transform(h, dt, T.M[l], Wc[l - 1], wstride[l - 1], T.H[l], m->dims[l - 1], m->dims[l], false,
+                               true, nullptr, st));
+    Hprev = T.H[l];
+  }
+  const int FL = m->dims[L - 1];
+  GNNCO_TRY(launch_gemv(h, dt, Hprev, Wc[L - 1], wstride[L - 1], T.u, FL, st));
+  GNNCO_TRY(launch_output_forward(h, T.u, out->z, out->p, st));
+  const bool fwd_only = (flags & GNNCO_FORWARD_ONLY) != 0;
+  GNNCO_TRY(launch_objective(h, out->p, obj->pen, obj->alpha, obj->beta, obj->lambda, T.item_loss, out->loss,
+                             fwd_only ? nullptr : T.t, st));
+  if (fwd_only) return GNNCO_OK;
+  // ---- backward
+  GNNCO_TRY(launch_output_backward(h, T.t, T.g, st));
+  float c1 = 1.0f, c2 = 1.0f;
+  if (opt) {
+    c1 = (float)(1.0 - pow((double)opt->beta1, (double)opt->step));
+    c2 = (float)(1.0 - pow((double)opt->beta2, (double)opt->step));
+  }
+  auto finish_layer = [&](int l, float* grad_sets_or_final) -> int32_t {
+    // grad_sets_or_final holds [sets x ...] already reduced; run Adam on layer l (0-based)
+    const int64_t wc = (int64_t)m->dims[l] * m->dims[l + 1] * sets;
+    if (opt) return launch_adam(h, m->W[l], opt->m[l], opt->v[l], grad_sets_or_final, wc, opt->lr, opt->beta1,
+                                opt->beta2, opt->eps, c1, c2, st);
+    return GNNCO_OK;
+  };
+  // gradient target of layer l: the caller's buffer or the scratch
+  auto grad_target = [&](int l) -> float* { return out->dW[l] ? out->dW[l] : T.dW_scratch; };
+  {
+    // last layer (0-based index L-1): dw = H^T g
+    float* target = grad_target(L - 1);
+    if (sets == 1) {
+      GNNCO_TRY(launch_weight_grad_vec(h, dt, Hprev, T.g, T.dW_sets, FL, st));
+      GNNCO_TRY(launch_sum_over_sets(h, T.dW_sets, target, FL, h->S, st));
+    } else {
+      GNNCO_TRY(launch_weight_grad_vec(h, dt, Hprev, T.g, target, FL, st));
+    }
+    if (L > 1) GNNCO_TRY(launch_rank1_masked(h, dt, T.g, Wc[L - 1], wstride[L - 1], Hprev, T.Ga, FL, st));
+    else if (flags & GNNCO_WANT_DX)
+      // L == 1: dX = A_hat^T (dz w_s^T) and w_s is constant inside a subgraph, so dX[i,:] = g_i w_s^T
+      GNNCO_TRY(launch_rank1_masked(h, dt, T.g, Wc[0], wstride[0], nullptr, out->dX, FL, st));
+    GNNCO_TRY(finish_layer(L - 1, target));
+  }
+  void* dZ = T.Ga;
+  void* other = T.Gb;
+  for (int l = L - 1; l >= 1; --l) {
+    // hidden layer l uses weight index l-1: widths d_{l-1} -> d_l
+    const int K = m->dims[l - 1], N = m->dims[l];
+    const bool need_input_grad = (l > 1) || (flags & GNNCO_WANT_DX);
+    if (need_input_grad)
+      GNNCO_TRY(launch_transform(h, dt, dZ, Wc[l - 1], wstride[l - 1], other, N, K, true, false, h->inv_deg, st));
+    float* target = grad_target(l - 1);
+    if (sets == 1) {
+      GNNCO_TRY(launch_weight_grad(h, dt, T.M[l], dZ, T.dW_sets, K, N, st));
+      GNNCO_TRY(launch_sum_over_sets(h, T.dW_sets, target, (int64_t)K * N, h->S, st));
+    } else {
+      GNNCO_TRY(launch_weight_grad(h, dt, T.M[l], dZ, target, K, N, st));
+    }
+    GNNCO_TRY(finish_layer(l - 1, target));
+    if (need_input_grad) {
+      if (l > 1) {
+        GNNCO_TRY(launch_aggregate(h, dt, other, dZ, K, nullptr, T.H[l - 1], st));   // new dZ in the old buffer
+      } else {
+        GNNCO_TRY(launch_aggregate(h, dt, other, out->dX, K, nullptr, nullptr, st));
+      }
+    }
+  }
+#undef GNNCO_TRY
+  return GNNCO_OK;
+}
+
+int32_t check_step_args(const gnnco_handle* h, const gnnco_model_desc* m, const gnnco_adam_state* opt,
+                        uint32_t flags) {
+  int32_t rc = check_model(h, m, true);
+  if (rc != GNNCO_OK) return rc;
+  if (flags & ~(GNNCO_WANT_DX | GNNCO_FORWARD_ONLY)) return GNNCO_INVALID_ARGUMENT;
+  if (opt && !(flags & GNNCO_FORWARD_ONLY)) {
+    if (opt->step < 1) return GNNCO_INVALID_ARGUMENT;
+    for (int l = 0; l < m->L; ++l)
+      if (!opt->m[l] || !opt->v[l]) return GNNCO_INVALID_ARGUMENT;
+  }
+  return GNNCO_OK;
+}
+
+}  // namespace
+
+extern "C" int32_t gnnco_train_workspace_bytes(const gnnco_handle* h, const gnnco_model_desc* m, uint32_t flags,
+                                              size_t* bytes) {
+  if (!bytes) return GNNCO_INVALID_ARGUMENT;
+  int32_t rc = check_model(h, m, false);
+  if (rc != GNNCO_OK) return rc;
+  *bytes = carve_train(h, m, flags, nullptr, false).bytes;
+  return GNNCO_OK;
+}
+
+extern "C" int32_t gnnco_train_host_workspace_bytes(const gnnco_handle* h, const gnnco_model_desc* m, uint32_t flags,
+                                                   size_t* bytes) {
+  if (!bytes) return GNNCO_INVALID_ARGUMENT;
+  int32_t rc = check_model(h, m, false);
+  if (rc != GNNCO_OK) return rc;
+  *bytes = carve_train(h, m, flags, nullptr, true).bytes;
+  return GNNCO_OK;
+}
+
+extern "C" int32_t gnnco_train_step(gnnco_handle* h, const gnnco_model_desc* m, const void* X,
+                                   const gnnco_objective* obj, gnnco_adam_state* opt, const gnnco_train_out* out,
+                                   uint32_t flags, void* ws, size_t ws_bytes, void* stream) {
+  if (!h || !m || !X || !obj || !out || !ws || !out->loss || !out->p) return GNNCO_INVALID_ARGUMENT;
+  int32_t rc = check_step_args(h, m, opt, flags);
+  if (rc != GNNCO_OK) return rc;
+  if ((flags & GNNCO_WANT_DX) && !out->dX) return GNNCO_INVALID_ARGUMENT;
+  if ((uintptr_t)ws & 255) return GNNCO_INVALID_ARGUMENT;
+  TrainLayout T = carve_train(h, m, flags, ws, false);
+  if (T.bytes > ws_bytes) return GNNCO_WORKSPACE_TOO_SMALL;
+  return run_step(h, m, X, obj, opt, out, flags, T, static_cast<cudaStream_t>(stream));
+}
+
+extern "C" int32_t gnnco_train_step_host(gnnco_handle* h, const gnnco_model_desc* m, const void* X_host, float alpha,
+                                        float beta, float lambda, const float* pen_host, gnnco_adam_state* opt,
+                                        float* loss_host, float* p_host, uint32_t flags, void* ws, size_t ws_bytes,
+                                        void* stream) {
+  if (!h || !m || !X_host || !loss_host || !p_host || !ws) return GNNCO_INVALID_ARGUMENT;
+  int32_t rc = check_step_args(h, m, opt, flags);
+  if (rc != GNNCO_OK) return rc;
+  if (flags & GNNCO_WANT_DX) return GNNCO_UNSUPPORTED;       // the host variant returns loss and p only
+  if ((uintptr_t)ws & 255) return GNNCO_INVALID_ARGUMENT;
+  TrainLayout T = carve_train(h, m, flags, ws, true);
+  if (T.bytes > ws_bytes) return GNNCO_WORKSPACE_TOO_SMALL;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  const size_t n = (size_t)h->n;
+  GNNCO_CUDA_TRY(cudaMemcpyAsync(T.X_stage, X_host, n * m->dims[0] * elem_size(m->feat_dtype),
+                                 cudaMemcpyHostToDevice, st));
+  gnnco_objective obj{alpha, beta, lambda, nullptr};
+  if (pen_host) {
+    GNNCO_CUDA_TRY(cudaMemcpyAsync(T.pen_stage, pen_host, n * sizeof(float), cudaMemcpyHostToDevice, st));
+    obj.pen = T.pen_stage;
+  }
+  gnnco_train_out out{};
+  out.loss = T.loss_stage;
+  out.p = T.p_stage;
+  rc = run_step(h, m, T.X_stage, &obj, opt, &out, flags, T, st);
+  if (rc != GNNCO_OK) return rc;
+  GNNCO_CUDA_TRY(cudaMemcpyAsync(loss_host, T.loss_stage, (size_t)h->S * sizeof(float), cudaMemcpyDeviceToHost, st));
+  GNNCO_CUDA_TRY(cudaMemcpyAsync(p_host, T.p_stage, n * sizeof(float), cudaMemcpyDeviceToHost, st));
+  GNNCO_CUDA_TRY(cudaStreamSynchronize(st));
+  return GNNCO_OK;
+}

@@ -1,0 +1,200 @@
+"""Helpers of the GPU parity tests: run the CUDA library through its binding and the
+oracle on the same seeded inputs, and compare element by element."""
+import numpy as np
+
+import oracle
+import synth_inputs as si
+
+# Tolerances (the ones the acceptance criteria state): float32 features rtol 1e-4 /
+# atol 1e-5; bfloat16 features rtol 2e-2, with an absolute floor of 1e-2 of the reference
+# tensor's RMS (stored bf16 values carry 2^-9 relative rounding error each, and an output
+# that is a cancelling sum of such values inherits an error proportional to the typical
+# magnitude of the tensor, not to the entry itself).
+F32_RTOL, F32_ATOL = 1e-4, 1e-5
+BF16_RTOL, BF16_ATOL_RMS = 2e-2, 1e-2
+
+
+def tolerances(dtype, ref):
+    if dtype == "bf16":
+        rms = float(np.sqrt(np.mean(np.square(ref)))) if ref.size else 0.0
+        return BF16_RTOL, BF16_ATOL_RMS * rms + 1e-6
+    return F32_RTOL, F32_ATOL
+
+
+def assert_close(got, ref, dtype, what, skip_mask=None):
+    got = np.asarray(got, dtype=np.float64)
+    ref = np.asarray(ref, dtype=np.float64)
+    assert got.shape == ref.shape, (what, got.shape, ref.shape)
+    rtol, atol = tolerances(dtype, ref)
+    err = np.abs(got - ref)
+    bad = err > atol + rtol * np.abs(ref)
+    if skip_mask is not None:
+        bad &= ~skip_mask
+    if bad.any():
+        k = np.unravel_index(np.argmax(np.where(bad, err, 0)), err.shape)
+        raise AssertionError("%s: %d of %d entries outside rtol=%g atol=%g; worst at %s: got %r, expected %r"
+                             % (what, int(bad.sum()), bad.size, rtol, atol, k, got[k], ref[k]))
+    return float(err.max()) if err.size else 0.0
+
+
+def torch_dev():
+    import torch
+    return torch.device("cuda:0")
+
+
+def to_dev(a, dtype=None):
+    import torch
+    t = torch.from_numpy(np.ascontiguousarray(a)).to(torch_dev())
+    return t if dtype is None else t.to(dtype)
+
+
+def load_graph(n, eu, ev, part, S):
+    import paper_2511_09261_b200 as gnnco
+    return gnnco.gnnco_partition_load(to_dev(eu.astype(np.int32)), to_dev(ev.astype(np.int32)),
+                                      to_dev(part.astype(np.int32)), S)
+
+
+def check_bookkeeping(graph, book):
+    """Bit-exact comparison of every array gnnco_partition_load builds."""
+    assert (graph.n, graph.S, graph.E_in, graph.E_b) == (book["n"], book["S"], book["E_in"], book["E_b"])
+    arr = graph.arrays()
+    for key in ("perm", "inv_perm", "part_ptr", "node_part", "rowptr", "colidx", "bnd_u", "bnd_v", "is_boundary"):
+        got = arr[key].cpu().numpy()
+        assert np.array_equal(got, book[key]), key
+    got = arr["inv_deg"].cpu().numpy()
+    assert np.array_equal(got.view(np.uint32), book["inv_deg"].view(np.uint32)), "inv_deg"
+    deg = np.diff(book["rowptr"])
+    assert graph.max_row == (int(deg.max()) if deg.size else 0)
+
+
+class StepCase:
+    """One teacher-forced step: same X, W, (m, v) on both sides; compares loss, p, z,
+    every dW, dX and the Adam-updated weights."""
+
+    def __init__(self, book, dims, dtype="f32", sets=None, alpha=2.0, beta=1.0, lam=0.0):
+        self.book, self.dims, self.dtype = book, list(dims), dtype
+        self.L = len(dims) - 1
+        self.S, self.n = int(book["S"]), int(book["n"])
+        self.sets = self.S if sets is None else sets
+        self.alpha, self.beta, self.lam = alpha, beta, lam
+
+    def run(self, graph, X_new, W, pen_new=None, want_dx=True, adam=None, threads=4, parts=None, label=""):
+        """X_new [n,F0] float32 numpy (bf16-representable when dtype is bf16), W list of
+        float32 numpy [sets,Fi,Fo]; adam = dict(m=[...], v=[...], step=t, lr=...) or None.
+        parts: compare only these subgraphs (the oracle then runs only them)."""
+        import torch
+        import paper_2511_09261_b200 as gnnco
+        bf16 = self.dtype == "bf16"
+        fd = gnnco.BF16 if bf16 else gnnco.F32
+        Xd = to_dev(X_new, torch.bfloat16 if bf16 else torch.float32)
+        Wd = [to_dev(w) for w in W]
+        model = gnnco.Model(self.dims, Wd, fd)
+        opt = None
+        if adam is not None:
+            opt = gnnco.Adam(model, lr=adam["lr"])
+            opt.step = adam["step"]
+            opt.m = [to_dev(m) for m in adam["m"]]
+            opt.v = [to_dev(v) for v in adam["v"]]
+        dW = [torch.full_like(w, float("nan")) for w in Wd]
+        z = torch.full((self.n,), float("nan"), device=Xd.device)
+        dX = torch.full_like(Xd, float("nan")) if want_dx else None
+        pen_d = to_dev(pen_new.astype(np.float32)) if pen_new is not None else None
+        flags = gnnco.WANT_DX if want_dx else 0
+        loss, p = graph.train_step(model, Xd, self.alpha, self.beta, self.lam, pen_d, opt, z=z, dW=dW, dX=dX,
+                                   flags=flags)
+        torch.cuda.synchronize()
+        assert graph.async_status() == 0
+        g = dict(loss=loss.cpu().numpy(), p=p.cpu().numpy(), z=z.cpu().numpy(),
+                 dW=[t.cpu().numpy() for t in dW], dX=None if dX is None else dX.float().cpu().numpy(),
+                 W=[t.cpu().numpy() for t in Wd])
+        if opt is not None:
+            g["m"] = [t.cpu().numpy() for t in opt.m]
+            g["v"] = [t.cpu().numpy() for t in opt.v]
+        # ---- oracle (weights as the matrix products see them: bf16-rounded for bf16 runs)
+        Wc = [si.round_to_bf16(w) if bf16 else w for w in W]
+        stats = {}
+        if parts is None:
+            r = oracle.train_step(self.book, self.dims, X_new, Wc, self.alpha, self.beta, self.lam, pen_new,
+                                  want_dX=want_dx, want_Z=True, threads=threads, store_bf16=bf16)
+            self._compare(g, r, slice(None), None, W, adam, stats, label)
+        else:
+            for s in parts:
+                lo, hi = int(self.book["part_ptr"][s]), int(self.book["part_ptr"][s + 1])
+                if hi == lo:
+                    continue
+                rp = self.book["rowptr"][lo:hi + 1] - self.book["rowptr"][lo]
+                ci = self.book["colidx"][self.book["rowptr"][lo]:self.book["rowptr"][hi]] - lo
+                ws = [w[s if self.sets > 1 else 0] for w in Wc]
+                one = oracle.subgraph_step(rp, ci, self.dims, X_new[lo:hi], ws, self.alpha, self.beta, self.lam,
+                                           None if pen_new is None else pen_new[lo:hi], want_dX=want_dx,
+                                           want_Z=True, store_bf16=bf16)
+                r = dict(loss=np.array([one["loss"]]), p=one["p"], z=one["z"], dX=one["dX"],
+                         dW=[d[None] for d in one["dW"]], Z=one["Z"])
+                self._compare(g, r, slice(lo, hi), s, W, adam, stats, "%s part %d" % (label, s))
+        return g, stats
+
+    def _compare(self, g, r, rows, s, W, adam, stats, label):
+        dt = self.dtype
+        sel = slice(None) if s is None else slice(s, s + 1)
+        stats["loss"] = max(stats.get("loss", 0), assert_close(g["loss"][sel], r["loss"], dt, label + " loss"))
+        stats["p"] = max(stats.get("p", 0), assert_close(g["p"][rows], r["p"], "f32" if dt == "f32" else dt, label + " p"))
+        stats["z"] = max(stats.get("z", 0), assert_close(g["z"][rows], r["z"], dt, label + " z"))
+        # pre-activations that sit on a ReLU kink decide a 0/1 mask; a subgraph (and hidden
+        # unit) holding one is excluded from the gradient comparison and counted
+        kink_parts = set()
+        if r["Z"]:
+            thr = 1e-6
+            for Z in r["Z"]:
+                near = np.abs(Z) < thr * (1.0 + np.abs(Z))
+                if near.any():
+                    base = 0 if s is None else rows.start
+                    node_rows = np.where(near.any(axis=1))[0] + base
+                    kink_parts.update(self.book["node_part"][node_rows].tolist())
+        stats["kink_parts"] = stats.get("kink_parts", 0) + len(kink_parts)
+        assert len(kink_parts) <= max(1, self.S // 50), "too many subgraphs sit on a ReLU kink"
+        shared = self.sets == 1
+        if shared and s is not None:
+            return
+        if shared and kink_parts:
+            return
+        for l in range(self.L):
+            gd = g["dW"][l][sel] if not shared else g["dW"][l]
+            rd = r["dW"][l]
+            skip = None
+            if kink_parts and not shared:
+                skip = np.zeros(rd.shape, bool)
+                for kp in kink_parts:
+                    skip[kp if s is None else 0] = True
+            stats["dW%d" % l] = max(stats.get("dW%d" % l, 0), assert_close(gd, rd, dt, label + " dW[%d]" % l, skip))
+        if r["dX"] is not None and g["dX"] is not None:
+            skip = None
+            if kink_parts:
+                skip = np.zeros(r["dX"].shape, bool)
+                base = 0 if s is None else rows.start
+                for kp in kink_parts:
+                    lo, hi = int(self.book["part_ptr"][kp]) - base, int(self.book["part_ptr"][kp + 1]) - base
+                    skip[max(lo, 0):max(hi, 0)] = True
+            stats["dX"] = max(stats.get("dX", 0), assert_close(g["dX"][rows], r["dX"], dt, label + " dX", skip))
+        if adam is not None and s is None and not kink_parts:
+            for l in range(self.L):
+                Wn = W[l].astype(np.float64).copy()
+                mn, vn = adam["m"][l].astype(np.float64).copy(), adam["v"][l].astype(np.float64).copy()
+                oracle.adam(Wn, mn, vn, r["dW"][l], adam["lr"], adam["step"])
+                assert_close(g["m"][l], mn, dt, label + " adam m[%d]" % l)
+                assert_close(g["v"][l], vn, dt, label + " adam v[%d]" % l)
+                assert_close(g["W"][l], Wn, dt, label + " adam W[%d]" % l)
+
+
+def check_decode(graph, book, p_new_f32):
+    """Bit-exact decode parity on the given float32 probabilities (new order)."""
+    import torch
+    d = graph.decode_boundary(to_dev(p_new_f32.astype(np.float32)))
+    torch.cuda.synchronize()
+    ref = oracle.decode(book, p_new_f32.astype(np.float32))
+    assert np.array_equal(d["x"].cpu().numpy(), ref["x"])
+    assert np.array_equal(d["viol"].cpu().numpy(), ref["viol"])
+    assert np.array_equal(d["per_part"].cpu().numpy(), ref["per_part"])
+    c = d["counts"].cpu().numpy().tolist()
+    assert c == [ref["set_size"], ref["intra_viol"], ref["boundary_viol"]]
+    assert int(ref["per_part"].sum()) == 2 * ref["boundary_viol"]
+    return ref

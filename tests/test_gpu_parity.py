@@ -1,0 +1,201 @@
+"""GPU parity: the CUDA library, called through its C ABI binding, against the CPU oracle
+on the same seeded inputs -- bit-exact for integer outputs, within the stated tolerances
+for floating point."""
+import numpy as np
+import pytest
+
+import oracle
+import synth_inputs as si
+from helpers import tiny_graph, rand_weights, rand_features
+from gpu_common import StepCase, check_bookkeeping, check_decode, load_graph, to_dev
+
+pytestmark = pytest.mark.gpu
+
+
+def _star_plus_isolated(n):
+    """Node 0 joined to every node of the first half (a hub row of length n/2-1), second
+    half isolated."""
+    half = n // 2
+    eu = np.zeros(half - 1, np.int32)
+    ev = np.arange(1, half, dtype=np.int32)
+    return eu, ev
+
+
+GRAPHS = {
+    "er_random_parts": lambda: tiny_graph(200, 0.06, 7, seed=3),
+    "one_part": lambda: tiny_graph(150, 0.08, 1, seed=4),
+    "every_node_own_part": lambda: tiny_graph(64, 0.1, 64, seed=5),
+    "empty_parts": lambda: (lambda g: (g[0], g[1], np.where(g[2] == 3, 2, g[2]).astype(np.int32)))(
+        tiny_graph(120, 0.08, 6, seed=6)),
+    "hub_and_isolated": lambda: _star_plus_isolated(300) + (np.zeros(300, np.int32),),
+    "no_edges": lambda: (np.zeros(0, np.int32), np.zeros(0, np.int32), si.contiguous_partition(50, 4)),
+    "dense_small": lambda: tiny_graph(90, 0.5, 2, seed=8, contiguous=True),
+}
+
+
+def _n_S(part):
+    return part.size, int(part.max()) + 1
+
+
+@pytest.mark.parametrize("name", sorted(GRAPHS))
+def test_bookkeeping_and_decode_small(name):
+    eu, ev, part = GRAPHS[name]()
+    n, S = _n_S(part)
+    if name == "empty_parts":
+        S = 6
+    book = oracle.bookkeeping(n, eu, ev, part, S)
+    graph = load_graph(n, eu, ev, part, S)
+    check_bookkeeping(graph, book)
+    p = si.uniform01(17, 0, n).astype(np.float32)
+    p[::5] = 0.5
+    check_decode(graph, book, p)
+    check_decode(graph, book, np.full(n, 0.5, np.float32))
+    check_decode(graph, book, np.zeros(n, np.float32))
+
+
+def test_partition_load_rejects_bad_graphs():
+    import paper_2511_09261_b200 as gnnco
+    part = np.zeros(4, np.int32)
+    cases = [
+        (np.array([0, 1, 2], np.int32), np.array([1, 2, 2], np.int32), part, 1, gnnco.NOT_SIMPLE_GRAPH),
+        (np.array([0, 1], np.int32), np.array([1, 0], np.int32), part, 1, gnnco.NOT_SIMPLE_GRAPH),
+        (np.array([0], np.int32), np.array([7], np.int32), part, 1, gnnco.OUT_OF_RANGE),
+        (np.array([0], np.int32), np.array([1], np.int32), np.array([0, 0, 3, 0], np.int32), 2, gnnco.OUT_OF_RANGE),
+        (np.array([0, 2], np.int32), np.array([2, 0], np.int32), np.array([0, 0, 1, 1], np.int32), 2,
+         gnnco.NOT_SIMPLE_GRAPH),
+    ]
+    for eu, ev, pt, S, code in cases:
+        with pytest.raises(gnnco.GnncoError) as e:
+            load_graph(pt.size, eu, ev, pt, S)
+        assert e.value.status == code
+
+
+STEP_CASES = [
+    ("er_random_parts", [5, 1], None, 0.0),
+    ("er_random_parts", [6, 4, 1], None, 0.7),
+    ("er_random_parts", [7, 5, 3, 1], None, 0.0),
+    ("er_random_parts", [64, 32, 1], None, 0.5),
+    ("er_random_parts", [20, 12, 8, 1], 1, 0.5),
+    ("one_part", [128, 64, 1], None, 0.0),
+    ("one_part", [16, 8, 1], 1, 1.0),
+    ("every_node_own_part", [8, 4, 1], None, 0.0),
+    ("empty_parts", [12, 12, 1], None, 0.3),
+    ("hub_and_isolated", [32, 16, 1], None, 0.0),
+    ("hub_and_isolated", [256, 8, 1], None, 0.0),
+    ("no_edges", [4, 4, 1], None, 0.0),
+    ("dense_small", [24, 40, 1], None, 0.2),
+    ("dense_small", [130, 70, 1], None, 0.0),
+]
+
+
+@pytest.mark.parametrize("name,dims,sets,lam", STEP_CASES)
+def test_train_step_small_f32(name, dims, sets, lam):
+    eu, ev, part = GRAPHS[name]()
+    n, S = _n_S(part)
+    if name == "empty_parts":
+        S = 6
+    book = oracle.bookkeeping(n, eu, ev, part, S)
+    graph = load_graph(n, eu, ev, part, S)
+    X = rand_features(n, dims[0], 11).astype(np.float32)
+    nsets = S if sets is None else sets
+    W = [w.astype(np.float32) for w in rand_weights(dims, nsets, 13, scale=1.5)]
+    pen = (si.uniform01(7, 0, n) < 0.3).astype(np.float32) if lam else None
+    case = StepCase(book, dims, "f32", nsets, lam=lam)
+    adam = dict(lr=1e-3, step=3, m=[0.01 * rand_weights(dims, nsets, 21)[l].astype(np.float32) for l in range(len(W))],
+                v=[np.square(0.02 * rand_weights(dims, nsets, 22)[l]).astype(np.float32) for l in range(len(W))])
+    g, stats = case.run(graph, X, W, pen, want_dx=True, adam=adam, label=name)
+    check_decode(graph, book, g["p"])
+
+
+@pytest.mark.parametrize("dims,sets", [([16, 8, 1], None), ([64, 32, 16, 1], None), ([256, 256, 1], None),
+                                       ([32, 16, 1], 1), ([6, 1], None)])
+def test_train_step_small_bf16(dims, sets):
+    eu, ev, part = tiny_graph(260, 0.05, 5, seed=9)
+    n, S = _n_S(part)
+    book = oracle.bookkeeping(n, eu, ev, part, S)
+    graph = load_graph(n, eu, ev, part, S)
+    X = si.round_to_bf16(rand_features(n, dims[0], 11).astype(np.float32))
+    nsets = S if sets is None else sets
+    W = [si.round_to_bf16(w.astype(np.float32)) for w in rand_weights(dims, nsets, 13, scale=1.5)]
+    case = StepCase(book, dims, "bf16", nsets, lam=0.4)
+    pen = (si.uniform01(7, 0, n) < 0.3).astype(np.float32)
+    adam = dict(lr=1e-3, step=1, m=[np.zeros_like(w) for w in W], v=[np.zeros_like(w) for w in W])
+    case.run(graph, X, W, pen, want_dx=True, adam=adam, label="bf16")
+
+
+def test_forward_only_matches_full_step_and_skips_update():
+    import torch
+    import paper_2511_09261_b200 as gnnco
+    eu, ev, part = tiny_graph(200, 0.06, 7, seed=3)
+    n, S = _n_S(part)
+    graph = load_graph(n, eu, ev, part, S)
+    dims = [16, 8, 1]
+    X = to_dev(rand_features(n, 16, 1).astype(np.float32))
+    W = [to_dev(w.astype(np.float32)) for w in rand_weights(dims, S, 2)]
+    W0 = [w.clone() for w in W]
+    model = gnnco.Model(dims, W)
+    opt = gnnco.Adam(model)
+    l1, p1 = graph.train_step(model, X, 2.0, 1.0, opt=opt, flags=gnnco.FORWARD_ONLY)
+    l1, p1 = l1.clone(), p1.clone()
+    assert opt.step == 1 and all(torch.equal(a, b) for a, b in zip(W, W0))
+    l2, p2 = graph.train_step(model, X, 2.0, 1.0, opt=None)
+    assert torch.equal(l1, l2) and torch.equal(p1, p2)
+    assert all(torch.equal(a, b) for a, b in zip(W, W0))          # opt=None: gradients only
+    graph.train_step(model, X, 2.0, 1.0, opt=opt)
+    assert opt.step == 2 and not torch.equal(W[0], W0[0])
+
+
+def test_step_is_deterministic_run_to_run():
+    import torch
+    import paper_2511_09261_b200 as gnnco
+    w = si.make_workload(3)
+    graph = load_graph(w.n, w.eu, w.ev, w.part, w.S)
+    perm = graph.arrays()["perm"].cpu().numpy()
+    X = to_dev(w.features_f32()[perm])
+    outs = []
+    for _ in range(2):
+        W = [to_dev(w.weights(l)) for l in range(w.L)]
+        model = gnnco.Model(w.dims, W)
+        dW = [torch.empty_like(t) for t in W]
+        dX = torch.empty_like(X)
+        loss, p = graph.train_step(model, X, 2.0, 1.0, dW=dW, dX=dX, flags=gnnco.WANT_DX)
+        outs.append([loss.clone(), p.clone(), dX.clone()] + [d.clone() for d in dW])
+    for a, b in zip(*outs):
+        assert torch.equal(a, b)
+
+
+def test_host_variant_matches_device_variant():
+    import torch
+    import paper_2511_09261_b200 as gnnco
+    w = si.make_workload(1)
+    graph = load_graph(w.n, w.eu, w.ev, w.part, w.S)
+    perm = graph.arrays()["perm"].cpu().numpy()
+    Xh = torch.from_numpy(w.features_f32()[perm]).pin_memory()
+    pen = torch.from_numpy(w.penalty()[perm]).pin_memory()
+    res = []
+    for host in (False, True):
+        W = [to_dev(w.weights(l)) for l in range(w.L)]
+        model = gnnco.Model(w.dims, W)
+        opt = gnnco.Adam(model)
+        if host:
+            loss, p = graph.train_step_host(model, Xh, 2.0, 1.0, 1.0, pen, opt)
+            res.append((loss.clone(), p.clone(), W[0].cpu()))
+        else:
+            loss, p = graph.train_step(model, Xh.cuda(), 2.0, 1.0, 1.0, pen.cuda(), opt)
+            res.append((loss.cpu(), p.cpu(), W[0].cpu()))
+    for a, b in zip(*res):
+        assert torch.equal(a, b)
+
+
+def test_gather_rows_roundtrip():
+    import torch
+    w = si.make_workload(1)
+    graph = load_graph(w.n, w.eu, w.ev, w.part, w.S)
+    arr = graph.arrays()
+    X = to_dev(w.features_f32())
+    Xn = graph.gather_rows(X, arr["perm"])
+    assert torch.equal(Xn, X[arr["perm"].long()])
+    back = graph.gather_rows(Xn, arr["inv_perm"])
+    assert torch.equal(back, X)
+    v = to_dev(np.arange(w.n, dtype=np.float32))
+    assert torch.equal(graph.gather_rows(v, arr["perm"]), arr["perm"].float())
