@@ -1,0 +1,428 @@
+#!/usr/bin/env python
+"""Benchmark of the partitioned-GNN training step (edges/s, fwd + bwd + Adam + decode).
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--config 1..5] [--impl ours|reference]
+
+One "step" is one pass of the whole hot path over one batch: gnnco_train_step (forward,
+objective, backward with input gradient, Adam) followed by gnnco_decode_boundary.  The
+default workload is configuration 5 (Chung-Lu, 10M nodes, 40M edges, 4096 subgraphs,
+256-256-256-1, bfloat16 features).  Bookkeeping (gnnco_partition_load) runs once per graph
+and is reported separately.
+
+With N > 1 (launched by torch.distributed.run) every rank runs an independent replica on
+its own GPU: subgraphs never exchange data during training, so there is no collective on
+the data path; the only communication is the barrier and the max-over-ranks of the time.
+
+`--impl reference` times the CPU oracle, as it stands, on the host cores.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import sys
+import threading
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+import synth_inputs as si  # noqa: E402
+
+METRIC = "partitioned-GNN train-step edges/s (fwd+bwd)"
+ORACLE_SAMPLE_PARTS = {1: 8, 2: 64, 3: 16, 4: 256, 5: 64}
+
+
+def _peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            d = json.load(f)
+        return float(d["hbm_gbs"]), "measured"
+    return 6650.0, "fallback"
+
+
+def _host_threads() -> int:
+    try:
+        return len(os.sched_getaffinity(0))
+    except AttributeError:
+        return os.cpu_count() or 1
+
+
+# ------------------------------------------------------------------ CPU oracle baseline
+def _oracle_sample(w, n_parts, seed=12345):
+    """Seeded sample of subgraphs with everything the oracle needs for them (inputs come
+    from the generators; the sample is the same on every call)."""
+    import oracle
+    t0 = time.time()
+    book = oracle.bookkeeping(w.n, w.eu, w.ev, w.part, w.S)
+    t_book = time.time() - t0
+    S = w.S
+    order = np.argsort(si.u64(seed, 0, S), kind="stable")
+    parts = sorted(order[: min(n_parts, S)].tolist())
+    items = []
+    edges = 0
+    for s in parts:
+        lo, hi = int(book["part_ptr"][s]), int(book["part_ptr"][s + 1])
+        if hi == lo:
+            continue
+        rp = book["rowptr"][lo:hi + 1] - book["rowptr"][lo]
+        ci = book["colidx"][book["rowptr"][lo]:book["rowptr"][hi]] - lo
+        X = w.features_f32(book["perm"][lo:hi]).astype(np.float64)
+        W = [w.weights(l, [s])[0].astype(np.float64) for l in range(w.L)]
+        items.append((rp, ci, X, W))
+        edges += int(ci.size) // 2
+    return book, parts, items, edges, t_book
+
+
+def _oracle_step(w, items, threads):
+    """One fwd+bwd+Adam pass of the oracle over the sampled subgraphs, subgraphs spread over
+    `threads` host threads (the C code releases the GIL inside each call)."""
+    import oracle
+    from concurrent.futures import ThreadPoolExecutor
+
+    def one(item):
+        rp, ci, X, W = item
+        r = oracle.subgraph_step(rp, ci, w.dims, X, W, w.alpha, w.beta, want_dX=True, store_bf16=(w.dtype == "bf16"))
+        for l in range(w.L):
+            m, v = np.zeros_like(W[l]), np.zeros_like(W[l])
+            Wc = W[l].copy()
+            oracle.adam(Wc, m, v, r["dW"][l], w.lr, 1)
+        return r["loss"]
+
+    with ThreadPoolExecutor(max_workers=threads) as ex:
+        return list(ex.map(one, items))
+
+
+def oracle_rate(w, cfg_index, steps=1, warmup=0):
+    threads = _host_threads()
+    n_parts = ORACLE_SAMPLE_PARTS[cfg_index]
+    book, parts, items, edges, t_book = _oracle_sample(w, n_parts)
+    for _ in range(warmup):
+        _oracle_step(w, items, threads)
+    t0 = time.time()
+    for _ in range(steps):
+        _oracle_step(w, items, threads)
+    dt = (time.time() - t0) / max(1, steps)
+    sample = "%d of %d subgraphs (seeded), %d intra edges, one fwd+bwd+Adam pass each step; bookkeeping of the " \
+             "whole graph took %.1f s single-threaded" % (len(items), w.S, edges, t_book)
+    return dict(value=edges / dt, unit="edges/s", cores=min(threads, max(1, len(items))), kind="oracle",
+                sample=sample, seconds_per_step=dt)
+
+
+# ------------------------------------------------------------------------ clock sampling
+class ClockSampler:
+    """Samples SM clock and throttle reasons of one GPU while the timed region runs
+    (read-only NVML queries)."""
+
+    def __init__(self, index: int):
+        self.index, self.samples, self.reasons, self.max_mhz = index, [], set(), None
+        self._stop = threading.Event()
+        self._thread = None
+        try:
+            import pynvml
+            pynvml.nvmlInit()
+            self.nv = pynvml
+            vis = os.environ.get("CUDA_VISIBLE_DEVICES")
+            phys = index
+            if vis:
+                ids = [x for x in vis.split(",") if x.strip() != ""]
+                if index < len(ids) and ids[index].strip().isdigit():
+                    phys = int(ids[index])
+            self.handle = pynvml.nvmlDeviceGetHandleByIndex(phys)
+            self.max_mhz = int(pynvml.nvmlDeviceGetMaxClockInfo(self.handle, pynvml.NVML_CLOCK_SM))
+        except Exception:
+            self.nv = None
+
+    def _loop(self):
+        nv = self.nv
+        names = {}
+        for k in dir(nv):
+            if k.startswith("nvmlClocksThrottleReason") or k.startswith("nvmlClocksEventReason"):
+                val = getattr(nv, k)
+                if isinstance(val, int) and val not in (0,) and "All" not in k:
+                    names[val] = k.replace("nvmlClocksThrottleReason", "").replace("nvmlClocksEventReason", "")
+        while not self._stop.is_set():
+            try:
+                self.samples.append(int(nv.nvmlDeviceGetClockInfo(self.handle, nv.NVML_CLOCK_SM)))
+                try:
+                    mask = int(nv.nvmlDeviceGetCurrentClocksEventReasons(self.handle))
+                except Exception:
+                    mask = int(nv.nvmlDeviceGetCurrentClocksThrottleReasons(self.handle))
+                for bit, name in names.items():
+                    if mask & bit and name not in ("GpuIdle", "None", "ApplicationsClocksSetting"):
+                        self.reasons.add(name)
+            except Exception:
+                pass
+            self._stop.wait(0.1)
+
+    def start(self):
+        if self.nv is not None:
+            self._thread = threading.Thread(target=self._loop, daemon=True)
+            self._thread.start()
+
+    def stop(self):
+        self._stop.set()
+        if self._thread is not None:
+            self._thread.join(timeout=2)
+        med = int(np.median(self.samples)) if self.samples else None
+        return dict(sm_mhz=med, sm_max_mhz=self.max_mhz, reasons=sorted(self.reasons), samples=len(self.samples))
+
+
+# ------------------------------------------------------------- algorithmic bytes per launch
+def algorithmic_bytes(kind, w, n, nnz, S):
+    """Compulsory bytes one launch of each kernel family moves: every tensor it must read or
+    write counted once (a subgraph's feature tile is assumed to stay on chip while its rows
+    are gathered, so neighbour re-reads are not counted)."""
+    b = 2 if w.dtype == "bf16" else 4
+    d = w.dims
+    L = w.L
+    hidden = list(range(1, L))                   # hidden layers, widths d[l-1] -> d[l]
+    csr = 4 * nnz + 4 * (n + 1)
+    per = {}
+    if hidden:
+        per["aggregate_fwd"] = np.mean([2 * n * d[l - 1] * b + csr + 4 * n for l in hidden])
+        per["aggregate_bwd"] = np.mean([2 * n * d[l - 1] * b + csr + (n * d[l - 1] * b if l > 1 else 0) for l in hidden])
+        per["transform_fwd"] = np.mean([n * (d[l - 1] + d[l]) * b + S * d[l - 1] * d[l] * b for l in hidden])
+        per["transform_bwd"] = np.mean([n * (d[l - 1] + d[l]) * b + 4 * n + S * d[l - 1] * d[l] * b for l in hidden])
+        per["weight_grad"] = np.mean([n * (d[l - 1] + d[l]) * b + S * d[l - 1] * d[l] * 4 for l in hidden])
+    F = d[L - 1]
+    per["gemv"] = n * F * b + 4 * n + S * F * b
+    per["weight_grad_vec"] = n * F * b + 4 * n + S * F * 4
+    per["rank1_masked"] = 2 * n * F * b + 4 * n
+    per["output_forward"] = csr + 4 * n * 3
+    per["objective"] = csr + 4 * n * 4
+    per["output_backward"] = csr + 4 * n * 2
+    wcounts = [S * d[l] * d[l + 1] for l in range(L)]
+    per["adam"] = np.mean([7 * 4 * c for c in wcounts])
+    per["cast_bf16"] = np.mean([6 * c for c in wcounts])
+    per["decode"] = 5 * n + csr + n
+    return float(per.get(kind, 0.0))
+
+
+# ------------------------------------------------------------------------------ our arm
+def run_ours(args):
+    import torch
+    import paper_2511_09261_b200 as gnnco
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    if args.gpus != world and world > 1:
+        raise SystemExit("--gpus must equal WORLD_SIZE")
+    if args.gpus > 1 and world == 1:
+        raise SystemExit("launch N > 1 with torch.distributed.run (one rank per GPU)")
+    dist = None
+    if world > 1:
+        import torch.distributed as dist_mod
+        dist = dist_mod
+        os.environ.setdefault("MASTER_ADDR", "127.0.0.1")
+        torch.cuda.set_device(local_rank)
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
+    dev = torch.device("cuda", local_rank)
+    torch.cuda.set_device(dev)
+
+    w = si.make_workload(args.config)
+    bf16 = w.dtype == "bf16"
+
+    # CPU baseline first (before the first GPU call), rank 0 of a single-GPU run only
+    cpu = None
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        cpu = oracle_rate(w, args.config)
+
+    # ---- device-resident inputs
+    t0 = time.time()
+    eu, ev, part = (torch.from_numpy(a).to(dev) for a in (w.eu, w.ev, w.part))
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    graph = gnnco.gnnco_partition_load(eu, ev, part, w.S)
+    e1.record()
+    torch.cuda.synchronize()
+    load_ms = e0.elapsed_time(e1)
+    arr = graph.arrays()
+    if bf16:
+        X_host_orig = torch.from_numpy(w.features_bf16_bits().view(np.int16)).view(torch.bfloat16)
+    else:
+        X_host_orig = torch.from_numpy(w.features_f32())
+    X_orig = X_host_orig.to(dev)
+    X = graph.gather_rows(X_orig, arr["perm"])          # embeddings in the library's node order
+    del X_orig
+    pen = graph.gather_rows(torch.from_numpy(w.penalty()).to(dev), arr["perm"])
+    W = [torch.from_numpy(w.weights(l)).to(dev) for l in range(w.L)]
+    model = gnnco.Model(w.dims, W, gnnco.BF16 if bf16 else gnnco.F32)
+    opt = gnnco.Adam(model, lr=w.lr)
+    loss = torch.empty(w.S, dtype=torch.float32, device=dev)
+    p = torch.empty(w.n, dtype=torch.float32, device=dev)
+    dX = torch.empty_like(X)
+    x = torch.empty(w.n, dtype=torch.uint8, device=dev)
+    viol = torch.empty(graph.E_b, dtype=torch.uint8, device=dev)
+    per_part = torch.empty(w.S, dtype=torch.int32, device=dev)
+    counts = torch.empty(3, dtype=torch.int64, device=dev)
+    flush = None
+    tensor_bytes = w.n * w.dims[0] * (2 if bf16 else 4)
+    if tensor_bytes < 256 * 1024 * 1024:
+        flush = torch.empty(256 * 1024 * 1024, dtype=torch.uint8, device=dev)
+
+    def step():
+        graph.train_step(model, X, w.alpha, w.beta, w.lam, pen, opt, loss=loss, p=p, dX=dX, flags=gnnco.WANT_DX)
+        graph.decode_boundary(p, 0.5, x=x, viol=viol, per_part=per_part, counts=counts)
+
+    for _ in range(args.warmup):
+        step()
+    torch.cuda.synchronize()
+    if dist is not None:
+        dist.barrier()
+    sampler = ClockSampler(local_rank)
+    sampler.start()
+    starts = [torch.cuda.Event(enable_timing=True) for _ in range(args.steps)]
+    ends = [torch.cuda.Event(enable_timing=True) for _ in range(args.steps)]
+    launches0 = graph.launch_count()
+    graph.profile_begin()
+    torch.cuda.synchronize()
+    for k in range(args.steps):
+        if flush is not None:
+            flush.fill_(k)                              # evict L2 between iterations (not timed)
+        starts[k].record()
+        step()
+        ends[k].record()
+    torch.cuda.synchronize()
+    prof = graph.profile_end()
+    launches = graph.launch_count() - launches0
+    clocks = sampler.stop()
+    if dist is not None:
+        dist.barrier()
+    total_ms = sum(s.elapsed_time(e) for s, e in zip(starts, ends))
+    if dist is not None:
+        t = torch.tensor([total_ms], dtype=torch.float64, device=dev)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        total_ms = float(t.item())
+    ms_per_step = total_ms / args.steps
+    value = world * graph.E_in / (ms_per_step * 1e-3)
+
+    # ---- per-kernel shares and the dominant kernel's roofline
+    nnz = 2 * graph.E_in
+    peak, peak_src = _peaks()
+    kern = {}
+    for name, (calls, ms) in prof.items():
+        ab = algorithmic_bytes(name, w, w.n, nnz, w.S)
+        per_call_ms = ms / calls
+        kern[name] = dict(calls=calls, total_ms=round(ms, 4), share=round(ms / max(total_ms, 1e-9), 4),
+                          algo_GBs=round(ab / (per_call_ms * 1e-3) / 1e9, 1) if per_call_ms > 0 else None)
+    top = max(prof.items(), key=lambda kv: kv[1][1])[0]
+    achieved = kern[top]["algo_GBs"]
+    roofline = dict(bound="hbm", kernel=top, achieved=achieved, peak=peak, unit="GB/s",
+                    frac=round(achieved / peak, 4), traffic=TRAFFIC_BYTES.get((args.config, top)),
+                    peak_source="%s (MEASURED_PEAKS.json hbm_gbs)" % peak_src if peak_src == "measured" else "fallback",
+                    algorithmic_bytes_per_launch=algorithmic_bytes(top, w, w.n, nnz, w.S))
+    agg = {k: kern[k] for k in ("aggregate_fwd", "aggregate_bwd") if k in kern}
+
+    # ---- end to end through the host-buffer entry point (rank-local; copies inside the timed region)
+    e2e = None
+    if not args.no_e2e:
+        Xh = torch.empty(X.shape, dtype=X.dtype).pin_memory()
+        Xh.copy_(X)                                    # the step's input, new node order, pinned
+        pen_h = pen.cpu().pin_memory()
+        loss_h = torch.empty(w.S, dtype=torch.float32).pin_memory()
+        p_h = torch.empty(w.n, dtype=torch.float32).pin_memory()
+        counts_h = torch.empty(3, dtype=torch.int64).pin_memory()
+
+        def step_host():
+            graph.train_step_host(model, Xh, w.alpha, w.beta, w.lam, pen_h, opt, loss_h, p_h)
+            p.copy_(p_h, non_blocking=True)
+            graph.decode_boundary(p, 0.5, x=x, viol=viol, per_part=per_part, counts=counts)
+            counts_h.copy_(counts, non_blocking=True)
+            torch.cuda.synchronize()
+
+        step_host()
+        n_e2e = args.steps
+        if dist is not None:
+            dist.barrier()
+        torch.cuda.synchronize()
+        t0 = time.perf_counter()
+        for _ in range(n_e2e):
+            step_host()
+        torch.cuda.synchronize()
+        dt = time.perf_counter() - t0
+        if dist is not None:
+            t = torch.tensor([dt], dtype=torch.float64, device=dev)
+            dist.all_reduce(t, op=dist.ReduceOp.MAX)
+            dt = float(t.item())
+        h2d = Xh.numel() * Xh.element_size() + pen_h.numel() * 4 + p_h.numel() * 4
+        d2h = loss_h.numel() * 4 + p_h.numel() * 4 + 24
+        e2e = dict(value=world * graph.E_in * n_e2e / dt, unit="edges/s", h2d_bytes_per_step=h2d,
+                   d2h_bytes_per_step=d2h, ms_per_step=dt / n_e2e * 1e3,
+                   note="gnnco_train_step_host: X, pen copied in and loss, p copied out every step; "
+                        "forward+loss+backward+Adam (no input gradient), then decode and its counts")
+
+    if rank == 0:
+        line = dict(
+            metric=METRIC, value=value, unit="edges/s", n_gpus=world, steps=args.steps, warmup=args.warmup,
+            ms_per_step=ms_per_step, higher_is_better=True, scaling="weak", vs_baseline=None,
+            dtype="bf16" if bf16 else "f32", data="synthetic",
+            config=dict(workload=w.name, index=args.config, n=w.n, E=w.E, E_in=graph.E_in, E_b=graph.E_b, S=w.S,
+                        dims=w.dims, max_intra_degree=graph.max_row, weight_sets=w.S, want_dx=True,
+                        l2="L2 flushed between steps (256 MB write, untimed)" if flush is not None
+                        else "inputs larger than L2",
+                        parallelism="replicas only (no collective on the data path)" if world > 1 else "1 GPU",
+                        partition_load_ms=round(load_ms, 3), edges_per_s_whole_graph=value * w.E / max(1, graph.E_in)),
+            roofline=roofline, aggregate_kernels=agg, kernels=kern, cpu_baseline=cpu, clocks=clocks, e2e=e2e,
+            gpu_launches=int(launches))
+        print(json.dumps(line))
+    if dist is not None:
+        dist.destroy_process_group()
+
+
+# DRAM traffic per launch (dram__bytes_read.sum + dram__bytes_write.sum) taken from ncu captures
+# of the kernel families as they stand; None until a capture of the current kernel exists.
+TRAFFIC_BYTES = {}
+
+
+# ----------------------------------------------------------------------- reference arm
+def run_reference(args):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    w = si.make_workload(args.config)
+    threads = _host_threads()
+    book, parts, items, edges, t_book = _oracle_sample(w, ORACLE_SAMPLE_PARTS[args.config])
+    for _ in range(args.warmup):
+        _oracle_step(w, items, threads)
+    t0 = time.time()
+    for _ in range(args.steps):
+        _oracle_step(w, items, threads)
+    dt = (time.time() - t0) / args.steps
+    value = edges / dt
+    sample = "%d of %d subgraphs (seeded), %d intra edges per step" % (len(items), w.S, edges)
+    line = dict(metric=METRIC, value=value, unit="edges/s", n_gpus=int(os.environ.get("WORLD_SIZE", "1")),
+                steps=args.steps, warmup=args.warmup, ms_per_step=dt * 1e3, higher_is_better=True, scaling="weak",
+                vs_baseline=None, dtype="f64", data="synthetic", impl="reference",
+                config=dict(workload=w.name, index=args.config, n=w.n, E=w.E, S=w.S, dims=w.dims),
+                cpu_baseline=dict(value=value, unit="edges/s", kind="oracle", cores=min(threads, len(items)),
+                                  sample=sample),
+                e2e=dict(value=value, unit="edges/s", h2d_bytes_per_step=0, d2h_bytes_per_step=0), gpu_launches=0)
+    print(json.dumps(line))
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=5)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--config", type=int, default=5, choices=[1, 2, 3, 4, 5])
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-e2e", action="store_true")
+    args = ap.parse_args()
+    if args.warmup < 3 and args.impl == "ours":
+        args.warmup = 3
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_ours(args)
+
+
+if __name__ == "__main__":
+    main()

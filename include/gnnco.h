@@ -203,6 +203,21 @@ int32_t gnnco_decode_boundary(const gnnco_handle* h, const float* p, float thres
 /* Host read of the device-side status word (synchronises `stream`). */
 int32_t gnnco_async_status(const gnnco_handle* h, void* stream, int32_t* status);
 
+/* Per-kernel timing (a measurement aid; Section 4.1 reports runtime as a metric).
+ * Between gnnco_profile_begin and gnnco_profile_end every kernel family of gnnco_train_step
+ * and gnnco_decode_boundary is bracketed by CUDA events on the launching stream.
+ * gnnco_profile_end synchronises `stream`, writes one entry per family that ran into
+ * `entries` (host array of `capacity` elements) and their number into *count; it returns
+ * GNNCO_WORKSPACE_TOO_SMALL if capacity was too small (*count then holds the need). */
+typedef struct {
+  char name[32];
+  int64_t calls;       /* launcher calls (a call may issue more than one kernel) */
+  double total_ms;     /* summed device time of those calls */
+} gnnco_profile_entry;
+int32_t gnnco_profile_begin(gnnco_handle* h);
+int32_t gnnco_profile_end(gnnco_handle* h, void* stream, gnnco_profile_entry* entries, int32_t capacity,
+                          int32_t* count);
+
 /* Number of kernels this handle has launched so far (for launch accounting). */
 int64_t gnnco_launch_count(const gnnco_handle* h);
 

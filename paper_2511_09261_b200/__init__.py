@@ -25,6 +25,7 @@ EXPORTS = [
     "gnnco_status_string", "gnnco_partition_workspace_bytes", "gnnco_partition_load", "gnnco_graph_info",
     "gnnco_gather_rows", "gnnco_train_workspace_bytes", "gnnco_train_step", "gnnco_train_host_workspace_bytes",
     "gnnco_train_step_host", "gnnco_decode_boundary", "gnnco_async_status", "gnnco_launch_count", "gnnco_destroy",
+    "gnnco_profile_begin", "gnnco_profile_end",
 ]
 
 _vp, _i32, _i64, _u32, _f32, _sz = (ctypes.c_void_p, ctypes.c_int32, ctypes.c_int64, ctypes.c_uint32, ctypes.c_float,
@@ -57,6 +58,10 @@ class AdamState(ctypes.Structure):
 
 class TrainOut(ctypes.Structure):
     _fields_ = [("loss", _vp), ("p", _vp), ("z", _vp), ("dW", _vp * MAX_LAYERS), ("dX", _vp)]
+
+
+class ProfileEntry(ctypes.Structure):
+    _fields_ = [("name", ctypes.c_char * 32), ("calls", _i64), ("total_ms", ctypes.c_double)]
 
 
 class GnncoError(RuntimeError):
@@ -100,6 +105,8 @@ def load_library(build_if_missing: bool = True):
     lib.gnnco_launch_count.argtypes = [_vp]
     lib.gnnco_launch_count.restype = _i64
     lib.gnnco_destroy.argtypes = [_vp]
+    lib.gnnco_profile_begin.argtypes = [_vp]
+    lib.gnnco_profile_end.argtypes = [_vp, _vp, ctypes.POINTER(ProfileEntry), _i32, ctypes.POINTER(_i32)]
     for name in EXPORTS:
         if name not in ("gnnco_status_string", "gnnco_launch_count"):
             getattr(lib, name).restype = _i32
@@ -343,6 +350,18 @@ class PartitionedGraph:
         s = _i32(0)
         _check(self._lib.gnnco_async_status(self._handle, _stream_ptr(stream), ctypes.byref(s)), "gnnco_async_status")
         return int(s.value)
+
+    def profile_begin(self) -> None:
+        _check(self._lib.gnnco_profile_begin(self._handle), "gnnco_profile_begin")
+
+    def profile_end(self, stream=None) -> dict:
+        """``gnnco_profile_end``: {kernel family: (calls, total_ms)} since profile_begin."""
+        entries = (ProfileEntry * 32)()
+        count = _i32(0)
+        _check(self._lib.gnnco_profile_end(self._handle, _stream_ptr(stream), entries, 32, ctypes.byref(count)),
+               "gnnco_profile_end")
+        return {entries[k].name.decode(): (int(entries[k].calls), float(entries[k].total_ms))
+                for k in range(count.value)}
 
     def launch_count(self) -> int:
         return int(self._lib.gnnco_launch_count(self._handle))

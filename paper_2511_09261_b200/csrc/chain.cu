@@ -114,6 +114,7 @@ __global__ void __launch_bounds__(256) output_backward(const float* __restrict__
 }  // namespace
 
 int32_t launch_output_forward(gnnco_handle* h, const float* u, float* z, float* p, cudaStream_t st) {
+  ProfScope prof_(h, K_OUT_FWD, st);
   unsigned grid = (unsigned)((h->n + 255) / 256);
   output_forward<<<grid, 256, 0, st>>>(u, h->rowptr, h->colidx, h->inv_deg, z, p, h->n);
   h->launches += 1;
@@ -123,6 +124,7 @@ int32_t launch_output_forward(gnnco_handle* h, const float* u, float* z, float* 
 
 int32_t launch_objective(gnnco_handle* h, const float* p, const float* pen, float alpha, float beta, float lambda,
                          float* item_loss, float* loss, float* t, cudaStream_t st) {
+  ProfScope prof_(h, K_OBJECTIVE, st);
   if (h->n_items > 0)
     objective_items<<<h->n_items, 256, 0, st>>>(p, pen, h->rowptr, h->colidx, h->inv_deg, h->item_row0, h->item_row1,
                                                 alpha, beta, lambda, item_loss, t);
@@ -133,6 +135,7 @@ int32_t launch_objective(gnnco_handle* h, const float* p, const float* pen, floa
 }
 
 int32_t launch_output_backward(gnnco_handle* h, const float* t, float* g, cudaStream_t st) {
+  ProfScope prof_(h, K_OUT_BWD, st);
   unsigned grid = (unsigned)((h->n + 255) / 256);
   output_backward<<<grid, 256, 0, st>>>(t, h->rowptr, h->colidx, g, h->n);
   h->launches += 1;

@@ -88,6 +88,7 @@ __global__ void __launch_bounds__(256) boundary_conflicts_kernel(const uint8_t* 
 
 int32_t launch_decode(gnnco_handle* h, const float* p, float thr, uint8_t* x, uint8_t* viol, int32_t* per_part,
                       gnnco_counts* counts, cudaStream_t st) {
+  ProfScope prof_(h, K_DECODE, st);
   GNNCO_CUDA_TRY(cudaMemsetAsync(counts, 0, sizeof(gnnco_counts), st));
   if (per_part) GNNCO_CUDA_TRY(cudaMemsetAsync(per_part, 0, (size_t)h->S * sizeof(int32_t), st));
   unsigned long long* c = reinterpret_cast<unsigned long long*>(counts);

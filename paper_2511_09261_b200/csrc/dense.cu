@@ -218,6 +218,7 @@ inline unsigned blocks_for(int64_t work, int threads) { return (unsigned)((work 
 
 int32_t launch_transform(gnnco_handle* h, int dtype, const void* A, const void* W, int64_t w_stride, void* Y, int K,
                          int N, bool transB, bool relu, const float* row_scale, cudaStream_t stream) {
+  ProfScope prof_(h, transB ? K_TRANSFORM_BWD : K_TRANSFORM_FWD, stream);
   if (h->n_tiles == 0) return GNNCO_OK;
   dim3 grid(h->n_tiles, (N + BN - 1) / BN);
   if (grid.y > 65535) return GNNCO_UNSUPPORTED;
@@ -241,6 +242,7 @@ int32_t launch_transform(gnnco_handle* h, int dtype, const void* A, const void* 
 
 int32_t launch_gemv(gnnco_handle* h, int dtype, const void* H, const void* w, int64_t w_stride, float* u, int F,
                     cudaStream_t stream) {
+  ProfScope prof_(h, K_GEMV, stream);
   unsigned grid = blocks_for(h->n, 8);
   if (dtype == GNNCO_F32)
     gemv_rows<float, float><<<grid, 256, 0, stream>>>((const float*)H, (const float*)w, w_stride, h->node_part, u,
@@ -257,6 +259,7 @@ int32_t launch_gemv(gnnco_handle* h, int dtype, const void* H, const void* w, in
 
 int32_t launch_weight_grad(gnnco_handle* h, int dtype, const void* A, const void* G, float* dW, int K, int N,
                            cudaStream_t stream) {
+  ProfScope prof_(h, K_WEIGHT_GRAD, stream);
   dim3 grid(h->S, (K + 63) / 64, (N + 63) / 64);
   if (grid.y > 65535 || grid.z > 65535) return GNNCO_UNSUPPORTED;
   if (dtype == GNNCO_F32)
@@ -273,6 +276,7 @@ int32_t launch_weight_grad(gnnco_handle* h, int dtype, const void* A, const void
 
 int32_t launch_weight_grad_vec(gnnco_handle* h, int dtype, const void* H, const float* g, float* dw, int F,
                                cudaStream_t stream) {
+  ProfScope prof_(h, K_WEIGHT_GRAD_VEC, stream);
   dim3 grid(h->S, (F + 255) / 256);
   if (grid.y > 65535) return GNNCO_UNSUPPORTED;
   if (dtype == GNNCO_F32)
@@ -288,6 +292,7 @@ int32_t launch_weight_grad_vec(gnnco_handle* h, int dtype, const void* H, const 
 
 int32_t launch_rank1_masked(gnnco_handle* h, int dtype, const float* g, const void* w, int64_t w_stride, const void* H,
                             void* dZ, int F, cudaStream_t stream) {
+  ProfScope prof_(h, K_RANK1, stream);
   unsigned grid = blocks_for(h->n * F, 256);
   if (dtype == GNNCO_F32)
     rank1_masked_kernel<float, float><<<grid, 256, 0, stream>>>(g, (const float*)w, w_stride, h->node_part,
@@ -304,6 +309,7 @@ int32_t launch_rank1_masked(gnnco_handle* h, int dtype, const float* g, const vo
 
 int32_t launch_sum_over_sets(gnnco_handle* h, const float* in, float* out, int64_t count, int32_t sets,
                              cudaStream_t stream) {
+  ProfScope prof_(h, K_SUM_SETS, stream);
   sum_over_sets_kernel<<<blocks_for(count, 256), 256, 0, stream>>>(in, out, count, sets);
   h->launches += 1;
   GNNCO_LAUNCH_CHECK();
@@ -311,6 +317,7 @@ int32_t launch_sum_over_sets(gnnco_handle* h, const float* in, float* out, int64
 }
 
 int32_t launch_cast_bf16(gnnco_handle* h, const float* in, __nv_bfloat16* out, int64_t count, cudaStream_t stream) {
+  ProfScope prof_(h, K_CAST, stream);
   cast_bf16_kernel<<<blocks_for(count, 256), 256, 0, stream>>>(in, out, count);
   h->launches += 1;
   GNNCO_LAUNCH_CHECK();
@@ -319,6 +326,7 @@ int32_t launch_cast_bf16(gnnco_handle* h, const float* in, __nv_bfloat16* out, i
 
 int32_t launch_adam(gnnco_handle* h, float* W, float* m, float* v, const float* g, int64_t count, float lr, float b1,
                     float b2, float eps, float c1, float c2, cudaStream_t stream) {
+  ProfScope prof_(h, K_ADAM, stream);
   adam_kernel<<<blocks_for(count, 256), 256, 0, stream>>>(W, m, v, g, count, lr, b1, b2, eps, 1.0f / c1, 1.0f / c2);
   h->launches += 1;
   GNNCO_LAUNCH_CHECK();

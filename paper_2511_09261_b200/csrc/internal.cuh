@@ -23,6 +23,30 @@
 constexpr int kGemmTileRows = 128;   // rows of one dense-transform tile (never straddles a subgraph)
 constexpr int kItemRows = 1024;      // rows of one objective work item (never straddles a subgraph)
 
+// Kernel families, for launch accounting and per-kernel timing.
+enum KernelKind {
+  K_AGG_FWD, K_AGG_BWD, K_TRANSFORM_FWD, K_TRANSFORM_BWD, K_WEIGHT_GRAD, K_GEMV, K_WEIGHT_GRAD_VEC, K_RANK1,
+  K_SUM_SETS, K_CAST, K_ADAM, K_OUT_FWD, K_OBJECTIVE, K_OUT_BWD, K_DECODE, K_KIND_COUNT
+};
+
+// Optional per-kernel timing: while `on`, every launcher brackets its launches with a pair
+// of CUDA events on the launching stream; gnnco_profile_end turns the pairs into totals.
+struct Profiler {
+  struct Rec { int kind; cudaEvent_t a, b; };
+  bool on = false;
+  std::vector<cudaEvent_t> pool;
+  size_t used = 0;
+  std::vector<Rec> recs;
+  cudaEvent_t get() {
+    if (used == pool.size()) {
+      cudaEvent_t e = nullptr;
+      if (cudaEventCreate(&e) != cudaSuccess) return nullptr;
+      pool.push_back(e);
+    }
+    return pool[used++];
+  }
+};
+
 struct gnnco_handle {
   int64_t n = 0, E = 0, E_in = 0, E_b = 0;
   int32_t S = 0, max_row = 0;
@@ -39,6 +63,25 @@ struct gnnco_handle {
   int32_t n_tiles = 0, n_items = 0;
   std::vector<int32_t> h_part_ptr;
   int64_t launches = 0;
+  Profiler prof;
+};
+
+struct ProfScope {
+  gnnco_handle* h;
+  cudaStream_t st;
+  Profiler::Rec rec{};
+  bool on = false;
+  ProfScope(gnnco_handle* h_, int kind, cudaStream_t st_) : h(h_), st(st_) {
+    if (!h->prof.on) return;
+    rec.kind = kind;
+    rec.a = h->prof.get();
+    rec.b = h->prof.get();
+    if (!rec.a || !rec.b) return;
+    on = cudaEventRecord(rec.a, st) == cudaSuccess;
+  }
+  ~ProfScope() {
+    if (on && cudaEventRecord(rec.b, st) == cudaSuccess) h->prof.recs.push_back(rec);
+  }
 };
 
 static inline size_t align_up(size_t x, size_t a = 256) { return (x + a - 1) / a * a; }
@@ -57,9 +100,6 @@ struct Carver {
   }
   bool ok() const { return off <= cap; }
 };
-
-// ---- partition.cu
-int32_t partition_scratch_bytes(int64_t n, int64_t E, int32_t S, size_t* bytes);
 
 // ---- spmm.cu : out[i] = scale[i] * (in[i] + sum_{j in row i} in[j]), optionally zeroed where mask[i,f] <= 0
 int32_t launch_aggregate(gnnco_handle* h, int dtype, const void* in, void* out, int F, const float* row_scale,

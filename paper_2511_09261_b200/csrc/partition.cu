@@ -539,6 +539,8 @@ extern "C" int32_t gnnco_async_status(const gnnco_handle* h, void* stream, int32
 extern "C" int64_t gnnco_launch_count(const gnnco_handle* h) { return h ? h->launches : 0; }
 
 extern "C" int32_t gnnco_destroy(gnnco_handle* h) {
+  if (h)
+    for (cudaEvent_t e : h->prof.pool) cudaEventDestroy(e);
   delete h;
   return GNNCO_OK;
 }

@@ -179,6 +179,7 @@ int32_t aggregate_typed(gnnco_handle* h, const T* in, T* out, int F, const float
 
 int32_t launch_aggregate(gnnco_handle* h, int dtype, const void* in, void* out, int F, const float* row_scale,
                          const void* relu_mask, cudaStream_t st) {
+  ProfScope prof_(h, row_scale ? K_AGG_FWD : K_AGG_BWD, st);
   if (dtype == GNNCO_F32)
     return aggregate_typed<float>(h, (const float*)in, (float*)out, F, row_scale, (const float*)relu_mask, st);
   if (dtype == GNNCO_BF16)
