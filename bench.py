@@ -98,7 +98,7 @@ def _oracle_step(w, items, threads):
 
 def oracle_rate(w, cfg_index, steps=1, warmup=0):
     threads = _host_threads()
-    n_parts = ORACLE_SAMPLE_PARTS[cfg_index]
+    n_parts = min(ORACLE_SAMPLE_PARTS[cfg_index], w.S)
     book, parts, items, edges, t_book = _oracle_sample(w, n_parts)
     for _ in range(warmup):
         _oracle_step(w, items, threads)
@@ -224,7 +224,7 @@ def run_ours(args):
     dev = torch.device("cuda", local_rank)
     torch.cuda.set_device(dev)
 
-    w = si.make_workload(args.config)
+    w = si.make_workload(args.config, args.scale)
     bf16 = w.dtype == "bf16"
 
     # CPU baseline first (before the first GPU call), rank 0 of a single-GPU run only
@@ -385,7 +385,7 @@ def run_reference(args):
     rank = int(os.environ.get("RANK", "0"))
     if rank != 0:
         return
-    w = si.make_workload(args.config)
+    w = si.make_workload(args.config, args.scale)
     threads = _host_threads()
     book, parts, items, edges, t_book = _oracle_sample(w, ORACLE_SAMPLE_PARTS[args.config])
     for _ in range(args.warmup):
@@ -412,6 +412,8 @@ def main():
     ap.add_argument("--steps", type=int, default=5)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--config", type=int, default=5, choices=[1, 2, 3, 4, 5])
+    ap.add_argument("--scale", type=float, default=1.0,
+                    help="shrink configuration 4 or 5 (nodes, edges, subgraphs) for profiler captures")
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
