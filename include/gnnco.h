@@ -200,6 +200,34 @@ int32_t gnnco_train_step_host(gnnco_handle* h, const gnnco_model_desc* m, const 
 int32_t gnnco_decode_boundary(const gnnco_handle* h, const float* p, float threshold, uint8_t* x, uint8_t* viol,
                               int32_t* per_part, gnnco_counts* counts, void* stream);
 
+/* Objective only, for callers that cannot allocate device memory.  (The paper has no
+ * counterpart to this call; it exists for the way the library is embedded.)
+ *
+ * Some users of this library run where no allocation is possible at the moment they need a
+ * loss value: a coordination loop living inside another program's callback or plug-in
+ * interface is handed `p` and a place for `loss` and nothing else -- it owns no allocator, the
+ * host program's memory pool is not its to grow, and a cudaMalloc there would stall every
+ * stream of the process.  gnnco_train_step cannot serve them, because it needs a work area.
+ * This entry point evaluates the per-subgraph objective of gnnco_objective for GIVEN
+ * probabilities `p` [n] (new node order) and writes loss [S]; it allocates nothing and takes
+ * no work area.  Its only scratch, one float per objective work item, is a fixed array of
+ * GNNCO_STATIC_OBJECTIVE_MAX_ITEMS floats (256 KiB) inside the library image, which every
+ * GPU that loads the library holds until the process exits.
+ *
+ *  - A graph needs  sum_s ceil(|V_s| / 1024)  work items; if that exceeds the maximum the call
+ *    returns GNNCO_WORKSPACE_TOO_SMALL and does nothing.
+ *  - The first call on a device looks up the array's device address (once per device, with
+ *    that device current); make that first call outside any stream capture.
+ *  - All calls share the one array and it keeps what the last call left: the part a call
+ *    uses is cleared and rewritten by that call, but two calls that overlap on the GPU
+ *    (different streams, or another thread) race on it.  Serialise them.
+ *  - The handle's device must be current.  Asynchronous on `stream`; results equal those of
+ *    gnnco_train_step's loss for the same p.
+ */
+#define GNNCO_STATIC_OBJECTIVE_MAX_ITEMS 65536
+int32_t gnnco_objective_static(gnnco_handle* h, const float* p, const gnnco_objective* obj, float* loss,
+                               void* stream);
+
 /* Host read of the device-side status word (synchronises `stream`). */
 int32_t gnnco_async_status(const gnnco_handle* h, void* stream, int32_t* status);
 

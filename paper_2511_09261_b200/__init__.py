@@ -25,7 +25,7 @@ EXPORTS = [
     "gnnco_status_string", "gnnco_partition_workspace_bytes", "gnnco_partition_load", "gnnco_graph_info",
     "gnnco_gather_rows", "gnnco_train_workspace_bytes", "gnnco_train_step", "gnnco_train_host_workspace_bytes",
     "gnnco_train_step_host", "gnnco_decode_boundary", "gnnco_async_status", "gnnco_launch_count", "gnnco_destroy",
-    "gnnco_profile_begin", "gnnco_profile_end",
+    "gnnco_profile_begin", "gnnco_profile_end", "gnnco_objective_static",
 ]
 
 _vp, _i32, _i64, _u32, _f32, _sz = (ctypes.c_void_p, ctypes.c_int32, ctypes.c_int64, ctypes.c_uint32, ctypes.c_float,
@@ -105,6 +105,7 @@ def load_library(build_if_missing: bool = True):
     lib.gnnco_launch_count.argtypes = [_vp]
     lib.gnnco_launch_count.restype = _i64
     lib.gnnco_destroy.argtypes = [_vp]
+    lib.gnnco_objective_static.argtypes = [_vp, _vp, ctypes.POINTER(Objective), _vp, _vp]
     lib.gnnco_profile_begin.argtypes = [_vp]
     lib.gnnco_profile_end.argtypes = [_vp, _vp, ctypes.POINTER(ProfileEntry), _i32, ctypes.POINTER(_i32)]
     for name in EXPORTS:
@@ -345,6 +346,19 @@ class PartitionedGraph:
                                              _dptr(per_part), counts.data_ptr(), _stream_ptr(stream))
         _check(st, "gnnco_decode_boundary")
         return dict(x=x, viol=viol, per_part=per_part, counts=counts)
+
+    def objective_static(self, p, alpha: float, beta: float, lam: float = 0.0, pen=None, loss=None, stream=None):
+        """``gnnco_objective_static``: per-subgraph objective of given probabilities, with no
+        work area and no allocation inside the library (``loss`` must be passed by callers
+        that cannot allocate; it is created here only as a convenience)."""
+        import torch
+        _require(p, torch.float32, "p")
+        if loss is None:
+            loss = torch.empty(self.S, dtype=torch.float32, device=self.device)
+        obj = Objective(alpha, beta, lam, _dptr(pen))
+        _check(self._lib.gnnco_objective_static(self._handle, p.data_ptr(), ctypes.byref(obj), loss.data_ptr(),
+                                                _stream_ptr(stream)), "gnnco_objective_static")
+        return loss
 
     def async_status(self, stream=None) -> int:
         s = _i32(0)

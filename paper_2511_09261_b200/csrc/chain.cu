@@ -142,3 +142,55 @@ int32_t launch_output_backward(gnnco_handle* h, const float* t, float* g, cudaSt
   GNNCO_LAUNCH_CHECK();
   return GNNCO_OK;
 }
+
+// ------------------------------------------------------------------------------------
+// Objective evaluation for callers that cannot allocate device memory (see gnnco.h).
+// The per-item partial sums, which launch_objective keeps in the caller's work area, live
+// here in a fixed device array that is part of the library image.
+namespace {
+
+static __device__ __align__(256) float g_static_item_loss[GNNCO_STATIC_OBJECTIVE_MAX_ITEMS];
+
+constexpr int kMaxDevices = 64;
+float* g_static_item_loss_addr[kMaxDevices] = {nullptr};   // device address of the array, per device
+
+// In host code the array's name is only a handle for the runtime, not a device address; the
+// address a kernel can use has to be asked for, once per device, with that device current.
+int32_t static_item_loss_address(float** out) {
+  int dev = -1;
+  GNNCO_CUDA_TRY(cudaGetDevice(&dev));
+  if (dev < 0 || dev >= kMaxDevices) return GNNCO_UNSUPPORTED;
+  if (!g_static_item_loss_addr[dev]) {
+    void* ptr = nullptr;
+    GNNCO_CUDA_TRY(cudaGetSymbolAddress(&ptr, g_static_item_loss));
+    if (!ptr) return GNNCO_CUDA_ERROR;
+    g_static_item_loss_addr[dev] = static_cast<float*>(ptr);
+  }
+  *out = g_static_item_loss_addr[dev];
+  return GNNCO_OK;
+}
+
+}  // namespace
+
+extern "C" int32_t gnnco_objective_static(gnnco_handle* h, const float* p, const gnnco_objective* obj, float* loss,
+                                         void* stream) {
+  if (!h || !p || !obj || !loss) return GNNCO_INVALID_ARGUMENT;
+  if (h->n_items > GNNCO_STATIC_OBJECTIVE_MAX_ITEMS) return GNNCO_WORKSPACE_TOO_SMALL;
+  int dev = -1;
+  GNNCO_CUDA_TRY(cudaGetDevice(&dev));
+  if (dev != h->device) return GNNCO_INVALID_ARGUMENT;
+  float* item_loss = nullptr;
+  int32_t rc = static_item_loss_address(&item_loss);
+  if (rc != GNNCO_OK) return rc;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  // every slot that is read below is written first by objective_items; the clear only makes
+  // sure nothing of an earlier call can be mistaken for a result
+  if (h->n_items > 0) GNNCO_CUDA_TRY(cudaMemsetAsync(item_loss, 0, (size_t)h->n_items * sizeof(float), st));
+  if (h->n_items > 0)
+    objective_items<<<h->n_items, 256, 0, st>>>(p, obj->pen, h->rowptr, h->colidx, h->inv_deg, h->item_row0,
+                                                h->item_row1, obj->alpha, obj->beta, obj->lambda, item_loss, nullptr);
+  sum_items_per_subgraph<<<(h->S + 255) / 256, 256, 0, st>>>(item_loss, h->part_item_ptr, loss, h->S);
+  h->launches += 2;
+  GNNCO_LAUNCH_CHECK();
+  return GNNCO_OK;
+}
