@@ -50,7 +50,7 @@ struct Profiler {
 struct gnnco_handle {
   int64_t n = 0, E = 0, E_in = 0, E_b = 0;
   int32_t S = 0, max_row = 0;
-  int device = 0;
+  int device = 0, sm_count = 0;
   // device arrays inside the caller's persistent work area
   int32_t *perm = nullptr, *inv_perm = nullptr, *part_ptr = nullptr, *node_part = nullptr;
   int32_t *rowptr = nullptr, *colidx = nullptr, *bnd_u = nullptr, *bnd_v = nullptr;
@@ -126,6 +126,15 @@ int32_t launch_sum_over_sets(gnnco_handle* h, const float* in, float* out, int64
 int32_t launch_cast_bf16(gnnco_handle* h, const float* in, __nv_bfloat16* out, int64_t count, cudaStream_t st);
 int32_t launch_adam(gnnco_handle* h, float* W, float* m, float* v, const float* g, int64_t count, float lr, float b1,
                     float b2, float eps, float c1, float c2, cudaStream_t st);
+
+// ---- tc_gemm.cu : the same transform on the tensor cores (bf16, widths 64/128/256)
+bool tc_transform_supported(int dtype, int K, int N);
+// Y = act(A B_s^T) * row_scale with A [n x K] and B [sets x N x K], K contiguous in both
+int32_t launch_transform_tc(gnnco_handle* h, const void* A, const void* B, int64_t b_stride, void* Y, int K, int N,
+                            bool relu, const float* row_scale, bool backward, cudaStream_t st);
+// Wt[s][n][k] = bf16(W[s][k][n])
+int32_t launch_cast_transpose_bf16(gnnco_handle* h, const float* W, __nv_bfloat16* Wt, int K, int N, int32_t sets,
+                                   cudaStream_t st);
 
 // ---- chain.cu : the width-1 part of the step
 int32_t launch_output_forward(gnnco_handle* h, const float* u, float* z, float* p, cudaStream_t st);

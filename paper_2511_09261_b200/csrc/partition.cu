@@ -391,6 +391,7 @@ extern "C" int32_t gnnco_partition_load(const gnnco_graph_desc* g, void* persist
     ~Guard() { delete h; }
   } guard{h};
   GNNCO_CUDA_TRY(cudaGetDevice(&h->device));
+  GNNCO_CUDA_TRY(cudaDeviceGetAttribute(&h->sm_count, cudaDevAttrMultiProcessorCount, h->device));
   h->n = n; h->E = E; h->S = S;
   h->perm = P.perm; h->inv_perm = P.inv_perm; h->node_part = P.node_part; h->part_ptr = P.part_ptr;
   h->rowptr = P.rowptr; h->colidx = P.colidx; h->bnd_u = P.bnd_u; h->bnd_v = P.bnd_v;

@@ -1,0 +1,219 @@
+// Dense per-subgraph transform on the sm_100a tensor cores (tcgen05 + TMEM), bf16 operands
+// with float32 accumulation (Eq. 3's "... W" and its input gradient).
+//
+//   Y[tile, :] = act( A[tile, 0:K] * B_s^T ) * row_scale,    B_s = [N x K], K contiguous
+//
+// Forward uses B = W^T (bf16 copy, transposed), the input gradient uses B = W (bf16 copy), so
+// both operands are K-major.  One CTA owns a run of consecutive 128-row tiles; consecutive
+// tiles mostly belong to the same subgraph, so its weight matrix stays in shared memory.
+// Operands are staged with 16-byte cp.async copies into the 128-byte-swizzled layout the
+// tensor core expects; one thread issues the MMAs, the accumulator (128 lanes x N columns of
+// TMEM) is read back by all eight warps, scaled / rectified, rounded to bf16 and stored.
+// The copies of the next tile are in flight while the current accumulator is drained.
+#include "internal.cuh"
+#include "tc_common.cuh"
+
+namespace {
+
+constexpr int kTileM = 128;
+constexpr int kThreads = 256;
+
+// Copy `rows_valid` rows (of `rows_total`) x KDIM bf16 from global (row stride KDIM) into
+// K-major SW128 shared memory: k-block kb at kb*rows_total*128, row r at (r/8)*1024 + (r%8)*128,
+// 16-byte chunk c at ((c ^ (r%8)) * 16).  Rows past rows_valid are zero-filled.
+template <int KDIM>
+__device__ __forceinline__ void stage_k_major(uint32_t sbase, const __nv_bfloat16* __restrict__ g, int rows_total,
+                                              int rows_valid) {
+  constexpr int CPR = KDIM / 8;                 // 16-byte chunks per row
+  const int total = rows_total * CPR;
+  for (int q = threadIdx.x; q < total; q += kThreads) {
+    const int r = q / CPR, c = q % CPR;
+    const int kb = c >> 3, cc = c & 7;
+    const uint32_t dst = sbase + kb * (rows_total * 128) + (r >> 3) * 1024 + (r & 7) * 128 + ((cc ^ (r & 7)) << 4);
+    if (r < rows_valid) tc::cp_async16(dst, g + (int64_t)r * KDIM + c * 8);
+    else tc::st_shared_zero16(dst);
+  }
+}
+
+template <int KDIM, int NDIM>
+__global__ void __launch_bounds__(kThreads, 1)
+transform_tc(const __nv_bfloat16* __restrict__ A, const __nv_bfloat16* __restrict__ B, int64_t b_stride,
+             __nv_bfloat16* __restrict__ Y, int relu, const float* __restrict__ row_scale,
+             const int32_t* __restrict__ tile_row0, const int32_t* __restrict__ tile_rows,
+             const int32_t* __restrict__ node_part, int n_tiles, int tiles_per_cta, int32_t* status) {
+  constexpr int KB = KDIM / 64;
+  constexpr uint32_t A_BYTES = KB * kTileM * 128;
+  constexpr uint32_t B_BYTES = KB * NDIM * 128;
+  extern __shared__ uint8_t smem_raw[];
+  const uint32_t sbase = (tc::smem_u32(smem_raw) + 1023u) & ~1023u;
+  const uint32_t sA = sbase, sB = sbase + A_BYTES;
+  uint8_t* gen_base = smem_raw + (sbase - tc::smem_u32(smem_raw));
+  uint64_t* bar = reinterpret_cast<uint64_t*>(gen_base + A_BYTES + B_BYTES);
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(gen_base + A_BYTES + B_BYTES + 8);
+  uint32_t* abort_flag = tmem_slot + 1;
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int t_begin = blockIdx.x * tiles_per_cta;
+  const int t_end = min(n_tiles, t_begin + tiles_per_cta);
+  if (t_begin >= t_end) return;
+
+  if (threadIdx.x == 0) {
+    tc::mbar_init(bar, 1);
+    *abort_flag = 0;
+    tc::fence_mbar_init();
+  }
+  if (warp == 0) tc::tmem_alloc(tmem_slot, NDIM);
+  tc::tc_fence_before_sync();
+  __syncthreads();
+  tc::tc_fence_after_sync();
+  const uint32_t tmem = *tmem_slot;
+  constexpr uint32_t IDESC = tc::idesc_bf16_f32(kTileM, NDIM, false, false);
+
+  int cur_part = -1;
+  uint32_t phase = 0;
+  // prologue: operands of the first tile
+  {
+    const int64_t row0 = tile_row0[t_begin];
+    cur_part = node_part[row0];
+    stage_k_major<KDIM>(sB, B + (int64_t)cur_part * b_stride, NDIM, NDIM);
+    stage_k_major<KDIM>(sA, A + row0 * KDIM, kTileM, tile_rows[t_begin]);
+    tc::cp_async_commit();
+  }
+  for (int t = t_begin; t < t_end; ++t) {
+    const int64_t row0 = tile_row0[t];
+    const int rows = tile_rows[t];
+    tc::cp_async_wait<0>();
+    tc::fence_proxy_async_smem();
+    __syncthreads();
+    if (threadIdx.x == 0) {
+      tc::tc_fence_after_sync();
+#pragma unroll
+      for (int kb = 0; kb < KB; ++kb)
+#pragma unroll
+        for (int ks = 0; ks < 4; ++ks) {
+          const uint64_t ad = tc::smem_desc_sw128(sA + kb * (kTileM * 128) + ks * 32, 16, 1024);
+          const uint64_t bd = tc::smem_desc_sw128(sB + kb * (NDIM * 128) + ks * 32, 16, 1024);
+          tc::mma_bf16(tmem, ad, bd, IDESC, (kb | ks) != 0);
+        }
+      tc::mma_commit(bar);
+    }
+    if (!tc::mbar_wait_bounded(bar, phase)) *abort_flag = 1;
+    phase ^= 1;
+    __syncthreads();
+    if (*abort_flag) {
+      if (threadIdx.x == 0) atomicMin(status, (int32_t)GNNCO_INTERNAL);
+      break;
+    }
+    tc::tc_fence_after_sync();
+    // operands are consumed: start the next tile's copies, they fly during the drain below
+    if (t + 1 < t_end) {
+      const int64_t nrow0 = tile_row0[t + 1];
+      const int npart = node_part[nrow0];
+      if (npart != cur_part) {
+        cur_part = npart;
+        stage_k_major<KDIM>(sB, B + (int64_t)cur_part * b_stride, NDIM, NDIM);
+      }
+      stage_k_major<KDIM>(sA, A + nrow0 * KDIM, kTileM, tile_rows[t + 1]);
+      tc::cp_async_commit();
+    }
+    // drain the accumulator: warp w reads lanes 32*(w%4).., columns half (w/4)
+    {
+      const int lg = warp & 3, ch = warp >> 2;
+      const int row = lg * 32 + lane;
+      const float s = (row_scale && row < rows) ? row_scale[row0 + row] : 1.0f;
+      constexpr int HALF = NDIM / 2;
+#pragma unroll
+      for (int c0 = 0; c0 < HALF; c0 += 32) {
+        uint32_t r[32];
+        tc::tmem_ld_32x32(tmem + ((uint32_t)(lg * 32) << 16) + ch * HALF + c0, r);
+        tc::tmem_ld_wait();
+        if (row < rows) {
+          uint4 out[4];
+          uint32_t* o = reinterpret_cast<uint32_t*>(out);
+#pragma unroll
+          for (int j = 0; j < 16; ++j) {
+            float a = __uint_as_float(r[2 * j]) * s, b = __uint_as_float(r[2 * j + 1]) * s;
+            if (relu) { a = a > 0.0f ? a : 0.0f; b = b > 0.0f ? b : 0.0f; }
+            __nv_bfloat162 v = __floats2bfloat162_rn(a, b);
+            o[j] = *reinterpret_cast<uint32_t*>(&v);
+          }
+          uint4* dst = reinterpret_cast<uint4*>(Y + (row0 + row) * NDIM + ch * HALF + c0);
+#pragma unroll
+          for (int j = 0; j < 4; ++j) dst[j] = out[j];
+        }
+      }
+    }
+    tc::tc_fence_before_sync();   // the next tile's MMA overwrites the accumulator after the sync at the loop top
+  }
+  tc::cp_async_wait<0>();
+  tc::tc_fence_before_sync();
+  __syncthreads();
+  if (warp == 0) tc::tmem_dealloc(tmem, NDIM);
+}
+
+template <int KDIM, int NDIM>
+int32_t launch_tc(gnnco_handle* h, const void* A, const void* B, int64_t b_stride, void* Y, bool relu,
+                  const float* row_scale, cudaStream_t st) {
+  constexpr int KB = KDIM / 64;
+  constexpr size_t smem = (size_t)KB * (kTileM + NDIM) * 128 + 64 + 1024;
+  GNNCO_CUDA_TRY(cudaFuncSetAttribute(transform_tc<KDIM, NDIM>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                      (int)smem));
+  int sms = h->sm_count > 0 ? h->sm_count : 148;
+  int grid = h->n_tiles < sms ? h->n_tiles : sms;
+  int per = (h->n_tiles + grid - 1) / grid;
+  grid = (h->n_tiles + per - 1) / per;
+  transform_tc<KDIM, NDIM><<<grid, kThreads, smem, st>>>(
+      (const __nv_bfloat16*)A, (const __nv_bfloat16*)B, b_stride, (__nv_bfloat16*)Y, relu ? 1 : 0, row_scale,
+      h->tile_row0, h->tile_rows, h->node_part, h->n_tiles, per, h->status);
+  h->launches += 1;
+  GNNCO_LAUNCH_CHECK();
+  return GNNCO_OK;
+}
+
+// W [sets][K][N] float32 -> Wt [sets][N][K] bf16
+__global__ void cast_transpose_bf16_kernel(const float* __restrict__ W, __nv_bfloat16* __restrict__ Wt, int K, int N) {
+  __shared__ float tile[32][33];
+  const int64_t base = (int64_t)blockIdx.z * K * N;
+  const int k0 = blockIdx.y * 32, n0 = blockIdx.x * 32;
+  for (int j = threadIdx.y; j < 32; j += 8) {
+    int k = k0 + j, n = n0 + threadIdx.x;
+    tile[j][threadIdx.x] = (k < K && n < N) ? W[base + (int64_t)k * N + n] : 0.0f;
+  }
+  __syncthreads();
+  for (int j = threadIdx.y; j < 32; j += 8) {
+    int n = n0 + j, k = k0 + threadIdx.x;
+    if (n < N && k < K) Wt[base + (int64_t)n * K + k] = __float2bfloat16_rn(tile[threadIdx.x][j]);
+  }
+}
+
+}  // namespace
+
+bool tc_transform_supported(int dtype, int K, int N) {
+  auto ok = [](int d) { return d == 64 || d == 128 || d == 256; };
+  return dtype == GNNCO_BF16 && ok(K) && ok(N);
+}
+
+// Y = act(A B_s^T) * row_scale with A [n x K], B [sets x N x K] (both bf16, K contiguous).
+int32_t launch_transform_tc(gnnco_handle* h, const void* A, const void* B, int64_t b_stride, void* Y, int K, int N,
+                            bool relu, const float* row_scale, bool backward, cudaStream_t st) {
+  if (h->n_tiles == 0) return GNNCO_OK;
+  ProfScope prof_(h, backward ? K_TRANSFORM_BWD : K_TRANSFORM_FWD, st);
+#define GNNCO_TC_CASE(KK, NN) \
+  if (K == KK && N == NN) return launch_tc<KK, NN>(h, A, B, b_stride, Y, relu, row_scale, st)
+  GNNCO_TC_CASE(64, 64); GNNCO_TC_CASE(64, 128); GNNCO_TC_CASE(64, 256);
+  GNNCO_TC_CASE(128, 64); GNNCO_TC_CASE(128, 128); GNNCO_TC_CASE(128, 256);
+  GNNCO_TC_CASE(256, 64); GNNCO_TC_CASE(256, 128); GNNCO_TC_CASE(256, 256);
+#undef GNNCO_TC_CASE
+  return GNNCO_UNSUPPORTED;
+}
+
+int32_t launch_cast_transpose_bf16(gnnco_handle* h, const float* W, __nv_bfloat16* Wt, int K, int N, int32_t sets,
+                                   cudaStream_t st) {
+  ProfScope prof_(h, K_CAST, st);
+  dim3 grid((N + 31) / 32, (K + 31) / 32, sets);
+  if (grid.y > 65535 || grid.z > 65535) return GNNCO_UNSUPPORTED;
+  cast_transpose_bf16_kernel<<<grid, dim3(32, 8), 0, st>>>(W, Wt, K, N);
+  h->launches += 1;
+  GNNCO_LAUNCH_CHECK();
+  return GNNCO_OK;
+}

@@ -27,6 +27,7 @@ struct TrainLayout {
   float* dW_scratch;                  // one layer's gradient (all sets), when the caller wants none
   float* dW_sets;                     // per-subgraph partials when the model shares one weight set
   __nv_bfloat16* W_lp[GNNCO_MAX_LAYERS];   // bf16 copies of the weights (bf16 features only)
+  __nv_bfloat16* W_lp_t[GNNCO_MAX_LAYERS]; // transposed bf16 copies [sets x F_out x F_in] for the tensor-core forward
   // host-variant staging
   void* X_stage;
   float *pen_stage, *loss_stage, *p_stage;
@@ -82,6 +83,9 @@ TrainLayout carve_train(const gnnco_handle* h, const gnnco_model_desc* m, uint32
   if (m->feat_dtype == GNNCO_BF16)
     for (int l = 0; l < L; ++l)
       T.W_lp[l] = c.take<__nv_bfloat16>((size_t)m->dims[l] * m->dims[l + 1] * m->weight_sets);
+  for (int l = 0; l + 1 < L; ++l)
+    if (tc_transform_supported(m->feat_dtype, m->dims[l], m->dims[l + 1]))
+      T.W_lp_t[l] = c.take<__nv_bfloat16>((size_t)m->dims[l] * m->dims[l + 1] * m->weight_sets);
   if (host) {
     T.X_stage = c.take<char>(n * m->dims[0] * es);
     T.pen_stage = c.take<float>(n);
@@ -109,6 +113,8 @@ int32_t run_step(gnnco_handle* h, const gnnco_model_desc* m, const void* X, cons
     if (bf16) {
       GNNCO_TRY(launch_cast_bf16(h, m->W[l], T.W_lp[l], wc * sets, st));
       Wc[l] = T.W_lp[l];
+      if (T.W_lp_t[l])
+        GNNCO_TRY(launch_cast_transpose_bf16(h, m->W[l], T.W_lp_t[l], m->dims[l], m->dims[l + 1], sets, st));
     } else {
       Wc[l] = m->W[l];
     }
@@ -117,8 +123,12 @@ int32_t run_step(gnnco_handle* h, const gnnco_model_desc* m, const void* X, cons
   const void* Hprev = X;
   for (int l = 1; l < L; ++l) {
     GNNCO_TRY(launch_aggregate(h, dt, Hprev, T.M[l], m->dims[l - 1], h->inv_deg, nullptr, st));
-    GNNCO_TRY(launch_transform(h, dt, T.M[l], Wc[l - 1], wstride[l - 1], T.H[l], m->dims[l - 1], m->dims[l], false,
-                               true, nullptr, st));
+    if (T.W_lp_t[l - 1])
+      GNNCO_TRY(launch_transform_tc(h, T.M[l], T.W_lp_t[l - 1], wstride[l - 1], T.H[l], m->dims[l - 1], m->dims[l], true,
+                                    nullptr, false, st));
+    else
+      GNNCO_TRY(launch_transform(h, dt, T.M[l], Wc[l - 1], wstride[l - 1], T.H[l], m->dims[l - 1], m->dims[l], false,
+                                 true, nullptr, st));
     Hprev = T.H[l];
   }
   const int FL = m->dims[L - 1];
@@ -165,8 +175,12 @@ int32_t run_step(gnnco_handle* h, const gnnco_model_desc* m, const void* X, cons
     // hidden layer l uses weight index l-1: widths d_{l-1} -> d_l
     const int K = m->dims[l - 1], N = m->dims[l];
     const bool need_input_grad = (l > 1) || (flags & GNNCO_WANT_DX);
-    if (need_input_grad)
-      GNNCO_TRY(launch_transform(h, dt, dZ, Wc[l - 1], wstride[l - 1], other, N, K, true, false, h->inv_deg, st));
+    if (need_input_grad) {
+      if (tc_transform_supported(dt, N, K))
+        GNNCO_TRY(launch_transform_tc(h, dZ, Wc[l - 1], wstride[l - 1], other, N, K, false, h->inv_deg, true, st));
+      else
+        GNNCO_TRY(launch_transform(h, dt, dZ, Wc[l - 1], wstride[l - 1], other, N, K, true, false, h->inv_deg, st));
+    }
     float* target = grad_target(l - 1);
     if (sets == 1) {
       GNNCO_TRY(launch_weight_grad(h, dt, T.M[l], dZ, T.dW_sets, K, N, st));

@@ -108,7 +108,9 @@ def test_train_step_small_f32(name, dims, sets, lam):
 
 
 @pytest.mark.parametrize("dims,sets", [([16, 8, 1], None), ([64, 32, 16, 1], None), ([256, 256, 1], None),
-                                       ([32, 16, 1], 1), ([6, 1], None)])
+                                       ([32, 16, 1], 1), ([6, 1], None), ([128, 64, 1], None),
+                                       ([64, 256, 128, 1], None), ([256, 256, 256, 1], None), ([128, 128, 1], 1),
+                                       ([64, 64, 64, 1], None)])
 def test_train_step_small_bf16(dims, sets):
     eu, ev, part = tiny_graph(260, 0.05, 5, seed=9)
     n, S = _n_S(part)
