@@ -132,6 +132,8 @@ bool tc_transform_supported(int dtype, int K, int N);
 // Y = act(A B_s^T) * row_scale with A [n x K] and B [sets x N x K], K contiguous in both
 int32_t launch_transform_tc(gnnco_handle* h, const void* A, const void* B, int64_t b_stride, void* Y, int K, int N,
                             bool relu, const float* row_scale, bool backward, cudaStream_t st);
+bool tc_weight_grad_supported(int dtype, int K, int N);
+int32_t launch_weight_grad_tc(gnnco_handle* h, const void* A, const void* G, float* dW, int K, int N, cudaStream_t st);
 // Wt[s][n][k] = bf16(W[s][k][n])
 int32_t launch_cast_transpose_bf16(gnnco_handle* h, const float* W, __nv_bfloat16* Wt, int K, int N, int32_t sets,
                                    cudaStream_t st);

@@ -170,6 +170,147 @@ int32_t launch_tc(gnnco_handle* h, const void* A, const void* B, int64_t b_strid
   return GNNCO_OK;
 }
 
+// ------------------------------------------------------------------------------------
+// Weight gradient on the tensor cores:  dW_s[KF x NF] = sum_{i in s} A[i, :]^T G[i, :]
+// (the reduction runs over the rows of subgraph s, so both operands are MN-major: a row of
+// A or G is 128-byte lines of 64 features, indexed by the reduction index).
+// One CTA per subgraph; rows stream through a 3-stage cp.async pipeline in chunks of 64;
+// the KF x NF accumulator lives in TMEM (two 128-lane halves when KF = 256) and is written
+// out in float32 once at the end, in a fixed order (deterministic, no atomics).
+constexpr int kWgRows = 64;      // reduction rows per pipeline stage
+constexpr int kWgStages = 3;
+
+// rows [r0, r0+64) of a [.. x DIM] bf16 matrix -> MN-major SW128 stage: feature block mb
+// (64 features) at mb*8192, row k at (k/8)*1024 + (k%8)*128, chunk c at ((c ^ (k%8)) * 16)
+template <int DIM>
+__device__ __forceinline__ void stage_mn_major(uint32_t sbase, const __nv_bfloat16* __restrict__ g, int64_t r0,
+                                               int64_t r_end) {
+  constexpr int CPR = DIM / 8;
+  constexpr int total = kWgRows * CPR;
+  for (int q = threadIdx.x; q < total; q += kThreads) {
+    const int k = q / CPR, c = q % CPR;
+    const int mb = c >> 3, cc = c & 7;
+    const uint32_t dst = sbase + mb * (kWgRows * 128) + (k >> 3) * 1024 + (k & 7) * 128 + ((cc ^ (k & 7)) << 4);
+    if (r0 + k < r_end) tc::cp_async16(dst, g + (r0 + k) * DIM + c * 8);
+    else tc::st_shared_zero16(dst);
+  }
+}
+
+template <int KF, int NF>
+__global__ void __launch_bounds__(kThreads, 1)
+weight_grad_tc(const __nv_bfloat16* __restrict__ A, const __nv_bfloat16* __restrict__ G, float* __restrict__ dW,
+               const int32_t* __restrict__ part_ptr, int32_t* status) {
+  constexpr int MH = KF / 128;                          // accumulator halves of 128 rows
+  constexpr uint32_t A_STAGE = KF * 128, G_STAGE = NF * 128;
+  constexpr uint32_t STAGE = A_STAGE + G_STAGE;
+  constexpr uint32_t TMEM_COLS = MH * NF < 32 ? 32 : MH * NF;
+  extern __shared__ uint8_t smem_raw[];
+  const uint32_t sbase = (tc::smem_u32(smem_raw) + 1023u) & ~1023u;
+  uint8_t* gen_base = smem_raw + (sbase - tc::smem_u32(smem_raw));
+  uint64_t* bars = reinterpret_cast<uint64_t*>(gen_base + kWgStages * STAGE);      // [stages] consumed, [stages] = all done
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + kWgStages + 1);
+  uint32_t* abort_flag = tmem_slot + 1;
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int s = blockIdx.x;
+  const int64_t ra = part_ptr[s], rb = part_ptr[s + 1];
+  float* out = dW + (int64_t)s * KF * NF;
+  const int iters = (int)((rb - ra + kWgRows - 1) / kWgRows);
+  if (iters == 0) {
+    for (int q = threadIdx.x; q < KF * NF; q += kThreads) out[q] = 0.0f;
+    return;
+  }
+  if (threadIdx.x == 0) {
+    for (int i = 0; i <= kWgStages; ++i) tc::mbar_init(bars + i, 1);
+    *abort_flag = 0;
+    tc::fence_mbar_init();
+  }
+  if (warp == 0) tc::tmem_alloc(tmem_slot, TMEM_COLS);
+  tc::tc_fence_before_sync();
+  __syncthreads();
+  tc::tc_fence_after_sync();
+  const uint32_t tmem = *tmem_slot;
+  constexpr uint32_t IDESC = tc::idesc_bf16_f32(128, NF, true, true);
+
+  auto load_stage = [&](int it) {
+    if (it < iters) {
+      const uint32_t sb = sbase + (it % kWgStages) * STAGE;
+      stage_mn_major<KF>(sb, A, ra + (int64_t)it * kWgRows, rb);
+      stage_mn_major<NF>(sb + A_STAGE, G, ra + (int64_t)it * kWgRows, rb);
+    }
+    tc::cp_async_commit();            // always commit: keeps the group count uniform
+  };
+  for (int it = 0; it < kWgStages - 1; ++it) load_stage(it);
+  bool failed = false;
+  for (int it = 0; it < iters; ++it) {
+    tc::cp_async_wait<kWgStages - 2>();
+    tc::fence_proxy_async_smem();
+    __syncthreads();
+    if (threadIdx.x == 0) {
+      tc::tc_fence_after_sync();
+      const uint32_t sb = sbase + (it % kWgStages) * STAGE;
+#pragma unroll
+      for (int j = 0; j < kWgRows / 16; ++j) {
+        const uint64_t gd = tc::smem_desc_sw128(sb + A_STAGE + j * 2048, kWgRows * 128, 1024);
+#pragma unroll
+        for (int hm = 0; hm < MH; ++hm) {
+          const uint64_t ad = tc::smem_desc_sw128(sb + hm * 2 * (kWgRows * 128) + j * 2048, kWgRows * 128, 1024);
+          tc::mma_bf16(tmem + hm * NF, ad, gd, IDESC, (it | j) != 0);
+        }
+      }
+      tc::mma_commit(bars + (it % kWgStages));
+      if (it == iters - 1) tc::mma_commit(bars + kWgStages);
+    }
+    // the slot that iteration it-1 used is free once its MMAs have completed; refill it
+    if (it >= 1) {
+      const int prev = it - 1;
+      if (!tc::mbar_wait_bounded(bars + (prev % kWgStages), (prev / kWgStages) & 1)) *abort_flag = 1;
+    }
+    __syncthreads();
+    if (*abort_flag) { failed = true; break; }
+    load_stage(it + kWgStages - 1);
+  }
+  if (!failed) {
+    if (!tc::mbar_wait_bounded(bars + kWgStages, 0)) *abort_flag = 1;
+    __syncthreads();
+    failed = *abort_flag != 0;
+  }
+  tc::cp_async_wait<0>();
+  if (failed) {
+    if (threadIdx.x == 0) atomicMin(status, (int32_t)GNNCO_INTERNAL);
+  } else {
+    tc::tc_fence_after_sync();
+    const int lg = warp & 3, ch = warp >> 2;
+    constexpr int HALF = NF / 2;
+#pragma unroll
+    for (int hm = 0; hm < MH; ++hm) {
+      const int f = hm * 128 + lg * 32 + lane;
+#pragma unroll
+      for (int c0 = 0; c0 < HALF; c0 += 32) {
+        uint32_t r[32];
+        tc::tmem_ld_32x32(tmem + ((uint32_t)(lg * 32) << 16) + hm * NF + ch * HALF + c0, r);
+        tc::tmem_ld_wait();
+        uint4* dst = reinterpret_cast<uint4*>(out + (int64_t)f * NF + ch * HALF + c0);
+#pragma unroll
+        for (int j = 0; j < 8; ++j) dst[j] = make_uint4(r[4 * j], r[4 * j + 1], r[4 * j + 2], r[4 * j + 3]);
+      }
+    }
+  }
+  tc::tc_fence_before_sync();
+  __syncthreads();
+  if (warp == 0) tc::tmem_dealloc(tmem, TMEM_COLS);
+}
+
+template <int KF, int NF>
+int32_t launch_wg(gnnco_handle* h, const void* A, const void* G, float* dW, cudaStream_t st) {
+  constexpr size_t smem = (size_t)kWgStages * (KF + NF) * 128 + 128 + 1024;
+  GNNCO_CUDA_TRY(cudaFuncSetAttribute(weight_grad_tc<KF, NF>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+  weight_grad_tc<KF, NF><<<h->S, kThreads, smem, st>>>((const __nv_bfloat16*)A, (const __nv_bfloat16*)G, dW,
+                                                       h->part_ptr, h->status);
+  h->launches += 1;
+  GNNCO_LAUNCH_CHECK();
+  return GNNCO_OK;
+}
+
 // W [sets][K][N] float32 -> Wt [sets][N][K] bf16
 __global__ void cast_transpose_bf16_kernel(const float* __restrict__ W, __nv_bfloat16* __restrict__ Wt, int K, int N) {
   __shared__ float tile[32][33];
@@ -204,6 +345,21 @@ int32_t launch_transform_tc(gnnco_handle* h, const void* A, const void* B, int64
   GNNCO_TC_CASE(128, 64); GNNCO_TC_CASE(128, 128); GNNCO_TC_CASE(128, 256);
   GNNCO_TC_CASE(256, 64); GNNCO_TC_CASE(256, 128); GNNCO_TC_CASE(256, 256);
 #undef GNNCO_TC_CASE
+  return GNNCO_UNSUPPORTED;
+}
+
+bool tc_weight_grad_supported(int dtype, int K, int N) {
+  return dtype == GNNCO_BF16 && (K == 128 || K == 256) && (N == 64 || N == 128 || N == 256);
+}
+
+// dW[s] (K x N, float32) = sum_{i in s} A[i,:]^T G[i,:], A [n x K], G [n x N] bf16
+int32_t launch_weight_grad_tc(gnnco_handle* h, const void* A, const void* G, float* dW, int K, int N, cudaStream_t st) {
+  ProfScope prof_(h, K_WEIGHT_GRAD, st);
+#define GNNCO_WG_CASE(KK, NN) \
+  if (K == KK && N == NN) return launch_wg<KK, NN>(h, A, G, dW, st)
+  GNNCO_WG_CASE(128, 64); GNNCO_WG_CASE(128, 128); GNNCO_WG_CASE(128, 256);
+  GNNCO_WG_CASE(256, 64); GNNCO_WG_CASE(256, 128); GNNCO_WG_CASE(256, 256);
+#undef GNNCO_WG_CASE
   return GNNCO_UNSUPPORTED;
 }
 

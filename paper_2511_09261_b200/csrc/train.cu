@@ -182,12 +182,10 @@ int32_t run_step(gnnco_handle* h, const gnnco_model_desc* m, const void* X, cons
         GNNCO_TRY(launch_transform(h, dt, dZ, Wc[l - 1], wstride[l - 1], other, N, K, true, false, h->inv_deg, st));
     }
     float* target = grad_target(l - 1);
-    if (sets == 1) {
-      GNNCO_TRY(launch_weight_grad(h, dt, T.M[l], dZ, T.dW_sets, K, N, st));
-      GNNCO_TRY(launch_sum_over_sets(h, T.dW_sets, target, (int64_t)K * N, h->S, st));
-    } else {
-      GNNCO_TRY(launch_weight_grad(h, dt, T.M[l], dZ, target, K, N, st));
-    }
+    float* wg_out = sets == 1 ? T.dW_sets : target;
+    if (tc_weight_grad_supported(dt, K, N)) GNNCO_TRY(launch_weight_grad_tc(h, T.M[l], dZ, wg_out, K, N, st));
+    else GNNCO_TRY(launch_weight_grad(h, dt, T.M[l], dZ, wg_out, K, N, st));
+    if (sets == 1) GNNCO_TRY(launch_sum_over_sets(h, T.dW_sets, target, (int64_t)K * N, h->S, st));
     GNNCO_TRY(finish_layer(l - 1, target));
     if (need_input_grad) {
       if (l > 1) {

@@ -201,3 +201,18 @@ def test_gather_rows_roundtrip():
     assert torch.equal(back, X)
     v = to_dev(np.arange(w.n, dtype=np.float32))
     assert torch.equal(graph.gather_rows(v, arr["perm"]), arr["perm"].float())
+
+
+@pytest.mark.parametrize("dims,n,S", [([256, 256, 256, 1], 3200, 8), ([128, 128, 1], 1500, 2), ([256, 64, 1], 900, 4),
+                                      ([128, 256, 1], 1300, 1)])
+def test_train_step_bf16_long_subgraphs(dims, n, S):
+    """Subgraphs of several hundred rows: many 128-row tiles per subgraph and a multi-stage
+    reduction in the weight-gradient kernel, with ragged tails."""
+    eu, ev, part = tiny_graph(n, 4.0 / n, S, seed=19)
+    book = oracle.bookkeeping(n, eu, ev, part, S)
+    graph = load_graph(n, eu, ev, part, S)
+    X = si.round_to_bf16(rand_features(n, dims[0], 23).astype(np.float32))
+    W = [si.round_to_bf16(w.astype(np.float32)) for w in rand_weights(dims, S, 29)]
+    case = StepCase(book, dims, "bf16", S, lam=0.0)
+    adam = dict(lr=1e-3, step=2, m=[np.zeros_like(w) for w in W], v=[np.zeros_like(w) for w in W])
+    case.run(graph, X, W, None, want_dx=True, adam=adam, label="bf16-long")
