@@ -185,6 +185,33 @@ __global__ void __launch_bounds__(256) rank1_masked_kernel(const float* __restri
   st(dZ + t, v);
 }
 
+// bf16, 8 features per thread (F a multiple of 8, 16-byte aligned rows)
+__global__ void __launch_bounds__(256) rank1_masked_bf16x8(const float* __restrict__ g,
+                                                           const __nv_bfloat16* __restrict__ w, int64_t w_stride,
+                                                           const int32_t* __restrict__ node_part,
+                                                           const __nv_bfloat16* __restrict__ H,
+                                                           __nv_bfloat16* __restrict__ dZ, int64_t n, int F) {
+  const int64_t t = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;      // one 8-element group
+  const int groups = F >> 3;
+  if (t >= n * groups) return;
+  const int64_t i = t / groups;
+  const int f = (int)(t - i * groups) << 3;
+  const float gi = __ldg(g + i);
+  const uint4 wv = __ldg(reinterpret_cast<const uint4*>(w + (int64_t)node_part[i] * w_stride + f));
+  uint4 hv = make_uint4(0x3f803f80u, 0x3f803f80u, 0x3f803f80u, 0x3f803f80u);   // ones when there is no mask
+  if (H) hv = __ldg(reinterpret_cast<const uint4*>(H + i * F + f));
+  const uint32_t wq[4] = {wv.x, wv.y, wv.z, wv.w}, hq[4] = {hv.x, hv.y, hv.z, hv.w};
+  uint32_t o[4];
+#pragma unroll
+  for (int k = 0; k < 4; ++k) {
+    const float w0 = __uint_as_float(wq[k] << 16), w1 = __uint_as_float(wq[k] & 0xffff0000u);
+    const float h0 = __uint_as_float(hq[k] << 16), h1 = __uint_as_float(hq[k] & 0xffff0000u);
+    __nv_bfloat162 v = __floats2bfloat162_rn(h0 > 0.0f ? gi * w0 : 0.0f, h1 > 0.0f ? gi * w1 : 0.0f);
+    o[k] = *reinterpret_cast<uint32_t*>(&v);
+  }
+  *reinterpret_cast<uint4*>(dZ + i * F + f) = make_uint4(o[0], o[1], o[2], o[3]);
+}
+
 __global__ void sum_over_sets_kernel(const float* __restrict__ in, float* __restrict__ out, int64_t count,
                                      int32_t sets) {
   const int64_t q = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
@@ -197,6 +224,16 @@ __global__ void sum_over_sets_kernel(const float* __restrict__ in, float* __rest
 __global__ void cast_bf16_kernel(const float* __restrict__ in, __nv_bfloat16* __restrict__ out, int64_t count) {
   const int64_t q = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
   if (q < count) out[q] = __float2bfloat16_rn(in[q]);
+}
+
+__global__ void cast_bf16x8_kernel(const float4* __restrict__ in, uint4* __restrict__ out, int64_t groups) {
+  const int64_t q = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+  if (q >= groups) return;
+  const float4 a = __ldg(in + 2 * q), b = __ldg(in + 2 * q + 1);
+  __nv_bfloat162 v0 = __floats2bfloat162_rn(a.x, a.y), v1 = __floats2bfloat162_rn(a.z, a.w);
+  __nv_bfloat162 v2 = __floats2bfloat162_rn(b.x, b.y), v3 = __floats2bfloat162_rn(b.z, b.w);
+  out[q] = make_uint4(*reinterpret_cast<uint32_t*>(&v0), *reinterpret_cast<uint32_t*>(&v1),
+                      *reinterpret_cast<uint32_t*>(&v2), *reinterpret_cast<uint32_t*>(&v3));
 }
 
 __global__ void adam_kernel(float* __restrict__ W, float* __restrict__ m, float* __restrict__ v,
@@ -297,6 +334,10 @@ int32_t launch_rank1_masked(gnnco_handle* h, int dtype, const float* g, const vo
   if (dtype == GNNCO_F32)
     rank1_masked_kernel<float, float><<<grid, 256, 0, stream>>>(g, (const float*)w, w_stride, h->node_part,
                                                                 (const float*)H, (float*)dZ, h->n, F);
+  else if (dtype == GNNCO_BF16 && F % 8 == 0 && w_stride % 8 == 0 &&
+           !(((uintptr_t)w | (uintptr_t)H | (uintptr_t)dZ) & 15))
+    rank1_masked_bf16x8<<<blocks_for(h->n * (F / 8), 256), 256, 0, stream>>>(
+        g, (const __nv_bfloat16*)w, w_stride, h->node_part, (const __nv_bfloat16*)H, (__nv_bfloat16*)dZ, h->n, F);
   else if (dtype == GNNCO_BF16)
     rank1_masked_kernel<__nv_bfloat16, __nv_bfloat16><<<grid, 256, 0, stream>>>(
         g, (const __nv_bfloat16*)w, w_stride, h->node_part, (const __nv_bfloat16*)H, (__nv_bfloat16*)dZ, h->n, F);
@@ -318,7 +359,11 @@ int32_t launch_sum_over_sets(gnnco_handle* h, const float* in, float* out, int64
 
 int32_t launch_cast_bf16(gnnco_handle* h, const float* in, __nv_bfloat16* out, int64_t count, cudaStream_t stream) {
   ProfScope prof_(h, K_CAST, stream);
-  cast_bf16_kernel<<<blocks_for(count, 256), 256, 0, stream>>>(in, out, count);
+  if (count % 8 == 0 && !(((uintptr_t)in | (uintptr_t)out) & 15))
+    cast_bf16x8_kernel<<<blocks_for(count / 8, 256), 256, 0, stream>>>(reinterpret_cast<const float4*>(in),
+                                                                       reinterpret_cast<uint4*>(out), count / 8);
+  else
+    cast_bf16_kernel<<<blocks_for(count, 256), 256, 0, stream>>>(in, out, count);
   h->launches += 1;
   GNNCO_LAUNCH_CHECK();
   return GNNCO_OK;
