@@ -131,7 +131,8 @@ int32_t launch_adam(gnnco_handle* h, float* W, float* m, float* v, const float* 
 bool tc_transform_supported(int dtype, int K, int N);
 // Y = act(A B_s^T) * row_scale with A [n x K] and B [sets x N x K], K contiguous in both
 int32_t launch_transform_tc(gnnco_handle* h, const void* A, const void* B, int64_t b_stride, void* Y, int K, int N,
-                            bool relu, const float* row_scale, bool backward, cudaStream_t st);
+                            bool relu, const float* row_scale, bool backward, const void* dot_w, int64_t dot_stride,
+                            float* dot_out, cudaStream_t st);
 bool tc_weight_grad_supported(int dtype, int K, int N);
 int32_t launch_weight_grad_tc(gnnco_handle* h, const void* A, const void* G, float* dW, int K, int N, cudaStream_t st);
 // Wt[s][n][k] = bf16(W[s][k][n])

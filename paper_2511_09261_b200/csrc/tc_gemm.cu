@@ -18,39 +18,52 @@ namespace {
 constexpr int kTileM = 128;
 constexpr int kThreads = 256;
 
-// Copy `rows_valid` rows (of `rows_total`) x KDIM bf16 from global (row stride KDIM) into
-// K-major SW128 shared memory: k-block kb at kb*rows_total*128, row r at (r/8)*1024 + (r%8)*128,
-// 16-byte chunk c at ((c ^ (r%8)) * 16).  Rows past rows_valid are zero-filled.
+// Roles of the eight warps of the transform kernel.
+constexpr int kEpiWarps = 4;                 // warps 0-3 drain the accumulator (one TMEM lane quarter each)
+constexpr int kMmaWarp = 4;                  // warp 4 issues the MMAs
+constexpr int kProdWarp0 = 5;                // warps 5-7 stage operands with cp.async
+constexpr int kProdLanes = 96;
+
+// One 64-wide k-block of `rows` rows (row stride KDIM elements) -> K-major SW128 shared memory:
+// row r at (r/8)*1024 + (r%8)*128, 16-byte chunk c at ((c ^ (r%8)) * 16).  Called by the 96
+// producer lanes; p = producer lane index.
 template <int KDIM>
-__device__ __forceinline__ void stage_k_major(uint32_t sbase, const __nv_bfloat16* __restrict__ g, int rows_total,
-                                              int rows_valid) {
-  constexpr int CPR = KDIM / 8;                 // 16-byte chunks per row
-  const int total = rows_total * CPR;
-  for (int q = threadIdx.x; q < total; q += kThreads) {
-    const int r = q / CPR, c = q % CPR;
-    const int kb = c >> 3, cc = c & 7;
-    const uint32_t dst = sbase + kb * (rows_total * 128) + (r >> 3) * 1024 + (r & 7) * 128 + ((cc ^ (r & 7)) << 4);
-    if (r < rows_valid) tc::cp_async16(dst, g + (int64_t)r * KDIM + c * 8);
-    else tc::st_shared_zero16(dst);
+__device__ __forceinline__ void stage_kblock(uint32_t sdst, const __nv_bfloat16* __restrict__ g, int rows, int p) {
+  for (int q = p; q < rows * 8; q += kProdLanes) {
+    const int r = q >> 3, cc = q & 7;
+    tc::cp_async16(sdst + (r >> 3) * 1024 + (r & 7) * 128 + ((cc ^ (r & 7)) << 4), g + (int64_t)r * KDIM + cc * 8);
   }
 }
 
+// Warp-specialised, persistent.  Shared memory: the subgraph's weight matrix (KB k-blocks of
+// NDIM rows) and one 128-row operand tile as KB independently recycled k-block slots.
+//   producers : wait until the MMAs that read slot kb are done, refill it (and the matching
+//               weight k-block when the subgraph changes), arrive on full[kb] when the copies land
+//   MMA warp  : for each k-block wait full[kb], issue 4 MMAs (K = 16 each) into accumulator
+//               buffer (tile & 1), commit -> empty[kb]; after the last k-block commit -> acc_full
+//   epilogue  : wait acc_full, read the accumulator (TMEM -> registers), scale / rectify /
+//               round to bf16, store; optionally the next layer's row dot product; arrive acc_empty
+// so the copies of tile t+1, the MMAs of tile t+1 and the drain of tile t overlap.
 template <int KDIM, int NDIM>
 __global__ void __launch_bounds__(kThreads, 1)
 transform_tc(const __nv_bfloat16* __restrict__ A, const __nv_bfloat16* __restrict__ B, int64_t b_stride,
              __nv_bfloat16* __restrict__ Y, int relu, const float* __restrict__ row_scale,
+             const __nv_bfloat16* __restrict__ dot_w, int64_t dot_stride, float* __restrict__ dot_out,
              const int32_t* __restrict__ tile_row0, const int32_t* __restrict__ tile_rows,
              const int32_t* __restrict__ node_part, int n_tiles, int tiles_per_cta, int32_t* status) {
   constexpr int KB = KDIM / 64;
-  constexpr uint32_t A_BYTES = KB * kTileM * 128;
-  constexpr uint32_t B_BYTES = KB * NDIM * 128;
+  constexpr uint32_t A_SLOT = kTileM * 128, B_SLOT = NDIM * 128;
+  constexpr uint32_t A_BYTES = KB * A_SLOT, B_BYTES = KB * B_SLOT;
   extern __shared__ uint8_t smem_raw[];
   const uint32_t sbase = (tc::smem_u32(smem_raw) + 1023u) & ~1023u;
   const uint32_t sA = sbase, sB = sbase + A_BYTES;
   uint8_t* gen_base = smem_raw + (sbase - tc::smem_u32(smem_raw));
-  uint64_t* bar = reinterpret_cast<uint64_t*>(gen_base + A_BYTES + B_BYTES);
-  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(gen_base + A_BYTES + B_BYTES + 8);
-  uint32_t* abort_flag = tmem_slot + 1;
+  uint64_t* full = reinterpret_cast<uint64_t*>(gen_base + A_BYTES + B_BYTES);   // [KB]
+  uint64_t* empty = full + KB;                                                  // [KB]
+  uint64_t* acc_full = empty + KB;                                              // [2]
+  uint64_t* acc_empty = acc_full + 2;                                           // [2]
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(acc_empty + 2);
+  volatile uint32_t* abort_flag = tmem_slot + 1;
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int t_begin = blockIdx.x * tiles_per_cta;
@@ -58,104 +71,133 @@ transform_tc(const __nv_bfloat16* __restrict__ A, const __nv_bfloat16* __restric
   if (t_begin >= t_end) return;
 
   if (threadIdx.x == 0) {
-    tc::mbar_init(bar, 1);
+    for (int kb = 0; kb < KB; ++kb) {
+      tc::mbar_init(full + kb, kProdLanes);
+      tc::mbar_init(empty + kb, 1);
+    }
+    for (int i = 0; i < 2; ++i) {
+      tc::mbar_init(acc_full + i, 1);
+      tc::mbar_init(acc_empty + i, kEpiWarps * 32);
+    }
     *abort_flag = 0;
     tc::fence_mbar_init();
   }
-  if (warp == 0) tc::tmem_alloc(tmem_slot, NDIM);
+  if (warp == 0) tc::tmem_alloc(tmem_slot, 2 * NDIM);
   tc::tc_fence_before_sync();
   __syncthreads();
   tc::tc_fence_after_sync();
   const uint32_t tmem = *tmem_slot;
-  constexpr uint32_t IDESC = tc::idesc_bf16_f32(kTileM, NDIM, false, false);
 
-  int cur_part = -1;
-  uint32_t phase = 0;
-  // prologue: operands of the first tile
-  {
-    const int64_t row0 = tile_row0[t_begin];
-    cur_part = node_part[row0];
-    stage_k_major<KDIM>(sB, B + (int64_t)cur_part * b_stride, NDIM, NDIM);
-    stage_k_major<KDIM>(sA, A + row0 * KDIM, kTileM, tile_rows[t_begin]);
-    tc::cp_async_commit();
-  }
-  for (int t = t_begin; t < t_end; ++t) {
-    const int64_t row0 = tile_row0[t];
-    const int rows = tile_rows[t];
+  if (warp >= kProdWarp0) {
+    // ------------------------------------------------------------------- producers
+    const int p = (warp - kProdWarp0) * 32 + lane;
+    int cur_part = -1;
+    for (int t = t_begin, j = 0; t < t_end && !*abort_flag; ++t, ++j) {
+      const int64_t row0 = tile_row0[t];
+      const int rows = tile_rows[t];
+      const int part = node_part[row0];
+      const bool new_b = part != cur_part;
+      cur_part = part;
+      for (int kb = 0; kb < KB; ++kb) {
+        if (j > 0 && !tc::mbar_wait_bounded(empty + kb, (j - 1) & 1)) *abort_flag = 1;
+        if (new_b) stage_kblock<KDIM>(sB + kb * B_SLOT, B + (int64_t)part * b_stride + kb * 64, NDIM, p);
+        stage_kblock<KDIM>(sA + kb * A_SLOT, A + row0 * KDIM + kb * 64, rows, p);   // rows past `rows` keep old bits: they only reach output rows that are never stored
+        tc::cp_async_arrive_noinc(full + kb);
+      }
+    }
     tc::cp_async_wait<0>();
-    tc::fence_proxy_async_smem();
-    __syncthreads();
-    if (threadIdx.x == 0) {
-      tc::tc_fence_after_sync();
+  } else if (warp == kMmaWarp) {
+    // -------------------------------------------------------------------- MMA issuer
+    constexpr uint32_t IDESC = tc::idesc_bf16_f32(kTileM, NDIM, false, false);
+    for (int t = t_begin, j = 0; t < t_end && !*abort_flag; ++t, ++j) {
+      const int buf = j & 1;
+      if (j >= 2 && !tc::mbar_wait_bounded(acc_empty + buf, ((j >> 1) - 1) & 1)) *abort_flag = 1;
+      for (int kb = 0; kb < KB; ++kb) {
+        if (!tc::mbar_wait_bounded(full + kb, j & 1)) *abort_flag = 1;
+        tc::fence_proxy_async_smem();
+        tc::tc_fence_after_sync();
+        if (lane == 0 && !*abort_flag) {
 #pragma unroll
-      for (int kb = 0; kb < KB; ++kb)
-#pragma unroll
-        for (int ks = 0; ks < 4; ++ks) {
-          const uint64_t ad = tc::smem_desc_sw128(sA + kb * (kTileM * 128) + ks * 32, 16, 1024);
-          const uint64_t bd = tc::smem_desc_sw128(sB + kb * (NDIM * 128) + ks * 32, 16, 1024);
-          tc::mma_bf16(tmem, ad, bd, IDESC, (kb | ks) != 0);
-        }
-      tc::mma_commit(bar);
-    }
-    if (!tc::mbar_wait_bounded(bar, phase)) *abort_flag = 1;
-    phase ^= 1;
-    __syncthreads();
-    if (*abort_flag) {
-      if (threadIdx.x == 0) atomicMin(status, (int32_t)GNNCO_INTERNAL);
-      break;
-    }
-    tc::tc_fence_after_sync();
-    // operands are consumed: start the next tile's copies, they fly during the drain below
-    if (t + 1 < t_end) {
-      const int64_t nrow0 = tile_row0[t + 1];
-      const int npart = node_part[nrow0];
-      if (npart != cur_part) {
-        cur_part = npart;
-        stage_k_major<KDIM>(sB, B + (int64_t)cur_part * b_stride, NDIM, NDIM);
-      }
-      stage_k_major<KDIM>(sA, A + nrow0 * KDIM, kTileM, tile_rows[t + 1]);
-      tc::cp_async_commit();
-    }
-    // drain the accumulator: warp w reads lanes 32*(w%4).., columns half (w/4)
-    {
-      const int lg = warp & 3, ch = warp >> 2;
-      const int row = lg * 32 + lane;
-      const float s = (row_scale && row < rows) ? row_scale[row0 + row] : 1.0f;
-      constexpr int HALF = NDIM / 2;
-#pragma unroll
-      for (int c0 = 0; c0 < HALF; c0 += 32) {
-        uint32_t r[32];
-        tc::tmem_ld_32x32(tmem + ((uint32_t)(lg * 32) << 16) + ch * HALF + c0, r);
-        tc::tmem_ld_wait();
-        if (row < rows) {
-          uint4 out[4];
-          uint32_t* o = reinterpret_cast<uint32_t*>(out);
-#pragma unroll
-          for (int j = 0; j < 16; ++j) {
-            float a = __uint_as_float(r[2 * j]) * s, b = __uint_as_float(r[2 * j + 1]) * s;
-            if (relu) { a = a > 0.0f ? a : 0.0f; b = b > 0.0f ? b : 0.0f; }
-            __nv_bfloat162 v = __floats2bfloat162_rn(a, b);
-            o[j] = *reinterpret_cast<uint32_t*>(&v);
+          for (int ks = 0; ks < 4; ++ks) {
+            const uint64_t ad = tc::smem_desc_sw128(sA + kb * A_SLOT + ks * 32, 16, 1024);
+            const uint64_t bd = tc::smem_desc_sw128(sB + kb * B_SLOT + ks * 32, 16, 1024);
+            tc::mma_bf16(tmem + buf * NDIM, ad, bd, IDESC, (kb | ks) != 0);
           }
-          uint4* dst = reinterpret_cast<uint4*>(Y + (row0 + row) * NDIM + ch * HALF + c0);
-#pragma unroll
-          for (int j = 0; j < 4; ++j) dst[j] = out[j];
+          tc::mma_commit(empty + kb);
+          if (kb == KB - 1) tc::mma_commit(acc_full + buf);
         }
+        __syncwarp();
       }
     }
-    tc::tc_fence_before_sync();   // the next tile's MMA overwrites the accumulator after the sync at the loop top
+  } else {
+    // ---------------------------------------------------------------------- epilogue
+    const int row = warp * 32 + lane;
+    int cur_part = -1;
+    for (int t = t_begin, j = 0; t < t_end && !*abort_flag; ++t, ++j) {
+      const int buf = j & 1;
+      const int64_t row0 = tile_row0[t];
+      const int rows = tile_rows[t];
+      const bool valid = row < rows;
+      const float s = (row_scale && valid) ? row_scale[row0 + row] : 1.0f;
+      const __nv_bfloat16* wv = nullptr;
+      if (dot_out) {
+        const int part = node_part[row0];
+        cur_part = part;
+        wv = dot_w + (int64_t)part * dot_stride;
+      }
+      float dot = 0.0f;
+      if (!tc::mbar_wait_bounded(acc_full + buf, (j >> 1) & 1)) { *abort_flag = 1; break; }
+      tc::tc_fence_after_sync();
+#pragma unroll 2
+      for (int c0 = 0; c0 < NDIM; c0 += 32) {
+        uint32_t r[32];
+        tc::tmem_ld_32x32(tmem + ((uint32_t)(warp * 32) << 16) + buf * NDIM + c0, r);
+        tc::tmem_ld_wait();
+        uint4 out[4];
+        uint32_t* o = reinterpret_cast<uint32_t*>(out);
+#pragma unroll
+        for (int q = 0; q < 16; ++q) {
+          float a = __uint_as_float(r[2 * q]) * s, b = __uint_as_float(r[2 * q + 1]) * s;
+          if (relu) { a = a > 0.0f ? a : 0.0f; b = b > 0.0f ? b : 0.0f; }
+          __nv_bfloat162 v = __floats2bfloat162_rn(a, b);
+          o[q] = *reinterpret_cast<uint32_t*>(&v);
+        }
+        if (wv) {   // dot product of the STORED (rounded) row with the next layer's weight vector
+#pragma unroll
+          for (int q4 = 0; q4 < 4; ++q4) {
+            const uint4 w8 = __ldg(reinterpret_cast<const uint4*>(wv + c0 + q4 * 8));
+            const uint32_t wq[4] = {w8.x, w8.y, w8.z, w8.w};
+#pragma unroll
+            for (int q = 0; q < 4; ++q) {
+              const uint32_t hv = o[q4 * 4 + q];
+              dot = fmaf(__uint_as_float(hv << 16), __uint_as_float(wq[q] << 16), dot);
+              dot = fmaf(__uint_as_float(hv & 0xffff0000u), __uint_as_float(wq[q] & 0xffff0000u), dot);
+            }
+          }
+        }
+        if (valid) {
+          uint4* dst = reinterpret_cast<uint4*>(Y + (row0 + row) * NDIM + c0);
+#pragma unroll
+          for (int q = 0; q < 4; ++q) dst[q] = out[q];
+        }
+      }
+      if (dot_out && valid) dot_out[row0 + row] = dot;
+      tc::tc_fence_before_sync();
+      tc::mbar_arrive(acc_empty + buf);
+    }
+    (void)cur_part;
   }
-  tc::cp_async_wait<0>();
+  if (*abort_flag && threadIdx.x == 0) atomicMin(status, (int32_t)GNNCO_INTERNAL);
   tc::tc_fence_before_sync();
   __syncthreads();
-  if (warp == 0) tc::tmem_dealloc(tmem, NDIM);
+  if (warp == 0) tc::tmem_dealloc(tmem, 2 * NDIM);
 }
 
 template <int KDIM, int NDIM>
 int32_t launch_tc(gnnco_handle* h, const void* A, const void* B, int64_t b_stride, void* Y, bool relu,
-                  const float* row_scale, cudaStream_t st) {
+                  const float* row_scale, const void* dot_w, int64_t dot_stride, float* dot_out, cudaStream_t st) {
   constexpr int KB = KDIM / 64;
-  constexpr size_t smem = (size_t)KB * (kTileM + NDIM) * 128 + 64 + 1024;
+  constexpr size_t smem = (size_t)KB * (kTileM + NDIM) * 128 + 256 + 1024;
   GNNCO_CUDA_TRY(cudaFuncSetAttribute(transform_tc<KDIM, NDIM>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                       (int)smem));
   int sms = h->sm_count > 0 ? h->sm_count : 148;
@@ -164,7 +206,8 @@ int32_t launch_tc(gnnco_handle* h, const void* A, const void* B, int64_t b_strid
   grid = (h->n_tiles + per - 1) / per;
   transform_tc<KDIM, NDIM><<<grid, kThreads, smem, st>>>(
       (const __nv_bfloat16*)A, (const __nv_bfloat16*)B, b_stride, (__nv_bfloat16*)Y, relu ? 1 : 0, row_scale,
-      h->tile_row0, h->tile_rows, h->node_part, h->n_tiles, per, h->status);
+      (const __nv_bfloat16*)dot_w, dot_stride, dot_out, h->tile_row0, h->tile_rows, h->node_part, h->n_tiles, per,
+      h->status);
   h->launches += 1;
   GNNCO_LAUNCH_CHECK();
   return GNNCO_OK;
@@ -335,12 +378,15 @@ bool tc_transform_supported(int dtype, int K, int N) {
 }
 
 // Y = act(A B_s^T) * row_scale with A [n x K], B [sets x N x K] (both bf16, K contiguous).
+// With dot_out != nullptr also dot_out[i] = Y[i,:] . dot_w[s,:] (the width-1 output layer's
+// product, taken on the rounded values that are stored).
 int32_t launch_transform_tc(gnnco_handle* h, const void* A, const void* B, int64_t b_stride, void* Y, int K, int N,
-                            bool relu, const float* row_scale, bool backward, cudaStream_t st) {
+                            bool relu, const float* row_scale, bool backward, const void* dot_w, int64_t dot_stride,
+                            float* dot_out, cudaStream_t st) {
   if (h->n_tiles == 0) return GNNCO_OK;
   ProfScope prof_(h, backward ? K_TRANSFORM_BWD : K_TRANSFORM_FWD, st);
 #define GNNCO_TC_CASE(KK, NN) \
-  if (K == KK && N == NN) return launch_tc<KK, NN>(h, A, B, b_stride, Y, relu, row_scale, st)
+  if (K == KK && N == NN) return launch_tc<KK, NN>(h, A, B, b_stride, Y, relu, row_scale, dot_w, dot_stride, dot_out, st)
   GNNCO_TC_CASE(64, 64); GNNCO_TC_CASE(64, 128); GNNCO_TC_CASE(64, 256);
   GNNCO_TC_CASE(128, 64); GNNCO_TC_CASE(128, 128); GNNCO_TC_CASE(128, 256);
   GNNCO_TC_CASE(256, 64); GNNCO_TC_CASE(256, 128); GNNCO_TC_CASE(256, 256);

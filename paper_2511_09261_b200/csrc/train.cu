@@ -121,18 +121,22 @@ int32_t run_step(gnnco_handle* h, const gnnco_model_desc* m, const void* X, cons
   }
   // ---- forward
   const void* Hprev = X;
+  bool u_done = false;
   for (int l = 1; l < L; ++l) {
     GNNCO_TRY(launch_aggregate(h, dt, Hprev, T.M[l], m->dims[l - 1], h->inv_deg, nullptr, st));
-    if (T.W_lp_t[l - 1])
+    if (T.W_lp_t[l - 1]) {
+      // the last hidden layer also produces u = H w_L in its epilogue
+      const bool fuse = (l == L - 1) && (m->dims[l] % 8 == 0);
       GNNCO_TRY(launch_transform_tc(h, T.M[l], T.W_lp_t[l - 1], wstride[l - 1], T.H[l], m->dims[l - 1], m->dims[l], true,
-                                    nullptr, false, st));
-    else
+                                    nullptr, false, fuse ? Wc[L - 1] : nullptr, wstride[L - 1], fuse ? T.u : nullptr, st));
+      u_done = fuse;
+    } else
       GNNCO_TRY(launch_transform(h, dt, T.M[l], Wc[l - 1], wstride[l - 1], T.H[l], m->dims[l - 1], m->dims[l], false,
                                  true, nullptr, st));
     Hprev = T.H[l];
   }
   const int FL = m->dims[L - 1];
-  GNNCO_TRY(launch_gemv(h, dt, Hprev, Wc[L - 1], wstride[L - 1], T.u, FL, st));
+  if (!u_done) GNNCO_TRY(launch_gemv(h, dt, Hprev, Wc[L - 1], wstride[L - 1], T.u, FL, st));
   GNNCO_TRY(launch_output_forward(h, T.u, out->z, out->p, st));
   const bool fwd_only = (flags & GNNCO_FORWARD_ONLY) != 0;
   GNNCO_TRY(launch_objective(h, out->p, obj->pen, obj->alpha, obj->beta, obj->lambda, T.item_loss, out->loss,
@@ -177,7 +181,8 @@ int32_t run_step(gnnco_handle* h, const gnnco_model_desc* m, const void* X, cons
     const bool need_input_grad = (l > 1) || (flags & GNNCO_WANT_DX);
     if (need_input_grad) {
       if (tc_transform_supported(dt, N, K))
-        GNNCO_TRY(launch_transform_tc(h, dZ, Wc[l - 1], wstride[l - 1], other, N, K, false, h->inv_deg, true, st));
+        GNNCO_TRY(launch_transform_tc(h, dZ, Wc[l - 1], wstride[l - 1], other, N, K, false, h->inv_deg, true, nullptr, 0,
+                                      nullptr, st));
       else
         GNNCO_TRY(launch_transform(h, dt, dZ, Wc[l - 1], wstride[l - 1], other, N, K, true, false, h->inv_deg, st));
     }
