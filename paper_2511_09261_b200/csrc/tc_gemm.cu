@@ -98,6 +98,8 @@ transform_tc(const __nv_bfloat16* __restrict__ A, const __nv_bfloat16* __restric
       const int part = node_part[row0];
       const bool new_b = part != cur_part;
       cur_part = part;
+      if (p == 0 && t + 2 < t_end)   // the tile after next: pull its rows (contiguous) into L2 ahead of the copies
+        tc::prefetch_l2(A + (int64_t)tile_row0[t + 2] * KDIM, (uint32_t)tile_rows[t + 2] * KDIM * 2);
       for (int kb = 0; kb < KB; ++kb) {
         if (j > 0 && !tc::mbar_wait_bounded(empty + kb, (j - 1) & 1)) *abort_flag = 1;
         if (new_b) stage_kblock<KDIM>(sB + kb * B_SLOT, B + (int64_t)part * b_stride + kb * 64, NDIM, p);
@@ -132,6 +134,7 @@ transform_tc(const __nv_bfloat16* __restrict__ A, const __nv_bfloat16* __restric
   } else {
     // ---------------------------------------------------------------------- epilogue
     const int row = warp * 32 + lane;
+    const uint32_t stage = sbase + A_BYTES + B_BYTES + 256 + warp * 4096;
     int cur_part = -1;
     for (int t = t_begin, j = 0; t < t_end && !*abort_flag; ++t, ++j) {
       const int buf = j & 1;
@@ -148,23 +151,26 @@ transform_tc(const __nv_bfloat16* __restrict__ A, const __nv_bfloat16* __restric
       float dot = 0.0f;
       if (!tc::mbar_wait_bounded(acc_full + buf, (j >> 1) & 1)) { *abort_flag = 1; break; }
       tc::tc_fence_after_sync();
-#pragma unroll 2
-      for (int c0 = 0; c0 < NDIM; c0 += 32) {
-        uint32_t r[32];
-        tc::tmem_ld_32x32(tmem + ((uint32_t)(warp * 32) << 16) + buf * NDIM + c0, r);
-        tc::tmem_ld_wait();
-        uint4 out[4];
-        uint32_t* o = reinterpret_cast<uint32_t*>(out);
+      const int rows_here = rows - warp * 32;          // valid rows of this warp's 32
+#pragma unroll 1
+      for (int c0 = 0; c0 < NDIM; c0 += 64) {
+        uint32_t o[32];                                // 64 bf16 of this thread's row, packed
 #pragma unroll
-        for (int q = 0; q < 16; ++q) {
-          float a = __uint_as_float(r[2 * q]) * s, b = __uint_as_float(r[2 * q + 1]) * s;
-          if (relu) { a = a > 0.0f ? a : 0.0f; b = b > 0.0f ? b : 0.0f; }
-          __nv_bfloat162 v = __floats2bfloat162_rn(a, b);
-          o[q] = *reinterpret_cast<uint32_t*>(&v);
+        for (int half = 0; half < 2; ++half) {
+          uint32_t r[32];
+          tc::tmem_ld_32x32(tmem + ((uint32_t)(warp * 32) << 16) + buf * NDIM + c0 + half * 32, r);
+          tc::tmem_ld_wait();
+#pragma unroll
+          for (int q = 0; q < 16; ++q) {
+            float a = __uint_as_float(r[2 * q]) * s, b = __uint_as_float(r[2 * q + 1]) * s;
+            if (relu) { a = a > 0.0f ? a : 0.0f; b = b > 0.0f ? b : 0.0f; }
+            __nv_bfloat162 v = __floats2bfloat162_rn(a, b);
+            o[half * 16 + q] = *reinterpret_cast<uint32_t*>(&v);
+          }
         }
         if (wv) {   // dot product of the STORED (rounded) row with the next layer's weight vector
 #pragma unroll
-          for (int q4 = 0; q4 < 4; ++q4) {
+          for (int q4 = 0; q4 < 8; ++q4) {
             const uint4 w8 = __ldg(reinterpret_cast<const uint4*>(wv + c0 + q4 * 8));
             const uint32_t wq[4] = {w8.x, w8.y, w8.z, w8.w};
 #pragma unroll
@@ -175,10 +181,20 @@ transform_tc(const __nv_bfloat16* __restrict__ A, const __nv_bfloat16* __restric
             }
           }
         }
-        if (valid) {
-          uint4* dst = reinterpret_cast<uint4*>(Y + (row0 + row) * NDIM + c0);
+        // through a per-warp staging tile (32 rows x 128 bytes, pieces XOR-swizzled by row) so
+        // that each store instruction writes whole 128-byte lines: 8 lanes per row, 4 rows
+        __syncwarp();
 #pragma unroll
-          for (int q = 0; q < 4; ++q) dst[q] = out[q];
+        for (int pc = 0; pc < 8; ++pc)
+          tc::st_shared16(stage + lane * 128 + ((pc ^ (lane & 7)) << 4), o[4 * pc], o[4 * pc + 1], o[4 * pc + 2],
+                          o[4 * pc + 3]);
+        __syncwarp();
+#pragma unroll
+        for (int it = 0; it < 8; ++it) {
+          const int rr = it * 4 + (lane >> 3), pc = lane & 7;
+          const uint4 v = tc::ld_shared16(stage + rr * 128 + ((pc ^ (rr & 7)) << 4));
+          if (rr < rows_here)
+            *reinterpret_cast<uint4*>(Y + (row0 + warp * 32 + rr) * NDIM + c0 + pc * 8) = v;
         }
       }
       if (dot_out && valid) dot_out[row0 + row] = dot;
@@ -197,7 +213,7 @@ template <int KDIM, int NDIM>
 int32_t launch_tc(gnnco_handle* h, const void* A, const void* B, int64_t b_stride, void* Y, bool relu,
                   const float* row_scale, const void* dot_w, int64_t dot_stride, float* dot_out, cudaStream_t st) {
   constexpr int KB = KDIM / 64;
-  constexpr size_t smem = (size_t)KB * (kTileM + NDIM) * 128 + 256 + 1024;
+  constexpr size_t smem = (size_t)KB * (kTileM + NDIM) * 128 + 256 + kEpiWarps * 4096 + 1024;
   GNNCO_CUDA_TRY(cudaFuncSetAttribute(transform_tc<KDIM, NDIM>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                       (int)smem));
   int sms = h->sm_count > 0 ? h->sm_count : 148;
