@@ -21,6 +21,7 @@
   } while (0)
 
 constexpr int kGemmTileRows = 128;   // rows of one dense-transform tile (never straddles a subgraph)
+constexpr int kLongRowDegree = 256;  // rows with more intra neighbours are aggregated by a whole block
 constexpr int kItemRows = 1024;      // rows of one objective work item (never straddles a subgraph)
 
 // Kernel families, for launch accounting and per-kernel timing.
@@ -60,10 +61,15 @@ struct gnnco_handle {
   int32_t *item_row0 = nullptr, *item_row1 = nullptr;      // objective work items
   int32_t* part_item_ptr = nullptr;                        // [S+1] items of each subgraph
   int32_t* status = nullptr;                               // device status word + counters
-  int32_t n_tiles = 0, n_items = 0;
+  int4* row_head = nullptr;                                // {first CSR slot, degree, first two neighbours} per row
+  int32_t* long_rows = nullptr;                            // ids of rows with degree > kLongRowDegree
+  int32_t n_tiles = 0, n_items = 0, n_long = 0;
   std::vector<int32_t> h_part_ptr;
   int64_t launches = 0;
   Profiler prof;
+  // long rows are aggregated on a side stream, concurrently with the short rows
+  cudaStream_t side_stream = nullptr;
+  cudaEvent_t ev_fork = nullptr, ev_join = nullptr;
 };
 
 struct ProfScope {

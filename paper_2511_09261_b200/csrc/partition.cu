@@ -200,7 +200,7 @@ __global__ void segment_starts(const uint64_t* keys, int64_t N, int32_t nseg, in
 }
 
 // ----------------------------------------------------------------------- the steps
-enum { kStatus = 0, kCntIn = 1, kCntB = 2, kMaxRow = 3, kStatusWords = 16 };
+enum { kStatus = 0, kCntIn = 1, kCntB = 2, kMaxRow = 3, kSelfLoop = 4, kLongCnt = 5, kStatusWords = 16 };
 
 __global__ void check_parts_make_keys(const int32_t* part, int64_t n, int32_t S, uint64_t* keys, int32_t* status) {
   int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
@@ -218,7 +218,7 @@ __global__ void check_edges(const int32_t* eu, const int32_t* ev, int64_t E, int
   if (e >= E) return;
   int32_t u = eu[e], v = ev[e];
   if (u < 0 || u >= n || v < 0 || v >= n) atomicMin(&status[kStatus], (int32_t)GNNCO_OUT_OF_RANGE);
-  else if (u == v) atomicMax(&status[kMaxRow + 1], 1);    // self loop seen (reported if ids are all in range)
+  else if (u == v) atomicMax(&status[kSelfLoop], 1);    // self loop seen (reported if ids are all in range)
 }
 
 __global__ void unpack_node_order(const uint64_t* keys, int64_t n, int32_t* perm, int32_t* inv_perm,
@@ -271,6 +271,25 @@ __global__ void degree_scale(const int32_t* rowptr, int64_t n, float* inv_deg, i
   if ((threadIdx.x & 31) == 0) atomicMax(&status[kMaxRow], m);
 }
 
+// row_head[i] = {rowptr[i], degree, first neighbour or -1, second neighbour or -1}
+__global__ void build_row_heads(const int32_t* rowptr, const int32_t* colidx, int64_t n, int4* row_head) {
+  int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+  if (i >= n) return;
+  const int32_t a = rowptr[i], d = rowptr[i + 1] - a;
+  row_head[i] = make_int4(a, d, d > 0 ? colidx[a] : -1, d > 1 ? colidx[a + 1] : -1);
+}
+
+// rows longer than kLongRowDegree, in no particular order (each is processed on its own)
+__global__ void collect_long_rows(const int32_t* rowptr, int64_t n, int32_t* long_rows, int32_t capacity,
+                                  int32_t* status) {
+  int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+  if (i >= n) return;
+  if (rowptr[i + 1] - rowptr[i] > kLongRowDegree) {
+    int32_t slot = atomicAdd(&status[kLongCnt], 1);
+    if (slot < capacity) long_rows[slot] = (int32_t)i;
+  }
+}
+
 template <int VEC>
 __global__ void gather_rows_kernel(const char* src, char* dst, const int32_t* index, int64_t rows, int64_t units) {
   int64_t t = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
@@ -293,8 +312,9 @@ struct PersistentLayout {
   int32_t *perm, *inv_perm, *node_part, *part_ptr, *rowptr, *colidx, *bnd_u, *bnd_v;
   float* inv_deg;
   uint8_t* is_boundary;
-  int32_t *tile_row0, *tile_rows, *item_row0, *item_row1, *part_item_ptr, *status;
-  int64_t max_tiles, max_items;
+  int32_t *tile_row0, *tile_rows, *item_row0, *item_row1, *part_item_ptr, *status, *long_rows;
+  int4* row_head;
+  int64_t max_tiles, max_items, max_long;
   size_t bytes;
 };
 
@@ -319,6 +339,9 @@ PersistentLayout carve_persistent(void* base, int64_t n, int64_t E, int32_t S) {
   L.item_row0 = c.take<int32_t>(L.max_items);
   L.item_row1 = c.take<int32_t>(L.max_items);
   L.part_item_ptr = c.take<int32_t>((size_t)S + 1);
+  L.max_long = 2 * E / kLongRowDegree + 1;
+  L.long_rows = c.take<int32_t>(L.max_long);
+  L.row_head = c.take<int4>(n);
   L.bytes = c.off;
   return L;
 }
@@ -388,7 +411,7 @@ extern "C" int32_t gnnco_partition_load(const gnnco_graph_desc* g, void* persist
   if (!h) return GNNCO_INTERNAL;
   struct Guard {
     gnnco_handle* h;
-    ~Guard() { delete h; }
+    ~Guard() { if (h) gnnco_destroy(h); }
   } guard{h};
   GNNCO_CUDA_TRY(cudaGetDevice(&h->device));
   GNNCO_CUDA_TRY(cudaDeviceGetAttribute(&h->sm_count, cudaDevAttrMultiProcessorCount, h->device));
@@ -397,7 +420,7 @@ extern "C" int32_t gnnco_partition_load(const gnnco_graph_desc* g, void* persist
   h->rowptr = P.rowptr; h->colidx = P.colidx; h->bnd_u = P.bnd_u; h->bnd_v = P.bnd_v;
   h->inv_deg = P.inv_deg; h->is_boundary = P.is_boundary;
   h->tile_row0 = P.tile_row0; h->tile_rows = P.tile_rows; h->item_row0 = P.item_row0; h->item_row1 = P.item_row1;
-  h->part_item_ptr = P.part_item_ptr; h->status = P.status;
+  h->part_item_ptr = P.part_item_ptr; h->status = P.status; h->long_rows = P.long_rows; h->row_head = P.row_head;
 
   const int T = 256;
   int32_t hs[kStatusWords];
@@ -414,7 +437,7 @@ extern "C" int32_t gnnco_partition_load(const gnnco_graph_desc* g, void* persist
   GNNCO_CUDA_TRY(cudaMemcpyAsync(hs, P.status, sizeof(hs), cudaMemcpyDeviceToHost, st));
   GNNCO_CUDA_TRY(cudaStreamSynchronize(st));
   if (hs[kStatus] != GNNCO_OK) return hs[kStatus];
-  if (hs[kMaxRow + 1] != 0) return GNNCO_NOT_SIMPLE_GRAPH;
+  if (hs[kSelfLoop] != 0) return GNNCO_NOT_SIMPLE_GRAPH;
 
   // 2. new node order: stable sort of (part, id) on the part bits
   uint64_t* sorted = nullptr;
@@ -466,7 +489,9 @@ extern "C" int32_t gnnco_partition_load(const gnnco_graph_desc* g, void* persist
     h->launches += 1;
   }
   degree_scale<<<grid_for(n, T), T, 0, st>>>(P.rowptr, n, P.inv_deg, P.status);
-  h->launches += 1;
+  collect_long_rows<<<grid_for(n, T), T, 0, st>>>(P.rowptr, n, P.long_rows, (int32_t)P.max_long, P.status);
+  build_row_heads<<<grid_for(n, T), T, 0, st>>>(P.rowptr, P.colidx, n, P.row_head);
+  h->launches += 3;
   GNNCO_LAUNCH_CHECK();
 
   // 5. host-built tables: dense-transform tiles and objective work items (from part_ptr)
@@ -500,6 +525,11 @@ extern "C" int32_t gnnco_partition_load(const gnnco_graph_desc* g, void* persist
   GNNCO_CUDA_TRY(cudaStreamSynchronize(st));
   if (hs[kStatus] != GNNCO_OK) return hs[kStatus];
   h->max_row = hs[kMaxRow];
+  GNNCO_CUDA_TRY(cudaStreamCreateWithFlags(&h->side_stream, cudaStreamNonBlocking));
+  GNNCO_CUDA_TRY(cudaEventCreateWithFlags(&h->ev_fork, cudaEventDisableTiming));
+  GNNCO_CUDA_TRY(cudaEventCreateWithFlags(&h->ev_join, cudaEventDisableTiming));
+  h->n_long = hs[kLongCnt];
+  if (h->n_long > P.max_long) return GNNCO_INTERNAL;
   guard.h = nullptr;
   *out = h;
   return GNNCO_OK;
@@ -540,8 +570,12 @@ extern "C" int32_t gnnco_async_status(const gnnco_handle* h, void* stream, int32
 extern "C" int64_t gnnco_launch_count(const gnnco_handle* h) { return h ? h->launches : 0; }
 
 extern "C" int32_t gnnco_destroy(gnnco_handle* h) {
-  if (h)
+  if (h) {
     for (cudaEvent_t e : h->prof.pool) cudaEventDestroy(e);
+    if (h->ev_fork) cudaEventDestroy(h->ev_fork);
+    if (h->ev_join) cudaEventDestroy(h->ev_join);
+    if (h->side_stream) cudaStreamDestroy(h->side_stream);
+  }
   delete h;
   return GNNCO_OK;
 }

@@ -25,6 +25,11 @@ struct Vec<float> {
     float4 v = __ldg(reinterpret_cast<const float4*>(p));
     f[0] = v.x; f[1] = v.y; f[2] = v.z; f[3] = v.w;
   }
+  __device__ static uint4 load_raw(const float* p) { return __ldg(reinterpret_cast<const uint4*>(p)); }
+  __device__ static void add_raw(float (&acc)[4], const uint4& v) {
+    acc[0] += __uint_as_float(v.x); acc[1] += __uint_as_float(v.y);
+    acc[2] += __uint_as_float(v.z); acc[3] += __uint_as_float(v.w);
+  }
   __device__ static void store(float* p, const float (&f)[4]) {
     *reinterpret_cast<float4*>(p) = make_float4(f[0], f[1], f[2], f[3]);
   }
@@ -39,6 +44,15 @@ struct Vec<__nv_bfloat16> {
     for (int k = 0; k < 4; ++k) {
       f[2 * k] = __uint_as_float(w[k] << 16);
       f[2 * k + 1] = __uint_as_float(w[k] & 0xffff0000u);
+    }
+  }
+  __device__ static uint4 load_raw(const __nv_bfloat16* p) { return __ldg(reinterpret_cast<const uint4*>(p)); }
+  __device__ static void add_raw(float (&acc)[8], const uint4& v) {
+    const uint32_t w[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+    for (int k = 0; k < 4; ++k) {
+      acc[2 * k] += __uint_as_float(w[k] << 16);
+      acc[2 * k + 1] += __uint_as_float(w[k] & 0xffff0000u);
     }
   }
   __device__ static void store(__nv_bfloat16* p, const float (&f)[8]) {
@@ -58,47 +72,67 @@ __device__ __forceinline__ void from_f32(float& d, float x) { d = x; }
 __device__ __forceinline__ void from_f32(__nv_bfloat16& d, float x) { d = __float2bfloat16_rn(x); }
 
 // LPR lanes per row, VPL vectors per lane: row width F = LPR * VPL * Vec<T>::N elements.
+// row_head[i] = {first CSR slot, degree, first neighbour, second neighbour}: one 16-byte load
+// tells a row its extent AND its first two neighbours, so for the many rows of degree <= 2
+// the neighbour features are only one round trip behind the head instead of two.
 template <typename T, int LPR, int VPL>
 __global__ void __launch_bounds__(256) aggregate_vec(const T* __restrict__ in, T* __restrict__ out,
-                                                     const int32_t* __restrict__ rowptr,
+                                                     const int4* __restrict__ row_head,
                                                      const int32_t* __restrict__ colidx,
                                                      const float* __restrict__ scale, const T* __restrict__ mask,
-                                                     int64_t n, int F) {
+                                                     int64_t n, int F, int skip_long) {
   constexpr int VN = Vec<T>::N;
   constexpr int ROWS_PER_BLOCK = 256 / LPR;
   const int sub = threadIdx.x % LPR;
   const int64_t row = (int64_t)blockIdx.x * ROWS_PER_BLOCK + threadIdx.x / LPR;
   if (row >= n) return;
-  const int32_t r0 = __ldg(rowptr + row), r1 = __ldg(rowptr + row + 1);
+  // the row's own features are requested before its CSR extent is known, so the two round
+  // trips overlap
   float acc[VPL][VN];
 #pragma unroll
   for (int v = 0; v < VPL; ++v) Vec<T>::load(in + row * F + (v * LPR + sub) * VN, acc[v]);
-  int32_t k = r0;
+  const int4 head = __ldg(row_head + row);
+  const int32_t deg = head.y;
+  if (skip_long && deg > kLongRowDegree) return;   // a whole block takes this row
+  {
+    uint4 t[2][VPL];
+    if (deg > 0) {
+#pragma unroll
+      for (int v = 0; v < VPL; ++v) t[0][v] = Vec<T>::load_raw(in + (int64_t)head.z * F + (v * LPR + sub) * VN);
+    }
+    if (deg > 1) {
+#pragma unroll
+      for (int v = 0; v < VPL; ++v) t[1][v] = Vec<T>::load_raw(in + (int64_t)head.w * F + (v * LPR + sub) * VN);
+    }
+    if (deg > 0) {
+#pragma unroll
+      for (int v = 0; v < VPL; ++v) Vec<T>::add_raw(acc[v], t[0][v]);
+    }
+    if (deg > 1) {
+#pragma unroll
+      for (int v = 0; v < VPL; ++v) Vec<T>::add_raw(acc[v], t[1][v]);
+    }
+  }
+  const int32_t r1 = head.x + deg;
+  int32_t k = head.x + 2;
   for (; k + 4 <= r1; k += 4) {
     int32_t j[4];
 #pragma unroll
     for (int u = 0; u < 4; ++u) j[u] = __ldg(colidx + k + u);
-    float t[4][VPL][VN];
+    uint4 t[4][VPL];
 #pragma unroll
     for (int u = 0; u < 4; ++u)
 #pragma unroll
-      for (int v = 0; v < VPL; ++v) Vec<T>::load(in + (int64_t)j[u] * F + (v * LPR + sub) * VN, t[u][v]);
+      for (int v = 0; v < VPL; ++v) t[u][v] = Vec<T>::load_raw(in + (int64_t)j[u] * F + (v * LPR + sub) * VN);
 #pragma unroll
     for (int u = 0; u < 4; ++u)
 #pragma unroll
-      for (int v = 0; v < VPL; ++v)
-#pragma unroll
-        for (int e = 0; e < VN; ++e) acc[v][e] += t[u][v][e];
+      for (int v = 0; v < VPL; ++v) Vec<T>::add_raw(acc[v], t[u][v]);
   }
   for (; k < r1; ++k) {
     const int64_t j = __ldg(colidx + k);
 #pragma unroll
-    for (int v = 0; v < VPL; ++v) {
-      float t[VN];
-      Vec<T>::load(in + j * F + (v * LPR + sub) * VN, t);
-#pragma unroll
-      for (int e = 0; e < VN; ++e) acc[v][e] += t[e];
-    }
+    for (int v = 0; v < VPL; ++v) Vec<T>::add_raw(acc[v], Vec<T>::load_raw(in + j * F + (v * LPR + sub) * VN));
   }
   const float s = scale ? __ldg(scale + row) : 1.0f;
 #pragma unroll
@@ -114,6 +148,60 @@ __global__ void __launch_bounds__(256) aggregate_vec(const T* __restrict__ in, T
       for (int e = 0; e < VN; ++e) acc[v][e] *= s;
     }
     Vec<T>::store(out + off, acc[v]);
+  }
+}
+
+// A row with more than kLongRowDegree neighbours: one block per row.  Each of the 8 warps sums
+// a contiguous eighth of the neighbour list with eight rows in flight, the partial sums
+// meet in shared memory in warp order (deterministic), and the block finishes the row.
+template <typename T, int LPR, int VPL>
+__global__ void __launch_bounds__(256) aggregate_long_row(const T* __restrict__ in, T* __restrict__ out,
+                                                          const int32_t* __restrict__ rowptr,
+                                                          const int32_t* __restrict__ colidx,
+                                                          const float* __restrict__ scale,
+                                                          const T* __restrict__ mask,
+                                                          const int32_t* __restrict__ long_rows, int F) {
+  constexpr int VN = Vec<T>::N;
+  constexpr int GROUPS = 256 / LPR;               // lane groups, each walks its own slice of the row
+  extern __shared__ float partial[];              // [GROUPS][F]
+  const int64_t row = long_rows[blockIdx.x];
+  const int sub = threadIdx.x % LPR, grp = threadIdx.x / LPR;
+  const int32_t r0 = rowptr[row], r1 = rowptr[row + 1];
+  const int32_t len = (r1 - r0 + GROUPS - 1) / GROUPS;
+  const int32_t a = r0 + grp * len, b = min(r1, a + len);
+  float acc[VPL][VN];
+#pragma unroll
+  for (int v = 0; v < VPL; ++v)
+#pragma unroll
+    for (int e = 0; e < VN; ++e) acc[v][e] = 0.0f;
+  for (int32_t k = a; k < b; k += 8) {
+    uint4 t[8][VPL];
+#pragma unroll
+    for (int u = 0; u < 8; ++u)
+      if (k + u < b) {
+        const int64_t c = __ldg(colidx + k + u);
+#pragma unroll
+        for (int v = 0; v < VPL; ++v) t[u][v] = Vec<T>::load_raw(in + c * F + (v * LPR + sub) * VN);
+      }
+#pragma unroll
+    for (int u = 0; u < 8; ++u)
+      if (k + u < b) {
+#pragma unroll
+        for (int v = 0; v < VPL; ++v) Vec<T>::add_raw(acc[v], t[u][v]);
+      }
+  }
+#pragma unroll
+  for (int v = 0; v < VPL; ++v)
+#pragma unroll
+    for (int e = 0; e < VN; ++e) partial[grp * F + (v * LPR + sub) * VN + e] = acc[v][e];
+  __syncthreads();
+  const float sc = scale ? scale[row] : 1.0f;
+  for (int f = threadIdx.x; f < F; f += 256) {
+    float tot = to_f32(in[row * F + f]);
+    for (int g = 0; g < GROUPS; ++g) tot += partial[g * F + f];
+    tot *= sc;
+    if (mask && !(to_f32(mask[row * F + f]) > 0.0f)) tot = 0.0f;
+    from_f32(out[row * F + f], tot);
   }
 }
 
@@ -139,11 +227,35 @@ __global__ void __launch_bounds__(256) aggregate_any(const T* __restrict__ in, T
 }
 
 template <typename T, int LPR, int VPL>
-void launch_vec(const T* in, T* out, const gnnco_handle* h, const float* scale, const T* mask, int F,
-                cudaStream_t st) {
+void launch_vec(const T* in, T* out, gnnco_handle* h, const float* scale, const T* mask, int F, cudaStream_t st) {
   constexpr int ROWS_PER_BLOCK = 256 / LPR;
-  unsigned grid = (unsigned)((h->n + ROWS_PER_BLOCK - 1) / ROWS_PER_BLOCK);
-  aggregate_vec<T, LPR, VPL><<<grid, 256, 0, st>>>(in, out, h->rowptr, h->colidx, scale, mask, h->n, F);
+  const unsigned main_blocks = (unsigned)((h->n + ROWS_PER_BLOCK - 1) / ROWS_PER_BLOCK);
+  if (h->n_long == 0) {
+    aggregate_vec<T, LPR, VPL><<<main_blocks, 256, 0, st>>>(in, out, h->row_head, h->colidx, scale, mask, h->n, F, 0);
+    return;
+  }
+  // A single warp walks a row of max_row entries in about max_row/4 dependent round trips of
+  // roughly a microsecond.  When streaming all rows takes several times longer than that, the
+  // long rows stay where they are (scattered through the grid, each a lightweight warp that
+  // overlaps with the streaming of its neighbours); otherwise (small or hub-dominated graphs,
+  // where one such walk would be the tail of the kernel) they get a block each, on a side
+  // stream, beside the short rows.
+  const double stream_us = 2.0 * (double)h->n * F * sizeof(T) / 4.0e6;          // at ~4 TB/s
+  const double walk_us = (double)h->max_row / 4.0;
+  const bool inline_first = stream_us > 3.0 * walk_us;
+  if (inline_first) {
+    aggregate_vec<T, LPR, VPL><<<main_blocks, 256, 0, st>>>(in, out, h->row_head, h->colidx, scale, mask, h->n, F, 0);
+    return;
+  }
+  const bool fork = h->side_stream && h->ev_fork && h->ev_join && cudaEventRecord(h->ev_fork, st) == cudaSuccess &&
+                    cudaStreamWaitEvent(h->side_stream, h->ev_fork, 0) == cudaSuccess;
+  cudaStream_t ls = fork ? h->side_stream : st;
+  aggregate_long_row<T, LPR, VPL><<<h->n_long, 256, (size_t)(256 / LPR) * F * sizeof(float), ls>>>(
+      in, out, h->rowptr, h->colidx, scale, mask, h->long_rows, F);
+  h->launches += 1;
+  if (fork) cudaEventRecord(h->ev_join, h->side_stream);
+  aggregate_vec<T, LPR, VPL><<<main_blocks, 256, 0, st>>>(in, out, h->row_head, h->colidx, scale, mask, h->n, F, 1);
+  if (fork) cudaStreamWaitEvent(st, h->ev_join, 0);
 }
 
 template <typename T>

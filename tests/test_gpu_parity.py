@@ -28,6 +28,7 @@ GRAPHS = {
     "empty_parts": lambda: (lambda g: (g[0], g[1], np.where(g[2] == 3, 2, g[2]).astype(np.int32)))(
         tiny_graph(120, 0.08, 6, seed=6)),
     "hub_and_isolated": lambda: _star_plus_isolated(300) + (np.zeros(300, np.int32),),
+    "big_hub": lambda: _star_plus_isolated(1100) + (np.zeros(1100, np.int32),),     # hub row of 549 entries
     "no_edges": lambda: (np.zeros(0, np.int32), np.zeros(0, np.int32), si.contiguous_partition(50, 4)),
     "dense_small": lambda: tiny_graph(90, 0.5, 2, seed=8, contiguous=True),
 }
@@ -82,6 +83,9 @@ STEP_CASES = [
     ("empty_parts", [12, 12, 1], None, 0.3),
     ("hub_and_isolated", [32, 16, 1], None, 0.0),
     ("hub_and_isolated", [256, 8, 1], None, 0.0),
+    ("big_hub", [32, 16, 1], None, 0.0),
+    ("big_hub", [128, 8, 1], None, 0.0),
+    ("big_hub", [256, 12, 1], None, 0.4),
     ("no_edges", [4, 4, 1], None, 0.0),
     ("dense_small", [24, 40, 1], None, 0.2),
     ("dense_small", [130, 70, 1], None, 0.0),
@@ -216,3 +220,16 @@ def test_train_step_bf16_long_subgraphs(dims, n, S):
     case = StepCase(book, dims, "bf16", S, lam=0.0)
     adam = dict(lr=1e-3, step=2, m=[np.zeros_like(w) for w in W], v=[np.zeros_like(w) for w in W])
     case.run(graph, X, W, None, want_dx=True, adam=adam, label="bf16-long")
+
+
+@pytest.mark.parametrize("dims", [[256, 64, 1], [64, 64, 1], [512, 64, 1]])
+def test_train_step_bf16_hub_row(dims):
+    """A hub row longer than the block-per-row threshold, bf16 features."""
+    eu, ev, part = GRAPHS["big_hub"]()
+    n, S = _n_S(part)
+    book = oracle.bookkeeping(n, eu, ev, part, S)
+    graph = load_graph(n, eu, ev, part, S)
+    assert graph.max_row > 256
+    X = si.round_to_bf16(rand_features(n, dims[0], 31).astype(np.float32))
+    W = [si.round_to_bf16(w.astype(np.float32)) for w in rand_weights(dims, S, 37)]
+    StepCase(book, dims, "bf16", S).run(graph, X, W, None, want_dx=True, label="bf16-hub")
