@@ -185,6 +185,24 @@ __global__ void __launch_bounds__(256) rank1_masked_kernel(const float* __restri
   st(dZ + t, v);
 }
 
+// float32, 4 features per thread (F a multiple of 4, 16-byte aligned rows)
+__global__ void __launch_bounds__(256) rank1_masked_f32x4(const float* __restrict__ g, const float* __restrict__ w,
+                                                          int64_t w_stride, const int32_t* __restrict__ node_part,
+                                                          const float* __restrict__ H, float* __restrict__ dZ,
+                                                          int64_t n, int F) {
+  const int64_t t = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+  const int groups = F >> 2;
+  if (t >= n * groups) return;
+  const int64_t i = t / groups;
+  const int f = (int)(t - i * groups) << 2;
+  const float gi = __ldg(g + i);
+  const float4 wv = __ldg(reinterpret_cast<const float4*>(w + (int64_t)node_part[i] * w_stride + f));
+  float4 hv = make_float4(1.f, 1.f, 1.f, 1.f);
+  if (H) hv = __ldg(reinterpret_cast<const float4*>(H + i * F + f));
+  *reinterpret_cast<float4*>(dZ + i * F + f) = make_float4(hv.x > 0.f ? gi * wv.x : 0.f, hv.y > 0.f ? gi * wv.y : 0.f,
+                                                           hv.z > 0.f ? gi * wv.z : 0.f, hv.w > 0.f ? gi * wv.w : 0.f);
+}
+
 // bf16, 8 features per thread (F a multiple of 8, 16-byte aligned rows)
 __global__ void __launch_bounds__(256) rank1_masked_bf16x8(const float* __restrict__ g,
                                                            const __nv_bfloat16* __restrict__ w, int64_t w_stride,
@@ -331,7 +349,10 @@ int32_t launch_rank1_masked(gnnco_handle* h, int dtype, const float* g, const vo
                             void* dZ, int F, cudaStream_t stream) {
   ProfScope prof_(h, K_RANK1, stream);
   unsigned grid = blocks_for(h->n * F, 256);
-  if (dtype == GNNCO_F32)
+  if (dtype == GNNCO_F32 && F % 4 == 0 && w_stride % 4 == 0 && !(((uintptr_t)w | (uintptr_t)H | (uintptr_t)dZ) & 15))
+    rank1_masked_f32x4<<<blocks_for(h->n * (F / 4), 256), 256, 0, stream>>>(g, (const float*)w, w_stride, h->node_part,
+                                                                            (const float*)H, (float*)dZ, h->n, F);
+  else if (dtype == GNNCO_F32)
     rank1_masked_kernel<float, float><<<grid, 256, 0, stream>>>(g, (const float*)w, w_stride, h->node_part,
                                                                 (const float*)H, (float*)dZ, h->n, F);
   else if (dtype == GNNCO_BF16 && F % 8 == 0 && w_stride % 8 == 0 &&

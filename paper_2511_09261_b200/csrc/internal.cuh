@@ -145,6 +145,18 @@ int32_t launch_weight_grad_tc(gnnco_handle* h, const void* A, const void* G, flo
 int32_t launch_cast_transpose_bf16(gnnco_handle* h, const float* W, __nv_bfloat16* Wt, int K, int N, int32_t sets,
                                    cudaStream_t st);
 
+// ---- tc_gemm_f32.cu : tensor-core path for float32 features (operands split into three bf16 limbs)
+bool tc_f32_transform_supported(int K, int N);
+bool tc_f32_weight_grad_supported(int K, int N);
+int32_t launch_transform_tc_f32(gnnco_handle* h, const void* A, const void* B_limbs, int64_t b_stride,
+                                int64_t b_limb_stride, void* Y, int K, int N, bool relu, const float* row_scale,
+                                bool backward, const void* dot_w, int64_t dot_stride, float* dot_out, cudaStream_t st);
+int32_t launch_weight_grad_tc_f32(gnnco_handle* h, const void* A, const void* G, float* dW, int K, int N,
+                                  cudaStream_t st);
+// three bf16 limb copies of W [sets x K x N] (transposed: [sets x N x K]); limb l at out + l*sets*K*N
+int32_t launch_cast_split3(gnnco_handle* h, const float* W, __nv_bfloat16* out, int K, int N, int32_t sets,
+                           bool transpose, cudaStream_t st);
+
 // ---- chain.cu : the width-1 part of the step
 int32_t launch_output_forward(gnnco_handle* h, const float* u, float* z, float* p, cudaStream_t st);
 int32_t launch_objective(gnnco_handle* h, const float* p, const float* pen, float alpha, float beta, float lambda,

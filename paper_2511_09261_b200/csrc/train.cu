@@ -28,6 +28,8 @@ struct TrainLayout {
   float* dW_sets;                     // per-subgraph partials when the model shares one weight set
   __nv_bfloat16* W_lp[GNNCO_MAX_LAYERS];   // bf16 copies of the weights (bf16 features only)
   __nv_bfloat16* W_lp_t[GNNCO_MAX_LAYERS]; // transposed bf16 copies [sets x F_out x F_in] for the tensor-core forward
+  __nv_bfloat16* W3[GNNCO_MAX_LAYERS];     // float32 features: three bf16 limbs of W (input-gradient operand)
+  __nv_bfloat16* W3_t[GNNCO_MAX_LAYERS];   // ... and of W^T (forward operand)
   // host-variant staging
   void* X_stage;
   float *pen_stage, *loss_stage, *p_stage;
@@ -86,6 +88,13 @@ TrainLayout carve_train(const gnnco_handle* h, const gnnco_model_desc* m, uint32
   for (int l = 0; l + 1 < L; ++l)
     if (tc_transform_supported(m->feat_dtype, m->dims[l], m->dims[l + 1]))
       T.W_lp_t[l] = c.take<__nv_bfloat16>((size_t)m->dims[l] * m->dims[l + 1] * m->weight_sets);
+  if (m->feat_dtype == GNNCO_F32)
+    for (int l = 0; l + 1 < L; ++l) {
+      const size_t wc3 = (size_t)3 * m->dims[l] * m->dims[l + 1] * m->weight_sets;
+      if (tc_f32_transform_supported(m->dims[l], m->dims[l + 1])) T.W3_t[l] = c.take<__nv_bfloat16>(wc3);
+      if (!(flags & GNNCO_FORWARD_ONLY) && tc_f32_transform_supported(m->dims[l + 1], m->dims[l]))
+        T.W3[l] = c.take<__nv_bfloat16>(wc3);
+    }
   if (host) {
     T.X_stage = c.take<char>(n * m->dims[0] * es);
     T.pen_stage = c.take<float>(n);
@@ -117,6 +126,10 @@ int32_t run_step(gnnco_handle* h, const gnnco_model_desc* m, const void* X, cons
         GNNCO_TRY(launch_cast_transpose_bf16(h, m->W[l], T.W_lp_t[l], m->dims[l], m->dims[l + 1], sets, st));
     } else {
       Wc[l] = m->W[l];
+      if (T.W3_t[l]) GNNCO_TRY(launch_cast_split3(h, m->W[l], T.W3_t[l], m->dims[l], m->dims[l + 1], sets, true, st));
+      const bool need_bwd = !(flags & GNNCO_FORWARD_ONLY) && (l > 0 || (flags & GNNCO_WANT_DX));
+      if (T.W3[l] && need_bwd)
+        GNNCO_TRY(launch_cast_split3(h, m->W[l], T.W3[l], m->dims[l], m->dims[l + 1], sets, false, st));
     }
   }
   // ---- forward
@@ -129,6 +142,13 @@ int32_t run_step(gnnco_handle* h, const gnnco_model_desc* m, const void* X, cons
       const bool fuse = (l == L - 1) && (m->dims[l] % 8 == 0);
       GNNCO_TRY(launch_transform_tc(h, T.M[l], T.W_lp_t[l - 1], wstride[l - 1], T.H[l], m->dims[l - 1], m->dims[l], true,
                                     nullptr, false, fuse ? Wc[L - 1] : nullptr, wstride[L - 1], fuse ? T.u : nullptr, st));
+      u_done = fuse;
+    } else if (T.W3_t[l - 1]) {
+      const bool fuse = (l == L - 1) && (m->dims[l] % 4 == 0);
+      GNNCO_TRY(launch_transform_tc_f32(h, T.M[l], T.W3_t[l - 1], wstride[l - 1],
+                                        (int64_t)m->dims[l - 1] * m->dims[l] * sets, T.H[l], m->dims[l - 1], m->dims[l],
+                                        true, nullptr, false, fuse ? Wc[L - 1] : nullptr, wstride[L - 1],
+                                        fuse ? T.u : nullptr, st));
       u_done = fuse;
     } else
       GNNCO_TRY(launch_transform(h, dt, T.M[l], Wc[l - 1], wstride[l - 1], T.H[l], m->dims[l - 1], m->dims[l], false,
@@ -183,12 +203,17 @@ int32_t run_step(gnnco_handle* h, const gnnco_model_desc* m, const void* X, cons
       if (tc_transform_supported(dt, N, K))
         GNNCO_TRY(launch_transform_tc(h, dZ, Wc[l - 1], wstride[l - 1], other, N, K, false, h->inv_deg, true, nullptr, 0,
                                       nullptr, st));
+      else if (T.W3[l - 1])
+        GNNCO_TRY(launch_transform_tc_f32(h, dZ, T.W3[l - 1], wstride[l - 1], (int64_t)K * N * sets, other, N, K, false,
+                                          h->inv_deg, true, nullptr, 0, nullptr, st));
       else
         GNNCO_TRY(launch_transform(h, dt, dZ, Wc[l - 1], wstride[l - 1], other, N, K, true, false, h->inv_deg, st));
     }
     float* target = grad_target(l - 1);
     float* wg_out = sets == 1 ? T.dW_sets : target;
     if (tc_weight_grad_supported(dt, K, N)) GNNCO_TRY(launch_weight_grad_tc(h, T.M[l], dZ, wg_out, K, N, st));
+    else if (dt == GNNCO_F32 && tc_f32_weight_grad_supported(K, N))
+      GNNCO_TRY(launch_weight_grad_tc_f32(h, T.M[l], dZ, wg_out, K, N, st));
     else GNNCO_TRY(launch_weight_grad(h, dt, T.M[l], dZ, wg_out, K, N, st));
     if (sets == 1) GNNCO_TRY(launch_sum_over_sets(h, T.dW_sets, target, (int64_t)K * N, h->S, st));
     GNNCO_TRY(finish_layer(l - 1, target));

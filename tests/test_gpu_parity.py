@@ -233,3 +233,23 @@ def test_train_step_bf16_hub_row(dims):
     X = si.round_to_bf16(rand_features(n, dims[0], 31).astype(np.float32))
     W = [si.round_to_bf16(w.astype(np.float32)) for w in rand_weights(dims, S, 37)]
     StepCase(book, dims, "bf16", S).run(graph, X, W, None, want_dx=True, label="bf16-hub")
+
+
+@pytest.mark.parametrize("dims,n,S,sets", [([128, 128, 128, 1], 2300, 5, None), ([128, 64, 1], 1500, 2, None),
+                                           ([64, 128, 64, 1], 900, 4, None), ([64, 64, 1], 700, 1, None),
+                                           ([128, 128, 1], 1000, 3, 1)])
+def test_train_step_f32_tensor_core_widths(dims, n, S, sets):
+    """float32 features at widths the tensor-core path takes (operands split into bf16 limbs):
+    the result must still meet the float32 tolerance."""
+    eu, ev, part = tiny_graph(n, 5.0 / n, S, seed=41)
+    book = oracle.bookkeeping(n, eu, ev, part, S)
+    graph = load_graph(n, eu, ev, part, S)
+    X = rand_features(n, dims[0], 43).astype(np.float32)
+    nsets = S if sets is None else sets
+    W = [w.astype(np.float32) for w in rand_weights(dims, nsets, 47, scale=1.5)]
+    pen = (si.uniform01(5, 0, n) < 0.2).astype(np.float32)
+    case = StepCase(book, dims, "f32", nsets, lam=0.3)
+    adam = dict(lr=1e-3, step=4, m=[0.01 * rand_weights(dims, nsets, 51)[l].astype(np.float32) for l in range(len(W))],
+                v=[np.square(0.02 * rand_weights(dims, nsets, 52)[l]).astype(np.float32) for l in range(len(W))])
+    g, stats = case.run(graph, X, W, pen, want_dx=True, adam=adam, label="f32-tc")
+    print({k: float("%.3g" % v) for k, v in stats.items()})
