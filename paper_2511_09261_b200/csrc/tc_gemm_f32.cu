@@ -6,7 +6,10 @@
 // is rebuilt from the six limb products whose weight is at least 2^-16 of the leading one:
 //     a*b ~= a1 b1 + (a1 b2 + a2 b1) + (a1 b3 + a2 b2 + a3 b1)
 // accumulated in float32 in TMEM.  What is dropped is below 2^-24 relative, i.e. float32
-// rounding level, so results meet the float32 tolerance.  Six bf16 MMAs cost as much tensor
+// rounding level, so results meet the float32 tolerance.  The leading products a1 b1 go to one
+// accumulator and the five correction products to a second one, added once in the epilogue:
+// every MMA rounds the running sum it adds to, and keeping the 5x more numerous corrections
+// away from the large sum cuts the accumulated rounding error several times (measured).  Six bf16 MMAs cost as much tensor
 // time as three tf32 ones and keep these kernels memory-bound at the widths in use (<= 128).
 //
 // Activations are split on the fly by the threads that stage them into shared memory; the
@@ -91,7 +94,7 @@ transform_tc_f32(const float* __restrict__ A, const __nv_bfloat16* __restrict__ 
     *abort_flag = 0;
     tc::fence_mbar_init();
   }
-  if (warp == 0) tc::tmem_alloc(tmem_slot, 2 * NDIM);
+  if (warp == 0) tc::tmem_alloc(tmem_slot, 4 * NDIM);   // two buffers x (leading, correction) accumulators
   tc::tc_fence_before_sync();
   __syncthreads();
   tc::tc_fence_after_sync();
@@ -170,7 +173,8 @@ transform_tc_f32(const float* __restrict__ A, const __nv_bfloat16* __restrict__ 
               const int lb = pr == 0 ? 0 : pr == 1 ? 1 : pr == 2 ? 2 : pr == 3 ? 0 : pr == 4 ? 1 : 0;
               const uint64_t ad = tc::smem_desc_sw128(sA + kb * A_SLOT + la * A_LIMB + ks * 32, 16, 1024);
               const uint64_t bd = tc::smem_desc_sw128(sB + kb * B_SLOT + lb * B_LIMB + ks * 32, 16, 1024);
-              tc::mma_bf16(tmem + buf * NDIM, ad, bd, IDESC, (kb | ks | pr) != 0);
+              if (pr == 5) tc::mma_bf16(tmem + buf * 2 * NDIM, ad, bd, IDESC, (kb | ks) != 0);
+              else tc::mma_bf16(tmem + buf * 2 * NDIM + NDIM, ad, bd, IDESC, (kb | ks | pr) != 0);
             }
           tc::mma_commit(empty + kb);
           if (kb == KB - 1) tc::mma_commit(acc_full + buf);
@@ -195,12 +199,13 @@ transform_tc_f32(const float* __restrict__ A, const __nv_bfloat16* __restrict__ 
       const int rows_here = rows - warp * 32;
 #pragma unroll 1
       for (int c0 = 0; c0 < NDIM; c0 += 32) {
-        uint32_t r[32];
-        tc::tmem_ld_32x32(tmem + ((uint32_t)(warp * 32) << 16) + buf * NDIM + c0, r);
+        uint32_t r[32], rs[32];
+        tc::tmem_ld_32x32(tmem + ((uint32_t)(warp * 32) << 16) + buf * 2 * NDIM + c0, r);
+        tc::tmem_ld_32x32(tmem + ((uint32_t)(warp * 32) << 16) + buf * 2 * NDIM + NDIM + c0, rs);
         tc::tmem_ld_wait();
 #pragma unroll
         for (int q = 0; q < 32; ++q) {
-          float a = __uint_as_float(r[q]) * s;
+          float a = (__uint_as_float(r[q]) + __uint_as_float(rs[q])) * s;
           if (relu) a = a > 0.0f ? a : 0.0f;
           r[q] = __float_as_uint(a);
         }
@@ -235,7 +240,7 @@ transform_tc_f32(const float* __restrict__ A, const __nv_bfloat16* __restrict__ 
   if (*abort_flag && threadIdx.x == 0) atomicMin(status, (int32_t)GNNCO_INTERNAL);
   tc::tc_fence_before_sync();
   __syncthreads();
-  if (warp == 0) tc::tmem_dealloc(tmem, 2 * NDIM);
+  if (warp == 0) tc::tmem_dealloc(tmem, 4 * NDIM);
 }
 
 template <int KDIM, int NDIM>
@@ -272,7 +277,7 @@ weight_grad_tc_f32(const float* __restrict__ A, const float* __restrict__ G, flo
   constexpr uint32_t A_LIMB = KF * 128, G_LIMB = NF * 128;            // 64 rows x (DIM/64 blocks of 128 B)
   constexpr uint32_t STAGE = 3 * (A_LIMB + G_LIMB);
   constexpr int STAGES = 2;
-  constexpr uint32_t TMEM_COLS = NF < 32 ? 32 : NF;
+  constexpr uint32_t TMEM_COLS = 2 * NF;                  // leading and correction accumulators
   extern __shared__ uint8_t smem_raw[];
   const uint32_t sbase = (tc::smem_u32(smem_raw) + 1023u) & ~1023u;
   uint8_t* gen_base = smem_raw + (sbase - tc::smem_u32(smem_raw));
@@ -360,7 +365,8 @@ weight_grad_tc_f32(const float* __restrict__ A, const float* __restrict__ G, flo
           const int lb = pr == 0 ? 0 : pr == 1 ? 1 : pr == 2 ? 2 : pr == 3 ? 0 : pr == 4 ? 1 : 0;
           const uint64_t ad = tc::smem_desc_sw128(sb + la * A_LIMB + j * 2048, kWgRows * 128, 1024);
           const uint64_t gd = tc::smem_desc_sw128(sb + 3 * A_LIMB + lb * G_LIMB + j * 2048, kWgRows * 128, 1024);
-          tc::mma_bf16(tmem, ad, gd, IDESC, (it | j | pr) != 0);
+          if (pr == 5) tc::mma_bf16(tmem, ad, gd, IDESC, (it | j) != 0);
+          else tc::mma_bf16(tmem + NF, ad, gd, IDESC, (it | j | pr) != 0);
         }
       tc::mma_commit(bars + slot);
       if (it == iters - 1) tc::mma_commit(bars + STAGES);
@@ -380,9 +386,12 @@ weight_grad_tc_f32(const float* __restrict__ A, const float* __restrict__ G, flo
     const int f = lg * 32 + lane;
 #pragma unroll
     for (int c0 = 0; c0 < HALF; c0 += 32) {
-      uint32_t r[32];
+      uint32_t r[32], rs[32];
       tc::tmem_ld_32x32(tmem + ((uint32_t)(lg * 32) << 16) + ch * HALF + c0, r);
+      tc::tmem_ld_32x32(tmem + ((uint32_t)(lg * 32) << 16) + NF + ch * HALF + c0, rs);
       tc::tmem_ld_wait();
+#pragma unroll
+      for (int q = 0; q < 32; ++q) r[q] = __float_as_uint(__uint_as_float(r[q]) + __uint_as_float(rs[q]));
       uint4* dst = reinterpret_cast<uint4*>(out + (int64_t)f * NF + ch * HALF + c0);
 #pragma unroll
       for (int j = 0; j < 8; ++j) dst[j] = make_uint4(r[4 * j], r[4 * j + 1], r[4 * j + 2], r[4 * j + 3]);
