@@ -158,6 +158,59 @@ __global__ void __launch_bounds__(256) gemv_rows(const TA* __restrict__ H, const
   if (lane == 0) u[row] = acc;
 }
 
+// dw[s][:] = sum_{i in s} H[i,:] g[i].  One block per subgraph; LPR lanes cover a row with
+// 16-byte loads, the 256/LPR row groups walk the subgraph's rows interleaved (four rows in
+// flight each) and meet in shared memory in a fixed order.
+template <typename TA, int LPR>
+__global__ void __launch_bounds__(256) weight_grad_vec_rows(const TA* __restrict__ H, const float* __restrict__ g,
+                                                            float* __restrict__ dw, int F,
+                                                            const int32_t* __restrict__ part_ptr) {
+  constexpr int VN = 16 / sizeof(TA);
+  constexpr int RG = 256 / LPR;
+  extern __shared__ float partial[];                       // [RG][F]
+  const int s = blockIdx.x;
+  const int sub = threadIdx.x % LPR, rg = threadIdx.x / LPR;
+  const int64_t ra = part_ptr[s], rb = part_ptr[s + 1];
+  float acc[VN];
+#pragma unroll
+  for (int e = 0; e < VN; ++e) acc[e] = 0.0f;
+  auto fma_row = [&](const uint4& v, float gi) {
+    if (sizeof(TA) == 4) {
+      acc[0] = fmaf(__uint_as_float(v.x), gi, acc[0]); acc[1] = fmaf(__uint_as_float(v.y), gi, acc[1]);
+      acc[2] = fmaf(__uint_as_float(v.z), gi, acc[2]); acc[3] = fmaf(__uint_as_float(v.w), gi, acc[3]);
+    } else {
+      const uint32_t w[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+      for (int k = 0; k < 4; ++k) {
+        acc[(2 * k) % VN] = fmaf(__uint_as_float(w[k] << 16), gi, acc[(2 * k) % VN]);
+        acc[(2 * k + 1) % VN] = fmaf(__uint_as_float(w[k] & 0xffff0000u), gi, acc[(2 * k + 1) % VN]);
+      }
+    }
+  };
+  int64_t i = ra + rg;
+  for (; i + 3 * RG < rb; i += 4 * RG) {
+    uint4 v[4];
+    float gi[4];
+#pragma unroll
+    for (int u = 0; u < 4; ++u) {
+      v[u] = __ldg(reinterpret_cast<const uint4*>(H + (i + u * RG) * F + sub * VN));
+      gi[u] = __ldg(g + i + u * RG);
+    }
+#pragma unroll
+    for (int u = 0; u < 4; ++u) fma_row(v[u], gi[u]);
+  }
+  for (; i < rb; i += RG) fma_row(__ldg(reinterpret_cast<const uint4*>(H + i * F + sub * VN)), __ldg(g + i));
+#pragma unroll
+  for (int e = 0; e < VN; ++e) partial[rg * F + sub * VN + e] = acc[e];
+  __syncthreads();
+  for (int f = threadIdx.x; f < F; f += 256) {
+    float tot = 0.0f;
+    for (int r = 0; r < RG; ++r) tot += partial[r * F + f];
+    dw[(int64_t)s * F + f] = tot;
+  }
+}
+
+// any width: one thread per column
 template <typename TA>
 __global__ void __launch_bounds__(256) weight_grad_vec_kernel(const TA* __restrict__ H, const float* __restrict__ g,
                                                               float* __restrict__ dw, int F,
@@ -332,14 +385,30 @@ int32_t launch_weight_grad(gnnco_handle* h, int dtype, const void* A, const void
 int32_t launch_weight_grad_vec(gnnco_handle* h, int dtype, const void* H, const float* g, float* dw, int F,
                                cudaStream_t stream) {
   ProfScope prof_(h, K_WEIGHT_GRAD_VEC, stream);
-  dim3 grid(h->S, (F + 255) / 256);
-  if (grid.y > 65535) return GNNCO_UNSUPPORTED;
-  if (dtype == GNNCO_F32)
-    weight_grad_vec_kernel<float><<<grid, 256, 0, stream>>>((const float*)H, g, dw, F, h->part_ptr);
-  else if (dtype == GNNCO_BF16)
-    weight_grad_vec_kernel<__nv_bfloat16><<<grid, 256, 0, stream>>>((const __nv_bfloat16*)H, g, dw, F, h->part_ptr);
-  else
-    return GNNCO_UNSUPPORTED;
+  const int vn = dtype == GNNCO_BF16 ? 8 : 4;
+  const int lpr = F % vn == 0 ? F / vn : 0;
+  const bool aligned = !((uintptr_t)H & 15);
+  const size_t sm = (size_t)(lpr ? 256 / lpr : 0) * F * sizeof(float);
+#define GNNCO_WGV(TT, L)                                                                                     \
+  weight_grad_vec_rows<TT, L><<<h->S, 256, sm, stream>>>((const TT*)H, g, dw, F, h->part_ptr)
+  bool done = aligned && (lpr == 8 || lpr == 16 || lpr == 32 || lpr == 64);
+  if (done && dtype == GNNCO_F32) {
+    if (lpr == 8) GNNCO_WGV(float, 8); else if (lpr == 16) GNNCO_WGV(float, 16);
+    else if (lpr == 32) GNNCO_WGV(float, 32); else GNNCO_WGV(float, 64);
+  } else if (done && dtype == GNNCO_BF16) {
+    if (lpr == 8) GNNCO_WGV(__nv_bfloat16, 8); else if (lpr == 16) GNNCO_WGV(__nv_bfloat16, 16);
+    else if (lpr == 32) GNNCO_WGV(__nv_bfloat16, 32); else GNNCO_WGV(__nv_bfloat16, 64);
+  } else {
+    dim3 grid(h->S, (F + 255) / 256);
+    if (grid.y > 65535) return GNNCO_UNSUPPORTED;
+    if (dtype == GNNCO_F32)
+      weight_grad_vec_kernel<float><<<grid, 256, 0, stream>>>((const float*)H, g, dw, F, h->part_ptr);
+    else if (dtype == GNNCO_BF16)
+      weight_grad_vec_kernel<__nv_bfloat16><<<grid, 256, 0, stream>>>((const __nv_bfloat16*)H, g, dw, F, h->part_ptr);
+    else
+      return GNNCO_UNSUPPORTED;
+  }
+#undef GNNCO_WGV
   h->launches += 1;
   GNNCO_LAUNCH_CHECK();
   return GNNCO_OK;
