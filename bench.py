@@ -202,6 +202,21 @@ def algorithmic_bytes(kind, w, n, nnz, S):
     return float(per.get(kind, 0.0))
 
 
+def max_over_ranks(dist, value: float, device) -> float:
+    """Max of a per-rank scalar over all ranks (identity without a process group)."""
+    if dist is None:
+        return float(value)
+    import torch
+    t = torch.tensor([value], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def whole_job_value(edges_per_replica: int, world: int, ms_per_step: float) -> float:
+    """Replicas only: every rank trains its own copy, so the job's rate is the sum."""
+    return world * edges_per_replica / (ms_per_step * 1e-3)
+
+
 # ------------------------------------------------------------------------------ our arm
 def run_ours(args):
     import torch
@@ -295,12 +310,9 @@ def run_ours(args):
     if dist is not None:
         dist.barrier()
     total_ms = sum(s.elapsed_time(e) for s, e in zip(starts, ends))
-    if dist is not None:
-        t = torch.tensor([total_ms], dtype=torch.float64, device=dev)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        total_ms = float(t.item())
+    total_ms = max_over_ranks(dist, total_ms, dev)
     ms_per_step = total_ms / args.steps
-    value = world * graph.E_in / (ms_per_step * 1e-3)
+    value = whole_job_value(graph.E_in, world, ms_per_step)
 
     # ---- per-kernel shares and the dominant kernel's roofline
     nnz = 2 * graph.E_in
@@ -346,10 +358,7 @@ def run_ours(args):
             step_host()
         torch.cuda.synchronize()
         dt = time.perf_counter() - t0
-        if dist is not None:
-            t = torch.tensor([dt], dtype=torch.float64, device=dev)
-            dist.all_reduce(t, op=dist.ReduceOp.MAX)
-            dt = float(t.item())
+        dt = max_over_ranks(dist, dt, dev)
         h2d = Xh.numel() * Xh.element_size() + pen_h.numel() * 4 + p_h.numel() * 4
         d2h = loss_h.numel() * 4 + p_h.numel() * 4 + 24
         e2e = dict(value=world * graph.E_in * n_e2e / dt, unit="edges/s", h2d_bytes_per_step=h2d,
