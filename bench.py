@@ -326,7 +326,7 @@ def run_ours(args):
     top = max(prof.items(), key=lambda kv: kv[1][1])[0]
     achieved = kern[top]["algo_GBs"]
     roofline = dict(bound="hbm", kernel=top, achieved=achieved, peak=peak, unit="GB/s",
-                    frac=round(achieved / peak, 4), traffic=TRAFFIC_BYTES.get((args.config, top)),
+                    frac=round(achieved / peak, 4), traffic=TRAFFIC_BYTES.get((args.config, top)) if args.scale == 1.0 else None,
                     peak_source="%s (MEASURED_PEAKS.json hbm_gbs)" % peak_src if peak_src == "measured" else "fallback",
                     algorithmic_bytes_per_launch=algorithmic_bytes(top, w, w.n, nnz, w.S))
     agg = {k: kern[k] for k in ("aggregate_fwd", "aggregate_bwd") if k in kern}
@@ -384,9 +384,16 @@ def run_ours(args):
         dist.destroy_process_group()
 
 
-# DRAM traffic per launch (dram__bytes_read.sum + dram__bytes_write.sum) taken from ncu captures
-# of the kernel families as they stand; None until a capture of the current kernel exists.
-TRAFFIC_BYTES = {}
+# DRAM traffic per launch (dram__bytes_read.sum + dram__bytes_write.sum) from ncu captures of the
+# kernels as they stand, taken on configuration 5 at one tenth of the size and scaled by 10 (the
+# traffic is proportional to the node count); an entry is removed when its kernel changes.
+TRAFFIC_BYTES = {
+    (5, "aggregate_bwd"): 15.37e9,
+    (5, "aggregate_fwd"): 10.07e9,
+    (5, "transform_fwd"): 11.53e9,
+    (5, "transform_bwd"): 11.63e9,
+    (5, "weight_grad"): 11.07e9,
+}
 
 
 # ----------------------------------------------------------------------- reference arm
