@@ -26,6 +26,7 @@ constexpr int kEpiWarps = 4;
 constexpr int kMmaWarp = 4;
 constexpr int kProdWarp0 = 5;
 constexpr int kProdLanes = 96;
+constexpr int kBatch = 11;                   // 32-byte source chunks a producer lane has in flight (a whole k-block)
 
 __device__ __forceinline__ uint32_t pack_bf16x2(float a, float b) {
   __nv_bfloat162 v = __floats2bfloat162_rn(a, b);
@@ -121,13 +122,13 @@ transform_tc_f32(const float* __restrict__ A, const __nv_bfloat16* __restrict__ 
                            B + limb * b_limb_stride + (int64_t)part * b_stride + (int64_t)r * KDIM + kb * 64 + cc * 8);
           }
         }
-        // activations: 32 bytes of float32 -> one 16-byte chunk in each limb tile, four chunks in flight
+        // activations: 32 bytes of float32 -> one 16-byte chunk in each limb tile, a whole k-block in flight
         const float* src = A + row0 * KDIM + kb * 64;
         const uint32_t dstA = sA + kb * A_SLOT;
-        for (int q0 = p; q0 < rows * 8; q0 += 4 * kProdLanes) {
-          float4 x[4], y[4];
+        for (int q0 = p; q0 < rows * 8; q0 += kBatch * kProdLanes) {
+          float4 x[kBatch], y[kBatch];
 #pragma unroll
-          for (int u = 0; u < 4; ++u) {
+          for (int u = 0; u < kBatch; ++u) {
             const int q = q0 + u * kProdLanes;
             if (q < rows * 8) {
               const float4* g = reinterpret_cast<const float4*>(src + (int64_t)(q >> 3) * KDIM + (q & 7) * 8);
@@ -136,7 +137,7 @@ transform_tc_f32(const float* __restrict__ A, const __nv_bfloat16* __restrict__ 
             }
           }
 #pragma unroll
-          for (int u = 0; u < 4; ++u) {
+          for (int u = 0; u < kBatch; ++u) {
             const int q = q0 + u * kProdLanes;
             if (q < rows * 8) {
               const int r = q >> 3, cc = q & 7;
