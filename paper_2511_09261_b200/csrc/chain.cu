@@ -22,15 +22,30 @@ __device__ __forceinline__ float row_sum(const float* __restrict__ val, const in
   const int lane = threadIdx.x & 31;
   const bool is_long = active && (r1 - r0 > kLongRow);
   float sum = 0.0f;
-  if (active && !is_long)
-    for (int32_t k = r0; k < r1; ++k) sum += __ldg(val + __ldg(colidx + k));
+  if (active && !is_long) {
+    int32_t k = r0;
+    for (; k + 4 <= r1; k += 4) {           // four independent gathers in flight
+      const int32_t c0 = __ldg(colidx + k), c1 = __ldg(colidx + k + 1), c2 = __ldg(colidx + k + 2),
+                    c3 = __ldg(colidx + k + 3);
+      const float v0 = __ldg(val + c0), v1 = __ldg(val + c1), v2 = __ldg(val + c2), v3 = __ldg(val + c3);
+      sum += (v0 + v1) + (v2 + v3);
+    }
+    for (; k < r1; ++k) sum += __ldg(val + __ldg(colidx + k));
+  }
   uint32_t todo = __ballot_sync(0xffffffffu, is_long);
   while (todo) {
     const int src = __ffs(todo) - 1;
     todo &= todo - 1;
     const int32_t a = __shfl_sync(0xffffffffu, r0, src), b = __shfl_sync(0xffffffffu, r1, src);
     float part = 0.0f;
-    for (int32_t k = a + lane; k < b; k += 32) part += __ldg(val + __ldg(colidx + k));
+    int32_t k = a + lane;
+    for (; k + 96 < b; k += 128) {          // four independent gathers in flight per lane
+      const int32_t c0 = __ldg(colidx + k), c1 = __ldg(colidx + k + 32), c2 = __ldg(colidx + k + 64),
+                    c3 = __ldg(colidx + k + 96);
+      const float v0 = __ldg(val + c0), v1 = __ldg(val + c1), v2 = __ldg(val + c2), v3 = __ldg(val + c3);
+      part += (v0 + v1) + (v2 + v3);
+    }
+    for (; k < b; k += 32) part += __ldg(val + __ldg(colidx + k));
 #pragma unroll
     for (int d = 16; d > 0; d >>= 1) part += __shfl_xor_sync(0xffffffffu, part, d);
     if (lane == src) sum = part;
