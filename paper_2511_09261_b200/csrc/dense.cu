@@ -292,6 +292,18 @@ __global__ void sum_over_sets_kernel(const float* __restrict__ in, float* __rest
   out[q] = acc;
 }
 
+__global__ void wg_combine_kernel(const float* __restrict__ scratch, float* __restrict__ dW, int64_t count,
+                                  const int32_t* __restrict__ mpart, const int32_t* __restrict__ mfirst,
+                                  const int32_t* __restrict__ mcount) {
+  const int64_t q = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+  if (q >= count) return;
+  const int m = blockIdx.y;
+  const float* src = scratch + (int64_t)mfirst[m] * count + q;
+  float acc = 0.0f;
+  for (int32_t c = 0; c < mcount[m]; ++c) acc += src[(int64_t)c * count];
+  dW[(int64_t)mpart[m] * count + q] = acc;
+}
+
 __global__ void cast_bf16_kernel(const float* __restrict__ in, __nv_bfloat16* __restrict__ out, int64_t count) {
   const int64_t q = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
   if (q < count) out[q] = __float2bfloat16_rn(in[q]);
@@ -433,6 +445,17 @@ int32_t launch_rank1_masked(gnnco_handle* h, int dtype, const float* g, const vo
         g, (const __nv_bfloat16*)w, w_stride, h->node_part, (const __nv_bfloat16*)H, (__nv_bfloat16*)dZ, h->n, F);
   else
     return GNNCO_UNSUPPORTED;
+  h->launches += 1;
+  GNNCO_LAUNCH_CHECK();
+  return GNNCO_OK;
+}
+
+int32_t launch_wg_combine(gnnco_handle* h, const float* scratch, float* dW, int64_t count, cudaStream_t stream) {
+  if (h->n_wg_multi == 0) return GNNCO_OK;
+  ProfScope prof_(h, K_WEIGHT_GRAD, stream);
+  dim3 grid(blocks_for(count, 256), h->n_wg_multi);
+  if (grid.y > 65535) return GNNCO_UNSUPPORTED;
+  wg_combine_kernel<<<grid, 256, 0, stream>>>(scratch, dW, count, h->wg_mpart, h->wg_mfirst, h->wg_mcount);
   h->launches += 1;
   GNNCO_LAUNCH_CHECK();
   return GNNCO_OK;

@@ -22,6 +22,7 @@
 
 constexpr int kGemmTileRows = 128;   // rows of one dense-transform tile (never straddles a subgraph)
 constexpr int kLongRowDegree = 256;  // rows with more intra neighbours are aggregated by a whole block
+constexpr int kWgChunkMinRows = 2048; // a subgraph is split for the weight gradient only in runs at least this long
 constexpr int kItemRows = 1024;      // rows of one objective work item (never straddles a subgraph)
 
 // Kernel families, for launch accounting and per-kernel timing.
@@ -64,6 +65,11 @@ struct gnnco_handle {
   int4* row_head = nullptr;                                // {first CSR slot, degree, first two neighbours} per row
   int32_t* long_rows = nullptr;                            // ids of rows with degree > kLongRowDegree
   int32_t n_tiles = 0, n_items = 0, n_long = 0;
+  // weight-gradient work: row ranges, output slot (>= 0 scratch slot, < 0 subgraph -(slot+1)), and the
+  // subgraphs that were split (id, first slot, slot count)
+  int32_t *wg_begin = nullptr, *wg_end = nullptr, *wg_slot = nullptr;
+  int32_t *wg_mpart = nullptr, *wg_mfirst = nullptr, *wg_mcount = nullptr;
+  int32_t n_wg_chunks = 0, n_wg_slots = 0, n_wg_multi = 0;
   std::vector<int32_t> h_part_ptr;
   int64_t launches = 0;
   Profiler prof;
@@ -127,6 +133,8 @@ int32_t launch_weight_grad_vec(gnnco_handle* h, int dtype, const void* H, const 
 // dZ[i,f] = g[i] * w_s[f] where H[i,f] > 0, else 0 (H == nullptr: no mask)
 int32_t launch_rank1_masked(gnnco_handle* h, int dtype, const float* g, const void* w, int64_t w_stride, const void* H,
                             void* dZ, int F, cudaStream_t st);
+// dW[part] = sum of the scratch slots of every split subgraph, in slot order
+int32_t launch_wg_combine(gnnco_handle* h, const float* scratch, float* dW, int64_t count, cudaStream_t st);
 // out[q] = sum_s in[s][q]
 int32_t launch_sum_over_sets(gnnco_handle* h, const float* in, float* out, int64_t count, int32_t sets, cudaStream_t st);
 int32_t launch_cast_bf16(gnnco_handle* h, const float* in, __nv_bfloat16* out, int64_t count, cudaStream_t st);
@@ -140,7 +148,8 @@ int32_t launch_transform_tc(gnnco_handle* h, const void* A, const void* B, int64
                             bool relu, const float* row_scale, bool backward, const void* dot_w, int64_t dot_stride,
                             float* dot_out, cudaStream_t st);
 bool tc_weight_grad_supported(int dtype, int K, int N);
-int32_t launch_weight_grad_tc(gnnco_handle* h, const void* A, const void* G, float* dW, int K, int N, cudaStream_t st);
+int32_t launch_weight_grad_tc(gnnco_handle* h, const void* A, const void* G, float* dW, float* scratch, int K, int N,
+                              cudaStream_t st);
 // Wt[s][n][k] = bf16(W[s][k][n])
 int32_t launch_cast_transpose_bf16(gnnco_handle* h, const float* W, __nv_bfloat16* Wt, int K, int N, int32_t sets,
                                    cudaStream_t st);
@@ -151,8 +160,8 @@ bool tc_f32_weight_grad_supported(int K, int N);
 int32_t launch_transform_tc_f32(gnnco_handle* h, const void* A, const void* B_limbs, int64_t b_stride,
                                 int64_t b_limb_stride, void* Y, int K, int N, bool relu, const float* row_scale,
                                 bool backward, const void* dot_w, int64_t dot_stride, float* dot_out, cudaStream_t st);
-int32_t launch_weight_grad_tc_f32(gnnco_handle* h, const void* A, const void* G, float* dW, int K, int N,
-                                  cudaStream_t st);
+int32_t launch_weight_grad_tc_f32(gnnco_handle* h, const void* A, const void* G, float* dW, float* scratch, int K,
+                                  int N, cudaStream_t st);
 // three bf16 limb copies of W [sets x K x N] (transposed: [sets x N x K]); limb l at out + l*sets*K*N
 int32_t launch_cast_split3(gnnco_handle* h, const float* W, __nv_bfloat16* out, int K, int N, int32_t sets,
                            bool transpose, cudaStream_t st);

@@ -314,6 +314,8 @@ struct PersistentLayout {
   uint8_t* is_boundary;
   int32_t *tile_row0, *tile_rows, *item_row0, *item_row1, *part_item_ptr, *status, *long_rows;
   int4* row_head;
+  int32_t *wg_begin, *wg_end, *wg_slot, *wg_mpart, *wg_mfirst, *wg_mcount;
+  int64_t max_chunks;
   int64_t max_tiles, max_items, max_long;
   size_t bytes;
 };
@@ -342,6 +344,13 @@ PersistentLayout carve_persistent(void* base, int64_t n, int64_t E, int32_t S) {
   L.max_long = 2 * E / kLongRowDegree + 1;
   L.long_rows = c.take<int32_t>(L.max_long);
   L.row_head = c.take<int4>(n);
+  L.max_chunks = (int64_t)S + n / kWgChunkMinRows + 1;
+  L.wg_begin = c.take<int32_t>(L.max_chunks);
+  L.wg_end = c.take<int32_t>(L.max_chunks);
+  L.wg_slot = c.take<int32_t>(L.max_chunks);
+  L.wg_mpart = c.take<int32_t>((size_t)S);
+  L.wg_mfirst = c.take<int32_t>((size_t)S);
+  L.wg_mcount = c.take<int32_t>((size_t)S);
   L.bytes = c.off;
   return L;
 }
@@ -421,6 +430,8 @@ extern "C" int32_t gnnco_partition_load(const gnnco_graph_desc* g, void* persist
   h->inv_deg = P.inv_deg; h->is_boundary = P.is_boundary;
   h->tile_row0 = P.tile_row0; h->tile_rows = P.tile_rows; h->item_row0 = P.item_row0; h->item_row1 = P.item_row1;
   h->part_item_ptr = P.part_item_ptr; h->status = P.status; h->long_rows = P.long_rows; h->row_head = P.row_head;
+  h->wg_begin = P.wg_begin; h->wg_end = P.wg_end; h->wg_slot = P.wg_slot;
+  h->wg_mpart = P.wg_mpart; h->wg_mfirst = P.wg_mfirst; h->wg_mcount = P.wg_mcount;
 
   const int T = 256;
   int32_t hs[kStatusWords];
@@ -509,6 +520,37 @@ extern "C" int32_t gnnco_partition_load(const gnnco_graph_desc* g, void* persist
     }
   }
   pip[S] = (int32_t)i0.size();
+  // weight-gradient chunks: a subgraph is one chunk unless it is so long that too few blocks
+  // would be busy; then it is cut into runs of chunk_rows rows whose partial results meet in a
+  // scratch area (slot >= 0) and are summed in chunk order afterwards.  slot = -(s+1) means
+  // "write subgraph s's result directly".
+  std::vector<int32_t> wb, we, wsl, mp, mf, mc;
+  {
+    int64_t per = (n + 4 * (int64_t)(h->sm_count > 0 ? h->sm_count : 148) - 1) / (4 * (int64_t)(h->sm_count > 0 ? h->sm_count : 148));
+    int64_t chunk_rows = (per + 63) / 64 * 64;
+    if (chunk_rows < kWgChunkMinRows) chunk_rows = kWgChunkMinRows;
+    int32_t slots = 0;
+    for (int32_t s = 0; s < S; ++s) {
+      int32_t a = h->h_part_ptr[s], b2 = h->h_part_ptr[s + 1];
+      if (b2 - a <= chunk_rows) {
+        wb.push_back(a); we.push_back(b2); wsl.push_back(-(s + 1));
+      } else {
+        mp.push_back(s); mf.push_back(slots);
+        int32_t cnt = 0;
+        for (int64_t r = a; r < b2; r += chunk_rows) {
+          wb.push_back((int32_t)r);
+          we.push_back((int32_t)(r + chunk_rows < b2 ? r + chunk_rows : b2));
+          wsl.push_back(slots++);
+          ++cnt;
+        }
+        mc.push_back(cnt);
+      }
+    }
+    h->n_wg_chunks = (int32_t)wb.size();
+    h->n_wg_slots = slots;
+    h->n_wg_multi = (int32_t)mp.size();
+    if (h->n_wg_chunks > P.max_chunks) return GNNCO_INTERNAL;
+  }
   h->n_tiles = (int32_t)t0.size();
   h->n_items = (int32_t)i0.size();
   if (h->n_tiles > P.max_tiles || h->n_items > P.max_items) return GNNCO_INTERNAL;
@@ -521,6 +563,12 @@ extern "C" int32_t gnnco_partition_load(const gnnco_graph_desc* g, void* persist
   GNNCO_CUDA_TRY(up(P.item_row0, i0));
   GNNCO_CUDA_TRY(up(P.item_row1, i1));
   GNNCO_CUDA_TRY(up(P.part_item_ptr, pip));
+  GNNCO_CUDA_TRY(up(P.wg_begin, wb));
+  GNNCO_CUDA_TRY(up(P.wg_end, we));
+  GNNCO_CUDA_TRY(up(P.wg_slot, wsl));
+  GNNCO_CUDA_TRY(up(P.wg_mpart, mp));
+  GNNCO_CUDA_TRY(up(P.wg_mfirst, mf));
+  GNNCO_CUDA_TRY(up(P.wg_mcount, mc));
   GNNCO_CUDA_TRY(cudaMemcpyAsync(hs, P.status, sizeof(hs), cudaMemcpyDeviceToHost, st));
   GNNCO_CUDA_TRY(cudaStreamSynchronize(st));
   if (hs[kStatus] != GNNCO_OK) return hs[kStatus];

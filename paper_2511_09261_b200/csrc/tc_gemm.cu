@@ -258,7 +258,8 @@ __device__ __forceinline__ void stage_mn_major(uint32_t sbase, const __nv_bfloat
 template <int KF, int NF>
 __global__ void __launch_bounds__(kThreads, 1)
 weight_grad_tc(const __nv_bfloat16* __restrict__ A, const __nv_bfloat16* __restrict__ G, float* __restrict__ dW,
-               const int32_t* __restrict__ part_ptr, int32_t* status) {
+               float* __restrict__ scratch, const int32_t* __restrict__ wg_begin,
+               const int32_t* __restrict__ wg_end, const int32_t* __restrict__ wg_slot, int32_t* status) {
   constexpr int MH = KF / 128;                          // accumulator halves of 128 rows
   constexpr uint32_t A_STAGE = KF * 128, G_STAGE = NF * 128;
   constexpr uint32_t STAGE = A_STAGE + G_STAGE;
@@ -270,9 +271,10 @@ weight_grad_tc(const __nv_bfloat16* __restrict__ A, const __nv_bfloat16* __restr
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + kWgStages + 1);
   uint32_t* abort_flag = tmem_slot + 1;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int s = blockIdx.x;
-  const int64_t ra = part_ptr[s], rb = part_ptr[s + 1];
-  float* out = dW + (int64_t)s * KF * NF;
+  // one block per chunk of rows; a chunk writes either a subgraph's result or a scratch slot
+  const int64_t ra = wg_begin[blockIdx.x], rb = wg_end[blockIdx.x];
+  const int32_t slot = wg_slot[blockIdx.x];
+  float* out = slot < 0 ? dW + (int64_t)(-(slot + 1)) * KF * NF : scratch + (int64_t)slot * KF * NF;
   const int iters = (int)((rb - ra + kWgRows - 1) / kWgRows);
   if (iters == 0) {
     for (int q = threadIdx.x; q < KF * NF; q += kThreads) out[q] = 0.0f;
@@ -360,14 +362,14 @@ weight_grad_tc(const __nv_bfloat16* __restrict__ A, const __nv_bfloat16* __restr
 }
 
 template <int KF, int NF>
-int32_t launch_wg(gnnco_handle* h, const void* A, const void* G, float* dW, cudaStream_t st) {
+int32_t launch_wg(gnnco_handle* h, const void* A, const void* G, float* dW, float* scratch, cudaStream_t st) {
   constexpr size_t smem = (size_t)kWgStages * (KF + NF) * 128 + 128 + 1024;
   GNNCO_CUDA_TRY(cudaFuncSetAttribute(weight_grad_tc<KF, NF>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-  weight_grad_tc<KF, NF><<<h->S, kThreads, smem, st>>>((const __nv_bfloat16*)A, (const __nv_bfloat16*)G, dW,
-                                                       h->part_ptr, h->status);
+  weight_grad_tc<KF, NF><<<h->n_wg_chunks, kThreads, smem, st>>>((const __nv_bfloat16*)A, (const __nv_bfloat16*)G, dW,
+                                                                 scratch, h->wg_begin, h->wg_end, h->wg_slot, h->status);
   h->launches += 1;
   GNNCO_LAUNCH_CHECK();
-  return GNNCO_OK;
+  return launch_wg_combine(h, scratch, dW, (int64_t)KF * NF, st);
 }
 
 // W [sets][K][N] float32 -> Wt [sets][N][K] bf16
@@ -415,10 +417,11 @@ bool tc_weight_grad_supported(int dtype, int K, int N) {
 }
 
 // dW[s] (K x N, float32) = sum_{i in s} A[i,:]^T G[i,:], A [n x K], G [n x N] bf16
-int32_t launch_weight_grad_tc(gnnco_handle* h, const void* A, const void* G, float* dW, int K, int N, cudaStream_t st) {
+int32_t launch_weight_grad_tc(gnnco_handle* h, const void* A, const void* G, float* dW, float* scratch, int K, int N,
+                              cudaStream_t st) {
   ProfScope prof_(h, K_WEIGHT_GRAD, st);
 #define GNNCO_WG_CASE(KK, NN) \
-  if (K == KK && N == NN) return launch_wg<KK, NN>(h, A, G, dW, st)
+  if (K == KK && N == NN) return launch_wg<KK, NN>(h, A, G, dW, scratch, st)
   GNNCO_WG_CASE(128, 64); GNNCO_WG_CASE(128, 128); GNNCO_WG_CASE(128, 256);
   GNNCO_WG_CASE(256, 64); GNNCO_WG_CASE(256, 128); GNNCO_WG_CASE(256, 256);
 #undef GNNCO_WG_CASE

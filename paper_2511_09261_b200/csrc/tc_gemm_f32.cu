@@ -273,7 +273,8 @@ constexpr int kWgRows = 64;
 template <int KF, int NF>
 __global__ void __launch_bounds__(kThreads, 1)
 weight_grad_tc_f32(const float* __restrict__ A, const float* __restrict__ G, float* __restrict__ dW,
-                   const int32_t* __restrict__ part_ptr, int32_t* status) {
+                   float* __restrict__ scratch, const int32_t* __restrict__ wg_begin,
+               const int32_t* __restrict__ wg_end, const int32_t* __restrict__ wg_slot, int32_t* status) {
   static_assert(KF == 128, "one 128-lane accumulator");
   constexpr uint32_t A_LIMB = KF * 128, G_LIMB = NF * 128;            // 64 rows x (DIM/64 blocks of 128 B)
   constexpr uint32_t STAGE = 3 * (A_LIMB + G_LIMB);
@@ -286,9 +287,10 @@ weight_grad_tc_f32(const float* __restrict__ A, const float* __restrict__ G, flo
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + STAGES + 1);
   uint32_t* abort_flag = tmem_slot + 1;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int s = blockIdx.x;
-  const int64_t ra = part_ptr[s], rb = part_ptr[s + 1];
-  float* out = dW + (int64_t)s * KF * NF;
+  // one block per chunk of rows; a chunk writes either a subgraph's result or a scratch slot
+  const int64_t ra = wg_begin[blockIdx.x], rb = wg_end[blockIdx.x];
+  const int32_t slot = wg_slot[blockIdx.x];
+  float* out = slot < 0 ? dW + (int64_t)(-(slot + 1)) * KF * NF : scratch + (int64_t)slot * KF * NF;
   const int iters = (int)((rb - ra + kWgRows - 1) / kWgRows);
   if (iters == 0) {
     for (int q = threadIdx.x; q < KF * NF; q += kThreads) out[q] = 0.0f;
@@ -404,16 +406,16 @@ weight_grad_tc_f32(const float* __restrict__ A, const float* __restrict__ G, flo
 }
 
 template <int KF, int NF>
-int32_t launch_wgf(gnnco_handle* h, const void* A, const void* G, float* dW, cudaStream_t st) {
+int32_t launch_wgf(gnnco_handle* h, const void* A, const void* G, float* dW, float* scratch, cudaStream_t st) {
   constexpr size_t smem = (size_t)2 * 3 * (KF + NF) * 128 + 128 + 1024;
   static_assert(smem <= 232448, "stages do not fit in shared memory");
   GNNCO_CUDA_TRY(cudaFuncSetAttribute(weight_grad_tc_f32<KF, NF>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                       (int)smem));
-  weight_grad_tc_f32<KF, NF><<<h->S, kThreads, smem, st>>>((const float*)A, (const float*)G, dW, h->part_ptr,
-                                                           h->status);
+  weight_grad_tc_f32<KF, NF><<<h->n_wg_chunks, kThreads, smem, st>>>((const float*)A, (const float*)G, dW, scratch,
+                                                                     h->wg_begin, h->wg_end, h->wg_slot, h->status);
   h->launches += 1;
   GNNCO_LAUNCH_CHECK();
-  return GNNCO_OK;
+  return launch_wg_combine(h, scratch, dW, (int64_t)KF * NF, st);
 }
 
 // W [sets][K][N] float32 -> three bf16 limb copies, either in place ([sets][K][N]) or
@@ -472,11 +474,11 @@ int32_t launch_transform_tc_f32(gnnco_handle* h, const void* A, const void* B_li
   return GNNCO_UNSUPPORTED;
 }
 
-int32_t launch_weight_grad_tc_f32(gnnco_handle* h, const void* A, const void* G, float* dW, int K, int N,
-                                  cudaStream_t st) {
+int32_t launch_weight_grad_tc_f32(gnnco_handle* h, const void* A, const void* G, float* dW, float* scratch, int K,
+                                  int N, cudaStream_t st) {
   ProfScope prof_(h, K_WEIGHT_GRAD, st);
-  if (K == 128 && N == 64) return launch_wgf<128, 64>(h, A, G, dW, st);
-  if (K == 128 && N == 128) return launch_wgf<128, 128>(h, A, G, dW, st);
+  if (K == 128 && N == 64) return launch_wgf<128, 64>(h, A, G, dW, scratch, st);
+  if (K == 128 && N == 128) return launch_wgf<128, 128>(h, A, G, dW, scratch, st);
   return GNNCO_UNSUPPORTED;
 }
 

@@ -26,6 +26,7 @@ struct TrainLayout {
   float *u, *t, *g, *item_loss;
   float* dW_scratch;                  // one layer's gradient (all sets), when the caller wants none
   float* dW_sets;                     // per-subgraph partials when the model shares one weight set
+  float* wg_scratch;                  // partial weight gradients of subgraphs that were split into row chunks
   __nv_bfloat16* W_lp[GNNCO_MAX_LAYERS];   // bf16 copies of the weights (bf16 features only)
   __nv_bfloat16* W_lp_t[GNNCO_MAX_LAYERS]; // transposed bf16 copies [sets x F_out x F_in] for the tensor-core forward
   __nv_bfloat16* W3[GNNCO_MAX_LAYERS];     // float32 features: three bf16 limbs of W (input-gradient operand)
@@ -81,6 +82,7 @@ TrainLayout carve_train(const gnnco_handle* h, const gnnco_model_desc* m, uint32
     T.Gb = c.take<char>(n * maxw * es);
     T.dW_scratch = c.take<float>(max_wcount * m->weight_sets);
     if (m->weight_sets == 1) T.dW_sets = c.take<float>(max_wcount * (size_t)h->S);
+    T.wg_scratch = c.take<float>(max_wcount * (size_t)h->n_wg_slots + 1);
   }
   if (m->feat_dtype == GNNCO_BF16)
     for (int l = 0; l < L; ++l)
@@ -211,9 +213,9 @@ int32_t run_step(gnnco_handle* h, const gnnco_model_desc* m, const void* X, cons
     }
     float* target = grad_target(l - 1);
     float* wg_out = sets == 1 ? T.dW_sets : target;
-    if (tc_weight_grad_supported(dt, K, N)) GNNCO_TRY(launch_weight_grad_tc(h, T.M[l], dZ, wg_out, K, N, st));
+    if (tc_weight_grad_supported(dt, K, N)) GNNCO_TRY(launch_weight_grad_tc(h, T.M[l], dZ, wg_out, T.wg_scratch, K, N, st));
     else if (dt == GNNCO_F32 && tc_f32_weight_grad_supported(K, N))
-      GNNCO_TRY(launch_weight_grad_tc_f32(h, T.M[l], dZ, wg_out, K, N, st));
+      GNNCO_TRY(launch_weight_grad_tc_f32(h, T.M[l], dZ, wg_out, T.wg_scratch, K, N, st));
     else GNNCO_TRY(launch_weight_grad(h, dt, T.M[l], dZ, wg_out, K, N, st));
     if (sets == 1) GNNCO_TRY(launch_sum_over_sets(h, T.dW_sets, target, (int64_t)K * N, h->S, st));
     GNNCO_TRY(finish_layer(l - 1, target));

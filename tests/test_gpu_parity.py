@@ -253,3 +253,26 @@ def test_train_step_f32_tensor_core_widths(dims, n, S, sets):
                 v=[np.square(0.02 * rand_weights(dims, nsets, 52)[l]).astype(np.float32) for l in range(len(W))])
     g, stats = case.run(graph, X, W, pen, want_dx=True, adam=adam, label="f32-tc")
     print({k: float("%.3g" % v) for k, v in stats.items()})
+
+
+@pytest.mark.parametrize("dtype,dims,n,S", [("bf16", [256, 128, 1], 9000, 2), ("f32", [128, 64, 1], 7000, 1),
+                                            ("bf16", [128, 128, 1], 6100, 3)])
+def test_train_step_few_very_long_subgraphs(dtype, dims, n, S):
+    """Few subgraphs of several thousand rows (the shape community detection gives): the
+    weight gradient of such a subgraph is cut into row chunks whose partial results are summed
+    in a fixed order."""
+    eu, ev, part = tiny_graph(n, 4.0 / n, S, seed=61, contiguous=True)
+    if S == 3:
+        part = np.where(np.arange(n) < 5000, 0, np.where(np.arange(n) < 6000, 1, 2)).astype(np.int32)   # uneven
+    book = oracle.bookkeeping(n, eu, ev, part, S)
+    graph = load_graph(n, eu, ev, part, S)
+    X = rand_features(n, dims[0], 63).astype(np.float32)
+    W = [w.astype(np.float32) for w in rand_weights(dims, S, 67)]
+    if dtype == "bf16":
+        X, W = si.round_to_bf16(X), [si.round_to_bf16(w) for w in W]
+    case = StepCase(book, dims, dtype, S)
+    case.run(graph, X, W, None, want_dx=True, label="long-subgraphs")
+    again = case.run(graph, X, W, None, want_dx=True, label="long-subgraphs")[0]
+    first = case.run(graph, X, W, None, want_dx=True, label="long-subgraphs")[0]
+    for a, b in zip(again["dW"], first["dW"]):
+        assert np.array_equal(a, b)                      # deterministic combine
