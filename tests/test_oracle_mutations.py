@@ -1,0 +1,85 @@
+"""Do the pins bite?  Each case plants ONE plausible mistake in a copy of the oracle's C
+source (on the CPU, in a temporary directory), builds it, swaps it in for the real oracle and
+runs the pin battery: at least one pin must fail.  A mutation that no pin notices would mean
+that part of the oracle is unpinned."""
+import ctypes
+import os
+import subprocess
+
+import pytest
+
+import oracle
+import test_oracle_pins as pins
+
+SRC = os.path.join(os.path.dirname(oracle.__file__), "gnnco_oracle.c")
+
+MUTATIONS = {
+    "aggregation drops the node's own features":
+        ("for (int32_t f = 0; f < fi; ++f) m[f] = Hp[(size_t)i * fi + f];", "for (int32_t f = 0; f < fi; ++f) m[f] = 0.0;"),
+    "normaliser is |N(i)|+2": ("double inv = 1.0 / (double)(rp[i + 1] - rp[i] + 1);", "double inv = 1.0 / (double)(rp[i + 1] - rp[i] + 2);"),
+    "size term has the wrong sign": ("alpha * edge_term - beta * node_term", "alpha * edge_term + beta * node_term"),
+    "every edge counted twice in the loss": ("if (ci[k] > i) edge_term += p[i] * p[ci[k]];", "edge_term += p[i] * p[ci[k]];"),
+    "penalty term dropped from the loss": ("+ lambda * pen_term;", "+ 0.0 * pen_term;"),
+    "sigmoid of -z": ("p[i] = 1.0 / (1.0 + exp(-z));", "p[i] = 1.0 / (1.0 + exp(z));"),
+    "edge gradient halved": ("double dp = alpha * nb - beta", "double dp = 0.5 * alpha * nb - beta"),
+    "penalty missing from the gradient": ("+ (pen ? lambda * pen[i] : 0.0);", "+ 0.0;"),
+    "transposed aggregation not normalised": ("dm[f] = acc / (double)(rp[i + 1] - rp[i] + 1);", "dm[f] = acc;"),
+    "transposed aggregation forgets the node itself":
+        ("for (int32_t f = 0; f < fi; ++f) dH[(size_t)i * fi + f] += dm[f];", ";"),
+    "ReLU derivative ignored": ("if (!(Z[l - 1][q] > 0.0)) dH[q] = 0.0;", ";"),
+    "input gradient uses W instead of W^T":
+        ("acc += dZ[(size_t)i * fo + h] * Wl[(size_t)f * fo + h];", "acc += dZ[(size_t)i * fo + h] * Wl[((size_t)h * fi + f) % ((size_t)fi * fo)];"),
+    "Adam without bias correction of m": ("W[q] -= lr * (m[q] / c1)", "W[q] -= lr * (m[q])"),
+    "Adam eps inside the root": ("/ (sqrt(v[q] / c2) + eps);", "/ sqrt(v[q] / c2 + eps);"),
+    "Adam second moment uses g instead of g^2": ("(1.0 - b2) * g[q] * g[q];", "(1.0 - b2) * g[q];"),
+    "threshold uses > instead of >=": ("x[i] = p[i] >= threshold ? 1 : 0;", "x[i] = p[i] > threshold ? 1 : 0;"),
+    "intra conflicts counted from both ends": ("if (colidx[k] > i && x[i] && x[colidx[k]]) ++intra;", "if (x[i] && x[colidx[k]]) ++intra;"),
+    "per-subgraph count misses the second endpoint": ("per_part[node_part[bnd_v[e]]]++;", ";"),
+    "boundary edge stored as (u, v) instead of (min, max)":
+        ("bpairs[2 * E_b] = a < b ? a : b;\n      bpairs[2 * E_b + 1] = a < b ? b : a;", "bpairs[2 * E_b] = a;\n      bpairs[2 * E_b + 1] = b;"),
+    "new ids ignore the original order inside a part":
+        ("int32_t id = fill[part[i]]++;", "int32_t id = part_ptr[part[i] + 1] - 1 - (fill[part[i]]++ - part_ptr[part[i]]);"),
+    "inv_deg without the +1": ("inv_deg[i] = 1.0f / (float)(hi - lo + 1);", "inv_deg[i] = 1.0f / (float)(hi - lo > 0 ? hi - lo : 1);"),
+}
+
+BATTERY = [
+    lambda: pins.test_bookkeeping_brute_force(40, 0.2, 5, 2),
+    lambda: pins.test_bookkeeping_brute_force(25, 0.3, 9, 5),
+    lambda: pins.test_forward_and_loss_match_dense_definition([6, 4, 1], False),
+    lambda: pins.test_forward_and_loss_match_dense_definition([7, 5, 3, 1], True),
+    pins.test_aggregation_preserves_constant_features_and_isolated_nodes,
+    pins.test_zero_weights_closed_forms,
+    pins.test_single_node_subgraph_by_hand,
+    pins.test_loss_on_binary_probabilities_is_the_qubo_value,
+    lambda: pins.test_gradients_match_central_finite_differences([5, 4, 1], False),
+    lambda: pins.test_gradients_match_central_finite_differences([6, 5, 4, 1], False),
+    pins.test_sigmoid_chain_identity_for_one_layer,
+    pins.test_adam_two_steps_against_exact_rational_arithmetic,
+    pins.test_adam_first_step_is_sign_step_and_zero_gradient_stays,
+    lambda: pins.test_decode_brute_force(1),
+    lambda: pins.test_decode_brute_force(2),
+]
+
+
+@pytest.mark.parametrize("name", sorted(MUTATIONS))
+def test_a_pin_fails_when_the_oracle_is_mutated(name, tmp_path, monkeypatch):
+    old, new = MUTATIONS[name]
+    text = open(SRC).read()
+    assert text.count(old) == 1, "mutation target not found exactly once: %r" % old
+    src = tmp_path / "mutant.c"
+    src.write_text(text.replace(old, new))
+    lib_path = str(tmp_path / "libmutant.so")
+    subprocess.check_call(["gcc", "-O1", "-fopenmp", "-shared", "-fPIC", "-o", lib_path, str(src), "-lm"])
+    real = oracle._native()
+    mutant = ctypes.CDLL(lib_path)
+    for fn in ("oracle_bookkeeping", "oracle_subgraph_step", "oracle_train_step", "oracle_adam", "oracle_decode"):
+        getattr(mutant, fn).argtypes = getattr(real, fn).argtypes
+        getattr(mutant, fn).restype = getattr(real, fn).restype
+    monkeypatch.setattr(oracle, "_lib", mutant)
+    caught = 0
+    for check in BATTERY:
+        try:
+            check()
+        except (AssertionError, oracle.OracleError, ValueError, IndexError, KeyError):
+            caught += 1
+    assert caught >= 1, "no pin noticed: " + name
