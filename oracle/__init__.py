@@ -47,6 +47,12 @@ def _native():
         lib.oracle_adam.restype = None
         lib.oracle_decode.argtypes = [i64, i32, vp, vp, vp, i64, vp, vp, vp, flt, vp, vp, vp, vp]
         lib.oracle_decode.restype = None
+        lib.oracle_conflict_list.argtypes = [i64, vp, vp]
+        lib.oracle_conflict_list.restype = i64
+        lib.oracle_base_action.argtypes = [i64, vp, vp, vp, vp, vp]
+        lib.oracle_base_action.restype = None
+        lib.oracle_apply_actions.argtypes = [i64, i32, i64, vp, vp, vp, vp, vp, vp, vp]
+        lib.oracle_apply_actions.restype = i64
         _lib = lib
     return _lib
 
@@ -178,3 +184,32 @@ def decode(book: Dict[str, np.ndarray], p: np.ndarray, threshold: float = 0.5) -
                             _ptr(per_part), _ptr(counts))
     return dict(x=x, viol=viol[: book["E_b"]], per_part=per_part, set_size=int(counts[0]), intra_viol=int(counts[1]),
                 boundary_viol=int(counts[2]))
+
+
+def conflict_list(book: Dict[str, np.ndarray], viol: np.ndarray) -> np.ndarray:
+    """Ascending indices (into the boundary list) of the violated boundary edges."""
+    viol = np.ascontiguousarray(viol, dtype=np.uint8)
+    idx = np.empty(max(1, viol.size), np.int32)
+    c = _native().oracle_conflict_list(viol.size, _ptr(viol), _ptr(idx))
+    return idx[:c].copy()
+
+
+def base_action(book: Dict[str, np.ndarray], conflicts: np.ndarray, p: np.ndarray) -> np.ndarray:
+    """0/1 per conflict: which endpoint (u or v of the stored pair) to push below the threshold."""
+    conflicts = np.ascontiguousarray(conflicts, dtype=np.int32)
+    p = np.ascontiguousarray(p, dtype=np.float32)
+    act = np.empty(max(1, conflicts.size), np.uint8)
+    _native().oracle_base_action(conflicts.size, _ptr(conflicts), _ptr(book["bnd_u"]), _ptr(book["bnd_v"]), _ptr(p),
+                                 _ptr(act))
+    return act[:conflicts.size].copy()
+
+
+def apply_actions(book: Dict[str, np.ndarray], conflicts: np.ndarray, action: np.ndarray) -> Dict[str, object]:
+    """Penalty node list (0/1 float per node), active-subgraph mask and number of chosen nodes."""
+    n, S = int(book["n"]), int(book["S"])
+    conflicts = np.ascontiguousarray(conflicts, dtype=np.int32)
+    action = np.ascontiguousarray(action, dtype=np.uint8)
+    pen, active = np.empty(n, np.float32), np.empty(S, np.uint8)
+    chosen = _native().oracle_apply_actions(n, S, conflicts.size, _ptr(conflicts), _ptr(action), _ptr(book["bnd_u"]),
+                                            _ptr(book["bnd_v"]), _ptr(book["node_part"]), _ptr(pen), _ptr(active))
+    return dict(pen=pen, active=active, chosen=int(chosen))

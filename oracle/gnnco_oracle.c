@@ -433,3 +433,54 @@ void oracle_decode(int64_t n, int32_t S, const int32_t* node_part, const int32_t
   counts[1] = intra;
   counts[2] = bviol;
 }
+
+/*
+ * Stage-3 glue (Algorithm 1, Stage 3, first lines; Section 3.3).
+ *
+ * Conflict list: the boundary edges whose two endpoints are both selected, as ascending
+ * indices into the boundary list ("compute conflict edges from m"; the set C of Section 3.3).
+ * Returns their number.
+ */
+int64_t oracle_conflict_list(int64_t E_b, const uint8_t* viol, int32_t* conflict_idx) {
+  int64_t c = 0;
+  for (int64_t e = 0; e < E_b; ++e)
+    if (viol[e]) conflict_idx[c++] = (int32_t)e;
+  return c;
+}
+
+/*
+ * Base action (Algorithm 1: "initialize agent base action"; the paper does not say how).
+ * Reading taken: for every conflict edge (u, v) the endpoint with the SMALLER probability is
+ * the one to push below the threshold; on equal probabilities the endpoint with the larger
+ * id.  action = 0 chooses u (the lower id of the stored pair), 1 chooses v.  Every conflict
+ * loses one endpoint, so removing all chosen nodes leaves no violated boundary edge.
+ */
+void oracle_base_action(int64_t count, const int32_t* conflict_idx, const int32_t* bnd_u, const int32_t* bnd_v,
+                        const float* p, uint8_t* action) {
+  for (int64_t c = 0; c < count; ++c) {
+    int32_t u = bnd_u[conflict_idx[c]], v = bnd_v[conflict_idx[c]];
+    action[c] = p[u] < p[v] ? 0 : 1;
+  }
+}
+
+/*
+ * Actions -> fine-tuning inputs (Section 3.3: each conflict offers two options, fine-tune the
+ * subgraph of node i or of node j so that this node's probability falls below the threshold;
+ * Algorithm 1: "group actions per subgraph").  pen[i] = 1 for every chosen node (the node
+ * list of the penalty term), 0 elsewhere; active[s] = 1 for every subgraph that holds a chosen
+ * node (the subgraphs whose models are fine-tuned).  Returns the number of distinct chosen nodes.
+ */
+int64_t oracle_apply_actions(int64_t n, int32_t S, int64_t count, const int32_t* conflict_idx, const uint8_t* action,
+                             const int32_t* bnd_u, const int32_t* bnd_v, const int32_t* node_part, float* pen,
+                             uint8_t* active) {
+  for (int64_t i = 0; i < n; ++i) pen[i] = 0.0f;
+  for (int32_t s = 0; s < S; ++s) active[s] = 0;
+  int64_t chosen = 0;
+  for (int64_t c = 0; c < count; ++c) {
+    int32_t node = action[c] ? bnd_v[conflict_idx[c]] : bnd_u[conflict_idx[c]];
+    if (pen[node] == 0.0f) ++chosen;
+    pen[node] = 1.0f;
+    active[node_part[node]] = 1;
+  }
+  return chosen;
+}

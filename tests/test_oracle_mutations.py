@@ -39,6 +39,9 @@ MUTATIONS = {
         ("bpairs[2 * E_b] = a < b ? a : b;\n      bpairs[2 * E_b + 1] = a < b ? b : a;", "bpairs[2 * E_b] = a;\n      bpairs[2 * E_b + 1] = b;"),
     "new ids ignore the original order inside a part":
         ("int32_t id = fill[part[i]]++;", "int32_t id = part_ptr[part[i] + 1] - 1 - (fill[part[i]]++ - part_ptr[part[i]]);"),
+    "base action picks u on equal probabilities": ("action[c] = p[u] < p[v] ? 0 : 1;", "action[c] = p[u] <= p[v] ? 0 : 1;"),
+    "actions mark the wrong endpoint's subgraph": ("active[node_part[node]] = 1;", "active[node_part[bnd_u[conflict_idx[c]]]] = 1;"),
+    "conflict list keeps non-violated edges": ("if (viol[e]) conflict_idx[c++] = (int32_t)e;", "conflict_idx[c++] = (int32_t)e;"),
     "inv_deg without the +1": ("inv_deg[i] = 1.0f / (float)(hi - lo + 1);", "inv_deg[i] = 1.0f / (float)(hi - lo > 0 ? hi - lo : 1);"),
 }
 
@@ -58,6 +61,8 @@ BATTERY = [
     pins.test_adam_first_step_is_sign_step_and_zero_gradient_stays,
     lambda: pins.test_decode_brute_force(1),
     lambda: pins.test_decode_brute_force(2),
+    lambda: pins.test_conflict_list_base_action_and_penalty_brute_force(1),
+    lambda: pins.test_conflict_list_base_action_and_penalty_brute_force(2),
 ]
 
 
@@ -72,7 +77,8 @@ def test_a_pin_fails_when_the_oracle_is_mutated(name, tmp_path, monkeypatch):
     subprocess.check_call(["gcc", "-O1", "-fopenmp", "-shared", "-fPIC", "-o", lib_path, str(src), "-lm"])
     real = oracle._native()
     mutant = ctypes.CDLL(lib_path)
-    for fn in ("oracle_bookkeeping", "oracle_subgraph_step", "oracle_train_step", "oracle_adam", "oracle_decode"):
+    for fn in ("oracle_bookkeeping", "oracle_subgraph_step", "oracle_train_step", "oracle_adam", "oracle_decode",
+               "oracle_conflict_list", "oracle_base_action", "oracle_apply_actions"):
         getattr(mutant, fn).argtypes = getattr(real, fn).argtypes
         getattr(mutant, fn).restype = getattr(real, fn).restype
     monkeypatch.setattr(oracle, "_lib", mutant)

@@ -553,3 +553,57 @@ def test_config1_training_lowers_every_subgraph_loss():
             oracle.adam(W[l], m[l], v[l], r["dW"][l], w.lr, t)
     last = oracle.train_step(b, w.dims, X, W, w.alpha, w.beta, want_dW=False)["loss"]
     assert np.all(last < first)
+
+
+# ------------------------------------------------- Stage-3 glue (conflicts -> fine-tune inputs)
+@pytest.mark.parametrize("seed", [1, 2, 3])
+def test_conflict_list_base_action_and_penalty_brute_force(seed):
+    n, S = 60, 6
+    eu, ev, part = tiny_graph(n, 0.15, S, seed=200 + seed)
+    b = oracle.bookkeeping(n, eu, ev, part, S)
+    p_orig = si.uniform01(300 + seed, 0, n).astype(np.float32)
+    p_orig[::9] = p_orig[1]                                      # some exact ties between endpoints
+    p_new = p_orig[b["perm"]]
+    d = oracle.decode(b, p_new)
+    conf = oracle.conflict_list(b, d["viol"])
+    # brute force over the ORIGINAL edge list
+    x = p_orig >= np.float32(0.5)
+    want = set()
+    for a, c in zip(eu.tolist(), ev.tolist()):
+        if part[a] != part[c] and x[a] and x[c]:
+            na, nc = int(b["inv_perm"][a]), int(b["inv_perm"][c])
+            want.add((min(na, nc), max(na, nc)))
+    got = [(int(b["bnd_u"][e]), int(b["bnd_v"][e])) for e in conf]
+    assert got == sorted(want) and len(conf) == d["boundary_viol"]
+    assert np.all(np.diff(conf) > 0)
+    act = oracle.base_action(b, conf, p_new)
+    chosen = set()
+    for e, a in zip(conf.tolist(), act.tolist()):
+        u, v = int(b["bnd_u"][e]), int(b["bnd_v"][e])
+        lower = u if p_new[u] < p_new[v] else v                 # smaller probability, ties -> larger id (v > u)
+        assert (u, v)[a] == lower
+        chosen.add(lower)
+    r = oracle.apply_actions(b, conf, act)
+    assert r["chosen"] == len(chosen)
+    assert set(np.nonzero(r["pen"])[0].tolist()) == chosen and set(np.unique(r["pen"]).tolist()) <= {0.0, 1.0}
+    assert set(np.nonzero(r["active"])[0].tolist()) == {int(b["node_part"][i]) for i in chosen}
+    # removing the chosen nodes resolves every boundary conflict and touches nothing else
+    p_fixed = p_new.copy()
+    p_fixed[sorted(chosen)] = 0.0
+    d2 = oracle.decode(b, p_fixed)
+    assert d2["boundary_viol"] == 0 and d2["set_size"] == d["set_size"] - len(chosen)
+    # the opposite choice is also a valid action vector and gives its own node list
+    r2 = oracle.apply_actions(b, conf, 1 - act)
+    other = {(int(b["bnd_u"][e]), int(b["bnd_v"][e]))[1 - a] for e, a in zip(conf.tolist(), act.tolist())}
+    assert set(np.nonzero(r2["pen"])[0].tolist()) == other
+
+
+def test_stage3_glue_on_empty_conflict_set():
+    n, S = 20, 4
+    eu, ev, part = tiny_graph(n, 0.2, S, seed=7)
+    b = oracle.bookkeeping(n, eu, ev, part, S)
+    d = oracle.decode(b, np.zeros(n, np.float32))
+    conf = oracle.conflict_list(b, d["viol"])
+    assert conf.size == 0
+    r = oracle.apply_actions(b, conf, np.zeros(0, np.uint8))
+    assert r["chosen"] == 0 and not r["pen"].any() and not r["active"].any()
