@@ -561,8 +561,8 @@ def test_conflict_list_base_action_and_penalty_brute_force(seed):
     n, S = 60, 6
     eu, ev, part = tiny_graph(n, 0.15, S, seed=200 + seed)
     b = oracle.bookkeeping(n, eu, ev, part, S)
-    p_orig = si.uniform01(300 + seed, 0, n).astype(np.float32)
-    p_orig[::9] = p_orig[1]                                      # some exact ties between endpoints
+    # three probability levels only, so that many conflict edges join endpoints with EQUAL p
+    p_orig = np.array([0.2, 0.6, 0.9], np.float32)[(si.u64(300 + seed, 0, n) % np.uint64(3)).astype(int)]
     p_new = p_orig[b["perm"]]
     d = oracle.decode(b, p_new)
     conf = oracle.conflict_list(b, d["viol"])
@@ -577,6 +577,7 @@ def test_conflict_list_base_action_and_penalty_brute_force(seed):
     assert got == sorted(want) and len(conf) == d["boundary_viol"]
     assert np.all(np.diff(conf) > 0)
     act = oracle.base_action(b, conf, p_new)
+    assert any(p_new[b["bnd_u"][e]] == p_new[b["bnd_v"][e]] for e in conf)      # ties are exercised
     chosen = set()
     for e, a in zip(conf.tolist(), act.tolist()):
         u, v = int(b["bnd_u"][e]), int(b["bnd_v"][e])
