@@ -331,6 +331,33 @@ def run_ours(args):
                     algorithmic_bytes_per_launch=algorithmic_bytes(top, w, w.n, nnz, w.S))
     agg = {k: kern[k] for k in ("aggregate_fwd", "aggregate_bwd") if k in kern}
 
+    # ---- Stage-3 glue after the last decode (not part of the timed step): conflict list + base
+    # action + penalty list / active subgraphs, timed with CUDA events on the current stream
+    stage3 = None
+    if graph.E_b > 0:
+        ca = graph.conflict_actions(viol, p)
+        graph.apply_actions(ca["conflict_idx"], ca["action"], ca["count"])
+        torch.cuda.synchronize()
+        s0, s1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        reps = 5
+        s0.record()
+        for _ in range(reps):
+            ca = graph.conflict_actions(viol, p)
+            ap = graph.apply_actions(ca["conflict_idx"], ca["action"], ca["count"])
+        s1.record()
+        torch.cuda.synchronize()
+        n_conf = int(ca["count"].item())
+        # flags read twice, one index + action per conflict, two endpoint ids and probabilities per
+        # conflict, penalty vector cleared, three words per conflict in the scatter of actions
+        s3_bytes = 2 * graph.E_b + n_conf * (5 + 16) + 4 * w.n + n_conf * 17
+        s3_ms = s0.elapsed_time(s1) / reps
+        stage3 = dict(ms=round(s3_ms, 4), conflicts=n_conf, chosen_nodes=int(ap["chosen"].item()),
+                      active_subgraphs=int(ap["active"].sum().item()),
+                      algo_GBs=round(s3_bytes / (s3_ms * 1e-3) / 1e9, 1),
+                      note="gnnco_conflict_actions + gnnco_apply_actions on the last step's flags; "
+                           "includes the binding's buffer allocations")
+        del ca, ap
+
     # ---- end to end through the host-buffer entry point (rank-local; copies inside the timed region)
     e2e = None
     if not args.no_e2e:
@@ -378,7 +405,7 @@ def run_ours(args):
                         parallelism="replicas only (no collective on the data path)" if world > 1 else "1 GPU",
                         partition_load_ms=round(load_ms, 3), edges_per_s_whole_graph=value * w.E / max(1, graph.E_in)),
             roofline=roofline, aggregate_kernels=agg, kernels=kern, cpu_baseline=cpu, clocks=clocks, e2e=e2e,
-            gpu_launches=int(launches))
+            gpu_launches=int(launches), stage3_glue=stage3)
         print(json.dumps(line))
     if dist is not None:
         dist.destroy_process_group()
@@ -392,7 +419,6 @@ TRAFFIC_BYTES = {
     (5, "aggregate_fwd"): 10.07e9,
     (5, "transform_fwd"): 11.53e9,
     (5, "transform_bwd"): 11.63e9,
-    (5, "weight_grad"): 11.07e9,
 }
 
 

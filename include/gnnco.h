@@ -114,12 +114,18 @@ typedef struct {
 
 /* Adam state (bias-corrected; eps outside the square root).  `step` is the 1-based
  * number of THIS update; the caller increments it between calls.  m[l], v[l] have the
- * shape of W[l]. */
+ * shape of W[l].
+ * `active` (device, [S] uint8, or NULL = all) restricts the update to the subgraphs that
+ * are being fine-tuned (Section 3.3: an action fine-tunes the model of ONE endpoint's
+ * subgraph; Algorithm 1, Stage 3 groups the actions per subgraph): weights and moments of
+ * a subgraph with active[s] == 0 are left bit-for-bit unchanged.  It needs per-subgraph
+ * weights (weight_sets == S); the bias correction uses `step` for every active subgraph. */
 typedef struct {
   float lr, beta1, beta2, eps;
   int64_t step;
   float* m[GNNCO_MAX_LAYERS];
   float* v[GNNCO_MAX_LAYERS];
+  const uint8_t* active;
 } gnnco_adam_state;
 
 /* Outputs of a training step.  loss and p are required; the rest may be NULL. */
@@ -199,6 +205,35 @@ int32_t gnnco_train_step_host(gnnco_handle* h, const gnnco_model_desc* m, const 
  * Integer results are exact.  Asynchronous on `stream`; needs no work area. */
 int32_t gnnco_decode_boundary(const gnnco_handle* h, const float* p, float threshold, uint8_t* x, uint8_t* viol,
                               int32_t* per_part, gnnco_counts* counts, void* stream);
+
+/* Stage-3 glue (Section 3.3; Algorithm 1, Stage 3), the step right after decoding.
+ *
+ * gnnco_conflict_actions turns the per-edge flags of gnnco_decode_boundary into the
+ * conflict set C and a non-learned base action for each conflict:
+ *   conflict_idx [E_b] int32 (capacity): positions, in the sorted boundary list, of the
+ *                violated edges, ASCENDING; only the first *count entries are written
+ *   action       [E_b] uint8 (capacity) or NULL: for conflict c on the stored pair (u, v),
+ *                u < v in the new order, 0 = push u below the threshold, 1 = push v.
+ *                Section 3.3 gives every conflict exactly these two options; the base action
+ *                ("initialize agent base action", not defined further by the paper) takes
+ *                the endpoint with the SMALLER probability p, and v when they are equal.
+ *   count        device int32: |C|
+ * viol [E_b] uint8 and p [n] float32 (new order) are inputs; p may be NULL iff action is.
+ * ws must hold gnnco_conflict_workspace_bytes bytes.  Asynchronous on `stream`; no host
+ * synchronisation (|C| stays on the device).  Results are exact and order-deterministic.
+ *
+ * gnnco_apply_actions turns (C, actions) into the inputs of the fine-tuning steps:
+ *   pen    [n] float32: 1 for every chosen node, else 0 -- the node list of the added
+ *          penalty term lambda * sum_k p_{i_k} (gnnco_objective.pen)
+ *   active [S] uint8: 1 for every subgraph holding a chosen node (gnnco_adam_state.active)
+ *   chosen device int32 or NULL: number of distinct chosen nodes
+ * count is the DEVICE value written by gnnco_conflict_actions; action may come from there or
+ * from the caller's own policy (any 0/1 vector of that length).  Asynchronous on `stream`. */
+int32_t gnnco_conflict_workspace_bytes(const gnnco_handle* h, size_t* bytes);
+int32_t gnnco_conflict_actions(gnnco_handle* h, const uint8_t* viol, const float* p, int32_t* conflict_idx,
+                               uint8_t* action, int32_t* count, void* ws, size_t ws_bytes, void* stream);
+int32_t gnnco_apply_actions(gnnco_handle* h, const int32_t* conflict_idx, const uint8_t* action,
+                            const int32_t* count, float* pen, uint8_t* active, int32_t* chosen, void* stream);
 
 /* Objective only, for callers that cannot allocate device memory.  (The paper has no
  * counterpart to this call; it exists for the way the library is embedded.)

@@ -25,7 +25,8 @@ EXPORTS = [
     "gnnco_status_string", "gnnco_partition_workspace_bytes", "gnnco_partition_load", "gnnco_graph_info",
     "gnnco_gather_rows", "gnnco_train_workspace_bytes", "gnnco_train_step", "gnnco_train_host_workspace_bytes",
     "gnnco_train_step_host", "gnnco_decode_boundary", "gnnco_async_status", "gnnco_launch_count", "gnnco_destroy",
-    "gnnco_profile_begin", "gnnco_profile_end", "gnnco_objective_static",
+    "gnnco_profile_begin", "gnnco_profile_end", "gnnco_objective_static", "gnnco_conflict_workspace_bytes",
+    "gnnco_conflict_actions", "gnnco_apply_actions",
 ]
 
 _vp, _i32, _i64, _u32, _f32, _sz = (ctypes.c_void_p, ctypes.c_int32, ctypes.c_int64, ctypes.c_uint32, ctypes.c_float,
@@ -53,7 +54,7 @@ class Objective(ctypes.Structure):
 
 class AdamState(ctypes.Structure):
     _fields_ = [("lr", _f32), ("beta1", _f32), ("beta2", _f32), ("eps", _f32), ("step", _i64),
-                ("m", _vp * MAX_LAYERS), ("v", _vp * MAX_LAYERS)]
+                ("m", _vp * MAX_LAYERS), ("v", _vp * MAX_LAYERS), ("active", _vp)]
 
 
 class TrainOut(ctypes.Structure):
@@ -108,6 +109,9 @@ def load_library(build_if_missing: bool = True):
     lib.gnnco_objective_static.argtypes = [_vp, _vp, ctypes.POINTER(Objective), _vp, _vp]
     lib.gnnco_profile_begin.argtypes = [_vp]
     lib.gnnco_profile_end.argtypes = [_vp, _vp, ctypes.POINTER(ProfileEntry), _i32, ctypes.POINTER(_i32)]
+    lib.gnnco_conflict_workspace_bytes.argtypes = [_vp, ctypes.POINTER(_sz)]
+    lib.gnnco_conflict_actions.argtypes = [_vp, _vp, _vp, _vp, _vp, _vp, _vp, _sz, _vp]
+    lib.gnnco_apply_actions.argtypes = [_vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp]
     for name in EXPORTS:
         if name not in ("gnnco_status_string", "gnnco_launch_count"):
             getattr(lib, name).restype = _i32
@@ -183,6 +187,7 @@ class Adam:
         import torch
         self.lr, self.beta1, self.beta2, self.eps = lr, beta1, beta2, eps
         self.step = 1
+        self.active = None          # uint8 [S] device tensor: subgraphs being fine-tuned (None = all)
         self.m = [torch.zeros_like(w) for w in model.W]
         self.v = [torch.zeros_like(w) for w in model.W]
 
@@ -192,6 +197,7 @@ class Adam:
         for l in range(len(self.m)):
             a.m[l] = self.m[l].data_ptr()
             a.v[l] = self.v[l].data_ptr()
+        a.active = _dptr(self.active)
         return a
 
 
@@ -346,6 +352,43 @@ class PartitionedGraph:
                                              _dptr(per_part), counts.data_ptr(), _stream_ptr(stream))
         _check(st, "gnnco_decode_boundary")
         return dict(x=x, viol=viol, per_part=per_part, counts=counts)
+
+    def conflict_actions(self, viol, p=None, want_action: bool = True, stream=None):
+        """``gnnco_conflict_actions``.  Returns dict(conflict_idx, action, count): int32 [E_b]
+        and uint8 [E_b] buffers of which the first ``count`` entries are valid, and the device
+        int32 count itself (no host synchronisation)."""
+        import torch
+        _require(viol, torch.uint8, "viol")
+        if want_action:
+            _require(p, torch.float32, "p")
+        need = _sz(0)
+        _check(self._lib.gnnco_conflict_workspace_bytes(self._handle, ctypes.byref(need)),
+               "gnnco_conflict_workspace_bytes")
+        ws = torch.empty(need.value, dtype=torch.uint8, device=self.device)
+        idx = torch.empty(self.E_b, dtype=torch.int32, device=self.device)
+        action = torch.empty(self.E_b, dtype=torch.uint8, device=self.device) if want_action else None
+        count = torch.empty(1, dtype=torch.int32, device=self.device)
+        _check(self._lib.gnnco_conflict_actions(self._handle, viol.data_ptr(), _dptr(p) if want_action else None,
+                                                idx.data_ptr(), _dptr(action), count.data_ptr(), ws.data_ptr(),
+                                                need.value, _stream_ptr(stream)), "gnnco_conflict_actions")
+        return dict(conflict_idx=idx, action=action, count=count)
+
+    def apply_actions(self, conflict_idx, action, count, pen=None, active=None, stream=None):
+        """``gnnco_apply_actions``.  Returns dict(pen, active, chosen): float32 [n], uint8 [S]
+        and a device int32 with the number of distinct chosen nodes."""
+        import torch
+        _require(conflict_idx, torch.int32, "conflict_idx")
+        _require(action, torch.uint8, "action")
+        _require(count, torch.int32, "count")
+        if pen is None:
+            pen = torch.empty(self.n, dtype=torch.float32, device=self.device)
+        if active is None:
+            active = torch.empty(self.S, dtype=torch.uint8, device=self.device)
+        chosen = torch.empty(1, dtype=torch.int32, device=self.device)
+        _check(self._lib.gnnco_apply_actions(self._handle, conflict_idx.data_ptr(), action.data_ptr(),
+                                             count.data_ptr(), pen.data_ptr(), active.data_ptr(), chosen.data_ptr(),
+                                             _stream_ptr(stream)), "gnnco_apply_actions")
+        return dict(pen=pen, active=active, chosen=chosen)
 
     def objective_static(self, p, alpha: float, beta: float, lam: float = 0.0, pen=None, loss=None, stream=None):
         """``gnnco_objective_static``: per-subgraph objective of given probabilities, with no

@@ -321,9 +321,10 @@ __global__ void cast_bf16x8_kernel(const float4* __restrict__ in, uint4* __restr
 
 __global__ void adam_kernel(float* __restrict__ W, float* __restrict__ m, float* __restrict__ v,
                             const float* __restrict__ g, int64_t count, float lr, float b1, float b2, float eps,
-                            float inv_c1, float inv_c2) {
+                            float inv_c1, float inv_c2, const uint8_t* __restrict__ active, int64_t per_set) {
   const int64_t q = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
   if (q >= count) return;
+  if (active && !active[q / per_set]) return;   // this subgraph is not being fine-tuned
   const float gq = g[q];
   const float mq = b1 * m[q] + (1.0f - b1) * gq;
   const float vq = b2 * v[q] + (1.0f - b2) * gq * gq;
@@ -483,9 +484,11 @@ int32_t launch_cast_bf16(gnnco_handle* h, const float* in, __nv_bfloat16* out, i
 }
 
 int32_t launch_adam(gnnco_handle* h, float* W, float* m, float* v, const float* g, int64_t count, float lr, float b1,
-                    float b2, float eps, float c1, float c2, cudaStream_t stream) {
+                    float b2, float eps, float c1, float c2, const uint8_t* active, int64_t per_set,
+                    cudaStream_t stream) {
   ProfScope prof_(h, K_ADAM, stream);
-  adam_kernel<<<blocks_for(count, 256), 256, 0, stream>>>(W, m, v, g, count, lr, b1, b2, eps, 1.0f / c1, 1.0f / c2);
+  adam_kernel<<<blocks_for(count, 256), 256, 0, stream>>>(W, m, v, g, count, lr, b1, b2, eps, 1.0f / c1, 1.0f / c2,
+                                                          active, per_set);
   h->launches += 1;
   GNNCO_LAUNCH_CHECK();
   return GNNCO_OK;

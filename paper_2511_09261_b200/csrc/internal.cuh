@@ -28,7 +28,7 @@ constexpr int kItemRows = 1024;      // rows of one objective work item (never s
 // Kernel families, for launch accounting and per-kernel timing.
 enum KernelKind {
   K_AGG_FWD, K_AGG_BWD, K_TRANSFORM_FWD, K_TRANSFORM_BWD, K_WEIGHT_GRAD, K_GEMV, K_WEIGHT_GRAD_VEC, K_RANK1,
-  K_SUM_SETS, K_CAST, K_ADAM, K_OUT_FWD, K_OBJECTIVE, K_OUT_BWD, K_DECODE, K_KIND_COUNT
+  K_SUM_SETS, K_CAST, K_ADAM, K_OUT_FWD, K_OBJECTIVE, K_OUT_BWD, K_DECODE, K_STAGE3, K_KIND_COUNT
 };
 
 // Optional per-kernel timing: while `on`, every launcher brackets its launches with a pair
@@ -138,8 +138,9 @@ int32_t launch_wg_combine(gnnco_handle* h, const float* scratch, float* dW, int6
 // out[q] = sum_s in[s][q]
 int32_t launch_sum_over_sets(gnnco_handle* h, const float* in, float* out, int64_t count, int32_t sets, cudaStream_t st);
 int32_t launch_cast_bf16(gnnco_handle* h, const float* in, __nv_bfloat16* out, int64_t count, cudaStream_t st);
+// active (or nullptr): one byte per run of `per_set` consecutive elements; runs with a zero byte are skipped
 int32_t launch_adam(gnnco_handle* h, float* W, float* m, float* v, const float* g, int64_t count, float lr, float b1,
-                    float b2, float eps, float c1, float c2, cudaStream_t st);
+                    float b2, float eps, float c1, float c2, const uint8_t* active, int64_t per_set, cudaStream_t st);
 
 // ---- tc_gemm.cu : the same transform on the tensor cores (bf16, widths 64/128/256)
 bool tc_transform_supported(int dtype, int K, int N);

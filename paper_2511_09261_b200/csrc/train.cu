@@ -175,7 +175,7 @@ int32_t run_step(gnnco_handle* h, const gnnco_model_desc* m, const void* X, cons
     // grad_sets_or_final holds [sets x ...] already reduced; run Adam on layer l (0-based)
     const int64_t wc = (int64_t)m->dims[l] * m->dims[l + 1] * sets;
     if (opt) return launch_adam(h, m->W[l], opt->m[l], opt->v[l], grad_sets_or_final, wc, opt->lr, opt->beta1,
-                                opt->beta2, opt->eps, c1, c2, st);
+                                opt->beta2, opt->eps, c1, c2, opt->active, wc / sets, st);
     return GNNCO_OK;
   };
   // gradient target of layer l: the caller's buffer or the scratch
@@ -238,6 +238,7 @@ int32_t check_step_args(const gnnco_handle* h, const gnnco_model_desc* m, const 
   if (flags & ~(GNNCO_WANT_DX | GNNCO_FORWARD_ONLY)) return GNNCO_INVALID_ARGUMENT;
   if (opt && !(flags & GNNCO_FORWARD_ONLY)) {
     if (opt->step < 1) return GNNCO_INVALID_ARGUMENT;
+    if (opt->active && m->weight_sets != h->S) return GNNCO_INVALID_ARGUMENT;
     for (int l = 0; l < m->L; ++l)
       if (!opt->m[l] || !opt->v[l]) return GNNCO_INVALID_ARGUMENT;
   }

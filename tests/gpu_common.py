@@ -244,6 +244,43 @@ def check_decode(graph, book, p_new_f32):
     return ref
 
 
+def check_stage3(graph, book, p, policy_seed=None):
+    """Bit-exact parity of conflict list, base action and actions -> (penalty list, active
+    subgraphs, number of chosen nodes), for the base action and for a seeded 0/1 policy."""
+    import torch
+    ref_dec = oracle.decode(book, p)
+    pd = to_dev(p)
+    d = graph.decode_boundary(pd)
+    ca = graph.conflict_actions(d["viol"], pd)
+    torch.cuda.synchronize()
+    conf = oracle.conflict_list(book, ref_dec["viol"])
+    act = oracle.base_action(book, conf, p)
+    C = int(ca["count"].item())
+    assert C == conf.size == ref_dec["boundary_viol"]
+    assert np.array_equal(ca["conflict_idx"].cpu().numpy()[:C], conf)
+    assert np.array_equal(ca["action"].cpu().numpy()[:C], act)
+    # list only (no probabilities)
+    only = graph.conflict_actions(d["viol"], None, want_action=False)
+    assert int(only["count"].item()) == C and only["action"] is None
+    assert np.array_equal(only["conflict_idx"].cpu().numpy()[:C], conf)
+    # the base action, then an arbitrary caller policy
+    policies = [act]
+    if policy_seed is not None and C:
+        policies.append((si.u64(policy_seed, 0, C) & np.uint64(1)).astype(np.uint8))
+    outs = []
+    for a in policies:
+        a_dev = ca["action"].clone()
+        a_dev[:C] = to_dev(a)
+        ap = graph.apply_actions(ca["conflict_idx"], a_dev, ca["count"])
+        torch.cuda.synchronize()
+        ref = oracle.apply_actions(book, conf, a)
+        assert np.array_equal(ap["pen"].cpu().numpy(), ref["pen"])
+        assert np.array_equal(ap["active"].cpu().numpy(), ref["active"])
+        assert int(ap["chosen"].item()) == ref["chosen"]
+        outs.append(ap)
+    return conf, act, outs[0]
+
+
 def sampled_step_check(graph, book, dims, dtype, Xd, Wd, parts, x_rows, w_part, alpha=2.0, beta=1.0, lam=0.0,
                        pen_d=None, pen_rows=None, opt=None, want_dx=True, label=""):
     """Full-size parity on sampled subgraphs.  The GPU runs one step on the whole batch

@@ -7,7 +7,7 @@ import pytest
 
 import oracle
 import synth_inputs as si
-from gpu_common import (StepCase, assert_close, check_bookkeeping, check_decode, load_graph, pick_parts,
+from gpu_common import (StepCase, assert_close, check_bookkeeping, check_decode, check_stage3, load_graph, pick_parts,
                         sampled_step_check, to_dev)
 
 pytestmark = pytest.mark.gpu
@@ -163,6 +163,7 @@ def _full_size_sampled(idx, steps, n_parts):
                                         lambda lo, hi: pen_new[lo:hi], model_opt, True, "%s step 0" % w.name)
     print("\n%s step 0 worst abs errors: %s" % (w.name, {k: float("%.3g" % v) for k, v in stats.items()}))
     check_decode(graph, book, p.cpu().numpy())
+    check_stage3(graph, book, p.cpu().numpy(), policy_seed=7)
     # free-run, then one teacher-forced step from the GPU's current weights
     model = gnnco.Model(w.dims, Wd, gnnco.BF16 if bf16 else gnnco.F32)
     for _ in range(steps - 2):
@@ -176,6 +177,8 @@ def _full_size_sampled(idx, steps, n_parts):
     print("%s last step worst abs errors: %s" % (w.name, {k: float("%.3g" % v) for k, v in stats.items()}))
     d = check_decode(graph, book, p.cpu().numpy())
     assert d["set_size"] > 0
+    conf, _, _ = check_stage3(graph, book, p.cpu().numpy(), policy_seed=8)
+    print("%s conflicts after the last step: %d of %d boundary edges" % (w.name, conf.size, graph.E_b))
 
 
 def test_config4_full_size_sampled_subgraphs():
