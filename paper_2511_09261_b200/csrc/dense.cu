@@ -333,6 +333,32 @@ __global__ void adam_kernel(float* __restrict__ W, float* __restrict__ m, float*
   W[q] -= lr * (mq * inv_c1) / (sqrtf(vq * inv_c2) + eps);
 }
 
+// the same update on four consecutive elements (count and per_set multiples of four, 16-byte aligned arrays)
+__global__ void __launch_bounds__(256) adam_vec4_kernel(float4* __restrict__ W, float4* __restrict__ m,
+                                                        float4* __restrict__ v, const float4* __restrict__ g,
+                                                        int64_t quads, float lr, float b1, float b2, float eps,
+                                                        float inv_c1, float inv_c2, const uint8_t* __restrict__ active,
+                                                        int64_t quads_per_set) {
+  const int64_t q = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+  if (q >= quads) return;
+  if (active && !active[q / quads_per_set]) return;
+  const float4 gq = __ldg(g + q);
+  float4 mq = m[q], vq = v[q], wq = W[q];
+  const float gs[4] = {gq.x, gq.y, gq.z, gq.w};
+  float* mp = reinterpret_cast<float*>(&mq);
+  float* vp = reinterpret_cast<float*>(&vq);
+  float* wp = reinterpret_cast<float*>(&wq);
+#pragma unroll
+  for (int c = 0; c < 4; ++c) {
+    mp[c] = b1 * mp[c] + (1.0f - b1) * gs[c];
+    vp[c] = b2 * vp[c] + (1.0f - b2) * gs[c] * gs[c];
+    wp[c] -= lr * (mp[c] * inv_c1) / (sqrtf(vp[c] * inv_c2) + eps);
+  }
+  m[q] = mq;
+  v[q] = vq;
+  W[q] = wq;
+}
+
 inline unsigned blocks_for(int64_t work, int threads) { return (unsigned)((work + threads - 1) / threads); }
 
 }  // namespace
@@ -487,7 +513,14 @@ int32_t launch_adam(gnnco_handle* h, float* W, float* m, float* v, const float* 
                     float b2, float eps, float c1, float c2, const uint8_t* active, int64_t per_set,
                     cudaStream_t stream) {
   ProfScope prof_(h, K_ADAM, stream);
-  adam_kernel<<<blocks_for(count, 256), 256, 0, stream>>>(W, m, v, g, count, lr, b1, b2, eps, 1.0f / c1, 1.0f / c2,
+  const bool vec = count % 4 == 0 && per_set % 4 == 0 &&
+                   (((uintptr_t)W | (uintptr_t)m | (uintptr_t)v | (uintptr_t)g) & 15) == 0;
+  if (vec)
+    adam_vec4_kernel<<<blocks_for(count / 4, 256), 256, 0, stream>>>(
+        reinterpret_cast<float4*>(W), reinterpret_cast<float4*>(m), reinterpret_cast<float4*>(v),
+        reinterpret_cast<const float4*>(g), count / 4, lr, b1, b2, eps, 1.0f / c1, 1.0f / c2, active, per_set / 4);
+  else
+    adam_kernel<<<blocks_for(count, 256), 256, 0, stream>>>(W, m, v, g, count, lr, b1, b2, eps, 1.0f / c1, 1.0f / c2,
                                                           active, per_set);
   h->launches += 1;
   GNNCO_LAUNCH_CHECK();

@@ -151,6 +151,9 @@ int32_t launch_transform_tc(gnnco_handle* h, const void* A, const void* B, int64
 bool tc_weight_grad_supported(int dtype, int K, int N);
 int32_t launch_weight_grad_tc(gnnco_handle* h, const void* A, const void* G, float* dW, float* scratch, int K, int N,
                               cudaStream_t st);
+// Wc[s][k][n] = bf16(W[s][k][n]) and Wt[s][n][k] = bf16(W[s][k][n]) in one pass over W
+int32_t launch_cast_both_bf16(gnnco_handle* h, const float* W, __nv_bfloat16* Wc, __nv_bfloat16* Wt, int K, int N,
+                              int32_t sets, cudaStream_t st);
 // Wt[s][n][k] = bf16(W[s][k][n])
 int32_t launch_cast_transpose_bf16(gnnco_handle* h, const float* W, __nv_bfloat16* Wt, int K, int N, int32_t sets,
                                    cudaStream_t st);

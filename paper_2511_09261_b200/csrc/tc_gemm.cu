@@ -388,6 +388,34 @@ __global__ void cast_transpose_bf16_kernel(const float* __restrict__ W, __nv_bfl
   }
 }
 
+// One pass over W [sets][K][N] float32 (K, N multiples of 64) that writes both bf16 copies the
+// tensor-core transforms read: Wc [sets][K][N] and Wt [sets][N][K].  A block owns a 64 x 64 tile.
+__global__ void __launch_bounds__(256) cast_both_bf16_kernel(const float* __restrict__ W, __nv_bfloat16* __restrict__ Wc,
+                                                             __nv_bfloat16* __restrict__ Wt, int K, int N) {
+  __shared__ float tile[64][65];
+  const int64_t base = (int64_t)blockIdx.z * K * N;
+  const int k0 = blockIdx.y * 64, n0 = blockIdx.x * 64;
+  const int q = threadIdx.x & 15, r = threadIdx.x >> 4;   // 16 threads of four elements across, 16 rows per pass
+#pragma unroll
+  for (int pass = 0; pass < 4; ++pass) {
+    const int k = r + 16 * pass;
+    const int64_t at = base + (int64_t)(k0 + k) * N + n0 + 4 * q;
+    const float4 v = __ldg(reinterpret_cast<const float4*>(W + at));
+    __nv_bfloat162 lo = __floats2bfloat162_rn(v.x, v.y), hi = __floats2bfloat162_rn(v.z, v.w);
+    *reinterpret_cast<uint2*>(Wc + at) = make_uint2(*reinterpret_cast<uint32_t*>(&lo), *reinterpret_cast<uint32_t*>(&hi));
+    tile[k][4 * q + 0] = v.x; tile[k][4 * q + 1] = v.y; tile[k][4 * q + 2] = v.z; tile[k][4 * q + 3] = v.w;
+  }
+  __syncthreads();
+#pragma unroll
+  for (int pass = 0; pass < 4; ++pass) {
+    const int n = r + 16 * pass;
+    __nv_bfloat162 lo = __floats2bfloat162_rn(tile[4 * q + 0][n], tile[4 * q + 1][n]);
+    __nv_bfloat162 hi = __floats2bfloat162_rn(tile[4 * q + 2][n], tile[4 * q + 3][n]);
+    *reinterpret_cast<uint2*>(Wt + base + (int64_t)(n0 + n) * K + k0 + 4 * q) =
+        make_uint2(*reinterpret_cast<uint32_t*>(&lo), *reinterpret_cast<uint32_t*>(&hi));
+  }
+}
+
 }  // namespace
 
 bool tc_transform_supported(int dtype, int K, int N) {
@@ -426,6 +454,19 @@ int32_t launch_weight_grad_tc(gnnco_handle* h, const void* A, const void* G, flo
   GNNCO_WG_CASE(256, 64); GNNCO_WG_CASE(256, 128); GNNCO_WG_CASE(256, 256);
 #undef GNNCO_WG_CASE
   return GNNCO_UNSUPPORTED;
+}
+
+int32_t launch_cast_both_bf16(gnnco_handle* h, const float* W, __nv_bfloat16* Wc, __nv_bfloat16* Wt, int K, int N,
+                              int32_t sets, cudaStream_t st) {
+  if ((K % 64) || (N % 64) || ((uintptr_t)W & 15) || ((uintptr_t)Wc & 7) || ((uintptr_t)Wt & 7) || sets > 65535) {
+    int32_t rc = launch_cast_bf16(h, W, Wc, (int64_t)K * N * sets, st);
+    return rc != GNNCO_OK ? rc : launch_cast_transpose_bf16(h, W, Wt, K, N, sets, st);
+  }
+  ProfScope prof_(h, K_CAST, st);
+  cast_both_bf16_kernel<<<dim3(N / 64, K / 64, sets), 256, 0, st>>>(W, Wc, Wt, K, N);
+  h->launches += 1;
+  GNNCO_LAUNCH_CHECK();
+  return GNNCO_OK;
 }
 
 int32_t launch_cast_transpose_bf16(gnnco_handle* h, const float* W, __nv_bfloat16* Wt, int K, int N, int32_t sets,

@@ -122,10 +122,11 @@ int32_t run_step(gnnco_handle* h, const gnnco_model_desc* m, const void* X, cons
     const int64_t wc = (int64_t)m->dims[l] * m->dims[l + 1];
     wstride[l] = sets == 1 ? 0 : wc;
     if (bf16) {
-      GNNCO_TRY(launch_cast_bf16(h, m->W[l], T.W_lp[l], wc * sets, st));
-      Wc[l] = T.W_lp[l];
       if (T.W_lp_t[l])
-        GNNCO_TRY(launch_cast_transpose_bf16(h, m->W[l], T.W_lp_t[l], m->dims[l], m->dims[l + 1], sets, st));
+        GNNCO_TRY(launch_cast_both_bf16(h, m->W[l], T.W_lp[l], T.W_lp_t[l], m->dims[l], m->dims[l + 1], sets, st));
+      else
+        GNNCO_TRY(launch_cast_bf16(h, m->W[l], T.W_lp[l], wc * sets, st));
+      Wc[l] = T.W_lp[l];
     } else {
       Wc[l] = m->W[l];
       if (T.W3_t[l]) GNNCO_TRY(launch_cast_split3(h, m->W[l], T.W3_t[l], m->dims[l], m->dims[l + 1], sets, true, st));
