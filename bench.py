@@ -156,7 +156,7 @@ class ClockSampler:
                         self.reasons.add(name)
             except Exception:
                 pass
-            self._stop.wait(0.1)
+            self._stop.wait(0.02)
 
     def start(self):
         if self.nv is not None:
@@ -184,9 +184,15 @@ def algorithmic_bytes(kind, w, n, nnz, S):
     per = {}
     if hidden:
         per["aggregate_fwd"] = np.mean([2 * n * d[l - 1] * b + csr + 4 * n for l in hidden])
-        per["aggregate_bwd"] = np.mean([2 * n * d[l - 1] * b + csr + (n * d[l - 1] * b if l > 1 else 0) for l in hidden])
+        # transposed aggregation of layers 2..L-1 (plain gather-sum, no scale, no mask)
+        per["aggregate_bwd"] = np.mean([2 * n * d[l - 1] * b + csr for l in hidden[1:]]) if L > 2 else 0.0
+        # rank-1 mode below the output layer: gathers H_{L-1}, reads coef and the weight vectors
+        per["aggregate_rank1"] = 2 * n * d[L - 1] * b + csr + 4 * n + S * d[L - 1] * b
         per["transform_fwd"] = np.mean([n * (d[l - 1] + d[l]) * b + S * d[l - 1] * d[l] * b for l in hidden])
-        per["transform_bwd"] = np.mean([n * (d[l - 1] + d[l]) * b + 4 * n + S * d[l - 1] * d[l] * b for l in hidden])
+        # input gradient: reads Q_l and the weights, writes n x d[l-1]; layers above the first also
+        # read the saved activation (ReLU mask) and inv_deg
+        per["transform_bwd"] = np.mean([n * (d[l - 1] + d[l]) * b + S * d[l - 1] * d[l] * b +
+                                        ((n * d[l - 1] * b + 4 * n) if l > 1 else 0) for l in hidden])
         per["weight_grad"] = np.mean([n * (d[l - 1] + d[l]) * b + S * d[l - 1] * d[l] * 4 for l in hidden])
     F = d[L - 1]
     per["gemv"] = n * F * b + 4 * n + S * F * b
@@ -329,7 +335,7 @@ def run_ours(args):
                     frac=round(achieved / peak, 4), traffic=TRAFFIC_BYTES.get((args.config, top)) if args.scale == 1.0 else None,
                     peak_source="%s (MEASURED_PEAKS.json hbm_gbs)" % peak_src if peak_src == "measured" else "fallback",
                     algorithmic_bytes_per_launch=algorithmic_bytes(top, w, w.n, nnz, w.S))
-    agg = {k: kern[k] for k in ("aggregate_fwd", "aggregate_bwd") if k in kern}
+    agg = {k: kern[k] for k in ("aggregate_fwd", "aggregate_bwd", "aggregate_rank1") if k in kern}
 
     # ---- Stage-3 glue after the last decode (not part of the timed step): conflict list + base
     # action + penalty list / active subgraphs, timed with CUDA events on the current stream
@@ -415,10 +421,8 @@ def run_ours(args):
 # kernels as they stand, taken on configuration 5 at one tenth of the size and scaled by 10 (the
 # traffic is proportional to the node count); an entry is removed when its kernel changes.
 TRAFFIC_BYTES = {
-    (5, "aggregate_bwd"): 15.37e9,
     (5, "aggregate_fwd"): 10.07e9,
     (5, "transform_fwd"): 11.53e9,
-    (5, "transform_bwd"): 11.63e9,
 }
 
 
@@ -451,7 +455,7 @@ def run_reference(args):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=5)
+    ap.add_argument("--steps", type=int, default=20)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--config", type=int, default=5, choices=[1, 2, 3, 4, 5])
     ap.add_argument("--scale", type=float, default=1.0,

@@ -7,6 +7,7 @@
 //   loss_s = sum_{i in s} ( alpha/2 * p_i q_i + c_i p_i ),  c_i = -beta + lambda * pen_i
 //   dz_i = (alpha q_i + c_i) p_i (1 - p_i),  t_i = inv_deg_i dz_i
 //   g_i  = t_i + sum_{j in N(i)} t_j            ( = (A_hat^T dz)_i, adjacency symmetric )
+//   coef_i = inv_deg_i g_i                      ( row scale of the next transposed aggregation )
 //
 // All three passes are one thread per row; a row longer than 32 entries is instead summed
 // by its whole warp, so a hub cannot stall its warp for thousands of dependent loads.
@@ -116,14 +117,19 @@ __global__ void sum_items_per_subgraph(const float* __restrict__ item_loss, cons
 }
 
 __global__ void __launch_bounds__(256) output_backward(const float* __restrict__ t, const int32_t* __restrict__ rowptr,
-                                                       const int32_t* __restrict__ colidx, float* __restrict__ g,
-                                                       int64_t n) {
+                                                       const int32_t* __restrict__ colidx,
+                                                       const float* __restrict__ inv_deg, float* __restrict__ g,
+                                                       float* __restrict__ coef, int64_t n) {
   const int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
   const bool active = i < n;
   int32_t r0 = 0, r1 = 0;
   if (active) { r0 = rowptr[i]; r1 = rowptr[i + 1]; }
   float s = row_sum(t, colidx, r0, r1, active);
-  if (active) g[i] = t[i] + s;
+  if (active) {
+    const float gi = t[i] + s;
+    g[i] = gi;
+    if (coef) coef[i] = inv_deg[i] * gi;
+  }
 }
 
 }  // namespace
@@ -149,10 +155,10 @@ int32_t launch_objective(gnnco_handle* h, const float* p, const float* pen, floa
   return GNNCO_OK;
 }
 
-int32_t launch_output_backward(gnnco_handle* h, const float* t, float* g, cudaStream_t st) {
+int32_t launch_output_backward(gnnco_handle* h, const float* t, float* g, float* coef, cudaStream_t st) {
   ProfScope prof_(h, K_OUT_BWD, st);
   unsigned grid = (unsigned)((h->n + 255) / 256);
-  output_backward<<<grid, 256, 0, st>>>(t, h->rowptr, h->colidx, g, h->n);
+  output_backward<<<grid, 256, 0, st>>>(t, h->rowptr, h->colidx, h->inv_deg, g, coef, h->n);
   h->launches += 1;
   GNNCO_LAUNCH_CHECK();
   return GNNCO_OK;

@@ -4,7 +4,8 @@
 // weight set.
 //
 //   transform      Y = act( A W_s ) or A W_s^T, optional per-row scale (folds D^-1 into
-//                  the tensor that feeds the transposed aggregation)
+//                  the tensor that feeds the transposed aggregation) and optional ReLU mask
+//                  taken from a saved activation of the same shape
 //   weight_grad    dW_s = A_s^T G_s        (one block per output tile, fixed row order)
 //   gemv / weight_grad_vec / rank1_masked  the same three roles for the last layer,
 //                  whose output width is 1 (Eq. 4)
@@ -26,6 +27,7 @@ template <typename TA, typename TW, bool TRANSB>
 __global__ void __launch_bounds__(256) transform_fma(const TA* __restrict__ A, const TW* __restrict__ W,
                                                      int64_t w_stride, TA* __restrict__ Y, int K, int N, int relu,
                                                      const float* __restrict__ row_scale,
+                                                     const TA* __restrict__ relu_mask,
                                                      const int32_t* __restrict__ tile_row0,
                                                      const int32_t* __restrict__ tile_rows,
                                                      const int32_t* __restrict__ node_part) {
@@ -91,6 +93,7 @@ __global__ void __launch_bounds__(256) transform_fma(const TA* __restrict__ A, c
       if (col >= N) continue;
       float v = acc[i][j] * s;
       if (relu) v = v > 0.0f ? v : 0.0f;
+      if (relu_mask && !(ld(relu_mask + (row0 + row) * N + col) > 0.0f)) v = 0.0f;
       st(Y + (row0 + row) * N + col, v);
     }
   }
@@ -364,14 +367,16 @@ inline unsigned blocks_for(int64_t work, int threads) { return (unsigned)((work 
 }  // namespace
 
 int32_t launch_transform(gnnco_handle* h, int dtype, const void* A, const void* W, int64_t w_stride, void* Y, int K,
-                         int N, bool transB, bool relu, const float* row_scale, cudaStream_t stream) {
+                         int N, bool transB, bool relu, const float* row_scale, const void* relu_mask,
+                         cudaStream_t stream) {
   ProfScope prof_(h, transB ? K_TRANSFORM_BWD : K_TRANSFORM_FWD, stream);
   if (h->n_tiles == 0) return GNNCO_OK;
   dim3 grid(h->n_tiles, (N + BN - 1) / BN);
   if (grid.y > 65535) return GNNCO_UNSUPPORTED;
 #define GNNCO_TRANSFORM(TA, TW, TB)                                                                            \
   transform_fma<TA, TW, TB><<<grid, 256, 0, stream>>>((const TA*)A, (const TW*)W, w_stride, (TA*)Y, K, N, relu, \
-                                                      row_scale, h->tile_row0, h->tile_rows, h->node_part)
+                                                      row_scale, (const TA*)relu_mask, h->tile_row0, h->tile_rows, \
+                                                      h->node_part)
   if (dtype == GNNCO_F32) {
     if (transB) GNNCO_TRANSFORM(float, float, true);
     else GNNCO_TRANSFORM(float, float, false);

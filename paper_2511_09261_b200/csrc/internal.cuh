@@ -28,7 +28,7 @@ constexpr int kItemRows = 1024;      // rows of one objective work item (never s
 // Kernel families, for launch accounting and per-kernel timing.
 enum KernelKind {
   K_AGG_FWD, K_AGG_BWD, K_TRANSFORM_FWD, K_TRANSFORM_BWD, K_WEIGHT_GRAD, K_GEMV, K_WEIGHT_GRAD_VEC, K_RANK1,
-  K_SUM_SETS, K_CAST, K_ADAM, K_OUT_FWD, K_OBJECTIVE, K_OUT_BWD, K_DECODE, K_STAGE3, K_KIND_COUNT
+  K_SUM_SETS, K_CAST, K_ADAM, K_OUT_FWD, K_OBJECTIVE, K_OUT_BWD, K_DECODE, K_STAGE3, K_AGG_RANK1, K_KIND_COUNT
 };
 
 // Optional per-kernel timing: while `on`, every launcher brackets its launches with a pair
@@ -116,11 +116,17 @@ struct Carver {
 // ---- spmm.cu : out[i] = scale[i] * (in[i] + sum_{j in row i} in[j]), optionally zeroed where mask[i,f] <= 0
 int32_t launch_aggregate(gnnco_handle* h, int dtype, const void* in, void* out, int F, const float* row_scale,
                          const void* relu_mask, cudaStream_t st);
+// out[i,f] = w_s[f] * sum_{j in {i} + row i} coef[j] * [H[j,f] > 0]: the transposed aggregation of
+// D^-1 (g w_s^T * [H > 0]) with coef = D^-1 g, gathered straight from the saved activation H
+int32_t launch_aggregate_rank1(gnnco_handle* h, int dtype, const void* H, const float* coef, const void* w,
+                               int64_t w_stride, void* out, int F, cudaStream_t st);
 
 // ---- dense.cu
-// Y[tile rows x N] = act( A[rows x K] * B_s ), B_s = W[s] (K x N) or, with transB, W[s]^T where W[s] is (N x K).
+// Y[tile rows x N] = act( A[rows x K] * B_s ), B_s = W[s] (K x N) or, with transB, W[s]^T where W[s] is (N x K);
+// with relu_mask (same shape as Y) the result is zeroed where relu_mask <= 0.
 int32_t launch_transform(gnnco_handle* h, int dtype, const void* A, const void* W, int64_t w_stride, void* Y, int K,
-                         int N, bool transB, bool relu, const float* row_scale, cudaStream_t st);
+                         int N, bool transB, bool relu, const float* row_scale, const void* relu_mask,
+                         cudaStream_t st);
 // u[i] = H[i,:] . w_s
 int32_t launch_gemv(gnnco_handle* h, int dtype, const void* H, const void* w, int64_t w_stride, float* u, int F,
                     cudaStream_t st);
@@ -144,10 +150,11 @@ int32_t launch_adam(gnnco_handle* h, float* W, float* m, float* v, const float* 
 
 // ---- tc_gemm.cu : the same transform on the tensor cores (bf16, widths 64/128/256)
 bool tc_transform_supported(int dtype, int K, int N);
-// Y = act(A B_s^T) * row_scale with A [n x K] and B [sets x N x K], K contiguous in both
+// Y = act(A B_s^T) * row_scale with A [n x K] and B [sets x N x K], K contiguous in both; zeroed where
+// relu_mask [n x N] <= 0 when that is given
 int32_t launch_transform_tc(gnnco_handle* h, const void* A, const void* B, int64_t b_stride, void* Y, int K, int N,
-                            bool relu, const float* row_scale, bool backward, const void* dot_w, int64_t dot_stride,
-                            float* dot_out, cudaStream_t st);
+                            bool relu, const float* row_scale, const void* relu_mask, bool backward, const void* dot_w,
+                            int64_t dot_stride, float* dot_out, cudaStream_t st);
 bool tc_weight_grad_supported(int dtype, int K, int N);
 int32_t launch_weight_grad_tc(gnnco_handle* h, const void* A, const void* G, float* dW, float* scratch, int K, int N,
                               cudaStream_t st);
@@ -163,7 +170,8 @@ bool tc_f32_transform_supported(int K, int N);
 bool tc_f32_weight_grad_supported(int K, int N);
 int32_t launch_transform_tc_f32(gnnco_handle* h, const void* A, const void* B_limbs, int64_t b_stride,
                                 int64_t b_limb_stride, void* Y, int K, int N, bool relu, const float* row_scale,
-                                bool backward, const void* dot_w, int64_t dot_stride, float* dot_out, cudaStream_t st);
+                                const void* relu_mask, bool backward, const void* dot_w, int64_t dot_stride,
+                                float* dot_out, cudaStream_t st);
 int32_t launch_weight_grad_tc_f32(gnnco_handle* h, const void* A, const void* G, float* dW, float* scratch, int K,
                                   int N, cudaStream_t st);
 // three bf16 limb copies of W [sets x K x N] (transposed: [sets x N x K]); limb l at out + l*sets*K*N
@@ -174,7 +182,8 @@ int32_t launch_cast_split3(gnnco_handle* h, const float* W, __nv_bfloat16* out, 
 int32_t launch_output_forward(gnnco_handle* h, const float* u, float* z, float* p, cudaStream_t st);
 int32_t launch_objective(gnnco_handle* h, const float* p, const float* pen, float alpha, float beta, float lambda,
                          float* item_loss, float* loss, float* t, cudaStream_t st);
-int32_t launch_output_backward(gnnco_handle* h, const float* t, float* g, cudaStream_t st);
+// g = t + sum of t over the row ( = A_hat^T dz ); coef (optional) = inv_deg * g
+int32_t launch_output_backward(gnnco_handle* h, const float* t, float* g, float* coef, cudaStream_t st);
 
 // ---- decode.cu
 int32_t launch_decode(gnnco_handle* h, const float* p, float thr, uint8_t* x, uint8_t* viol, int32_t* per_part,

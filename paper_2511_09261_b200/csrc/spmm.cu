@@ -8,6 +8,11 @@
 // producer of G folds D^-1 in, and this kernel runs with scale = NULL.  With `mask` the
 // result is zeroed where mask[i,f] <= 0 (ReLU derivative taken from the saved activation).
 //
+// Rank-1 mode (template flag R1), for the layer below the width-1 output layer: its incoming
+// gradient is dZ[j,f] = g_j w_s[f] [H[j,f] > 0], so the transposed aggregation of D^-1 dZ is
+//   out[i,f] = w_s[f] * sum_{j in {i} + row i} coef[j] [H[j,f] > 0],     coef = D^-1 g,
+// which gathers the saved activation H directly; dZ itself is never written.
+//
 // Mapping: a group of LPR lanes owns one row; every lane keeps VPL 16-byte vectors of the
 // row in float32 registers, so a feature row is read with 128-bit loads and each
 // neighbour row is one fully coalesced request.  Rows of one subgraph are adjacent in
@@ -26,9 +31,17 @@ struct Vec<float> {
     f[0] = v.x; f[1] = v.y; f[2] = v.z; f[3] = v.w;
   }
   __device__ static uint4 load_raw(const float* p) { return __ldg(reinterpret_cast<const uint4*>(p)); }
+  __device__ static void unpack(const uint4& v, float (&f)[4]) {
+    f[0] = __uint_as_float(v.x); f[1] = __uint_as_float(v.y); f[2] = __uint_as_float(v.z); f[3] = __uint_as_float(v.w);
+  }
   __device__ static void add_raw(float (&acc)[4], const uint4& v) {
     acc[0] += __uint_as_float(v.x); acc[1] += __uint_as_float(v.y);
     acc[2] += __uint_as_float(v.z); acc[3] += __uint_as_float(v.w);
+  }
+  // acc[e] += c where the element is positive
+  __device__ static void add_where_positive(float (&acc)[4], const uint4& v, float c) {
+    acc[0] += __uint_as_float(v.x) > 0.0f ? c : 0.0f; acc[1] += __uint_as_float(v.y) > 0.0f ? c : 0.0f;
+    acc[2] += __uint_as_float(v.z) > 0.0f ? c : 0.0f; acc[3] += __uint_as_float(v.w) > 0.0f ? c : 0.0f;
   }
   __device__ static void store(float* p, const float (&f)[4]) {
     *reinterpret_cast<float4*>(p) = make_float4(f[0], f[1], f[2], f[3]);
@@ -47,12 +60,28 @@ struct Vec<__nv_bfloat16> {
     }
   }
   __device__ static uint4 load_raw(const __nv_bfloat16* p) { return __ldg(reinterpret_cast<const uint4*>(p)); }
+  __device__ static void unpack(const uint4& v, float (&f)[8]) {
+    const uint32_t w[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+    for (int k = 0; k < 4; ++k) {
+      f[2 * k] = __uint_as_float(w[k] << 16);
+      f[2 * k + 1] = __uint_as_float(w[k] & 0xffff0000u);
+    }
+  }
   __device__ static void add_raw(float (&acc)[8], const uint4& v) {
     const uint32_t w[4] = {v.x, v.y, v.z, v.w};
 #pragma unroll
     for (int k = 0; k < 4; ++k) {
       acc[2 * k] += __uint_as_float(w[k] << 16);
       acc[2 * k + 1] += __uint_as_float(w[k] & 0xffff0000u);
+    }
+  }
+  __device__ static void add_where_positive(float (&acc)[8], const uint4& v, float c) {
+    const uint32_t w[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+    for (int k = 0; k < 4; ++k) {
+      acc[2 * k] += __uint_as_float(w[k] << 16) > 0.0f ? c : 0.0f;
+      acc[2 * k + 1] += __uint_as_float(w[k] & 0xffff0000u) > 0.0f ? c : 0.0f;
     }
   }
   __device__ static void store(__nv_bfloat16* p, const float (&f)[8]) {
@@ -71,16 +100,31 @@ __device__ __forceinline__ float to_f32(__nv_bfloat16 x) { return __bfloat162flo
 __device__ __forceinline__ void from_f32(float& d, float x) { d = x; }
 __device__ __forceinline__ void from_f32(__nv_bfloat16& d, float x) { d = __float2bfloat16_rn(x); }
 
+// Arguments of the rank-1 mode.
+template <typename T>
+struct Rank1Args {
+  const float* coef;            // D^-1 g, one value per node
+  const T* w;                   // output-layer weight vectors [sets x F], in the features' type
+  int64_t w_stride;             // 0 when all subgraphs share one vector
+  const int32_t* node_part;
+};
+
+template <typename T, bool R1>
+__device__ __forceinline__ void accumulate(float (&acc)[Vec<T>::N], const uint4& v, float c) {
+  if constexpr (R1) Vec<T>::add_where_positive(acc, v, c);
+  else Vec<T>::add_raw(acc, v);
+}
+
 // LPR lanes per row, VPL vectors per lane: row width F = LPR * VPL * Vec<T>::N elements.
 // row_head[i] = {first CSR slot, degree, first neighbour, second neighbour}: one 16-byte load
 // tells a row its extent AND its first two neighbours, so for the many rows of degree <= 2
 // the neighbour features are only one round trip behind the head instead of two.
-template <typename T, int LPR, int VPL>
+template <typename T, int LPR, int VPL, bool R1>
 __global__ void __launch_bounds__(256) aggregate_vec(const T* __restrict__ in, T* __restrict__ out,
                                                      const int4* __restrict__ row_head,
                                                      const int32_t* __restrict__ colidx,
                                                      const float* __restrict__ scale, const T* __restrict__ mask,
-                                                     int64_t n, int F, int skip_long) {
+                                                     const Rank1Args<T> r1, int64_t n, int F, int skip_long) {
   constexpr int VN = Vec<T>::N;
   constexpr int ROWS_PER_BLOCK = 256 / LPR;
   const int sub = threadIdx.x % LPR;
@@ -89,86 +133,127 @@ __global__ void __launch_bounds__(256) aggregate_vec(const T* __restrict__ in, T
   // the row's own features are requested before its CSR extent is known, so the two round
   // trips overlap
   float acc[VPL][VN];
+  uint4 own[VPL];
 #pragma unroll
-  for (int v = 0; v < VPL; ++v) Vec<T>::load(in + row * F + (v * LPR + sub) * VN, acc[v]);
+  for (int v = 0; v < VPL; ++v) own[v] = Vec<T>::load_raw(in + row * F + (v * LPR + sub) * VN);
+  float c_own = 0.0f;
+  int32_t part = 0;
+  if constexpr (R1) {
+    c_own = __ldg(r1.coef + row);
+    part = __ldg(r1.node_part + row);
+  }
   const int4 head = __ldg(row_head + row);
   const int32_t deg = head.y;
   if (skip_long && deg > kLongRowDegree) return;   // a whole block takes this row
   {
     uint4 t[2][VPL];
+    float c[2] = {0.0f, 0.0f};
     if (deg > 0) {
 #pragma unroll
       for (int v = 0; v < VPL; ++v) t[0][v] = Vec<T>::load_raw(in + (int64_t)head.z * F + (v * LPR + sub) * VN);
+      if constexpr (R1) c[0] = __ldg(r1.coef + head.z);
     }
     if (deg > 1) {
 #pragma unroll
       for (int v = 0; v < VPL; ++v) t[1][v] = Vec<T>::load_raw(in + (int64_t)head.w * F + (v * LPR + sub) * VN);
+      if constexpr (R1) c[1] = __ldg(r1.coef + head.w);
+    }
+#pragma unroll
+    for (int v = 0; v < VPL; ++v) {
+#pragma unroll
+      for (int e = 0; e < VN; ++e) acc[v][e] = 0.0f;
+      accumulate<T, R1>(acc[v], own[v], c_own);
     }
     if (deg > 0) {
 #pragma unroll
-      for (int v = 0; v < VPL; ++v) Vec<T>::add_raw(acc[v], t[0][v]);
+      for (int v = 0; v < VPL; ++v) accumulate<T, R1>(acc[v], t[0][v], c[0]);
     }
     if (deg > 1) {
 #pragma unroll
-      for (int v = 0; v < VPL; ++v) Vec<T>::add_raw(acc[v], t[1][v]);
+      for (int v = 0; v < VPL; ++v) accumulate<T, R1>(acc[v], t[1][v], c[1]);
     }
   }
-  const int32_t r1 = head.x + deg;
+  // rank-1 mode: this lane's piece of the subgraph's weight vector, requested while the
+  // neighbour rows are still in flight
+  uint4 wraw[VPL];
+  if constexpr (R1) {
+    const T* wv = r1.w + (int64_t)part * r1.w_stride;
+#pragma unroll
+    for (int v = 0; v < VPL; ++v) wraw[v] = Vec<T>::load_raw(wv + (v * LPR + sub) * VN);
+  }
+  const int32_t r1_end = head.x + deg;
   int32_t k = head.x + 2;
-  for (; k + 4 <= r1; k += 4) {
+  for (; k + 4 <= r1_end; k += 4) {
     int32_t j[4];
 #pragma unroll
     for (int u = 0; u < 4; ++u) j[u] = __ldg(colidx + k + u);
     uint4 t[4][VPL];
+    float c[4] = {0.0f, 0.0f, 0.0f, 0.0f};
 #pragma unroll
-    for (int u = 0; u < 4; ++u)
+    for (int u = 0; u < 4; ++u) {
 #pragma unroll
       for (int v = 0; v < VPL; ++v) t[u][v] = Vec<T>::load_raw(in + (int64_t)j[u] * F + (v * LPR + sub) * VN);
+      if constexpr (R1) c[u] = __ldg(r1.coef + j[u]);
+    }
 #pragma unroll
     for (int u = 0; u < 4; ++u)
 #pragma unroll
-      for (int v = 0; v < VPL; ++v) Vec<T>::add_raw(acc[v], t[u][v]);
+      for (int v = 0; v < VPL; ++v) accumulate<T, R1>(acc[v], t[u][v], c[u]);
   }
-  for (; k < r1; ++k) {
+  for (; k < r1_end; ++k) {
     const int64_t j = __ldg(colidx + k);
+    float c = 0.0f;
+    if constexpr (R1) c = __ldg(r1.coef + j);
 #pragma unroll
-    for (int v = 0; v < VPL; ++v) Vec<T>::add_raw(acc[v], Vec<T>::load_raw(in + j * F + (v * LPR + sub) * VN));
+    for (int v = 0; v < VPL; ++v)
+      accumulate<T, R1>(acc[v], Vec<T>::load_raw(in + j * F + (v * LPR + sub) * VN), c);
   }
-  const float s = scale ? __ldg(scale + row) : 1.0f;
+  if constexpr (R1) {
 #pragma unroll
-  for (int v = 0; v < VPL; ++v) {
-    const int64_t off = row * F + (v * LPR + sub) * VN;
-    if (mask) {
-      float m[VN];
-      Vec<T>::load(mask + off, m);
+    for (int v = 0; v < VPL; ++v) {
+      float wf[VN];
+      Vec<T>::unpack(wraw[v], wf);
 #pragma unroll
-      for (int e = 0; e < VN; ++e) acc[v][e] = m[e] > 0.0f ? acc[v][e] * s : 0.0f;
-    } else {
-#pragma unroll
-      for (int e = 0; e < VN; ++e) acc[v][e] *= s;
+      for (int e = 0; e < VN; ++e) acc[v][e] *= wf[e];
+      Vec<T>::store(out + row * F + (v * LPR + sub) * VN, acc[v]);
     }
-    Vec<T>::store(out + off, acc[v]);
+  } else {
+    const float s = scale ? __ldg(scale + row) : 1.0f;
+#pragma unroll
+    for (int v = 0; v < VPL; ++v) {
+      const int64_t off = row * F + (v * LPR + sub) * VN;
+      if (mask) {
+        float m[VN];
+        Vec<T>::load(mask + off, m);
+#pragma unroll
+        for (int e = 0; e < VN; ++e) acc[v][e] = m[e] > 0.0f ? acc[v][e] * s : 0.0f;
+      } else {
+#pragma unroll
+        for (int e = 0; e < VN; ++e) acc[v][e] *= s;
+      }
+      Vec<T>::store(out + off, acc[v]);
+    }
   }
 }
 
 // A row with more than kLongRowDegree neighbours: one block per row.  Each of the 8 warps sums
 // a contiguous eighth of the neighbour list with eight rows in flight, the partial sums
 // meet in shared memory in warp order (deterministic), and the block finishes the row.
-template <typename T, int LPR, int VPL>
+template <typename T, int LPR, int VPL, bool R1>
 __global__ void __launch_bounds__(256) aggregate_long_row(const T* __restrict__ in, T* __restrict__ out,
                                                           const int32_t* __restrict__ rowptr,
                                                           const int32_t* __restrict__ colidx,
                                                           const float* __restrict__ scale,
-                                                          const T* __restrict__ mask,
+                                                          const T* __restrict__ mask, const Rank1Args<T> r1,
                                                           const int32_t* __restrict__ long_rows, int F) {
   constexpr int VN = Vec<T>::N;
   constexpr int GROUPS = 256 / LPR;               // lane groups, each walks its own slice of the row
   extern __shared__ float partial[];              // [GROUPS][F]
   const int64_t row = long_rows[blockIdx.x];
   const int sub = threadIdx.x % LPR, grp = threadIdx.x / LPR;
-  const int32_t r0 = rowptr[row], r1 = rowptr[row + 1];
-  const int32_t len = (r1 - r0 + GROUPS - 1) / GROUPS;
-  const int32_t a = r0 + grp * len, b = min(r1, a + len);
+  const int32_t r0 = rowptr[row], r1_end = rowptr[row + 1];
+  const int32_t len = (r1_end - r0 + GROUPS - 1) / GROUPS;
+  const int32_t a = r0 + grp * len, b = min(r1_end, a + len);
   float acc[VPL][VN];
 #pragma unroll
   for (int v = 0; v < VPL; ++v)
@@ -176,18 +261,22 @@ __global__ void __launch_bounds__(256) aggregate_long_row(const T* __restrict__ 
     for (int e = 0; e < VN; ++e) acc[v][e] = 0.0f;
   for (int32_t k = a; k < b; k += 8) {
     uint4 t[8][VPL];
+    float c[8];
 #pragma unroll
-    for (int u = 0; u < 8; ++u)
+    for (int u = 0; u < 8; ++u) {
+      c[u] = 0.0f;
       if (k + u < b) {
-        const int64_t c = __ldg(colidx + k + u);
+        const int64_t col = __ldg(colidx + k + u);
 #pragma unroll
-        for (int v = 0; v < VPL; ++v) t[u][v] = Vec<T>::load_raw(in + c * F + (v * LPR + sub) * VN);
+        for (int v = 0; v < VPL; ++v) t[u][v] = Vec<T>::load_raw(in + col * F + (v * LPR + sub) * VN);
+        if constexpr (R1) c[u] = __ldg(r1.coef + col);
       }
+    }
 #pragma unroll
     for (int u = 0; u < 8; ++u)
       if (k + u < b) {
 #pragma unroll
-        for (int v = 0; v < VPL; ++v) Vec<T>::add_raw(acc[v], t[u][v]);
+        for (int v = 0; v < VPL; ++v) accumulate<T, R1>(acc[v], t[u][v], c[u]);
       }
   }
 #pragma unroll
@@ -195,43 +284,68 @@ __global__ void __launch_bounds__(256) aggregate_long_row(const T* __restrict__ 
 #pragma unroll
     for (int e = 0; e < VN; ++e) partial[grp * F + (v * LPR + sub) * VN + e] = acc[v][e];
   __syncthreads();
-  const float sc = scale ? scale[row] : 1.0f;
-  for (int f = threadIdx.x; f < F; f += 256) {
-    float tot = to_f32(in[row * F + f]);
-    for (int g = 0; g < GROUPS; ++g) tot += partial[g * F + f];
-    tot *= sc;
-    if (mask && !(to_f32(mask[row * F + f]) > 0.0f)) tot = 0.0f;
-    from_f32(out[row * F + f], tot);
+  if constexpr (R1) {
+    const float ci = r1.coef[row];
+    const T* wv = r1.w + (int64_t)r1.node_part[row] * r1.w_stride;
+    for (int f = threadIdx.x; f < F; f += 256) {
+      float tot = to_f32(in[row * F + f]) > 0.0f ? ci : 0.0f;
+      for (int g = 0; g < GROUPS; ++g) tot += partial[g * F + f];
+      from_f32(out[row * F + f], tot * to_f32(wv[f]));
+    }
+  } else {
+    const float sc = scale ? scale[row] : 1.0f;
+    for (int f = threadIdx.x; f < F; f += 256) {
+      float tot = to_f32(in[row * F + f]);
+      for (int g = 0; g < GROUPS; ++g) tot += partial[g * F + f];
+      tot *= sc;
+      if (mask && !(to_f32(mask[row * F + f]) > 0.0f)) tot = 0.0f;
+      from_f32(out[row * F + f], tot);
+    }
   }
 }
 
 // Any width: one warp per row, lanes stride over the features with scalar accesses.
-template <typename T>
+template <typename T, bool R1>
 __global__ void __launch_bounds__(256) aggregate_any(const T* __restrict__ in, T* __restrict__ out,
                                                      const int32_t* __restrict__ rowptr,
                                                      const int32_t* __restrict__ colidx,
                                                      const float* __restrict__ scale, const T* __restrict__ mask,
-                                                     int64_t n, int F) {
+                                                     const Rank1Args<T> r1, int64_t n, int F) {
   const int lane = threadIdx.x & 31;
   const int64_t row = (int64_t)blockIdx.x * 8 + (threadIdx.x >> 5);
   if (row >= n) return;
-  const int32_t r0 = rowptr[row], r1 = rowptr[row + 1];
-  const float s = scale ? scale[row] : 1.0f;
-  for (int f = lane; f < F; f += 32) {
-    float acc = to_f32(in[row * F + f]);
-    for (int32_t k = r0; k < r1; ++k) acc += to_f32(in[(int64_t)colidx[k] * F + f]);
-    acc *= s;
-    if (mask && !(to_f32(mask[row * F + f]) > 0.0f)) acc = 0.0f;
-    from_f32(out[row * F + f], acc);
+  const int32_t r0 = rowptr[row], r1_end = rowptr[row + 1];
+  if constexpr (R1) {
+    const float ci = r1.coef[row];
+    const T* wv = r1.w + (int64_t)r1.node_part[row] * r1.w_stride;
+    for (int f = lane; f < F; f += 32) {
+      float acc = to_f32(in[row * F + f]) > 0.0f ? ci : 0.0f;
+      for (int32_t k = r0; k < r1_end; ++k) {
+        const int64_t j = colidx[k];
+        acc += to_f32(in[j * F + f]) > 0.0f ? r1.coef[j] : 0.0f;
+      }
+      from_f32(out[row * F + f], acc * to_f32(wv[f]));
+    }
+  } else {
+    const float s = scale ? scale[row] : 1.0f;
+    for (int f = lane; f < F; f += 32) {
+      float acc = to_f32(in[row * F + f]);
+      for (int32_t k = r0; k < r1_end; ++k) acc += to_f32(in[(int64_t)colidx[k] * F + f]);
+      acc *= s;
+      if (mask && !(to_f32(mask[row * F + f]) > 0.0f)) acc = 0.0f;
+      from_f32(out[row * F + f], acc);
+    }
   }
 }
 
-template <typename T, int LPR, int VPL>
-void launch_vec(const T* in, T* out, gnnco_handle* h, const float* scale, const T* mask, int F, cudaStream_t st) {
+template <typename T, int LPR, int VPL, bool R1>
+void launch_vec(const T* in, T* out, gnnco_handle* h, const float* scale, const T* mask, const Rank1Args<T>& r1, int F,
+                cudaStream_t st) {
   constexpr int ROWS_PER_BLOCK = 256 / LPR;
   const unsigned main_blocks = (unsigned)((h->n + ROWS_PER_BLOCK - 1) / ROWS_PER_BLOCK);
   if (h->n_long == 0) {
-    aggregate_vec<T, LPR, VPL><<<main_blocks, 256, 0, st>>>(in, out, h->row_head, h->colidx, scale, mask, h->n, F, 0);
+    aggregate_vec<T, LPR, VPL, R1><<<main_blocks, 256, 0, st>>>(in, out, h->row_head, h->colidx, scale, mask, r1, h->n,
+                                                                F, 0);
     return;
   }
   // A single warp walks a row of max_row entries in about max_row/4 dependent round trips of
@@ -244,43 +358,46 @@ void launch_vec(const T* in, T* out, gnnco_handle* h, const float* scale, const 
   const double walk_us = (double)h->max_row / 4.0;
   const bool inline_first = stream_us > 3.0 * walk_us;
   if (inline_first) {
-    aggregate_vec<T, LPR, VPL><<<main_blocks, 256, 0, st>>>(in, out, h->row_head, h->colidx, scale, mask, h->n, F, 0);
+    aggregate_vec<T, LPR, VPL, R1><<<main_blocks, 256, 0, st>>>(in, out, h->row_head, h->colidx, scale, mask, r1, h->n,
+                                                                F, 0);
     return;
   }
   const bool fork = h->side_stream && h->ev_fork && h->ev_join && cudaEventRecord(h->ev_fork, st) == cudaSuccess &&
                     cudaStreamWaitEvent(h->side_stream, h->ev_fork, 0) == cudaSuccess;
   cudaStream_t ls = fork ? h->side_stream : st;
-  aggregate_long_row<T, LPR, VPL><<<h->n_long, 256, (size_t)(256 / LPR) * F * sizeof(float), ls>>>(
-      in, out, h->rowptr, h->colidx, scale, mask, h->long_rows, F);
+  aggregate_long_row<T, LPR, VPL, R1><<<h->n_long, 256, (size_t)(256 / LPR) * F * sizeof(float), ls>>>(
+      in, out, h->rowptr, h->colidx, scale, mask, r1, h->long_rows, F);
   h->launches += 1;
   if (fork) cudaEventRecord(h->ev_join, h->side_stream);
-  aggregate_vec<T, LPR, VPL><<<main_blocks, 256, 0, st>>>(in, out, h->row_head, h->colidx, scale, mask, h->n, F, 1);
+  aggregate_vec<T, LPR, VPL, R1><<<main_blocks, 256, 0, st>>>(in, out, h->row_head, h->colidx, scale, mask, r1, h->n, F,
+                                                              1);
   if (fork) cudaStreamWaitEvent(st, h->ev_join, 0);
 }
 
-template <typename T>
+template <typename T, bool R1>
 int32_t aggregate_typed(gnnco_handle* h, const T* in, T* out, int F, const float* scale, const T* mask,
-                        cudaStream_t st) {
+                        const Rank1Args<T>& r1, cudaStream_t st) {
   constexpr int VN = Vec<T>::N;
   bool aligned = !((uintptr_t)in & 15) && !((uintptr_t)out & 15) && !((uintptr_t)mask & 15);
+  if (R1) aligned = aligned && !((uintptr_t)r1.w & 15) && (r1.w_stride % VN == 0);
   int vecs = F / VN;
   bool done = false;
   if (aligned && F % VN == 0) {
     done = true;
     switch (vecs) {
-      case 1: launch_vec<T, 1, 1>(in, out, h, scale, mask, F, st); break;
-      case 2: launch_vec<T, 2, 1>(in, out, h, scale, mask, F, st); break;
-      case 4: launch_vec<T, 4, 1>(in, out, h, scale, mask, F, st); break;
-      case 8: launch_vec<T, 8, 1>(in, out, h, scale, mask, F, st); break;
-      case 16: launch_vec<T, 16, 1>(in, out, h, scale, mask, F, st); break;
-      case 32: launch_vec<T, 32, 1>(in, out, h, scale, mask, F, st); break;
-      case 64: launch_vec<T, 32, 2>(in, out, h, scale, mask, F, st); break;
+      case 1: launch_vec<T, 1, 1, R1>(in, out, h, scale, mask, r1, F, st); break;
+      case 2: launch_vec<T, 2, 1, R1>(in, out, h, scale, mask, r1, F, st); break;
+      case 4: launch_vec<T, 4, 1, R1>(in, out, h, scale, mask, r1, F, st); break;
+      case 8: launch_vec<T, 8, 1, R1>(in, out, h, scale, mask, r1, F, st); break;
+      case 16: launch_vec<T, 16, 1, R1>(in, out, h, scale, mask, r1, F, st); break;
+      case 32: launch_vec<T, 32, 1, R1>(in, out, h, scale, mask, r1, F, st); break;
+      case 64: launch_vec<T, 32, 2, R1>(in, out, h, scale, mask, r1, F, st); break;
       default: done = false;
     }
   }
   if (!done) {
     unsigned grid = (unsigned)((h->n + 7) / 8);
-    aggregate_any<T><<<grid, 256, 0, st>>>(in, out, h->rowptr, h->colidx, scale, mask, h->n, F);
+    aggregate_any<T, R1><<<grid, 256, 0, st>>>(in, out, h->rowptr, h->colidx, scale, mask, r1, h->n, F);
   }
   h->launches += 1;
   GNNCO_LAUNCH_CHECK();
@@ -291,11 +408,27 @@ int32_t aggregate_typed(gnnco_handle* h, const T* in, T* out, int F, const float
 
 int32_t launch_aggregate(gnnco_handle* h, int dtype, const void* in, void* out, int F, const float* row_scale,
                          const void* relu_mask, cudaStream_t st) {
+  if (h->n == 0) return GNNCO_OK;
   ProfScope prof_(h, row_scale ? K_AGG_FWD : K_AGG_BWD, st);
   if (dtype == GNNCO_F32)
-    return aggregate_typed<float>(h, (const float*)in, (float*)out, F, row_scale, (const float*)relu_mask, st);
+    return aggregate_typed<float, false>(h, (const float*)in, (float*)out, F, row_scale, (const float*)relu_mask,
+                                         Rank1Args<float>{}, st);
   if (dtype == GNNCO_BF16)
-    return aggregate_typed<__nv_bfloat16>(h, (const __nv_bfloat16*)in, (__nv_bfloat16*)out, F, row_scale,
-                                          (const __nv_bfloat16*)relu_mask, st);
+    return aggregate_typed<__nv_bfloat16, false>(h, (const __nv_bfloat16*)in, (__nv_bfloat16*)out, F, row_scale,
+                                                 (const __nv_bfloat16*)relu_mask, Rank1Args<__nv_bfloat16>{}, st);
+  return GNNCO_UNSUPPORTED;
+}
+
+int32_t launch_aggregate_rank1(gnnco_handle* h, int dtype, const void* H, const float* coef, const void* w,
+                               int64_t w_stride, void* out, int F, cudaStream_t st) {
+  if (h->n == 0) return GNNCO_OK;
+  ProfScope prof_(h, K_AGG_RANK1, st);
+  if (dtype == GNNCO_F32)
+    return aggregate_typed<float, true>(h, (const float*)H, (float*)out, F, nullptr, nullptr,
+                                        Rank1Args<float>{coef, (const float*)w, w_stride, h->node_part}, st);
+  if (dtype == GNNCO_BF16)
+    return aggregate_typed<__nv_bfloat16, true>(
+        h, (const __nv_bfloat16*)H, (__nv_bfloat16*)out, F, nullptr, nullptr,
+        Rank1Args<__nv_bfloat16>{coef, (const __nv_bfloat16*)w, w_stride, h->node_part}, st);
   return GNNCO_UNSUPPORTED;
 }

@@ -2,6 +2,7 @@
 // with float32 accumulation (Eq. 3's "... W" and its input gradient).
 //
 //   Y[tile, :] = act( A[tile, 0:K] * B_s^T ) * row_scale,    B_s = [N x K], K contiguous
+//   (optionally zeroed where a saved activation of Y's shape is <= 0: the ReLU derivative)
 //
 // Forward uses B = W^T (bf16 copy, transposed), the input gradient uses B = W (bf16 copy), so
 // both operands are K-major.  One CTA owns a run of consecutive 128-row tiles; consecutive
@@ -16,13 +17,16 @@
 namespace {
 
 constexpr int kTileM = 128;
-constexpr int kThreads = 256;
+constexpr int kThreads = 256;                // weight-gradient kernel
+constexpr int kTfThreads = 384;              // transform kernel
 
-// Roles of the eight warps of the transform kernel.
-constexpr int kEpiWarps = 4;                 // warps 0-3 drain the accumulator (one TMEM lane quarter each)
-constexpr int kMmaWarp = 4;                  // warp 4 issues the MMAs
-constexpr int kProdWarp0 = 5;                // warps 5-7 stage operands with cp.async
+// Roles of the twelve warps of the transform kernel.
+constexpr int kEpiWarps = 8;                 // warps 0-7 drain the accumulator: TMEM lane quarter (warp % 4), column half (warp / 4)
+constexpr int kMmaWarp = 8;                  // warp 8 issues the MMAs
+constexpr int kProdWarp0 = 9;                // warps 9-11 stage operands with cp.async
 constexpr int kProdLanes = 96;
+
+constexpr uint32_t kTfMiscBytes = 1536;      // barriers (256 B) + two 128-float dot-product exchange buffers
 
 // One 64-wide k-block of `rows` rows (row stride KDIM elements) -> K-major SW128 shared memory:
 // row r at (r/8)*1024 + (r%8)*128, 16-byte chunk c at ((c ^ (r%8)) * 16).  Called by the 96
@@ -35,20 +39,30 @@ __device__ __forceinline__ void stage_kblock(uint32_t sdst, const __nv_bfloat16*
   }
 }
 
+// keep the bf16 halves of v where the matching halves of m are positive
+__device__ __forceinline__ uint32_t keep_where_positive(uint32_t v, uint32_t m) {
+  const uint32_t lo = __uint_as_float(m << 16) > 0.0f ? 0x0000ffffu : 0u;
+  const uint32_t hi = __uint_as_float(m & 0xffff0000u) > 0.0f ? 0xffff0000u : 0u;
+  return v & (lo | hi);
+}
+
 // Warp-specialised, persistent.  Shared memory: the subgraph's weight matrix (KB k-blocks of
 // NDIM rows) and one 128-row operand tile as KB independently recycled k-block slots.
 //   producers : wait until the MMAs that read slot kb are done, refill it (and the matching
 //               weight k-block when the subgraph changes), arrive on full[kb] when the copies land
 //   MMA warp  : for each k-block wait full[kb], issue 4 MMAs (K = 16 each) into accumulator
 //               buffer (tile & 1), commit -> empty[kb]; after the last k-block commit -> acc_full
-//   epilogue  : wait acc_full, read the accumulator (TMEM -> registers), scale / rectify /
-//               round to bf16, store; optionally the next layer's row dot product; arrive acc_empty
+//   epilogue  : two warps per TMEM lane quarter, each owning half of the columns: request the
+//               ReLU-mask lines of the tile (if any), wait acc_full, read the accumulator
+//               (TMEM -> registers), scale / rectify / round to bf16, store; optionally the
+//               next layer's row dot product (the two column halves meet in shared memory);
+//               arrive acc_empty
 // so the copies of tile t+1, the MMAs of tile t+1 and the drain of tile t overlap.
 template <int KDIM, int NDIM>
-__global__ void __launch_bounds__(kThreads, 1)
+__global__ void __launch_bounds__(kTfThreads, 1)
 transform_tc(const __nv_bfloat16* __restrict__ A, const __nv_bfloat16* __restrict__ B, int64_t b_stride,
              __nv_bfloat16* __restrict__ Y, int relu, const float* __restrict__ row_scale,
-             const __nv_bfloat16* __restrict__ dot_w, int64_t dot_stride, float* __restrict__ dot_out,
+             const __nv_bfloat16* __restrict__ relu_mask, const __nv_bfloat16* __restrict__ dot_w, int64_t dot_stride, float* __restrict__ dot_out,
              const int32_t* __restrict__ tile_row0, const int32_t* __restrict__ tile_rows,
              const int32_t* __restrict__ node_part, int n_tiles, int tiles_per_cta, int32_t* status) {
   constexpr int KB = KDIM / 64;
@@ -62,8 +76,10 @@ transform_tc(const __nv_bfloat16* __restrict__ A, const __nv_bfloat16* __restric
   uint64_t* empty = full + KB;                                                  // [KB]
   uint64_t* acc_full = empty + KB;                                              // [2]
   uint64_t* acc_empty = acc_full + 2;                                           // [2]
-  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(acc_empty + 2);
+  uint64_t* dot_bar = acc_empty + 2;                                            // [4 quarters][2 buffers]
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(dot_bar + 8);
   volatile uint32_t* abort_flag = tmem_slot + 1;
+  float* dot_x = reinterpret_cast<float*>(gen_base + A_BYTES + B_BYTES + 256);  // [2][128] upper column half's share
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int t_begin = blockIdx.x * tiles_per_cta;
@@ -79,6 +95,7 @@ transform_tc(const __nv_bfloat16* __restrict__ A, const __nv_bfloat16* __restric
       tc::mbar_init(acc_full + i, 1);
       tc::mbar_init(acc_empty + i, kEpiWarps * 32);
     }
+    for (int i = 0; i < 8; ++i) tc::mbar_init(dot_bar + i, 32);
     *abort_flag = 0;
     tc::fence_mbar_init();
   }
@@ -133,39 +150,55 @@ transform_tc(const __nv_bfloat16* __restrict__ A, const __nv_bfloat16* __restric
     }
   } else {
     // ---------------------------------------------------------------------- epilogue
-    const int row = warp * 32 + lane;
-    const uint32_t stage = sbase + A_BYTES + B_BYTES + 256 + warp * 4096;
-    int cur_part = -1;
+    constexpr int CHUNKS = NDIM / 64;                 // 64-column chunks of the tile
+    constexpr int PER = (CHUNKS + 1) / 2;             // chunks per column half
+    const int quarter = warp & 3, half = warp >> 2;
+    const int ch_begin = half * PER, ch_end = min(CHUNKS, ch_begin + PER);
+    const int row = quarter * 32 + lane;
+    const uint32_t stage = sbase + A_BYTES + B_BYTES + kTfMiscBytes + warp * 4096;
     for (int t = t_begin, j = 0; t < t_end && !*abort_flag; ++t, ++j) {
       const int buf = j & 1;
       const int64_t row0 = tile_row0[t];
       const int rows = tile_rows[t];
       const bool valid = row < rows;
+      const int rows_here = rows - quarter * 32;       // valid rows of this warp's 32
+      // the mask is read where the result will be stored (whole lines); every line of the tile
+      // that this warp needs is requested before the accumulator is waited for
+      uint4 mk[PER][8];
+      if (relu_mask) {
+#pragma unroll
+        for (int c = 0; c < PER; ++c)
+#pragma unroll
+          for (int it = 0; it < 8; ++it) {
+            const int rr = it * 4 + (lane >> 3);
+            mk[c][it] = make_uint4(0u, 0u, 0u, 0u);
+            if (rr < rows_here && ch_begin + c < ch_end)
+              mk[c][it] = __ldg(reinterpret_cast<const uint4*>(relu_mask + (row0 + quarter * 32 + rr) * NDIM +
+                                                               (ch_begin + c) * 64 + (lane & 7) * 8));
+          }
+      }
       const float s = (row_scale && valid) ? row_scale[row0 + row] : 1.0f;
       const __nv_bfloat16* wv = nullptr;
-      if (dot_out) {
-        const int part = node_part[row0];
-        cur_part = part;
-        wv = dot_w + (int64_t)part * dot_stride;
-      }
+      if (dot_out) wv = dot_w + (int64_t)node_part[row0] * dot_stride;
       float dot = 0.0f;
       if (!tc::mbar_wait_bounded(acc_full + buf, (j >> 1) & 1)) { *abort_flag = 1; break; }
       tc::tc_fence_after_sync();
-      const int rows_here = rows - warp * 32;          // valid rows of this warp's 32
-#pragma unroll 1
-      for (int c0 = 0; c0 < NDIM; c0 += 64) {
+#pragma unroll
+      for (int c = 0; c < PER; ++c) {
+        if (ch_begin + c >= ch_end) break;
+        const int c0 = (ch_begin + c) * 64;
         uint32_t o[32];                                // 64 bf16 of this thread's row, packed
 #pragma unroll
-        for (int half = 0; half < 2; ++half) {
+        for (int hh = 0; hh < 2; ++hh) {
           uint32_t r[32];
-          tc::tmem_ld_32x32(tmem + ((uint32_t)(warp * 32) << 16) + buf * NDIM + c0 + half * 32, r);
+          tc::tmem_ld_32x32(tmem + ((uint32_t)(quarter * 32) << 16) + buf * NDIM + c0 + hh * 32, r);
           tc::tmem_ld_wait();
 #pragma unroll
           for (int q = 0; q < 16; ++q) {
             float a = __uint_as_float(r[2 * q]) * s, b = __uint_as_float(r[2 * q + 1]) * s;
             if (relu) { a = a > 0.0f ? a : 0.0f; b = b > 0.0f ? b : 0.0f; }
             __nv_bfloat162 v = __floats2bfloat162_rn(a, b);
-            o[half * 16 + q] = *reinterpret_cast<uint32_t*>(&v);
+            o[hh * 16 + q] = *reinterpret_cast<uint32_t*>(&v);
           }
         }
         if (wv) {   // dot product of the STORED (rounded) row with the next layer's weight vector
@@ -192,16 +225,34 @@ transform_tc(const __nv_bfloat16* __restrict__ A, const __nv_bfloat16* __restric
 #pragma unroll
         for (int it = 0; it < 8; ++it) {
           const int rr = it * 4 + (lane >> 3), pc = lane & 7;
-          const uint4 v = tc::ld_shared16(stage + rr * 128 + ((pc ^ (rr & 7)) << 4));
+          uint4 v = tc::ld_shared16(stage + rr * 128 + ((pc ^ (rr & 7)) << 4));
+          if (relu_mask) {
+            v.x = keep_where_positive(v.x, mk[c][it].x); v.y = keep_where_positive(v.y, mk[c][it].y);
+            v.z = keep_where_positive(v.z, mk[c][it].z); v.w = keep_where_positive(v.w, mk[c][it].w);
+          }
           if (rr < rows_here)
-            *reinterpret_cast<uint4*>(Y + (row0 + warp * 32 + rr) * NDIM + c0 + pc * 8) = v;
+            *reinterpret_cast<uint4*>(Y + (row0 + quarter * 32 + rr) * NDIM + c0 + pc * 8) = v;
         }
       }
-      if (dot_out && valid) dot_out[row0 + row] = dot;
+      if (dot_out) {
+        // lower column half + upper column half, in that order.  The exchange buffer of this
+        // accumulator buffer is free again once the lower half has arrived on acc_empty below:
+        // the upper half cannot reach its next write before the MMAs of tile j + 2 are done.
+        if (CHUNKS > 1 && half == 1) {
+          dot_x[buf * 128 + row] = dot;
+          tc::mbar_arrive(dot_bar + quarter * 2 + buf);
+        }
+        if (half == 0) {
+          if (CHUNKS > 1) {
+            if (!tc::mbar_wait_bounded(dot_bar + quarter * 2 + buf, (j >> 1) & 1)) { *abort_flag = 1; break; }
+            dot += dot_x[buf * 128 + row];
+          }
+          if (valid) dot_out[row0 + row] = dot;
+        }
+      }
       tc::tc_fence_before_sync();
       tc::mbar_arrive(acc_empty + buf);
     }
-    (void)cur_part;
   }
   if (*abort_flag && threadIdx.x == 0) atomicMin(status, (int32_t)GNNCO_INTERNAL);
   tc::tc_fence_before_sync();
@@ -211,18 +262,21 @@ transform_tc(const __nv_bfloat16* __restrict__ A, const __nv_bfloat16* __restric
 
 template <int KDIM, int NDIM>
 int32_t launch_tc(gnnco_handle* h, const void* A, const void* B, int64_t b_stride, void* Y, bool relu,
-                  const float* row_scale, const void* dot_w, int64_t dot_stride, float* dot_out, cudaStream_t st) {
+                  const float* row_scale, const void* relu_mask, const void* dot_w, int64_t dot_stride, float* dot_out,
+                  cudaStream_t st) {
   constexpr int KB = KDIM / 64;
-  constexpr size_t smem = (size_t)KB * (kTileM + NDIM) * 128 + 256 + kEpiWarps * 4096 + 1024;
+  // operands, barriers and dot-product exchange, one 4 KB staging tile per epilogue warp, alignment slack
+  constexpr size_t smem = (size_t)KB * (kTileM + NDIM) * 128 + kTfMiscBytes + kEpiWarps * 4096 + 1024;
+  static_assert(smem <= 232448, "tile does not fit in shared memory");
   GNNCO_CUDA_TRY(cudaFuncSetAttribute(transform_tc<KDIM, NDIM>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                       (int)smem));
   int sms = h->sm_count > 0 ? h->sm_count : 148;
   int grid = h->n_tiles < sms ? h->n_tiles : sms;
   int per = (h->n_tiles + grid - 1) / grid;
   grid = (h->n_tiles + per - 1) / per;
-  transform_tc<KDIM, NDIM><<<grid, kThreads, smem, st>>>(
+  transform_tc<KDIM, NDIM><<<grid, kTfThreads, smem, st>>>(
       (const __nv_bfloat16*)A, (const __nv_bfloat16*)B, b_stride, (__nv_bfloat16*)Y, relu ? 1 : 0, row_scale,
-      (const __nv_bfloat16*)dot_w, dot_stride, dot_out, h->tile_row0, h->tile_rows, h->node_part, h->n_tiles, per,
+      (const __nv_bfloat16*)relu_mask, (const __nv_bfloat16*)dot_w, dot_stride, dot_out, h->tile_row0, h->tile_rows, h->node_part, h->n_tiles, per,
       h->status);
   h->launches += 1;
   GNNCO_LAUNCH_CHECK();
@@ -423,16 +477,18 @@ bool tc_transform_supported(int dtype, int K, int N) {
   return dtype == GNNCO_BF16 && ok(K) && ok(N);
 }
 
-// Y = act(A B_s^T) * row_scale with A [n x K], B [sets x N x K] (both bf16, K contiguous).
+// Y = act(A B_s^T) * row_scale with A [n x K], B [sets x N x K] (both bf16, K contiguous),
+// zeroed where relu_mask [n x N] (bf16, optional) is not positive.
 // With dot_out != nullptr also dot_out[i] = Y[i,:] . dot_w[s,:] (the width-1 output layer's
 // product, taken on the rounded values that are stored).
 int32_t launch_transform_tc(gnnco_handle* h, const void* A, const void* B, int64_t b_stride, void* Y, int K, int N,
-                            bool relu, const float* row_scale, bool backward, const void* dot_w, int64_t dot_stride,
-                            float* dot_out, cudaStream_t st) {
+                            bool relu, const float* row_scale, const void* relu_mask, bool backward, const void* dot_w,
+                            int64_t dot_stride, float* dot_out, cudaStream_t st) {
   if (h->n_tiles == 0) return GNNCO_OK;
   ProfScope prof_(h, backward ? K_TRANSFORM_BWD : K_TRANSFORM_FWD, st);
 #define GNNCO_TC_CASE(KK, NN) \
-  if (K == KK && N == NN) return launch_tc<KK, NN>(h, A, B, b_stride, Y, relu, row_scale, dot_w, dot_stride, dot_out, st)
+  if (K == KK && N == NN)       \
+  return launch_tc<KK, NN>(h, A, B, b_stride, Y, relu, row_scale, relu_mask, dot_w, dot_stride, dot_out, st)
   GNNCO_TC_CASE(64, 64); GNNCO_TC_CASE(64, 128); GNNCO_TC_CASE(64, 256);
   GNNCO_TC_CASE(128, 64); GNNCO_TC_CASE(128, 128); GNNCO_TC_CASE(128, 256);
   GNNCO_TC_CASE(256, 64); GNNCO_TC_CASE(256, 128); GNNCO_TC_CASE(256, 256);

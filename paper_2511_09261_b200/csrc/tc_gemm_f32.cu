@@ -60,7 +60,7 @@ template <int KDIM, int NDIM>
 __global__ void __launch_bounds__(kThreads, 1)
 transform_tc_f32(const float* __restrict__ A, const __nv_bfloat16* __restrict__ B, int64_t b_stride,
                  int64_t b_limb_stride, float* __restrict__ Y, int relu, const float* __restrict__ row_scale,
-                 const float* __restrict__ dot_w, int64_t dot_stride, float* __restrict__ dot_out,
+                 const float* __restrict__ relu_mask, const float* __restrict__ dot_w, int64_t dot_stride, float* __restrict__ dot_out,
                  const int32_t* __restrict__ tile_row0, const int32_t* __restrict__ tile_rows,
                  const int32_t* __restrict__ node_part, int n_tiles, int tiles_per_cta, int32_t* status) {
   constexpr int KB = KDIM / 64;
@@ -200,6 +200,17 @@ transform_tc_f32(const float* __restrict__ A, const __nv_bfloat16* __restrict__ 
       const int rows_here = rows - warp * 32;
 #pragma unroll 1
       for (int c0 = 0; c0 < NDIM; c0 += 32) {
+        // ReLU-derivative mask, read where the result will be stored, requested before the accumulator
+        float4 mk[8];
+        if (relu_mask) {
+#pragma unroll
+          for (int it = 0; it < 8; ++it) {
+            const int rr = it * 4 + (lane >> 3);
+            mk[it] = make_float4(0.f, 0.f, 0.f, 0.f);
+            if (rr < rows_here)
+              mk[it] = __ldg(reinterpret_cast<const float4*>(relu_mask + (row0 + warp * 32 + rr) * NDIM + c0 + (lane & 7) * 4));
+          }
+        }
         uint32_t r[32], rs[32];
         tc::tmem_ld_32x32(tmem + ((uint32_t)(warp * 32) << 16) + buf * 2 * NDIM + c0, r);
         tc::tmem_ld_32x32(tmem + ((uint32_t)(warp * 32) << 16) + buf * 2 * NDIM + NDIM + c0, rs);
@@ -229,7 +240,13 @@ transform_tc_f32(const float* __restrict__ A, const __nv_bfloat16* __restrict__ 
 #pragma unroll
         for (int it = 0; it < 8; ++it) {
           const int rr = it * 4 + (lane >> 3), pc = lane & 7;
-          const uint4 v = tc::ld_shared16(stage + rr * 128 + ((pc ^ (rr & 7)) << 4));
+          uint4 v = tc::ld_shared16(stage + rr * 128 + ((pc ^ (rr & 7)) << 4));
+          if (relu_mask) {
+            if (!(mk[it].x > 0.0f)) v.x = 0u;
+            if (!(mk[it].y > 0.0f)) v.y = 0u;
+            if (!(mk[it].z > 0.0f)) v.z = 0u;
+            if (!(mk[it].w > 0.0f)) v.w = 0u;
+          }
           if (rr < rows_here) *reinterpret_cast<uint4*>(Y + (row0 + warp * 32 + rr) * NDIM + c0 + pc * 4) = v;
         }
       }
@@ -246,8 +263,8 @@ transform_tc_f32(const float* __restrict__ A, const __nv_bfloat16* __restrict__ 
 
 template <int KDIM, int NDIM>
 int32_t launch_tf(gnnco_handle* h, const void* A, const void* B, int64_t b_stride, int64_t b_limb_stride, void* Y,
-                  bool relu, const float* row_scale, const void* dot_w, int64_t dot_stride, float* dot_out,
-                  cudaStream_t st) {
+                  bool relu, const float* row_scale, const void* relu_mask, const void* dot_w, int64_t dot_stride,
+                  float* dot_out, cudaStream_t st) {
   constexpr int KB = KDIM / 64;
   constexpr size_t smem = (size_t)KB * 3 * (kTileM + NDIM) * 128 + 256 + kEpiWarps * 4096 + 1024;
   static_assert(smem <= 232448, "tile does not fit in shared memory");
@@ -259,7 +276,7 @@ int32_t launch_tf(gnnco_handle* h, const void* A, const void* B, int64_t b_strid
   grid = (h->n_tiles + per - 1) / per;
   transform_tc_f32<KDIM, NDIM><<<grid, kThreads, smem, st>>>(
       (const float*)A, (const __nv_bfloat16*)B, b_stride, b_limb_stride, (float*)Y, relu ? 1 : 0, row_scale,
-      (const float*)dot_w, dot_stride, dot_out, h->tile_row0, h->tile_rows, h->node_part, h->n_tiles, per, h->status);
+      (const float*)relu_mask, (const float*)dot_w, dot_stride, dot_out, h->tile_row0, h->tile_rows, h->node_part, h->n_tiles, per, h->status);
   h->launches += 1;
   GNNCO_LAUNCH_CHECK();
   return GNNCO_OK;
@@ -462,13 +479,14 @@ bool tc_f32_weight_grad_supported(int K, int N) { return K == 128 && (N == 64 ||
 // Y = act(A B_s^T) * row_scale, A float32 [n x K], B = three bf16 limb copies of [sets x N x K]
 int32_t launch_transform_tc_f32(gnnco_handle* h, const void* A, const void* B_limbs, int64_t b_stride,
                                 int64_t b_limb_stride, void* Y, int K, int N, bool relu, const float* row_scale,
-                                bool backward, const void* dot_w, int64_t dot_stride, float* dot_out,
-                                cudaStream_t st) {
+                                const void* relu_mask, bool backward, const void* dot_w, int64_t dot_stride,
+                                float* dot_out, cudaStream_t st) {
   if (h->n_tiles == 0) return GNNCO_OK;
   ProfScope prof_(h, backward ? K_TRANSFORM_BWD : K_TRANSFORM_FWD, st);
 #define GNNCO_TF_CASE(KK, NN)    \
   if (K == KK && N == NN)        \
-  return launch_tf<KK, NN>(h, A, B_limbs, b_stride, b_limb_stride, Y, relu, row_scale, dot_w, dot_stride, dot_out, st)
+  return launch_tf<KK, NN>(h, A, B_limbs, b_stride, b_limb_stride, Y, relu, row_scale, relu_mask, dot_w, dot_stride, \
+                           dot_out, st)
   GNNCO_TF_CASE(64, 64); GNNCO_TF_CASE(64, 128); GNNCO_TF_CASE(128, 64); GNNCO_TF_CASE(128, 128);
 #undef GNNCO_TF_CASE
   return GNNCO_UNSUPPORTED;

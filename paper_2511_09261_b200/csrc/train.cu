@@ -3,13 +3,18 @@
 // launches happen here; every arithmetic step runs on the device.
 //
 // Forward, hidden layer l (1-based, widths d_{l-1} -> d_l):
-//     M_l = A_hat H_{l-1}            aggregate   (spmm.cu)
-//     H_l = ReLU(M_l W_l)            transform   (dense.cu)
+//     M_l = A_hat H_{l-1}            aggregate   (spmm.cu; M_l is a temporary, not kept)
+//     H_l = ReLU(M_l W_l)            transform   (dense.cu / tc_gemm*.cu)
 // Output layer:  u = H_{L-1} w_L ;  z = A_hat u ;  p = sigmoid(z)      (chain.cu)
 // Objective:     q = A p, per-subgraph loss, t = D^-1 dz ;  g = (A+I) t = A_hat^T dz
-// Backward:      dw_L = H_{L-1}^T g ;  dZ_{L-1} = (g w_L^T) * [H_{L-1} > 0]
-//     for l = L-1 .. 1:  dM_l = D^-1 (dZ_l W_l^T) ;  dW_l = M_l^T dZ_l ;  Adam on W_l
-//                        dZ_{l-1} = ((A+I) dM_l) * [H_{l-1} > 0]      (dX when l = 1)
+// Backward.  With Q_l = A_hat^T dZ_l = (A+I)(D^-1 dZ_l) the chain rule through
+// Z_l = A_hat H_{l-1} W_l reads  dW_l = H_{l-1}^T Q_l  and  dH_{l-1} = Q_l W_l^T, so only the
+// activations H_l are kept from the forward pass:
+//     dw_L = H_{L-1}^T g
+//     Q_{L-1} = (A+I) D^-1 (g w_L^T * [H_{L-1} > 0])                  aggregate, rank-1 mode
+//     for l = L-1 .. 1:  R = D^-1 ((Q_l W_l^T) * [H_{l-1} > 0])       transform with mask (dX = Q_1 W_1^T when l = 1)
+//                        dW_l = H_{l-1}^T Q_l ;  Adam on W_l
+//                        Q_{l-1} = (A+I) R                            aggregate
 // The transposed aggregation reuses the forward CSR because the intra adjacency is
 // symmetric: A_hat^T G = (A+I)(D^-1 G).
 #include <math.h>
@@ -19,10 +24,9 @@
 namespace {
 
 struct TrainLayout {
-  void* M[GNNCO_MAX_LAYERS];          // M[l], l = 1..L-1: aggregated input of hidden layer l
   void* H[GNNCO_MAX_LAYERS];          // H[l], l = 1..L-1: activation of hidden layer l
-  void* Ga;                           // gradient ping-pong buffers, n x max width
-  void* Gb;
+  void* Ga;                           // n x max width: aggregated input M_l (forward), then gradient ping-pong
+  void* Gb;                           // second gradient buffer (three or more layers, backward)
   float *u, *t, *g, *item_loss;
   float* dW_scratch;                  // one layer's gradient (all sets), when the caller wants none
   float* dW_sets;                     // per-subgraph partials when the model shares one weight set
@@ -69,17 +73,14 @@ TrainLayout carve_train(const gnnco_handle* h, const gnnco_model_desc* m, uint32
     size_t wc = (size_t)m->dims[l] * m->dims[l + 1];
     if (wc > max_wcount) max_wcount = wc;
   }
-  for (int l = 1; l < L; ++l) {
-    T.M[l] = c.take<char>(n * m->dims[l - 1] * es);
-    T.H[l] = c.take<char>(n * m->dims[l] * es);
-  }
+  for (int l = 1; l < L; ++l) T.H[l] = c.take<char>(n * m->dims[l] * es);
+  if (L > 1) T.Ga = c.take<char>(n * maxw * es);
   T.u = c.take<float>(n);
   T.t = c.take<float>(n);
   T.g = c.take<float>(n);
   T.item_loss = c.take<float>((size_t)h->n_items + 1);
   if (!(flags & GNNCO_FORWARD_ONLY)) {
-    T.Ga = c.take<char>(n * maxw * es);
-    T.Gb = c.take<char>(n * maxw * es);
+    if (L > 2) T.Gb = c.take<char>(n * maxw * es);
     T.dW_scratch = c.take<float>(max_wcount * m->weight_sets);
     if (m->weight_sets == 1) T.dW_sets = c.take<float>(max_wcount * (size_t)h->S);
     T.wg_scratch = c.take<float>(max_wcount * (size_t)h->n_wg_slots + 1);
@@ -139,23 +140,24 @@ int32_t run_step(gnnco_handle* h, const gnnco_model_desc* m, const void* X, cons
   const void* Hprev = X;
   bool u_done = false;
   for (int l = 1; l < L; ++l) {
-    GNNCO_TRY(launch_aggregate(h, dt, Hprev, T.M[l], m->dims[l - 1], h->inv_deg, nullptr, st));
+    GNNCO_TRY(launch_aggregate(h, dt, Hprev, T.Ga, m->dims[l - 1], h->inv_deg, nullptr, st));
     if (T.W_lp_t[l - 1]) {
       // the last hidden layer also produces u = H w_L in its epilogue
       const bool fuse = (l == L - 1) && (m->dims[l] % 8 == 0);
-      GNNCO_TRY(launch_transform_tc(h, T.M[l], T.W_lp_t[l - 1], wstride[l - 1], T.H[l], m->dims[l - 1], m->dims[l], true,
-                                    nullptr, false, fuse ? Wc[L - 1] : nullptr, wstride[L - 1], fuse ? T.u : nullptr, st));
+      GNNCO_TRY(launch_transform_tc(h, T.Ga, T.W_lp_t[l - 1], wstride[l - 1], T.H[l], m->dims[l - 1], m->dims[l], true,
+                                    nullptr, nullptr, false, fuse ? Wc[L - 1] : nullptr, wstride[L - 1],
+                                    fuse ? T.u : nullptr, st));
       u_done = fuse;
     } else if (T.W3_t[l - 1]) {
       const bool fuse = (l == L - 1) && (m->dims[l] % 4 == 0);
-      GNNCO_TRY(launch_transform_tc_f32(h, T.M[l], T.W3_t[l - 1], wstride[l - 1],
+      GNNCO_TRY(launch_transform_tc_f32(h, T.Ga, T.W3_t[l - 1], wstride[l - 1],
                                         (int64_t)m->dims[l - 1] * m->dims[l] * sets, T.H[l], m->dims[l - 1], m->dims[l],
-                                        true, nullptr, false, fuse ? Wc[L - 1] : nullptr, wstride[L - 1],
+                                        true, nullptr, nullptr, false, fuse ? Wc[L - 1] : nullptr, wstride[L - 1],
                                         fuse ? T.u : nullptr, st));
       u_done = fuse;
     } else
-      GNNCO_TRY(launch_transform(h, dt, T.M[l], Wc[l - 1], wstride[l - 1], T.H[l], m->dims[l - 1], m->dims[l], false,
-                                 true, nullptr, st));
+      GNNCO_TRY(launch_transform(h, dt, T.Ga, Wc[l - 1], wstride[l - 1], T.H[l], m->dims[l - 1], m->dims[l], false,
+                                 true, nullptr, nullptr, st));
     Hprev = T.H[l];
   }
   const int FL = m->dims[L - 1];
@@ -166,7 +168,8 @@ int32_t run_step(gnnco_handle* h, const gnnco_model_desc* m, const void* X, cons
                              fwd_only ? nullptr : T.t, st));
   if (fwd_only) return GNNCO_OK;
   // ---- backward
-  GNNCO_TRY(launch_output_backward(h, T.t, T.g, st));
+  // coef = D^-1 g takes the place of u, which the forward pass is done with
+  GNNCO_TRY(launch_output_backward(h, T.t, T.g, L > 1 ? T.u : nullptr, st));
   float c1 = 1.0f, c2 = 1.0f;
   if (opt) {
     c1 = (float)(1.0 - pow((double)opt->beta1, (double)opt->step));
@@ -181,6 +184,8 @@ int32_t run_step(gnnco_handle* h, const gnnco_model_desc* m, const void* X, cons
   };
   // gradient target of layer l: the caller's buffer or the scratch
   auto grad_target = [&](int l) -> float* { return out->dW[l] ? out->dW[l] : T.dW_scratch; };
+  void* Q = T.Ga;          // Q_l = A_hat^T dZ_l of the layer being processed
+  void* other = T.Gb;
   {
     // last layer (0-based index L-1): dw = H^T g
     float* target = grad_target(L - 1);
@@ -190,43 +195,41 @@ int32_t run_step(gnnco_handle* h, const gnnco_model_desc* m, const void* X, cons
     } else {
       GNNCO_TRY(launch_weight_grad_vec(h, dt, Hprev, T.g, target, FL, st));
     }
-    if (L > 1) GNNCO_TRY(launch_rank1_masked(h, dt, T.g, Wc[L - 1], wstride[L - 1], Hprev, T.Ga, FL, st));
+    // everything that reads the weights of a layer runs before that layer's Adam update
+    if (L > 1) GNNCO_TRY(launch_aggregate_rank1(h, dt, Hprev, T.u, Wc[L - 1], wstride[L - 1], Q, FL, st));
     else if (flags & GNNCO_WANT_DX)
       // L == 1: dX = A_hat^T (dz w_s^T) and w_s is constant inside a subgraph, so dX[i,:] = g_i w_s^T
       GNNCO_TRY(launch_rank1_masked(h, dt, T.g, Wc[0], wstride[0], nullptr, out->dX, FL, st));
     GNNCO_TRY(finish_layer(L - 1, target));
   }
-  void* dZ = T.Ga;
-  void* other = T.Gb;
   for (int l = L - 1; l >= 1; --l) {
     // hidden layer l uses weight index l-1: widths d_{l-1} -> d_l
     const int K = m->dims[l - 1], N = m->dims[l];
+    const void* Hin = l > 1 ? T.H[l - 1] : X;
     const bool need_input_grad = (l > 1) || (flags & GNNCO_WANT_DX);
     if (need_input_grad) {
+      // l > 1: R = D^-1 ((Q W^T) * [H_{l-1} > 0]);  l == 1: dX = Q W^T
+      void* dst = l > 1 ? other : out->dX;
+      const float* scale = l > 1 ? h->inv_deg : nullptr;
+      const void* mask = l > 1 ? T.H[l - 1] : nullptr;
       if (tc_transform_supported(dt, N, K))
-        GNNCO_TRY(launch_transform_tc(h, dZ, Wc[l - 1], wstride[l - 1], other, N, K, false, h->inv_deg, true, nullptr, 0,
+        GNNCO_TRY(launch_transform_tc(h, Q, Wc[l - 1], wstride[l - 1], dst, N, K, false, scale, mask, true, nullptr, 0,
                                       nullptr, st));
       else if (T.W3[l - 1])
-        GNNCO_TRY(launch_transform_tc_f32(h, dZ, T.W3[l - 1], wstride[l - 1], (int64_t)K * N * sets, other, N, K, false,
-                                          h->inv_deg, true, nullptr, 0, nullptr, st));
+        GNNCO_TRY(launch_transform_tc_f32(h, Q, T.W3[l - 1], wstride[l - 1], (int64_t)K * N * sets, dst, N, K, false,
+                                          scale, mask, true, nullptr, 0, nullptr, st));
       else
-        GNNCO_TRY(launch_transform(h, dt, dZ, Wc[l - 1], wstride[l - 1], other, N, K, true, false, h->inv_deg, st));
+        GNNCO_TRY(launch_transform(h, dt, Q, Wc[l - 1], wstride[l - 1], dst, N, K, true, false, scale, mask, st));
     }
     float* target = grad_target(l - 1);
     float* wg_out = sets == 1 ? T.dW_sets : target;
-    if (tc_weight_grad_supported(dt, K, N)) GNNCO_TRY(launch_weight_grad_tc(h, T.M[l], dZ, wg_out, T.wg_scratch, K, N, st));
+    if (tc_weight_grad_supported(dt, K, N)) GNNCO_TRY(launch_weight_grad_tc(h, Hin, Q, wg_out, T.wg_scratch, K, N, st));
     else if (dt == GNNCO_F32 && tc_f32_weight_grad_supported(K, N))
-      GNNCO_TRY(launch_weight_grad_tc_f32(h, T.M[l], dZ, wg_out, T.wg_scratch, K, N, st));
-    else GNNCO_TRY(launch_weight_grad(h, dt, T.M[l], dZ, wg_out, K, N, st));
+      GNNCO_TRY(launch_weight_grad_tc_f32(h, Hin, Q, wg_out, T.wg_scratch, K, N, st));
+    else GNNCO_TRY(launch_weight_grad(h, dt, Hin, Q, wg_out, K, N, st));
     if (sets == 1) GNNCO_TRY(launch_sum_over_sets(h, T.dW_sets, target, (int64_t)K * N, h->S, st));
     GNNCO_TRY(finish_layer(l - 1, target));
-    if (need_input_grad) {
-      if (l > 1) {
-        GNNCO_TRY(launch_aggregate(h, dt, other, dZ, K, nullptr, T.H[l - 1], st));   // new dZ in the old buffer
-      } else {
-        GNNCO_TRY(launch_aggregate(h, dt, other, out->dX, K, nullptr, nullptr, st));
-      }
-    }
+    if (l > 1) GNNCO_TRY(launch_aggregate(h, dt, other, Q, K, nullptr, nullptr, st));   // Q_{l-1} = (A+I) R
   }
 #undef GNNCO_TRY
   return GNNCO_OK;
