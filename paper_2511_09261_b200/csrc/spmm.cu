@@ -124,11 +124,38 @@ __global__ void __launch_bounds__(256) aggregate_vec(const T* __restrict__ in, T
                                                      const int4* __restrict__ row_head,
                                                      const int32_t* __restrict__ colidx,
                                                      const float* __restrict__ scale, const T* __restrict__ mask,
-                                                     const Rank1Args<T> r1, int64_t n, int F, int skip_long) {
+                                                     const Rank1Args<T> r1, int64_t n, int F, int skip_long,
+                                                     int prefetch_blocks) {
   constexpr int VN = Vec<T>::N;
   constexpr int ROWS_PER_BLOCK = 256 / LPR;
   const int sub = threadIdx.x % LPR;
   const int64_t row = (int64_t)blockIdx.x * ROWS_PER_BLOCK + threadIdx.x / LPR;
+  // Blocks are dispatched roughly in index order, so the block `prefetch_blocks` further on
+  // will run a few microseconds from now: ask for its rows and head records to be brought
+  // into L2 (no data returns to the SM, nothing to wait for), so that its first round trip
+  // is an L2 hit instead of a DRAM access.
+  if (threadIdx.x == 0 && prefetch_blocks > 0) {
+    const int64_t r0 = ((int64_t)blockIdx.x + prefetch_blocks) * ROWS_PER_BLOCK;
+    if (r0 + ROWS_PER_BLOCK <= n) {
+      asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;" ::"l"(in + r0 * F),
+                   "r"((uint32_t)(ROWS_PER_BLOCK * VPL * LPR * 16)) : "memory");
+      asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;" ::"l"(row_head + r0),
+                   "r"((uint32_t)(ROWS_PER_BLOCK * 16)) : "memory");
+      // per-row scalars: 4 bytes a row; the instruction wants 16-byte granules
+      auto prefetch_words = [&](const void* base) {
+        const char* a = static_cast<const char*>(base) + r0 * 4;
+        if ((ROWS_PER_BLOCK * 4) % 16 == 0 && ((uintptr_t)a & 15) == 0)
+          asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;" ::"l"(a), "r"((uint32_t)(ROWS_PER_BLOCK * 4))
+                       : "memory");
+      };
+      if constexpr (R1) {
+        prefetch_words(r1.coef);
+        prefetch_words(r1.node_part);
+      } else if (scale) {
+        prefetch_words(scale);
+      }
+    }
+  }
   if (row >= n) return;
   // the row's own features are requested before its CSR extent is known, so the two round
   // trips overlap
@@ -136,11 +163,13 @@ __global__ void __launch_bounds__(256) aggregate_vec(const T* __restrict__ in, T
   uint4 own[VPL];
 #pragma unroll
   for (int v = 0; v < VPL; ++v) own[v] = Vec<T>::load_raw(in + row * F + (v * LPR + sub) * VN);
-  float c_own = 0.0f;
+  float c_own = 0.0f, s = 1.0f;
   int32_t part = 0;
   if constexpr (R1) {
     c_own = __ldg(r1.coef + row);
     part = __ldg(r1.node_part + row);
+  } else if (scale) {
+    s = __ldg(scale + row);                          // with the first round trip, not after the last
   }
   const int4 head = __ldg(row_head + row);
   const int32_t deg = head.y;
@@ -183,20 +212,22 @@ __global__ void __launch_bounds__(256) aggregate_vec(const T* __restrict__ in, T
   }
   const int32_t r1_end = head.x + deg;
   int32_t k = head.x + 2;
-  for (; k + 4 <= r1_end; k += 4) {
-    int32_t j[4];
+  constexpr int U = 4;                               // neighbour rows in flight
+  for (; k + U <= r1_end; k += U) {
+    int32_t j[U];
 #pragma unroll
-    for (int u = 0; u < 4; ++u) j[u] = __ldg(colidx + k + u);
-    uint4 t[4][VPL];
-    float c[4] = {0.0f, 0.0f, 0.0f, 0.0f};
+    for (int u = 0; u < U; ++u) j[u] = __ldg(colidx + k + u);
+    uint4 t[U][VPL];
+    float c[U];
 #pragma unroll
-    for (int u = 0; u < 4; ++u) {
+    for (int u = 0; u < U; ++u) {
 #pragma unroll
       for (int v = 0; v < VPL; ++v) t[u][v] = Vec<T>::load_raw(in + (int64_t)j[u] * F + (v * LPR + sub) * VN);
+      c[u] = 0.0f;
       if constexpr (R1) c[u] = __ldg(r1.coef + j[u]);
     }
 #pragma unroll
-    for (int u = 0; u < 4; ++u)
+    for (int u = 0; u < U; ++u)
 #pragma unroll
       for (int v = 0; v < VPL; ++v) accumulate<T, R1>(acc[v], t[u][v], c[u]);
   }
@@ -218,7 +249,6 @@ __global__ void __launch_bounds__(256) aggregate_vec(const T* __restrict__ in, T
       Vec<T>::store(out + row * F + (v * LPR + sub) * VN, acc[v]);
     }
   } else {
-    const float s = scale ? __ldg(scale + row) : 1.0f;
 #pragma unroll
     for (int v = 0; v < VPL; ++v) {
       const int64_t off = row * F + (v * LPR + sub) * VN;
@@ -343,9 +373,24 @@ void launch_vec(const T* in, T* out, gnnco_handle* h, const float* scale, const 
                 cudaStream_t st) {
   constexpr int ROWS_PER_BLOCK = 256 / LPR;
   const unsigned main_blocks = (unsigned)((h->n + ROWS_PER_BLOCK - 1) / ROWS_PER_BLOCK);
+  const size_t long_smem = (size_t)(256 / LPR) * F * sizeof(float);
+  // L2 prefetch distance: one full wave of resident blocks (8 per SM) ahead; pointless on small grids
+  const int sms = h->sm_count > 0 ? h->sm_count : 148;
+  const int pf_blocks = main_blocks > 4u * 8u * (unsigned)sms ? 8 * sms : 0;
+  // the block-per-row kernel on the side stream, beside the kernel that follows on `st`
+  auto fork_long_rows = [&](const int32_t* list, int32_t count) -> bool {
+    const bool fork = h->side_stream && h->ev_fork && h->ev_join && cudaEventRecord(h->ev_fork, st) == cudaSuccess &&
+                      cudaStreamWaitEvent(h->side_stream, h->ev_fork, 0) == cudaSuccess;
+    cudaStream_t ls = fork ? h->side_stream : st;
+    aggregate_long_row<T, LPR, VPL, R1><<<count, 256, long_smem, ls>>>(in, out, h->rowptr, h->colidx, scale, mask, r1,
+                                                                       list, F);
+    h->launches += 1;
+    if (fork) cudaEventRecord(h->ev_join, h->side_stream);
+    return fork;
+  };
   if (h->n_long == 0) {
     aggregate_vec<T, LPR, VPL, R1><<<main_blocks, 256, 0, st>>>(in, out, h->row_head, h->colidx, scale, mask, r1, h->n,
-                                                                F, 0);
+                                                                F, 0, pf_blocks);
     return;
   }
   // A single warp walks a row of max_row entries in about max_row/4 dependent round trips of
@@ -359,18 +404,12 @@ void launch_vec(const T* in, T* out, gnnco_handle* h, const float* scale, const 
   const bool inline_first = stream_us > 3.0 * walk_us;
   if (inline_first) {
     aggregate_vec<T, LPR, VPL, R1><<<main_blocks, 256, 0, st>>>(in, out, h->row_head, h->colidx, scale, mask, r1, h->n,
-                                                                F, 0);
+                                                                F, 0, pf_blocks);
     return;
   }
-  const bool fork = h->side_stream && h->ev_fork && h->ev_join && cudaEventRecord(h->ev_fork, st) == cudaSuccess &&
-                    cudaStreamWaitEvent(h->side_stream, h->ev_fork, 0) == cudaSuccess;
-  cudaStream_t ls = fork ? h->side_stream : st;
-  aggregate_long_row<T, LPR, VPL, R1><<<h->n_long, 256, (size_t)(256 / LPR) * F * sizeof(float), ls>>>(
-      in, out, h->rowptr, h->colidx, scale, mask, r1, h->long_rows, F);
-  h->launches += 1;
-  if (fork) cudaEventRecord(h->ev_join, h->side_stream);
+  const bool fork = fork_long_rows(h->long_rows, h->n_long);
   aggregate_vec<T, LPR, VPL, R1><<<main_blocks, 256, 0, st>>>(in, out, h->row_head, h->colidx, scale, mask, r1, h->n, F,
-                                                              1);
+                                                              1, pf_blocks);
   if (fork) cudaStreamWaitEvent(st, h->ev_join, 0);
 }
 
