@@ -364,6 +364,28 @@ def run_ours(args):
                            "includes the binding's buffer allocations")
         del ca, ap
 
+    # ---- the same step with the first layer's aggregated input kept across steps (X is a fixed
+    # input, so this is legal; it is NOT the headline number, which recomputes it every step)
+    cached = None
+    if w.L > 1:
+        ax = torch.empty_like(X)
+        graph.train_step(model, X, w.alpha, w.beta, w.lam, pen, opt, loss=loss, p=p, dX=dX,
+                         flags=gnnco.WANT_DX | gnnco.AX_STORE, ax_cache=ax)
+        torch.cuda.synchronize()
+        c0, c1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        c0.record()
+        for _ in range(args.steps):
+            graph.train_step(model, X, w.alpha, w.beta, w.lam, pen, opt, loss=loss, p=p, dX=dX,
+                             flags=gnnco.WANT_DX | gnnco.AX_REUSE, ax_cache=ax)
+            graph.decode_boundary(p, 0.5, x=x, viol=viol, per_part=per_part, counts=counts)
+        c1.record()
+        torch.cuda.synchronize()
+        cms = max_over_ranks(dist, c0.elapsed_time(c1) / args.steps, dev)
+        cached = dict(ms_per_step=round(cms, 4), value=whole_job_value(graph.E_in, world, cms), unit="edges/s",
+                      note="GNNCO_AX_REUSE: first-layer aggregation of the fixed embeddings computed once, "
+                           "outside the timed steps; reported beside the headline, not instead of it")
+        del ax
+
     # ---- end to end through the host-buffer entry point (rank-local; copies inside the timed region)
     e2e = None
     if not args.no_e2e:
@@ -411,7 +433,7 @@ def run_ours(args):
                         parallelism="replicas only (no collective on the data path)" if world > 1 else "1 GPU",
                         partition_load_ms=round(load_ms, 3), edges_per_s_whole_graph=value * w.E / max(1, graph.E_in)),
             roofline=roofline, aggregate_kernels=agg, kernels=kern, cpu_baseline=cpu, clocks=clocks, e2e=e2e,
-            gpu_launches=int(launches), stage3_glue=stage3)
+            gpu_launches=int(launches), stage3_glue=stage3, cached_first_aggregation=cached)
         print(json.dumps(line))
     if dist is not None:
         dist.destroy_process_group()
@@ -419,10 +441,14 @@ def run_ours(args):
 
 # DRAM traffic per launch (dram__bytes_read.sum + dram__bytes_write.sum) from ncu captures of the
 # kernels as they stand, taken on configuration 5 at one tenth of the size and scaled by 10 (the
-# traffic is proportional to the node count); an entry is removed when its kernel changes.
+# traffic is proportional to the node count); averaged over the launches of a family inside one
+# step; an entry is removed when its kernel changes.
 TRAFFIC_BYTES = {
-    (5, "aggregate_fwd"): 10.07e9,
-    (5, "transform_fwd"): 11.53e9,
+    (5, "aggregate_fwd"): 10.03e9,
+    (5, "aggregate_bwd"): 10.00e9,
+    (5, "aggregate_rank1"): 10.17e9,
+    (5, "transform_fwd"): 11.62e9,
+    (5, "transform_bwd"): 15.05e9,
 }
 
 

@@ -54,6 +54,14 @@ typedef enum { GNNCO_F32 = 0, GNNCO_BF16 = 1 } gnnco_dtype;
 /* flags of gnnco_train_step */
 #define GNNCO_WANT_DX 1u        /* also compute d loss / d X (runs the transposed aggregation of layer 1) */
 #define GNNCO_FORWARD_ONLY 2u   /* stop after loss and p (Algorithm 1, Stage 2: "run forward to get p_i") */
+/* The embeddings X are fixed inputs (Section 3.2 updates "the weight matrix W" only), so the
+ * first layer's aggregated input  mean_{self + intra neighbours}(X)  of Eq. 3 is the same in
+ * every step of a run.  With GNNCO_AX_STORE the step keeps it in gnnco_train_out.ax_cache;
+ * with GNNCO_AX_REUSE the step skips that aggregation and reads ax_cache instead (the caller
+ * vouches that graph and X are those of the storing step).  Both need L >= 2 and a non-NULL
+ * ax_cache; results are bit-identical to the plain step. */
+#define GNNCO_AX_STORE 4u
+#define GNNCO_AX_REUSE 8u
 
 typedef struct gnnco_handle gnnco_handle;
 
@@ -135,6 +143,7 @@ typedef struct {
   float* z;                      /* [n]  pre-sigmoid values, or NULL */
   float* dW[GNNCO_MAX_LAYERS];   /* gradient of sum_s loss_s wrt W[l], shape of W[l], or NULL */
   void* dX;                      /* [n x dims[0]] in feat_dtype; written only with GNNCO_WANT_DX */
+  void* ax_cache;                /* [n x dims[0]] in feat_dtype; see GNNCO_AX_STORE / GNNCO_AX_REUSE; else NULL */
 } gnnco_train_out;
 
 typedef struct {

@@ -19,7 +19,7 @@ OK = 0
 INVALID_ARGUMENT, OUT_OF_RANGE, NOT_SIMPLE_GRAPH, UNSUPPORTED, WORKSPACE_TOO_SMALL, CUDA_ERROR, INTERNAL = (
     -1, -2, -3, -4, -5, -6, -7)
 F32, BF16 = 0, 1
-WANT_DX, FORWARD_ONLY = 1, 2
+WANT_DX, FORWARD_ONLY, AX_STORE, AX_REUSE = 1, 2, 4, 8
 
 EXPORTS = [
     "gnnco_status_string", "gnnco_partition_workspace_bytes", "gnnco_partition_load", "gnnco_graph_info",
@@ -58,7 +58,7 @@ class AdamState(ctypes.Structure):
 
 
 class TrainOut(ctypes.Structure):
-    _fields_ = [("loss", _vp), ("p", _vp), ("z", _vp), ("dW", _vp * MAX_LAYERS), ("dX", _vp)]
+    _fields_ = [("loss", _vp), ("p", _vp), ("z", _vp), ("dW", _vp * MAX_LAYERS), ("dX", _vp), ("ax_cache", _vp)]
 
 
 class ProfileEntry(ctypes.Structure):
@@ -284,9 +284,10 @@ class PartitionedGraph:
 
     def train_step(self, model: Model, X, alpha: float, beta: float, lam: float = 0.0, pen=None,
                    opt: Optional[Adam] = None, loss=None, p=None, z=None, dW: Optional[List] = None, dX=None,
-                   flags: int = 0, stream=None):
+                   flags: int = 0, stream=None, ax_cache=None):
         """One ``gnnco_train_step``.  Returns (loss, p).  Optional outputs are written
-        into the tensors passed as ``z``, ``dW`` (list, entries may be None) and ``dX``."""
+        into the tensors passed as ``z``, ``dW`` (list, entries may be None) and ``dX``;
+        ``ax_cache`` ([n, dims[0]], the features' type) goes with AX_STORE / AX_REUSE."""
         import torch
         _require(X, model.torch_feat_dtype, "X")
         if tuple(X.shape) != (self.n, model.dims[0]):
@@ -300,6 +301,11 @@ class PartitionedGraph:
         obj = Objective(alpha, beta, lam, _dptr(pen))
         out = TrainOut()
         out.loss, out.p, out.z, out.dX = _dptr(loss), _dptr(p), _dptr(z), _dptr(dX)
+        if ax_cache is not None:
+            _require(ax_cache, model.torch_feat_dtype, "ax_cache")
+            if tuple(ax_cache.shape) != (self.n, model.dims[0]):
+                raise ValueError("ax_cache must be [n, dims[0]]")
+            out.ax_cache = ax_cache.data_ptr()
         if dW is not None:
             for l, t in enumerate(dW):
                 out.dW[l] = _dptr(t)

@@ -140,23 +140,27 @@ int32_t run_step(gnnco_handle* h, const gnnco_model_desc* m, const void* X, cons
   const void* Hprev = X;
   bool u_done = false;
   for (int l = 1; l < L; ++l) {
-    GNNCO_TRY(launch_aggregate(h, dt, Hprev, T.Ga, m->dims[l - 1], h->inv_deg, nullptr, st));
+    // aggregated input M_l; the first layer's can be kept across steps (X does not change)
+    const void* Min = T.Ga;
+    if (l == 1 && (flags & (GNNCO_AX_STORE | GNNCO_AX_REUSE))) Min = out->ax_cache;
+    if (!(l == 1 && (flags & GNNCO_AX_REUSE)))
+      GNNCO_TRY(launch_aggregate(h, dt, Hprev, const_cast<void*>(Min), m->dims[l - 1], h->inv_deg, nullptr, st));
     if (T.W_lp_t[l - 1]) {
       // the last hidden layer also produces u = H w_L in its epilogue
       const bool fuse = (l == L - 1) && (m->dims[l] % 8 == 0);
-      GNNCO_TRY(launch_transform_tc(h, T.Ga, T.W_lp_t[l - 1], wstride[l - 1], T.H[l], m->dims[l - 1], m->dims[l], true,
+      GNNCO_TRY(launch_transform_tc(h, Min, T.W_lp_t[l - 1], wstride[l - 1], T.H[l], m->dims[l - 1], m->dims[l], true,
                                     nullptr, nullptr, false, fuse ? Wc[L - 1] : nullptr, wstride[L - 1],
                                     fuse ? T.u : nullptr, st));
       u_done = fuse;
     } else if (T.W3_t[l - 1]) {
       const bool fuse = (l == L - 1) && (m->dims[l] % 4 == 0);
-      GNNCO_TRY(launch_transform_tc_f32(h, T.Ga, T.W3_t[l - 1], wstride[l - 1],
+      GNNCO_TRY(launch_transform_tc_f32(h, Min, T.W3_t[l - 1], wstride[l - 1],
                                         (int64_t)m->dims[l - 1] * m->dims[l] * sets, T.H[l], m->dims[l - 1], m->dims[l],
                                         true, nullptr, nullptr, false, fuse ? Wc[L - 1] : nullptr, wstride[L - 1],
                                         fuse ? T.u : nullptr, st));
       u_done = fuse;
     } else
-      GNNCO_TRY(launch_transform(h, dt, T.Ga, Wc[l - 1], wstride[l - 1], T.H[l], m->dims[l - 1], m->dims[l], false,
+      GNNCO_TRY(launch_transform(h, dt, Min, Wc[l - 1], wstride[l - 1], T.H[l], m->dims[l - 1], m->dims[l], false,
                                  true, nullptr, nullptr, st));
     Hprev = T.H[l];
   }
@@ -239,7 +243,9 @@ int32_t check_step_args(const gnnco_handle* h, const gnnco_model_desc* m, const 
                         uint32_t flags) {
   int32_t rc = check_model(h, m, true);
   if (rc != GNNCO_OK) return rc;
-  if (flags & ~(GNNCO_WANT_DX | GNNCO_FORWARD_ONLY)) return GNNCO_INVALID_ARGUMENT;
+  if (flags & ~(GNNCO_WANT_DX | GNNCO_FORWARD_ONLY | GNNCO_AX_STORE | GNNCO_AX_REUSE)) return GNNCO_INVALID_ARGUMENT;
+  if ((flags & GNNCO_AX_STORE) && (flags & GNNCO_AX_REUSE)) return GNNCO_INVALID_ARGUMENT;
+  if ((flags & (GNNCO_AX_STORE | GNNCO_AX_REUSE)) && m->L < 2) return GNNCO_INVALID_ARGUMENT;
   if (opt && !(flags & GNNCO_FORWARD_ONLY)) {
     if (opt->step < 1) return GNNCO_INVALID_ARGUMENT;
     if (opt->active && m->weight_sets != h->S) return GNNCO_INVALID_ARGUMENT;
@@ -276,6 +282,7 @@ extern "C" int32_t gnnco_train_step(gnnco_handle* h, const gnnco_model_desc* m, 
   int32_t rc = check_step_args(h, m, opt, flags);
   if (rc != GNNCO_OK) return rc;
   if ((flags & GNNCO_WANT_DX) && !out->dX) return GNNCO_INVALID_ARGUMENT;
+  if ((flags & (GNNCO_AX_STORE | GNNCO_AX_REUSE)) && !out->ax_cache) return GNNCO_INVALID_ARGUMENT;
   if ((uintptr_t)ws & 255) return GNNCO_INVALID_ARGUMENT;
   TrainLayout T = carve_train(h, m, flags, ws, false);
   if (T.bytes > ws_bytes) return GNNCO_WORKSPACE_TOO_SMALL;
@@ -289,7 +296,8 @@ extern "C" int32_t gnnco_train_step_host(gnnco_handle* h, const gnnco_model_desc
   if (!h || !m || !X_host || !loss_host || !p_host || !ws) return GNNCO_INVALID_ARGUMENT;
   int32_t rc = check_step_args(h, m, opt, flags);
   if (rc != GNNCO_OK) return rc;
-  if (flags & GNNCO_WANT_DX) return GNNCO_UNSUPPORTED;       // the host variant returns loss and p only
+  // the host variant returns loss and p only and takes fresh inputs every step
+  if (flags & (GNNCO_WANT_DX | GNNCO_AX_STORE | GNNCO_AX_REUSE)) return GNNCO_UNSUPPORTED;
   if ((uintptr_t)ws & 255) return GNNCO_INVALID_ARGUMENT;
   TrainLayout T = carve_train(h, m, flags, ws, true);
   if (T.bytes > ws_bytes) return GNNCO_WORKSPACE_TOO_SMALL;

@@ -170,6 +170,41 @@ def test_step_is_deterministic_run_to_run():
         assert torch.equal(a, b)
 
 
+@pytest.mark.parametrize("cfg", [1, 3])
+def test_cached_first_aggregation_is_bit_identical(cfg):
+    """Three Adam steps with the first layer's aggregated input stored on step 1 and
+    reused afterwards equal three plain steps bit for bit; bad flag combinations are refused."""
+    import torch
+    import paper_2511_09261_b200 as gnnco
+    w = si.make_workload(cfg)
+    graph = load_graph(w.n, w.eu, w.ev, w.part, w.S)
+    perm = graph.arrays()["perm"].cpu().numpy()
+    X = to_dev(w.features_f32()[perm])
+    runs = []
+    for cached in (False, True):
+        W = [to_dev(w.weights(l)) for l in range(w.L)]
+        model = gnnco.Model(w.dims, W)
+        opt = gnnco.Adam(model, lr=1e-2)
+        cache = torch.empty_like(X) if cached else None
+        trace = []
+        for step in range(3):
+            flags = gnnco.WANT_DX
+            if cached:
+                flags |= gnnco.AX_STORE if step == 0 else gnnco.AX_REUSE
+            dX = torch.empty_like(X)
+            loss, p = graph.train_step(model, X, 2.0, 1.0, opt=opt, dX=dX, flags=flags, ax_cache=cache)
+            trace += [loss.clone(), p.clone(), dX]
+        runs.append(trace + [t.clone() for t in W])
+    for a, b in zip(*runs):
+        assert torch.equal(a, b)
+    W = [to_dev(w.weights(l)) for l in range(w.L)]
+    model = gnnco.Model(w.dims, W)
+    for flags, cache in ((gnnco.AX_STORE, None), (gnnco.AX_STORE | gnnco.AX_REUSE, torch.empty_like(X))):
+        with pytest.raises(gnnco.GnncoError) as e:
+            graph.train_step(model, X, 2.0, 1.0, flags=flags, ax_cache=cache)
+        assert e.value.status == gnnco.INVALID_ARGUMENT
+
+
 def test_host_variant_matches_device_variant():
     import torch
     import paper_2511_09261_b200 as gnnco
