@@ -29,6 +29,7 @@ GRAPHS = {
         tiny_graph(120, 0.08, 6, seed=6)),
     "hub_and_isolated": lambda: _star_plus_isolated(300) + (np.zeros(300, np.int32),),
     "big_hub": lambda: _star_plus_isolated(1100) + (np.zeros(1100, np.int32),),     # hub row of 549 entries
+    "huge_hub": lambda: _star_plus_isolated(9000) + (np.zeros(9000, np.int32),),   # hub row of 4499 entries (block-summed)
     "no_edges": lambda: (np.zeros(0, np.int32), np.zeros(0, np.int32), si.contiguous_partition(50, 4)),
     "dense_small": lambda: tiny_graph(90, 0.5, 2, seed=8, contiguous=True),
 }
@@ -86,6 +87,7 @@ STEP_CASES = [
     ("big_hub", [32, 16, 1], None, 0.0),
     ("big_hub", [128, 8, 1], None, 0.0),
     ("big_hub", [256, 12, 1], None, 0.4),
+    ("huge_hub", [16, 8, 1], None, 0.3),
     ("no_edges", [4, 4, 1], None, 0.0),
     ("dense_small", [24, 40, 1], None, 0.2),
     ("dense_small", [130, 70, 1], None, 0.0),
