@@ -21,12 +21,13 @@
 namespace {
 
 constexpr int kTileM = 128;
-constexpr int kThreads = 256;
+constexpr int kThreads = 256;                // weight-gradient kernel
+constexpr int kTfThreads = 384;              // transform kernel: 4 epilogue warps, 1 MMA warp, 7 producer warps
 constexpr int kEpiWarps = 4;
 constexpr int kMmaWarp = 4;
 constexpr int kProdWarp0 = 5;
-constexpr int kProdLanes = 96;
-constexpr int kBatch = 11;                   // 32-byte source chunks a producer lane has in flight (a whole k-block)
+constexpr int kProdLanes = 224;              // splitting float32 into limbs is the producers' work: most warps do it
+constexpr int kBatch = 5;                    // 32-byte source chunks a producer lane has in flight (a whole k-block)
 
 __device__ __forceinline__ uint32_t pack_bf16x2(float a, float b) {
   __nv_bfloat162 v = __floats2bfloat162_rn(a, b);
@@ -57,7 +58,7 @@ __device__ __forceinline__ void split3(const float4& x, const float4& y, uint4& 
 // Shared memory: A slot of k-block kb = 3 limb tiles of 128 rows x 128 bytes (K-major SW128);
 // B k-block kb = 3 limb tiles of NDIM rows x 128 bytes.
 template <int KDIM, int NDIM>
-__global__ void __launch_bounds__(kThreads, 1)
+__global__ void __launch_bounds__(kTfThreads, 1)
 transform_tc_f32(const float* __restrict__ A, const __nv_bfloat16* __restrict__ B, int64_t b_stride,
                  int64_t b_limb_stride, float* __restrict__ Y, int relu, const float* __restrict__ row_scale,
                  const float* __restrict__ relu_mask, const float* __restrict__ dot_w, int64_t dot_stride, float* __restrict__ dot_out,
@@ -274,7 +275,7 @@ int32_t launch_tf(gnnco_handle* h, const void* A, const void* B, int64_t b_strid
   int grid = h->n_tiles < sms ? h->n_tiles : sms;
   int per = (h->n_tiles + grid - 1) / grid;
   grid = (h->n_tiles + per - 1) / per;
-  transform_tc_f32<KDIM, NDIM><<<grid, kThreads, smem, st>>>(
+  transform_tc_f32<KDIM, NDIM><<<grid, kTfThreads, smem, st>>>(
       (const float*)A, (const __nv_bfloat16*)B, b_stride, b_limb_stride, (float*)Y, relu ? 1 : 0, row_scale,
       (const float*)relu_mask, (const float*)dot_w, dot_stride, dot_out, h->tile_row0, h->tile_rows, h->node_part, h->n_tiles, per, h->status);
   h->launches += 1;
