@@ -170,6 +170,23 @@ def adam(W: np.ndarray, m: np.ndarray, v: np.ndarray, g: np.ndarray, lr: float, 
     _native().oracle_adam(W.size, _ptr(W), _ptr(m), _ptr(v), _ptr(g), lr, b1, b2, eps, t)
 
 
+def gumbel_softmax(E: np.ndarray, U: Optional[np.ndarray], tau: float) -> np.ndarray:
+    """Gumbel-softmax processing of the initial embeddings (Section 3.2, first paragraph of
+    "Subgraph training"): row i of the result is softmax((e_i + g_i) / tau) over the feature
+    axis, with Gumbel noise g = -log(-log u) from uniforms u in (0, 1) that the caller passes
+    in (``U`` None: no noise).  Reading of the paper where it is silent: the soft (relaxed)
+    form, one temperature ``tau`` for all nodes, noise drawn once with the embeddings.
+    Plain float64 numpy; the row maximum is subtracted before exponentiating, which changes
+    nothing in exact arithmetic."""
+    a = np.asarray(E, dtype=np.float64)
+    if U is not None:
+        a = a + (-np.log(-np.log(np.asarray(U, dtype=np.float64))))
+    a = a / float(tau)
+    a = a - a.max(axis=1, keepdims=True)
+    e = np.exp(a)
+    return e / e.sum(axis=1, keepdims=True)
+
+
 def decode(book: Dict[str, np.ndarray], p: np.ndarray, threshold: float = 0.5) -> Dict[str, object]:
     """Threshold float32 probabilities and count selected nodes and violated edges."""
     n, S = int(book["n"]), int(book["S"])

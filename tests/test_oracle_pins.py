@@ -508,6 +508,60 @@ def test_adam_first_step_is_sign_step_and_zero_gradient_stays():
     assert W[2] == 1.0
 
 
+# ------------------------------------------------- Gumbel-softmax input processing (Section 3.2)
+def test_gumbel_softmax_without_noise_is_the_library_softmax():
+    from scipy.special import softmax
+    E = rand_features(37, 12, 5)
+    for tau in (0.3, 1.0, 4.0):
+        np.testing.assert_allclose(oracle.gumbel_softmax(E, None, tau), softmax(E / tau, axis=1), rtol=1e-13, atol=0)
+
+
+def test_gumbel_softmax_two_features_closed_form():
+    # e = (0, 0), tau = 1:  x_0 = 1 / (1 + exp(g_1 - g_0)) with exp(-g) = -ln u, i.e. x_0 = ln u_1 / ln(u_0 u_1)
+    U = np.array([[0.2, 0.7], [0.9, 0.05], [0.5, 0.5]])
+    x = oracle.gumbel_softmax(np.zeros((3, 2)), U, 1.0)
+    expect0 = np.log(U[:, 1]) / np.log(U[:, 0] * U[:, 1])
+    np.testing.assert_allclose(x[:, 0], expect0, rtol=1e-13)
+    np.testing.assert_allclose(x[:, 1], 1.0 - expect0, rtol=1e-13)
+    # temperature divides BOTH the embedding and the noise: e = (ln 3, 0), tau = 1/2, no noise -> odds 9 : 1
+    y = oracle.gumbel_softmax(np.array([[np.log(3.0), 0.0]]), None, 0.5)
+    np.testing.assert_allclose(y, [[0.9, 0.1]], rtol=1e-13)
+    z = oracle.gumbel_softmax(np.zeros((1, 2)), np.array([[0.2, 0.7]]), 0.5)
+    odds = (np.log(0.7) / np.log(0.2)) ** 2                      # exp((g_0 - g_1) / tau)
+    np.testing.assert_allclose(z[0, 0] / z[0, 1], odds, rtol=1e-12)
+
+
+def test_gumbel_softmax_invariants_and_temperature_limits():
+    n, F = 50, 9
+    E = rand_features(n, F, 8)
+    U = si.uniform01(91, 0, n * F).reshape(n, F)
+    x = oracle.gumbel_softmax(E, U, 0.7)
+    assert np.all(x > 0) and np.all(x < 1)
+    np.testing.assert_allclose(x.sum(axis=1), 1.0, rtol=1e-14)
+    # a constant added to a row changes nothing; rows do not interact
+    np.testing.assert_allclose(oracle.gumbel_softmax(E + 3.25, U, 0.7), x, rtol=1e-12)
+    np.testing.assert_allclose(oracle.gumbel_softmax(E[7:8], U[7:8], 0.7), x[7:8], rtol=1e-14)
+    # hot: close to uniform; cold: one-hot at the arg max of embedding + noise
+    hot = oracle.gumbel_softmax(E, U, 1e6)
+    assert np.max(np.abs(hot - 1.0 / F)) < 1e-4
+    cold = oracle.gumbel_softmax(E, U, 1e-3)
+    winner = np.argmax(E - np.log(-np.log(U)), axis=1)
+    assert np.array_equal(np.argmax(cold, axis=1), winner) and np.all(cold.max(axis=1) > 1 - 1e-3)
+
+
+def test_gumbel_max_trick_reproduces_the_softmax_distribution():
+    # arg max of (e + g) is distributed as softmax(e): pins the noise law -log(-log u) statistically
+    from scipy.special import softmax
+    e = np.array([0.5, -1.0, 1.5, 0.0])
+    N = 200_000
+    U = si.uniform01(123, 0, N * 4).reshape(N, 4)
+    cold = oracle.gumbel_softmax(np.broadcast_to(e, (N, 4)), U, 1e-2)
+    freq = np.bincount(np.argmax(cold, axis=1), minlength=4) / N
+    prob = softmax(e)
+    sigma = np.sqrt(prob * (1 - prob) / N)
+    assert np.all(np.abs(freq - prob) < 5 * sigma)
+
+
 # --------------------------------------------------------------------- decode (a8, a9)
 @pytest.mark.parametrize("seed", [1, 2, 3])
 def test_decode_brute_force(seed):
