@@ -244,6 +244,29 @@ int32_t gnnco_conflict_actions(gnnco_handle* h, const uint8_t* viol, const float
 int32_t gnnco_apply_actions(gnnco_handle* h, const int32_t* conflict_idx, const uint8_t* action,
                             const int32_t* count, float* pen, uint8_t* active, int32_t* chosen, void* stream);
 
+/* Input embeddings (Section 3.2, "Subgraph training": "node embeddings are initialized as random
+ * vectors ... processed using the Gumbel-softmax trick").
+ *
+ * gnnco_gumbel_softmax: X[i,:] = softmax( (E[i,:] + g[i,:]) / tau ) over the F features of node i,
+ * with Gumbel noise g = -log(-log U) from uniforms U in (0, 1), exclusive, that the caller draws
+ * (U == NULL: no noise).  The paper fixes neither the temperature, nor hard versus soft, nor
+ * when the noise is redrawn; this is the soft form with one temperature, and the noise is an
+ * input, so the call is deterministic.  E and X are [n x F] in feat_dtype (any node order, rows
+ * are independent; E == X is allowed), U is [n x F] float32.  tau > 0.  Asynchronous on `stream`.
+ *
+ * gnnco_embedding_update: the variant in which the embeddings are trained (the paper only says
+ * that W is updated; gnnco_train_step leaves X alone).  One Adam step, same rule as for the
+ * weights, on the float32 master copy X_master [n x F] with the gradient dX [n x F] (feat_dtype)
+ * that gnnco_train_step wrote under GNNCO_WANT_DX; m and v are its moments (float32, zero
+ * before the first step), `step` is the 1-based number of this update.  X [n x F] (feat_dtype)
+ * receives the updated embeddings in the type the next gnnco_train_step reads; a cached
+ * first-layer aggregation (GNNCO_AX_REUSE) is stale after this call.  Asynchronous on `stream`. */
+int32_t gnnco_gumbel_softmax(gnnco_handle* h, int32_t feat_dtype, int32_t F, const void* E, const float* U, float tau,
+                             void* X, void* stream);
+int32_t gnnco_embedding_update(gnnco_handle* h, int32_t feat_dtype, int32_t F, const void* dX, float* X_master,
+                               float* m, float* v, void* X, float lr, float beta1, float beta2, float eps,
+                               int64_t step, void* stream);
+
 /* Objective only, for callers that cannot allocate device memory.  (The paper has no
  * counterpart to this call; it exists for the way the library is embedded.)
  *

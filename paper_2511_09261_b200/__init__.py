@@ -26,7 +26,7 @@ EXPORTS = [
     "gnnco_gather_rows", "gnnco_train_workspace_bytes", "gnnco_train_step", "gnnco_train_host_workspace_bytes",
     "gnnco_train_step_host", "gnnco_decode_boundary", "gnnco_async_status", "gnnco_launch_count", "gnnco_destroy",
     "gnnco_profile_begin", "gnnco_profile_end", "gnnco_objective_static", "gnnco_conflict_workspace_bytes",
-    "gnnco_conflict_actions", "gnnco_apply_actions",
+    "gnnco_conflict_actions", "gnnco_apply_actions", "gnnco_gumbel_softmax", "gnnco_embedding_update",
 ]
 
 _vp, _i32, _i64, _u32, _f32, _sz = (ctypes.c_void_p, ctypes.c_int32, ctypes.c_int64, ctypes.c_uint32, ctypes.c_float,
@@ -112,6 +112,8 @@ def load_library(build_if_missing: bool = True):
     lib.gnnco_conflict_workspace_bytes.argtypes = [_vp, ctypes.POINTER(_sz)]
     lib.gnnco_conflict_actions.argtypes = [_vp, _vp, _vp, _vp, _vp, _vp, _vp, _sz, _vp]
     lib.gnnco_apply_actions.argtypes = [_vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp]
+    lib.gnnco_gumbel_softmax.argtypes = [_vp, _i32, _i32, _vp, _vp, _f32, _vp, _vp]
+    lib.gnnco_embedding_update.argtypes = [_vp, _i32, _i32, _vp, _vp, _vp, _vp, _vp, _f32, _f32, _f32, _f32, _i64, _vp]
     for name in EXPORTS:
         if name not in ("gnnco_status_string", "gnnco_launch_count"):
             getattr(lib, name).restype = _i32
@@ -395,6 +397,46 @@ class PartitionedGraph:
                                              count.data_ptr(), pen.data_ptr(), active.data_ptr(), chosen.data_ptr(),
                                              _stream_ptr(stream)), "gnnco_apply_actions")
         return dict(pen=pen, active=active, chosen=chosen)
+
+    def gumbel_softmax(self, E, U=None, tau: float = 1.0, out=None, stream=None):
+        """``gnnco_gumbel_softmax``: rows of ``E`` ([n, F], float32 or bfloat16) through the
+        Gumbel-softmax with uniforms ``U`` ([n, F] float32 in (0, 1), or None for no noise)."""
+        import torch
+        if E.dtype not in (torch.float32, torch.bfloat16) or E.dim() != 2 or E.shape[0] != self.n:
+            raise ValueError("E must be [n, F] float32 or bfloat16")
+        _require(E, E.dtype, "E")
+        if U is not None:
+            _require(U, torch.float32, "U")
+            if tuple(U.shape) != tuple(E.shape):
+                raise ValueError("U must have the shape of E")
+        if out is None:
+            out = torch.empty_like(E)
+        _require(out, E.dtype, "out")
+        dt = BF16 if E.dtype == torch.bfloat16 else F32
+        _check(self._lib.gnnco_gumbel_softmax(self._handle, dt, int(E.shape[1]), E.data_ptr(), _dptr(U), float(tau),
+                                              out.data_ptr(), _stream_ptr(stream)), "gnnco_gumbel_softmax")
+        return out
+
+    def embedding_update(self, dX, X_master, m, v, X, lr: float, step: int, beta1: float = 0.9,
+                         beta2: float = 0.999, eps: float = 1e-8, stream=None):
+        """``gnnco_embedding_update``: one Adam step on the float32 master embeddings with the
+        gradient ``dX`` of a WANT_DX training step; ``X`` receives them in the features' type."""
+        import torch
+        for t, what in ((X_master, "X_master"), (m, "m"), (v, "v")):
+            _require(t, torch.float32, what)
+        _require(dX, X.dtype, "dX")
+        _require(X, X.dtype, "X")
+        if X.dtype not in (torch.float32, torch.bfloat16) or X.dim() != 2 or X.shape[0] != self.n:
+            raise ValueError("X must be [n, F] float32 or bfloat16")
+        for t in (dX, X_master, m, v):
+            if tuple(t.shape) != tuple(X.shape):
+                raise ValueError("dX, X_master, m, v and X must have the same shape")
+        dt = BF16 if X.dtype == torch.bfloat16 else F32
+        _check(self._lib.gnnco_embedding_update(self._handle, dt, int(X.shape[1]), dX.data_ptr(), X_master.data_ptr(),
+                                                m.data_ptr(), v.data_ptr(), X.data_ptr(), float(lr), float(beta1),
+                                                float(beta2), float(eps), int(step), _stream_ptr(stream)),
+               "gnnco_embedding_update")
+        return X
 
     def objective_static(self, p, alpha: float, beta: float, lam: float = 0.0, pen=None, loss=None, stream=None):
         """``gnnco_objective_static``: per-subgraph objective of given probabilities, with no

@@ -28,7 +28,7 @@ constexpr int kItemRows = 1024;      // rows of one objective work item (never s
 // Kernel families, for launch accounting and per-kernel timing.
 enum KernelKind {
   K_AGG_FWD, K_AGG_BWD, K_TRANSFORM_FWD, K_TRANSFORM_BWD, K_WEIGHT_GRAD, K_GEMV, K_WEIGHT_GRAD_VEC, K_RANK1,
-  K_SUM_SETS, K_CAST, K_ADAM, K_OUT_FWD, K_OBJECTIVE, K_OUT_BWD, K_DECODE, K_STAGE3, K_AGG_RANK1, K_KIND_COUNT
+  K_SUM_SETS, K_CAST, K_ADAM, K_OUT_FWD, K_OBJECTIVE, K_OUT_BWD, K_DECODE, K_STAGE3, K_AGG_RANK1, K_EMBED, K_KIND_COUNT
 };
 
 // Optional per-kernel timing: while `on`, every launcher brackets its launches with a pair
