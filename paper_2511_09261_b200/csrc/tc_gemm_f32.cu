@@ -112,6 +112,10 @@ transform_tc_f32(const float* __restrict__ A, const __nv_bfloat16* __restrict__ 
       const int part = node_part[row0];
       const bool new_b = part != cur_part;
       cur_part = part;
+      // the operand loads below go through registers, a k-block at a time, so their latency is
+      // on this pipeline's critical path: have the next tile's rows (contiguous) waiting in L2
+      if (p == 0 && t + 1 < t_end)
+        tc::prefetch_l2(A + (int64_t)tile_row0[t + 1] * KDIM, (uint32_t)tile_rows[t + 1] * KDIM * 4);
       for (int kb = 0; kb < KB; ++kb) {
         if (j > 0 && !tc::mbar_wait_bounded(empty + kb, (j - 1) & 1)) *abort_flag = 1;
         if (new_b) {
@@ -338,6 +342,14 @@ weight_grad_tc_f32(const float* __restrict__ A, const float* __restrict__ G, flo
     }
     const uint32_t sb = sbase + slot * STAGE;
     const int64_t r0 = ra + (int64_t)it * kWgRows;
+    // the loads below go through registers and wait for their data: have the rows of the
+    // iteration after next (contiguous in both operands) on their way into L2
+    if (threadIdx.x < 2 && it + 2 < iters) {
+      const int64_t rp = r0 + 2 * kWgRows;
+      const uint32_t nrows = (uint32_t)min((int64_t)kWgRows, rb - rp);
+      if (threadIdx.x == 0) tc::prefetch_l2(A + rp * KF, nrows * KF * 4);
+      else tc::prefetch_l2(G + rp * NF, nrows * NF * 4);
+    }
     // stage 64 rows of A and G: load float32, split, store the three limbs
 #pragma unroll
     for (int half = 0; half < 2; ++half) {
