@@ -447,8 +447,8 @@ TRAFFIC_BYTES = {
     (5, "aggregate_fwd"): 10.03e9,
     (5, "aggregate_bwd"): 10.00e9,
     (5, "aggregate_rank1"): 10.17e9,
-    (5, "transform_fwd"): 11.62e9,
-    (5, "transform_bwd"): 15.05e9,
+    (5, "transform_fwd"): 10.49e9,
+    (5, "transform_bwd"): 13.10e9,
 }
 
 
