@@ -53,12 +53,14 @@ __device__ __forceinline__ uint32_t keep_where_positive(uint32_t v, uint32_t m) 
 //   MMA warp  : for each k-block wait full[kb], issue 4 MMAs (K = 16 each) into accumulator
 //               buffer (tile & 1), commit -> empty[kb]; after the last k-block commit -> acc_full
 //   epilogue  : two warps per TMEM lane quarter, each owning half of the columns: request the
-//               ReLU-mask lines of the tile (if any), wait acc_full, read the accumulator
-//               (TMEM -> registers), scale / rectify / round to bf16, store; optionally the
+//               ReLU-mask lines of the tile (MASKED instantiation), wait acc_full, read the
+//               accumulator (TMEM -> registers; without a mask the next chunk's read is issued
+//               before the current chunk is stored, so its latency hides behind the stores),
+//               scale / rectify / round to bf16, store; optionally the
 //               next layer's row dot product (the two column halves meet in shared memory);
 //               arrive acc_empty
 // so the copies of tile t+1, the MMAs of tile t+1 and the drain of tile t overlap.
-template <int KDIM, int NDIM>
+template <int KDIM, int NDIM, bool MASKED>
 __global__ void __launch_bounds__(kTfThreads, 1)
 transform_tc(const __nv_bfloat16* __restrict__ A, const __nv_bfloat16* __restrict__ B, int64_t b_stride,
              __nv_bfloat16* __restrict__ Y, int relu, const float* __restrict__ row_scale,
@@ -164,8 +166,8 @@ transform_tc(const __nv_bfloat16* __restrict__ A, const __nv_bfloat16* __restric
       const int rows_here = rows - quarter * 32;       // valid rows of this warp's 32
       // the mask is read where the result will be stored (whole lines); every line of the tile
       // that this warp needs is requested before the accumulator is waited for
-      uint4 mk[PER][8];
-      if (relu_mask) {
+      uint4 mk[MASKED ? PER : 1][8];
+      if (MASKED) {
 #pragma unroll
         for (int c = 0; c < PER; ++c)
 #pragma unroll
@@ -183,23 +185,43 @@ transform_tc(const __nv_bfloat16* __restrict__ A, const __nv_bfloat16* __restric
       float dot = 0.0f;
       if (!tc::mbar_wait_bounded(acc_full + buf, (j >> 1) & 1)) { *abort_flag = 1; break; }
       tc::tc_fence_after_sync();
+      // the 64 columns of a chunk are read with two 32-column loads and one wait
+      uint32_t ra[32], rb[32];
+      auto read_chunk = [&](int c) {
+        const uint32_t at = tmem + ((uint32_t)(quarter * 32) << 16) + buf * NDIM + (ch_begin + c) * 64;
+        tc::tmem_ld_32x32(at, ra);
+        tc::tmem_ld_32x32(at + 32, rb);
+      };
+      if (!MASKED && ch_begin < ch_end) read_chunk(0);
 #pragma unroll
       for (int c = 0; c < PER; ++c) {
         if (ch_begin + c >= ch_end) break;
         const int c0 = (ch_begin + c) * 64;
         uint32_t o[32];                                // 64 bf16 of this thread's row, packed
-#pragma unroll
-        for (int hh = 0; hh < 2; ++hh) {
-          uint32_t r[32];
-          tc::tmem_ld_32x32(tmem + ((uint32_t)(quarter * 32) << 16) + buf * NDIM + c0 + hh * 32, r);
-          tc::tmem_ld_wait();
+        auto convert = [&](const uint32_t (&r)[32], int at) {
 #pragma unroll
           for (int q = 0; q < 16; ++q) {
             float a = __uint_as_float(r[2 * q]) * s, b = __uint_as_float(r[2 * q + 1]) * s;
             if (relu) { a = a > 0.0f ? a : 0.0f; b = b > 0.0f ? b : 0.0f; }
             __nv_bfloat162 v = __floats2bfloat162_rn(a, b);
-            o[hh * 16 + q] = *reinterpret_cast<uint32_t*>(&v);
+            o[at + q] = *reinterpret_cast<uint32_t*>(&v);
           }
+        };
+        if (MASKED) {
+          // the mask lines hold 64 registers: one 32-column read at a time
+#pragma unroll
+          for (int hh = 0; hh < 2; ++hh) {
+            tc::tmem_ld_32x32(tmem + ((uint32_t)(quarter * 32) << 16) + buf * NDIM + c0 + hh * 32, ra);
+            tc::tmem_ld_wait();
+            convert(ra, hh * 16);
+          }
+        } else {
+          tc::tmem_ld_wait();
+          convert(ra, 0);
+          convert(rb, 16);
+          // the accumulator registers are free again: the next chunk's read goes out now and
+          // lands while this chunk is being stored
+          if (c + 1 < PER && ch_begin + c + 1 < ch_end) read_chunk(c + 1);
         }
         if (wv) {   // dot product of the STORED (rounded) row with the next layer's weight vector
 #pragma unroll
@@ -226,7 +248,7 @@ transform_tc(const __nv_bfloat16* __restrict__ A, const __nv_bfloat16* __restric
         for (int it = 0; it < 8; ++it) {
           const int rr = it * 4 + (lane >> 3), pc = lane & 7;
           uint4 v = tc::ld_shared16(stage + rr * 128 + ((pc ^ (rr & 7)) << 4));
-          if (relu_mask) {
+          if (MASKED) {
             v.x = keep_where_positive(v.x, mk[c][it].x); v.y = keep_where_positive(v.y, mk[c][it].y);
             v.z = keep_where_positive(v.z, mk[c][it].z); v.w = keep_where_positive(v.w, mk[c][it].w);
           }
@@ -268,13 +290,21 @@ int32_t launch_tc(gnnco_handle* h, const void* A, const void* B, int64_t b_strid
   // operands, barriers and dot-product exchange, one 4 KB staging tile per epilogue warp, alignment slack
   constexpr size_t smem = (size_t)KB * (kTileM + NDIM) * 128 + kTfMiscBytes + kEpiWarps * 4096 + 1024;
   static_assert(smem <= 232448, "tile does not fit in shared memory");
-  GNNCO_CUDA_TRY(cudaFuncSetAttribute(transform_tc<KDIM, NDIM>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+  GNNCO_CUDA_TRY(cudaFuncSetAttribute(transform_tc<KDIM, NDIM, false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                      (int)smem));
+  GNNCO_CUDA_TRY(cudaFuncSetAttribute(transform_tc<KDIM, NDIM, true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                       (int)smem));
   int sms = h->sm_count > 0 ? h->sm_count : 148;
   int grid = h->n_tiles < sms ? h->n_tiles : sms;
   int per = (h->n_tiles + grid - 1) / grid;
   grid = (h->n_tiles + per - 1) / per;
-  transform_tc<KDIM, NDIM><<<grid, kTfThreads, smem, st>>>(
+  if (relu_mask)
+    transform_tc<KDIM, NDIM, true><<<grid, kTfThreads, smem, st>>>(
+      (const __nv_bfloat16*)A, (const __nv_bfloat16*)B, b_stride, (__nv_bfloat16*)Y, relu ? 1 : 0, row_scale,
+      (const __nv_bfloat16*)relu_mask, (const __nv_bfloat16*)dot_w, dot_stride, dot_out, h->tile_row0, h->tile_rows, h->node_part, h->n_tiles, per,
+      h->status);
+  else
+    transform_tc<KDIM, NDIM, false><<<grid, kTfThreads, smem, st>>>(
       (const __nv_bfloat16*)A, (const __nv_bfloat16*)B, b_stride, (__nv_bfloat16*)Y, relu ? 1 : 0, row_scale,
       (const __nv_bfloat16*)relu_mask, (const __nv_bfloat16*)dot_w, dot_stride, dot_out, h->tile_row0, h->tile_rows, h->node_part, h->n_tiles, per,
       h->status);
