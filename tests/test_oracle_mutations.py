@@ -89,3 +89,39 @@ def test_a_pin_fails_when_the_oracle_is_mutated(name, tmp_path, monkeypatch):
         except (AssertionError, oracle.OracleError, ValueError, IndexError, KeyError):
             caught += 1
     assert caught >= 1, "no pin noticed: " + name
+
+
+# The Gumbel-softmax oracle is numpy, not C: the same game on its Python source.
+PY_MUTATIONS = {
+    "Gumbel noise subtracted": ("a = a + (-np.log(-np.log(", "a = a - (-np.log(-np.log("),
+    "noise with a single logarithm": ("(-np.log(-np.log(np.asarray(U, dtype=np.float64))))", "(-np.log(np.asarray(U, dtype=np.float64)))"),
+    "temperature multiplies": ("a = a / float(tau)", "a = a * float(tau)"),
+    "normalised over nodes instead of features": ("e / e.sum(axis=1, keepdims=True)", "e / e.sum(axis=0, keepdims=True)"),
+    "softmax without the exponential": ("e = np.exp(a)", "e = a - a.min() + 1.0"),
+}
+
+PY_BATTERY = [
+    pins.test_gumbel_softmax_without_noise_is_the_library_softmax,
+    pins.test_gumbel_softmax_two_features_closed_form,
+    pins.test_gumbel_softmax_invariants_and_temperature_limits,
+    pins.test_gumbel_max_trick_reproduces_the_softmax_distribution,
+]
+
+
+@pytest.mark.parametrize("name", sorted(PY_MUTATIONS))
+def test_a_pin_fails_when_the_gumbel_softmax_oracle_is_mutated(name, monkeypatch):
+    import inspect
+    import numpy as np
+    old, new = PY_MUTATIONS[name]
+    text = inspect.getsource(oracle.gumbel_softmax)
+    assert text.count(old) == 1, "mutation target not found exactly once: %r" % old
+    scope = {"np": np, "Optional": __import__("typing").Optional}
+    exec(text.replace(old, new), scope)
+    monkeypatch.setattr(oracle, "gumbel_softmax", scope["gumbel_softmax"])
+    caught = 0
+    for check in PY_BATTERY:
+        try:
+            check()
+        except (AssertionError, ValueError, FloatingPointError):
+            caught += 1
+    assert caught >= 1, "no pin noticed: " + name
