@@ -53,6 +53,8 @@ def _native():
         lib.oracle_base_action.restype = None
         lib.oracle_apply_actions.argtypes = [i64, i32, i64, vp, vp, vp, vp, vp, vp, vp]
         lib.oracle_apply_actions.restype = i64
+        lib.oracle_repair.argtypes = [i64, vp, vp]
+        lib.oracle_repair.restype = i64
         _lib = lib
     return _lib
 
@@ -168,6 +170,15 @@ def adam(W: np.ndarray, m: np.ndarray, v: np.ndarray, g: np.ndarray, lr: float, 
         assert a.dtype == np.float64 and a.flags.c_contiguous
     g = _as_f64(g)
     _native().oracle_adam(W.size, _ptr(W), _ptr(m), _ptr(v), _ptr(g), lr, b1, b2, eps, t)
+
+
+def repair(x: np.ndarray, pen: np.ndarray) -> Dict[str, object]:
+    """Carry the chosen actions out on the mask: a copy of ``x`` with every chosen node
+    (``pen`` != 0) cleared, and the number of selected nodes that were removed."""
+    out = np.ascontiguousarray(x, dtype=np.uint8).copy()
+    pen = np.ascontiguousarray(pen, dtype=np.float32)
+    removed = _native().oracle_repair(out.size, _ptr(pen), _ptr(out))
+    return dict(x=out, removed=int(removed))
 
 
 def gumbel_softmax(E: np.ndarray, U: Optional[np.ndarray], tau: float) -> np.ndarray:

@@ -484,3 +484,19 @@ int64_t oracle_apply_actions(int64_t n, int32_t S, int64_t count, const int32_t*
   }
   return chosen;
 }
+
+/*
+ * Non-learned repair (Section 3.3: an action on conflict (i, j) "directly eliminates the conflict
+ * by removing node i [or j] from the candidate set"; Algorithm 1, Stage 3 starts from a base
+ * action).  Carrying the chosen actions out on the bit mask itself, without fine-tuning:
+ * x[i] <- 0 for every chosen node i (pen[i] != 0).  Returns how many selected nodes were removed.
+ */
+int64_t oracle_repair(int64_t n, const float* pen, uint8_t* x) {
+  int64_t removed = 0;
+  for (int64_t i = 0; i < n; ++i)
+    if (pen[i] != 0.0f && x[i]) {
+      x[i] = 0;
+      ++removed;
+    }
+  return removed;
+}

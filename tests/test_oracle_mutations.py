@@ -42,6 +42,8 @@ MUTATIONS = {
     "base action picks u on equal probabilities": ("action[c] = p[u] < p[v] ? 0 : 1;", "action[c] = p[u] <= p[v] ? 0 : 1;"),
     "actions mark the wrong endpoint's subgraph": ("active[node_part[node]] = 1;", "active[node_part[bnd_u[conflict_idx[c]]]] = 1;"),
     "conflict list keeps non-violated edges": ("if (viol[e]) conflict_idx[c++] = (int32_t)e;", "conflict_idx[c++] = (int32_t)e;"),
+    "repair clears the nodes that were NOT chosen": ("if (pen[i] != 0.0f && x[i]) {", "if (pen[i] == 0.0f && x[i]) {"),
+    "repair counts chosen nodes that were not selected": ("if (pen[i] != 0.0f && x[i]) {", "if (pen[i] != 0.0f) {"),
     "inv_deg without the +1": ("inv_deg[i] = 1.0f / (float)(hi - lo + 1);", "inv_deg[i] = 1.0f / (float)(hi - lo > 0 ? hi - lo : 1);"),
 }
 
@@ -63,6 +65,7 @@ BATTERY = [
     lambda: pins.test_decode_brute_force(2),
     lambda: pins.test_conflict_list_base_action_and_penalty_brute_force(1),
     lambda: pins.test_conflict_list_base_action_and_penalty_brute_force(2),
+    lambda: pins.test_repair_removes_exactly_the_chosen_nodes_brute_force(1),
 ]
 
 
@@ -78,7 +81,7 @@ def test_a_pin_fails_when_the_oracle_is_mutated(name, tmp_path, monkeypatch):
     real = oracle._native()
     mutant = ctypes.CDLL(lib_path)
     for fn in ("oracle_bookkeeping", "oracle_subgraph_step", "oracle_train_step", "oracle_adam", "oracle_decode",
-               "oracle_conflict_list", "oracle_base_action", "oracle_apply_actions"):
+               "oracle_conflict_list", "oracle_base_action", "oracle_apply_actions", "oracle_repair"):
         getattr(mutant, fn).argtypes = getattr(real, fn).argtypes
         getattr(mutant, fn).restype = getattr(real, fn).restype
     monkeypatch.setattr(oracle, "_lib", mutant)

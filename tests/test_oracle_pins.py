@@ -653,6 +653,39 @@ def test_conflict_list_base_action_and_penalty_brute_force(seed):
     assert set(np.nonzero(r2["pen"])[0].tolist()) == other
 
 
+@pytest.mark.parametrize("seed", [1, 2, 3])
+def test_repair_removes_exactly_the_chosen_nodes_brute_force(seed):
+    n, S = 70, 5
+    eu, ev, part = tiny_graph(n, 0.15, S, seed=400 + seed)
+    b = oracle.bookkeeping(n, eu, ev, part, S)
+    p_new = si.uniform01(500 + seed, 0, n).astype(np.float32)
+    d = oracle.decode(b, p_new)
+    conf = oracle.conflict_list(b, d["viol"])
+    assert conf.size > 0
+    for act in (oracle.base_action(b, conf, p_new), (si.u64(600 + seed, 0, conf.size) & np.uint64(1)).astype(np.uint8)):
+        pen = oracle.apply_actions(b, conf, act)["pen"]
+        r = oracle.repair(d["x"], pen)
+        # brute force on the ORIGINAL graph: drop the chosen endpoint of every violated cross edge
+        x0 = p_new[b["inv_perm"]] >= np.float32(0.5)                 # original order
+        drop = set()
+        for e, a in zip(conf.tolist(), act.tolist()):
+            drop.add(int(b["perm"][(int(b["bnd_u"][e]), int(b["bnd_v"][e]))[a]]))
+        x1 = x0.copy()
+        x1[sorted(drop)] = False
+        assert np.array_equal(r["x"], x1[b["perm"]].astype(np.uint8)) and r["removed"] == len(drop)
+        # no cross edge of the original graph has both ends selected any more; intra conflicts are untouched
+        cross_left = sum(1 for a, c in zip(eu.tolist(), ev.tolist()) if part[a] != part[c] and x1[a] and x1[c])
+        assert cross_left == 0
+        d2 = oracle.decode(b, r["x"].astype(np.float32))
+        assert d2["boundary_viol"] == 0 and d2["set_size"] == d["set_size"] - len(drop)
+        assert d2["intra_viol"] <= d["intra_viol"]
+    # nodes that are not selected are not counted, and a zero vector changes nothing
+    pen = np.zeros(n, np.float32)
+    pen[np.nonzero(d["x"] == 0)[0][:3]] = 1.0
+    r = oracle.repair(d["x"], pen)
+    assert r["removed"] == 0 and np.array_equal(r["x"], d["x"])
+
+
 def test_stage3_glue_on_empty_conflict_set():
     n, S = 20, 4
     eu, ev, part = tiny_graph(n, 0.2, S, seed=7)
