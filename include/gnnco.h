@@ -238,6 +238,14 @@ int32_t gnnco_decode_boundary(const gnnco_handle* h, const float* p, float thres
  *   chosen device int32 or NULL: number of distinct chosen nodes
  * count is the DEVICE value written by gnnco_conflict_actions; action may come from there or
  * from the caller's own policy (any 0/1 vector of that length).  Asynchronous on `stream`. */
+/*
+ * gnnco_repair_boundary carries the chosen actions out on the mask itself, without any
+ * fine-tuning -- the non-learned baseline of Stage 3 (Section 3.3: an action "directly eliminates
+ * the conflict by removing node i from the candidate set"):  x[i] <- 0 for every chosen node
+ * (pen[i] != 0, the vector written by gnnco_apply_actions).  Afterwards no boundary edge has both
+ * ends selected; intra-subgraph conflicts are not touched.  removed (device int32, or NULL)
+ * receives the number of selected nodes that were cleared.  Asynchronous on `stream`. */
+int32_t gnnco_repair_boundary(gnnco_handle* h, const float* pen, uint8_t* x, int32_t* removed, void* stream);
 int32_t gnnco_conflict_workspace_bytes(const gnnco_handle* h, size_t* bytes);
 int32_t gnnco_conflict_actions(gnnco_handle* h, const uint8_t* viol, const float* p, int32_t* conflict_idx,
                                uint8_t* action, int32_t* count, void* ws, size_t ws_bytes, void* stream);

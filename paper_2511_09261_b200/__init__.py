@@ -27,6 +27,7 @@ EXPORTS = [
     "gnnco_train_step_host", "gnnco_decode_boundary", "gnnco_async_status", "gnnco_launch_count", "gnnco_destroy",
     "gnnco_profile_begin", "gnnco_profile_end", "gnnco_objective_static", "gnnco_conflict_workspace_bytes",
     "gnnco_conflict_actions", "gnnco_apply_actions", "gnnco_gumbel_softmax", "gnnco_embedding_update",
+    "gnnco_repair_boundary",
 ]
 
 _vp, _i32, _i64, _u32, _f32, _sz = (ctypes.c_void_p, ctypes.c_int32, ctypes.c_int64, ctypes.c_uint32, ctypes.c_float,
@@ -112,6 +113,7 @@ def load_library(build_if_missing: bool = True):
     lib.gnnco_conflict_workspace_bytes.argtypes = [_vp, ctypes.POINTER(_sz)]
     lib.gnnco_conflict_actions.argtypes = [_vp, _vp, _vp, _vp, _vp, _vp, _vp, _sz, _vp]
     lib.gnnco_apply_actions.argtypes = [_vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp]
+    lib.gnnco_repair_boundary.argtypes = [_vp, _vp, _vp, _vp, _vp]
     lib.gnnco_gumbel_softmax.argtypes = [_vp, _i32, _i32, _vp, _vp, _f32, _vp, _vp]
     lib.gnnco_embedding_update.argtypes = [_vp, _i32, _i32, _vp, _vp, _vp, _vp, _vp, _f32, _f32, _f32, _f32, _i64, _vp]
     for name in EXPORTS:
@@ -397,6 +399,17 @@ class PartitionedGraph:
                                              count.data_ptr(), pen.data_ptr(), active.data_ptr(), chosen.data_ptr(),
                                              _stream_ptr(stream)), "gnnco_apply_actions")
         return dict(pen=pen, active=active, chosen=chosen)
+
+    def repair_boundary(self, pen, x, stream=None):
+        """``gnnco_repair_boundary``: clears, in place, every chosen node (``pen`` != 0) from the
+        mask ``x``; returns a device int32 with the number of selected nodes removed."""
+        import torch
+        _require(pen, torch.float32, "pen")
+        _require(x, torch.uint8, "x")
+        removed = torch.empty(1, dtype=torch.int32, device=self.device)
+        _check(self._lib.gnnco_repair_boundary(self._handle, pen.data_ptr(), x.data_ptr(), removed.data_ptr(),
+                                               _stream_ptr(stream)), "gnnco_repair_boundary")
+        return removed
 
     def gumbel_softmax(self, E, U=None, tau: float = 1.0, out=None, stream=None):
         """``gnnco_gumbel_softmax``: rows of ``E`` ([n, F], float32 or bfloat16) through the

@@ -127,6 +127,22 @@ __global__ void __launch_bounds__(256) apply_actions_kernel(const int32_t* __res
   }
 }
 
+// x[i] <- 0 for every chosen node (pen[i] != 0); counts the selected nodes that were removed
+__global__ void __launch_bounds__(256) repair_kernel(const float* __restrict__ pen, uint8_t* __restrict__ x, int64_t n,
+                                                     int32_t* __restrict__ removed) {
+  const int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+  int32_t hit = 0;
+  if (i < n && pen[i] != 0.0f && x[i]) {
+    x[i] = 0;
+    hit = 1;
+  }
+  if (removed) {
+#pragma unroll
+    for (int d = 16; d > 0; d >>= 1) hit += __shfl_xor_sync(0xffffffffu, hit, d);
+    if ((threadIdx.x & 31) == 0 && hit) atomicAdd(removed, hit);
+  }
+}
+
 inline int32_t tiles_for(int64_t E_b) { return (int32_t)((E_b + kTileEdges - 1) / kTileEdges); }
 
 }  // namespace
@@ -176,6 +192,17 @@ extern "C" int32_t gnnco_apply_actions(gnnco_handle* h, const int32_t* conflict_
   const unsigned grid = (unsigned)(want < cap ? want : cap);
   apply_actions_kernel<<<grid, 256, 0, st>>>(conflict_idx, action, count, h->bnd_u, h->bnd_v, h->node_part, h->E_b,
                                              pen, active, chosen);
+  h->launches += 1;
+  GNNCO_LAUNCH_CHECK();
+  return GNNCO_OK;
+}
+
+extern "C" int32_t gnnco_repair_boundary(gnnco_handle* h, const float* pen, uint8_t* x, int32_t* removed, void* stream) {
+  if (!h || !pen || !x) return GNNCO_INVALID_ARGUMENT;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  ProfScope prof_(h, K_STAGE3, st);
+  if (removed) GNNCO_CUDA_TRY(cudaMemsetAsync(removed, 0, sizeof(int32_t), st));
+  repair_kernel<<<(unsigned)((h->n + 255) / 256), 256, 0, st>>>(pen, x, h->n, removed);
   h->launches += 1;
   GNNCO_LAUNCH_CHECK();
   return GNNCO_OK;

@@ -277,6 +277,14 @@ def check_stage3(graph, book, p, policy_seed=None):
         assert np.array_equal(ap["pen"].cpu().numpy(), ref["pen"])
         assert np.array_equal(ap["active"].cpu().numpy(), ref["active"])
         assert int(ap["chosen"].item()) == ref["chosen"]
+        # the non-learned repair: clear the chosen nodes from the mask, then no boundary conflict is left
+        xr = d["x"].clone()
+        removed = graph.repair_boundary(ap["pen"], xr)
+        fix = oracle.repair(ref_dec["x"], ref["pen"])
+        assert np.array_equal(xr.cpu().numpy(), fix["x"]) and int(removed.item()) == fix["removed"] == ref["chosen"]
+        again = graph.decode_boundary(xr.float())
+        counts = again["counts"].cpu().tolist()
+        assert counts[2] == 0 and counts[0] == ref_dec["set_size"] - fix["removed"]
         outs.append(ap)
     return conf, act, outs[0]
 
