@@ -53,6 +53,8 @@ def _native():
         lib.oracle_base_action.restype = None
         lib.oracle_apply_actions.argtypes = [i64, i32, i64, vp, vp, vp, vp, vp, vp, vp]
         lib.oracle_apply_actions.restype = i64
+        lib.oracle_partition_quality.argtypes = [i64, vp, vp, vp, i32, vp, vp]
+        lib.oracle_partition_quality.restype = dbl
         lib.oracle_repair.argtypes = [i64, vp, vp]
         lib.oracle_repair.restype = i64
         _lib = lib
@@ -170,6 +172,25 @@ def adam(W: np.ndarray, m: np.ndarray, v: np.ndarray, g: np.ndarray, lr: float, 
         assert a.dtype == np.float64 and a.flags.c_contiguous
     g = _as_f64(g)
     _native().oracle_adam(W.size, _ptr(W), _ptr(m), _ptr(v), _ptr(g), lr, b1, b2, eps, t)
+
+
+def partition_quality(eu: np.ndarray, ev: np.ndarray, part: np.ndarray, S: int) -> Dict[str, object]:
+    """Per-community internal edge counts and degree sums (the Sigma of Eq. 1) and the
+    modularity Q of the partition, from the original edge list."""
+    eu = np.ascontiguousarray(eu, dtype=np.int32)
+    ev = np.ascontiguousarray(ev, dtype=np.int32)
+    part = np.ascontiguousarray(part, dtype=np.int32)
+    in_edges, tot = np.empty(S, np.int64), np.empty(S, np.int64)
+    q = _native().oracle_partition_quality(eu.size, _ptr(eu), _ptr(ev), _ptr(part), S, _ptr(in_edges), _ptr(tot))
+    return dict(in_edges=in_edges, tot=tot, Q=float(q))
+
+
+def delta_q(k_i_in: float, sigma_tot: float, k_i: float, m: float) -> float:
+    """Gain in modularity when an isolated node i joins a community (Section 3.1, the
+    simplified form, Eq. 2):  k_i_in / m - sigma_tot * k_i / (2 m^2).  Eq. 1 as printed differs
+    from it by a factor of two in its first term unless k_i_in and Sigma_in count every edge
+    from both ends; Eq. 2 is the one that equals the exact difference of Q."""
+    return k_i_in / m - sigma_tot * k_i / (2.0 * m * m)
 
 
 def repair(x: np.ndarray, pen: np.ndarray) -> Dict[str, object]:

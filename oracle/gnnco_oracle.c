@@ -500,3 +500,29 @@ int64_t oracle_repair(int64_t n, const float* pen, uint8_t* x) {
     }
   return removed;
 }
+
+/*
+ * Quality of a partition in the terms of Section 3.1 (the quantities of Eq. 1): for every
+ * community s, in_edges[s] = number of edges with both ends in s and tot[s] = Sigma_tot = sum of
+ * the degrees of its nodes; m = E.  With Sigma_in = 2 * in_edges (every internal edge seen from
+ * both ends, the convention under which a bracket of Eq. 1 is one community's share), the
+ * modularity is  Q = sum_s [ Sigma_in(s) / 2m - (Sigma_tot(s) / 2m)^2 ].  Works on the ORIGINAL
+ * edge list and part vector.  Returns Q (0 for a graph without edges).
+ */
+double oracle_partition_quality(int64_t E, const int32_t* eu, const int32_t* ev, const int32_t* part, int32_t S,
+                                int64_t* in_edges, int64_t* tot) {
+  for (int32_t s = 0; s < S; ++s) in_edges[s] = tot[s] = 0;
+  for (int64_t e = 0; e < E; ++e) {
+    int32_t a = part[eu[e]], b = part[ev[e]];
+    if (a == b) in_edges[a] += 1;
+    tot[a] += 1;
+    tot[b] += 1;
+  }
+  if (E == 0) return 0.0;
+  double two_m = 2.0 * (double)E, q = 0.0;
+  for (int32_t s = 0; s < S; ++s) {
+    double share = (double)tot[s] / two_m;
+    q += 2.0 * (double)in_edges[s] / two_m - share * share;
+  }
+  return q;
+}

@@ -44,6 +44,8 @@ MUTATIONS = {
     "conflict list keeps non-violated edges": ("if (viol[e]) conflict_idx[c++] = (int32_t)e;", "conflict_idx[c++] = (int32_t)e;"),
     "repair clears the nodes that were NOT chosen": ("if (pen[i] != 0.0f && x[i]) {", "if (pen[i] == 0.0f && x[i]) {"),
     "repair counts chosen nodes that were not selected": ("if (pen[i] != 0.0f && x[i]) {", "if (pen[i] != 0.0f) {"),
+    "modularity counts internal edges once": ("q += 2.0 * (double)in_edges[s] / two_m - share * share;", "q += (double)in_edges[s] / two_m - share * share;"),
+    "degree sum misses the second endpoint": ("    tot[a] += 1;\n    tot[b] += 1;", "    tot[a] += 1;"),
     "inv_deg without the +1": ("inv_deg[i] = 1.0f / (float)(hi - lo + 1);", "inv_deg[i] = 1.0f / (float)(hi - lo > 0 ? hi - lo : 1);"),
 }
 
@@ -66,6 +68,7 @@ BATTERY = [
     lambda: pins.test_conflict_list_base_action_and_penalty_brute_force(1),
     lambda: pins.test_conflict_list_base_action_and_penalty_brute_force(2),
     lambda: pins.test_repair_removes_exactly_the_chosen_nodes_brute_force(1),
+    lambda: pins.test_partition_quality_matches_networkx_and_the_pairwise_definition(30, 0.2, 4, 1),
 ]
 
 
@@ -81,7 +84,7 @@ def test_a_pin_fails_when_the_oracle_is_mutated(name, tmp_path, monkeypatch):
     real = oracle._native()
     mutant = ctypes.CDLL(lib_path)
     for fn in ("oracle_bookkeeping", "oracle_subgraph_step", "oracle_train_step", "oracle_adam", "oracle_decode",
-               "oracle_conflict_list", "oracle_base_action", "oracle_apply_actions", "oracle_repair"):
+               "oracle_conflict_list", "oracle_base_action", "oracle_apply_actions", "oracle_repair", "oracle_partition_quality"):
         getattr(mutant, fn).argtypes = getattr(real, fn).argtypes
         getattr(mutant, fn).restype = getattr(real, fn).restype
     monkeypatch.setattr(oracle, "_lib", mutant)

@@ -508,6 +508,54 @@ def test_adam_first_step_is_sign_step_and_zero_gradient_stays():
     assert W[2] == 1.0
 
 
+# ------------------------------------------------------------- partition quality (Section 3.1)
+@pytest.mark.parametrize("n,p,S,seed", [(30, 0.2, 4, 1), (60, 0.1, 7, 2), (25, 0.3, 1, 3), (40, 0.15, 40, 4)])
+def test_partition_quality_matches_networkx_and_the_pairwise_definition(n, p, S, seed):
+    import networkx as nx
+    eu, ev, part = tiny_graph(n, p, S, seed=700 + seed)
+    S = max(S, int(part.max()) + 1)
+    r = oracle.partition_quality(eu, ev, part, S)
+    G = nx.Graph()
+    G.add_nodes_from(range(n))
+    G.add_edges_from(zip(eu.tolist(), ev.tolist()))
+    groups = [set(np.nonzero(part == s)[0].tolist()) for s in range(S)]
+    groups = [g for g in groups if g]
+    np.testing.assert_allclose(r["Q"], nx.community.modularity(G, groups), rtol=1e-12, atol=1e-15)
+    # pairwise definition: Q = 1/(2m) sum_ij [A_ij - k_i k_j / 2m] [c_i = c_j]
+    A = np.zeros((n, n))
+    A[eu, ev] = 1.0
+    A[ev, eu] = 1.0
+    k = A.sum(axis=1)
+    m = eu.size
+    same = part[:, None] == part[None, :]
+    np.testing.assert_allclose(r["Q"], ((A - np.outer(k, k) / (2 * m)) * same).sum() / (2 * m), rtol=1e-12, atol=1e-15)
+    # integer parts, brute force
+    for s in range(S):
+        inside = sum(1 for a, c in zip(eu.tolist(), ev.tolist()) if part[a] == s and part[c] == s)
+        assert r["in_edges"][s] == inside and r["tot"][s] == int(k[part == s].sum())
+    assert r["tot"].sum() == 2 * m
+
+
+def test_delta_q_is_the_exact_change_of_modularity():
+    # move node i out of its own singleton community into a neighbour's community: Q changes by Eq. 2
+    n, S0 = 24, 3
+    eu, ev, part = tiny_graph(n, 0.25, S0, seed=801)
+    m = eu.size
+    deg = np.bincount(np.concatenate([eu, ev]), minlength=n)
+    for i in (2, 7, 13):
+        alone = part.copy()
+        alone[i] = S0                                    # i in a community of its own
+        before = oracle.partition_quality(eu, ev, alone, S0 + 1)
+        for target in range(S0):
+            joined = alone.copy()
+            joined[i] = target
+            after = oracle.partition_quality(eu, ev, joined, S0 + 1)
+            k_i_in = sum(1 for a, c in zip(eu.tolist(), ev.tolist())
+                         if (a == i and alone[c] == target) or (c == i and alone[a] == target))
+            gain = oracle.delta_q(k_i_in, before["tot"][target], deg[i], m)
+            np.testing.assert_allclose(after["Q"] - before["Q"], gain, rtol=1e-10, atol=1e-14)
+
+
 # ------------------------------------------------- Gumbel-softmax input processing (Section 3.2)
 def test_gumbel_softmax_without_noise_is_the_library_softmax():
     from scipy.special import softmax
