@@ -171,6 +171,13 @@ int32_t gnnco_partition_load(const gnnco_graph_desc* g, void* persistent_ws, siz
 
 int32_t gnnco_graph_info(const gnnco_handle* h, gnnco_graph_view* out);
 
+/* Quality of the loaded partition in the terms of Section 3.1 (the quantities of Eq. 1), all device
+ * outputs:  in_edges [S] int64 = edges with both ends in subgraph s;  tot [S] int64 = Sigma_tot, the
+ * degree sum of its nodes in the whole graph;  Q = sum_s [ 2 in_edges(s) / 2m - (tot(s) / 2m)^2 ],
+ * m = E, the modularity that the paper's partitioner maximises (float64; 0 when E = 0).  The
+ * integers are exact.  Asynchronous on `stream`. */
+int32_t gnnco_partition_quality(gnnco_handle* h, int64_t* in_edges, int64_t* tot, double* Q, void* stream);
+
 /* dst[i] = src[index[i]] for i < rows, rows of row_bytes bytes each (row_bytes a
  * multiple of 4).  With index = perm it brings a per-node array from the caller's
  * original order into the new order (Algorithm 1, Stage 2 uses the inverse to "map

@@ -27,7 +27,7 @@ EXPORTS = [
     "gnnco_train_step_host", "gnnco_decode_boundary", "gnnco_async_status", "gnnco_launch_count", "gnnco_destroy",
     "gnnco_profile_begin", "gnnco_profile_end", "gnnco_objective_static", "gnnco_conflict_workspace_bytes",
     "gnnco_conflict_actions", "gnnco_apply_actions", "gnnco_gumbel_softmax", "gnnco_embedding_update",
-    "gnnco_repair_boundary",
+    "gnnco_repair_boundary", "gnnco_partition_quality",
 ]
 
 _vp, _i32, _i64, _u32, _f32, _sz = (ctypes.c_void_p, ctypes.c_int32, ctypes.c_int64, ctypes.c_uint32, ctypes.c_float,
@@ -113,6 +113,7 @@ def load_library(build_if_missing: bool = True):
     lib.gnnco_conflict_workspace_bytes.argtypes = [_vp, ctypes.POINTER(_sz)]
     lib.gnnco_conflict_actions.argtypes = [_vp, _vp, _vp, _vp, _vp, _vp, _vp, _sz, _vp]
     lib.gnnco_apply_actions.argtypes = [_vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp]
+    lib.gnnco_partition_quality.argtypes = [_vp, _vp, _vp, _vp, _vp]
     lib.gnnco_repair_boundary.argtypes = [_vp, _vp, _vp, _vp, _vp]
     lib.gnnco_gumbel_softmax.argtypes = [_vp, _i32, _i32, _vp, _vp, _f32, _vp, _vp]
     lib.gnnco_embedding_update.argtypes = [_vp, _i32, _i32, _vp, _vp, _vp, _vp, _vp, _f32, _f32, _f32, _f32, _i64, _vp]
@@ -399,6 +400,16 @@ class PartitionedGraph:
                                              count.data_ptr(), pen.data_ptr(), active.data_ptr(), chosen.data_ptr(),
                                              _stream_ptr(stream)), "gnnco_apply_actions")
         return dict(pen=pen, active=active, chosen=chosen)
+
+    def partition_quality(self, stream=None):
+        """``gnnco_partition_quality``: dict(in_edges int64 [S], tot int64 [S], Q float64 [1]) on the device."""
+        import torch
+        in_edges = torch.empty(self.S, dtype=torch.int64, device=self.device)
+        tot = torch.empty(self.S, dtype=torch.int64, device=self.device)
+        Q = torch.empty(1, dtype=torch.float64, device=self.device)
+        _check(self._lib.gnnco_partition_quality(self._handle, in_edges.data_ptr(), tot.data_ptr(), Q.data_ptr(),
+                                                 _stream_ptr(stream)), "gnnco_partition_quality")
+        return dict(in_edges=in_edges, tot=tot, Q=Q)
 
     def repair_boundary(self, pen, x, stream=None):
         """``gnnco_repair_boundary``: clears, in place, every chosen node (``pen`` != 0) from the

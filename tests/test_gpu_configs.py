@@ -142,6 +142,10 @@ def _full_size_sampled(idx, steps, n_parts):
     book = oracle.bookkeeping(w.n, w.eu, w.ev, w.part, w.S)
     graph = load_graph(w.n, w.eu, w.ev, w.part, w.S)
     check_bookkeeping(graph, book)
+    quality, ref_quality = graph.partition_quality(), oracle.partition_quality(w.eu, w.ev, w.part, w.S)
+    assert np.array_equal(quality["in_edges"].cpu().numpy(), ref_quality["in_edges"])
+    assert np.array_equal(quality["tot"].cpu().numpy(), ref_quality["tot"])
+    np.testing.assert_allclose(float(quality["Q"].item()), ref_quality["Q"], rtol=1e-12)
     arr = graph.arrays()
     bf16 = w.dtype == "bf16"
     if bf16:

@@ -55,6 +55,20 @@ def test_bookkeeping_and_decode_small(name):
     check_decode(graph, book, np.zeros(n, np.float32))
 
 
+@pytest.mark.parametrize("name", sorted(GRAPHS))
+def test_partition_quality_small(name):
+    eu, ev, part = GRAPHS[name]()
+    n, S = _n_S(part)
+    if name == "empty_parts":
+        S = 6
+    graph = load_graph(n, eu, ev, part, S)
+    ref = oracle.partition_quality(eu, ev, part, S)
+    got = graph.partition_quality()
+    assert np.array_equal(got["in_edges"].cpu().numpy(), ref["in_edges"])
+    assert np.array_equal(got["tot"].cpu().numpy(), ref["tot"])
+    np.testing.assert_allclose(float(got["Q"].item()), ref["Q"], rtol=1e-12, atol=1e-15)
+
+
 def test_partition_load_rejects_bad_graphs():
     import paper_2511_09261_b200 as gnnco
     part = np.zeros(4, np.int32)
