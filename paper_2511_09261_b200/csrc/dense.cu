@@ -161,19 +161,24 @@ __global__ void __launch_bounds__(256) gemv_rows(const TA* __restrict__ H, const
   if (lane == 0) u[row] = acc;
 }
 
-// dw[s][:] = sum_{i in s} H[i,:] g[i].  One block per subgraph; LPR lanes cover a row with
-// 16-byte loads, the 256/LPR row groups walk the subgraph's rows interleaved (four rows in
-// flight each) and meet in shared memory in a fixed order.
+// dw[s][:] = sum_{i in s} H[i,:] g[i].  One block per row chunk of the weight-gradient chunk
+// table (a whole subgraph, or a run of rows of a very long one whose partial result goes to a
+// scratch slot and is combined in chunk order afterwards); LPR lanes cover a row with 16-byte
+// loads, the 256/LPR row groups walk the chunk's rows interleaved (four rows in flight each)
+// and meet in shared memory in a fixed order.
 template <typename TA, int LPR>
 __global__ void __launch_bounds__(256) weight_grad_vec_rows(const TA* __restrict__ H, const float* __restrict__ g,
-                                                            float* __restrict__ dw, int F,
-                                                            const int32_t* __restrict__ part_ptr) {
+                                                            float* __restrict__ dw, float* __restrict__ scratch, int F,
+                                                            const int32_t* __restrict__ wg_begin,
+                                                            const int32_t* __restrict__ wg_end,
+                                                            const int32_t* __restrict__ wg_slot) {
   constexpr int VN = 16 / sizeof(TA);
   constexpr int RG = 256 / LPR;
   extern __shared__ float partial[];                       // [RG][F]
-  const int s = blockIdx.x;
   const int sub = threadIdx.x % LPR, rg = threadIdx.x / LPR;
-  const int64_t ra = part_ptr[s], rb = part_ptr[s + 1];
+  const int64_t ra = wg_begin[blockIdx.x], rb = wg_end[blockIdx.x];
+  const int32_t slot = wg_slot[blockIdx.x];
+  float* out = slot < 0 ? dw + (int64_t)(-(slot + 1)) * F : scratch + (int64_t)slot * F;
   float acc[VN];
 #pragma unroll
   for (int e = 0; e < VN; ++e) acc[e] = 0.0f;
@@ -209,22 +214,25 @@ __global__ void __launch_bounds__(256) weight_grad_vec_rows(const TA* __restrict
   for (int f = threadIdx.x; f < F; f += 256) {
     float tot = 0.0f;
     for (int r = 0; r < RG; ++r) tot += partial[r * F + f];
-    dw[(int64_t)s * F + f] = tot;
+    out[f] = tot;
   }
 }
 
 // any width: one thread per column
 template <typename TA>
 __global__ void __launch_bounds__(256) weight_grad_vec_kernel(const TA* __restrict__ H, const float* __restrict__ g,
-                                                              float* __restrict__ dw, int F,
-                                                              const int32_t* __restrict__ part_ptr) {
-  const int s = blockIdx.x;
+                                                              float* __restrict__ dw, float* __restrict__ scratch,
+                                                              int F, const int32_t* __restrict__ wg_begin,
+                                                              const int32_t* __restrict__ wg_end,
+                                                              const int32_t* __restrict__ wg_slot) {
   const int f = blockIdx.y * 256 + threadIdx.x;
   if (f >= F) return;
-  const int64_t ra = part_ptr[s], rb = part_ptr[s + 1];
+  const int64_t ra = wg_begin[blockIdx.x], rb = wg_end[blockIdx.x];
+  const int32_t slot = wg_slot[blockIdx.x];
+  float* out = slot < 0 ? dw + (int64_t)(-(slot + 1)) * F : scratch + (int64_t)slot * F;
   float acc = 0.0f;
   for (int64_t i = ra; i < rb; ++i) acc = fmaf(ld(H + i * F + f), __ldg(g + i), acc);
-  dw[(int64_t)s * F + f] = acc;
+  out[f] = acc;
 }
 
 template <typename TA, typename TW>
@@ -426,15 +434,17 @@ int32_t launch_weight_grad(gnnco_handle* h, int dtype, const void* A, const void
   return GNNCO_OK;
 }
 
-int32_t launch_weight_grad_vec(gnnco_handle* h, int dtype, const void* H, const float* g, float* dw, int F,
-                               cudaStream_t stream) {
+int32_t launch_weight_grad_vec(gnnco_handle* h, int dtype, const void* H, const float* g, float* dw, float* scratch,
+                               int F, cudaStream_t stream) {
   ProfScope prof_(h, K_WEIGHT_GRAD_VEC, stream);
+  if (h->n_wg_slots > 0 && !scratch) return GNNCO_INTERNAL;
   const int vn = dtype == GNNCO_BF16 ? 8 : 4;
   const int lpr = F % vn == 0 ? F / vn : 0;
   const bool aligned = !((uintptr_t)H & 15);
   const size_t sm = (size_t)(lpr ? 256 / lpr : 0) * F * sizeof(float);
 #define GNNCO_WGV(TT, L)                                                                                     \
-  weight_grad_vec_rows<TT, L><<<h->S, 256, sm, stream>>>((const TT*)H, g, dw, F, h->part_ptr)
+  weight_grad_vec_rows<TT, L><<<h->n_wg_chunks, 256, sm, stream>>>((const TT*)H, g, dw, scratch, F, h->wg_begin, \
+                                                                   h->wg_end, h->wg_slot)
   bool done = aligned && (lpr == 8 || lpr == 16 || lpr == 32 || lpr == 64);
   if (done && dtype == GNNCO_F32) {
     if (lpr == 8) GNNCO_WGV(float, 8); else if (lpr == 16) GNNCO_WGV(float, 16);
@@ -443,19 +453,21 @@ int32_t launch_weight_grad_vec(gnnco_handle* h, int dtype, const void* H, const 
     if (lpr == 8) GNNCO_WGV(__nv_bfloat16, 8); else if (lpr == 16) GNNCO_WGV(__nv_bfloat16, 16);
     else if (lpr == 32) GNNCO_WGV(__nv_bfloat16, 32); else GNNCO_WGV(__nv_bfloat16, 64);
   } else {
-    dim3 grid(h->S, (F + 255) / 256);
+    dim3 grid(h->n_wg_chunks, (F + 255) / 256);
     if (grid.y > 65535) return GNNCO_UNSUPPORTED;
     if (dtype == GNNCO_F32)
-      weight_grad_vec_kernel<float><<<grid, 256, 0, stream>>>((const float*)H, g, dw, F, h->part_ptr);
+      weight_grad_vec_kernel<float><<<grid, 256, 0, stream>>>((const float*)H, g, dw, scratch, F, h->wg_begin,
+                                                              h->wg_end, h->wg_slot);
     else if (dtype == GNNCO_BF16)
-      weight_grad_vec_kernel<__nv_bfloat16><<<grid, 256, 0, stream>>>((const __nv_bfloat16*)H, g, dw, F, h->part_ptr);
+      weight_grad_vec_kernel<__nv_bfloat16><<<grid, 256, 0, stream>>>((const __nv_bfloat16*)H, g, dw, scratch, F,
+                                                                      h->wg_begin, h->wg_end, h->wg_slot);
     else
       return GNNCO_UNSUPPORTED;
   }
 #undef GNNCO_WGV
   h->launches += 1;
   GNNCO_LAUNCH_CHECK();
-  return GNNCO_OK;
+  return launch_wg_combine(h, scratch, dw, F, stream);
 }
 
 int32_t launch_rank1_masked(gnnco_handle* h, int dtype, const float* g, const void* w, int64_t w_stride, const void* H,

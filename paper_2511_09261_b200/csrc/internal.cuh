@@ -133,9 +133,9 @@ int32_t launch_gemv(gnnco_handle* h, int dtype, const void* H, const void* w, in
 // dW[s] (K x N) = sum_{i in s} A[i,:]^T G[i,:]
 int32_t launch_weight_grad(gnnco_handle* h, int dtype, const void* A, const void* G, float* dW, int K, int N,
                            cudaStream_t st);
-// dw[s][f] = sum_{i in s} H[i,f] g[i]
-int32_t launch_weight_grad_vec(gnnco_handle* h, int dtype, const void* H, const float* g, float* dw, int F,
-                               cudaStream_t st);
+// dw[s][f] = sum_{i in s} H[i,f] g[i]; scratch: F floats per slot of the weight-gradient chunk table
+int32_t launch_weight_grad_vec(gnnco_handle* h, int dtype, const void* H, const float* g, float* dw, float* scratch,
+                               int F, cudaStream_t st);
 // dZ[i,f] = g[i] * w_s[f] where H[i,f] > 0, else 0 (H == nullptr: no mask)
 int32_t launch_rank1_masked(gnnco_handle* h, int dtype, const float* g, const void* w, int64_t w_stride, const void* H,
                             void* dZ, int F, cudaStream_t st);

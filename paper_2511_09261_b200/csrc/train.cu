@@ -194,10 +194,10 @@ int32_t run_step(gnnco_handle* h, const gnnco_model_desc* m, const void* X, cons
     // last layer (0-based index L-1): dw = H^T g
     float* target = grad_target(L - 1);
     if (sets == 1) {
-      GNNCO_TRY(launch_weight_grad_vec(h, dt, Hprev, T.g, T.dW_sets, FL, st));
+      GNNCO_TRY(launch_weight_grad_vec(h, dt, Hprev, T.g, T.dW_sets, T.wg_scratch, FL, st));
       GNNCO_TRY(launch_sum_over_sets(h, T.dW_sets, target, FL, h->S, st));
     } else {
-      GNNCO_TRY(launch_weight_grad_vec(h, dt, Hprev, T.g, target, FL, st));
+      GNNCO_TRY(launch_weight_grad_vec(h, dt, Hprev, T.g, target, T.wg_scratch, FL, st));
     }
     // everything that reads the weights of a layer runs before that layer's Adam update
     if (L > 1) GNNCO_TRY(launch_aggregate_rank1(h, dt, Hprev, T.u, Wc[L - 1], wstride[L - 1], Q, FL, st));
