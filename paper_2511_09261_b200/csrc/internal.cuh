@@ -22,6 +22,7 @@
 
 constexpr int kGemmTileRows = 128;   // rows of one dense-transform tile (never straddles a subgraph)
 constexpr int kLongRowDegree = 256;  // rows with more intra neighbours are aggregated by a whole block
+constexpr int kLongRowSegment = 2048; // ... and in segments of this many neighbours, one block each
 constexpr int kWgChunkMinRows = 2048; // a subgraph is split for the weight gradient only in runs at least this long
 constexpr int kItemRows = 1024;      // rows of one objective work item (never straddles a subgraph)
 
@@ -63,7 +64,12 @@ struct gnnco_handle {
   int32_t* part_item_ptr = nullptr;                        // [S+1] items of each subgraph
   int32_t* status = nullptr;                               // device status word + counters
   int4* row_head = nullptr;                                // {first CSR slot, degree, first two neighbours} per row
-  int32_t* long_rows = nullptr;                            // ids of rows with degree > kLongRowDegree
+  int32_t* long_rows = nullptr;                            // ids of rows with degree > kLongRowDegree, ascending
+  // the long rows' neighbour lists cut into segments: CSR slots [seg_begin, seg_end) of each segment, and
+  // for long row k its segments long_first_seg[k] .. long_first_seg[k+1]-1
+  int32_t *seg_begin = nullptr, *seg_end = nullptr, *long_first_seg = nullptr;
+  int32_t n_long_segs = 0;
+  float* agg_partial = nullptr;                            // [n_long_segs x width] float32, set for the running step
   int32_t n_tiles = 0, n_items = 0, n_long = 0;
   // weight-gradient work: row ranges, output slot (>= 0 scratch slot, < 0 subgraph -(slot+1)), and the
   // subgraphs that were split (id, first slot, slot count)

@@ -7,6 +7,7 @@
 // stable least-significant-digit radix sort of 64-bit keys, and "segment starts of a
 // sorted key array".  Slot allocation for the two edge classes uses integer atomics, but
 // both lists are sorted afterwards, so every output is uniquely defined.
+#include <algorithm>
 #include <new>
 
 #include "internal.cuh"
@@ -290,6 +291,14 @@ __global__ void collect_long_rows(const int32_t* rowptr, int64_t n, int32_t* lon
   }
 }
 
+// extents of the listed rows: ext[2k] = rowptr[rows[k]], ext[2k+1] = rowptr[rows[k] + 1]
+__global__ void gather_extents(const int32_t* rows, const int32_t* rowptr, int32_t count, int32_t* ext) {
+  const int32_t k = blockIdx.x * blockDim.x + threadIdx.x;
+  if (k >= count) return;
+  ext[2 * k] = rowptr[rows[k]];
+  ext[2 * k + 1] = rowptr[rows[k] + 1];
+}
+
 template <int VEC>
 __global__ void gather_rows_kernel(const char* src, char* dst, const int32_t* index, int64_t rows, int64_t units) {
   int64_t t = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
@@ -312,11 +321,11 @@ struct PersistentLayout {
   int32_t *perm, *inv_perm, *node_part, *part_ptr, *rowptr, *colidx, *bnd_u, *bnd_v;
   float* inv_deg;
   uint8_t* is_boundary;
-  int32_t *tile_row0, *tile_rows, *item_row0, *item_row1, *part_item_ptr, *status, *long_rows;
+  int32_t *tile_row0, *tile_rows, *item_row0, *item_row1, *part_item_ptr, *status, *long_rows, *seg_begin, *seg_end, *long_first_seg;
   int4* row_head;
   int32_t *wg_begin, *wg_end, *wg_slot, *wg_mpart, *wg_mfirst, *wg_mcount;
   int64_t max_chunks;
-  int64_t max_tiles, max_items, max_long;
+  int64_t max_tiles, max_items, max_long, max_segs;
   size_t bytes;
 };
 
@@ -343,6 +352,10 @@ PersistentLayout carve_persistent(void* base, int64_t n, int64_t E, int32_t S) {
   L.part_item_ptr = c.take<int32_t>((size_t)S + 1);
   L.max_long = 2 * E / kLongRowDegree + 1;
   L.long_rows = c.take<int32_t>(L.max_long);
+  L.max_segs = 2 * E / kLongRowSegment + L.max_long + 1;
+  L.seg_begin = c.take<int32_t>(L.max_segs);
+  L.seg_end = c.take<int32_t>(L.max_segs);
+  L.long_first_seg = c.take<int32_t>(L.max_long + 1);
   L.row_head = c.take<int4>(n);
   L.max_chunks = (int64_t)S + n / kWgChunkMinRows + 1;
   L.wg_begin = c.take<int32_t>(L.max_chunks);
@@ -429,7 +442,8 @@ extern "C" int32_t gnnco_partition_load(const gnnco_graph_desc* g, void* persist
   h->rowptr = P.rowptr; h->colidx = P.colidx; h->bnd_u = P.bnd_u; h->bnd_v = P.bnd_v;
   h->inv_deg = P.inv_deg; h->is_boundary = P.is_boundary;
   h->tile_row0 = P.tile_row0; h->tile_rows = P.tile_rows; h->item_row0 = P.item_row0; h->item_row1 = P.item_row1;
-  h->part_item_ptr = P.part_item_ptr; h->status = P.status; h->long_rows = P.long_rows; h->row_head = P.row_head;
+  h->part_item_ptr = P.part_item_ptr; h->status = P.status; h->long_rows = P.long_rows; h->seg_begin = P.seg_begin; h->seg_end = P.seg_end;
+  h->long_first_seg = P.long_first_seg; h->row_head = P.row_head;
   h->wg_begin = P.wg_begin; h->wg_end = P.wg_end; h->wg_slot = P.wg_slot;
   h->wg_mpart = P.wg_mpart; h->wg_mfirst = P.wg_mfirst; h->wg_mcount = P.wg_mcount;
 
@@ -578,6 +592,37 @@ extern "C" int32_t gnnco_partition_load(const gnnco_graph_desc* g, void* persist
   GNNCO_CUDA_TRY(cudaEventCreateWithFlags(&h->ev_join, cudaEventDisableTiming));
   h->n_long = hs[kLongCnt];
   if (h->n_long > P.max_long) return GNNCO_INTERNAL;
+  if (h->n_long > 0) {
+    // The long rows were collected in no particular order: sort them, then cut every row's
+    // neighbour list into segments of at most kLongRowSegment entries (one block each in the
+    // aggregation; a row's segments are consecutive, so its partial sums are added in a fixed order).
+    std::vector<int32_t> lr((size_t)h->n_long), ext(2 * (size_t)h->n_long);
+    GNNCO_CUDA_TRY(cudaMemcpyAsync(lr.data(), P.long_rows, lr.size() * sizeof(int32_t), cudaMemcpyDeviceToHost, st));
+    GNNCO_CUDA_TRY(cudaStreamSynchronize(st));
+    std::sort(lr.begin(), lr.end());
+    GNNCO_CUDA_TRY(cudaMemcpyAsync(P.long_rows, lr.data(), lr.size() * sizeof(int32_t), cudaMemcpyHostToDevice, st));
+    // 2 * n_long <= 2 * max_long <= max_segs + max_long: seg_begin is large enough to hold the extents for a moment
+    if (2 * (int64_t)h->n_long > P.max_segs) return GNNCO_INTERNAL;
+    gather_extents<<<grid_for(h->n_long, T), T, 0, st>>>(P.long_rows, P.rowptr, h->n_long, P.seg_begin);
+    h->launches += 1;
+    GNNCO_CUDA_TRY(cudaMemcpyAsync(ext.data(), P.seg_begin, ext.size() * sizeof(int32_t), cudaMemcpyDeviceToHost, st));
+    GNNCO_CUDA_TRY(cudaStreamSynchronize(st));
+    std::vector<int32_t> sb, se, first((size_t)h->n_long + 1);
+    for (int32_t k = 0; k < h->n_long; ++k) {
+      first[k] = (int32_t)sb.size();
+      for (int64_t a = ext[2 * k]; a < ext[2 * k + 1]; a += kLongRowSegment) {
+        sb.push_back((int32_t)a);
+        se.push_back((int32_t)(a + kLongRowSegment < ext[2 * k + 1] ? a + kLongRowSegment : ext[2 * k + 1]));
+      }
+    }
+    first[h->n_long] = (int32_t)sb.size();
+    if ((int64_t)sb.size() > P.max_segs) return GNNCO_INTERNAL;
+    h->n_long_segs = (int32_t)sb.size();
+    GNNCO_CUDA_TRY(up(P.seg_begin, sb));
+    GNNCO_CUDA_TRY(up(P.seg_end, se));
+    GNNCO_CUDA_TRY(up(P.long_first_seg, first));
+    GNNCO_CUDA_TRY(cudaStreamSynchronize(st));      // the host vectors go out of scope
+  }
   guard.h = nullptr;
   *out = h;
   return GNNCO_OK;

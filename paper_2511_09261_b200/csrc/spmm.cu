@@ -269,19 +269,27 @@ __global__ void __launch_bounds__(256) aggregate_vec(const T* __restrict__ in, T
 // A row with more than kLongRowDegree neighbours: one block per row.  Each of the 8 warps sums
 // a contiguous eighth of the neighbour list with eight rows in flight, the partial sums
 // meet in shared memory in warp order (deterministic), and the block finishes the row.
+// With a segment table (seg_out != nullptr) a block instead sums ONE SEGMENT of a long row's
+// neighbour list (at most kLongRowSegment entries) into seg_out[segment][F], float32, and
+// aggregate_long_finish adds a row's segments up in order: a hub of tens of thousands of
+// neighbours then occupies a dozen blocks for a moment instead of one block for a millisecond.
 template <typename T, int LPR, int VPL, bool R1>
 __global__ void __launch_bounds__(256) aggregate_long_row(const T* __restrict__ in, T* __restrict__ out,
                                                           const int32_t* __restrict__ rowptr,
                                                           const int32_t* __restrict__ colidx,
                                                           const float* __restrict__ scale,
                                                           const T* __restrict__ mask, const Rank1Args<T> r1,
-                                                          const int32_t* __restrict__ long_rows, int F) {
+                                                          const int32_t* __restrict__ long_rows, int F,
+                                                          const int32_t* __restrict__ seg_begin,
+                                                          const int32_t* __restrict__ seg_end,
+                                                          float* __restrict__ seg_out) {
   constexpr int VN = Vec<T>::N;
   constexpr int GROUPS = 256 / LPR;               // lane groups, each walks its own slice of the row
   extern __shared__ float partial[];              // [GROUPS][F]
-  const int64_t row = long_rows[blockIdx.x];
+  const int64_t row = seg_out ? 0 : long_rows[blockIdx.x];
   const int sub = threadIdx.x % LPR, grp = threadIdx.x / LPR;
-  const int32_t r0 = rowptr[row], r1_end = rowptr[row + 1];
+  const int32_t r0 = seg_out ? seg_begin[blockIdx.x] : rowptr[row];
+  const int32_t r1_end = seg_out ? seg_end[blockIdx.x] : rowptr[row + 1];
   const int32_t len = (r1_end - r0 + GROUPS - 1) / GROUPS;
   const int32_t a = r0 + grp * len, b = min(r1_end, a + len);
   float acc[VPL][VN];
@@ -314,6 +322,14 @@ __global__ void __launch_bounds__(256) aggregate_long_row(const T* __restrict__ 
 #pragma unroll
     for (int e = 0; e < VN; ++e) partial[grp * F + (v * LPR + sub) * VN + e] = acc[v][e];
   __syncthreads();
+  if (seg_out) {
+    for (int f = threadIdx.x; f < F; f += 256) {
+      float tot = 0.0f;
+      for (int g = 0; g < GROUPS; ++g) tot += partial[g * F + f];
+      seg_out[(int64_t)blockIdx.x * F + f] = tot;
+    }
+    return;
+  }
   if constexpr (R1) {
     const float ci = r1.coef[row];
     const T* wv = r1.w + (int64_t)r1.node_part[row] * r1.w_stride;
@@ -331,6 +347,32 @@ __global__ void __launch_bounds__(256) aggregate_long_row(const T* __restrict__ 
       if (mask && !(to_f32(mask[row * F + f]) > 0.0f)) tot = 0.0f;
       from_f32(out[row * F + f], tot);
     }
+  }
+}
+
+// Second half of the segmented long rows: one block per long row adds the row's own features
+// and its segments' partial sums (in segment order) and applies the epilogue of the mode.
+template <typename T, bool R1>
+__global__ void __launch_bounds__(256) aggregate_long_finish(const T* __restrict__ in, T* __restrict__ out,
+                                                             const float* __restrict__ scale,
+                                                             const T* __restrict__ mask, const Rank1Args<T> r1,
+                                                             const int32_t* __restrict__ long_rows,
+                                                             const int32_t* __restrict__ long_first_seg,
+                                                             const float* __restrict__ seg_part, int F) {
+  const int64_t row = long_rows[blockIdx.x];
+  const int32_t s0 = long_first_seg[blockIdx.x], s1 = long_first_seg[blockIdx.x + 1];
+  for (int f = threadIdx.x; f < F; f += 256) {
+    float tot;
+    if constexpr (R1) tot = to_f32(in[row * F + f]) > 0.0f ? r1.coef[row] : 0.0f;
+    else tot = to_f32(in[row * F + f]);
+    for (int32_t sg = s0; sg < s1; ++sg) tot += seg_part[(int64_t)sg * F + f];
+    if constexpr (R1) {
+      tot *= to_f32(r1.w[(int64_t)r1.node_part[row] * r1.w_stride + f]);
+    } else {
+      tot *= scale ? scale[row] : 1.0f;
+      if (mask && !(to_f32(mask[row * F + f]) > 0.0f)) tot = 0.0f;
+    }
+    from_f32(out[row * F + f], tot);
   }
 }
 
@@ -382,9 +424,18 @@ void launch_vec(const T* in, T* out, gnnco_handle* h, const float* scale, const 
     const bool fork = h->side_stream && h->ev_fork && h->ev_join && cudaEventRecord(h->ev_fork, st) == cudaSuccess &&
                       cudaStreamWaitEvent(h->side_stream, h->ev_fork, 0) == cudaSuccess;
     cudaStream_t ls = fork ? h->side_stream : st;
-    aggregate_long_row<T, LPR, VPL, R1><<<count, 256, long_smem, ls>>>(in, out, h->rowptr, h->colidx, scale, mask, r1,
-                                                                       list, F);
-    h->launches += 1;
+    if (h->agg_partial && h->n_long_segs > 0) {
+      // long rows cut into segments: partial sums by one block per segment, then one block per row
+      aggregate_long_row<T, LPR, VPL, R1><<<h->n_long_segs, 256, long_smem, ls>>>(
+          in, out, h->rowptr, h->colidx, scale, mask, r1, list, F, h->seg_begin, h->seg_end, h->agg_partial);
+      aggregate_long_finish<T, R1><<<count, 256, 0, ls>>>(in, out, scale, mask, r1, list, h->long_first_seg,
+                                                          h->agg_partial, F);
+      h->launches += 2;
+    } else {
+      aggregate_long_row<T, LPR, VPL, R1><<<count, 256, long_smem, ls>>>(in, out, h->rowptr, h->colidx, scale, mask,
+                                                                         r1, list, F, nullptr, nullptr, nullptr);
+      h->launches += 1;
+    }
     if (fork) cudaEventRecord(h->ev_join, h->side_stream);
     return fork;
   };

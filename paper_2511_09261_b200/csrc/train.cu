@@ -31,6 +31,7 @@ struct TrainLayout {
   float* dW_scratch;                  // one layer's gradient (all sets), when the caller wants none
   float* dW_sets;                     // per-subgraph partials when the model shares one weight set
   float* wg_scratch;                  // partial weight gradients of subgraphs that were split into row chunks
+  float* agg_partial;                 // partial sums of the segments of long rows (aggregation)
   __nv_bfloat16* W_lp[GNNCO_MAX_LAYERS];   // bf16 copies of the weights (bf16 features only)
   __nv_bfloat16* W_lp_t[GNNCO_MAX_LAYERS]; // transposed bf16 copies [sets x F_out x F_in] for the tensor-core forward
   __nv_bfloat16* W3[GNNCO_MAX_LAYERS];     // float32 features: three bf16 limbs of W (input-gradient operand)
@@ -79,6 +80,7 @@ TrainLayout carve_train(const gnnco_handle* h, const gnnco_model_desc* m, uint32
   T.t = c.take<float>(n);
   T.g = c.take<float>(n);
   T.item_loss = c.take<float>((size_t)h->n_items + 1);
+  T.agg_partial = h->n_long_segs > 0 ? c.take<float>((size_t)h->n_long_segs * maxw) : nullptr;
   if (!(flags & GNNCO_FORWARD_ONLY)) {
     if (L > 2) T.Gb = c.take<char>(n * maxw * es);
     T.dW_scratch = c.take<float>(max_wcount * m->weight_sets);
@@ -113,6 +115,7 @@ int32_t run_step(gnnco_handle* h, const gnnco_model_desc* m, const void* X, cons
                  cudaStream_t st) {
   const int L = m->L, dt = m->feat_dtype;
   const bool bf16 = dt == GNNCO_BF16;
+  h->agg_partial = T.agg_partial;       // where this step's aggregations keep the segments of long rows
   const int32_t sets = m->weight_sets;
   int32_t rc;
 #define GNNCO_TRY(call) do { rc = (call); if (rc != GNNCO_OK) return rc; } while (0)
