@@ -56,32 +56,64 @@ __global__ void __launch_bounds__(256) intra_conflicts_kernel(const uint8_t* __r
   block_add_u64(cnt, intra);
 }
 
+// Four consecutive boundary edges per thread: the eight endpoint bits are gathered together
+// (they are the kernel's only dependent loads), endpoints and flags move as 16- and 4-byte words.
 __global__ void __launch_bounds__(256) boundary_conflicts_kernel(const uint8_t* __restrict__ x,
                                                                  const int32_t* __restrict__ bnd_u,
                                                                  const int32_t* __restrict__ bnd_v,
                                                                  const int32_t* __restrict__ node_part, int64_t E_b,
                                                                  uint8_t* __restrict__ viol,
                                                                  int32_t* __restrict__ per_part,
-                                                                 unsigned long long* total) {
-  const int64_t e = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+                                                                 unsigned long long* total, int vectorised) {
+  const int64_t e0 = ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) * 4;
   const int lane = threadIdx.x & 31;
-  unsigned long long v = 0;
-  int32_t su = -1, sv = -1;
-  if (e < E_b) {
-    const int32_t a = bnd_u[e], b = bnd_v[e];
-    v = (x[a] & x[b]) ? 1 : 0;
-    if (viol) viol[e] = (uint8_t)v;
-    if (v && per_part) { su = node_part[a]; sv = node_part[b]; }
+  int32_t a[4], b[4];
+  if (vectorised && e0 + 4 <= E_b) {
+    const int4 ua = __ldg(reinterpret_cast<const int4*>(bnd_u + e0)), va = __ldg(reinterpret_cast<const int4*>(bnd_v + e0));
+    a[0] = ua.x; a[1] = ua.y; a[2] = ua.z; a[3] = ua.w;
+    b[0] = va.x; b[1] = va.y; b[2] = va.z; b[3] = va.w;
+  } else {
+#pragma unroll
+    for (int k = 0; k < 4; ++k) {
+      a[k] = e0 + k < E_b ? bnd_u[e0 + k] : -1;
+      b[k] = e0 + k < E_b ? bnd_v[e0 + k] : -1;
+    }
+  }
+  uint8_t xa[4], xb[4];
+#pragma unroll
+  for (int k = 0; k < 4; ++k) {
+    xa[k] = a[k] >= 0 ? x[a[k]] : 0;
+    xb[k] = b[k] >= 0 ? x[b[k]] : 0;
+  }
+  unsigned long long count = 0;
+  uint8_t v[4];
+#pragma unroll
+  for (int k = 0; k < 4; ++k) {
+    v[k] = (xa[k] & xb[k]) ? 1 : 0;
+    count += v[k];
+  }
+  if (viol) {
+    if (vectorised && e0 + 4 <= E_b) {
+      *reinterpret_cast<uchar4*>(viol + e0) = make_uchar4(v[0], v[1], v[2], v[3]);
+    } else {
+#pragma unroll
+      for (int k = 0; k < 4; ++k)
+        if (e0 + k < E_b) viol[e0 + k] = v[k];
+    }
   }
   if (per_part) {
     // edges are sorted by their lower endpoint, so neighbouring lanes mostly share su:
-    // one atomic per distinct subgraph in the warp
-    uint32_t peers = __match_any_sync(0xffffffffu, su);
-    if (su >= 0 && lane == __ffs(peers) - 1) atomicAdd(per_part + su, __popc(peers));
-    peers = __match_any_sync(0xffffffffu, sv);
-    if (sv >= 0 && lane == __ffs(peers) - 1) atomicAdd(per_part + sv, __popc(peers));
+    // one atomic per distinct subgraph in the warp and edge slot
+#pragma unroll
+    for (int k = 0; k < 4; ++k) {
+      const int32_t su = v[k] ? node_part[a[k]] : -1, sv = v[k] ? node_part[b[k]] : -1;
+      uint32_t peers = __match_any_sync(0xffffffffu, su);
+      if (su >= 0 && lane == __ffs(peers) - 1) atomicAdd(per_part + su, __popc(peers));
+      peers = __match_any_sync(0xffffffffu, sv);
+      if (sv >= 0 && lane == __ffs(peers) - 1) atomicAdd(per_part + sv, __popc(peers));
+    }
   }
-  block_add_u64(v, total);
+  block_add_u64(count, total);
 }
 
 }  // namespace
@@ -97,8 +129,10 @@ int32_t launch_decode(gnnco_handle* h, const float* p, float thr, uint8_t* x, ui
   intra_conflicts_kernel<<<grid, 256, 0, st>>>(x, h->rowptr, h->colidx, h->n, c + 1);
   h->launches += 2;
   if (h->E_b > 0) {
-    unsigned gb = (unsigned)((h->E_b + 255) / 256);
-    boundary_conflicts_kernel<<<gb, 256, 0, st>>>(x, h->bnd_u, h->bnd_v, h->node_part, h->E_b, viol, per_part, c + 2);
+    unsigned gb = (unsigned)((h->E_b + 1023) / 1024);
+    const int vectorised = (((uintptr_t)h->bnd_u | (uintptr_t)h->bnd_v) & 15) == 0 && ((uintptr_t)viol & 3) == 0;
+    boundary_conflicts_kernel<<<gb, 256, 0, st>>>(x, h->bnd_u, h->bnd_v, h->node_part, h->E_b, viol, per_part, c + 2,
+                                                  vectorised);
     h->launches += 1;
   }
   GNNCO_LAUNCH_CHECK();
