@@ -187,7 +187,9 @@ def algorithmic_bytes(kind, w, n, nnz, S):
         # transposed aggregation of layers 2..L-1 (plain gather-sum, no scale, no mask)
         per["aggregate_bwd"] = np.mean([2 * n * d[l - 1] * b + csr for l in hidden[1:]]) if L > 2 else 0.0
         # rank-1 mode below the output layer: gathers H_{L-1}, reads coef and the weight vectors
-        per["aggregate_rank1"] = 2 * n * d[L - 1] * b + csr + 4 * n + S * d[L - 1] * b
+        # (bfloat16: it gathers the mask bits that the last layer's weight gradient left, n*F/8 bytes)
+        per["aggregate_rank1"] = (n * d[L - 1] * b + n * d[L - 1] // 8 if b == 2 and d[L - 1] % 8 == 0
+                                  else 2 * n * d[L - 1] * b) + csr + 4 * n + S * d[L - 1] * b
         per["transform_fwd"] = np.mean([n * (d[l - 1] + d[l]) * b + S * d[l - 1] * d[l] * b for l in hidden])
         # input gradient: reads Q_l and the weights, writes n x d[l-1]; layers above the first also
         # read the saved activation (ReLU mask) and inv_deg
@@ -196,7 +198,7 @@ def algorithmic_bytes(kind, w, n, nnz, S):
         per["weight_grad"] = np.mean([n * (d[l - 1] + d[l]) * b + S * d[l - 1] * d[l] * 4 for l in hidden])
     F = d[L - 1]
     per["gemv"] = n * F * b + 4 * n + S * F * b
-    per["weight_grad_vec"] = n * F * b + 4 * n + S * F * 4
+    per["weight_grad_vec"] = n * F * b + 4 * n + S * F * 4 + (n * F // 8 if b == 2 and F % 8 == 0 and L > 1 else 0)
     per["rank1_masked"] = 2 * n * F * b + 4 * n
     per["output_forward"] = csr + 4 * n * 3
     per["objective"] = csr + 4 * n * 4
@@ -446,7 +448,6 @@ def run_ours(args):
 TRAFFIC_BYTES = {
     (5, "aggregate_fwd"): 10.03e9,
     (5, "aggregate_bwd"): 10.00e9,
-    (5, "aggregate_rank1"): 10.17e9,
     (5, "transform_fwd"): 10.49e9,
     (5, "transform_bwd"): 13.10e9,
 }

@@ -165,10 +165,14 @@ __global__ void __launch_bounds__(256) gemv_rows(const TA* __restrict__ H, const
 // table (a whole subgraph, or a run of rows of a very long one whose partial result goes to a
 // scratch slot and is combined in chunk order afterwards); LPR lanes cover a row with 16-byte
 // loads, the 256/LPR row groups walk the chunk's rows interleaved (four rows in flight each)
-// and meet in shared memory in a fixed order.
+// and meet in shared memory in a fixed order.  This pass reads every element of H exactly once,
+// so (bfloat16) it can leave [H > 0] behind as one bit per element (bits_out: element f of a row
+// = bit f%8 of byte f/8) for the rank-1 aggregation that follows, which then gathers 32 bytes
+// a row instead of 512.
 template <typename TA, int LPR>
 __global__ void __launch_bounds__(256) weight_grad_vec_rows(const TA* __restrict__ H, const float* __restrict__ g,
-                                                            float* __restrict__ dw, float* __restrict__ scratch, int F,
+                                                            float* __restrict__ dw, float* __restrict__ scratch,
+                                                            uint8_t* __restrict__ bits_out, int F,
                                                             const int32_t* __restrict__ wg_begin,
                                                             const int32_t* __restrict__ wg_end,
                                                             const int32_t* __restrict__ wg_slot) {
@@ -182,7 +186,24 @@ __global__ void __launch_bounds__(256) weight_grad_vec_rows(const TA* __restrict
   float acc[VN];
 #pragma unroll
   for (int e = 0; e < VN; ++e) acc[e] = 0.0f;
-  auto fma_row = [&](const uint4& v, float gi) {
+  auto fma_row = [&](const uint4& v, float gi, int64_t row) {
+    if (sizeof(TA) == 2 && bits_out) {
+      const uint32_t w[4] = {v.x, v.y, v.z, v.w};
+      uint32_t m = 0;
+#pragma unroll
+      for (int k = 0; k < 4; ++k) {
+        m |= (__uint_as_float(w[k] << 16) > 0.0f ? 1u : 0u) << (2 * k);
+        m |= (__uint_as_float(w[k] & 0xffff0000u) > 0.0f ? 1u : 0u) << (2 * k + 1);
+      }
+      if (LPR >= 32) {
+        // a row group is one or two whole warps here (uniform trip counts): four lanes' bytes in one word
+        m |= __shfl_down_sync(0xffffffffu, m, 1) << 8;
+        m |= __shfl_down_sync(0xffffffffu, m, 2) << 16;
+        if ((sub & 3) == 0) *reinterpret_cast<uint32_t*>(bits_out + row * (F >> 3) + sub) = m;
+      } else {
+        bits_out[row * (F >> 3) + sub] = (uint8_t)m;
+      }
+    }
     if (sizeof(TA) == 4) {
       acc[0] = fmaf(__uint_as_float(v.x), gi, acc[0]); acc[1] = fmaf(__uint_as_float(v.y), gi, acc[1]);
       acc[2] = fmaf(__uint_as_float(v.z), gi, acc[2]); acc[3] = fmaf(__uint_as_float(v.w), gi, acc[3]);
@@ -205,9 +226,9 @@ __global__ void __launch_bounds__(256) weight_grad_vec_rows(const TA* __restrict
       gi[u] = __ldg(g + i + u * RG);
     }
 #pragma unroll
-    for (int u = 0; u < 4; ++u) fma_row(v[u], gi[u]);
+    for (int u = 0; u < 4; ++u) fma_row(v[u], gi[u], i + u * RG);
   }
-  for (; i < rb; i += RG) fma_row(__ldg(reinterpret_cast<const uint4*>(H + i * F + sub * VN)), __ldg(g + i));
+  for (; i < rb; i += RG) fma_row(__ldg(reinterpret_cast<const uint4*>(H + i * F + sub * VN)), __ldg(g + i), i);
 #pragma unroll
   for (int e = 0; e < VN; ++e) partial[rg * F + sub * VN + e] = acc[e];
   __syncthreads();
@@ -435,17 +456,20 @@ int32_t launch_weight_grad(gnnco_handle* h, int dtype, const void* A, const void
 }
 
 int32_t launch_weight_grad_vec(gnnco_handle* h, int dtype, const void* H, const float* g, float* dw, float* scratch,
-                               int F, cudaStream_t stream) {
+                               int F, uint8_t* bits_out, bool* wrote_bits, cudaStream_t stream) {
   ProfScope prof_(h, K_WEIGHT_GRAD_VEC, stream);
+  if (wrote_bits) *wrote_bits = false;
   if (h->n_wg_slots > 0 && !scratch) return GNNCO_INTERNAL;
   const int vn = dtype == GNNCO_BF16 ? 8 : 4;
   const int lpr = F % vn == 0 ? F / vn : 0;
   const bool aligned = !((uintptr_t)H & 15);
   const size_t sm = (size_t)(lpr ? 256 / lpr : 0) * F * sizeof(float);
 #define GNNCO_WGV(TT, L)                                                                                     \
-  weight_grad_vec_rows<TT, L><<<h->n_wg_chunks, 256, sm, stream>>>((const TT*)H, g, dw, scratch, F, h->wg_begin, \
-                                                                   h->wg_end, h->wg_slot)
+  weight_grad_vec_rows<TT, L><<<h->n_wg_chunks, 256, sm, stream>>>((const TT*)H, g, dw, scratch, bits, F, \
+                                                                   h->wg_begin, h->wg_end, h->wg_slot)
   bool done = aligned && (lpr == 8 || lpr == 16 || lpr == 32 || lpr == 64);
+  uint8_t* bits = (done && dtype == GNNCO_BF16) ? bits_out : nullptr;   // every row is in exactly one chunk
+  if (bits && wrote_bits) *wrote_bits = true;
   if (done && dtype == GNNCO_F32) {
     if (lpr == 8) GNNCO_WGV(float, 8); else if (lpr == 16) GNNCO_WGV(float, 16);
     else if (lpr == 32) GNNCO_WGV(float, 32); else GNNCO_WGV(float, 64);

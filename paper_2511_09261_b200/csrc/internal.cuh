@@ -126,6 +126,10 @@ int32_t launch_aggregate(gnnco_handle* h, int dtype, const void* in, void* out, 
 // D^-1 (g w_s^T * [H > 0]) with coef = D^-1 g, gathered straight from the saved activation H
 int32_t launch_aggregate_rank1(gnnco_handle* h, int dtype, const void* H, const float* coef, const void* w,
                                int64_t w_stride, void* out, int F, cudaStream_t st);
+// the same from the bits [H > 0] (n x F/8 bytes, element f of a row = bit f%8 of byte f/8) instead of H
+bool aggregate_rank1_bits_supported(const gnnco_handle* h, int dtype, int F);
+int32_t launch_aggregate_rank1_bits(gnnco_handle* h, int dtype, const uint8_t* bits, const float* coef, const void* w,
+                                    int64_t w_stride, void* out, int F, cudaStream_t st);
 
 // ---- dense.cu
 // Y[tile rows x N] = act( A[rows x K] * B_s ), B_s = W[s] (K x N) or, with transB, W[s]^T where W[s] is (N x K);
@@ -139,9 +143,11 @@ int32_t launch_gemv(gnnco_handle* h, int dtype, const void* H, const void* w, in
 // dW[s] (K x N) = sum_{i in s} A[i,:]^T G[i,:]
 int32_t launch_weight_grad(gnnco_handle* h, int dtype, const void* A, const void* G, float* dW, int K, int N,
                            cudaStream_t st);
-// dw[s][f] = sum_{i in s} H[i,f] g[i]; scratch: F floats per slot of the weight-gradient chunk table
+// dw[s][f] = sum_{i in s} H[i,f] g[i]; scratch: F floats per slot of the weight-gradient chunk table.
+// bits_out (optional, n x F/8 bytes): receives [H > 0], one bit per element, when the kernel that runs
+// can produce it; *wrote_bits says whether it did.
 int32_t launch_weight_grad_vec(gnnco_handle* h, int dtype, const void* H, const float* g, float* dw, float* scratch,
-                               int F, cudaStream_t st);
+                               int F, uint8_t* bits_out, bool* wrote_bits, cudaStream_t st);
 // dZ[i,f] = g[i] * w_s[f] where H[i,f] > 0, else 0 (H == nullptr: no mask)
 int32_t launch_rank1_masked(gnnco_handle* h, int dtype, const float* g, const void* w, int64_t w_stride, const void* H,
                             void* dZ, int F, cudaStream_t st);

@@ -266,6 +266,128 @@ __global__ void __launch_bounds__(256) aggregate_vec(const T* __restrict__ in, T
   }
 }
 
+// Rank-1 mode from mask bits: the pass that reads H just before (the last layer's weight
+// gradient) can leave [H > 0] as one bit per element (element f of a row = bit f%8 of byte
+// f/8, F/8 bytes a row).  The gather then moves 1/16 (bfloat16) of the bytes of an activation
+// row.  Same sums in the same order as the activation-gathering mode.
+template <int VN>
+__device__ __forceinline__ void add_where_bits(float (&acc)[VN], uint32_t m, float c) {
+#pragma unroll
+  for (int e = 0; e < VN; ++e) acc[e] += ((m >> e) & 1u) ? c : 0.0f;
+}
+
+template <typename T, int LPR, int VPL>
+__global__ void __launch_bounds__(256) aggregate_rank1_bits(const uint8_t* __restrict__ bits, T* __restrict__ out,
+                                                            const int4* __restrict__ row_head,
+                                                            const int32_t* __restrict__ colidx,
+                                                            const Rank1Args<T> r1, int64_t n, int F,
+                                                            int prefetch_blocks) {
+  constexpr int VN = Vec<T>::N;
+  constexpr int ROWS_PER_BLOCK = 256 / LPR;
+  constexpr uint32_t PIECE = (1u << VN) - 1u;
+  const int sub = threadIdx.x % LPR;
+  const int64_t row = (int64_t)blockIdx.x * ROWS_PER_BLOCK + threadIdx.x / LPR;
+  const int64_t rb = F >> 3;                                   // bytes of bits per row
+  if (threadIdx.x == 0 && prefetch_blocks > 0) {               // see aggregate_vec
+    const int64_t r0 = ((int64_t)blockIdx.x + prefetch_blocks) * ROWS_PER_BLOCK;
+    if (r0 + ROWS_PER_BLOCK <= n) {
+      asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;" ::"l"(row_head + r0),
+                   "r"((uint32_t)(ROWS_PER_BLOCK * 16)) : "memory");
+      const uint8_t* b0 = bits + r0 * rb;
+      const uint32_t nb = (uint32_t)(ROWS_PER_BLOCK * rb);
+      if ((nb & 15u) == 0 && ((uintptr_t)b0 & 15) == 0)
+        asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;" ::"l"(b0), "r"(nb) : "memory");
+    }
+  }
+  if (row >= n) return;
+  // piece v of this lane: elements (v*LPR + sub)*VN .. +VN  ->  VN bits inside one byte
+  int byte_of[VPL], shift_of[VPL];
+#pragma unroll
+  for (int v = 0; v < VPL; ++v) {
+    const int off = (v * LPR + sub) * VN;
+    byte_of[v] = off >> 3;
+    shift_of[v] = off & 7;
+  }
+  uint32_t own[VPL];
+#pragma unroll
+  for (int v = 0; v < VPL; ++v) own[v] = __ldg(bits + row * rb + byte_of[v]);
+  const float c_own = __ldg(r1.coef + row);
+  const int32_t part = __ldg(r1.node_part + row);
+  const int4 head = __ldg(row_head + row);
+  const int32_t deg = head.y;
+  float acc[VPL][VN];
+  {
+    uint32_t t[2][VPL];
+    float c[2] = {0.0f, 0.0f};
+    if (deg > 0) {
+#pragma unroll
+      for (int v = 0; v < VPL; ++v) t[0][v] = __ldg(bits + (int64_t)head.z * rb + byte_of[v]);
+      c[0] = __ldg(r1.coef + head.z);
+    }
+    if (deg > 1) {
+#pragma unroll
+      for (int v = 0; v < VPL; ++v) t[1][v] = __ldg(bits + (int64_t)head.w * rb + byte_of[v]);
+      c[1] = __ldg(r1.coef + head.w);
+    }
+#pragma unroll
+    for (int v = 0; v < VPL; ++v) {
+#pragma unroll
+      for (int e = 0; e < VN; ++e) acc[v][e] = 0.0f;
+      add_where_bits<VN>(acc[v], (own[v] >> shift_of[v]) & PIECE, c_own);
+    }
+    if (deg > 0) {
+#pragma unroll
+      for (int v = 0; v < VPL; ++v) add_where_bits<VN>(acc[v], (t[0][v] >> shift_of[v]) & PIECE, c[0]);
+    }
+    if (deg > 1) {
+#pragma unroll
+      for (int v = 0; v < VPL; ++v) add_where_bits<VN>(acc[v], (t[1][v] >> shift_of[v]) & PIECE, c[1]);
+    }
+  }
+  // this lane's piece of the subgraph's weight vector, requested while the rest of the row is walked
+  uint4 wraw[VPL];
+  {
+    const T* wv = r1.w + (int64_t)part * r1.w_stride;
+#pragma unroll
+    for (int v = 0; v < VPL; ++v) wraw[v] = Vec<T>::load_raw(wv + (v * LPR + sub) * VN);
+  }
+  const int32_t r_end = head.x + deg;
+  int32_t k = head.x + 2;
+  constexpr int U = 8;                                         // neighbour rows in flight
+  for (; k + U <= r_end; k += U) {
+    int32_t j[U];
+#pragma unroll
+    for (int u = 0; u < U; ++u) j[u] = __ldg(colidx + k + u);
+    uint32_t t[U][VPL];
+    float c[U];
+#pragma unroll
+    for (int u = 0; u < U; ++u) {
+#pragma unroll
+      for (int v = 0; v < VPL; ++v) t[u][v] = __ldg(bits + (int64_t)j[u] * rb + byte_of[v]);
+      c[u] = __ldg(r1.coef + j[u]);
+    }
+#pragma unroll
+    for (int u = 0; u < U; ++u)
+#pragma unroll
+      for (int v = 0; v < VPL; ++v) add_where_bits<VN>(acc[v], (t[u][v] >> shift_of[v]) & PIECE, c[u]);
+  }
+  for (; k < r_end; ++k) {
+    const int64_t j = __ldg(colidx + k);
+    const float cj = __ldg(r1.coef + j);
+#pragma unroll
+    for (int v = 0; v < VPL; ++v)
+      add_where_bits<VN>(acc[v], ((uint32_t)__ldg(bits + j * rb + byte_of[v]) >> shift_of[v]) & PIECE, cj);
+  }
+#pragma unroll
+  for (int v = 0; v < VPL; ++v) {
+    float wf[VN];
+    Vec<T>::unpack(wraw[v], wf);
+#pragma unroll
+    for (int e = 0; e < VN; ++e) acc[v][e] *= wf[e];
+    Vec<T>::store(out + row * F + (v * LPR + sub) * VN, acc[v]);
+  }
+}
+
 // A row with more than kLongRowDegree neighbours: one block per row.  Each of the 8 warps sums
 // a contiguous eighth of the neighbour list with eight rows in flight, the partial sums
 // meet in shared memory in warp order (deterministic), and the block finishes the row.
@@ -521,4 +643,61 @@ int32_t launch_aggregate_rank1(gnnco_handle* h, int dtype, const void* H, const 
         h, (const __nv_bfloat16*)H, (__nv_bfloat16*)out, F, nullptr, nullptr,
         Rank1Args<__nv_bfloat16>{coef, (const __nv_bfloat16*)w, w_stride, h->node_part}, st);
   return GNNCO_UNSUPPORTED;
+}
+
+namespace {
+
+// The bit-gathering kernel walks every row inline, so it is used where the plain kernel would
+// do the same (no separate pass for long rows).
+bool rows_stay_inline(const gnnco_handle* h, int F, size_t elem) {
+  if (h->n_long == 0) return true;
+  const double stream_us = 2.0 * (double)h->n * F * elem / 4.0e6;
+  const double walk_us = (double)h->max_row / 4.0;
+  return stream_us > 3.0 * walk_us;
+}
+
+template <typename T>
+int32_t rank1_bits_typed(gnnco_handle* h, const uint8_t* bits, T* out, int F, const Rank1Args<T>& r1, cudaStream_t st) {
+  constexpr int VN = Vec<T>::N;
+  const int sms = h->sm_count > 0 ? h->sm_count : 148;
+#define GNNCO_R1B(LPR, VPL)                                                                                      \
+  do {                                                                                                           \
+    const unsigned blocks = (unsigned)((h->n + (256 / LPR) - 1) / (256 / LPR));                                  \
+    const int pf = blocks > 4u * 8u * (unsigned)sms ? 8 * sms : 0;                                               \
+    aggregate_rank1_bits<T, LPR, VPL><<<blocks, 256, 0, st>>>(bits, out, h->row_head, h->colidx, r1, h->n, F, pf); \
+  } while (0)
+  switch (F / VN) {
+    case 1: GNNCO_R1B(1, 1); break;
+    case 2: GNNCO_R1B(2, 1); break;
+    case 4: GNNCO_R1B(4, 1); break;
+    case 8: GNNCO_R1B(8, 1); break;
+    case 16: GNNCO_R1B(16, 1); break;
+    case 32: GNNCO_R1B(32, 1); break;
+    case 64: GNNCO_R1B(32, 2); break;
+    default: return GNNCO_UNSUPPORTED;
+  }
+#undef GNNCO_R1B
+  h->launches += 1;
+  GNNCO_LAUNCH_CHECK();
+  return GNNCO_OK;
+}
+
+}  // namespace
+
+bool aggregate_rank1_bits_supported(const gnnco_handle* h, int dtype, int F) {
+  if (dtype != GNNCO_BF16) return false;
+  if (F % 8) return false;
+  const int vecs = F / 8;
+  if (!(vecs == 1 || vecs == 2 || vecs == 4 || vecs == 8 || vecs == 16 || vecs == 32 || vecs == 64)) return false;
+  return rows_stay_inline(h, F, 2);
+}
+
+int32_t launch_aggregate_rank1_bits(gnnco_handle* h, int dtype, const uint8_t* bits, const float* coef, const void* w,
+                                    int64_t w_stride, void* out, int F, cudaStream_t st) {
+  if (!aggregate_rank1_bits_supported(h, dtype, F)) return GNNCO_UNSUPPORTED;
+  if (((uintptr_t)out & 15) || ((uintptr_t)w & 15) || (w_stride % 8)) return GNNCO_UNSUPPORTED;
+  ProfScope prof_(h, K_AGG_RANK1, st);
+  return rank1_bits_typed<__nv_bfloat16>(
+      h, bits, (__nv_bfloat16*)out, F,
+      Rank1Args<__nv_bfloat16>{coef, (const __nv_bfloat16*)w, w_stride, h->node_part}, st);
 }

@@ -32,6 +32,7 @@ struct TrainLayout {
   float* dW_sets;                     // per-subgraph partials when the model shares one weight set
   float* wg_scratch;                  // partial weight gradients of subgraphs that were split into row chunks
   float* agg_partial;                 // partial sums of the segments of long rows (aggregation)
+  uint8_t* Hbits;                     // [H_{L-1} > 0], one bit per element (bfloat16, written by the last layer's weight gradient)
   __nv_bfloat16* W_lp[GNNCO_MAX_LAYERS];   // bf16 copies of the weights (bf16 features only)
   __nv_bfloat16* W_lp_t[GNNCO_MAX_LAYERS]; // transposed bf16 copies [sets x F_out x F_in] for the tensor-core forward
   __nv_bfloat16* W3[GNNCO_MAX_LAYERS];     // float32 features: three bf16 limbs of W (input-gradient operand)
@@ -82,6 +83,8 @@ TrainLayout carve_train(const gnnco_handle* h, const gnnco_model_desc* m, uint32
   T.item_loss = c.take<float>((size_t)h->n_items + 1);
   T.agg_partial = h->n_long_segs > 0 ? c.take<float>((size_t)h->n_long_segs * maxw) : nullptr;
   if (!(flags & GNNCO_FORWARD_ONLY)) {
+    if (L > 1 && m->feat_dtype == GNNCO_BF16 && m->dims[L - 1] % 8 == 0)
+      T.Hbits = c.take<uint8_t>(n * (size_t)(m->dims[L - 1] / 8));
     if (L > 2) T.Gb = c.take<char>(n * maxw * es);
     T.dW_scratch = c.take<float>(max_wcount * m->weight_sets);
     if (m->weight_sets == 1) T.dW_sets = c.take<float>(max_wcount * (size_t)h->S);
@@ -196,14 +199,23 @@ int32_t run_step(gnnco_handle* h, const gnnco_model_desc* m, const void* X, cons
   {
     // last layer (0-based index L-1): dw = H^T g
     float* target = grad_target(L - 1);
+    bool have_bits = false;
     if (sets == 1) {
-      GNNCO_TRY(launch_weight_grad_vec(h, dt, Hprev, T.g, T.dW_sets, T.wg_scratch, FL, st));
+      GNNCO_TRY(launch_weight_grad_vec(h, dt, Hprev, T.g, T.dW_sets, T.wg_scratch, FL, T.Hbits, &have_bits, st));
       GNNCO_TRY(launch_sum_over_sets(h, T.dW_sets, target, FL, h->S, st));
     } else {
-      GNNCO_TRY(launch_weight_grad_vec(h, dt, Hprev, T.g, target, T.wg_scratch, FL, st));
+      GNNCO_TRY(launch_weight_grad_vec(h, dt, Hprev, T.g, target, T.wg_scratch, FL, T.Hbits, &have_bits, st));
     }
     // everything that reads the weights of a layer runs before that layer's Adam update
-    if (L > 1) GNNCO_TRY(launch_aggregate_rank1(h, dt, Hprev, T.u, Wc[L - 1], wstride[L - 1], Q, FL, st));
+    if (L > 1) {
+      // from the mask bits that the weight-gradient pass above left behind, where it could
+      const bool from_bits = have_bits && aggregate_rank1_bits_supported(h, dt, FL) &&
+                             !((uintptr_t)Wc[L - 1] & 15) && wstride[L - 1] % 8 == 0 && !((uintptr_t)Q & 15);
+      if (from_bits)
+        GNNCO_TRY(launch_aggregate_rank1_bits(h, dt, T.Hbits, T.u, Wc[L - 1], wstride[L - 1], Q, FL, st));
+      else
+        GNNCO_TRY(launch_aggregate_rank1(h, dt, Hprev, T.u, Wc[L - 1], wstride[L - 1], Q, FL, st));
+    }
     else if (flags & GNNCO_WANT_DX)
       // L == 1: dX = A_hat^T (dz w_s^T) and w_s is constant inside a subgraph, so dX[i,:] = g_i w_s^T
       GNNCO_TRY(launch_rank1_masked(h, dt, T.g, Wc[0], wstride[0], nullptr, out->dX, FL, st));
