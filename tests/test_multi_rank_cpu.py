@@ -27,7 +27,7 @@ def _worker(rank, world, port, out):
 
 def test_time_is_max_over_ranks_and_value_sums_replicas():
     world, port = 2, 29611
-    with mp.Manager() as mgr:
+    with mp.get_context("spawn").Manager() as mgr:       # never fork a process that already runs threads
         out = mgr.dict()
         mp.spawn(_worker, args=(world, port, out), nprocs=world, join=True)
         res = dict(out)
