@@ -145,6 +145,20 @@ def test_train_step_small_bf16(dims, sets):
     case.run(graph, X, W, pen, want_dx=True, adam=adam, label="bf16")
 
 
+@pytest.mark.parametrize("name,dims", [("big_hub", [64, 16, 1]), ("huge_hub", [128, 64, 1]), ("hub_and_isolated", [64, 64, 8, 1])])
+def test_train_step_bf16_with_hub_rows(name, dims):
+    """bfloat16 on graphs whose hub row goes through the block-per-segment aggregation (plain and
+    rank-1 mode) and the pre-summed long rows of the width-1 kernels."""
+    eu, ev, part = GRAPHS[name]()
+    n, S = _n_S(part)
+    book = oracle.bookkeeping(n, eu, ev, part, S)
+    graph = load_graph(n, eu, ev, part, S)
+    X = si.round_to_bf16(rand_features(n, dims[0], 11).astype(np.float32))
+    W = [si.round_to_bf16(w.astype(np.float32)) for w in rand_weights(dims, S, 13, scale=1.5)]
+    case = StepCase(book, dims, "bf16", S)
+    case.run(graph, X, W, None, want_dx=True, label=name + "-bf16")
+
+
 def test_forward_only_matches_full_step_and_skips_update():
     import torch
     import paper_2511_09261_b200 as gnnco
