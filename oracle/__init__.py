@@ -57,6 +57,8 @@ def _native():
         lib.oracle_partition_quality.restype = dbl
         lib.oracle_repair.argtypes = [i64, vp, vp]
         lib.oracle_repair.restype = i64
+        lib.oracle_round_bf16.argtypes = [dbl]
+        lib.oracle_round_bf16.restype = dbl
         _lib = lib
     return _lib
 
@@ -163,6 +165,12 @@ def train_step(book: Dict[str, np.ndarray], dims: Sequence[int], X, W: Sequence[
     if rc <= 0:
         raise OracleError(rc, "oracle_train_step")
     return dict(loss=loss, z=z, p=p, dW=dW, dX=dX, Z=Z, threads=rc)
+
+
+def round_bf16(x: float) -> float:
+    """The rounding that the bfloat16-storage mode applies to a stored value: double ->
+    nearest float -> nearest bfloat16 (ties to even both times), as a Python float."""
+    return float(_native().oracle_round_bf16(float(x)))
 
 
 def adam(W: np.ndarray, m: np.ndarray, v: np.ndarray, g: np.ndarray, lr: float, t: int, b1: float = 0.9,

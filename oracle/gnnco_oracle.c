@@ -16,7 +16,10 @@
  *
  * Pins (see tests, "not gpu"): finite differences for every gradient, closed forms at
  * W = 0, row-stochastic aggregation, per-subgraph runs equal the batched run, brute
- * force on graphs of at most 16 nodes, hand-computed Adam steps, brute-force decode.
+ * force on graphs of at most 16 nodes, hand-computed Adam steps, brute-force decode;
+ * the bfloat16-storage mode: exact rational rounding, a dense restatement with the rounding
+ * written out at the stored tensors, and bit-equality with the plain mode on inputs whose
+ * stored values are all bfloat16 numbers.
  * Parity unpinned: nothing here can be compared with the paper's result tables
  * (they need the original datasets, trained weights and the RL stage).
  */
@@ -41,8 +44,11 @@ static int cmp_pair(const void* a, const void* b) {
   return (x[1] > y[1]) - (x[1] < y[1]);
 }
 
-/* Round a double to the nearest-even bfloat16 value (via float), returned as double.
- * Used only where a workload fixes bfloat16 STORAGE of activations. */
+/* Round a double to bfloat16 the way a value that was accumulated in float32 and is then STORED
+ * in bfloat16 gets there: first to the nearest float (ties to even), then that float to the
+ * nearest bfloat16 (8 significant bits, float's exponent range; ties to even; overflow gives
+ * infinity), returned as double.  Used only where a workload fixes bfloat16 storage of
+ * activations with float32 accumulation. */
 static double round_bf16(double x) {
   float f = (float)x;
   uint32_t u;
@@ -53,6 +59,9 @@ static double round_bf16(double x) {
   memcpy(&f, &u, 4);
   return (double)f;
 }
+
+/* round_bf16 for the pins (exact rational arithmetic checks it from outside). */
+double oracle_round_bf16(double x) { return round_bf16(x); }
 
 /*
  * Bookkeeping (Section 3.3, first paragraph: the graph is split into subgraphs, and

@@ -46,6 +46,17 @@ MUTATIONS = {
     "repair counts chosen nodes that were not selected": ("if (pen[i] != 0.0f && x[i]) {", "if (pen[i] != 0.0f) {"),
     "modularity counts internal edges once": ("q += 2.0 * (double)in_edges[s] / two_m - share * share;", "q += (double)in_edges[s] / two_m - share * share;"),
     "degree sum misses the second endpoint": ("    tot[a] += 1;\n    tot[b] += 1;", "    tot[a] += 1;"),
+    "bf16 storage truncates instead of rounding to nearest": ("u += 0x7FFFu + ((u >> 16) & 1u);", ";"),
+    "bf16 storage rounds ties away from zero": ("u += 0x7FFFu + ((u >> 16) & 1u);", "u += 0x8000u;"),
+    "bf16 storage rounds the double directly (one rounding)":
+        ("  float f = (float)x;\n  uint32_t u;\n  memcpy(&u, &f, 4);\n  if ((u & 0x7F800000u) == 0x7F800000u) return (double)f;",
+         "  float f = (float)x;\n  uint32_t u;\n  memcpy(&u, &f, 4);\n  if ((u & 0x7F800000u) == 0x7F800000u) return (double)f;\n"
+         "  if ((u & 0xFFFFu) == 0x8000u && (double)f != x) u += (fabs(x) > fabs((double)f)) ? 1u : 0xFFFFFFFFu;"),
+    "bf16 storage leaves the aggregated input unrounded":
+        ("if (store_bf16 && l < L)\n        for (int32_t f = 0; f < fi; ++f) m[f] = round_bf16(m[f]);", ";"),
+    "bf16 storage also rounds the output layer's aggregate": ("if (store_bf16 && l < L)", "if (store_bf16)"),
+    "bf16 storage leaves the activation unrounded":
+        ("if (store_bf16)\n          for (int32_t h = 0; h < fo; ++h) hr[h] = round_bf16(hr[h]);", ";"),
     "inv_deg without the +1": ("inv_deg[i] = 1.0f / (float)(hi - lo + 1);", "inv_deg[i] = 1.0f / (float)(hi - lo > 0 ? hi - lo : 1);"),
 }
 
@@ -69,6 +80,11 @@ BATTERY = [
     lambda: pins.test_conflict_list_base_action_and_penalty_brute_force(2),
     lambda: pins.test_repair_removes_exactly_the_chosen_nodes_brute_force(1),
     lambda: pins.test_partition_quality_matches_networkx_and_the_pairwise_definition(30, 0.2, 4, 1),
+    pins.test_round_bf16_is_exact_round_to_nearest_even,
+    lambda: pins.test_bf16_storage_forward_matches_dense_definition_with_rounding_written_out([7, 5, 3, 1], False),
+    pins.test_bf16_storage_hidden_preactivations_and_output_layer_keep_full_precision,
+    pins.test_bf16_storage_mode_is_a_no_op_when_every_stored_value_is_a_bf16_number,
+    pins.test_bf16_storage_gradients_are_those_of_the_rounded_forward_values,
 ]
 
 
@@ -84,7 +100,8 @@ def test_a_pin_fails_when_the_oracle_is_mutated(name, tmp_path, monkeypatch):
     real = oracle._native()
     mutant = ctypes.CDLL(lib_path)
     for fn in ("oracle_bookkeeping", "oracle_subgraph_step", "oracle_train_step", "oracle_adam", "oracle_decode",
-               "oracle_conflict_list", "oracle_base_action", "oracle_apply_actions", "oracle_repair", "oracle_partition_quality"):
+               "oracle_conflict_list", "oracle_base_action", "oracle_apply_actions", "oracle_repair", "oracle_partition_quality",
+               "oracle_round_bf16"):
         getattr(mutant, fn).argtypes = getattr(real, fn).argtypes
         getattr(mutant, fn).restype = getattr(real, fn).restype
     monkeypatch.setattr(oracle, "_lib", mutant)

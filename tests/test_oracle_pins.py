@@ -430,6 +430,193 @@ def test_sigmoid_chain_identity_for_one_layer():
     np.testing.assert_allclose(r["dW"][0][0][:, 0], X.T @ Ahat.T @ dz, rtol=1e-11, atol=1e-13)
 
 
+# ------------------------------------------------- bfloat16-storage mode of the oracle
+def _exact_bf16_of_float32(f):
+    """Nearest bfloat16 (8 significant bits, float32's exponent range, ties to even, overflow
+    to infinity) of a finite float32, in exact rational arithmetic."""
+    x = Fraction(float(f))
+    if x == 0:
+        return float(f)                                         # keeps the sign of zero
+    a = abs(x)
+    e = 0
+    while Fraction(2) ** (e + 1) <= a:
+        e += 1
+    while Fraction(2) ** e > a:
+        e -= 1
+    q = Fraction(2) ** (max(e, -126) - 7)                       # spacing of bfloat16 numbers around a
+    k = a / q
+    lo = k.numerator // k.denominator
+    rem = k - lo
+    if rem > Fraction(1, 2) or (rem == Fraction(1, 2) and lo % 2 == 1):
+        lo += 1
+    r = lo * q
+    if r >= Fraction(2) ** 128:
+        return float("inf") if x > 0 else float("-inf")
+    return float(r) if x > 0 else -float(r)
+
+
+def test_round_bf16_is_exact_round_to_nearest_even():
+    vals = []
+    for base in (1.0, 2.0, 0.75, 3.0e-5, 1.0e20, 2.0 ** -126, 2.0 ** -130, 2.0 ** 127):
+        ulp = 2.0 ** (int(np.floor(np.log2(base))) - 7)
+        for k in range(0, 9):
+            for tweak in (0.0, 2.0 ** -20, -(2.0 ** -20)):
+                # k/4 of a bfloat16 spacing above a bfloat16 number: k = 2, 6 are exact ties with an even
+                # and an odd neighbour below; the tweaks fall just off the ties on either side
+                vals.append(base + ulp * (k / 4.0) * (1.0 + tweak))
+    vals += [2.0 - 2.0 ** -9, 2.0 - 2.0 ** -8, 4.0 - 2.0 ** -8, 2.0 ** -133, 2.0 ** -134, 1.5 * 2.0 ** -133, 3.0 * 2.0 ** -134,
+             3.3895313892515355e38, 3.3961775292304601e38, 3.4028234663852886e38, 0.0, -0.0]
+    vals += si.normal_f32(4242, 0, 400).astype(np.float64).tolist()
+    vals += (si.normal_f32(4243, 0, 200).astype(np.float64) * 1e-39).tolist()      # float32 subnormals
+    for v in vals:
+        for x in (v, -v):
+            f = np.float32(x)                                     # IEEE round-to-nearest-even to float32
+            want = _exact_bf16_of_float32(f)
+            got = oracle.round_bf16(x)
+            assert got == want and np.signbit(got) == np.signbit(want), (x, got, want)
+    assert oracle.round_bf16(float("inf")) == float("inf") and oracle.round_bf16(float("-inf")) == float("-inf")
+    assert np.isnan(oracle.round_bf16(float("nan")))
+    # two roundings, not one: a double just above a bfloat16 tie first becomes the tie (as float32)
+    assert oracle.round_bf16(1.0 + 2.0 ** -8 + 2.0 ** -40) == 1.0
+    # every bfloat16 number is a fixed point
+    for v in (1.0, 1.0078125, -3.5, 2.0 ** -133, 255.0, 0.00390625):
+        assert oracle.round_bf16(v) == v
+
+
+def _bf16_lib(a):
+    """Library rounding float64 -> float32 -> bfloat16 (torch's conversion routines)."""
+    import torch
+    return torch.from_numpy(np.ascontiguousarray(a, dtype=np.float64)).to(torch.float32).to(torch.bfloat16).to(
+        torch.float64).numpy()
+
+
+def _dense_forward_loss_bf16_storage(n, eu, ev, part, dims, X, W, pen, lam):
+    """The dense restatement of Eqs. 3-5 with the two tensors that a bfloat16 run STORES per hidden
+    layer -- the aggregated input M_l and the activation H_l -- rounded to bfloat16; the output
+    layer's aggregate, z, p and the loss stay in double."""
+    A = dense_intra_adjacency(n, eu, ev, part)
+    Ahat = (A + np.eye(n)) / (A.sum(1) + 1.0)[:, None]
+    H = X
+    L = len(dims) - 1
+    for l in range(L):
+        M = Ahat @ H
+        if l < L - 1:
+            M = _bf16_lib(M)
+        Z = np.stack([M[i] @ W[l][part[i] if W[l].shape[0] > 1 else 0] for i in range(n)])
+        H = _bf16_lib(np.maximum(Z, 0.0)) if l < L - 1 else Z
+    z = H[:, 0]
+    p = 1.0 / (1.0 + np.exp(-z))
+    S = int(part.max()) + 1
+    loss = np.zeros(S)
+    for s in range(S):
+        ps = p * (part == s)
+        loss[s] = ALPHA * 0.5 * ps @ A @ ps - BETA * ps.sum() + lam * (pen * ps).sum()
+    return z, p, loss
+
+
+@pytest.mark.parametrize("dims,sets_shared", [([6, 4, 1], False), ([7, 5, 3, 1], False), ([7, 5, 3, 1], True)])
+def test_bf16_storage_forward_matches_dense_definition_with_rounding_written_out(dims, sets_shared):
+    n, S = 40, 4
+    eu, ev, part = tiny_graph(n, 0.25, S, seed=11)
+    b = oracle.bookkeeping(n, eu, ev, part, S)
+    X = si.round_to_bf16(rand_features(n, dims[0], 5).astype(np.float32)).astype(np.float64)
+    W = [si.round_to_bf16(w.astype(np.float32)).astype(np.float64)
+         for w in rand_weights(dims, 1 if sets_shared else S, 7, scale=2.0)]
+    pen = (si.uniform01(99, 0, n) < 0.3).astype(np.float64)
+    z, p, loss = _dense_forward_loss_bf16_storage(n, eu, ev, part, dims, X, W, pen, 0.7)
+    r = oracle.train_step(b, dims, X[b["perm"]], W, ALPHA, BETA, 0.7, pen[b["perm"]], store_bf16=True)
+    # sums of a handful of double products in a different order: a few ulps of double, far below the
+    # 2^-9 relative size of one bfloat16 rounding (a missing or an extra rounding shows at ~1e-3)
+    np.testing.assert_allclose(r["z"], z[b["perm"]], rtol=1e-11, atol=1e-12)
+    np.testing.assert_allclose(r["p"], p[b["perm"]], rtol=1e-11, atol=1e-12)
+    np.testing.assert_allclose(r["loss"], loss, rtol=1e-11, atol=1e-11)
+    # and the mode does change the result on such inputs (otherwise the check above says nothing)
+    plain = oracle.train_step(b, dims, X[b["perm"]], W, ALPHA, BETA, 0.7, pen[b["perm"]], store_bf16=False)
+    assert np.abs(plain["z"] - r["z"]).max() > 1e-5
+
+
+def test_bf16_storage_hidden_preactivations_and_output_layer_keep_full_precision():
+    # what is rounded is what is stored: Z_l (never stored) is the double product of the ROUNDED M_l,
+    # and the last layer's aggregate is not rounded
+    n, S, dims = 30, 3, [5, 4, 1]
+    eu, ev, part = tiny_graph(n, 0.3, S, seed=17)
+    b = oracle.bookkeeping(n, eu, ev, part, S)
+    perm = b["perm"]
+    X = si.round_to_bf16(rand_features(n, dims[0], 8).astype(np.float32)).astype(np.float64)
+    W = [si.round_to_bf16(w.astype(np.float32)).astype(np.float64) for w in rand_weights(dims, S, 9, scale=2.0)]
+    r = oracle.train_step(b, dims, X[perm], W, ALPHA, BETA, want_Z=True, store_bf16=True)
+    A = dense_intra_adjacency(n, eu, ev, part)
+    Ahat = (A + np.eye(n)) / (A.sum(1) + 1.0)[:, None]
+    M1 = _bf16_lib(Ahat @ X)
+    Z1 = np.stack([M1[i] @ W[0][part[i]] for i in range(n)])
+    np.testing.assert_allclose(r["Z"][0], Z1[perm], rtol=1e-12, atol=1e-13)
+    H1 = _bf16_lib(np.maximum(Z1, 0.0))
+    M2 = Ahat @ H1                                               # output layer: not rounded
+    z = np.array([M2[i] @ W[1][part[i]][:, 0] for i in range(n)])
+    np.testing.assert_allclose(r["z"], z[perm], rtol=1e-12, atol=1e-13)
+    assert np.abs(_bf16_lib(M2) - M2).max() > 1e-4               # rounding M2 would have been visible
+
+
+def test_bf16_storage_mode_is_a_no_op_when_every_stored_value_is_a_bf16_number():
+    # degrees 0, 1 and 3 (means divide by 1, 2, 4), small integer features, weights in {-1, 0, 1} with a
+    # signed permutation in the second layer: every M_l and H_l is a multiple of 1/16 below 2^4, i.e.
+    # a bfloat16 number, so the two modes must agree bit for bit -- loss, p and every gradient
+    n, S, dims = 24, 2, [4, 4, 4, 1]
+    edges = [(0, 1), (2, 3), (4, 5), (4, 6), (4, 7), (5, 6), (5, 7), (6, 7),          # part 0: pairs and a K4
+             (12, 13), (14, 15), (16, 17), (16, 18), (16, 19), (17, 18), (17, 19), (18, 19), (20, 21)]
+    eu = np.array([a for a, _ in edges], np.int32)
+    ev = np.array([c for _, c in edges], np.int32)
+    part = (np.arange(n) >= 12).astype(np.int32)
+    b = oracle.bookkeeping(n, eu, ev, part, S)
+    assert set(np.diff(b["rowptr"]).tolist()) == {0, 1, 3}
+    X = (si.u64(5, 0, n * 4) % np.uint64(5)).astype(np.float64).reshape(n, 4) - 2.0
+    W0 = (si.u64(6, 0, S * 16) % np.uint64(3)).astype(np.float64).reshape(S, 4, 4) - 1.0
+    P = np.zeros((S, 4, 4))
+    for s in range(S):
+        for k, (j, sign) in enumerate(zip([2, 0, 3, 1], [1.0, -1.0, 1.0, 1.0])):
+            P[s, k, (j + s) % 4] = sign
+    W2 = (si.u64(7, 0, S * 4) % np.uint64(3)).astype(np.float64).reshape(S, 4, 1) - 1.0
+    W = [W0, P, W2]
+    a = oracle.train_step(b, dims, X, W, ALPHA, BETA, want_dX=True, want_Z=True, store_bf16=False)
+    c = oracle.train_step(b, dims, X, W, ALPHA, BETA, want_dX=True, want_Z=True, store_bf16=True)
+    assert np.abs(a["Z"][0]).max() > 0 and (a["Z"][1] > 0).any()
+    for key in ("loss", "p", "z", "dX"):
+        assert np.array_equal(a[key], c[key]), key
+    for l in range(3):
+        assert np.array_equal(a["dW"][l], c["dW"][l])
+        if l < 2:
+            assert np.array_equal(a["Z"][l], c["Z"][l])
+
+
+def test_bf16_storage_gradients_are_those_of_the_rounded_forward_values():
+    # The backward pass of the bfloat16 mode is the exact derivative taken AT the stored values
+    # (straight-through: the rounding itself has no derivative).  With one hidden layer,
+    #   dW_2 = (A_hat H_1)^T dz       with H_1 the rounded activation,
+    #   dW_1 = M_1^T ((A_hat^T dz w_2^T) * [Z_1 > 0])   with M_1 the rounded aggregate.
+    n, S, dims = 36, 3, [5, 4, 1]
+    eu, ev, part = tiny_graph(n, 0.25, S, seed=23)
+    b = oracle.bookkeeping(n, eu, ev, part, S)
+    perm = b["perm"]
+    X = si.round_to_bf16(rand_features(n, dims[0], 2).astype(np.float32)).astype(np.float64)
+    W = [si.round_to_bf16(w.astype(np.float32)).astype(np.float64) for w in rand_weights(dims, S, 3, scale=2.0)]
+    r = oracle.train_step(b, dims, X[perm], W, ALPHA, BETA, store_bf16=True)
+    A = dense_intra_adjacency(n, eu, ev, part)
+    Ahat = (A + np.eye(n)) / (A.sum(1) + 1.0)[:, None]
+    M1 = _bf16_lib(Ahat @ X)
+    Z1 = np.stack([M1[i] @ W[0][part[i]] for i in range(n)])
+    H1 = _bf16_lib(np.maximum(Z1, 0.0))
+    M2 = Ahat @ H1
+    z = np.array([M2[i] @ W[1][part[i]][:, 0] for i in range(n)])
+    p = 1.0 / (1.0 + np.exp(-z))
+    dz = (ALPHA * (A @ p) - BETA) * p * (1 - p)
+    g = Ahat.T @ dz
+    for s in range(S):
+        msk = part == s
+        np.testing.assert_allclose(r["dW"][1][s][:, 0], M2[msk].T @ dz[msk], rtol=1e-10, atol=1e-12)
+        dZ1 = np.outer(g[msk], W[1][s][:, 0]) * (Z1[msk] > 0)
+        np.testing.assert_allclose(r["dW"][0][s], M1[msk].T @ dZ1, rtol=1e-10, atol=1e-12)
+
+
 # ----------------------------------------------------------- block-diagonal batch pin
 def test_batch_equals_independent_subgraph_runs_bit_for_bit():
     n, S, dims = 90, 6, [6, 5, 4, 1]
