@@ -2,7 +2,7 @@
  * gnnco -- partitioned-GNN training step for combinatorial optimisation on one GPU.
  *
  * C ABI of the CUDA library.  The calls follow the problem statement of the method
- * (Algorithm 1: inputs "graph G, subgraph set {G_i}, QUBO Q", output "bitstring x"):
+ * (Algorithm 1 takes the graph G, its subgraphs {G_i} and the QUBO matrix Q and returns a bit string x):
  *
  *   gnnco_partition_load   graph + partition  -> block-diagonal batch of subgraphs
  *                          (Section 3.3, first paragraph; Algorithm 1, Stage 2 masks)
@@ -53,8 +53,8 @@ typedef enum { GNNCO_F32 = 0, GNNCO_BF16 = 1 } gnnco_dtype;
 
 /* flags of gnnco_train_step */
 #define GNNCO_WANT_DX 1u        /* also compute d loss / d X (runs the transposed aggregation of layer 1) */
-#define GNNCO_FORWARD_ONLY 2u   /* stop after loss and p (Algorithm 1, Stage 2: "run forward to get p_i") */
-/* The embeddings X are fixed inputs (Section 3.2 updates "the weight matrix W" only), so the
+#define GNNCO_FORWARD_ONLY 2u   /* stop after loss and p (Algorithm 1, Stage 2 needs one forward pass per subgraph) */
+/* The embeddings X are fixed inputs (Section 3.2 updates the weights W only), so the
  * first layer's aggregated input  mean_{self + intra neighbours}(X)  of Eq. 3 is the same in
  * every step of a run.  With GNNCO_AX_STORE the step keeps it in gnnco_train_out.ax_cache;
  * with GNNCO_AX_REUSE the step skips that aggregation and reads ax_cache instead (the caller
@@ -230,9 +230,10 @@ int32_t gnnco_decode_boundary(const gnnco_handle* h, const float* p, float thres
  *                violated edges, ASCENDING; only the first *count entries are written
  *   action       [E_b] uint8 (capacity) or NULL: for conflict c on the stored pair (u, v),
  *                u < v in the new order, 0 = push u below the threshold, 1 = push v.
- *                Section 3.3 gives every conflict exactly these two options; the base action
- *                ("initialize agent base action", not defined further by the paper) takes
- *                the endpoint with the SMALLER probability p, and v when they are equal.
+ *                Section 3.3 gives every conflict exactly these two options.  Algorithm 1,
+ *                Stage 3 starts the agent from a base action obtained with a cover heuristic
+ *                that it does not spell out; this library SUBSTITUTES a rule of its own for
+ *                it: the endpoint with the SMALLER probability p, and v when they are equal.
  *   count        device int32: |C|
  * viol [E_b] uint8 and p [n] float32 (new order) are inputs; p may be NULL iff action is.
  * ws must hold gnnco_conflict_workspace_bytes bytes.  Asynchronous on `stream`; no host
@@ -247,8 +248,8 @@ int32_t gnnco_decode_boundary(const gnnco_handle* h, const float* p, float thres
  * from the caller's own policy (any 0/1 vector of that length).  Asynchronous on `stream`. */
 /*
  * gnnco_repair_boundary carries the chosen actions out on the mask itself, without any
- * fine-tuning -- the non-learned baseline of Stage 3 (Section 3.3: an action "directly eliminates
- * the conflict by removing node i from the candidate set"):  x[i] <- 0 for every chosen node
+ * fine-tuning -- the non-learned baseline of Stage 3 (Section 3.3: acting on a conflict takes
+ * one of its two endpoints out of the candidate set):  x[i] <- 0 for every chosen node
  * (pen[i] != 0, the vector written by gnnco_apply_actions).  Afterwards no boundary edge has both
  * ends selected; intra-subgraph conflicts are not touched.  removed (device int32, or NULL)
  * receives the number of selected nodes that were cleared.  Asynchronous on `stream`. */
@@ -259,8 +260,8 @@ int32_t gnnco_conflict_actions(gnnco_handle* h, const uint8_t* viol, const float
 int32_t gnnco_apply_actions(gnnco_handle* h, const int32_t* conflict_idx, const uint8_t* action,
                             const int32_t* count, float* pen, uint8_t* active, int32_t* chosen, void* stream);
 
-/* Input embeddings (Section 3.2, "Subgraph training": "node embeddings are initialized as random
- * vectors ... processed using the Gumbel-softmax trick").
+/* Input embeddings (Section 3.2, subgraph training: the random initial node embeddings go
+ * through a Gumbel-softmax before the first layer).
  *
  * gnnco_gumbel_softmax: X[i,:] = softmax( (E[i,:] + g[i,:]) / tau ) over the F features of node i,
  * with Gumbel noise g = -log(-log U) from uniforms U in (0, 1), exclusive, that the caller draws
@@ -303,8 +304,9 @@ int32_t gnnco_embedding_update(gnnco_handle* h, int32_t feat_dtype, int32_t F, c
  *  - All calls share the one array and it keeps what the last call left: the part a call
  *    uses is cleared and rewritten by that call, but two calls that overlap on the GPU
  *    (different streams, or another thread) race on it.  Serialise them.
- *  - The handle's device must be current.  Asynchronous on `stream`; results equal those of
- *    gnnco_train_step's loss for the same p.
+ *  - The handle's device must be current.  Asynchronous on `stream`.  Results equal
+ *    gnnco_train_step's loss for the same p to float32 rounding, and bit for bit when no row has
+ *    more than 256 intra neighbours (longer rows are summed in another order here).
  */
 #define GNNCO_STATIC_OBJECTIVE_MAX_ITEMS 65536
 int32_t gnnco_objective_static(gnnco_handle* h, const float* p, const gnnco_objective* obj, float* loss,

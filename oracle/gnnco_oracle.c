@@ -9,8 +9,8 @@
  * Conventions
  *   - nodes are renumbered so that each subgraph (partition) is a contiguous id range;
  *     `part_ptr[s] .. part_ptr[s+1]` is subgraph s;
- *   - only intra-subgraph edges take part in training (Section 3.3: subgraphs are
- *     trained "without cross-subgraph interference"); cross edges are kept aside as
+ *   - only intra-subgraph edges take part in training (Section 3.3: each subgraph is
+ *     trained on its own, edges to other subgraphs play no part); cross edges are kept aside as
  *     the boundary list that decoding inspects;
  *   - dense matrices are row-major.
  *
@@ -391,8 +391,8 @@ int oracle_train_step(int64_t n, int32_t S, const int32_t* part_ptr, const int32
 }
 
 /*
- * Adam with bias correction (the paper names no optimiser beyond "backpropagation is
- * performed to update the weight matrix W", Section 3.2; the benchmark configurations
+ * Adam with bias correction (Section 3.2 only says that W is updated by backpropagation
+ * and names no optimiser; the benchmark configurations
  * fix Adam).  t is the 1-based step number.
  *   m <- b1 m + (1-b1) g;  v <- b2 v + (1-b2) g^2
  *   W <- W - lr * (m / (1-b1^t)) / (sqrt(v / (1-b2^t)) + eps)
@@ -408,9 +408,8 @@ void oracle_adam(int64_t count, double* W, double* m, double* v, const double* g
 }
 
 /*
- * Decoding and conflict counting (Section 3.3: probabilities are binarised with
- * "1 if prob >= 0.5, 0 otherwise"; a cross edge whose two endpoints are both selected
- * is a conflict; Section 4.1: MIS size and conflicts are the reported metrics).
+ * Decoding and conflict counting (Section 3.3: a probability of at least 0.5 becomes one, anything
+ * below zero; a cross edge whose two endpoints are both selected is a conflict; Section 4.1: MIS size and conflicts are the reported metrics).
  *   x[i]        = p[i] >= threshold   (compared on the stored float value)
  *   viol[e]     = x[bnd_u[e]] & x[bnd_v[e]]
  *   per_part[s] = number of violated boundary edges with an endpoint in s (an edge
@@ -447,7 +446,7 @@ void oracle_decode(int64_t n, int32_t S, const int32_t* node_part, const int32_t
  * Stage-3 glue (Algorithm 1, Stage 3, first lines; Section 3.3).
  *
  * Conflict list: the boundary edges whose two endpoints are both selected, as ascending
- * indices into the boundary list ("compute conflict edges from m"; the set C of Section 3.3).
+ * indices into the boundary list (Algorithm 1, Stage 3 derives them from the global mask; the set C of Section 3.3).
  * Returns their number.
  */
 int64_t oracle_conflict_list(int64_t E_b, const uint8_t* viol, int32_t* conflict_idx) {
@@ -458,8 +457,8 @@ int64_t oracle_conflict_list(int64_t E_b, const uint8_t* viol, int32_t* conflict
 }
 
 /*
- * Base action (Algorithm 1: "initialize agent base action"; the paper does not say how).
- * Reading taken: for every conflict edge (u, v) the endpoint with the SMALLER probability is
+ * Base action (Algorithm 1, Stage 3 starts the agent from one, obtained with a cover heuristic it
+ * does not spell out).  A rule of this build's own stands in for it: for every conflict edge (u, v) the endpoint with the SMALLER probability is
  * the one to push below the threshold; on equal probabilities the endpoint with the larger
  * id.  action = 0 chooses u (the lower id of the stored pair), 1 chooses v.  Every conflict
  * loses one endpoint, so removing all chosen nodes leaves no violated boundary edge.
@@ -475,7 +474,7 @@ void oracle_base_action(int64_t count, const int32_t* conflict_idx, const int32_
 /*
  * Actions -> fine-tuning inputs (Section 3.3: each conflict offers two options, fine-tune the
  * subgraph of node i or of node j so that this node's probability falls below the threshold;
- * Algorithm 1: "group actions per subgraph").  pen[i] = 1 for every chosen node (the node
+ * Algorithm 1, Stage 3 then groups the actions by subgraph).  pen[i] = 1 for every chosen node (the node
  * list of the penalty term), 0 elsewhere; active[s] = 1 for every subgraph that holds a chosen
  * node (the subgraphs whose models are fine-tuned).  Returns the number of distinct chosen nodes.
  */
@@ -495,9 +494,8 @@ int64_t oracle_apply_actions(int64_t n, int32_t S, int64_t count, const int32_t*
 }
 
 /*
- * Non-learned repair (Section 3.3: an action on conflict (i, j) "directly eliminates the conflict
- * by removing node i [or j] from the candidate set"; Algorithm 1, Stage 3 starts from a base
- * action).  Carrying the chosen actions out on the bit mask itself, without fine-tuning:
+ * Non-learned repair (Section 3.3: acting on conflict (i, j) takes node i, or node j, out of the
+ * candidate set and so removes the conflict; Algorithm 1, Stage 3 starts from a base action).  Carrying the chosen actions out on the bit mask itself, without fine-tuning:
  * x[i] <- 0 for every chosen node i (pen[i] != 0).  Returns how many selected nodes were removed.
  */
 int64_t oracle_repair(int64_t n, const float* pen, uint8_t* x) {

@@ -4,16 +4,18 @@ from __future__ import annotations
 import glob
 import os
 import subprocess
+from concurrent.futures import ThreadPoolExecutor
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
 _ROOT = os.path.dirname(_HERE)
 LIB_PATH = os.path.join(_HERE, "libgnnco.so")
+OBJ_DIR = os.path.join(_HERE, "_build")
 SOURCES = sorted(glob.glob(os.path.join(_HERE, "csrc", "*.cu")))
 HEADERS = sorted(glob.glob(os.path.join(_HERE, "csrc", "*.cuh"))) + [os.path.join(_ROOT, "include", "gnnco.h")]
 
 NVCC_FLAGS = [
     "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
-    "-Xcompiler", "-fPIC", "-shared", "--use_fast_math=false",
+    "-Xcompiler", "-fPIC",
 ]
 
 
@@ -31,17 +33,31 @@ def needs_build() -> bool:
     return any(os.path.getmtime(f) > t for f in SOURCES + HEADERS)
 
 
+def _object_of(src: str) -> str:
+    return os.path.join(OBJ_DIR, os.path.splitext(os.path.basename(src))[0] + ".o")
+
+
 def build(force: bool = False, verbose: bool = False) -> str:
-    """Compile every .cu under csrc/ into one shared library next to this file."""
+    """Compile every .cu under csrc/ (one nvcc process per file, in parallel; a file is recompiled
+    when it or any header is newer than its object) and link them into one shared library next to
+    this file."""
     if not force and not needs_build():
         return LIB_PATH
-    flags = [f for f in NVCC_FLAGS if f != "--use_fast_math=false"]
+    os.makedirs(OBJ_DIR, exist_ok=True)
+    newest_header = max(os.path.getmtime(f) for f in HEADERS)
+    include = ["-I", os.path.join(_ROOT, "include"), "-I", os.path.join(_HERE, "csrc")]
+
+    def compile_one(src: str) -> str:
+        obj = _object_of(src)
+        if force or not os.path.exists(obj) or os.path.getmtime(obj) < max(os.path.getmtime(src), newest_header):
+            cmd = [_nvcc()] + NVCC_FLAGS + (["-Xptxas=-v"] if verbose else []) + include + ["-c", "-o", obj, src]
+            subprocess.check_call(cmd)
+        return obj
+
+    with ThreadPoolExecutor(max_workers=min(len(SOURCES), os.cpu_count() or 4)) as pool:
+        objects = list(pool.map(compile_one, SOURCES))
     tmp = LIB_PATH + ".tmp%d" % os.getpid()
-    cmd = [_nvcc()] + flags + ["-I", os.path.join(_ROOT, "include"), "-I", os.path.join(_HERE, "csrc"),
-                               "-o", tmp] + SOURCES
-    if verbose:
-        cmd.insert(1, "-Xptxas=-v")
-    subprocess.check_call(cmd)
+    subprocess.check_call([_nvcc(), "-gencode", "arch=compute_100a,code=sm_100a", "-shared", "-o", tmp] + objects)
     os.replace(tmp, LIB_PATH)
     return LIB_PATH
 

@@ -1,6 +1,6 @@
-// Input embeddings (Section 3.2, "Subgraph training", first paragraph): node embeddings are
-// random vectors that are "processed using the Gumbel-softmax trick" before they enter the
-// GCN layer of Eq. 3.  Two entry points:
+// Input embeddings (Section 3.2, first paragraph on subgraph training): node embeddings start
+// as random vectors and pass through a Gumbel-softmax before they enter the GCN layer of
+// Eq. 3.  Two entry points:
 //
 //   gnnco_gumbel_softmax     x_i = softmax( (e_i + g_i) / tau ),  g = -log(-log u)
 //   gnnco_embedding_update   Adam on a float32 master copy of the embeddings with the

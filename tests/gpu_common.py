@@ -5,60 +5,102 @@ import numpy as np
 import oracle
 import synth_inputs as si
 
-# Tolerances (the ones the acceptance criteria state): float32 features rtol 1e-4 /
-# atol 1e-5; bfloat16 features rtol 2e-2.
-# Absolute tolerances are taken in units of the compared tensor's scale:
-#   float32:  1e-5 * max(1, largest |reference|).  A gradient entry is a sum of up to
-#             thousands of products, and when the tensor's entries reach the hundreds (hub
-#             subgraphs of the power-law configurations) a float32 sum cannot resolve 1e-5 of
-#             a cancelling entry -- its round-off is eps * sqrt(terms) * (size of the partial
-#             sums), a fraction of the tensor's scale.
-#   bfloat16: 2^-6 * largest |reference|.  Every stored bf16 value carries up to 2^-9
-#             relative rounding error; an entry that is a cancelling sum of K stored values
-#             inherits up to 2^-9 * (sum of the |terms|) per rounding along the chain, and with
-#             a hub node in the subgraph a single term can be larger than any entry of the
-#             result.  Measured worst errors are about 2^-7 of the tensor's largest entry.
+# Tolerances.  The acceptance criteria state: float32 features rtol 1e-4 / atol 1e-5; bfloat16
+# features rtol 2e-2.  They are applied FLAT (exactly as stated) to every tensor first:
+#   float32:   |err| <= 1e-4 |ref| + 1e-5
+#   bfloat16:  |err| <= 2e-2 |ref| + BF16_ATOL   (the criteria give bfloat16 no absolute part; a value
+#              next to zero needs one.  A stored bf16 value carries 2^-9 relative rounding; both sides
+#              round the same tensors, so they differ only where float32 and double sums fall on two
+#              sides of a rounding boundary: one bf16 ulp (2^-8) of one O(1) activation times one
+#              O(0.1) weight, a few 1e-4 in z.  BF16_ATOL = 2e-3 leaves a margin over that.)
+# loss, p and z are held to the flat bound, always.
+# GRADIENT tensors that miss the flat bound get a second, scaled bound, and every use of it is
+# counted and printed (``Report``): the absolute part is taken in units of the scale of the entry's
+# own group -- the subgraph's matrix for dW, the node's row for dX:
+#   float32:   atol = 1e-5 * max(1, largest |ref| of the group).  A gradient entry is a sum of up to
+#              thousands of products; in hub subgraphs entries reach the hundreds, and a float32 sum
+#              cannot resolve 1e-5 of a cancelling entry (round-off eps * sqrt(terms) * partial sums).
+#   bfloat16:  atol = 2^-6 * largest |ref| of the group (an entry that is a cancelling sum of K stored
+#              values inherits 2^-9 * sum |terms| per rounding along the chain).
+# bfloat16 gradients only: a hidden activation on a bf16 rounding boundary can differ by one ulp between
+# the float32-accumulating kernel and the double-accumulating oracle; the next layer's pre-activations
+# move by ~1e-4 and the few units that close to zero flip their ReLU mask, which changes a handful of
+# gradient rows by a few percent.  Neither side is wrong, so at most BF16_GRAD_OUTLIER_FRAC of a bf16
+# gradient tensor's entries may miss the scaled bound provided ||err||_F <= BF16_GRAD_NORM_RTOL ||ref||_F.
 F32_RTOL, F32_ATOL = 1e-4, 1e-5
-BF16_RTOL, BF16_ATOL_SCALE = 2e-2, 2.0 ** -6
+BF16_RTOL, BF16_ATOL = 2e-2, 2e-3
+BF16_GROUP_ATOL_SCALE = 2.0 ** -6
+BF16_GRAD_OUTLIER_FRAC = 2e-3
+BF16_GRAD_NORM_RTOL = 2e-2
 
 
-def tolerances(dtype, ref):
-    top = float(np.abs(ref).max()) if ref.size else 0.0
-    if dtype == "bf16":
-        return BF16_RTOL, BF16_ATOL_SCALE * top + 1e-6
-    return F32_RTOL, F32_ATOL * max(1.0, top)
+class Report:
+    """Which bound each compared tensor needed; printed by the tests so that a drift inside the
+    wider bounds is seen."""
+
+    def __init__(self):
+        self.rows = {}
+
+    def add(self, name, entries, worst, scaled, outliers):
+        r = self.rows.setdefault(name, dict(entries=0, worst=0.0, scaled=0, outliers=0))
+        r["entries"] += entries
+        r["worst"] = max(r["worst"], worst)
+        r["scaled"] += scaled
+        r["outliers"] += outliers
+
+    def needs_only_flat(self, name):
+        r = self.rows.get(name)
+        return r is None or (r["scaled"] == 0 and r["outliers"] == 0)
+
+    def __str__(self):
+        out = []
+        for name in sorted(self.rows):
+            r = self.rows[name]
+            how = "flat bound" if not (r["scaled"] or r["outliers"]) else (
+                "%d entries needed the group-scaled bound, %d outliers under the norm rule" % (r["scaled"], r["outliers"]))
+            out.append("  %-6s %10d entries, worst |err| %.3g: %s" % (name, r["entries"], r["worst"], how))
+        return "\n".join(out)
 
 
-# bfloat16 GRADIENTS only: a hidden activation that lands on a bf16 rounding boundary can
-# differ by one bf16 ulp between the float32-accumulating kernel and the double-accumulating
-# oracle; that ulp moves the next layer's pre-activations by ~1e-4 and flips the ReLU mask
-# of the few units that sit that close to zero, which changes a handful of gradient rows by
-# a few percent.  Neither side is wrong, so for bf16 gradient tensors a small fraction of
-# entries may miss the element-wise bound, provided the tensor as a whole agrees:
-BF16_GRAD_OUTLIER_FRAC = 2e-3      # at most this share of entries outside the bound
-BF16_GRAD_NORM_RTOL = 2e-2         # and ||got - ref||_F <= this * ||ref||_F
+def flat_tolerances(dtype):
+    return (BF16_RTOL, BF16_ATOL) if dtype == "bf16" else (F32_RTOL, F32_ATOL)
 
 
-def assert_close(got, ref, dtype, what, skip_mask=None, bf16_gradient=False):
+def assert_close(got, ref, dtype, what, skip_mask=None, group_axes=None, report=None, name=None):
+    """Element-wise comparison.  Without ``group_axes`` only the flat bound applies (loss, p, z).
+    ``group_axes`` (gradient tensors) names the axes over which an entry's group extends -- (1, 2) for
+    dW [sets, F_in, F_out], (1,) for dX [rows, F] -- and enables the scaled bound and, for bfloat16,
+    the outlier rule.  Returns the largest absolute error."""
     got = np.asarray(got, dtype=np.float64)
     ref = np.asarray(ref, dtype=np.float64)
     assert got.shape == ref.shape, (what, got.shape, ref.shape)
-    rtol, atol = tolerances(dtype, ref)
+    rtol, atol = flat_tolerances(dtype)
     err = np.abs(got - ref)
-    bad = err > atol + rtol * np.abs(ref)
-    if skip_mask is not None:
-        bad &= ~skip_mask
-    if bad.any() and bf16_gradient and dtype == "bf16":
-        frac = bad.mean()
-        rel = float(np.linalg.norm(got - ref) / max(np.linalg.norm(ref), 1e-30))
-        assert frac <= BF16_GRAD_OUTLIER_FRAC and rel <= BF16_GRAD_NORM_RTOL, (
-            "%s: %.3g of entries outside the element-wise bound, norm-wise error %.3g" % (what, frac, rel))
-        return float(err.max())
+    checked = np.ones(err.shape, bool) if skip_mask is None else ~skip_mask
+    bad = (err > atol + rtol * np.abs(ref)) & checked
+    n_scaled = n_out = 0
+    if bad.any() and group_axes is not None:
+        top = np.abs(ref).max(axis=tuple(group_axes), keepdims=True) if ref.size else 0.0
+        wide = BF16_GROUP_ATOL_SCALE * top + atol if dtype == "bf16" else F32_ATOL * np.maximum(1.0, top)
+        still = (err > wide + rtol * np.abs(ref)) & checked
+        n_scaled = int(bad.sum() - still.sum())
+        bad = still
+        if bad.any() and dtype == "bf16":
+            frac = bad.sum() / max(1, checked.sum())
+            rel = float(np.linalg.norm((got - ref)[checked]) / max(np.linalg.norm(ref[checked]), 1e-30))
+            assert frac <= BF16_GRAD_OUTLIER_FRAC and rel <= BF16_GRAD_NORM_RTOL, (
+                "%s: %.3g of entries outside the scaled bound, norm-wise error %.3g" % (what, frac, rel))
+            n_out = int(bad.sum())
+            bad = np.zeros_like(bad)
     if bad.any():
         k = np.unravel_index(np.argmax(np.where(bad, err, 0)), err.shape)
-        raise AssertionError("%s: %d of %d entries outside rtol=%g atol=%g; worst at %s: got %r, expected %r"
-                             % (what, int(bad.sum()), bad.size, rtol, atol, k, got[k], ref[k]))
-    return float(err.max()) if err.size else 0.0
+        raise AssertionError("%s: %d of %d entries outside rtol=%g atol=%g%s; worst at %s: got %r, expected %r"
+                             % (what, int(bad.sum()), bad.size, rtol, atol,
+                                " (group-scaled)" if group_axes is not None else "", k, got[k], ref[k]))
+    worst = float(err[checked].max()) if checked.any() else 0.0
+    if report is not None:
+        report.add(name or what, int(checked.sum()), worst, n_scaled, n_out)
+    return worst
 
 
 def _adam_hyper(adam):
@@ -107,6 +149,7 @@ class StepCase:
         self.S, self.n = int(book["S"]), int(book["n"])
         self.sets = self.S if sets is None else sets
         self.alpha, self.beta, self.lam = alpha, beta, lam
+        self.report = Report()
 
     def run(self, graph, X_new, W, pen_new=None, want_dx=True, adam=None, threads=4, parts=None, label=""):
         """X_new [n,F0] float32 numpy (bf16-representable when dtype is bf16), W list of
@@ -166,9 +209,10 @@ class StepCase:
     def _compare(self, g, r, rows, s, W, adam, stats, label):
         dt = self.dtype
         sel = slice(None) if s is None else slice(s, s + 1)
-        stats["loss"] = max(stats.get("loss", 0), assert_close(g["loss"][sel], r["loss"], dt, label + " loss"))
-        stats["p"] = max(stats.get("p", 0), assert_close(g["p"][rows], r["p"], "f32" if dt == "f32" else dt, label + " p"))
-        stats["z"] = max(stats.get("z", 0), assert_close(g["z"][rows], r["z"], dt, label + " z"))
+        rep = self.report
+        stats["loss"] = max(stats.get("loss", 0), assert_close(g["loss"][sel], r["loss"], dt, label + " loss", report=rep, name="loss"))
+        stats["p"] = max(stats.get("p", 0), assert_close(g["p"][rows], r["p"], dt, label + " p", report=rep, name="p"))
+        stats["z"] = max(stats.get("z", 0), assert_close(g["z"][rows], r["z"], dt, label + " z", report=rep, name="z"))
         # A pre-activation that sits on a ReLU kink (|Z| below float32 round-off) decides a 0/1
         # mask that the two sides may round differently.  Such an entry of hidden layer l, in
         # subgraph q and unit h, can only touch column h of dW[l][q], all of dW[l'][q] for
@@ -199,13 +243,13 @@ class StepCase:
             # expected; most of the tensor must still be compared
             stats["kink_skipped_frac"] = max(stats.get("kink_skipped_frac", 0), float(skip.mean()))
             assert skip.mean() <= 0.3, "too many gradient entries sit behind a ReLU kink"
-            stats["dW%d" % l] = max(stats.get("dW%d" % l, 0), assert_close(gd, rd, dt, label + " dW[%d]" % l, skip, True))
+            stats["dW%d" % l] = max(stats.get("dW%d" % l, 0), assert_close(gd, rd, dt, label + " dW[%d]" % l, skip, (1, 2), rep, "dW%d" % l))
         if r["dX"] is not None and g["dX"] is not None:
             skip = np.zeros(r["dX"].shape, bool)
             for kp in kink_parts:
                 lo, hi = int(self.book["part_ptr"][kp]) - base, int(self.book["part_ptr"][kp + 1]) - base
                 skip[max(lo, 0):max(hi, 0)] = True
-            stats["dX"] = max(stats.get("dX", 0), assert_close(g["dX"][rows], r["dX"], dt, label + " dX", skip, True))
+            stats["dX"] = max(stats.get("dX", 0), assert_close(g["dX"][rows], r["dX"], dt, label + " dX", skip, (1,), rep, "dX"))
         if adam is not None and s is None:
             for l in range(self.L):
                 # (a) the update rule itself: the oracle's Adam fed with the GPU's own float32
@@ -224,9 +268,9 @@ class StepCase:
                     Wn = W[l].astype(np.float64).copy()
                     mn, vn = adam["m"][l].astype(np.float64).copy(), adam["v"][l].astype(np.float64).copy()
                     oracle.adam(Wn, mn, vn, r["dW"][l], *_adam_hyper(adam))
-                    assert_close(g["m"][l], mn, dt, label + " adam m[%d]" % l)
-                    assert_close(g["v"][l], vn, dt, label + " adam v[%d]" % l)
-                    assert_close(g["W"][l], Wn, dt, label + " adam W[%d]" % l)
+                    assert_close(g["m"][l], mn, dt, label + " adam m[%d]" % l, None, (1, 2), rep, "adam m")
+                    assert_close(g["v"][l], vn, dt, label + " adam v[%d]" % l, None, (1, 2), rep, "adam v")
+                    assert_close(g["W"][l], Wn, dt, label + " adam W[%d]" % l, report=rep, name="adam W")
 
 
 def check_decode(graph, book, p_new_f32):
@@ -290,7 +334,7 @@ def check_stage3(graph, book, p, policy_seed=None):
 
 
 def sampled_step_check(graph, book, dims, dtype, Xd, Wd, parts, x_rows, w_part, alpha=2.0, beta=1.0, lam=0.0,
-                       pen_d=None, pen_rows=None, opt=None, want_dx=True, label=""):
+                       pen_d=None, pen_rows=None, opt=None, want_dx=True, label="", report=None):
     """Full-size parity on sampled subgraphs.  The GPU runs one step on the whole batch
     (device tensors Xd, Wd, optional gnnco.Adam ``opt``); for every subgraph in ``parts``
     the oracle runs that subgraph alone and is compared on loss, p, z, dW, dX and the Adam
@@ -317,31 +361,44 @@ def sampled_step_check(graph, book, dims, dtype, Xd, Wd, parts, x_rows, w_part, 
                                flags=gnnco.WANT_DX if want_dx else 0)
     torch.cuda.synchronize()
     assert graph.async_status() == 0
-    case = StepCase(book, dims, dtype, sets, alpha, beta, lam)
     stats = {}
-    for s in parts:
+    # the oracle runs the sampled subgraphs one by one, several at a time on host threads (the C
+    # call releases the interpreter lock; nothing inside a subgraph's arithmetic changes)
+    import os
+    from concurrent.futures import ThreadPoolExecutor
+
+    def oracle_part(s):
         lo, hi = int(book["part_ptr"][s]), int(book["part_ptr"][s + 1])
         if hi == lo:
-            continue
-        k = s if sets > 1 else 0
+            return None
         Xs = x_rows(lo, hi)
-        got_x = Xd[lo:hi].float().cpu().numpy()
-        assert np.array_equal(got_x, Xs), "device X rows differ from the generator's"
         ws = [w_part(l, s) for l in range(L)]
         wc = [si.round_to_bf16(w) if bf16 else w for w in ws]
         rp = book["rowptr"][lo:hi + 1] - book["rowptr"][lo]
         ci = book["colidx"][book["rowptr"][lo]:book["rowptr"][hi]] - lo
         one = oracle.subgraph_step(rp, ci, dims, Xs, wc, alpha, beta, lam, None if pen_rows is None else pen_rows(lo, hi),
                                    want_dX=want_dx, want_Z=True, store_bf16=bf16)
+        return Xs, one
+
+    with ThreadPoolExecutor(max_workers=min(16, len(os.sched_getaffinity(0)))) as pool:
+        oracle_out = dict(zip(parts, pool.map(oracle_part, parts)))
+    for s in parts:
+        lo, hi = int(book["part_ptr"][s]), int(book["part_ptr"][s + 1])
+        if oracle_out[s] is None:
+            continue
+        k = s if sets > 1 else 0
+        Xs, one = oracle_out[s]
+        got_x = Xd[lo:hi].float().cpu().numpy()
+        assert np.array_equal(got_x, Xs), "device X rows differ from the generator's"
         r = dict(loss=np.array([one["loss"]]), p=one["p"], z=one["z"], dX=one["dX"], dW=[d[None] for d in one["dW"]],
                  Z=one["Z"])
         g = dict(loss=loss[s:s + 1].cpu().numpy(), p=p[lo:hi].cpu().numpy(), z=z[lo:hi].cpu().numpy(),
                  dW=[dW[l][k:k + 1].cpu().numpy() for l in range(L)],
                  dX=None if dX is None else dX[lo:hi].float().cpu().numpy())
         tag = "%s part %d" % (label, s)
-        stats["loss"] = max(stats.get("loss", 0), assert_close(g["loss"], r["loss"], dtype, tag + " loss"))
-        stats["p"] = max(stats.get("p", 0), assert_close(g["p"], r["p"], dtype, tag + " p"))
-        stats["z"] = max(stats.get("z", 0), assert_close(g["z"], r["z"], dtype, tag + " z"))
+        stats["loss"] = max(stats.get("loss", 0), assert_close(g["loss"], r["loss"], dtype, tag + " loss", report=report, name="loss"))
+        stats["p"] = max(stats.get("p", 0), assert_close(g["p"], r["p"], dtype, tag + " p", report=report, name="p"))
+        stats["z"] = max(stats.get("z", 0), assert_close(g["z"], r["z"], dtype, tag + " z", report=report, name="z"))
         kinks = [set(np.nonzero((np.abs(Z) < 1e-6 * (1.0 + np.abs(Z))).any(axis=0))[0].tolist()) for Z in (r["Z"] or [])]
         kinks += [set()] * (L - len(kinks))
         near = any(kinks)
@@ -357,9 +414,9 @@ def sampled_step_check(graph, book, dims, dtype, Xd, Wd, parts, x_rows, w_part, 
                     else:
                         skip[:] = True
             stats["dW%d" % l] = max(stats.get("dW%d" % l, 0),
-                                    assert_close(g["dW"][l], r["dW"][l], dtype, tag + " dW[%d]" % l, skip, True))
+                                    assert_close(g["dW"][l], r["dW"][l], dtype, tag + " dW[%d]" % l, skip, (1, 2), report, "dW%d" % l))
         if want_dx and not near:
-            stats["dX"] = max(stats.get("dX", 0), assert_close(g["dX"], r["dX"], dtype, tag + " dX", None, True))
+            stats["dX"] = max(stats.get("dX", 0), assert_close(g["dX"], r["dX"], dtype, tag + " dX", None, (1,), report, "dX"))
         if opt is not None:
             hyper = _adam_hyper(dict(lr=lr, step=step_no))
             for l in range(L):
@@ -372,15 +429,16 @@ def sampled_step_check(graph, book, dims, dtype, Xd, Wd, parts, x_rows, w_part, 
 
 
 def pick_parts(book, count, seed):
-    """Seeded sample of subgraphs plus the one with the most intra edges and the one that
-    holds the longest row."""
+    """Seeded sample of ``count`` subgraphs plus the first, the last, the one with the most intra
+    edges and the one that holds the longest row."""
     S = int(book["S"])
     pp = book["part_ptr"].astype(np.int64)
     nnz = book["rowptr"][pp[1:]].astype(np.int64) - book["rowptr"][pp[:-1]].astype(np.int64)
     deg = np.diff(book["rowptr"])
-    picks = {int(np.argmax(nnz)), int(book["node_part"][int(np.argmax(deg))])}
-    for r in si.u64(seed, 0, 4 * count).tolist():
-        if len(picks) >= count + 2:
+    picks = {0, S - 1, int(np.argmax(nnz)), int(book["node_part"][int(np.argmax(deg))])}
+    want = min(S, len(picks) + count)
+    for r in si.u64(seed, 0, 8 * count + 64).tolist():
+        if len(picks) >= want:
             break
         picks.add(int(r % S))
     return sorted(picks)
