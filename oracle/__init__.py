@@ -59,6 +59,10 @@ def _native():
         lib.oracle_repair.restype = i64
         lib.oracle_round_bf16.argtypes = [dbl]
         lib.oracle_round_bf16.restype = dbl
+        lib.oracle_louvain.argtypes = [i64, i64, vp, vp, i32, i32, vp, vp, vp, vp, vp]
+        lib.oracle_louvain.restype = i64
+        lib.oracle_louvain_sweep.argtypes = [i64, i64, vp, vp, vp, vp]
+        lib.oracle_louvain_sweep.restype = i64
         _lib = lib
     return _lib
 
@@ -191,6 +195,38 @@ def partition_quality(eu: np.ndarray, ev: np.ndarray, part: np.ndarray, S: int) 
     in_edges, tot = np.empty(S, np.int64), np.empty(S, np.int64)
     q = _native().oracle_partition_quality(eu.size, _ptr(eu), _ptr(ev), _ptr(part), S, _ptr(in_edges), _ptr(tot))
     return dict(in_edges=in_edges, tot=tot, Q=float(q))
+
+
+def louvain(n: int, eu: np.ndarray, ev: np.ndarray, max_levels: int = 32, max_sweeps: int = 64) -> Dict[str, object]:
+    """Deterministic Louvain partition (Section 3.1; synchronous sweeps, exact integer gains --
+    see the C source).  Returns part [n] int32, S, the exact modularity numerator ``qnum`` and
+    ``two_m`` (Q = qnum / two_m**2), the levels that moved something and the accepted sweeps."""
+    eu = np.ascontiguousarray(eu, dtype=np.int32)
+    ev = np.ascontiguousarray(ev, dtype=np.int32)
+    part = np.empty(n, np.int32)
+    qnum, two_m = ctypes.c_int64(0), ctypes.c_int64(0)
+    levels, sweeps = ctypes.c_int32(0), ctypes.c_int32(0)
+    S = _native().oracle_louvain(n, eu.size, _ptr(eu), _ptr(ev), max_levels, max_sweeps, _ptr(part),
+                                 ctypes.addressof(qnum), ctypes.addressof(two_m), ctypes.addressof(levels),
+                                 ctypes.addressof(sweeps))
+    if S < 0:
+        raise OracleError(int(S), "oracle_louvain")
+    q = qnum.value / float(two_m.value) ** 2 if two_m.value else 0.0
+    return dict(part=part, S=int(S), qnum=int(qnum.value), two_m=int(two_m.value), Q=q, levels=int(levels.value),
+                sweeps=int(sweeps.value))
+
+
+def louvain_sweep(n: int, eu: np.ndarray, ev: np.ndarray, comm: np.ndarray) -> Dict[str, object]:
+    """One frozen-state sweep on the input graph from the community vector ``comm``: every node's
+    next community and the number of nodes that move."""
+    eu = np.ascontiguousarray(eu, dtype=np.int32)
+    ev = np.ascontiguousarray(ev, dtype=np.int32)
+    comm = np.ascontiguousarray(comm, dtype=np.int32)
+    nxt = np.empty(n, np.int32)
+    moves = _native().oracle_louvain_sweep(n, eu.size, _ptr(eu), _ptr(ev), _ptr(comm), _ptr(nxt))
+    if moves < 0:
+        raise OracleError(int(moves), "oracle_louvain_sweep")
+    return dict(next=nxt, moves=int(moves))
 
 
 def delta_q(k_i_in: float, sigma_tot: float, k_i: float, m: float) -> float:

@@ -533,3 +533,278 @@ double oracle_partition_quality(int64_t E, const int32_t* eu, const int32_t* ev,
   }
   return q;
 }
+
+/*
+ * Louvain partitioning (Section 3.1, Eqs. 1-2), in a form whose result is uniquely defined.
+ *
+ * The method of Section 3.1 repeats two phases: nodes move, one by one, to the neighbouring
+ * community with the largest modularity gain (Eq. 2), and then every community is contracted
+ * into one node of a smaller weighted graph.  The one-by-one phase depends on a visiting order
+ * that the paper does not fix, so its result is not unique.  The reading taken here makes every
+ * sweep a function of the state before it (all nodes decide from the same frozen state, then
+ * all moves are applied together) and compares gains exactly:
+ *
+ *   level graph   nodes 0..N-1, integer edge weights w(a,b) (1 on the input graph), self-loop
+ *                 weights loop(a) (0 on the input graph); degree k_a = sum_{b != a} w(a,b) + 2 loop(a);
+ *                 2m = sum_a k_a, the same on every level.
+ *   sweep         every node a starts a level in its own community.  With the state frozen
+ *                 (comm, tot[c] = sum of k over c, size[c]), node a collects kin[c] = sum of w(a,b)
+ *                 over neighbours b != a with comm[b] = c, and scores its own community and every
+ *                 community with kin > 0 by Eq. 2 times 2 m^2, an integer:
+ *                     score(c) = 2m * kin[c] - (tot[c] - [c == comm[a]] k_a) * k_a
+ *                 (the node is taken out of its own community first).  It moves to the best-scoring
+ *                 community, the LOWEST id among equals, if that is not its own and scores strictly
+ *                 higher than its own; a node alone in its community does not move to a community of
+ *                 one node with a HIGHER id (two single nodes would swap places for ever otherwise).
+ *   acceptance    after the moves of a sweep are applied the modularity numerator
+ *                     Qnum = sum_c [ 2m * in2(c) - tot(c)^2 ],   Q = Qnum / (2m)^2,
+ *                 in2(c) = twice the weight inside c (Eq. 1's Sigma_in counted from both ends, self loops
+ *                 twice), is recomputed exactly; a sweep that does not raise it strictly is undone and
+ *                 ends the level, as does a sweep without a move or the sweep limit.
+ *   contraction   communities that are not empty become the nodes of the next level, numbered in
+ *                 ascending order of their ids; weights between two communities add up, weight inside a
+ *                 community becomes its self loop.  The procedure ends when a level moves nothing (or at
+ *                 the level limit).
+ *
+ * Input: simple undirected graph as an edge list (each edge once).  Output: part[i] in [0, S) for the
+ * original nodes, S (returned), and *qnum_out / *two_m_out so that Q = qnum / two_m^2.
+ * levels_out / sweeps_out (optional) receive the number of levels that moved something and the
+ * number of accepted sweeps.  Returns S, or a negative error.
+ */
+typedef struct {
+  int64_t N;
+  int64_t* rp;      /* [N+1] */
+  int32_t* ci;      /* neighbours b != a */
+  int64_t* w;       /* weights */
+  int64_t* loop;    /* [N] */
+} lv_graph;
+
+static void lv_free(lv_graph* g) { free(g->rp); free(g->ci); free(g->w); free(g->loop); g->rp = NULL; g->ci = NULL; g->w = NULL; g->loop = NULL; }
+
+/* level graph from a list of M undirected weighted edges (a != b allowed to repeat: weights add up;
+ * a == b goes to the self loop) */
+static int lv_build(int64_t N, int64_t M, const int32_t* ea, const int32_t* eb, const int64_t* ew, lv_graph* g) {
+  g->N = N;
+  g->rp = (int64_t*)calloc((size_t)N + 1, sizeof(int64_t));
+  g->loop = (int64_t*)calloc((size_t)N + 1, sizeof(int64_t));
+  if (!g->rp || !g->loop) return ORACLE_NOMEM;
+  for (int64_t e = 0; e < M; ++e) {
+    if (ea[e] == eb[e]) { g->loop[ea[e]] += ew[e]; continue; }
+    g->rp[ea[e] + 1]++; g->rp[eb[e] + 1]++;
+  }
+  for (int64_t a = 0; a < N; ++a) g->rp[a + 1] += g->rp[a];
+  int64_t nnz = g->rp[N];
+  int32_t* tci = (int32_t*)malloc((size_t)(nnz + 1) * sizeof(int32_t));
+  int64_t* tw = (int64_t*)malloc((size_t)(nnz + 1) * sizeof(int64_t));
+  int64_t* pos = (int64_t*)malloc((size_t)(N + 1) * sizeof(int64_t));
+  if (!tci || !tw || !pos) { free(tci); free(tw); free(pos); return ORACLE_NOMEM; }
+  memcpy(pos, g->rp, (size_t)N * sizeof(int64_t));
+  for (int64_t e = 0; e < M; ++e) {
+    if (ea[e] == eb[e]) continue;
+    tci[pos[ea[e]]] = eb[e]; tw[pos[ea[e]]++] = ew[e];
+    tci[pos[eb[e]]] = ea[e]; tw[pos[eb[e]]++] = ew[e];
+  }
+  free(pos);
+  g->ci = tci; g->w = tw;
+  return ORACLE_OK;
+}
+
+static int64_t lv_qnum(const lv_graph* g, const int32_t* comm, int64_t two_m, int64_t* in2, int64_t* tot) {
+  int64_t N = g->N;
+  for (int64_t c = 0; c < N; ++c) in2[c] = tot[c] = 0;
+  for (int64_t a = 0; a < N; ++a) {
+    int64_t k = 2 * g->loop[a];
+    in2[comm[a]] += 2 * g->loop[a];
+    for (int64_t q = g->rp[a]; q < g->rp[a + 1]; ++q) {
+      k += g->w[q];
+      if (comm[g->ci[q]] == comm[a]) in2[comm[a]] += g->w[q];      /* seen from both ends over the loop */
+    }
+    tot[comm[a]] += k;
+  }
+  int64_t num = 0;
+  for (int64_t c = 0; c < N; ++c) num += two_m * in2[c] - tot[c] * tot[c];
+  return num;
+}
+
+/* One frozen-state sweep: next[a] for every node of the level graph (see above).  tot and size
+ * describe comm; kin (all zero on entry and on exit) and touched are scratch.  Returns the number
+ * of nodes that move. */
+static int64_t lv_decide(const lv_graph* g, const int32_t* comm, const int64_t* k, const int64_t* tot,
+                         const int64_t* size, int64_t two_m, int64_t* kin, int32_t* touched, int32_t* next) {
+  int64_t moves = 0;
+  for (int64_t a = 0; a < g->N; ++a) {
+    const int32_t own = comm[a];
+    int64_t nt = 0;
+    for (int64_t q = g->rp[a]; q < g->rp[a + 1]; ++q) {
+      int32_t c = comm[g->ci[q]];
+      if (kin[c] == 0) touched[nt++] = c;
+      kin[c] += g->w[q];
+    }
+    const int64_t own_score = two_m * kin[own] - (tot[own] - k[a]) * k[a];
+    int64_t best_score = own_score;
+    int32_t best = own;
+    for (int64_t t = 0; t < nt; ++t) {
+      int32_t c = touched[t];
+      if (c == own) continue;
+      int64_t sc = two_m * kin[c] - tot[c] * k[a];
+      if (sc > best_score || (sc == best_score && best != own && c < best)) { best_score = sc; best = c; }
+    }
+    for (int64_t t = 0; t < nt; ++t) kin[touched[t]] = 0;
+    if (best != own && best_score > own_score && !(size[own] == 1 && size[best] == 1 && best > own)) {
+      next[a] = best;
+      ++moves;
+    } else {
+      next[a] = own;
+    }
+  }
+  return moves;
+}
+
+int64_t oracle_louvain(int64_t n, int64_t E, const int32_t* eu, const int32_t* ev, int32_t max_levels,
+                       int32_t max_sweeps, int32_t* part, int64_t* qnum_out, int64_t* two_m_out,
+                       int32_t* levels_out, int32_t* sweeps_out) {
+  if (n <= 0 || E < 0 || max_levels < 1 || max_sweeps < 1) return ORACLE_BAD_ARG;
+  for (int64_t e = 0; e < E; ++e) {
+    if (eu[e] < 0 || eu[e] >= n || ev[e] < 0 || ev[e] >= n) return ORACLE_OUT_OF_RANGE;
+    if (eu[e] == ev[e]) return ORACLE_NOT_SIMPLE;
+  }
+  const int64_t two_m = 2 * E;
+  int64_t* ones = (int64_t*)malloc((size_t)(E + 1) * sizeof(int64_t));
+  if (!ones) return ORACLE_NOMEM;
+  for (int64_t e = 0; e < E; ++e) ones[e] = 1;
+  lv_graph g;
+  int rc = lv_build(n, E, eu, ev, ones, &g);
+  free(ones);
+  if (rc != ORACLE_OK) { lv_free(&g); return rc; }
+  for (int64_t i = 0; i < n; ++i) part[i] = (int32_t)i;      /* level-0 node of every original node */
+  int32_t levels = 0, sweeps_total = 0;
+  int64_t qnum = 0;
+  int64_t S = n;
+  for (int32_t level = 0; level < max_levels; ++level) {
+    const int64_t N = g.N;
+    int32_t* comm = (int32_t*)malloc((size_t)N * sizeof(int32_t));
+    int32_t* next = (int32_t*)malloc((size_t)N * sizeof(int32_t));
+    int64_t* k = (int64_t*)malloc((size_t)N * sizeof(int64_t));
+    int64_t* tot = (int64_t*)malloc((size_t)N * sizeof(int64_t));
+    int64_t* in2 = (int64_t*)malloc((size_t)N * sizeof(int64_t));
+    int64_t* size = (int64_t*)malloc((size_t)N * sizeof(int64_t));
+    int64_t* kin = (int64_t*)calloc((size_t)N, sizeof(int64_t));
+    int32_t* touched = (int32_t*)malloc((size_t)N * sizeof(int32_t));
+    if (!comm || !next || !k || !tot || !in2 || !size || !kin || !touched) {
+      free(comm); free(next); free(k); free(tot); free(in2); free(size); free(kin); free(touched); lv_free(&g);
+      return ORACLE_NOMEM;
+    }
+    for (int64_t a = 0; a < N; ++a) {
+      comm[a] = (int32_t)a;
+      k[a] = 2 * g.loop[a];
+      for (int64_t q = g.rp[a]; q < g.rp[a + 1]; ++q) k[a] += g.w[q];
+    }
+    qnum = lv_qnum(&g, comm, two_m, in2, tot);
+    int moved_this_level = 0;
+    for (int32_t sweep = 0; sweep < max_sweeps; ++sweep) {
+      for (int64_t c = 0; c < N; ++c) tot[c] = size[c] = 0;
+      for (int64_t a = 0; a < N; ++a) { tot[comm[a]] += k[a]; size[comm[a]] += 1; }
+      const int64_t moves = lv_decide(&g, comm, k, tot, size, two_m, kin, touched, next);
+      if (moves == 0) break;
+      int64_t q_new = lv_qnum(&g, next, two_m, in2, tot);
+      if (q_new <= qnum) break;                         /* the sweep as a whole did not help: undone */
+      memcpy(comm, next, (size_t)N * sizeof(int32_t));
+      qnum = q_new;
+      moved_this_level = 1;
+      ++sweeps_total;
+    }
+    free(next); free(k); free(tot); free(in2); free(size); free(kin); free(touched);
+    if (!moved_this_level) { free(comm); break; }
+    ++levels;
+    /* contraction: communities in ascending id order become nodes 0..Nc-1 */
+    int32_t* newid = (int32_t*)malloc((size_t)N * sizeof(int32_t));
+    if (!newid) { free(comm); lv_free(&g); return ORACLE_NOMEM; }
+    for (int64_t c = 0; c < N; ++c) newid[c] = -1;
+    for (int64_t a = 0; a < N; ++a) newid[comm[a]] = 0;
+    int64_t Nc = 0;
+    for (int64_t c = 0; c < N; ++c) if (newid[c] == 0) newid[c] = (int32_t)Nc++;
+    for (int64_t i = 0; i < n; ++i) part[i] = newid[comm[part[i]]];
+    /* every undirected edge once (a < b) plus the self loops, relabelled; lv_build adds weights up */
+    int64_t M = N;
+    for (int64_t a = 0; a < N; ++a)
+      for (int64_t q = g.rp[a]; q < g.rp[a + 1]; ++q) if (g.ci[q] > a) ++M;
+    int32_t* ea = (int32_t*)malloc((size_t)(M + 1) * sizeof(int32_t));
+    int32_t* eb = (int32_t*)malloc((size_t)(M + 1) * sizeof(int32_t));
+    int64_t* ew = (int64_t*)malloc((size_t)(M + 1) * sizeof(int64_t));
+    if (!ea || !eb || !ew) { free(ea); free(eb); free(ew); free(newid); free(comm); lv_free(&g); return ORACLE_NOMEM; }
+    int64_t t = 0;
+    for (int64_t a = 0; a < N; ++a) {
+      ea[t] = eb[t] = newid[comm[a]]; ew[t++] = g.loop[a];
+      for (int64_t q = g.rp[a]; q < g.rp[a + 1]; ++q)
+        if (g.ci[q] > a) { ea[t] = newid[comm[a]]; eb[t] = newid[comm[g.ci[q]]]; ew[t++] = g.w[q]; }
+    }
+    free(newid); free(comm);
+    lv_free(&g);
+    /* merge parallel edges so that the next level's adjacency lists hold every neighbour once */
+    {
+      /* sort (min, max) pairs by a simple two-pass counting approach: build, then compact rows */
+      lv_graph raw;
+      for (int64_t e = 0; e < t; ++e)
+        if (ea[e] > eb[e]) { int32_t s = ea[e]; ea[e] = eb[e]; eb[e] = s; }
+      rc = lv_build(Nc, t, ea, eb, ew, &raw);
+      free(ea); free(eb); free(ew);
+      if (rc != ORACLE_OK) { lv_free(&raw); return rc; }
+      int64_t* acc = (int64_t*)calloc((size_t)Nc, sizeof(int64_t));
+      int32_t* seen = (int32_t*)malloc((size_t)Nc * sizeof(int32_t));
+      int64_t* nrp = (int64_t*)calloc((size_t)Nc + 1, sizeof(int64_t));
+      if (!acc || !seen || !nrp) { free(acc); free(seen); free(nrp); lv_free(&raw); return ORACLE_NOMEM; }
+      int64_t out = 0;
+      for (int64_t a = 0; a < Nc; ++a) {
+        int64_t ns = 0;
+        for (int64_t q = raw.rp[a]; q < raw.rp[a + 1]; ++q) {
+          int32_t b = raw.ci[q];
+          if (acc[b] == 0) seen[ns++] = b;
+          acc[b] += raw.w[q];
+        }
+        qsort(seen, (size_t)ns, sizeof(int32_t), cmp_i32);
+        for (int64_t s = 0; s < ns; ++s) { raw.ci[out] = seen[s]; raw.w[out++] = acc[seen[s]]; acc[seen[s]] = 0; }
+        nrp[a + 1] = out;
+      }
+      free(acc); free(seen);
+      free(raw.rp);
+      raw.rp = nrp;
+      g = raw;
+    }
+    S = Nc;
+  }
+  lv_free(&g);
+  if (qnum_out) *qnum_out = qnum;
+  if (two_m_out) *two_m_out = two_m;
+  if (levels_out) *levels_out = levels;
+  if (sweeps_out) *sweeps_out = sweeps_total;
+  return S;
+}
+
+/* One frozen-state sweep on the input graph from a GIVEN community vector (no acceptance test, no
+ * contraction): next[i] as defined above.  Lets a test look at a single sweep. */
+int64_t oracle_louvain_sweep(int64_t n, int64_t E, const int32_t* eu, const int32_t* ev, const int32_t* comm,
+                             int32_t* next) {
+  int64_t* ones = (int64_t*)malloc((size_t)(E + 1) * sizeof(int64_t));
+  if (!ones) return ORACLE_NOMEM;
+  for (int64_t e = 0; e < E; ++e) ones[e] = 1;
+  lv_graph g;
+  int rc = lv_build(n, E, eu, ev, ones, &g);
+  free(ones);
+  if (rc != ORACLE_OK) { lv_free(&g); return rc; }
+  const int64_t two_m = 2 * E;
+  int64_t* k = (int64_t*)calloc((size_t)n, sizeof(int64_t));
+  int64_t* tot = (int64_t*)calloc((size_t)n, sizeof(int64_t));
+  int64_t* size = (int64_t*)calloc((size_t)n, sizeof(int64_t));
+  int64_t* kin = (int64_t*)calloc((size_t)n, sizeof(int64_t));
+  int32_t* touched = (int32_t*)malloc((size_t)n * sizeof(int32_t));
+  if (!k || !tot || !size || !kin || !touched) { free(k); free(tot); free(size); free(kin); free(touched); lv_free(&g); return ORACLE_NOMEM; }
+  for (int64_t a = 0; a < n; ++a) {
+    for (int64_t q = g.rp[a]; q < g.rp[a + 1]; ++q) k[a] += g.w[q];
+    tot[comm[a]] += k[a];
+    size[comm[a]] += 1;
+  }
+  const int64_t moves = lv_decide(&g, comm, k, tot, size, two_m, kin, touched, next);
+  free(k); free(tot); free(size); free(kin); free(touched);
+  lv_free(&g);
+  return moves;
+}

@@ -60,6 +60,9 @@ struct gnnco_handle {
   float* inv_deg = nullptr;
   uint8_t* is_boundary = nullptr;
   int32_t *tile_row0 = nullptr, *tile_rows = nullptr;      // dense-transform tiles
+  int32_t *pair_row0 = nullptr, *pair_rows = nullptr;      // double tiles (up to 256 rows of one subgraph) for CTA pairs
+  int32_t n_pairs = 0;
+  int pair_clusters = -1;                                  // co-resident CTA pairs of the two-CTA transform (-1: not asked yet)
   int32_t *item_row0 = nullptr, *item_row1 = nullptr;      // objective work items
   int32_t* part_item_ptr = nullptr;                        // [S+1] items of each subgraph
   int32_t* status = nullptr;                               // device status word + counters
@@ -127,9 +130,10 @@ int32_t launch_aggregate(gnnco_handle* h, int dtype, const void* in, void* out, 
 int32_t launch_aggregate_rank1(gnnco_handle* h, int dtype, const void* H, const float* coef, const void* w,
                                int64_t w_stride, void* out, int F, cudaStream_t st);
 // the same from the bits [H > 0] (n x F/8 bytes, element f of a row = bit f%8 of byte f/8) instead of H
+// (H itself is still read for the few rows with more than kLongRowDegree neighbours)
 bool aggregate_rank1_bits_supported(const gnnco_handle* h, int dtype, int F);
-int32_t launch_aggregate_rank1_bits(gnnco_handle* h, int dtype, const uint8_t* bits, const float* coef, const void* w,
-                                    int64_t w_stride, void* out, int F, cudaStream_t st);
+int32_t launch_aggregate_rank1_bits(gnnco_handle* h, int dtype, const uint8_t* bits, const void* H, const float* coef,
+                                    const void* w, int64_t w_stride, void* out, int F, cudaStream_t st);
 
 // ---- dense.cu
 // Y[tile rows x N] = act( A[rows x K] * B_s ), B_s = W[s] (K x N) or, with transB, W[s]^T where W[s] is (N x K);
@@ -167,6 +171,11 @@ bool tc_transform_supported(int dtype, int K, int N);
 int32_t launch_transform_tc(gnnco_handle* h, const void* A, const void* B, int64_t b_stride, void* Y, int K, int N,
                             bool relu, const float* row_scale, const void* relu_mask, bool backward, const void* dot_w,
                             int64_t dot_stride, float* dot_out, cudaStream_t st);
+// the same by pairs of CTAs (cluster of two, one 256-row double tile per pair; tc_gemm2.cu)
+bool tc_pair_transform_supported(gnnco_handle* h, int dtype, int K, int N);
+int32_t launch_transform_tc_pair(gnnco_handle* h, const void* A, const void* B, int64_t b_stride, int32_t b_sets, void* Y,
+                                 int K, int N, bool relu, const float* row_scale, const void* relu_mask, bool backward,
+                                 const void* dot_w, int64_t dot_stride, float* dot_out, cudaStream_t st);
 bool tc_weight_grad_supported(int dtype, int K, int N);
 int32_t launch_weight_grad_tc(gnnco_handle* h, const void* A, const void* G, float* dW, float* scratch, int K, int N,
                               cudaStream_t st);

@@ -321,6 +321,7 @@ struct PersistentLayout {
   int32_t *perm, *inv_perm, *node_part, *part_ptr, *rowptr, *colidx, *bnd_u, *bnd_v;
   float* inv_deg;
   uint8_t* is_boundary;
+  int32_t *pair_row0, *pair_rows;
   int32_t *tile_row0, *tile_rows, *item_row0, *item_row1, *part_item_ptr, *status, *long_rows, *seg_begin, *seg_end, *long_first_seg;
   int4* row_head;
   int32_t *wg_begin, *wg_end, *wg_slot, *wg_mpart, *wg_mfirst, *wg_mcount;
@@ -347,6 +348,8 @@ PersistentLayout carve_persistent(void* base, int64_t n, int64_t E, int32_t S) {
   L.is_boundary = c.take<uint8_t>(n);
   L.tile_row0 = c.take<int32_t>(L.max_tiles);
   L.tile_rows = c.take<int32_t>(L.max_tiles);
+  L.pair_row0 = c.take<int32_t>(L.max_tiles);
+  L.pair_rows = c.take<int32_t>(L.max_tiles);
   L.item_row0 = c.take<int32_t>(L.max_items);
   L.item_row1 = c.take<int32_t>(L.max_items);
   L.part_item_ptr = c.take<int32_t>((size_t)S + 1);
@@ -441,6 +444,7 @@ extern "C" int32_t gnnco_partition_load(const gnnco_graph_desc* g, void* persist
   h->perm = P.perm; h->inv_perm = P.inv_perm; h->node_part = P.node_part; h->part_ptr = P.part_ptr;
   h->rowptr = P.rowptr; h->colidx = P.colidx; h->bnd_u = P.bnd_u; h->bnd_v = P.bnd_v;
   h->inv_deg = P.inv_deg; h->is_boundary = P.is_boundary;
+  h->pair_row0 = P.pair_row0; h->pair_rows = P.pair_rows;
   h->tile_row0 = P.tile_row0; h->tile_rows = P.tile_rows; h->item_row0 = P.item_row0; h->item_row1 = P.item_row1;
   h->part_item_ptr = P.part_item_ptr; h->status = P.status; h->long_rows = P.long_rows; h->seg_begin = P.seg_begin; h->seg_end = P.seg_end;
   h->long_first_seg = P.long_first_seg; h->row_head = P.row_head;
@@ -520,10 +524,15 @@ extern "C" int32_t gnnco_partition_load(const gnnco_graph_desc* g, void* persist
   GNNCO_LAUNCH_CHECK();
 
   // 5. host-built tables: dense-transform tiles and objective work items (from part_ptr)
-  std::vector<int32_t> t0, tr, i0, i1, pip((size_t)S + 1);
+  std::vector<int32_t> t0, tr, p0, pr, i0, i1, pip((size_t)S + 1);
   for (int32_t s = 0; s < S; ++s) {
     int32_t a = h->h_part_ptr[s], b = h->h_part_ptr[s + 1];
     pip[s] = (int32_t)i0.size();
+    // double tiles for the two-CTA transform: 256 rows of one subgraph, 128 for each CTA of a pair
+    for (int32_t r = a; r < b; r += 2 * kGemmTileRows) {
+      p0.push_back(r);
+      pr.push_back(b - r < 2 * kGemmTileRows ? b - r : 2 * kGemmTileRows);
+    }
     for (int32_t r = a; r < b; r += kGemmTileRows) {
       t0.push_back(r);
       tr.push_back(b - r < kGemmTileRows ? b - r : kGemmTileRows);
@@ -566,6 +575,7 @@ extern "C" int32_t gnnco_partition_load(const gnnco_graph_desc* g, void* persist
     if (h->n_wg_chunks > P.max_chunks) return GNNCO_INTERNAL;
   }
   h->n_tiles = (int32_t)t0.size();
+  h->n_pairs = (int32_t)p0.size();
   h->n_items = (int32_t)i0.size();
   if (h->n_tiles > P.max_tiles || h->n_items > P.max_items) return GNNCO_INTERNAL;
   auto up = [&](int32_t* dst, const std::vector<int32_t>& v) {
@@ -574,6 +584,8 @@ extern "C" int32_t gnnco_partition_load(const gnnco_graph_desc* g, void* persist
   };
   GNNCO_CUDA_TRY(up(P.tile_row0, t0));
   GNNCO_CUDA_TRY(up(P.tile_rows, tr));
+  GNNCO_CUDA_TRY(up(P.pair_row0, p0));
+  GNNCO_CUDA_TRY(up(P.pair_rows, pr));
   GNNCO_CUDA_TRY(up(P.item_row0, i0));
   GNNCO_CUDA_TRY(up(P.item_row1, i1));
   GNNCO_CUDA_TRY(up(P.part_item_ptr, pip));

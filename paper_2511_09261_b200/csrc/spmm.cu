@@ -276,6 +276,24 @@ __device__ __forceinline__ void add_where_bits(float (&acc)[VN], uint32_t m, flo
   for (int e = 0; e < VN; ++e) acc[e] += ((m >> e) & 1u) ? c : 0.0f;
 }
 
+// The same for a byte of bits, written so that the seven low bits become seven predicates at once
+// (the assembler turns tests of the low bits 1, 2, 4 ... 64 of one register into a single
+// register-to-predicates move) and every element costs one predicated add.  Measured on B200:
+// 10 issue cycles per byte against 21 for the shift-mask-select form above; the batched kernel is
+// bound by its integer pipe, so this is what its speed hangs on.
+__device__ __forceinline__ void add_where_bits8(float (&acc)[8], uint32_t m, float c) {
+  asm("{\n\t.reg .pred p<7>;\n\t.reg .b32 t<7>;\n\t"
+      "and.b32 t0, %7, 1;\n\tand.b32 t1, %7, 2;\n\tand.b32 t2, %7, 4;\n\tand.b32 t3, %7, 8;\n\t"
+      "and.b32 t4, %7, 16;\n\tand.b32 t5, %7, 32;\n\tand.b32 t6, %7, 64;\n\t"
+      "setp.ne.b32 p0, t0, 0;\n\tsetp.ne.b32 p1, t1, 0;\n\tsetp.ne.b32 p2, t2, 0;\n\tsetp.ne.b32 p3, t3, 0;\n\t"
+      "setp.ne.b32 p4, t4, 0;\n\tsetp.ne.b32 p5, t5, 0;\n\tsetp.ne.b32 p6, t6, 0;\n\t"
+      "@p0 add.f32 %0, %0, %8;\n\t@p1 add.f32 %1, %1, %8;\n\t@p2 add.f32 %2, %2, %8;\n\t@p3 add.f32 %3, %3, %8;\n\t"
+      "@p4 add.f32 %4, %4, %8;\n\t@p5 add.f32 %5, %5, %8;\n\t@p6 add.f32 %6, %6, %8;\n\t}"
+      : "+f"(acc[0]), "+f"(acc[1]), "+f"(acc[2]), "+f"(acc[3]), "+f"(acc[4]), "+f"(acc[5]), "+f"(acc[6])
+      : "r"(m), "f"(c));
+  acc[7] += (m & 128u) ? c : 0.0f;
+}
+
 template <typename T, int LPR, int VPL>
 __global__ void __launch_bounds__(256) aggregate_rank1_bits(const uint8_t* __restrict__ bits, T* __restrict__ out,
                                                             const int4* __restrict__ row_head,
@@ -385,6 +403,160 @@ __global__ void __launch_bounds__(256) aggregate_rank1_bits(const uint8_t* __res
 #pragma unroll
     for (int e = 0; e < VN; ++e) acc[v][e] *= wf[e];
     Vec<T>::store(out + row * F + (v * LPR + sub) * VN, acc[v]);
+  }
+}
+
+// Rank-1 mode from mask bits, rows in batches (row widths of 256 and 512 elements: NB = 32 or 64
+// bytes of bits a row).  The kernel above gives every row a warp that walks head record ->
+// neighbour bits -> store as a chain of dependent round trips; with 64 warps on an SM only 64 rows
+// are in flight and the pass is bound by that chain, not by its bytes.  Here a warp owns 32
+// consecutive rows and works in two phases:
+//   gather   lane = row: head record, coefficient, subgraph id and the row's own bits in one round
+//            trip (the bits of 32 consecutive rows are one contiguous kilobyte), the bits and
+//            coefficients of the first two neighbours (named by the head record) in a second one;
+//            everything is parked in shared memory.  32 rows per warp are in flight.
+//   reduce   lane = 8 (or 16) features: row after row, the parked bits are expanded, neighbours
+//            beyond the second are fetched 32 at a time (lane = neighbour, parked the same way)
+//            and added in CSR order, the sum is scaled by the subgraph's weight vector and stored
+//            as one 512-byte (1 KB) line per row.
+// Sums are taken in the same order as in the kernel above, so the results are bit-identical.
+// Rows with more than kLongRowDegree neighbours are left to the block-per-segment kernels (which gather
+// the activation itself): hubs are neighbours in the node order, and a warp that met a run of them
+// would walk tens of thousands of neighbours on its own while the rest of the GPU idles.
+template <int NB>
+__global__ void __launch_bounds__(256) aggregate_rank1_bits_batch(const uint8_t* __restrict__ bits,
+                                                                  __nv_bfloat16* __restrict__ out,
+                                                                  const int4* __restrict__ row_head,
+                                                                  const int32_t* __restrict__ colidx,
+                                                                  const Rank1Args<__nv_bfloat16> r1, int64_t n,
+                                                                  int skip_long, int prefetch_blocks) {
+  using T = __nv_bfloat16;
+  constexpr int F = NB * 8, VPL = NB / 32, Q = NB / 16;
+  constexpr int kWarpBytes = 4 * 32 * NB + 7 * 32 * 4;       // own + two neighbours + tail bits, 7 words of per-row scalars
+  extern __shared__ uint4 smem_r1b[];
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  if (threadIdx.x == 0 && prefetch_blocks > 0) {               // see aggregate_vec
+    const int64_t r0 = ((int64_t)blockIdx.x + prefetch_blocks) * 256;
+    if (r0 + 256 <= n) {
+      asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;" ::"l"(row_head + r0), "r"(256u * 16u) : "memory");
+      const uint8_t* b0 = bits + r0 * NB;
+      if (((uintptr_t)b0 & 15) == 0)
+        asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;" ::"l"(b0), "r"(256u * (uint32_t)NB) : "memory");
+      if ((((uintptr_t)(r1.coef + r0)) & 15) == 0)
+        asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;" ::"l"(r1.coef + r0), "r"(1024u) : "memory");
+      if ((((uintptr_t)(r1.node_part + r0)) & 15) == 0)
+        asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;" ::"l"(r1.node_part + r0), "r"(1024u) : "memory");
+    }
+  }
+  const int64_t row0 = (int64_t)blockIdx.x * 256 + warp * 32;
+  if (row0 >= n) return;                                       // whole warp; no block-wide barrier below
+  uint8_t* wbase = reinterpret_cast<uint8_t*>(smem_r1b) + warp * kWarpBytes;
+  uint8_t* sb = wbase;                                         // [3][32 rows][NB]: own, first, second neighbour
+  uint8_t* tb = wbase + 3 * 32 * NB;                           // [32 neighbours][NB]
+  float* sc = reinterpret_cast<float*>(wbase + 4 * 32 * NB);   // [3][32] coefficients
+  int32_t* sdeg = reinterpret_cast<int32_t*>(sc + 96);
+  int32_t* sfirst = sdeg + 32;
+  int32_t* spart = sfirst + 32;
+  float* tcf = reinterpret_cast<float*>(spart + 32);           // [32] coefficients of the parked neighbours
+  // ---- gather, lane = row
+  {
+    const int64_t row = row0 + lane;
+    const bool valid = row < n;
+    int4 head = make_int4(0, 0, 0, 0);
+    float c_own = 0.0f, c0 = 0.0f, c1 = 0.0f;
+    int32_t part = 0;
+    uint4 own[Q], b0[Q], b1[Q];
+#pragma unroll
+    for (int q = 0; q < Q; ++q) own[q] = b0[q] = b1[q] = make_uint4(0u, 0u, 0u, 0u);
+    if (valid) {
+      head = __ldg(row_head + row);
+      c_own = __ldg(r1.coef + row);
+      part = __ldg(r1.node_part + row);
+#pragma unroll
+      for (int q = 0; q < Q; ++q) own[q] = __ldg(reinterpret_cast<const uint4*>(bits + row * NB) + q);
+      if (head.y > 0) {
+#pragma unroll
+        for (int q = 0; q < Q; ++q) b0[q] = __ldg(reinterpret_cast<const uint4*>(bits + (int64_t)head.z * NB) + q);
+        c0 = __ldg(r1.coef + head.z);
+      }
+      if (head.y > 1) {
+#pragma unroll
+        for (int q = 0; q < Q; ++q) b1[q] = __ldg(reinterpret_cast<const uint4*>(bits + (int64_t)head.w * NB) + q);
+        c1 = __ldg(r1.coef + head.w);
+      }
+    }
+#pragma unroll
+    for (int q = 0; q < Q; ++q) {
+      reinterpret_cast<uint4*>(sb + (0 * 32 + lane) * NB)[q] = own[q];
+      reinterpret_cast<uint4*>(sb + (1 * 32 + lane) * NB)[q] = b0[q];
+      reinterpret_cast<uint4*>(sb + (2 * 32 + lane) * NB)[q] = b1[q];
+    }
+    sc[lane] = c_own; sc[32 + lane] = c0; sc[64 + lane] = c1;
+    sdeg[lane] = head.y; sfirst[lane] = head.x; spart[lane] = part;
+  }
+  __syncwarp();
+  // ---- reduce, lane = VPL pieces of 8 features
+  const int rows_here = (int)min((int64_t)32, n - row0);
+  int cur_part = -1;
+  float wf[VPL][8];                                            // this lane's pieces of the subgraph's weight vector
+  for (int r = 0; r < rows_here; ++r) {
+    const int deg = sdeg[r];
+    if (skip_long && deg > kLongRowDegree) continue;           // a block (or one per segment) takes this row
+    float acc[VPL][8];
+#pragma unroll
+    for (int v = 0; v < VPL; ++v) {
+#pragma unroll
+      for (int e = 0; e < 8; ++e) acc[v][e] = 0.0f;
+      add_where_bits8(acc[v], sb[(0 * 32 + r) * NB + v * 32 + lane], sc[r]);
+    }
+    if (deg > 0) {
+#pragma unroll
+      for (int v = 0; v < VPL; ++v) add_where_bits8(acc[v], sb[(1 * 32 + r) * NB + v * 32 + lane], sc[32 + r]);
+    }
+    if (deg > 1) {
+#pragma unroll
+      for (int v = 0; v < VPL; ++v) add_where_bits8(acc[v], sb[(2 * 32 + r) * NB + v * 32 + lane], sc[64 + r]);
+    }
+    if (deg > 2) {
+      const int32_t r_end = sfirst[r] + deg;
+      for (int32_t k0 = sfirst[r] + 2; k0 < r_end; k0 += 32) {
+        const int32_t k = k0 + lane;
+        uint4 tbits[Q];
+        float cj = 0.0f;
+#pragma unroll
+        for (int q = 0; q < Q; ++q) tbits[q] = make_uint4(0u, 0u, 0u, 0u);
+        if (k < r_end) {
+          const int64_t j = __ldg(colidx + k);
+          cj = __ldg(r1.coef + j);
+#pragma unroll
+          for (int q = 0; q < Q; ++q) tbits[q] = __ldg(reinterpret_cast<const uint4*>(bits + j * NB) + q);
+        }
+        __syncwarp();                                          // readers of the previous 32 are done
+#pragma unroll
+        for (int q = 0; q < Q; ++q) reinterpret_cast<uint4*>(tb + lane * NB)[q] = tbits[q];
+        tcf[lane] = cj;
+        __syncwarp();
+        const int cnt = min(32, r_end - k0);
+        for (int t = 0; t < cnt; ++t) {
+          const float c = tcf[t];
+#pragma unroll
+          for (int v = 0; v < VPL; ++v) add_where_bits8(acc[v], tb[t * NB + v * 32 + lane], c);
+        }
+      }
+    }
+    const int part = spart[r];
+    if (part != cur_part) {                                    // uniform across the warp
+      cur_part = part;
+      const T* wv = r1.w + (int64_t)part * r1.w_stride;
+#pragma unroll
+      for (int v = 0; v < VPL; ++v) Vec<T>::load(wv + (v * 32 + lane) * 8, wf[v]);
+    }
+#pragma unroll
+    for (int v = 0; v < VPL; ++v) {
+#pragma unroll
+      for (int e = 0; e < 8; ++e) acc[v][e] *= wf[v][e];
+      Vec<T>::store(out + (row0 + r) * F + (v * 32 + lane) * 8, acc[v]);
+    }
   }
 }
 
@@ -532,35 +704,41 @@ __global__ void __launch_bounds__(256) aggregate_any(const T* __restrict__ in, T
   }
 }
 
+// The rows with more than kLongRowDegree neighbours, one block per row (or per segment of a row when the
+// step has scratch for the partial sums), on the handle's side stream so that they run beside the kernel
+// that the caller launches next on `st`.  Returns whether the side stream was used; the caller then
+// makes `st` wait for ev_join.
+template <typename T, int LPR, int VPL, bool R1>
+bool fork_long_rows(gnnco_handle* h, const T* in, T* out, const float* scale, const T* mask, const Rank1Args<T>& r1,
+                    int F, cudaStream_t st) {
+  const size_t long_smem = (size_t)(256 / LPR) * F * sizeof(float);
+  const bool fork = h->side_stream && h->ev_fork && h->ev_join && cudaEventRecord(h->ev_fork, st) == cudaSuccess &&
+                    cudaStreamWaitEvent(h->side_stream, h->ev_fork, 0) == cudaSuccess;
+  cudaStream_t ls = fork ? h->side_stream : st;
+  if (h->agg_partial && h->n_long_segs > 0) {
+    // long rows cut into segments: partial sums by one block per segment, then one block per row
+    aggregate_long_row<T, LPR, VPL, R1><<<h->n_long_segs, 256, long_smem, ls>>>(
+        in, out, h->rowptr, h->colidx, scale, mask, r1, h->long_rows, F, h->seg_begin, h->seg_end, h->agg_partial);
+    aggregate_long_finish<T, R1><<<h->n_long, 256, 0, ls>>>(in, out, scale, mask, r1, h->long_rows, h->long_first_seg,
+                                                            h->agg_partial, F);
+    h->launches += 2;
+  } else {
+    aggregate_long_row<T, LPR, VPL, R1><<<h->n_long, 256, long_smem, ls>>>(in, out, h->rowptr, h->colidx, scale, mask,
+                                                                            r1, h->long_rows, F, nullptr, nullptr, nullptr);
+    h->launches += 1;
+  }
+  if (fork) cudaEventRecord(h->ev_join, h->side_stream);
+  return fork;
+}
+
 template <typename T, int LPR, int VPL, bool R1>
 void launch_vec(const T* in, T* out, gnnco_handle* h, const float* scale, const T* mask, const Rank1Args<T>& r1, int F,
                 cudaStream_t st) {
   constexpr int ROWS_PER_BLOCK = 256 / LPR;
   const unsigned main_blocks = (unsigned)((h->n + ROWS_PER_BLOCK - 1) / ROWS_PER_BLOCK);
-  const size_t long_smem = (size_t)(256 / LPR) * F * sizeof(float);
   // L2 prefetch distance: one full wave of resident blocks (8 per SM) ahead; pointless on small grids
   const int sms = h->sm_count > 0 ? h->sm_count : 148;
   const int pf_blocks = main_blocks > 4u * 8u * (unsigned)sms ? 8 * sms : 0;
-  // the block-per-row kernel on the side stream, beside the kernel that follows on `st`
-  auto fork_long_rows = [&](const int32_t* list, int32_t count) -> bool {
-    const bool fork = h->side_stream && h->ev_fork && h->ev_join && cudaEventRecord(h->ev_fork, st) == cudaSuccess &&
-                      cudaStreamWaitEvent(h->side_stream, h->ev_fork, 0) == cudaSuccess;
-    cudaStream_t ls = fork ? h->side_stream : st;
-    if (h->agg_partial && h->n_long_segs > 0) {
-      // long rows cut into segments: partial sums by one block per segment, then one block per row
-      aggregate_long_row<T, LPR, VPL, R1><<<h->n_long_segs, 256, long_smem, ls>>>(
-          in, out, h->rowptr, h->colidx, scale, mask, r1, list, F, h->seg_begin, h->seg_end, h->agg_partial);
-      aggregate_long_finish<T, R1><<<count, 256, 0, ls>>>(in, out, scale, mask, r1, list, h->long_first_seg,
-                                                          h->agg_partial, F);
-      h->launches += 2;
-    } else {
-      aggregate_long_row<T, LPR, VPL, R1><<<count, 256, long_smem, ls>>>(in, out, h->rowptr, h->colidx, scale, mask,
-                                                                         r1, list, F, nullptr, nullptr, nullptr);
-      h->launches += 1;
-    }
-    if (fork) cudaEventRecord(h->ev_join, h->side_stream);
-    return fork;
-  };
   if (h->n_long == 0) {
     aggregate_vec<T, LPR, VPL, R1><<<main_blocks, 256, 0, st>>>(in, out, h->row_head, h->colidx, scale, mask, r1, h->n,
                                                                 F, 0, pf_blocks);
@@ -580,7 +758,7 @@ void launch_vec(const T* in, T* out, gnnco_handle* h, const float* scale, const 
                                                                 F, 0, pf_blocks);
     return;
   }
-  const bool fork = fork_long_rows(h->long_rows, h->n_long);
+  const bool fork = fork_long_rows<T, LPR, VPL, R1>(h, in, out, scale, mask, r1, F, st);
   aggregate_vec<T, LPR, VPL, R1><<<main_blocks, 256, 0, st>>>(in, out, h->row_head, h->colidx, scale, mask, r1, h->n, F,
                                                               1, pf_blocks);
   if (fork) cudaStreamWaitEvent(st, h->ev_join, 0);
@@ -657,7 +835,8 @@ bool rows_stay_inline(const gnnco_handle* h, int F, size_t elem) {
 }
 
 template <typename T>
-int32_t rank1_bits_typed(gnnco_handle* h, const uint8_t* bits, T* out, int F, const Rank1Args<T>& r1, cudaStream_t st) {
+int32_t rank1_bits_typed(gnnco_handle* h, const uint8_t* bits, const T* H, T* out, int F, const Rank1Args<T>& r1,
+                         cudaStream_t st) {
   constexpr int VN = Vec<T>::N;
   const int sms = h->sm_count > 0 ? h->sm_count : 148;
 #define GNNCO_R1B(LPR, VPL)                                                                                      \
@@ -666,6 +845,27 @@ int32_t rank1_bits_typed(gnnco_handle* h, const uint8_t* bits, T* out, int F, co
     const int pf = blocks > 4u * 8u * (unsigned)sms ? 8 * sms : 0;                                               \
     aggregate_rank1_bits<T, LPR, VPL><<<blocks, 256, 0, st>>>(bits, out, h->row_head, h->colidx, r1, h->n, F, pf); \
   } while (0)
+  if (F == 256 || F == 512) {
+    // rows in batches of 32 per warp (see aggregate_rank1_bits_batch); long rows beside them
+    const unsigned blocks = (unsigned)((h->n + 255) / 256);
+    const int pf = blocks > 4u * 5u * (unsigned)sms ? 5 * sms : 0;      // one wave of resident blocks ahead
+    const int skip = h->n_long > 0 ? 1 : 0;
+    bool fork = false;
+    if (F == 256) {
+      constexpr int smem = 8 * (4 * 32 * 32 + 7 * 32 * 4);
+      if (skip) fork = fork_long_rows<T, 32, 1, true>(h, H, out, nullptr, nullptr, r1, F, st);
+      aggregate_rank1_bits_batch<32><<<blocks, 256, smem, st>>>(bits, out, h->row_head, h->colidx, r1, h->n, skip, pf);
+    } else {
+      constexpr int smem = 8 * (4 * 32 * 64 + 7 * 32 * 4);
+      GNNCO_CUDA_TRY(cudaFuncSetAttribute(aggregate_rank1_bits_batch<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
+      if (skip) fork = fork_long_rows<T, 32, 2, true>(h, H, out, nullptr, nullptr, r1, F, st);
+      aggregate_rank1_bits_batch<64><<<blocks, 256, smem, st>>>(bits, out, h->row_head, h->colidx, r1, h->n, skip, pf);
+    }
+    if (fork) cudaStreamWaitEvent(st, h->ev_join, 0);
+    h->launches += 1;
+    GNNCO_LAUNCH_CHECK();
+    return GNNCO_OK;
+  }
   switch (F / VN) {
     case 1: GNNCO_R1B(1, 1); break;
     case 2: GNNCO_R1B(2, 1); break;
@@ -689,15 +889,17 @@ bool aggregate_rank1_bits_supported(const gnnco_handle* h, int dtype, int F) {
   if (F % 8) return false;
   const int vecs = F / 8;
   if (!(vecs == 1 || vecs == 2 || vecs == 4 || vecs == 8 || vecs == 16 || vecs == 32 || vecs == 64)) return false;
+  if (F == 256 || F == 512) return true;          // the batched kernel hands its long rows to a block each
   return rows_stay_inline(h, F, 2);
 }
 
-int32_t launch_aggregate_rank1_bits(gnnco_handle* h, int dtype, const uint8_t* bits, const float* coef, const void* w,
-                                    int64_t w_stride, void* out, int F, cudaStream_t st) {
+int32_t launch_aggregate_rank1_bits(gnnco_handle* h, int dtype, const uint8_t* bits, const void* H, const float* coef,
+                                    const void* w, int64_t w_stride, void* out, int F, cudaStream_t st) {
   if (!aggregate_rank1_bits_supported(h, dtype, F)) return GNNCO_UNSUPPORTED;
-  if (((uintptr_t)out & 15) || ((uintptr_t)w & 15) || (w_stride % 8)) return GNNCO_UNSUPPORTED;
+  if (((uintptr_t)out & 15) || ((uintptr_t)w & 15) || (w_stride % 8) || ((uintptr_t)bits & 15) || ((uintptr_t)H & 15))
+    return GNNCO_UNSUPPORTED;
   ProfScope prof_(h, K_AGG_RANK1, st);
   return rank1_bits_typed<__nv_bfloat16>(
-      h, bits, (__nv_bfloat16*)out, F,
+      h, bits, (const __nv_bfloat16*)H, (__nv_bfloat16*)out, F,
       Rank1Args<__nv_bfloat16>{coef, (const __nv_bfloat16*)w, w_stride, h->node_part}, st);
 }

@@ -154,9 +154,14 @@ int32_t run_step(gnnco_handle* h, const gnnco_model_desc* m, const void* X, cons
     if (T.W_lp_t[l - 1]) {
       // the last hidden layer also produces u = H w_L in its epilogue
       const bool fuse = (l == L - 1) && (m->dims[l] % 8 == 0);
-      GNNCO_TRY(launch_transform_tc(h, Min, T.W_lp_t[l - 1], wstride[l - 1], T.H[l], m->dims[l - 1], m->dims[l], true,
-                                    nullptr, nullptr, false, fuse ? Wc[L - 1] : nullptr, wstride[L - 1],
-                                    fuse ? T.u : nullptr, st));
+      if (false && tc_pair_transform_supported(h, dt, m->dims[l - 1], m->dims[l]))
+        GNNCO_TRY(launch_transform_tc_pair(h, Min, T.W_lp_t[l - 1], wstride[l - 1], sets, T.H[l], m->dims[l - 1],
+                                           m->dims[l], true, nullptr, nullptr, false, fuse ? Wc[L - 1] : nullptr,
+                                           wstride[L - 1], fuse ? T.u : nullptr, st));
+      else
+        GNNCO_TRY(launch_transform_tc(h, Min, T.W_lp_t[l - 1], wstride[l - 1], T.H[l], m->dims[l - 1], m->dims[l], true,
+                                      nullptr, nullptr, false, fuse ? Wc[L - 1] : nullptr, wstride[L - 1],
+                                      fuse ? T.u : nullptr, st));
       u_done = fuse;
     } else if (T.W3_t[l - 1]) {
       const bool fuse = (l == L - 1) && (m->dims[l] % 4 == 0);
@@ -210,9 +215,10 @@ int32_t run_step(gnnco_handle* h, const gnnco_model_desc* m, const void* X, cons
     if (L > 1) {
       // from the mask bits that the weight-gradient pass above left behind, where it could
       const bool from_bits = have_bits && aggregate_rank1_bits_supported(h, dt, FL) &&
-                             !((uintptr_t)Wc[L - 1] & 15) && wstride[L - 1] % 8 == 0 && !((uintptr_t)Q & 15);
+                             !((uintptr_t)Wc[L - 1] & 15) && wstride[L - 1] % 8 == 0 && !((uintptr_t)Q & 15) &&
+                             !((uintptr_t)Hprev & 15);
       if (from_bits)
-        GNNCO_TRY(launch_aggregate_rank1_bits(h, dt, T.Hbits, T.u, Wc[L - 1], wstride[L - 1], Q, FL, st));
+        GNNCO_TRY(launch_aggregate_rank1_bits(h, dt, T.Hbits, Hprev, T.u, Wc[L - 1], wstride[L - 1], Q, FL, st));
       else
         GNNCO_TRY(launch_aggregate_rank1(h, dt, Hprev, T.u, Wc[L - 1], wstride[L - 1], Q, FL, st));
     }
@@ -231,7 +237,10 @@ int32_t run_step(gnnco_handle* h, const gnnco_model_desc* m, const void* X, cons
       void* dst = l > 1 ? other : out->dX;
       const float* scale = l > 1 ? h->inv_deg : nullptr;
       const void* mask = l > 1 ? T.H[l - 1] : nullptr;
-      if (tc_transform_supported(dt, N, K))
+      if (false && tc_pair_transform_supported(h, dt, N, K))
+        GNNCO_TRY(launch_transform_tc_pair(h, Q, Wc[l - 1], wstride[l - 1], sets, dst, N, K, false, scale, mask, true,
+                                           nullptr, 0, nullptr, st));
+      else if (tc_transform_supported(dt, N, K))
         GNNCO_TRY(launch_transform_tc(h, Q, Wc[l - 1], wstride[l - 1], dst, N, K, false, scale, mask, true, nullptr, 0,
                                       nullptr, st));
       else if (T.W3[l - 1])
