@@ -173,9 +173,12 @@ int32_t launch_transform_tc(gnnco_handle* h, const void* A, const void* B, int64
                             int64_t dot_stride, float* dot_out, cudaStream_t st);
 // the same by pairs of CTAs (cluster of two, one 256-row double tile per pair; tc_gemm2.cu)
 bool tc_pair_transform_supported(gnnco_handle* h, int dtype, int K, int N);
+// modes: relu (optionally bits_out = [Y > 0], one bit per element, and the row dot product), plain, or
+// row_scale + mask_bits (result zeroed where the bit of the saved activation is clear)
 int32_t launch_transform_tc_pair(gnnco_handle* h, const void* A, const void* B, int64_t b_stride, int32_t b_sets, void* Y,
-                                 int K, int N, bool relu, const float* row_scale, const void* relu_mask, bool backward,
-                                 const void* dot_w, int64_t dot_stride, float* dot_out, cudaStream_t st);
+                                 int K, int N, bool relu, const float* row_scale, const uint8_t* mask_bits,
+                                 uint8_t* bits_out, bool backward, const void* dot_w, int64_t dot_stride, float* dot_out,
+                                 cudaStream_t st);
 bool tc_weight_grad_supported(int dtype, int K, int N);
 int32_t launch_weight_grad_tc(gnnco_handle* h, const void* A, const void* G, float* dW, float* scratch, int K, int N,
                               cudaStream_t st);

@@ -11,17 +11,25 @@
 // slots.  Each SM still streams only its own rows from HBM; B crosses the SM-to-SM link, not L2.
 //
 // Operands arrive by TMA (cp.async.bulk.tensor, 2-D boxes of 128 rows x 64 bf16 with the
-// 128-byte swizzle that the MMA descriptors expect) issued by one thread per CTA; the tensor maps
-// cover this GPU's own buffers and no load is multicast.  Roles per CTA (ten warps):
-//   warp 9    one lane: waits for a free A slot, announces the bytes on the EVEN CTA's `full` barrier
+// 128-byte swizzle that the MMA descriptors expect) issued by one thread per CTA; results leave by
+// TMA too (boxes of 32 rows x 32 columns from a per-warp staging tile).  The tensor maps cover this
+// GPU's own buffers and no load is multicast.  Roles per CTA (eighteen warps):
+//   warp 17   one lane: waits for a free A slot, announces the bytes on the EVEN CTA's `full` barrier
 //             (which counts the boxes of both CTAs) and issues the boxes: one A k-block per slot, plus
 //             this CTA's half of the B k-block when the subgraph changes
-//   warp 8    even CTA only, one lane: per k-block wait `full`, issue 4 MMAs of 256 x N x 16 for
+//   warp 16   even CTA only, one lane: per k-block wait `full`, issue 4 MMAs of 256 x N x 16 for
 //             the pair, commit -> `empty` of that slot in BOTH CTAs; after the last k-block commit
 //             -> `acc_full` in both CTAs
-//   warps 0-7 epilogue of this CTA's 128 rows, as in tc_gemm.cu (TMEM -> registers -> scale / ReLU /
-//             mask / round -> staged 128-byte lines -> global; optional row dot product with the
-//             next layer's weight vector); then one arrival per warp on the even CTA's `acc_empty`
+//   warps 0-15 epilogue of this CTA's 128 rows: warp w owns TMEM lanes 32 (w % 4) .. +32 (one row per
+//             lane) and columns 64 (w / 4) .. +64.  It copies its part of the accumulator to registers and
+//             gives the accumulator buffer back AT ONCE (one arrival per warp on the even CTA's
+//             `acc_empty`), so the next tile's MMAs never wait for conversions or stores; then, 32
+//             columns at a time: scale / ReLU (inside the conversion to bf16) / mask (one bit per element of
+//             the saved activation; a rectifying launch can leave those bits behind), optional dot
+//             product with the next layer's weight vector, staging, one TMA store.  The last, ragged
+//             tile of a subgraph is stored with plain stores (a TMA box would spill into the next subgraph).
+// The drain used to be the bottleneck: with eight warps doing all of this the on-chip part alone took as
+// long per tile as the tile's memory traffic, and the two did not overlap.
 // Every wait has a time limit; a CTA that gives up raises the handle's status word and still takes
 // part in the cluster barriers at the end, so nothing is left waiting.
 #include <cuda.h>
@@ -31,12 +39,18 @@
 
 namespace {
 
-constexpr int kPairThreads = 320;
-constexpr int kPairEpiWarps = 8;
-constexpr int kPairMmaWarp = 8;
-constexpr int kPairTmaWarp = 9;
-constexpr uint32_t kPairMisc = 1536;         // barriers (512 B) + two 128-float dot-product exchange buffers
+constexpr int kPairEpiWarps = 16;
+constexpr int kPairMmaWarp = 16;
+constexpr int kPairTmaWarp = 17;
+constexpr int kPairThreads = 32 * 18;
+constexpr uint32_t kPairStage = 2048;        // per epilogue warp: 32 rows x 32 bf16
+constexpr uint32_t kPairMisc = 3584;         // barriers (512 B) + dot-product exchange [2 buffers][3 column groups][128 rows]
 constexpr uint32_t kPairSmemLimit = 232448;  // 227 KB
+
+// epilogue modes
+constexpr int kModePlain = 0;                // Y = A B^T
+constexpr int kModeRelu = 1;                 // Y = max(A B^T, 0), optional row dot product
+constexpr int kModeScaledMasked = 2;         // Y = row_scale * (A B^T) where mask > 0, else 0
 
 template <int KDIM, int NDIM>
 struct PairCfg {
@@ -44,45 +58,59 @@ struct PairCfg {
   static constexpr uint32_t A_SLOT = 128 * 128;             // 128 rows x 64 bf16
   static constexpr uint32_t B_SLOT = (NDIM / 2) * 128;      // this CTA's N/2 rows of one k-block
   static constexpr uint32_t B_BYTES = KB * B_SLOT;
-  static constexpr uint32_t EPI_BYTES = kPairEpiWarps * 4096;
+  static constexpr uint32_t EPI_BYTES = kPairEpiWarps * kPairStage;
   static constexpr int kFit = (int)((kPairSmemLimit - 1024 - kPairMisc - EPI_BYTES - B_BYTES) / A_SLOT);
-  static constexpr int kTiles = (kFit / KB) < 4 ? (kFit / KB) : 4;      // tiles of A in flight (at most four)
-  static constexpr int NSLOT = kTiles * KB;
+  static constexpr int NSLOT = kFit < 4 * KB ? kFit : 4 * KB;           // k-block slots of A in flight (at most four tiles)
   static constexpr uint32_t A_BYTES = NSLOT * A_SLOT;
-  static constexpr size_t SMEM = 1024 + A_BYTES + B_BYTES + kPairMisc + EPI_BYTES;
-  static_assert(kTiles >= 2, "the pair form needs at least two tiles of A slots");
+  static constexpr size_t SMEM = 1024 + A_BYTES + B_BYTES + EPI_BYTES + kPairMisc;
+  static_assert(NDIM == 64 * (kPairEpiWarps / 4), "sixteen epilogue warps cover four column groups of 64");
+  static_assert(NSLOT > KB, "the ring must hold more than one tile of A slots");
   static_assert(NSLOT <= 16, "barrier area holds 16 slots");
+  static_assert(SMEM <= kPairSmemLimit, "does not fit in shared memory");
 };
 
-// keep the bf16 halves of v where the matching halves of m are positive
-__device__ __forceinline__ uint32_t keep_positive_pair(uint32_t v, uint32_t m) {
-  const uint32_t lo = __uint_as_float(m << 16) > 0.0f ? 0x0000ffffu : 0u;
-  const uint32_t hi = __uint_as_float(m & 0xffff0000u) > 0.0f ? 0xffff0000u : 0u;
-  return v & (lo | hi);
+// two float32 -> packed bf16 pair (first argument in the low half), optionally rectified by the conversion itself
+template <bool RELU>
+__device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
+  uint32_t d;
+  if (RELU) asm("cvt.rn.relu.bf16x2.f32 %0, %1, %2;" : "=r"(d) : "f"(hi), "f"(lo));
+  else asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(d) : "f"(hi), "f"(lo));
+  return d;
 }
 
-template <int KDIM, int NDIM, bool MASKED>
+__device__ __forceinline__ void tma_store_2d(const void* tmap, uint32_t smem_src, int32_t x, int32_t y) {
+  asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.bulk_group [%0, {%1, %2}], [%3];"
+               ::"l"(tmap), "r"(x), "r"(y), "r"(smem_src) : "memory");
+  asm volatile("cp.async.bulk.commit_group;" ::: "memory");
+}
+// the bulk stores committed so far have read their shared-memory source
+__device__ __forceinline__ void tma_store_wait_read() { asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory"); }
+// ... and have been written
+__device__ __forceinline__ void tma_store_wait_all() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
+
+template <int KDIM, int NDIM, int MODE>
 __global__ void __launch_bounds__(kPairThreads, 1)
 transform_tc_pair(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
-                  int32_t b_per_part, __nv_bfloat16* __restrict__ Y, int relu, const float* __restrict__ row_scale,
-                  const __nv_bfloat16* __restrict__ relu_mask, const __nv_bfloat16* __restrict__ dot_w,
-                  int64_t dot_stride, float* __restrict__ dot_out, const int32_t* __restrict__ pair_row0,
-                  const int32_t* __restrict__ pair_rows, const int32_t* __restrict__ node_part, int n_pairs,
-                  int pairs_per_cluster, int32_t* status) {
+                  const __grid_constant__ CUtensorMap map_y, int32_t b_per_part, __nv_bfloat16* __restrict__ Y,
+                  const float* __restrict__ row_scale, const uint8_t* __restrict__ mask_bits,
+                  uint8_t* __restrict__ bits_out, const __nv_bfloat16* __restrict__ dot_w, int64_t dot_stride, float* __restrict__ dot_out,
+                  const int32_t* __restrict__ pair_row0, const int32_t* __restrict__ pair_rows,
+                  const int32_t* __restrict__ node_part, int n_pairs, int pairs_per_cluster, int32_t* status) {
   using C = PairCfg<KDIM, NDIM>;
   constexpr int KB = C::KB, NSLOT = C::NSLOT;
   extern __shared__ uint8_t smem_raw[];
   const uint32_t sbase = (tc::smem_u32(smem_raw) + 1023u) & ~1023u;
-  const uint32_t sA = sbase, sB = sbase + C::A_BYTES;
+  const uint32_t sA = sbase, sB = sbase + C::A_BYTES, sStage = sB + C::B_BYTES;
   uint8_t* gen_base = smem_raw + (sbase - tc::smem_u32(smem_raw));
-  uint64_t* full = reinterpret_cast<uint64_t*>(gen_base + C::A_BYTES + C::B_BYTES);   // [16]  (even CTA's copy is used)
-  uint64_t* empty = full + 16;                                                        // [16]  both CTAs
-  uint64_t* acc_full = empty + 16;                                                    // [2]   both CTAs
-  uint64_t* acc_empty = acc_full + 2;                                                 // [2]   even CTA's copy is used
-  uint64_t* dot_bar = acc_empty + 2;                                                  // [4 quarters][2 buffers]
+  uint8_t* misc = gen_base + C::A_BYTES + C::B_BYTES + C::EPI_BYTES;
+  uint64_t* full = reinterpret_cast<uint64_t*>(misc);          // [16]  (even CTA's copy is used)
+  uint64_t* empty = full + 16;                                 // [16]  both CTAs
+  uint64_t* acc_full = empty + 16;                             // [2]   both CTAs
+  uint64_t* acc_empty = acc_full + 2;                          // [2]   even CTA's copy is used
+  uint64_t* dot_bar = acc_empty + 2;                           // [4 quarters][2 buffers]
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(dot_bar + 8);
   volatile uint32_t* abort_flag = tmem_slot + 1;
-  float* dot_x = reinterpret_cast<float*>(gen_base + C::A_BYTES + C::B_BYTES + 512);  // [2][128]
+  float* dot_x = reinterpret_cast<float*>(misc + 512);         // [2 buffers][3 column groups][128 rows]
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const uint32_t rank = tc::cluster_ctarank();                 // 0 = even CTA (issues the MMAs), 1 = odd CTA
@@ -100,7 +128,7 @@ transform_tc_pair(const __grid_constant__ CUtensorMap map_a, const __grid_consta
       tc::mbar_init(acc_full + i, 1);
       tc::mbar_init(acc_empty + i, 2 * kPairEpiWarps);         // one arrival per epilogue warp of both CTAs
     }
-    for (int i = 0; i < 8; ++i) tc::mbar_init(dot_bar + i, 32);
+    for (int i = 0; i < 8; ++i) tc::mbar_init(dot_bar + i, 96);  // the three upper column groups of a lane quarter
     *abort_flag = 0;
     tc::fence_mbar_init();
   }
@@ -165,12 +193,10 @@ transform_tc_pair(const __grid_constant__ CUtensorMap map_a, const __grid_consta
     }
   } else {
     // ---------------------------------------------------------------------- epilogue (this CTA's 128 rows)
-    constexpr int CHUNKS = NDIM / 64;                 // 64-column chunks of the tile
-    constexpr int PER = (CHUNKS + 1) / 2;             // chunks per column half
-    const int quarter = warp & 3, half = warp >> 2;
-    const int ch_begin = half * PER, ch_end = min(CHUNKS, ch_begin + PER);
+    const int quarter = warp & 3, cg = warp >> 2;     // TMEM lane quarter, column group of 64
     const int row = quarter * 32 + lane;
-    const uint32_t stage = sbase + C::A_BYTES + C::B_BYTES + kPairMisc + warp * 4096;
+    const int c0 = cg * 64;
+    const uint32_t stage = sStage + warp * kPairStage;
     const uint32_t acc_empty_even = tc::map_to_cta(tc::smem_u32(acc_empty), 0);
     for (int t = t_begin, j = 0; t < t_end && !*abort_flag; ++t, ++j) {
       const int buf = j & 1;
@@ -178,63 +204,63 @@ transform_tc_pair(const __grid_constant__ CUtensorMap map_a, const __grid_consta
       const int rows = max(0, min(128, pair_rows[t] - (int)rank * 128));
       const bool valid = row < rows;
       const int rows_here = rows - quarter * 32;       // valid rows of this warp's 32
-      uint4 mk[MASKED ? PER : 1][8];
-      if (MASKED) {
-#pragma unroll
-        for (int c = 0; c < PER; ++c)
-#pragma unroll
-          for (int it = 0; it < 8; ++it) {
-            const int rr = it * 4 + (lane >> 3);
-            mk[c][it] = make_uint4(0u, 0u, 0u, 0u);
-            if (rr < rows_here && ch_begin + c < ch_end)
-              mk[c][it] = __ldg(reinterpret_cast<const uint4*>(relu_mask + (row0 + quarter * 32 + rr) * NDIM +
-                                                               (ch_begin + c) * 64 + (lane & 7) * 8));
-          }
+      float s = 1.0f;
+      uint2 mk = make_uint2(0u, 0u);
+      if (MODE == kModeScaledMasked && valid) {
+        // this row's scale and the 64 mask bits under this warp's columns, requested before the wait
+        s = row_scale[row0 + row];
+        mk = __ldg(reinterpret_cast<const uint2*>(mask_bits + (row0 + row) * (NDIM / 8) + c0 / 8));
       }
-      const float s = (row_scale && valid) ? row_scale[row0 + row] : 1.0f;
       const __nv_bfloat16* wv = nullptr;
-      if (dot_out) wv = dot_w + (int64_t)node_part[pair_row0[t]] * dot_stride;
+      if (MODE == kModeRelu && dot_out) wv = dot_w + (int64_t)node_part[pair_row0[t]] * dot_stride + c0;
       float dot = 0.0f;
+      uint32_t sign_words[2] = {0u, 0u};
       if (!tc::mbar_wait_bounded(acc_full + buf, (j >> 1) & 1)) { *abort_flag = 1; break; }
       tc::tc_fence_after_sync();
       uint32_t ra[32], rb[32];
-      auto read_chunk = [&](int c) {
-        const uint32_t at = tmem + ((uint32_t)(quarter * 32) << 16) + buf * NDIM + (ch_begin + c) * 64;
+      {
+        const uint32_t at = tmem + ((uint32_t)(quarter * 32) << 16) + buf * NDIM + c0;
         tc::tmem_ld_32x32(at, ra);
         tc::tmem_ld_32x32(at + 32, rb);
-      };
-      if (!MASKED && ch_begin < ch_end) read_chunk(0);
+        tc::tmem_ld_wait();
+      }
+      // the accumulator is in registers: hand the buffer back before converting and storing (the warps
+      // that collect the row dot products do it after they have read the exchange slots of this buffer,
+      // so that nobody can be two tiles ahead and overwrite them)
+      const bool late_release = MODE == kModeRelu && dot_out && cg == 0;
+      tc::tc_fence_before_sync();
+      __syncwarp();
+      if (lane == 0 && !late_release) tc::mbar_arrive_cluster(acc_empty_even + buf * 8);
 #pragma unroll
-      for (int c = 0; c < PER; ++c) {
-        if (ch_begin + c >= ch_end) break;
-        const int c0 = (ch_begin + c) * 64;
-        uint32_t o[32];                                // 64 bf16 of this thread's row, packed
-        auto convert = [&](const uint32_t (&r)[32], int at) {
+      for (int hh = 0; hh < 2; ++hh) {
+        uint32_t o[16];                                // 32 bf16 of this thread's row, packed
+#pragma unroll
+        for (int q = 0; q < 16; ++q) {
+          float a = __uint_as_float(hh ? rb[2 * q] : ra[2 * q]), b = __uint_as_float(hh ? rb[2 * q + 1] : ra[2 * q + 1]);
+          if (MODE == kModeScaledMasked) {
+            const uint32_t mw = hh ? mk.y : mk.x;          // bit k: column c0 + 32 hh + k of the saved activation was positive
+            a = (mw >> (2 * q)) & 1u ? a * s : 0.0f;
+            b = (mw >> (2 * q + 1)) & 1u ? b * s : 0.0f;
+          }
+          o[q] = pack_bf16<MODE == kModeRelu>(a, b);
+        }
+        if (MODE == kModeRelu && bits_out) {
+          // [stored value > 0], one bit per element, for the backward pass (element f of a row = bit f % 8 of
+          // byte f / 8): the 32 columns of this round are one word of the row
+          uint32_t word = 0;
 #pragma unroll
           for (int q = 0; q < 16; ++q) {
-            float a = __uint_as_float(r[2 * q]) * s, b = __uint_as_float(r[2 * q + 1]) * s;
-            if (relu) { a = a > 0.0f ? a : 0.0f; b = b > 0.0f ? b : 0.0f; }
-            __nv_bfloat162 v = __floats2bfloat162_rn(a, b);
-            o[at + q] = *reinterpret_cast<uint32_t*>(&v);
+            word |= (o[q] & 0x0000ffffu) ? (1u << (2 * q)) : 0u;
+            word |= (o[q] & 0xffff0000u) ? (2u << (2 * q)) : 0u;
           }
-        };
-        if (MASKED) {
-#pragma unroll
-          for (int hh = 0; hh < 2; ++hh) {
-            tc::tmem_ld_32x32(tmem + ((uint32_t)(quarter * 32) << 16) + buf * NDIM + c0 + hh * 32, ra);
-            tc::tmem_ld_wait();
-            convert(ra, hh * 16);
-          }
-        } else {
-          tc::tmem_ld_wait();
-          convert(ra, 0);
-          convert(rb, 16);
-          if (c + 1 < PER && ch_begin + c + 1 < ch_end) read_chunk(c + 1);
+          sign_words[hh] = word;
+          if (hh == 1 && valid)
+            *reinterpret_cast<uint2*>(bits_out + (row0 + row) * (NDIM / 8) + c0 / 8) = make_uint2(sign_words[0], word);
         }
         if (wv) {   // dot product of the STORED (rounded) row with the next layer's weight vector
 #pragma unroll
-          for (int q4 = 0; q4 < 8; ++q4) {
-            const uint4 w8 = __ldg(reinterpret_cast<const uint4*>(wv + c0 + q4 * 8));
+          for (int q4 = 0; q4 < 4; ++q4) {
+            const uint4 w8 = __ldg(reinterpret_cast<const uint4*>(wv + hh * 32) + q4);
             const uint32_t wq[4] = {w8.x, w8.y, w8.z, w8.w};
 #pragma unroll
             for (int q = 0; q < 4; ++q) {
@@ -244,42 +270,41 @@ transform_tc_pair(const __grid_constant__ CUtensorMap map_a, const __grid_consta
             }
           }
         }
-        __syncwarp();
+        if (rows_here >= 32) {
+          // staging tile: 32 rows of 64 bytes, dense; the previous store of this warp must have read it
+          if (lane == 0) tma_store_wait_read();
+          __syncwarp();
 #pragma unroll
-        for (int pc = 0; pc < 8; ++pc)
-          tc::st_shared16(stage + lane * 128 + ((pc ^ (lane & 7)) << 4), o[4 * pc], o[4 * pc + 1], o[4 * pc + 2],
-                          o[4 * pc + 3]);
-        __syncwarp();
+          for (int pc = 0; pc < 4; ++pc)
+            tc::st_shared16(stage + lane * 64 + pc * 16, o[4 * pc], o[4 * pc + 1], o[4 * pc + 2], o[4 * pc + 3]);
+          tc::fence_proxy_async_smem();
+          __syncwarp();
+          if (lane == 0) tma_store_2d(&map_y, stage, c0 + hh * 32, (int32_t)(row0 + quarter * 32));
+        } else if (valid) {
+          // ragged end of a subgraph: a box would reach into the next subgraph's rows
+          uint4* dst = reinterpret_cast<uint4*>(Y + (row0 + row) * NDIM + c0 + hh * 32);
 #pragma unroll
-        for (int it = 0; it < 8; ++it) {
-          const int rr = it * 4 + (lane >> 3), pc = lane & 7;
-          uint4 v = tc::ld_shared16(stage + rr * 128 + ((pc ^ (rr & 7)) << 4));
-          if (MASKED) {
-            v.x = keep_positive_pair(v.x, mk[c][it].x); v.y = keep_positive_pair(v.y, mk[c][it].y);
-            v.z = keep_positive_pair(v.z, mk[c][it].z); v.w = keep_positive_pair(v.w, mk[c][it].w);
-          }
-          if (rr < rows_here)
-            *reinterpret_cast<uint4*>(Y + (row0 + quarter * 32 + rr) * NDIM + c0 + pc * 8) = v;
+          for (int pc = 0; pc < 4; ++pc) dst[pc] = make_uint4(o[4 * pc], o[4 * pc + 1], o[4 * pc + 2], o[4 * pc + 3]);
         }
       }
-      if (dot_out) {
-        // lower column half + upper column half, in that order (see tc_gemm.cu)
-        if (CHUNKS > 1 && half == 1) {
-          dot_x[buf * 128 + row] = dot;
+      if (MODE == kModeRelu && dot_out) {
+        // column groups are added in the order 0, 1, 2, 3
+        if (cg > 0) {
+          dot_x[(buf * 3 + cg - 1) * 128 + row] = dot;
           tc::mbar_arrive(dot_bar + quarter * 2 + buf);
-        }
-        if (half == 0) {
-          if (CHUNKS > 1) {
-            if (!tc::mbar_wait_bounded(dot_bar + quarter * 2 + buf, (j >> 1) & 1)) { *abort_flag = 1; break; }
-            dot += dot_x[buf * 128 + row];
-          }
+        } else {
+          if (!tc::mbar_wait_bounded(dot_bar + quarter * 2 + buf, (j >> 1) & 1)) { *abort_flag = 1; break; }
+          dot += dot_x[(buf * 3 + 0) * 128 + row];
+          dot += dot_x[(buf * 3 + 1) * 128 + row];
+          dot += dot_x[(buf * 3 + 2) * 128 + row];
           if (valid) dot_out[row0 + row] = dot;
+          __syncwarp();
+          if (lane == 0) tc::mbar_arrive_cluster(acc_empty_even + buf * 8);
         }
       }
-      tc::tc_fence_before_sync();
-      __syncwarp();
-      if (lane == 0) tc::mbar_arrive_cluster(acc_empty_even + buf * 8);
     }
+    if (lane == 0) tma_store_wait_all();
+    __syncwarp();
   }
   if (*abort_flag && threadIdx.x == 0) atomicMin(status, (int32_t)GNNCO_INTERNAL);
   tc::tc_fence_before_sync();
@@ -307,25 +332,27 @@ EncodeTiledFn encode_tiled() {
   return fn;
 }
 
-// [rows x KDIM] bf16 row-major, boxes of box_rows x 64 elements, 128-byte swizzle
-bool make_map(CUtensorMap* m, const void* base, uint64_t rows, int kdim, int box_rows) {
+// [rows x width] bf16 row-major, boxes of box_rows x box_cols elements; operand boxes (64 columns) use the
+// 128-byte swizzle of the MMA descriptors, result boxes are dense
+bool make_map(CUtensorMap* m, const void* base, uint64_t rows, int width, int box_rows, int box_cols, bool swizzle) {
   EncodeTiledFn enc = encode_tiled();
   if (!enc) return false;
-  const cuuint64_t dims[2] = {(cuuint64_t)kdim, (cuuint64_t)rows};
-  const cuuint64_t strides[1] = {(cuuint64_t)kdim * 2};
-  const cuuint32_t box[2] = {64u, (cuuint32_t)box_rows};
+  const cuuint64_t dims[2] = {(cuuint64_t)width, (cuuint64_t)rows};
+  const cuuint64_t strides[1] = {(cuuint64_t)width * 2};
+  const cuuint32_t box[2] = {(cuuint32_t)box_cols, (cuuint32_t)box_rows};
   const cuuint32_t estr[2] = {1u, 1u};
   return enc(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides, box, estr,
-             CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
-             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+             CU_TENSOR_MAP_INTERLEAVE_NONE, swizzle ? CU_TENSOR_MAP_SWIZZLE_128B : CU_TENSOR_MAP_SWIZZLE_NONE,
+             CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
-template <int KDIM, int NDIM, bool MASKED>
-int32_t launch_pair_kernel(gnnco_handle* h, const CUtensorMap& ma, const CUtensorMap& mb, int32_t b_per_part, void* Y,
-                           bool relu, const float* row_scale, const void* relu_mask, const void* dot_w,
-                           int64_t dot_stride, float* dot_out, int clusters, int per, cudaStream_t st) {
+template <int KDIM, int NDIM, int MODE>
+int32_t launch_pair_kernel(gnnco_handle* h, const CUtensorMap& ma, const CUtensorMap& mb, const CUtensorMap& my,
+                           int32_t b_per_part, void* Y, const float* row_scale, const uint8_t* mask_bits,
+                           uint8_t* bits_out, const void* dot_w, int64_t dot_stride, float* dot_out, int clusters,
+                           int per, cudaStream_t st) {
   using C = PairCfg<KDIM, NDIM>;
-  auto kernel = transform_tc_pair<KDIM, NDIM, MASKED>;
+  auto kernel = transform_tc_pair<KDIM, NDIM, MODE>;
   GNNCO_CUDA_TRY(cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)C::SMEM));
   cudaLaunchConfig_t cfg{};
   cfg.gridDim = dim3(2 * clusters);
@@ -337,8 +364,8 @@ int32_t launch_pair_kernel(gnnco_handle* h, const CUtensorMap& ma, const CUtenso
   attr[0].val.clusterDim.x = 2; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
   cfg.attrs = attr;
   cfg.numAttrs = 1;
-  GNNCO_CUDA_TRY(cudaLaunchKernelEx(&cfg, kernel, ma, mb, b_per_part, (__nv_bfloat16*)Y, relu ? 1 : 0, row_scale,
-                                    (const __nv_bfloat16*)relu_mask, (const __nv_bfloat16*)dot_w, dot_stride, dot_out,
+  GNNCO_CUDA_TRY(cudaLaunchKernelEx(&cfg, kernel, ma, mb, my, b_per_part, (__nv_bfloat16*)Y, row_scale, mask_bits,
+                                    bits_out, (const __nv_bfloat16*)dot_w, dot_stride, dot_out,
                                     (const int32_t*)h->pair_row0, (const int32_t*)h->pair_rows,
                                     (const int32_t*)h->node_part, (int)h->n_pairs, per, h->status));
   h->launches += 1;
@@ -349,7 +376,7 @@ int32_t launch_pair_kernel(gnnco_handle* h, const CUtensorMap& ma, const CUtenso
 template <int KDIM, int NDIM>
 int resident_pairs() {
   using C = PairCfg<KDIM, NDIM>;
-  auto kernel = transform_tc_pair<KDIM, NDIM, false>;
+  auto kernel = transform_tc_pair<KDIM, NDIM, kModePlain>;
   if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)C::SMEM) != cudaSuccess) {
     cudaGetLastError();
     return 0;
@@ -373,21 +400,30 @@ int resident_pairs() {
 
 template <int KDIM, int NDIM>
 int32_t launch_pair(gnnco_handle* h, const void* A, const void* B, int64_t b_stride, int32_t b_sets, void* Y, bool relu,
-                    const float* row_scale, const void* relu_mask, const void* dot_w, int64_t dot_stride,
-                    float* dot_out, cudaStream_t st) {
-  CUtensorMap ma, mb;
-  // rows past the end of A read as zeros; B holds b_sets matrices of NDIM rows
-  if (!make_map(&ma, A, (uint64_t)h->n, KDIM, 128)) return GNNCO_CUDA_ERROR;
-  if (!make_map(&mb, B, (uint64_t)b_sets * NDIM, KDIM, NDIM / 2)) return GNNCO_CUDA_ERROR;
+                    const float* row_scale, const uint8_t* mask_bits, uint8_t* bits_out, const void* dot_w,
+                    int64_t dot_stride, float* dot_out, cudaStream_t st) {
+  int mode;
+  if (relu && !row_scale && !mask_bits) mode = kModeRelu;
+  else if (!relu && row_scale && mask_bits && !dot_out && !bits_out) mode = kModeScaledMasked;
+  else if (!relu && !row_scale && !mask_bits && !dot_out && !bits_out) mode = kModePlain;
+  else return GNNCO_UNSUPPORTED;
+  CUtensorMap ma, mb, my;
+  // rows past the end of A read as zeros; B holds b_sets matrices of NDIM rows; result boxes of 32 x 32
+  if (!make_map(&ma, A, (uint64_t)h->n, KDIM, 128, 64, true)) return GNNCO_CUDA_ERROR;
+  if (!make_map(&mb, B, (uint64_t)b_sets * NDIM, KDIM, NDIM / 2, 64, true)) return GNNCO_CUDA_ERROR;
+  if (!make_map(&my, Y, (uint64_t)h->n, NDIM, 32, 32, false)) return GNNCO_CUDA_ERROR;
   int clusters = h->pair_clusters < h->n_pairs ? h->pair_clusters : h->n_pairs;
   const int per = (h->n_pairs + clusters - 1) / clusters;
   clusters = (h->n_pairs + per - 1) / per;
   const int32_t b_per_part = b_stride == 0 ? 0 : NDIM;
-  if (relu_mask)
-    return launch_pair_kernel<KDIM, NDIM, true>(h, ma, mb, b_per_part, Y, relu, row_scale, relu_mask, dot_w, dot_stride,
-                                                dot_out, clusters, per, st);
-  return launch_pair_kernel<KDIM, NDIM, false>(h, ma, mb, b_per_part, Y, relu, row_scale, relu_mask, dot_w, dot_stride,
-                                               dot_out, clusters, per, st);
+  if (mode == kModeRelu)
+    return launch_pair_kernel<KDIM, NDIM, kModeRelu>(h, ma, mb, my, b_per_part, Y, row_scale, mask_bits, bits_out, dot_w,
+                                                     dot_stride, dot_out, clusters, per, st);
+  if (mode == kModeScaledMasked)
+    return launch_pair_kernel<KDIM, NDIM, kModeScaledMasked>(h, ma, mb, my, b_per_part, Y, row_scale, mask_bits, bits_out,
+                                                             dot_w, dot_stride, dot_out, clusters, per, st);
+  return launch_pair_kernel<KDIM, NDIM, kModePlain>(h, ma, mb, my, b_per_part, Y, row_scale, mask_bits, bits_out, dot_w,
+                                                    dot_stride, dot_out, clusters, per, st);
 }
 
 }  // namespace
@@ -401,10 +437,14 @@ bool tc_pair_transform_supported(gnnco_handle* h, int dtype, int K, int N) {
 }
 
 int32_t launch_transform_tc_pair(gnnco_handle* h, const void* A, const void* B, int64_t b_stride, int32_t b_sets, void* Y,
-                                 int K, int N, bool relu, const float* row_scale, const void* relu_mask, bool backward,
-                                 const void* dot_w, int64_t dot_stride, float* dot_out, cudaStream_t st) {
+                                 int K, int N, bool relu, const float* row_scale, const uint8_t* mask_bits,
+                                 uint8_t* bits_out, bool backward, const void* dot_w, int64_t dot_stride, float* dot_out,
+                                 cudaStream_t st) {
   if (!tc_pair_transform_supported(h, GNNCO_BF16, K, N)) return GNNCO_UNSUPPORTED;
-  if (((uintptr_t)A & 15) || ((uintptr_t)B & 15) || (b_stride != 0 && b_stride != (int64_t)K * N)) return GNNCO_UNSUPPORTED;
+  if (((uintptr_t)A & 15) || ((uintptr_t)B & 15) || ((uintptr_t)Y & 15) || (b_stride != 0 && b_stride != (int64_t)K * N))
+    return GNNCO_UNSUPPORTED;
   ProfScope prof_(h, backward ? K_TRANSFORM_BWD : K_TRANSFORM_FWD, st);
-  return launch_pair<256, 256>(h, A, B, b_stride, b_sets, Y, relu, row_scale, relu_mask, dot_w, dot_stride, dot_out, st);
+  if (((uintptr_t)mask_bits & 7) || ((uintptr_t)bits_out & 7)) return GNNCO_UNSUPPORTED;
+  return launch_pair<256, 256>(h, A, B, b_stride, b_sets, Y, relu, row_scale, mask_bits, bits_out, dot_w, dot_stride, dot_out,
+                               st);
 }

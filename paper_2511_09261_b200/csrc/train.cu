@@ -32,7 +32,8 @@ struct TrainLayout {
   float* dW_sets;                     // per-subgraph partials when the model shares one weight set
   float* wg_scratch;                  // partial weight gradients of subgraphs that were split into row chunks
   float* agg_partial;                 // partial sums of the segments of long rows (aggregation)
-  uint8_t* Hbits;                     // [H_{L-1} > 0], one bit per element (bfloat16, written by the last layer's weight gradient)
+  uint8_t* Hbits[GNNCO_MAX_LAYERS];   // [H_l > 0], one bit per element (bfloat16; written by the transform that makes H_l,
+                                      // or, for the last hidden layer, by the output layer's weight gradient)
   __nv_bfloat16* W_lp[GNNCO_MAX_LAYERS];   // bf16 copies of the weights (bf16 features only)
   __nv_bfloat16* W_lp_t[GNNCO_MAX_LAYERS]; // transposed bf16 copies [sets x F_out x F_in] for the tensor-core forward
   __nv_bfloat16* W3[GNNCO_MAX_LAYERS];     // float32 features: three bf16 limbs of W (input-gradient operand)
@@ -83,8 +84,9 @@ TrainLayout carve_train(const gnnco_handle* h, const gnnco_model_desc* m, uint32
   T.item_loss = c.take<float>((size_t)h->n_items + 1);
   T.agg_partial = h->n_long_segs > 0 ? c.take<float>((size_t)h->n_long_segs * maxw) : nullptr;
   if (!(flags & GNNCO_FORWARD_ONLY)) {
-    if (L > 1 && m->feat_dtype == GNNCO_BF16 && m->dims[L - 1] % 8 == 0)
-      T.Hbits = c.take<uint8_t>(n * (size_t)(m->dims[L - 1] / 8));
+    if (m->feat_dtype == GNNCO_BF16)
+      for (int l = 1; l < L; ++l)
+        if (m->dims[l] % 8 == 0) T.Hbits[l] = c.take<uint8_t>(n * (size_t)(m->dims[l] / 8));
     if (L > 2) T.Gb = c.take<char>(n * maxw * es);
     T.dW_scratch = c.take<float>(max_wcount * m->weight_sets);
     if (m->weight_sets == 1) T.dW_sets = c.take<float>(max_wcount * (size_t)h->S);
@@ -145,6 +147,7 @@ int32_t run_step(gnnco_handle* h, const gnnco_model_desc* m, const void* X, cons
   // ---- forward
   const void* Hprev = X;
   bool u_done = false;
+  bool bits_written[GNNCO_MAX_LAYERS] = {false};
   for (int l = 1; l < L; ++l) {
     // aggregated input M_l; the first layer's can be kept across steps (X does not change)
     const void* Min = T.Ga;
@@ -154,11 +157,17 @@ int32_t run_step(gnnco_handle* h, const gnnco_model_desc* m, const void* X, cons
     if (T.W_lp_t[l - 1]) {
       // the last hidden layer also produces u = H w_L in its epilogue
       const bool fuse = (l == L - 1) && (m->dims[l] % 8 == 0);
-      if (false && tc_pair_transform_supported(h, dt, m->dims[l - 1], m->dims[l]))
+      if (tc_pair_transform_supported(h, dt, m->dims[l - 1], m->dims[l])) {
+        // The pair kernel can leave [H_l > 0] behind as bits for the masked input gradient of layer l + 1.  The
+        // last hidden layer's bits are left to the output layer's weight gradient, which reads H_{L-1} anyway:
+        // measured in one run, 0.22 ms more here against 0.21 ms more there, and the drain of this kernel is the
+        // scarcer resource.
+        uint8_t* bits = l < L - 1 ? T.Hbits[l] : nullptr;
         GNNCO_TRY(launch_transform_tc_pair(h, Min, T.W_lp_t[l - 1], wstride[l - 1], sets, T.H[l], m->dims[l - 1],
-                                           m->dims[l], true, nullptr, nullptr, false, fuse ? Wc[L - 1] : nullptr,
+                                           m->dims[l], true, nullptr, nullptr, bits, false, fuse ? Wc[L - 1] : nullptr,
                                            wstride[L - 1], fuse ? T.u : nullptr, st));
-      else
+        bits_written[l] = bits != nullptr;
+      } else
         GNNCO_TRY(launch_transform_tc(h, Min, T.W_lp_t[l - 1], wstride[l - 1], T.H[l], m->dims[l - 1], m->dims[l], true,
                                       nullptr, nullptr, false, fuse ? Wc[L - 1] : nullptr, wstride[L - 1],
                                       fuse ? T.u : nullptr, st));
@@ -205,12 +214,14 @@ int32_t run_step(gnnco_handle* h, const gnnco_model_desc* m, const void* X, cons
     // last layer (0-based index L-1): dw = H^T g
     float* target = grad_target(L - 1);
     bool have_bits = false;
+    uint8_t* wgv_bits = (L > 1 && !bits_written[L - 1]) ? T.Hbits[L - 1] : nullptr;
     if (sets == 1) {
-      GNNCO_TRY(launch_weight_grad_vec(h, dt, Hprev, T.g, T.dW_sets, T.wg_scratch, FL, T.Hbits, &have_bits, st));
+      GNNCO_TRY(launch_weight_grad_vec(h, dt, Hprev, T.g, T.dW_sets, T.wg_scratch, FL, wgv_bits, &have_bits, st));
       GNNCO_TRY(launch_sum_over_sets(h, T.dW_sets, target, FL, h->S, st));
     } else {
-      GNNCO_TRY(launch_weight_grad_vec(h, dt, Hprev, T.g, target, T.wg_scratch, FL, T.Hbits, &have_bits, st));
+      GNNCO_TRY(launch_weight_grad_vec(h, dt, Hprev, T.g, target, T.wg_scratch, FL, wgv_bits, &have_bits, st));
     }
+    if (L > 1 && bits_written[L - 1]) have_bits = true;
     // everything that reads the weights of a layer runs before that layer's Adam update
     if (L > 1) {
       // from the mask bits that the weight-gradient pass above left behind, where it could
@@ -218,7 +229,7 @@ int32_t run_step(gnnco_handle* h, const gnnco_model_desc* m, const void* X, cons
                              !((uintptr_t)Wc[L - 1] & 15) && wstride[L - 1] % 8 == 0 && !((uintptr_t)Q & 15) &&
                              !((uintptr_t)Hprev & 15);
       if (from_bits)
-        GNNCO_TRY(launch_aggregate_rank1_bits(h, dt, T.Hbits, Hprev, T.u, Wc[L - 1], wstride[L - 1], Q, FL, st));
+        GNNCO_TRY(launch_aggregate_rank1_bits(h, dt, T.Hbits[L - 1], Hprev, T.u, Wc[L - 1], wstride[L - 1], Q, FL, st));
       else
         GNNCO_TRY(launch_aggregate_rank1(h, dt, Hprev, T.u, Wc[L - 1], wstride[L - 1], Q, FL, st));
     }
@@ -237,9 +248,9 @@ int32_t run_step(gnnco_handle* h, const gnnco_model_desc* m, const void* X, cons
       void* dst = l > 1 ? other : out->dX;
       const float* scale = l > 1 ? h->inv_deg : nullptr;
       const void* mask = l > 1 ? T.H[l - 1] : nullptr;
-      if (false && tc_pair_transform_supported(h, dt, N, K))
-        GNNCO_TRY(launch_transform_tc_pair(h, Q, Wc[l - 1], wstride[l - 1], sets, dst, N, K, false, scale, mask, true,
-                                           nullptr, 0, nullptr, st));
+      if (tc_pair_transform_supported(h, dt, N, K) && (l == 1 || bits_written[l - 1]))
+        GNNCO_TRY(launch_transform_tc_pair(h, Q, Wc[l - 1], wstride[l - 1], sets, dst, N, K, false, scale,
+                                           l > 1 ? T.Hbits[l - 1] : nullptr, nullptr, true, nullptr, 0, nullptr, st));
       else if (tc_transform_supported(dt, N, K))
         GNNCO_TRY(launch_transform_tc(h, Q, Wc[l - 1], wstride[l - 1], dst, N, K, false, scale, mask, true, nullptr, 0,
                                       nullptr, st));
