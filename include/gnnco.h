@@ -62,6 +62,14 @@ typedef enum { GNNCO_F32 = 0, GNNCO_BF16 = 1 } gnnco_dtype;
  * ax_cache; results are bit-identical to the plain step. */
 #define GNNCO_AX_STORE 4u
 #define GNNCO_AX_REUSE 8u
+/* bfloat16 features only.  A step that runs Adam writes, together with the updated master weights, the
+ * bfloat16 copies of them that the matrix products of the NEXT step read (inside the work area).  With
+ * GNNCO_WEIGHTS_UNTOUCHED the caller vouches that nobody but this library has written W[l] since the
+ * previous gnnco_train_step on this handle returned, and that the work area is the same one and has not
+ * been written either; the step then skips rounding the master weights again.  Without the flag (or when
+ * the previous step left no copies: first step, forward only, no optimiser, other buffers) the copies
+ * are rebuilt from W at the start of the step.  Results are bit-identical either way. */
+#define GNNCO_WEIGHTS_UNTOUCHED 16u
 
 typedef struct gnnco_handle gnnco_handle;
 

@@ -82,6 +82,11 @@ struct gnnco_handle {
   std::vector<int32_t> h_part_ptr;
   int64_t launches = 0;
   Profiler prof;
+  // bf16 copies of the weights that the last updating step left in its work area (GNNCO_WEIGHTS_UNTOUCHED):
+  // which master weights and which copies they belong to; fresh[l] says whether layer l's copies are current
+  const float* shadow_W[GNNCO_MAX_LAYERS] = {nullptr};
+  const void* shadow_copy[GNNCO_MAX_LAYERS] = {nullptr};
+  bool shadow_fresh[GNNCO_MAX_LAYERS] = {false};
   // long rows are aggregated on a side stream, concurrently with the short rows
   cudaStream_t side_stream = nullptr;
   cudaEvent_t ev_fork = nullptr, ev_join = nullptr;
@@ -185,6 +190,12 @@ int32_t launch_weight_grad_tc(gnnco_handle* h, const void* A, const void* G, flo
 // Wc[s][k][n] = bf16(W[s][k][n]) and Wt[s][n][k] = bf16(W[s][k][n]) in one pass over W
 int32_t launch_cast_both_bf16(gnnco_handle* h, const float* W, __nv_bfloat16* Wc, __nv_bfloat16* Wt, int K, int N,
                               int32_t sets, cudaStream_t st);
+// Adam on W [sets x K x N] that also writes both bf16 copies of the updated weights (for the next step)
+bool adam_cast_both_supported(const float* W, const float* m, const float* v, const float* g, const __nv_bfloat16* Wc,
+                              const __nv_bfloat16* Wt, int K, int N, int32_t sets);
+int32_t launch_adam_cast_both(gnnco_handle* h, float* W, float* m, float* v, const float* g, __nv_bfloat16* Wc,
+                              __nv_bfloat16* Wt, int K, int N, int32_t sets, float lr, float b1, float b2, float eps,
+                              float c1, float c2, const uint8_t* active, cudaStream_t st);
 // Wt[s][n][k] = bf16(W[s][k][n])
 int32_t launch_cast_transpose_bf16(gnnco_handle* h, const float* W, __nv_bfloat16* Wt, int K, int N, int32_t sets,
                                    cudaStream_t st);

@@ -500,6 +500,59 @@ __global__ void __launch_bounds__(256) cast_both_bf16_kernel(const float* __rest
   }
 }
 
+// Adam (same rule as adam_vec4_kernel) on W [sets][K][N] that also leaves behind the two bf16 copies of the
+// UPDATED weights which the next step's tensor-core transforms read (Wc [sets][K][N], Wt [sets][N][K]),
+// so that the next step need not read the master weights again just to round them.  A block owns a
+// 64 x 64 tile.  Subgraphs that are not being fine-tuned keep W, m and v bit for bit; their copies
+// are still written (from the unchanged W).
+__global__ void __launch_bounds__(256) adam_cast_both_kernel(float* __restrict__ W, float* __restrict__ m,
+                                                             float* __restrict__ v, const float* __restrict__ g,
+                                                             __nv_bfloat16* __restrict__ Wc, __nv_bfloat16* __restrict__ Wt,
+                                                             int K, int N, float lr, float b1, float b2, float eps,
+                                                             float inv_c1, float inv_c2,
+                                                             const uint8_t* __restrict__ active) {
+  __shared__ float tile[64][65];
+  const int64_t base = (int64_t)blockIdx.z * K * N;
+  const int k0 = blockIdx.y * 64, n0 = blockIdx.x * 64;
+  const int q = threadIdx.x & 15, r = threadIdx.x >> 4;   // 16 threads of four elements across, 16 rows per pass
+  const bool on = !active || active[blockIdx.z];
+#pragma unroll
+  for (int pass = 0; pass < 4; ++pass) {
+    const int k = r + 16 * pass;
+    const int64_t at = base + (int64_t)(k0 + k) * N + n0 + 4 * q;
+    float4 wq = *reinterpret_cast<const float4*>(W + at);
+    if (on) {
+      const float4 gq = __ldg(reinterpret_cast<const float4*>(g + at));
+      float4 mq = *reinterpret_cast<const float4*>(m + at), vq = *reinterpret_cast<const float4*>(v + at);
+      const float gs[4] = {gq.x, gq.y, gq.z, gq.w};
+      float* mp = reinterpret_cast<float*>(&mq);
+      float* vp = reinterpret_cast<float*>(&vq);
+      float* wp = reinterpret_cast<float*>(&wq);
+#pragma unroll
+      for (int c = 0; c < 4; ++c) {
+        mp[c] = b1 * mp[c] + (1.0f - b1) * gs[c];
+        vp[c] = b2 * vp[c] + (1.0f - b2) * gs[c] * gs[c];
+        wp[c] -= lr * (mp[c] * inv_c1) / (sqrtf(vp[c] * inv_c2) + eps);
+      }
+      *reinterpret_cast<float4*>(m + at) = mq;
+      *reinterpret_cast<float4*>(v + at) = vq;
+      *reinterpret_cast<float4*>(W + at) = wq;
+    }
+    __nv_bfloat162 lo = __floats2bfloat162_rn(wq.x, wq.y), hi = __floats2bfloat162_rn(wq.z, wq.w);
+    *reinterpret_cast<uint2*>(Wc + at) = make_uint2(*reinterpret_cast<uint32_t*>(&lo), *reinterpret_cast<uint32_t*>(&hi));
+    tile[k][4 * q + 0] = wq.x; tile[k][4 * q + 1] = wq.y; tile[k][4 * q + 2] = wq.z; tile[k][4 * q + 3] = wq.w;
+  }
+  __syncthreads();
+#pragma unroll
+  for (int pass = 0; pass < 4; ++pass) {
+    const int n = r + 16 * pass;
+    __nv_bfloat162 lo = __floats2bfloat162_rn(tile[4 * q + 0][n], tile[4 * q + 1][n]);
+    __nv_bfloat162 hi = __floats2bfloat162_rn(tile[4 * q + 2][n], tile[4 * q + 3][n]);
+    *reinterpret_cast<uint2*>(Wt + base + (int64_t)(n0 + n) * K + k0 + 4 * q) =
+        make_uint2(*reinterpret_cast<uint32_t*>(&lo), *reinterpret_cast<uint32_t*>(&hi));
+  }
+}
+
 }  // namespace
 
 bool tc_transform_supported(int dtype, int K, int N) {
@@ -561,6 +614,24 @@ int32_t launch_cast_transpose_bf16(gnnco_handle* h, const float* W, __nv_bfloat1
   dim3 grid((N + 31) / 32, (K + 31) / 32, sets);
   if (grid.y > 65535 || grid.z > 65535) return GNNCO_UNSUPPORTED;
   cast_transpose_bf16_kernel<<<grid, dim3(32, 8), 0, st>>>(W, Wt, K, N);
+  h->launches += 1;
+  GNNCO_LAUNCH_CHECK();
+  return GNNCO_OK;
+}
+
+bool adam_cast_both_supported(const float* W, const float* m, const float* v, const float* g, const __nv_bfloat16* Wc,
+                              const __nv_bfloat16* Wt, int K, int N, int32_t sets) {
+  return Wc && Wt && (K % 64) == 0 && (N % 64) == 0 && sets <= 65535 &&
+         !(((uintptr_t)W | (uintptr_t)m | (uintptr_t)v | (uintptr_t)g) & 15) && !(((uintptr_t)Wc | (uintptr_t)Wt) & 7);
+}
+
+int32_t launch_adam_cast_both(gnnco_handle* h, float* W, float* m, float* v, const float* g, __nv_bfloat16* Wc,
+                              __nv_bfloat16* Wt, int K, int N, int32_t sets, float lr, float b1, float b2, float eps,
+                              float c1, float c2, const uint8_t* active, cudaStream_t st) {
+  if (!adam_cast_both_supported(W, m, v, g, Wc, Wt, K, N, sets)) return GNNCO_UNSUPPORTED;
+  ProfScope prof_(h, K_ADAM, st);
+  adam_cast_both_kernel<<<dim3(N / 64, K / 64, sets), 256, 0, st>>>(W, m, v, g, Wc, Wt, K, N, lr, b1, b2, eps, 1.0f / c1,
+                                                                     1.0f / c2, active);
   h->launches += 1;
   GNNCO_LAUNCH_CHECK();
   return GNNCO_OK;

@@ -131,7 +131,12 @@ int32_t run_step(gnnco_handle* h, const gnnco_model_desc* m, const void* X, cons
     const int64_t wc = (int64_t)m->dims[l] * m->dims[l + 1];
     wstride[l] = sets == 1 ? 0 : wc;
     if (bf16) {
-      if (T.W_lp_t[l])
+      // copies that the previous step's Adam left behind are used as they are when the caller vouches for them
+      const bool fresh = (flags & GNNCO_WEIGHTS_UNTOUCHED) && h->shadow_fresh[l] && h->shadow_W[l] == m->W[l] &&
+                         h->shadow_copy[l] == (const void*)T.W_lp[l];
+      h->shadow_fresh[l] = false;
+      if (fresh) {
+      } else if (T.W_lp_t[l])
         GNNCO_TRY(launch_cast_both_bf16(h, m->W[l], T.W_lp[l], T.W_lp_t[l], m->dims[l], m->dims[l + 1], sets, st));
       else
         GNNCO_TRY(launch_cast_bf16(h, m->W[l], T.W_lp[l], wc * sets, st));
@@ -202,9 +207,23 @@ int32_t run_step(gnnco_handle* h, const gnnco_model_desc* m, const void* X, cons
   auto finish_layer = [&](int l, float* grad_sets_or_final) -> int32_t {
     // grad_sets_or_final holds [sets x ...] already reduced; run Adam on layer l (0-based)
     const int64_t wc = (int64_t)m->dims[l] * m->dims[l + 1] * sets;
-    if (opt) return launch_adam(h, m->W[l], opt->m[l], opt->v[l], grad_sets_or_final, wc, opt->lr, opt->beta1,
-                                opt->beta2, opt->eps, c1, c2, opt->active, wc / sets, st);
-    return GNNCO_OK;
+    if (!opt) return GNNCO_OK;
+    if (bf16 && T.W_lp_t[l] &&
+        adam_cast_both_supported(m->W[l], opt->m[l], opt->v[l], grad_sets_or_final, T.W_lp[l], T.W_lp_t[l], m->dims[l],
+                                 m->dims[l + 1], sets)) {
+      // everything that reads this layer's bf16 copies in this step has been launched before this point
+      int32_t rc2 = launch_adam_cast_both(h, m->W[l], opt->m[l], opt->v[l], grad_sets_or_final, T.W_lp[l], T.W_lp_t[l],
+                                          m->dims[l], m->dims[l + 1], sets, opt->lr, opt->beta1, opt->beta2, opt->eps,
+                                          c1, c2, opt->active, st);
+      if (rc2 == GNNCO_OK) {
+        h->shadow_W[l] = m->W[l];
+        h->shadow_copy[l] = T.W_lp[l];
+        h->shadow_fresh[l] = true;
+      }
+      return rc2;
+    }
+    return launch_adam(h, m->W[l], opt->m[l], opt->v[l], grad_sets_or_final, wc, opt->lr, opt->beta1, opt->beta2,
+                       opt->eps, c1, c2, opt->active, wc / sets, st);
   };
   // gradient target of layer l: the caller's buffer or the scratch
   auto grad_target = [&](int l) -> float* { return out->dW[l] ? out->dW[l] : T.dW_scratch; };
@@ -278,7 +297,8 @@ int32_t check_step_args(const gnnco_handle* h, const gnnco_model_desc* m, const 
                         uint32_t flags) {
   int32_t rc = check_model(h, m, true);
   if (rc != GNNCO_OK) return rc;
-  if (flags & ~(GNNCO_WANT_DX | GNNCO_FORWARD_ONLY | GNNCO_AX_STORE | GNNCO_AX_REUSE)) return GNNCO_INVALID_ARGUMENT;
+  if (flags & ~(GNNCO_WANT_DX | GNNCO_FORWARD_ONLY | GNNCO_AX_STORE | GNNCO_AX_REUSE | GNNCO_WEIGHTS_UNTOUCHED))
+    return GNNCO_INVALID_ARGUMENT;
   if ((flags & GNNCO_AX_STORE) && (flags & GNNCO_AX_REUSE)) return GNNCO_INVALID_ARGUMENT;
   if ((flags & (GNNCO_AX_STORE | GNNCO_AX_REUSE)) && m->L < 2) return GNNCO_INVALID_ARGUMENT;
   if (opt && !(flags & GNNCO_FORWARD_ONLY)) {

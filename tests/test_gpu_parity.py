@@ -235,6 +235,37 @@ def test_cached_first_aggregation_is_bit_identical(cfg):
         assert e.value.status == gnnco.INVALID_ARGUMENT
 
 
+def test_weight_copies_left_by_adam_are_bit_identical_to_fresh_ones():
+    """bfloat16 run: with GNNCO_WEIGHTS_UNTOUCHED the step reuses the bfloat16 weight copies that the
+    previous step's Adam kernel wrote; four steps (the third with only some subgraphs active, then a
+    forward-only step) equal the same steps without the flag bit for bit."""
+    import torch
+    import paper_2511_09261_b200 as gnnco
+    eu, ev, part = tiny_graph(700, 0.02, 5, seed=29)
+    n, S = _n_S(part)
+    graph = load_graph(n, eu, ev, part, S)
+    dims = [256, 256, 128, 1]
+    X = to_dev(si.round_to_bf16(rand_features(n, dims[0], 11).astype(np.float32)), torch.bfloat16)
+    active = to_dev(np.array([1, 0, 1, 1, 0], np.uint8))
+    runs = []
+    for reuse in (0, gnnco.WEIGHTS_UNTOUCHED):
+        W = [to_dev(si.round_to_bf16(w.astype(np.float32))) for w in rand_weights(dims, S, 13, scale=1.5)]
+        model = gnnco.Model(dims, W, gnnco.BF16)
+        opt = gnnco.Adam(model, lr=1e-2)
+        trace = []
+        for step in range(4):
+            opt.active = active if step == 2 else None
+            dX = torch.empty_like(X)
+            loss, p = graph.train_step(model, X, 2.0, 1.0, opt=opt, dX=dX, flags=gnnco.WANT_DX | reuse)
+            trace += [loss.clone(), p.clone(), dX]
+        loss, p = graph.train_step(model, X, 2.0, 1.0, flags=gnnco.FORWARD_ONLY | reuse)
+        runs.append(trace + [loss.clone(), p.clone()] + [t.clone() for t in W] + [t.clone() for t in opt.m])
+    torch.cuda.synchronize()
+    assert graph.async_status() == 0
+    for a, b in zip(*runs):
+        assert torch.equal(a, b)
+
+
 def test_host_variant_matches_device_variant():
     import torch
     import paper_2511_09261_b200 as gnnco
