@@ -367,6 +367,34 @@ def run_ours(args):
                       algo_GBs=round(s3_bytes / (s3_ms * 1e-3) / 1e9, 1),
                       note="gnnco_conflict_actions + gnnco_apply_actions on the last step's flags; "
                            "includes the binding's buffer allocations")
+        # ---- fine-tuning steps on the subgraphs that those actions name (Section 3.3): same model, penalty
+        # list and active flags from the glue above, GNNCO_ACTIVE_ONLY; not part of the headline
+        fine = None
+        n_active = graph.active_plan(ap["active"])
+        if n_active > 0:
+            opt.active = ap["active"]
+            ft_flags = gnnco.ACTIVE_ONLY | gnnco.WEIGHTS_UNTOUCHED
+            for _ in range(3):
+                graph.train_step(model, X, w.alpha, w.beta, 1.0, ap["pen"], opt, loss=loss, p=p, flags=ft_flags)
+            torch.cuda.synchronize()
+            f0, f1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            f0.record()
+            for _ in range(args.steps):
+                graph.train_step(model, X, w.alpha, w.beta, 1.0, ap["pen"], opt, loss=loss, p=p, flags=ft_flags)
+            f1.record()
+            torch.cuda.synchronize()
+            opt.active = None
+            act_np = ap["active"].cpu().numpy().astype(bool)
+            pp = arr["part_ptr"].cpu().numpy()
+            rp = arr["rowptr"].cpu().numpy()
+            act_rows = int((np.diff(pp)[act_np]).sum())
+            act_edges = int(((rp[pp[1:]] - rp[pp[:-1]])[act_np]).sum()) // 2
+            fms = f0.elapsed_time(f1) / args.steps
+            fine = dict(ms_per_step=round(fms, 4), active_subgraphs=n_active, subgraphs=w.S, active_rows=act_rows,
+                        active_intra_edges=act_edges, edges_per_s=act_edges / (fms * 1e-3),
+                        note="gnnco_active_plan + GNNCO_ACTIVE_ONLY steps (forward, objective with the penalty list, "
+                             "backward, Adam) on the subgraphs named by the base actions of the last decode")
+        stage3["fine_tune_step"] = fine
         del ca, ap
 
     # ---- the same step with the first layer's aggregated input kept across steps (X is a fixed
@@ -438,7 +466,8 @@ def run_ours(args):
                         parallelism="replicas only (no collective on the data path)" if world > 1 else "1 GPU",
                         partition_load_ms=round(load_ms, 3), edges_per_s_whole_graph=value * w.E / max(1, graph.E_in)),
             roofline=roofline, aggregate_kernels=agg, kernels=kern, cpu_baseline=cpu, clocks=clocks, e2e=e2e,
-            gpu_launches=int(launches), stage3_glue=stage3, cached_first_aggregation=cached)
+            gpu_launches=int(launches), stage3_glue=stage3, fine_tune_step=(stage3 or {}).get("fine_tune_step"),
+            cached_first_aggregation=cached)
         print(json.dumps(line))
     if dist is not None:
         dist.destroy_process_group()

@@ -70,6 +70,8 @@ typedef enum { GNNCO_F32 = 0, GNNCO_BF16 = 1 } gnnco_dtype;
  * the previous step left no copies: first step, forward only, no optimiser, other buffers) the copies
  * are rebuilt from W at the start of the step.  Results are bit-identical either way. */
 #define GNNCO_WEIGHTS_UNTOUCHED 16u
+/* Fine-tuning on the active subgraphs only; see gnnco_active_plan. */
+#define GNNCO_ACTIVE_ONLY 32u
 
 typedef struct gnnco_handle gnnco_handle;
 
@@ -207,6 +209,26 @@ int32_t gnnco_train_workspace_bytes(const gnnco_handle* h, const gnnco_model_des
 int32_t gnnco_train_step(gnnco_handle* h, const gnnco_model_desc* m, const void* X, const gnnco_objective* obj,
                          gnnco_adam_state* opt, const gnnco_train_out* out, uint32_t flags, void* ws,
                          size_t ws_bytes, void* stream);
+
+/* Fine-tuning steps that cost what the ACTIVE subgraphs cost (Section 3.3: a conflict is resolved by
+ * fine-tuning the model of one endpoint's subgraph; Algorithm 1, Stage 3 fine-tunes the subgraphs that
+ * the grouped actions name -- typically a small share of all subgraphs).
+ *
+ * gnnco_active_plan reads `active` (device, [S] uint8, e.g. the vector written by gnnco_apply_actions)
+ * and lays out, inside `plan_ws` (device, gnnco_active_plan_bytes bytes, 256-byte aligned, owned by the
+ * caller and kept until the plan is replaced or the handle destroyed), the work lists of the active
+ * subgraphs.  It synchronises `stream` (the flags must reach the host) and stores the number of active
+ * subgraphs in *active_count (host, may be NULL).  A new call replaces the plan.
+ *
+ * gnnco_train_step with GNNCO_ACTIVE_ONLY then runs forward, objective, backward and Adam over those
+ * subgraphs only.  It needs a plan, opt != NULL with opt->active equal to the pointer the plan was built
+ * from (the caller vouches that the flags have not changed since), per-subgraph weights and L >= 2.
+ * For every INACTIVE subgraph the step leaves loss[s], its rows of p, z and dX, its dW[l][s] and its
+ * weights and moments exactly as they were; for every active subgraph all results are bit-identical to
+ * those of a full step.  Not combined with GNNCO_AX_STORE / GNNCO_AX_REUSE. */
+int32_t gnnco_active_plan_bytes(const gnnco_handle* h, size_t* bytes);
+int32_t gnnco_active_plan(gnnco_handle* h, const uint8_t* active, void* plan_ws, size_t plan_bytes, void* stream,
+                          int32_t* active_count);
 
 /* Same step with HOST buffers for the per-step data: X_host [n x dims[0]] (feat_dtype,
  * new order; pinned memory recommended), pen_host [n] or NULL, loss_host [S], p_host [n].

@@ -19,7 +19,7 @@ OK = 0
 INVALID_ARGUMENT, OUT_OF_RANGE, NOT_SIMPLE_GRAPH, UNSUPPORTED, WORKSPACE_TOO_SMALL, CUDA_ERROR, INTERNAL = (
     -1, -2, -3, -4, -5, -6, -7)
 F32, BF16 = 0, 1
-WANT_DX, FORWARD_ONLY, AX_STORE, AX_REUSE, WEIGHTS_UNTOUCHED = 1, 2, 4, 8, 16
+WANT_DX, FORWARD_ONLY, AX_STORE, AX_REUSE, WEIGHTS_UNTOUCHED, ACTIVE_ONLY = 1, 2, 4, 8, 16, 32
 
 EXPORTS = [
     "gnnco_status_string", "gnnco_partition_workspace_bytes", "gnnco_partition_load", "gnnco_graph_info",
@@ -27,7 +27,7 @@ EXPORTS = [
     "gnnco_train_step_host", "gnnco_decode_boundary", "gnnco_async_status", "gnnco_launch_count", "gnnco_destroy",
     "gnnco_profile_begin", "gnnco_profile_end", "gnnco_objective_static", "gnnco_conflict_workspace_bytes",
     "gnnco_conflict_actions", "gnnco_apply_actions", "gnnco_gumbel_softmax", "gnnco_embedding_update",
-    "gnnco_repair_boundary", "gnnco_partition_quality",
+    "gnnco_repair_boundary", "gnnco_partition_quality", "gnnco_active_plan_bytes", "gnnco_active_plan",
 ]
 
 _vp, _i32, _i64, _u32, _f32, _sz = (ctypes.c_void_p, ctypes.c_int32, ctypes.c_int64, ctypes.c_uint32, ctypes.c_float,
@@ -115,6 +115,8 @@ def load_library(build_if_missing: bool = True):
     lib.gnnco_apply_actions.argtypes = [_vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp]
     lib.gnnco_partition_quality.argtypes = [_vp, _vp, _vp, _vp, _vp]
     lib.gnnco_repair_boundary.argtypes = [_vp, _vp, _vp, _vp, _vp]
+    lib.gnnco_active_plan_bytes.argtypes = [_vp, ctypes.POINTER(_sz)]
+    lib.gnnco_active_plan.argtypes = [_vp, _vp, _vp, _sz, _vp, ctypes.POINTER(_i32)]
     lib.gnnco_gumbel_softmax.argtypes = [_vp, _i32, _i32, _vp, _vp, _f32, _vp, _vp]
     lib.gnnco_embedding_update.argtypes = [_vp, _i32, _i32, _vp, _vp, _vp, _vp, _vp, _f32, _f32, _f32, _f32, _i64, _vp]
     for name in EXPORTS:
@@ -239,6 +241,8 @@ class PartitionedGraph:
         self._view = v
         self._ws = None
         self._ws_key = None
+        self._plan_ws = None
+        self._plan_active = None
 
     # ---- views of the persistent area as torch tensors (no copies)
     def _view_tensor(self, ptr: int, count: int, dtype):
@@ -363,6 +367,25 @@ class PartitionedGraph:
                                              _dptr(per_part), counts.data_ptr(), _stream_ptr(stream))
         _check(st, "gnnco_decode_boundary")
         return dict(x=x, viol=viol, per_part=per_part, counts=counts)
+
+    def active_plan(self, active, stream=None) -> int:
+        """``gnnco_active_plan``: work lists of the subgraphs with ``active[s] != 0`` (uint8 [S] device tensor,
+        kept alive by the caller while the plan is in use) for steps with ACTIVE_ONLY.  Synchronises the
+        stream; returns the number of active subgraphs."""
+        import torch
+        _require(active, torch.uint8, "active")
+        if tuple(active.shape) != (self.S,):
+            raise ValueError("active must be [S]")
+        need = _sz(0)
+        _check(self._lib.gnnco_active_plan_bytes(self._handle, ctypes.byref(need)), "gnnco_active_plan_bytes")
+        if self._plan_ws is None or self._plan_ws.numel() < need.value:
+            self._plan_ws = torch.empty(max(256, need.value), dtype=torch.uint8, device=self.device)
+        count = _i32(0)
+        _check(self._lib.gnnco_active_plan(self._handle, active.data_ptr(), self._plan_ws.data_ptr(),
+                                           self._plan_ws.numel(), _stream_ptr(stream), ctypes.byref(count)),
+               "gnnco_active_plan")
+        self._plan_active = active
+        return int(count.value)
 
     def conflict_actions(self, viol, p=None, want_action: bool = True, stream=None):
         """``gnnco_conflict_actions``.  Returns dict(conflict_idx, action, count): int32 [E_b]

@@ -149,9 +149,10 @@ __device__ __forceinline__ float row_sum(const float* __restrict__ val, const in
 __global__ void __launch_bounds__(256) output_forward(const float* __restrict__ u, const int32_t* __restrict__ rowptr,
                                                       const int32_t* __restrict__ colidx,
                                                       const float* __restrict__ inv_deg, float* __restrict__ z_out,
-                                                      float* __restrict__ p_out, int64_t n, const LongRows lr) {
-  const int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
-  const bool active = i < n;
+                                                      float* __restrict__ p_out, int64_t n, const LongRows lr,
+                                                      const RowChunks rc) {
+  int64_t i;
+  const bool active = chunk_row(rc, (int64_t)blockIdx.x * blockDim.x + threadIdx.x, n, i);
   int32_t r0 = 0, r1 = 0;
   if (active) { r0 = rowptr[i]; r1 = rowptr[i + 1]; }
   float s = row_sum(u, colidx, r0, r1, active, i, lr);
@@ -200,9 +201,10 @@ __global__ void __launch_bounds__(256) objective_items(const float* __restrict__
 }
 
 __global__ void sum_items_per_subgraph(const float* __restrict__ item_loss, const int32_t* __restrict__ part_item_ptr,
-                                       float* __restrict__ loss, int32_t S) {
+                                       float* __restrict__ loss, int32_t S, const uint8_t* __restrict__ only) {
   const int32_t s = blockIdx.x * blockDim.x + threadIdx.x;
   if (s >= S) return;
+  if (only && !only[s]) return;             // a step on the active subgraphs leaves the other losses alone
   float tot = 0.0f;
   for (int32_t k = part_item_ptr[s]; k < part_item_ptr[s + 1]; ++k) tot += item_loss[k];
   loss[s] = tot;
@@ -211,9 +213,10 @@ __global__ void sum_items_per_subgraph(const float* __restrict__ item_loss, cons
 __global__ void __launch_bounds__(256) output_backward(const float* __restrict__ t, const int32_t* __restrict__ rowptr,
                                                        const int32_t* __restrict__ colidx,
                                                        const float* __restrict__ inv_deg, float* __restrict__ g,
-                                                       float* __restrict__ coef, int64_t n, const LongRows lr) {
-  const int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
-  const bool active = i < n;
+                                                       float* __restrict__ coef, int64_t n, const LongRows lr,
+                                                       const RowChunks rc) {
+  int64_t i;
+  const bool active = chunk_row(rc, (int64_t)blockIdx.x * blockDim.x + threadIdx.x, n, i);
   int32_t r0 = 0, r1 = 0;
   if (active) { r0 = rowptr[i]; r1 = rowptr[i + 1]; }
   float s = row_sum(t, colidx, r0, r1, active, i, lr);
@@ -242,9 +245,9 @@ LongRows long_rows_prepass(gnnco_handle* h, const float* val, cudaStream_t st) {
 
 int32_t launch_output_forward(gnnco_handle* h, const float* u, float* z, float* p, cudaStream_t st) {
   ProfScope prof_(h, K_OUT_FWD, st);
-  unsigned grid = (unsigned)((h->n + 255) / 256);
+  unsigned grid = (unsigned)((linear_rows(h) + 255) / 256);
   const LongRows lr = long_rows_prepass(h, u, st);
-  output_forward<<<grid, 256, 0, st>>>(u, h->rowptr, h->colidx, h->inv_deg, z, p, h->n, lr);
+  output_forward<<<grid, 256, 0, st>>>(u, h->rowptr, h->colidx, h->inv_deg, z, p, h->n, lr, h->row_chunks);
   h->launches += 1;
   GNNCO_LAUNCH_CHECK();
   return GNNCO_OK;
@@ -257,7 +260,8 @@ int32_t launch_objective(gnnco_handle* h, const float* p, const float* pen, floa
   if (h->n_items > 0)
     objective_items<<<h->n_items, 256, 0, st>>>(p, pen, h->rowptr, h->colidx, h->inv_deg, h->item_row0, h->item_row1,
                                                 alpha, beta, lambda, item_loss, t, lr);
-  sum_items_per_subgraph<<<(h->S + 255) / 256, 256, 0, st>>>(item_loss, h->part_item_ptr, loss, h->S);
+  sum_items_per_subgraph<<<(h->S + 255) / 256, 256, 0, st>>>(item_loss, h->part_item_ptr, loss, h->S,
+                                                             h->row_chunks.row0 ? h->plan_active : nullptr);
   h->launches += 2;
   GNNCO_LAUNCH_CHECK();
   return GNNCO_OK;
@@ -265,9 +269,9 @@ int32_t launch_objective(gnnco_handle* h, const float* p, const float* pen, floa
 
 int32_t launch_output_backward(gnnco_handle* h, const float* t, float* g, float* coef, cudaStream_t st) {
   ProfScope prof_(h, K_OUT_BWD, st);
-  unsigned grid = (unsigned)((h->n + 255) / 256);
+  unsigned grid = (unsigned)((linear_rows(h) + 255) / 256);
   const LongRows lr = long_rows_prepass(h, t, st);
-  output_backward<<<grid, 256, 0, st>>>(t, h->rowptr, h->colidx, h->inv_deg, g, coef, h->n, lr);
+  output_backward<<<grid, 256, 0, st>>>(t, h->rowptr, h->colidx, h->inv_deg, g, coef, h->n, lr, h->row_chunks);
   h->launches += 1;
   GNNCO_LAUNCH_CHECK();
   return GNNCO_OK;
@@ -320,7 +324,7 @@ extern "C" int32_t gnnco_objective_static(gnnco_handle* h, const float* p, const
     objective_items<<<h->n_items, 256, 0, st>>>(p, obj->pen, h->rowptr, h->colidx, h->inv_deg, h->item_row0,
                                                 h->item_row1, obj->alpha, obj->beta, obj->lambda, item_loss, nullptr,
                                                 LongRows{});
-  sum_items_per_subgraph<<<(h->S + 255) / 256, 256, 0, st>>>(item_loss, h->part_item_ptr, loss, h->S);
+  sum_items_per_subgraph<<<(h->S + 255) / 256, 256, 0, st>>>(item_loss, h->part_item_ptr, loss, h->S, nullptr);
   h->launches += 2;
   GNNCO_LAUNCH_CHECK();
   return GNNCO_OK;

@@ -103,11 +103,13 @@ __global__ void __launch_bounds__(256) transform_fma(const TA* __restrict__ A, c
 template <typename TA>
 __global__ void __launch_bounds__(256) weight_grad_fma(const TA* __restrict__ A, const TA* __restrict__ G,
                                                        float* __restrict__ dW, int K, int N,
-                                                       const int32_t* __restrict__ part_ptr) {
+                                                       const int32_t* __restrict__ part_ptr,
+                                                       const uint8_t* __restrict__ only) {
   __shared__ __align__(16) float As[16][64 + 4];
   __shared__ __align__(16) float Gs[16][64 + 4];
   const int tid = threadIdx.x, tx = tid & 15, ty = tid >> 4;
   const int s = blockIdx.x, k0 = blockIdx.y * 64, n0 = blockIdx.z * 64;
+  if (only && !only[s]) return;               // a step on the active subgraphs only (uniform across the block)
   const int64_t ra = part_ptr[s], rb = part_ptr[s + 1];
   float acc[4][4];
 #pragma unroll
@@ -149,10 +151,10 @@ __global__ void __launch_bounds__(256) weight_grad_fma(const TA* __restrict__ A,
 template <typename TA, typename TW>
 __global__ void __launch_bounds__(256) gemv_rows(const TA* __restrict__ H, const TW* __restrict__ w, int64_t w_stride,
                                                  const int32_t* __restrict__ node_part, float* __restrict__ u,
-                                                 int64_t n, int F) {
+                                                 int64_t n, int F, const RowChunks rc) {
   const int lane = threadIdx.x & 31;
-  const int64_t row = (int64_t)blockIdx.x * 8 + (threadIdx.x >> 5);
-  if (row >= n) return;
+  int64_t row;
+  if (!chunk_row(rc, (int64_t)blockIdx.x * 8 + (threadIdx.x >> 5), n, row)) return;
   const TW* ws = w + (int64_t)node_part[row] * w_stride;
   float acc = 0.0f;
   for (int f = lane; f < F; f += 32) acc = fmaf(ld(H + row * F + f), ld(ws + f), acc);
@@ -424,13 +426,14 @@ int32_t launch_transform(gnnco_handle* h, int dtype, const void* A, const void* 
 int32_t launch_gemv(gnnco_handle* h, int dtype, const void* H, const void* w, int64_t w_stride, float* u, int F,
                     cudaStream_t stream) {
   ProfScope prof_(h, K_GEMV, stream);
-  unsigned grid = blocks_for(h->n, 8);
+  unsigned grid = blocks_for(linear_rows(h), 8);
   if (dtype == GNNCO_F32)
     gemv_rows<float, float><<<grid, 256, 0, stream>>>((const float*)H, (const float*)w, w_stride, h->node_part, u,
-                                                      h->n, F);
+                                                      h->n, F, h->row_chunks);
   else if (dtype == GNNCO_BF16)
     gemv_rows<__nv_bfloat16, __nv_bfloat16><<<grid, 256, 0, stream>>>(
-        (const __nv_bfloat16*)H, (const __nv_bfloat16*)w, w_stride, h->node_part, u, h->n, F);
+        (const __nv_bfloat16*)H, (const __nv_bfloat16*)w, w_stride, h->node_part, u, h->n, F,
+        h->row_chunks);
   else
     return GNNCO_UNSUPPORTED;
   h->launches += 1;
@@ -444,10 +447,12 @@ int32_t launch_weight_grad(gnnco_handle* h, int dtype, const void* A, const void
   dim3 grid(h->S, (K + 63) / 64, (N + 63) / 64);
   if (grid.y > 65535 || grid.z > 65535) return GNNCO_UNSUPPORTED;
   if (dtype == GNNCO_F32)
-    weight_grad_fma<float><<<grid, 256, 0, stream>>>((const float*)A, (const float*)G, dW, K, N, h->part_ptr);
+    weight_grad_fma<float><<<grid, 256, 0, stream>>>((const float*)A, (const float*)G, dW, K, N, h->part_ptr,
+                                                     h->row_chunks.row0 ? h->plan_active : nullptr);
   else if (dtype == GNNCO_BF16)
     weight_grad_fma<__nv_bfloat16><<<grid, 256, 0, stream>>>((const __nv_bfloat16*)A, (const __nv_bfloat16*)G, dW, K,
-                                                             N, h->part_ptr);
+                                                             N, h->part_ptr,
+                                                             h->row_chunks.row0 ? h->plan_active : nullptr);
   else
     return GNNCO_UNSUPPORTED;
   h->launches += 1;

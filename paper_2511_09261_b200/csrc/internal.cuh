@@ -50,6 +50,39 @@ struct Profiler {
   }
 };
 
+// Rows of a step that runs on SOME subgraphs only (fine-tuning, Section 3.3): the active subgraphs'
+// row ranges cut into chunks of at most 256 rows.  row0 == nullptr means "all n rows".  A kernel that
+// gives every block R rows (R divides 256) is launched with linear_rows() / R blocks and turns its linear
+// row index into a row with chunk_row().
+struct RowChunks {
+  const int32_t* row0 = nullptr;
+  const int32_t* rows = nullptr;
+  int32_t count = 0;
+};
+__device__ __forceinline__ bool chunk_row(const RowChunks& rc, int64_t linear, int64_t n, int64_t& row) {
+  if (!rc.row0) {
+    row = linear;
+    return linear < n;
+  }
+  const int64_t c = linear >> 8;
+  const int off = (int)(linear & 255);
+  if (c >= rc.count) return false;
+  row = (int64_t)rc.row0[c] + off;
+  return off < rc.rows[c];
+}
+
+// The per-graph work tables that the kernels of a step walk.  The handle holds the set for all
+// subgraphs; gnnco_active_plan builds a second set for the active subgraphs only, and a step with
+// GNNCO_ACTIVE_ONLY runs with that set swapped in.
+struct WorkSet {
+  int32_t *tile_row0 = nullptr, *tile_rows = nullptr, *pair_row0 = nullptr, *pair_rows = nullptr;
+  int32_t *item_row0 = nullptr, *item_row1 = nullptr, *part_item_ptr = nullptr;
+  int32_t *wg_begin = nullptr, *wg_end = nullptr, *wg_slot = nullptr;
+  int32_t *wg_mpart = nullptr, *wg_mfirst = nullptr, *wg_mcount = nullptr;
+  int32_t n_tiles = 0, n_pairs = 0, n_items = 0, n_wg_chunks = 0, n_wg_multi = 0;
+  RowChunks row_chunks;
+};
+
 struct gnnco_handle {
   int64_t n = 0, E = 0, E_in = 0, E_b = 0;
   int32_t S = 0, max_row = 0;
@@ -80,6 +113,12 @@ struct gnnco_handle {
   int32_t *wg_mpart = nullptr, *wg_mfirst = nullptr, *wg_mcount = nullptr;
   int32_t n_wg_chunks = 0, n_wg_slots = 0, n_wg_multi = 0;
   std::vector<int32_t> h_part_ptr;
+  // a step on the active subgraphs only: the rows it covers (nullptr: all), the plan built by
+  // gnnco_active_plan and the device flags it was built from
+  RowChunks row_chunks;
+  WorkSet plan;
+  const uint8_t* plan_active = nullptr;
+  int32_t plan_active_count = -1;                            // -1: no plan
   int64_t launches = 0;
   Profiler prof;
   // bf16 copies of the weights that the last updating step left in its work area (GNNCO_WEIGHTS_UNTOUCHED):
@@ -111,6 +150,20 @@ struct ProfScope {
 };
 
 static inline size_t align_up(size_t x, size_t a = 256) { return (x + a - 1) / a * a; }
+
+// rows a row-per-thread (or row-group-per-block) kernel has to cover in the running step
+static inline int64_t linear_rows(const gnnco_handle* h) {
+  return h->row_chunks.row0 ? (int64_t)h->row_chunks.count * 256 : h->n;
+}
+
+// Host side of the work tables: what partition_load uploads for all subgraphs and what
+// gnnco_active_plan uploads for the active ones (active == nullptr: all).  Defined in partition.cu.
+struct HostWorkTables {
+  std::vector<int32_t> t0, tr, p0, pr, i0, i1, pip, wb, we, wsl, mp, mf, mc, c0, cr;
+  int32_t n_wg_slots = 0;
+};
+void build_work_tables(const std::vector<int32_t>& part_ptr, int32_t S, int64_t n, int sm_count, const uint8_t* active,
+                       HostWorkTables& out);
 
 // A bump allocator over a caller-provided work area.
 struct Carver {

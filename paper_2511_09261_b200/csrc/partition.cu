@@ -398,6 +398,65 @@ bool valid_sizes(int64_t n, int64_t E, int32_t S) {
 
 }  // namespace
 
+// Work tables of the subgraphs with active[s] != 0 (all when active == nullptr), in subgraph order:
+//   tiles of 128 rows and double tiles of 256 rows of one subgraph (dense transforms), objective work items
+//   of kItemRows rows with the item range of every subgraph (empty for an inactive one), row chunks of
+//   256 rows, and the weight-gradient chunks: a subgraph is one chunk unless it is so long that too few
+//   blocks would be busy; then it is cut into runs of chunk_rows rows whose partial results meet in a
+//   scratch area (slot >= 0) and are summed in chunk order afterwards; slot = -(s+1) means "write
+//   subgraph s's result directly".  Scratch slots are numbered over ALL subgraphs, so a plan for some
+//   subgraphs uses the same slots as the full set.
+void build_work_tables(const std::vector<int32_t>& part_ptr, int32_t S, int64_t n, int sm_count, const uint8_t* active,
+                       HostWorkTables& o) {
+  o = HostWorkTables();
+  o.pip.assign((size_t)S + 1, 0);
+  const int64_t sms = sm_count > 0 ? sm_count : 148;
+  const int64_t per = (n + 4 * sms - 1) / (4 * sms);
+  int64_t chunk_rows = (per + 63) / 64 * 64;
+  if (chunk_rows < kWgChunkMinRows) chunk_rows = kWgChunkMinRows;
+  int32_t slots = 0;
+  for (int32_t s = 0; s < S; ++s) {
+    const int32_t a = part_ptr[s], b = part_ptr[s + 1];
+    const bool on = !active || active[s];
+    o.pip[s] = (int32_t)o.i0.size();
+    const bool split = b - a > chunk_rows;
+    int32_t first_slot = slots;
+    if (split) slots += (int32_t)((b - a + chunk_rows - 1) / chunk_rows);
+    if (!on) continue;
+    for (int32_t r = a; r < b; r += kGemmTileRows) {
+      o.t0.push_back(r);
+      o.tr.push_back(b - r < kGemmTileRows ? b - r : kGemmTileRows);
+    }
+    for (int32_t r = a; r < b; r += 2 * kGemmTileRows) {
+      o.p0.push_back(r);
+      o.pr.push_back(b - r < 2 * kGemmTileRows ? b - r : 2 * kGemmTileRows);
+    }
+    for (int32_t r = a; r < b; r += 256) {
+      o.c0.push_back(r);
+      o.cr.push_back(b - r < 256 ? b - r : 256);
+    }
+    for (int32_t r = a; r < b; r += kItemRows) {
+      o.i0.push_back(r);
+      o.i1.push_back(b - r < kItemRows ? b : r + kItemRows);
+    }
+    if (!split) {
+      o.wb.push_back(a); o.we.push_back(b); o.wsl.push_back(-(s + 1));
+    } else {
+      o.mp.push_back(s); o.mf.push_back(first_slot);
+      int32_t cnt = 0;
+      for (int64_t r = a; r < b; r += chunk_rows) {
+        o.wb.push_back((int32_t)r);
+        o.we.push_back((int32_t)(r + chunk_rows < b ? r + chunk_rows : b));
+        o.wsl.push_back(first_slot + cnt);
+        ++cnt;
+      }
+      o.mc.push_back(cnt);
+    }
+  }
+  o.pip[S] = (int32_t)o.i0.size();
+  o.n_wg_slots = slots;
+}
+
 extern "C" const char* gnnco_status_string(int32_t status) {
   switch (status) {
     case GNNCO_OK: return "ok";
@@ -523,57 +582,15 @@ extern "C" int32_t gnnco_partition_load(const gnnco_graph_desc* g, void* persist
   h->launches += 3;
   GNNCO_LAUNCH_CHECK();
 
-  // 5. host-built tables: dense-transform tiles and objective work items (from part_ptr)
-  std::vector<int32_t> t0, tr, p0, pr, i0, i1, pip((size_t)S + 1);
-  for (int32_t s = 0; s < S; ++s) {
-    int32_t a = h->h_part_ptr[s], b = h->h_part_ptr[s + 1];
-    pip[s] = (int32_t)i0.size();
-    // double tiles for the two-CTA transform: 256 rows of one subgraph, 128 for each CTA of a pair
-    for (int32_t r = a; r < b; r += 2 * kGemmTileRows) {
-      p0.push_back(r);
-      pr.push_back(b - r < 2 * kGemmTileRows ? b - r : 2 * kGemmTileRows);
-    }
-    for (int32_t r = a; r < b; r += kGemmTileRows) {
-      t0.push_back(r);
-      tr.push_back(b - r < kGemmTileRows ? b - r : kGemmTileRows);
-    }
-    for (int32_t r = a; r < b; r += kItemRows) {
-      i0.push_back(r);
-      i1.push_back(b - r < kItemRows ? b : r + kItemRows);
-    }
-  }
-  pip[S] = (int32_t)i0.size();
-  // weight-gradient chunks: a subgraph is one chunk unless it is so long that too few blocks
-  // would be busy; then it is cut into runs of chunk_rows rows whose partial results meet in a
-  // scratch area (slot >= 0) and are summed in chunk order afterwards.  slot = -(s+1) means
-  // "write subgraph s's result directly".
-  std::vector<int32_t> wb, we, wsl, mp, mf, mc;
-  {
-    int64_t per = (n + 4 * (int64_t)(h->sm_count > 0 ? h->sm_count : 148) - 1) / (4 * (int64_t)(h->sm_count > 0 ? h->sm_count : 148));
-    int64_t chunk_rows = (per + 63) / 64 * 64;
-    if (chunk_rows < kWgChunkMinRows) chunk_rows = kWgChunkMinRows;
-    int32_t slots = 0;
-    for (int32_t s = 0; s < S; ++s) {
-      int32_t a = h->h_part_ptr[s], b2 = h->h_part_ptr[s + 1];
-      if (b2 - a <= chunk_rows) {
-        wb.push_back(a); we.push_back(b2); wsl.push_back(-(s + 1));
-      } else {
-        mp.push_back(s); mf.push_back(slots);
-        int32_t cnt = 0;
-        for (int64_t r = a; r < b2; r += chunk_rows) {
-          wb.push_back((int32_t)r);
-          we.push_back((int32_t)(r + chunk_rows < b2 ? r + chunk_rows : b2));
-          wsl.push_back(slots++);
-          ++cnt;
-        }
-        mc.push_back(cnt);
-      }
-    }
-    h->n_wg_chunks = (int32_t)wb.size();
-    h->n_wg_slots = slots;
-    h->n_wg_multi = (int32_t)mp.size();
-    if (h->n_wg_chunks > P.max_chunks) return GNNCO_INTERNAL;
-  }
+  // 5. host-built tables: dense-transform tiles, objective work items, weight-gradient chunks (from part_ptr)
+  HostWorkTables tab;
+  build_work_tables(h->h_part_ptr, S, n, h->sm_count, nullptr, tab);
+  const std::vector<int32_t>&t0 = tab.t0, &tr = tab.tr, &p0 = tab.p0, &pr = tab.pr, &i0 = tab.i0, &i1 = tab.i1, &pip = tab.pip,
+                            &wb = tab.wb, &we = tab.we, &wsl = tab.wsl, &mp = tab.mp, &mf = tab.mf, &mc = tab.mc;
+  h->n_wg_chunks = (int32_t)wb.size();
+  h->n_wg_slots = tab.n_wg_slots;
+  h->n_wg_multi = (int32_t)mp.size();
+  if (h->n_wg_chunks > P.max_chunks) return GNNCO_INTERNAL;
   h->n_tiles = (int32_t)t0.size();
   h->n_pairs = (int32_t)p0.size();
   h->n_items = (int32_t)i0.size();

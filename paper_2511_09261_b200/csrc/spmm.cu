@@ -125,16 +125,17 @@ __global__ void __launch_bounds__(256) aggregate_vec(const T* __restrict__ in, T
                                                      const int32_t* __restrict__ colidx,
                                                      const float* __restrict__ scale, const T* __restrict__ mask,
                                                      const Rank1Args<T> r1, int64_t n, int F, int skip_long,
-                                                     int prefetch_blocks) {
+                                                     int prefetch_blocks, const RowChunks rc) {
   constexpr int VN = Vec<T>::N;
   constexpr int ROWS_PER_BLOCK = 256 / LPR;
   const int sub = threadIdx.x % LPR;
-  const int64_t row = (int64_t)blockIdx.x * ROWS_PER_BLOCK + threadIdx.x / LPR;
+  int64_t row;
+  const bool has_row = chunk_row(rc, (int64_t)blockIdx.x * ROWS_PER_BLOCK + threadIdx.x / LPR, n, row);
   // Blocks are dispatched roughly in index order, so the block `prefetch_blocks` further on
   // will run a few microseconds from now: ask for its rows and head records to be brought
   // into L2 (no data returns to the SM, nothing to wait for), so that its first round trip
   // is an L2 hit instead of a DRAM access.
-  if (threadIdx.x == 0 && prefetch_blocks > 0) {
+  if (threadIdx.x == 0 && prefetch_blocks > 0 && !rc.row0) {
     const int64_t r0 = ((int64_t)blockIdx.x + prefetch_blocks) * ROWS_PER_BLOCK;
     if (r0 + ROWS_PER_BLOCK <= n) {
       asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;" ::"l"(in + r0 * F),
@@ -156,7 +157,7 @@ __global__ void __launch_bounds__(256) aggregate_vec(const T* __restrict__ in, T
       }
     }
   }
-  if (row >= n) return;
+  if (!has_row) return;
   // the row's own features are requested before its CSR extent is known, so the two round
   // trips overlap
   float acc[VPL][VN];
@@ -299,14 +300,15 @@ __global__ void __launch_bounds__(256) aggregate_rank1_bits(const uint8_t* __res
                                                             const int4* __restrict__ row_head,
                                                             const int32_t* __restrict__ colidx,
                                                             const Rank1Args<T> r1, int64_t n, int F,
-                                                            int prefetch_blocks) {
+                                                            int prefetch_blocks, const RowChunks rc) {
   constexpr int VN = Vec<T>::N;
   constexpr int ROWS_PER_BLOCK = 256 / LPR;
   constexpr uint32_t PIECE = (1u << VN) - 1u;
   const int sub = threadIdx.x % LPR;
-  const int64_t row = (int64_t)blockIdx.x * ROWS_PER_BLOCK + threadIdx.x / LPR;
+  int64_t row;
+  const bool has_row = chunk_row(rc, (int64_t)blockIdx.x * ROWS_PER_BLOCK + threadIdx.x / LPR, n, row);
   const int64_t rb = F >> 3;                                   // bytes of bits per row
-  if (threadIdx.x == 0 && prefetch_blocks > 0) {               // see aggregate_vec
+  if (threadIdx.x == 0 && prefetch_blocks > 0 && !rc.row0) {   // see aggregate_vec
     const int64_t r0 = ((int64_t)blockIdx.x + prefetch_blocks) * ROWS_PER_BLOCK;
     if (r0 + ROWS_PER_BLOCK <= n) {
       asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;" ::"l"(row_head + r0),
@@ -317,7 +319,7 @@ __global__ void __launch_bounds__(256) aggregate_rank1_bits(const uint8_t* __res
         asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;" ::"l"(b0), "r"(nb) : "memory");
     }
   }
-  if (row >= n) return;
+  if (!has_row) return;
   // piece v of this lane: elements (v*LPR + sub)*VN .. +VN  ->  VN bits inside one byte
   int byte_of[VPL], shift_of[VPL];
 #pragma unroll
@@ -429,13 +431,14 @@ __global__ void __launch_bounds__(256) aggregate_rank1_bits_batch(const uint8_t*
                                                                   const int4* __restrict__ row_head,
                                                                   const int32_t* __restrict__ colidx,
                                                                   const Rank1Args<__nv_bfloat16> r1, int64_t n,
-                                                                  int skip_long, int prefetch_blocks) {
+                                                                  int skip_long, int prefetch_blocks,
+                                                                  const RowChunks rc) {
   using T = __nv_bfloat16;
   constexpr int F = NB * 8, VPL = NB / 32, Q = NB / 16;
   constexpr int kWarpBytes = 4 * 32 * NB + 7 * 32 * 4;       // own + two neighbours + tail bits, 7 words of per-row scalars
   extern __shared__ uint4 smem_r1b[];
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  if (threadIdx.x == 0 && prefetch_blocks > 0) {               // see aggregate_vec
+  if (threadIdx.x == 0 && prefetch_blocks > 0 && !rc.row0) {   // see aggregate_vec
     const int64_t r0 = ((int64_t)blockIdx.x + prefetch_blocks) * 256;
     if (r0 + 256 <= n) {
       asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;" ::"l"(row_head + r0), "r"(256u * 16u) : "memory");
@@ -448,8 +451,13 @@ __global__ void __launch_bounds__(256) aggregate_rank1_bits_batch(const uint8_t*
         asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;" ::"l"(r1.node_part + r0), "r"(1024u) : "memory");
     }
   }
-  const int64_t row0 = (int64_t)blockIdx.x * 256 + warp * 32;
-  if (row0 >= n) return;                                       // whole warp; no block-wide barrier below
+  // the warp's 32 consecutive rows: of the whole graph, or of one 256-row chunk of an active subgraph
+  int64_t row0 = (int64_t)blockIdx.x * 256 + warp * 32, row_end = n;
+  if (rc.row0) {
+    row0 = (int64_t)rc.row0[blockIdx.x] + warp * 32;
+    row_end = (int64_t)rc.row0[blockIdx.x] + rc.rows[blockIdx.x];
+  }
+  if (row0 >= row_end) return;                                 // whole warp; no block-wide barrier below
   uint8_t* wbase = reinterpret_cast<uint8_t*>(smem_r1b) + warp * kWarpBytes;
   uint8_t* sb = wbase;                                         // [3][32 rows][NB]: own, first, second neighbour
   uint8_t* tb = wbase + 3 * 32 * NB;                           // [32 neighbours][NB]
@@ -461,7 +469,7 @@ __global__ void __launch_bounds__(256) aggregate_rank1_bits_batch(const uint8_t*
   // ---- gather, lane = row
   {
     const int64_t row = row0 + lane;
-    const bool valid = row < n;
+    const bool valid = row < row_end;
     int4 head = make_int4(0, 0, 0, 0);
     float c_own = 0.0f, c0 = 0.0f, c1 = 0.0f;
     int32_t part = 0;
@@ -496,7 +504,7 @@ __global__ void __launch_bounds__(256) aggregate_rank1_bits_batch(const uint8_t*
   }
   __syncwarp();
   // ---- reduce, lane = VPL pieces of 8 features
-  const int rows_here = (int)min((int64_t)32, n - row0);
+  const int rows_here = (int)min((int64_t)32, row_end - row0);
   int cur_part = -1;
   float wf[VPL][8];                                            // this lane's pieces of the subgraph's weight vector
   for (int r = 0; r < rows_here; ++r) {
@@ -676,10 +684,10 @@ __global__ void __launch_bounds__(256) aggregate_any(const T* __restrict__ in, T
                                                      const int32_t* __restrict__ rowptr,
                                                      const int32_t* __restrict__ colidx,
                                                      const float* __restrict__ scale, const T* __restrict__ mask,
-                                                     const Rank1Args<T> r1, int64_t n, int F) {
+                                                     const Rank1Args<T> r1, int64_t n, int F, const RowChunks rc) {
   const int lane = threadIdx.x & 31;
-  const int64_t row = (int64_t)blockIdx.x * 8 + (threadIdx.x >> 5);
-  if (row >= n) return;
+  int64_t row;
+  if (!chunk_row(rc, (int64_t)blockIdx.x * 8 + (threadIdx.x >> 5), n, row)) return;
   const int32_t r0 = rowptr[row], r1_end = rowptr[row + 1];
   if constexpr (R1) {
     const float ci = r1.coef[row];
@@ -735,13 +743,13 @@ template <typename T, int LPR, int VPL, bool R1>
 void launch_vec(const T* in, T* out, gnnco_handle* h, const float* scale, const T* mask, const Rank1Args<T>& r1, int F,
                 cudaStream_t st) {
   constexpr int ROWS_PER_BLOCK = 256 / LPR;
-  const unsigned main_blocks = (unsigned)((h->n + ROWS_PER_BLOCK - 1) / ROWS_PER_BLOCK);
+  const unsigned main_blocks = (unsigned)((linear_rows(h) + ROWS_PER_BLOCK - 1) / ROWS_PER_BLOCK);
   // L2 prefetch distance: one full wave of resident blocks (8 per SM) ahead; pointless on small grids
   const int sms = h->sm_count > 0 ? h->sm_count : 148;
   const int pf_blocks = main_blocks > 4u * 8u * (unsigned)sms ? 8 * sms : 0;
   if (h->n_long == 0) {
     aggregate_vec<T, LPR, VPL, R1><<<main_blocks, 256, 0, st>>>(in, out, h->row_head, h->colidx, scale, mask, r1, h->n,
-                                                                F, 0, pf_blocks);
+                                                                F, 0, pf_blocks, h->row_chunks);
     return;
   }
   // A single warp walks a row of max_row entries in about max_row/4 dependent round trips of
@@ -755,12 +763,12 @@ void launch_vec(const T* in, T* out, gnnco_handle* h, const float* scale, const 
   const bool inline_first = stream_us > 3.0 * walk_us;
   if (inline_first) {
     aggregate_vec<T, LPR, VPL, R1><<<main_blocks, 256, 0, st>>>(in, out, h->row_head, h->colidx, scale, mask, r1, h->n,
-                                                                F, 0, pf_blocks);
+                                                                F, 0, pf_blocks, h->row_chunks);
     return;
   }
   const bool fork = fork_long_rows<T, LPR, VPL, R1>(h, in, out, scale, mask, r1, F, st);
   aggregate_vec<T, LPR, VPL, R1><<<main_blocks, 256, 0, st>>>(in, out, h->row_head, h->colidx, scale, mask, r1, h->n, F,
-                                                              1, pf_blocks);
+                                                              1, pf_blocks, h->row_chunks);
   if (fork) cudaStreamWaitEvent(st, h->ev_join, 0);
 }
 
@@ -786,8 +794,8 @@ int32_t aggregate_typed(gnnco_handle* h, const T* in, T* out, int F, const float
     }
   }
   if (!done) {
-    unsigned grid = (unsigned)((h->n + 7) / 8);
-    aggregate_any<T, R1><<<grid, 256, 0, st>>>(in, out, h->rowptr, h->colidx, scale, mask, r1, h->n, F);
+    unsigned grid = (unsigned)((linear_rows(h) + 7) / 8);
+    aggregate_any<T, R1><<<grid, 256, 0, st>>>(in, out, h->rowptr, h->colidx, scale, mask, r1, h->n, F, h->row_chunks);
   }
   h->launches += 1;
   GNNCO_LAUNCH_CHECK();
@@ -841,25 +849,28 @@ int32_t rank1_bits_typed(gnnco_handle* h, const uint8_t* bits, const T* H, T* ou
   const int sms = h->sm_count > 0 ? h->sm_count : 148;
 #define GNNCO_R1B(LPR, VPL)                                                                                      \
   do {                                                                                                           \
-    const unsigned blocks = (unsigned)((h->n + (256 / LPR) - 1) / (256 / LPR));                                  \
+    const unsigned blocks = (unsigned)((linear_rows(h) + (256 / LPR) - 1) / (256 / LPR));                        \
     const int pf = blocks > 4u * 8u * (unsigned)sms ? 8 * sms : 0;                                               \
-    aggregate_rank1_bits<T, LPR, VPL><<<blocks, 256, 0, st>>>(bits, out, h->row_head, h->colidx, r1, h->n, F, pf); \
+    aggregate_rank1_bits<T, LPR, VPL><<<blocks, 256, 0, st>>>(bits, out, h->row_head, h->colidx, r1, h->n, F, pf, \
+                                                              h->row_chunks);                                    \
   } while (0)
   if (F == 256 || F == 512) {
     // rows in batches of 32 per warp (see aggregate_rank1_bits_batch); long rows beside them
-    const unsigned blocks = (unsigned)((h->n + 255) / 256);
+    const unsigned blocks = (unsigned)((linear_rows(h) + 255) / 256);
     const int pf = blocks > 4u * 5u * (unsigned)sms ? 5 * sms : 0;      // one wave of resident blocks ahead
     const int skip = h->n_long > 0 ? 1 : 0;
     bool fork = false;
     if (F == 256) {
       constexpr int smem = 8 * (4 * 32 * 32 + 7 * 32 * 4);
       if (skip) fork = fork_long_rows<T, 32, 1, true>(h, H, out, nullptr, nullptr, r1, F, st);
-      aggregate_rank1_bits_batch<32><<<blocks, 256, smem, st>>>(bits, out, h->row_head, h->colidx, r1, h->n, skip, pf);
+      aggregate_rank1_bits_batch<32><<<blocks, 256, smem, st>>>(bits, out, h->row_head, h->colidx, r1, h->n, skip, pf,
+                                                                h->row_chunks);
     } else {
       constexpr int smem = 8 * (4 * 32 * 64 + 7 * 32 * 4);
       GNNCO_CUDA_TRY(cudaFuncSetAttribute(aggregate_rank1_bits_batch<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
       if (skip) fork = fork_long_rows<T, 32, 2, true>(h, H, out, nullptr, nullptr, r1, F, st);
-      aggregate_rank1_bits_batch<64><<<blocks, 256, smem, st>>>(bits, out, h->row_head, h->colidx, r1, h->n, skip, pf);
+      aggregate_rank1_bits_batch<64><<<blocks, 256, smem, st>>>(bits, out, h->row_head, h->colidx, r1, h->n, skip, pf,
+                                                                h->row_chunks);
     }
     if (fork) cudaStreamWaitEvent(st, h->ev_join, 0);
     h->launches += 1;

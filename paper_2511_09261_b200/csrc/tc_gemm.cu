@@ -503,8 +503,8 @@ __global__ void __launch_bounds__(256) cast_both_bf16_kernel(const float* __rest
 // Adam (same rule as adam_vec4_kernel) on W [sets][K][N] that also leaves behind the two bf16 copies of the
 // UPDATED weights which the next step's tensor-core transforms read (Wc [sets][K][N], Wt [sets][N][K]),
 // so that the next step need not read the master weights again just to round them.  A block owns a
-// 64 x 64 tile.  Subgraphs that are not being fine-tuned keep W, m and v bit for bit; their copies
-// are still written (from the unchanged W).
+// 64 x 64 tile.  Subgraphs that are not being fine-tuned are skipped: W, m and v stay bit for bit, and
+// their copies are current already (the step made or vouched for them before its first matrix product).
 __global__ void __launch_bounds__(256) adam_cast_both_kernel(float* __restrict__ W, float* __restrict__ m,
                                                              float* __restrict__ v, const float* __restrict__ g,
                                                              __nv_bfloat16* __restrict__ Wc, __nv_bfloat16* __restrict__ Wt,
@@ -515,13 +515,13 @@ __global__ void __launch_bounds__(256) adam_cast_both_kernel(float* __restrict__
   const int64_t base = (int64_t)blockIdx.z * K * N;
   const int k0 = blockIdx.y * 64, n0 = blockIdx.x * 64;
   const int q = threadIdx.x & 15, r = threadIdx.x >> 4;   // 16 threads of four elements across, 16 rows per pass
-  const bool on = !active || active[blockIdx.z];
+  if (active && !active[blockIdx.z]) return;                // uniform across the block
 #pragma unroll
   for (int pass = 0; pass < 4; ++pass) {
     const int k = r + 16 * pass;
     const int64_t at = base + (int64_t)(k0 + k) * N + n0 + 4 * q;
     float4 wq = *reinterpret_cast<const float4*>(W + at);
-    if (on) {
+    {
       const float4 gq = __ldg(reinterpret_cast<const float4*>(g + at));
       float4 mq = *reinterpret_cast<const float4*>(m + at), vq = *reinterpret_cast<const float4*>(v + at);
       const float gs[4] = {gq.x, gq.y, gq.z, gq.w};

@@ -115,9 +115,49 @@ TrainLayout carve_train(const gnnco_handle* h, const gnnco_model_desc* m, uint32
   return T;
 }
 
+int32_t run_step_on(gnnco_handle* h, const gnnco_model_desc* m, const void* X, const gnnco_objective* obj,
+                    gnnco_adam_state* opt, const gnnco_train_out* out, uint32_t flags, const TrainLayout& T,
+                    cudaStream_t st);
+
+WorkSet capture_work(const gnnco_handle* h) {
+  WorkSet w;
+  w.tile_row0 = h->tile_row0; w.tile_rows = h->tile_rows; w.pair_row0 = h->pair_row0; w.pair_rows = h->pair_rows;
+  w.item_row0 = h->item_row0; w.item_row1 = h->item_row1; w.part_item_ptr = h->part_item_ptr;
+  w.wg_begin = h->wg_begin; w.wg_end = h->wg_end; w.wg_slot = h->wg_slot;
+  w.wg_mpart = h->wg_mpart; w.wg_mfirst = h->wg_mfirst; w.wg_mcount = h->wg_mcount;
+  w.n_tiles = h->n_tiles; w.n_pairs = h->n_pairs; w.n_items = h->n_items; w.n_wg_chunks = h->n_wg_chunks;
+  w.n_wg_multi = h->n_wg_multi;
+  w.row_chunks = h->row_chunks;
+  return w;
+}
+
+void apply_work(gnnco_handle* h, const WorkSet& w) {
+  h->tile_row0 = w.tile_row0; h->tile_rows = w.tile_rows; h->pair_row0 = w.pair_row0; h->pair_rows = w.pair_rows;
+  h->item_row0 = w.item_row0; h->item_row1 = w.item_row1; h->part_item_ptr = w.part_item_ptr;
+  h->wg_begin = w.wg_begin; h->wg_end = w.wg_end; h->wg_slot = w.wg_slot;
+  h->wg_mpart = w.wg_mpart; h->wg_mfirst = w.wg_mfirst; h->wg_mcount = w.wg_mcount;
+  h->n_tiles = w.n_tiles; h->n_pairs = w.n_pairs; h->n_items = w.n_items; h->n_wg_chunks = w.n_wg_chunks;
+  h->n_wg_multi = w.n_wg_multi;
+  h->row_chunks = w.row_chunks;
+}
+
+// A step over all subgraphs, or (GNNCO_ACTIVE_ONLY) the same launch sequence with the plan's work tables
+// swapped in for its duration.
 int32_t run_step(gnnco_handle* h, const gnnco_model_desc* m, const void* X, const gnnco_objective* obj,
                  gnnco_adam_state* opt, const gnnco_train_out* out, uint32_t flags, const TrainLayout& T,
                  cudaStream_t st) {
+  if (!(flags & GNNCO_ACTIVE_ONLY)) return run_step_on(h, m, X, obj, opt, out, flags, T, st);
+  if (h->plan.row_chunks.count == 0) return GNNCO_OK;          // no active subgraph has a node: nothing to do
+  const WorkSet full = capture_work(h);
+  apply_work(h, h->plan);
+  const int32_t rc = run_step_on(h, m, X, obj, opt, out, flags, T, st);
+  apply_work(h, full);
+  return rc;
+}
+
+int32_t run_step_on(gnnco_handle* h, const gnnco_model_desc* m, const void* X, const gnnco_objective* obj,
+                    gnnco_adam_state* opt, const gnnco_train_out* out, uint32_t flags, const TrainLayout& T,
+                    cudaStream_t st) {
   const int L = m->L, dt = m->feat_dtype;
   const bool bf16 = dt == GNNCO_BF16;
   h->agg_partial = T.agg_partial;       // where this step's aggregations keep the segments of long rows
@@ -297,8 +337,14 @@ int32_t check_step_args(const gnnco_handle* h, const gnnco_model_desc* m, const 
                         uint32_t flags) {
   int32_t rc = check_model(h, m, true);
   if (rc != GNNCO_OK) return rc;
-  if (flags & ~(GNNCO_WANT_DX | GNNCO_FORWARD_ONLY | GNNCO_AX_STORE | GNNCO_AX_REUSE | GNNCO_WEIGHTS_UNTOUCHED))
+  if (flags & ~(GNNCO_WANT_DX | GNNCO_FORWARD_ONLY | GNNCO_AX_STORE | GNNCO_AX_REUSE | GNNCO_WEIGHTS_UNTOUCHED |
+                GNNCO_ACTIVE_ONLY))
     return GNNCO_INVALID_ARGUMENT;
+  if (flags & GNNCO_ACTIVE_ONLY) {
+    if (flags & (GNNCO_AX_STORE | GNNCO_AX_REUSE)) return GNNCO_INVALID_ARGUMENT;
+    if (h->plan_active_count < 0 || !opt || opt->active != h->plan_active || m->weight_sets != h->S || m->L < 2)
+      return GNNCO_INVALID_ARGUMENT;
+  }
   if ((flags & GNNCO_AX_STORE) && (flags & GNNCO_AX_REUSE)) return GNNCO_INVALID_ARGUMENT;
   if ((flags & (GNNCO_AX_STORE | GNNCO_AX_REUSE)) && m->L < 2) return GNNCO_INVALID_ARGUMENT;
   if (opt && !(flags & GNNCO_FORWARD_ONLY)) {

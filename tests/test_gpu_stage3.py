@@ -118,3 +118,94 @@ def test_fine_tune_updates_active_subgraphs_only():
     with pytest.raises(gnnco.GnncoError) as e:
         graph.train_step(shared, Xd, 2.0, 1.0, opt=opt2)
     assert e.value.status == gnnco.INVALID_ARGUMENT
+
+
+@pytest.mark.parametrize("dtype,dims,n,S", [("f32", [48, 24, 1], 900, 7), ("f32", [128, 128, 64, 1], 3000, 9),
+                                            ("bf16", [256, 256, 256, 1], 6000, 11), ("bf16", [64, 32, 1], 700, 5)])
+def test_active_only_step_equals_the_full_step_on_active_subgraphs(dtype, dims, n, S):
+    """A fine-tuning step restricted to the active subgraphs (gnnco_active_plan + GNNCO_ACTIVE_ONLY): loss, p, z,
+    dW, dX and the updated weights and moments of every ACTIVE subgraph are bit-identical to those of a full
+    step with the same Adam mask; everything that belongs to an inactive subgraph keeps the value it had
+    before the step (checked with canaries); with every subgraph active the step equals the plain one."""
+    import torch
+    import paper_2511_09261_b200 as gnnco
+    from helpers import tiny_graph, rand_weights, rand_features
+    eu, ev, part = tiny_graph(n, 8.0 / n, S, seed=41)
+    part[part == 2] = 3                                         # an empty subgraph
+    graph = load_graph(n, eu, ev, part, S)
+    pp = graph.arrays()["part_ptr"].cpu().numpy()
+    bf16 = dtype == "bf16"
+    tdt = torch.bfloat16 if bf16 else torch.float32
+    X = rand_features(n, dims[0], 3).astype(np.float32)
+    X = to_dev(si.round_to_bf16(X) if bf16 else X, tdt)
+    pen = to_dev((si.uniform01(5, 0, n) < 0.2).astype(np.float32))
+    L = len(dims) - 1
+    for flags_np in (np.array([(s * 7 + 3) % 3 == 0 for s in range(S)], np.uint8), np.ones(S, np.uint8),
+                     np.zeros(S, np.uint8)):
+        active = to_dev(flags_np)
+        outs = []
+        for only in (False, True):
+            W = [to_dev(w.astype(np.float32)) for w in rand_weights(dims, S, 13, scale=1.5)]
+            model = gnnco.Model(dims, W, gnnco.BF16 if bf16 else gnnco.F32)
+            opt = gnnco.Adam(model, lr=1e-2)
+            opt.active = active
+            # one full step first so that the Adam moments are not zero, then the step under test
+            graph.train_step(model, X, 2.0, 1.0, 0.5, pen, opt)
+            canary = 1024.0
+            loss = torch.full((S,), canary, device=X.device)
+            p = torch.full((n,), canary, device=X.device)
+            z = torch.full((n,), canary, device=X.device)
+            dW = [torch.full_like(w, canary) for w in W]
+            dX = torch.full_like(X, canary)
+            flags = gnnco.WANT_DX
+            if only:
+                assert graph.active_plan(active) == int(flags_np.sum())
+                flags |= gnnco.ACTIVE_ONLY
+            graph.train_step(model, X, 2.0, 1.0, 0.5, pen, opt, loss=loss, p=p, z=z, dW=dW, dX=dX, flags=flags)
+            torch.cuda.synchronize()
+            assert graph.async_status() == 0
+            outs.append(dict(loss=loss, p=p, z=z, dW=dW, dX=dX, W=[w.clone() for w in W], m=[t.clone() for t in opt.m],
+                             v=[t.clone() for t in opt.v]))
+        full, act = outs
+        for s in range(S):
+            lo, hi = int(pp[s]), int(pp[s + 1])
+            if flags_np[s] and hi > lo:
+                assert torch.equal(full["loss"][s], act["loss"][s])
+                for key in ("p", "z", "dX"):
+                    assert torch.equal(full[key][lo:hi], act[key][lo:hi]), (key, s)
+                for l in range(L):
+                    assert torch.equal(full["dW"][l][s], act["dW"][l][s]), ("dW", l, s)
+            elif not flags_np[s]:
+                assert float(act["loss"][s]) == 1024.0
+                for key in ("p", "z", "dX"):
+                    assert bool((act[key][lo:hi].float() == 1024.0).all()), (key, s)
+                for l in range(L):
+                    assert bool((act["dW"][l][s] == 1024.0).all())
+            for l in range(L):
+                for key in ("W", "m", "v"):
+                    assert torch.equal(full[key][l][s], act[key][l][s]), (key, l, s)
+
+
+def test_active_only_needs_a_matching_plan():
+    import torch
+    import paper_2511_09261_b200 as gnnco
+    from helpers import tiny_graph, rand_weights, rand_features
+    n, S, dims = 300, 4, [16, 8, 1]
+    eu, ev, part = tiny_graph(n, 0.03, S, seed=43)
+    graph = load_graph(n, eu, ev, part, S)
+    X = to_dev(rand_features(n, dims[0], 3).astype(np.float32))
+    W = [to_dev(w.astype(np.float32)) for w in rand_weights(dims, S, 13)]
+    model = gnnco.Model(dims, W)
+    opt = gnnco.Adam(model, lr=1e-2)
+    opt.active = to_dev(np.ones(S, np.uint8))
+    with pytest.raises(gnnco.GnncoError) as e:                  # no plan yet
+        graph.train_step(model, X, 2.0, 1.0, opt=opt, flags=gnnco.ACTIVE_ONLY)
+    assert e.value.status == gnnco.INVALID_ARGUMENT
+    graph.active_plan(opt.active)
+    graph.train_step(model, X, 2.0, 1.0, opt=opt, flags=gnnco.ACTIVE_ONLY)
+    opt.active = to_dev(np.ones(S, np.uint8))                   # other flags than the plan's
+    with pytest.raises(gnnco.GnncoError) as e:
+        graph.train_step(model, X, 2.0, 1.0, opt=opt, flags=gnnco.ACTIVE_ONLY)
+    assert e.value.status == gnnco.INVALID_ARGUMENT
+    with pytest.raises(gnnco.GnncoError):                       # no optimiser
+        graph.train_step(model, X, 2.0, 1.0, flags=gnnco.ACTIVE_ONLY)
