@@ -57,6 +57,14 @@ MUTATIONS = {
     "bf16 storage also rounds the output layer's aggregate": ("if (store_bf16 && l < L)", "if (store_bf16)"),
     "bf16 storage leaves the activation unrounded":
         ("if (store_bf16)\n          for (int32_t h = 0; h < fo; ++h) hr[h] = round_bf16(hr[h]);", ";"),
+    "Louvain: ties go to the highest community id":
+        ("if (sc > best_score || (sc == best_score && best != own && c < best))", "if (sc > best_score || (sc == best_score && best != own && c > best))"),
+    "Louvain: two single nodes may swap": (" && !(size[own] == 1 && size[best] == 1 && best > own)) {\n      next[a] = best;", ") {\n      next[a] = best;"),
+    "Louvain: the node's own degree stays in its community's total":
+        ("const int64_t own_score = two_m * kin[own] - (tot[own] - k[a]) * k[a];", "const int64_t own_score = two_m * kin[own] - tot[own] * k[a];"),
+    "Louvain: gain without the factor 2m": ("int64_t sc = two_m * kin[c] - tot[c] * k[a];", "int64_t sc = kin[c] - tot[c] * k[a];"),
+    "Louvain: a sweep that lowers Q is kept": ("if (q_new <= qnum) break;", "if (q_new <= qnum && 0) break;"),
+    "Louvain: internal weight counted once in Q": ("in2[comm[a]] += 2 * g->loop[a];", "in2[comm[a]] += g->loop[a];"),
     "inv_deg without the +1": ("inv_deg[i] = 1.0f / (float)(hi - lo + 1);", "inv_deg[i] = 1.0f / (float)(hi - lo > 0 ? hi - lo : 1);"),
 }
 
@@ -80,6 +88,13 @@ BATTERY = [
     lambda: pins.test_conflict_list_base_action_and_penalty_brute_force(2),
     lambda: pins.test_repair_removes_exactly_the_chosen_nodes_brute_force(1),
     lambda: pins.test_partition_quality_matches_networkx_and_the_pairwise_definition(30, 0.2, 4, 1),
+    lambda: pins.test_louvain_sweep_picks_the_brute_force_best_community(12, 0.3, 2),
+    lambda: pins.test_louvain_sweep_picks_the_brute_force_best_community(11, 0.5, 3),
+    pins.test_eq2_gain_is_what_the_sweep_compares,
+    lambda: pins.test_louvain_level_keeps_a_sweep_only_if_exact_modularity_rises(8, 0.3, 5),
+    lambda: pins.test_louvain_level_keeps_a_sweep_only_if_exact_modularity_rises(12, 0.3, 7),
+    pins.test_louvain_recovers_planted_blocks_and_reports_their_exact_modularity,
+    pins.test_louvain_small_cases_by_hand,
     pins.test_round_bf16_is_exact_round_to_nearest_even,
     lambda: pins.test_bf16_storage_forward_matches_dense_definition_with_rounding_written_out([7, 5, 3, 1], False),
     pins.test_bf16_storage_hidden_preactivations_and_output_layer_keep_full_precision,
@@ -101,7 +116,7 @@ def test_a_pin_fails_when_the_oracle_is_mutated(name, tmp_path, monkeypatch):
     mutant = ctypes.CDLL(lib_path)
     for fn in ("oracle_bookkeeping", "oracle_subgraph_step", "oracle_train_step", "oracle_adam", "oracle_decode",
                "oracle_conflict_list", "oracle_base_action", "oracle_apply_actions", "oracle_repair", "oracle_partition_quality",
-               "oracle_round_bf16"):
+               "oracle_round_bf16", "oracle_louvain", "oracle_louvain_sweep"):
         getattr(mutant, fn).argtypes = getattr(real, fn).argtypes
         getattr(mutant, fn).restype = getattr(real, fn).restype
     monkeypatch.setattr(oracle, "_lib", mutant)

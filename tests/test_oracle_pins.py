@@ -430,6 +430,160 @@ def test_sigmoid_chain_identity_for_one_layer():
     np.testing.assert_allclose(r["dW"][0][0][:, 0], X.T @ Ahat.T @ dz, rtol=1e-11, atol=1e-13)
 
 
+# ------------------------------------------------------- Louvain partitioning (Section 3.1)
+def _exact_modularity(n, edges, comm):
+    """Q of Eq. 1's terms, sum_c [ Sigma_in(c)/2m - (Sigma_tot(c)/2m)^2 ] with Sigma_in counted from both ends,
+    as an exact fraction, straight from the edge list."""
+    two_m = 2 * len(edges)
+    if two_m == 0:
+        return Fraction(0)
+    deg = [0] * n
+    for a, b in edges:
+        deg[a] += 1
+        deg[b] += 1
+    q = Fraction(0)
+    for c in set(comm):
+        inside = sum(2 for a, b in edges if comm[a] == c and comm[b] == c)
+        tot = sum(deg[i] for i in range(n) if comm[i] == c)
+        q += Fraction(inside, two_m) - Fraction(tot, two_m) ** 2
+    return q
+
+
+def _brute_force_sweep(n, edges, comm):
+    """Every node's move by exhaustive evaluation: the change of the exact modularity when the node alone is
+    re-assigned, over its own and its neighbours' communities."""
+    nbrs = [set() for _ in range(n)]
+    for a, b in edges:
+        nbrs[a].add(b)
+        nbrs[b].add(a)
+    size = {c: comm.count(c) for c in set(comm)}
+    nxt = list(comm)
+    for i in range(n):
+        own = comm[i]
+        alone = list(comm)
+        alone[i] = -1                                            # the node taken out of its community
+        base = _exact_modularity(n, edges, alone)
+        gain = {}
+        for c in {comm[j] for j in nbrs[i]} | {own}:
+            trial = list(comm)
+            trial[i] = c
+            gain[c] = _exact_modularity(n, edges, trial) - base
+        best = own
+        for c in sorted(gain):
+            if c != own and (gain[c] > gain[best] or (gain[c] == gain[best] and best != own and c < best)):
+                best = c
+        if best != own and gain[best] > gain[own] and not (size[own] == 1 and size[best] == 1 and best > own):
+            nxt[i] = best
+    return nxt
+
+
+@pytest.mark.parametrize("n,p,seed", [(9, 0.4, 1), (12, 0.3, 2), (11, 0.5, 3), (12, 0.2, 4), (10, 0.35, 5)])
+def test_louvain_sweep_picks_the_brute_force_best_community(n, p, seed):
+    eu, ev = si.erdos_renyi(n, p, seed)
+    edges = list(zip(eu.tolist(), ev.tolist()))
+    vectors = [list(range(n)),                                                    # every node alone
+               (si.u64(seed + 50, 0, n) % np.uint64(3)).astype(int).tolist(),     # three random communities
+               [i // 2 * 2 for i in range(n)]]                                    # pairs, ids with gaps
+    for comm in vectors:
+        got = oracle.louvain_sweep(n, eu, ev, np.array(comm, np.int32))
+        want = _brute_force_sweep(n, edges, comm)
+        assert got["next"].tolist() == want, (comm, got["next"].tolist(), want)
+        assert got["moves"] == sum(1 for a, b in zip(comm, want) if a != b)
+
+
+def test_eq2_gain_is_what_the_sweep_compares():
+    # the integer score of the sweep is Eq. 2 times 2 m^2: both rank the candidate communities alike, and the
+    # difference of two scores is the exact change of Q times 2 m^2 ... checked through single applied moves
+    n = 12
+    eu, ev = si.erdos_renyi(n, 0.35, 9)
+    edges = list(zip(eu.tolist(), ev.tolist()))
+    m = len(edges)
+    comm = (si.u64(77, 0, n) % np.uint64(4)).astype(int).tolist()
+    deg = np.bincount(np.concatenate([eu, ev]), minlength=n)
+    nxt = oracle.louvain_sweep(n, eu, ev, np.array(comm, np.int32))["next"].tolist()
+    moved = [i for i in range(n) if nxt[i] != comm[i]]
+    assert moved
+    for i in moved:
+        one = list(comm)
+        one[i] = nxt[i]
+        dq = _exact_modularity(n, edges, one) - _exact_modularity(n, edges, comm)
+        assert dq > 0                                           # a single applied move never lowers Q
+        k_in_new = sum(1 for a, b in edges if (a == i and comm[b] == nxt[i]) or (b == i and comm[a] == nxt[i]))
+        k_in_old = sum(1 for a, b in edges if (a == i and comm[b] == comm[i] and b != i) or (b == i and comm[a] == comm[i] and a != i))
+        tot_new = sum(int(deg[j]) for j in range(n) if comm[j] == nxt[i])
+        tot_old = sum(int(deg[j]) for j in range(n) if comm[j] == comm[i] and j != i)
+        eq2 = lambda k_in, tot: Fraction(k_in, m) - Fraction(tot * int(deg[i]), 2 * m * m)
+        assert dq == eq2(k_in_new, tot_new) - eq2(k_in_old, tot_old)
+
+
+def test_louvain_recovers_planted_blocks_and_reports_their_exact_modularity():
+    import networkx as nx
+    blocks, size = 6, 30
+    G = nx.planted_partition_graph(blocks, size, 0.5, 0.004, seed=5)
+    e = np.array(G.edges(), dtype=np.int32)
+    n = blocks * size
+    r = oracle.louvain(n, e[:, 0].copy(), e[:, 1].copy())
+    assert r["S"] == blocks
+    truth = np.arange(n) // size
+    # same partition up to the names of the parts; parts are numbered 0..S-1
+    pairs = set(zip(truth.tolist(), r["part"].tolist()))
+    assert len(pairs) == blocks and sorted(set(r["part"].tolist())) == list(range(blocks))
+    comms = [set(np.where(r["part"] == s)[0].tolist()) for s in range(r["S"])]
+    np.testing.assert_allclose(r["Q"], nx.community.modularity(G, comms), rtol=1e-12)
+    assert Fraction(r["qnum"], r["two_m"] ** 2) == _exact_modularity(n, [tuple(x) for x in e.tolist()], r["part"].tolist())
+    q = oracle.partition_quality(e[:, 0].copy(), e[:, 1].copy(), r["part"], r["S"])
+    np.testing.assert_allclose(q["Q"], r["Q"], rtol=1e-12)
+
+
+def test_louvain_small_cases_by_hand():
+    # no edges: nobody moves
+    r = oracle.louvain(5, np.zeros(0, np.int32), np.zeros(0, np.int32))
+    assert r["S"] == 5 and r["part"].tolist() == [0, 1, 2, 3, 4] and r["levels"] == 0 and r["qnum"] == 0
+    # one edge: the higher-numbered end joins the lower one (two single nodes never swap), Q goes from -1/2 to 0
+    r = oracle.louvain(2, np.array([1], np.int32), np.array([0], np.int32))
+    assert r["S"] == 1 and r["part"].tolist() == [0, 0] and r["qnum"] == 0
+    # two triangles joined by one edge: the two triangles, Q = 2 * (6/14 - (7/14)^2) = 5/14
+    eu = np.array([0, 1, 2, 3, 4, 5, 2], np.int32)
+    ev = np.array([1, 2, 0, 4, 5, 3, 3], np.int32)
+    r = oracle.louvain(6, eu, ev)
+    assert r["part"].tolist() == [0, 0, 0, 1, 1, 1]
+    assert Fraction(r["qnum"], r["two_m"] ** 2) == Fraction(5, 14)
+    # a sweep that lowers Q is undone: the result is never worse than what it started from
+    for seed in (1, 2, 3):
+        eu, ev = si.erdos_renyi(60, 0.08, seed)
+        r = oracle.louvain(60, eu, ev)
+        edges = list(zip(eu.tolist(), ev.tolist()))
+        assert Fraction(r["qnum"], r["two_m"] ** 2) == _exact_modularity(60, edges, r["part"].tolist())
+        assert Fraction(r["qnum"], r["two_m"] ** 2) > _exact_modularity(60, edges, list(range(60)))
+        bound = oracle.louvain(60, eu, ev, max_levels=1, max_sweeps=1)
+        assert bound["qnum"] <= r["qnum"]
+
+
+@pytest.mark.parametrize("n,p,seed", [(8, 0.2, 1), (8, 0.3, 5), (8, 0.4, 1), (12, 0.3, 7), (16, 0.2, 3)])
+def test_louvain_level_keeps_a_sweep_only_if_exact_modularity_rises(n, p, seed):
+    # first level replayed from outside: frozen-state sweeps, each kept only when the exact modularity of
+    # the whole assignment rises strictly (synchronous moves can lower it; these graphs have such a sweep)
+    eu, ev = si.erdos_renyi(n, p, seed)
+    edges = list(zip(eu.tolist(), ev.tolist()))
+    comm = list(range(n))
+    q = _exact_modularity(n, edges, comm)
+    rejected = False
+    for _ in range(64):
+        nxt = oracle.louvain_sweep(n, eu, ev, np.array(comm, np.int32))
+        if nxt["moves"] == 0:
+            break
+        q2 = _exact_modularity(n, edges, nxt["next"].tolist())
+        if q2 <= q:
+            rejected = True
+            break
+        comm, q = nxt["next"].tolist(), q2
+    r = oracle.louvain(n, eu, ev, max_levels=1)
+    rank = {c: k for k, c in enumerate(sorted(set(comm)))}
+    assert r["part"].tolist() == [rank[c] for c in comm]
+    assert Fraction(r["qnum"], r["two_m"] ** 2) == q
+    assert rejected or (n, p, seed) == (16, 0.2, 3)
+
+
 # ------------------------------------------------- bfloat16-storage mode of the oracle
 def _exact_bf16_of_float32(f):
     """Nearest bfloat16 (8 significant bits, float32's exponent range, ties to even, overflow
