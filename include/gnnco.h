@@ -188,6 +188,28 @@ int32_t gnnco_graph_info(const gnnco_handle* h, gnnco_graph_view* out);
  * integers are exact.  Asynchronous on `stream`. */
 int32_t gnnco_partition_quality(gnnco_handle* h, int64_t* in_edges, int64_t* tot, double* Q, void* stream);
 
+/* Louvain partitioning (Section 3.1, Eqs. 1-2): the subgraphs that the method trains on.  The paper's
+ * procedure moves nodes one by one in an order it does not fix, so its result is not unique; this is the
+ * variant whose result is: every node of a level decides from the same frozen state (best gain of Eq. 2
+ * over its own and its neighbours' communities, compared exactly in 64-bit integers, lowest community id
+ * among equals, a move only on a strictly better gain, a node alone in its community never joins a
+ * single node with a higher id), all moves of a sweep are applied together and kept only if the exact
+ * modularity rises; then communities are contracted into the nodes of the next level, until a level moves
+ * nothing.  Levels and sweeps per level are capped by max_levels / max_sweeps (32 and 64 are plenty).
+ *   edge_u, edge_v [E] device: the graph as in gnnco_graph_desc (simple, undirected, each edge once)
+ *   part [n] device int32 (out): community of every node, numbered 0 .. S-1; pass it to
+ *        gnnco_partition_load with S = *S_out
+ *   S_out, qnum_out, two_m_out, levels_out, sweeps_out: HOST values (the last four may be NULL): number of
+ *        communities, exact modularity numerator and 2m (Q = qnum / two_m^2, Eq. 1's sum with Sigma_in counted
+ *        from both ends), levels that moved a node, sweeps kept
+ * ws: gnnco_louvain_workspace_bytes bytes, 256-byte aligned, free again when the call returns.  The call
+ * synchronises `stream` several times per sweep (two integers decide whether a sweep is kept).
+ * Errors: GNNCO_OUT_OF_RANGE, GNNCO_NOT_SIMPLE_GRAPH (self loop), GNNCO_WORKSPACE_TOO_SMALL. */
+int32_t gnnco_louvain_workspace_bytes(int64_t n, int64_t E, size_t* bytes);
+int32_t gnnco_louvain(int64_t n, int64_t E, const int32_t* edge_u, const int32_t* edge_v, int32_t max_levels,
+                      int32_t max_sweeps, int32_t* part, int32_t* S_out, int64_t* qnum_out, int64_t* two_m_out,
+                      int32_t* levels_out, int32_t* sweeps_out, void* ws, size_t ws_bytes, void* stream);
+
 /* dst[i] = src[index[i]] for i < rows, rows of row_bytes bytes each (row_bytes a
  * multiple of 4).  With index = perm it brings a per-node array from the caller's
  * original order into the new order (Algorithm 1, Stage 2 uses the inverse to "map

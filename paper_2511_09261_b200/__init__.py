@@ -28,6 +28,7 @@ EXPORTS = [
     "gnnco_profile_begin", "gnnco_profile_end", "gnnco_objective_static", "gnnco_conflict_workspace_bytes",
     "gnnco_conflict_actions", "gnnco_apply_actions", "gnnco_gumbel_softmax", "gnnco_embedding_update",
     "gnnco_repair_boundary", "gnnco_partition_quality", "gnnco_active_plan_bytes", "gnnco_active_plan",
+    "gnnco_louvain_workspace_bytes", "gnnco_louvain",
 ]
 
 _vp, _i32, _i64, _u32, _f32, _sz = (ctypes.c_void_p, ctypes.c_int32, ctypes.c_int64, ctypes.c_uint32, ctypes.c_float,
@@ -115,6 +116,9 @@ def load_library(build_if_missing: bool = True):
     lib.gnnco_apply_actions.argtypes = [_vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp]
     lib.gnnco_partition_quality.argtypes = [_vp, _vp, _vp, _vp, _vp]
     lib.gnnco_repair_boundary.argtypes = [_vp, _vp, _vp, _vp, _vp]
+    lib.gnnco_louvain_workspace_bytes.argtypes = [_i64, _i64, ctypes.POINTER(_sz)]
+    lib.gnnco_louvain.argtypes = [_i64, _i64, _vp, _vp, _i32, _i32, _vp, ctypes.POINTER(_i32), ctypes.POINTER(_i64),
+                                  ctypes.POINTER(_i64), ctypes.POINTER(_i32), ctypes.POINTER(_i32), _vp, _sz, _vp]
     lib.gnnco_active_plan_bytes.argtypes = [_vp, ctypes.POINTER(_sz)]
     lib.gnnco_active_plan.argtypes = [_vp, _vp, _vp, _sz, _vp, ctypes.POINTER(_i32)]
     lib.gnnco_gumbel_softmax.argtypes = [_vp, _i32, _i32, _vp, _vp, _f32, _vp, _vp]
@@ -540,3 +544,26 @@ def gnnco_train_step(graph: PartitionedGraph, *args, **kwargs):
 
 def gnnco_decode_boundary(graph: PartitionedGraph, *args, **kwargs):
     return graph.decode_boundary(*args, **kwargs)
+
+
+def gnnco_louvain(edge_u, edge_v, n: int, max_levels: int = 32, max_sweeps: int = 64, stream=None):
+    """``gnnco_louvain``: deterministic Louvain partition of the graph (int32 device tensors ``edge_u``,
+    ``edge_v``).  Returns dict(part [n] int32 device tensor, S, qnum, two_m, Q, levels, sweeps)."""
+    import torch
+    lib = load_library()
+    _require(edge_u, torch.int32, "edge_u")
+    _require(edge_v, torch.int32, "edge_v")
+    E = int(edge_u.numel())
+    need = _sz(0)
+    _check(lib.gnnco_louvain_workspace_bytes(n, E, ctypes.byref(need)), "gnnco_louvain_workspace_bytes")
+    ws = torch.empty(max(256, need.value), dtype=torch.uint8, device=edge_u.device)
+    part = torch.empty(n, dtype=torch.int32, device=edge_u.device)
+    S, levels, sweeps = _i32(0), _i32(0), _i32(0)
+    qnum, two_m = _i64(0), _i64(0)
+    _check(lib.gnnco_louvain(n, E, edge_u.data_ptr() if E else None, edge_v.data_ptr() if E else None, max_levels,
+                             max_sweeps, part.data_ptr(), ctypes.byref(S), ctypes.byref(qnum), ctypes.byref(two_m),
+                             ctypes.byref(levels), ctypes.byref(sweeps), ws.data_ptr(), ws.numel(), _stream_ptr(stream)),
+           "gnnco_louvain")
+    q = qnum.value / float(two_m.value) ** 2 if two_m.value else 0.0
+    return dict(part=part, S=int(S.value), qnum=int(qnum.value), two_m=int(two_m.value), Q=q, levels=int(levels.value),
+                sweeps=int(sweeps.value))

@@ -180,6 +180,14 @@ struct Carver {
   bool ok() const { return off <= cap; }
 };
 
+// ---- partition.cu : device primitives (stable LSD radix sort of 64-bit keys on bits [bit_lo, bit_hi) with an
+// optional 32-bit payload, exclusive scan of int32) and the sizes of their scratch arrays
+int32_t device_exclusive_scan(int32_t* data, int64_t N, int32_t* tile_sums, cudaStream_t st);
+int32_t device_radix_sort(uint64_t* a, uint64_t* b, int64_t N, int bit_lo, int bit_hi, int32_t* hist, int32_t* tile_sums,
+                          cudaStream_t st, uint64_t** result, int32_t* va, int32_t* vb, int32_t** vresult);
+void device_sort_scratch_sizes(int64_t N, size_t* hist_ints, size_t* tile_sum_ints);
+void device_scan_scratch_size(int64_t N, size_t* tile_sum_ints);
+
 // ---- spmm.cu : out[i] = scale[i] * (in[i] + sum_{j in row i} in[j]), optionally zeroed where mask[i,f] <= 0
 int32_t launch_aggregate(gnnco_handle* h, int dtype, const void* in, void* out, int F, const float* row_scale,
                          const void* relu_mask, cudaStream_t st);

@@ -97,7 +97,7 @@ int32_t exclusive_scan(gnnco_handle* h, int32_t* data, int64_t N, int32_t* tile_
   scan_tiles<<<tiles, kScanThreads, 0, st>>>(data, N, tile_sums);
   scan_tile_sums<<<1, 1024, 0, st>>>(tile_sums, tiles);
   scan_add_offsets<<<tiles, kScanThreads, 0, st>>>(data, N, tile_sums);
-  h->launches += 3;
+  if (h) h->launches += 3;
   GNNCO_LAUNCH_CHECK();
   return GNNCO_OK;
 }
@@ -136,7 +136,7 @@ __global__ void sort_histogram(const uint64_t* keys, int64_t N, int shift, int32
 }
 
 __global__ void sort_scatter(const uint64_t* keys, uint64_t* out, int64_t N, int shift, const int32_t* offs,
-                             int32_t nblocks) {
+                             int32_t nblocks, const int32_t* vals, int32_t* vals_out) {
   __shared__ int32_t cnt[kSortWarps][256];
   for (int i = threadIdx.x; i < kSortWarps * 256; i += kSortThreads) (&cnt[0][0])[i] = 0;
   __syncthreads();
@@ -167,27 +167,35 @@ __global__ void sort_scatter(const uint64_t* keys, uint64_t* out, int64_t N, int
     __syncwarp();
     if (valid && rank == 0) cnt[warp][d] += __popc(peers);
     __syncwarp();
-    if (valid) out[pos] = key;
+    if (valid) {
+      out[pos] = key;
+      if (vals) vals_out[pos] = vals[idx];        // optional 32-bit payload travels with its key
+    }
   }
 }
 
-// Stable sort of keys on bits [bit_lo, bit_hi).  Returns the buffer that holds the result.
+// Stable sort of keys on bits [bit_lo, bit_hi), optionally with a 32-bit payload per key (va / vb ping-pong
+// like the keys).  Returns the buffers that hold the result.
 int32_t radix_sort(gnnco_handle* h, uint64_t* a, uint64_t* b, int64_t N, int bit_lo, int bit_hi, int32_t* hist,
-                   int32_t* tile_sums, cudaStream_t st, uint64_t** result) {
+                   int32_t* tile_sums, cudaStream_t st, uint64_t** result, int32_t* va = nullptr, int32_t* vb = nullptr,
+                   int32_t** vresult = nullptr) {
   *result = a;
+  if (vresult) *vresult = va;
   if (N <= 1) return GNNCO_OK;
   int32_t nblocks = (int32_t)((N + kSortTile - 1) / kSortTile);
   for (int shift = bit_lo; shift < bit_hi; shift += 8) {
     sort_histogram<<<nblocks, kSortThreads, 0, st>>>(a, N, shift, hist, nblocks);
-    h->launches += 1;
+    if (h) h->launches += 1;
     int32_t rc = exclusive_scan(h, hist, (int64_t)256 * nblocks, tile_sums, st);
     if (rc != GNNCO_OK) return rc;
-    sort_scatter<<<nblocks, kSortThreads, 0, st>>>(a, b, N, shift, hist, nblocks);
-    h->launches += 1;
+    sort_scatter<<<nblocks, kSortThreads, 0, st>>>(a, b, N, shift, hist, nblocks, va, vb);
+    if (h) h->launches += 1;
     GNNCO_LAUNCH_CHECK();
     uint64_t* t = a; a = b; b = t;
+    int32_t* tv = va; va = vb; vb = tv;
   }
   *result = a;
+  if (vresult) *vresult = va;
   return GNNCO_OK;
 }
 
@@ -397,6 +405,21 @@ bool valid_sizes(int64_t n, int64_t E, int32_t S) {
 }
 
 }  // namespace
+
+// The sort and scan primitives for the other translation units (louvain.cu).
+int32_t device_exclusive_scan(int32_t* data, int64_t N, int32_t* tile_sums, cudaStream_t st) {
+  return exclusive_scan(nullptr, data, N, tile_sums, st);
+}
+int32_t device_radix_sort(uint64_t* a, uint64_t* b, int64_t N, int bit_lo, int bit_hi, int32_t* hist, int32_t* tile_sums,
+                          cudaStream_t st, uint64_t** result, int32_t* va, int32_t* vb, int32_t** vresult) {
+  return radix_sort(nullptr, a, b, N, bit_lo, bit_hi, hist, tile_sums, st, result, va, vb, vresult);
+}
+void device_sort_scratch_sizes(int64_t N, size_t* hist_ints, size_t* tile_sum_ints) {
+  const int64_t nblocks = (N + kSortTile - 1) / kSortTile + 1;
+  *hist_ints = (size_t)(256 * nblocks);
+  *tile_sum_ints = (size_t)((256 * nblocks + kScanTile - 1) / kScanTile + 1);
+}
+void device_scan_scratch_size(int64_t N, size_t* tile_sum_ints) { *tile_sum_ints = (size_t)((N + kScanTile - 1) / kScanTile + 1); }
 
 // Work tables of the subgraphs with active[s] != 0 (all when active == nullptr), in subgraph order:
 //   tiles of 128 rows and double tiles of 256 rows of one subgraph (dense transforms), objective work items
