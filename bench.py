@@ -61,7 +61,12 @@ def _oracle_sample(w, n_parts, seed=12345):
     t_book = time.time() - t0
     S = w.S
     order = np.argsort(si.u64(seed, 0, S), kind="stable")
-    parts = sorted(order[: min(n_parts, S)].tolist())
+    pp = book["part_ptr"].astype(np.int64)
+    nnz = book["rowptr"][pp[1:]].astype(np.int64) - book["rowptr"][pp[:-1]].astype(np.int64)
+    deg = np.diff(book["rowptr"])
+    # seeded sample plus the subgraph with the most intra edges and the one that holds the longest row
+    picks = set(order[: min(n_parts, S)].tolist()) | {int(np.argmax(nnz)), int(book["node_part"][int(np.argmax(deg))])}
+    parts = sorted(picks)
     items = []
     edges = 0
     for s in parts:
@@ -106,10 +111,14 @@ def oracle_rate(w, cfg_index, steps=1, warmup=0):
     for _ in range(steps):
         _oracle_step(w, items, threads)
     dt = (time.time() - t0) / max(1, steps)
-    sample = "%d of %d subgraphs (seeded), %d intra edges, one fwd+bwd+Adam pass each step; bookkeeping of the " \
-             "whole graph took %.1f s single-threaded" % (len(items), w.S, edges, t_book)
+    total_edges = int(book["E_in"])
+    sample = "%d of %d subgraphs (seeded, plus the one with the most intra edges and the one with the longest row), " \
+             "%d of %d intra edges, one fwd+bwd+Adam pass each step; bookkeeping of the whole graph took %.1f s " \
+             "single-threaded" % (len(items), w.S, edges, total_edges, t_book)
     return dict(value=edges / dt, unit="edges/s", cores=min(threads, max(1, len(items))), kind="oracle",
-                sample=sample, seconds_per_step=dt)
+                sample=sample, seconds_per_step=dt,
+                extrapolated_whole_graph_seconds_per_step=dt * total_edges / max(1, edges),
+                extrapolation="by intra edges (sample time x all intra edges / sampled intra edges); not measured")
 
 
 # ------------------------------------------------------------------------ clock sampling
@@ -190,12 +199,11 @@ def algorithmic_bytes(kind, w, n, nnz, S):
         # (bfloat16: it gathers the mask bits that the last layer's weight gradient left, n*F/8 bytes)
         per["aggregate_rank1"] = (n * d[L - 1] * b + n * d[L - 1] // 8 if b == 2 and d[L - 1] % 8 == 0
                                   else 2 * n * d[L - 1] * b) + csr + 4 * n + S * d[L - 1] * b
-        per["transform_fwd"] = np.mean([n * (d[l - 1] + d[l]) * b + S * d[l - 1] * d[l] * b for l in hidden])
-        # input gradient: reads Q_l and the weights, writes n x d[l-1]; layers above the first also
-        # read the saved activation (ReLU mask) and inv_deg
-        per["transform_bwd"] = np.mean([n * (d[l - 1] + d[l]) * b + S * d[l - 1] * d[l] * b +
-                                        ((n * d[l - 1] * b + 4 * n) if l > 1 else 0) for l in hidden])
-        per["weight_grad"] = np.mean([n * (d[l - 1] + d[l]) * b + S * d[l - 1] * d[l] * 4 for l in hidden])
+        # dense transforms (forward, input gradient, weight gradient): one n x F and one n x H tensor each;
+        # the weights (S x F x H), the mask bits and the per-row scale are not counted
+        per["transform_fwd"] = np.mean([n * (d[l - 1] + d[l]) * b for l in hidden])
+        per["transform_bwd"] = np.mean([n * (d[l - 1] + d[l]) * b for l in hidden])
+        per["weight_grad"] = np.mean([n * (d[l - 1] + d[l]) * b for l in hidden])
     F = d[L - 1]
     per["gemv"] = n * F * b + 4 * n + S * F * b
     per["weight_grad_vec"] = n * F * b + 4 * n + S * F * 4 + (n * F // 8 if b == 2 and F % 8 == 0 and L > 1 else 0)
@@ -249,6 +257,26 @@ def run_ours(args):
 
     w = si.make_workload(args.config, args.scale)
     bf16 = w.dtype == "bf16"
+    partition_note = "the configuration's own partition"
+    louvain_info = None
+    if args.partition.startswith("bfs:"):
+        import dataclasses
+        S2 = int(args.partition.split(":")[1])
+        w = dataclasses.replace(w, part=si.bfs_partition(w.n, w.eu, w.ev, S2), S=S2, name="%s-bfs%d" % (w.name, S2))
+        partition_note = "%d breadth-first grown parts" % S2
+    elif args.partition == "louvain":
+        # Section 3.1: the partition comes from gnnco_louvain (run on the GPU before anything else; timed below)
+        import dataclasses
+        t_lv = time.time()
+        lv = gnnco.gnnco_louvain(torch.from_numpy(w.eu).to(dev), torch.from_numpy(w.ev).to(dev), w.n)
+        torch.cuda.synchronize()
+        louvain_info = dict(seconds=round(time.time() - t_lv, 4), S=lv["S"], Q=lv["Q"], levels=lv["levels"],
+                            sweeps=lv["sweeps"])
+        w = dataclasses.replace(w, part=lv["part"].cpu().numpy(), S=lv["S"], name="%s-louvain" % w.name)
+        partition_note = "gnnco_louvain: %d communities, modularity %.4f" % (lv["S"], lv["Q"])
+        del lv
+    elif args.partition != "config":
+        raise SystemExit("--partition must be config, louvain or bfs:<S>")
 
     # CPU baseline first (before the first GPU call), rank 0 of a single-GPU run only
     cpu = None
@@ -336,11 +364,22 @@ def run_ours(args):
                           algo_GBs=round(ab / (per_call_ms * 1e-3) / 1e9, 1) if per_call_ms > 0 else None)
     top = max(prof.items(), key=lambda kv: kv[1][1])[0]
     achieved = kern[top]["algo_GBs"]
+    nominal = 8000.0                              # the nominal HBM3e rate the target is quoted against
     roofline = dict(bound="hbm", kernel=top, achieved=achieved, peak=peak, unit="GB/s",
-                    frac=round(achieved / peak, 4), traffic=TRAFFIC_BYTES.get((args.config, top)) if args.scale == 1.0 else None,
+                    frac=round(achieved / peak, 4), frac_of_nominal_8TBs=round(achieved / nominal, 4),
+                    traffic=measured_traffic(args, top),
                     peak_source="%s (MEASURED_PEAKS.json hbm_gbs)" % peak_src if peak_src == "measured" else "fallback",
                     algorithmic_bytes_per_launch=algorithmic_bytes(top, w, w.n, nnz, w.S))
     agg = {k: kern[k] for k in ("aggregate_fwd", "aggregate_bwd", "aggregate_rank1") if k in kern}
+    # the neighbour aggregation forward + backward as one figure (all its launches of the timed steps)
+    agg_bytes = sum(algorithmic_bytes(k, w, w.n, nnz, w.S) * prof[k][0] for k in agg)
+    agg_ms = sum(prof[k][1] for k in agg)
+    spmm = None
+    if agg_ms > 0:
+        rate = agg_bytes / (agg_ms * 1e-3) / 1e9
+        spmm = dict(launches=int(sum(prof[k][0] for k in agg)), total_ms=round(agg_ms, 4), achieved=round(rate, 1),
+                    unit="GB/s", frac=round(rate / peak, 4), frac_of_nominal_8TBs=round(rate / nominal, 4),
+                    note="aggregation forward + transposed + rank-1, algorithmic bytes over their summed device time")
 
     # ---- Stage-3 glue after the last decode (not part of the timed step): conflict list + base
     # action + penalty list / active subgraphs, timed with CUDA events on the current stream
@@ -463,9 +502,10 @@ def run_ours(args):
                         dims=w.dims, max_intra_degree=graph.max_row, weight_sets=w.S, want_dx=True,
                         l2="L2 flushed between steps (256 MB write, untimed)" if flush is not None
                         else "inputs larger than L2",
+                        partition=partition_note, louvain=louvain_info,
                         parallelism="replicas only (no collective on the data path)" if world > 1 else "1 GPU",
                         partition_load_ms=round(load_ms, 3), edges_per_s_whole_graph=value * w.E / max(1, graph.E_in)),
-            roofline=roofline, aggregate_kernels=agg, kernels=kern, cpu_baseline=cpu, clocks=clocks, e2e=e2e,
+            roofline=roofline, spmm_fwd_bwd=spmm, aggregate_kernels=agg, kernels=kern, cpu_baseline=cpu, clocks=clocks, e2e=e2e,
             gpu_launches=int(launches), stage3_glue=stage3, fine_tune_step=(stage3 or {}).get("fine_tune_step"),
             cached_first_aggregation=cached)
         print(json.dumps(line))
@@ -473,16 +513,35 @@ def run_ours(args):
         dist.destroy_process_group()
 
 
-# DRAM traffic per launch (dram__bytes_read.sum + dram__bytes_write.sum) from ncu captures of the
-# kernels as they stand, taken on configuration 5 at one tenth of the size and scaled by 10 (the
-# traffic is proportional to the node count); averaged over the launches of a family inside one
-# step; an entry is removed when its kernel changes.
+# DRAM traffic per launch (dram__bytes_read.sum + dram__bytes_write.sum) of configuration 5's kernel families,
+# from ncu captures of one tenth of the workload (three tenths for the rank-1 aggregation) scaled to the full
+# node count (the traffic is proportional to it); see profiles/ncu_counters_config5_scaled.md.  Every entry
+# names the source file of its kernel and that file's SHA-1 when the counters were taken: when the file has
+# changed since, the entry no longer describes the kernel and the bench reports null.
 TRAFFIC_BYTES = {
-    (5, "aggregate_fwd"): 10.03e9,
-    (5, "aggregate_bwd"): 10.00e9,
-    (5, "transform_fwd"): 10.49e9,
-    (5, "transform_bwd"): 13.10e9,
+    "transform_fwd": (10.46e9, "tc_gemm2.cu", "69db3cca4022"),
+    "transform_bwd": (10.61e9, "tc_gemm2.cu", "69db3cca4022"),
+    "weight_grad": (12.15e9, "tc_gemm.cu", "834b9463b12c"),
+    "aggregate_fwd": (10.00e9, "spmm.cu", "621aa0f900a3"),
+    "aggregate_bwd": (10.00e9, "spmm.cu", "621aa0f900a3"),
+    "aggregate_rank1": (6.09e9, "spmm.cu", "621aa0f900a3"),
+    "weight_grad_vec": (5.46e9, "dense.cu", "6104b880bc2f"),
+    "adam": (8.12e9, "tc_gemm.cu", "834b9463b12c"),
 }
+
+
+def measured_traffic(args, kind):
+    if args.config != 5 or args.scale != 1.0 or args.partition != "config" or kind not in TRAFFIC_BYTES:
+        return None
+    import hashlib
+    nbytes, fname, sha = TRAFFIC_BYTES[kind]
+    path = os.path.join(ROOT, "paper_2511_09261_b200", "csrc", fname)
+    try:
+        with open(path, "rb") as f:
+            now = hashlib.sha1(f.read()).hexdigest()[:12]
+    except OSError:
+        return None
+    return nbytes if now == sha else None
 
 
 # ----------------------------------------------------------------------- reference arm
@@ -519,6 +578,8 @@ def main():
     ap.add_argument("--config", type=int, default=5, choices=[1, 2, 3, 4, 5])
     ap.add_argument("--scale", type=float, default=1.0,
                     help="shrink configuration 4 or 5 (nodes, edges, subgraphs) for profiler captures")
+    ap.add_argument("--partition", default="config",
+                    help="config (the configuration's partition), louvain (gnnco_louvain on the GPU) or bfs:<S>")
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")

@@ -459,8 +459,8 @@ int32_t launch_wg(gnnco_handle* h, const void* A, const void* G, float* dW, floa
 // W [sets][K][N] float32 -> Wt [sets][N][K] bf16
 __global__ void cast_transpose_bf16_kernel(const float* __restrict__ W, __nv_bfloat16* __restrict__ Wt, int K, int N) {
   __shared__ float tile[32][33];
-  const int64_t base = (int64_t)blockIdx.z * K * N;
-  const int k0 = blockIdx.y * 32, n0 = blockIdx.x * 32;
+  const int64_t base = (int64_t)blockIdx.x * K * N;          // the set index is on x (no 65,535 limit there)
+  const int k0 = blockIdx.y * 32, n0 = blockIdx.z * 32;
   for (int j = threadIdx.y; j < 32; j += 8) {
     int k = k0 + j, n = n0 + threadIdx.x;
     tile[j][threadIdx.x] = (k < K && n < N) ? W[base + (int64_t)k * N + n] : 0.0f;
@@ -477,8 +477,8 @@ __global__ void cast_transpose_bf16_kernel(const float* __restrict__ W, __nv_bfl
 __global__ void __launch_bounds__(256) cast_both_bf16_kernel(const float* __restrict__ W, __nv_bfloat16* __restrict__ Wc,
                                                              __nv_bfloat16* __restrict__ Wt, int K, int N) {
   __shared__ float tile[64][65];
-  const int64_t base = (int64_t)blockIdx.z * K * N;
-  const int k0 = blockIdx.y * 64, n0 = blockIdx.x * 64;
+  const int64_t base = (int64_t)blockIdx.x * K * N;          // the set index is on x (no 65,535 limit there)
+  const int k0 = blockIdx.y * 64, n0 = blockIdx.z * 64;
   const int q = threadIdx.x & 15, r = threadIdx.x >> 4;   // 16 threads of four elements across, 16 rows per pass
 #pragma unroll
   for (int pass = 0; pass < 4; ++pass) {
@@ -512,10 +512,10 @@ __global__ void __launch_bounds__(256) adam_cast_both_kernel(float* __restrict__
                                                              float inv_c1, float inv_c2,
                                                              const uint8_t* __restrict__ active) {
   __shared__ float tile[64][65];
-  const int64_t base = (int64_t)blockIdx.z * K * N;
-  const int k0 = blockIdx.y * 64, n0 = blockIdx.x * 64;
+  const int64_t base = (int64_t)blockIdx.x * K * N;          // the set index is on x (no 65,535 limit there)
+  const int k0 = blockIdx.y * 64, n0 = blockIdx.z * 64;
   const int q = threadIdx.x & 15, r = threadIdx.x >> 4;   // 16 threads of four elements across, 16 rows per pass
-  if (active && !active[blockIdx.z]) return;                // uniform across the block
+  if (active && !active[blockIdx.x]) return;                // uniform across the block
 #pragma unroll
   for (int pass = 0; pass < 4; ++pass) {
     const int k = r + 16 * pass;
@@ -597,12 +597,12 @@ int32_t launch_weight_grad_tc(gnnco_handle* h, const void* A, const void* G, flo
 
 int32_t launch_cast_both_bf16(gnnco_handle* h, const float* W, __nv_bfloat16* Wc, __nv_bfloat16* Wt, int K, int N,
                               int32_t sets, cudaStream_t st) {
-  if ((K % 64) || (N % 64) || ((uintptr_t)W & 15) || ((uintptr_t)Wc & 7) || ((uintptr_t)Wt & 7) || sets > 65535) {
+  if ((K % 64) || (N % 64) || ((uintptr_t)W & 15) || ((uintptr_t)Wc & 7) || ((uintptr_t)Wt & 7)) {
     int32_t rc = launch_cast_bf16(h, W, Wc, (int64_t)K * N * sets, st);
     return rc != GNNCO_OK ? rc : launch_cast_transpose_bf16(h, W, Wt, K, N, sets, st);
   }
   ProfScope prof_(h, K_CAST, st);
-  cast_both_bf16_kernel<<<dim3(N / 64, K / 64, sets), 256, 0, st>>>(W, Wc, Wt, K, N);
+  cast_both_bf16_kernel<<<dim3(sets, K / 64, N / 64), 256, 0, st>>>(W, Wc, Wt, K, N);
   h->launches += 1;
   GNNCO_LAUNCH_CHECK();
   return GNNCO_OK;
@@ -611,7 +611,7 @@ int32_t launch_cast_both_bf16(gnnco_handle* h, const float* W, __nv_bfloat16* Wc
 int32_t launch_cast_transpose_bf16(gnnco_handle* h, const float* W, __nv_bfloat16* Wt, int K, int N, int32_t sets,
                                    cudaStream_t st) {
   ProfScope prof_(h, K_CAST, st);
-  dim3 grid((N + 31) / 32, (K + 31) / 32, sets);
+  dim3 grid(sets, (K + 31) / 32, (N + 31) / 32);
   if (grid.y > 65535 || grid.z > 65535) return GNNCO_UNSUPPORTED;
   cast_transpose_bf16_kernel<<<grid, dim3(32, 8), 0, st>>>(W, Wt, K, N);
   h->launches += 1;
@@ -621,7 +621,7 @@ int32_t launch_cast_transpose_bf16(gnnco_handle* h, const float* W, __nv_bfloat1
 
 bool adam_cast_both_supported(const float* W, const float* m, const float* v, const float* g, const __nv_bfloat16* Wc,
                               const __nv_bfloat16* Wt, int K, int N, int32_t sets) {
-  return Wc && Wt && (K % 64) == 0 && (N % 64) == 0 && sets <= 65535 &&
+  return Wc && Wt && (K % 64) == 0 && (N % 64) == 0 && sets >= 1 &&
          !(((uintptr_t)W | (uintptr_t)m | (uintptr_t)v | (uintptr_t)g) & 15) && !(((uintptr_t)Wc | (uintptr_t)Wt) & 7);
 }
 
@@ -630,7 +630,7 @@ int32_t launch_adam_cast_both(gnnco_handle* h, float* W, float* m, float* v, con
                               float c1, float c2, const uint8_t* active, cudaStream_t st) {
   if (!adam_cast_both_supported(W, m, v, g, Wc, Wt, K, N, sets)) return GNNCO_UNSUPPORTED;
   ProfScope prof_(h, K_ADAM, st);
-  adam_cast_both_kernel<<<dim3(N / 64, K / 64, sets), 256, 0, st>>>(W, m, v, g, Wc, Wt, K, N, lr, b1, b2, eps, 1.0f / c1,
+  adam_cast_both_kernel<<<dim3(sets, K / 64, N / 64), 256, 0, st>>>(W, m, v, g, Wc, Wt, K, N, lr, b1, b2, eps, 1.0f / c1,
                                                                      1.0f / c2, active);
   h->launches += 1;
   GNNCO_LAUNCH_CHECK();

@@ -453,8 +453,8 @@ int32_t launch_wgf(gnnco_handle* h, const void* A, const void* G, float* dW, flo
 __global__ void cast_split3_kernel(const float* __restrict__ W, __nv_bfloat16* __restrict__ out, int K, int N,
                                    int64_t limb_stride, int transpose) {
   __shared__ float tile[32][33];
-  const int64_t base = (int64_t)blockIdx.z * K * N;
-  const int k0 = blockIdx.y * 32, n0 = blockIdx.x * 32;
+  const int64_t base = (int64_t)blockIdx.x * K * N;          // the set index is on x (no 65,535 limit there)
+  const int k0 = blockIdx.y * 32, n0 = blockIdx.z * 32;
   for (int j = threadIdx.y; j < 32; j += 8) {
     int k = k0 + j, n = n0 + threadIdx.x;
     tile[j][threadIdx.x] = (k < K && n < N) ? W[base + (int64_t)k * N + n] : 0.0f;
@@ -516,7 +516,7 @@ int32_t launch_weight_grad_tc_f32(gnnco_handle* h, const void* A, const void* G,
 int32_t launch_cast_split3(gnnco_handle* h, const float* W, __nv_bfloat16* out, int K, int N, int32_t sets,
                            bool transpose, cudaStream_t st) {
   ProfScope prof_(h, K_CAST, st);
-  dim3 grid((N + 31) / 32, (K + 31) / 32, sets);
+  dim3 grid(sets, (K + 31) / 32, (N + 31) / 32);
   if (grid.y > 65535 || grid.z > 65535) return GNNCO_UNSUPPORTED;
   cast_split3_kernel<<<grid, dim3(32, 8), 0, st>>>(W, out, K, N, (int64_t)sets * K * N, transpose ? 1 : 0);
   h->launches += 1;

@@ -120,3 +120,42 @@ def test_training_the_embeddings_lowers_the_objective():
         graph.embedding_update(dX, Xm, m, v, X, lr=1e-2, step=step)
     assert totals[-1] < totals[0]
     assert graph.async_status() == gnnco.OK
+
+
+@pytest.mark.parametrize("n,d,S", [(100, 10, 2), (500, 20, 4), (1000, 40, 8), (1000, 10, 1)])
+def test_small_regular_workload_pipeline_matches_the_oracle(n, d, S):
+    """The paper's small-graph experiment shape (Section 4: d-regular graphs of 100 to 1,000 nodes, degree 10 to
+    40), through the whole variant in which embeddings are processed and trained: Gumbel-softmax of the random
+    initial embeddings, one training step with the input gradient, Adam on the embeddings -- every stage
+    against the oracle on the same seeded inputs."""
+    import torch
+    import paper_2511_09261_b200 as gnnco
+    from gpu_common import StepCase, check_bookkeeping, check_decode
+    w = si.small_regular_workload(n, d, S, [32, 16, 1], seed=100 + d)
+    deg = np.bincount(np.concatenate([w.eu, w.ev]), minlength=n)
+    assert deg.max() == d and (deg >= d - 2).mean() > 0.9          # configuration model: a few nodes lose an edge
+    book = oracle.bookkeeping(w.n, w.eu, w.ev, w.part, w.S)
+    graph = load_graph(w.n, w.eu, w.ev, w.part, w.S)
+    check_bookkeeping(graph, book)
+    E = w.features_f32()[book["perm"]]
+    U = _uniforms(n, w.dims[0], 7)
+    X_d = graph.gumbel_softmax(to_dev(E), to_dev(U), 0.7)
+    X = X_d.cpu().numpy()
+    np.testing.assert_allclose(X, oracle.gumbel_softmax(E, U, 0.7), **TOL["f32"])
+    # the step is compared on the GPU's own float32 embeddings (teacher-forced at the stage boundary)
+    W = [w.weights(l) for l in range(w.L)]
+    case = StepCase(book, w.dims, "f32", w.S, w.alpha, w.beta)
+    adam = dict(lr=1e-2, step=1, m=[np.zeros_like(x) for x in W], v=[np.zeros_like(x) for x in W])
+    g, _ = case.run(graph, X, W, None, want_dx=True, adam=adam, label="regular-%d-%d" % (n, d))
+    check_decode(graph, book, g["p"])
+    for name in ("loss", "p", "z", "dW0", "dW1", "dX"):
+        assert case.report.needs_only_flat(name), name
+    # Adam on the embeddings with the GPU's own input gradient
+    Xm, m, v = X_d.clone(), torch.zeros_like(X_d), torch.zeros_like(X_d)
+    out = torch.empty_like(X_d)
+    graph.embedding_update(to_dev(g["dX"].astype(np.float32)), Xm, m, v, out, lr=1e-2, step=1)
+    Xr, mr, vr = X.astype(np.float64), np.zeros_like(X, np.float64), np.zeros_like(X, np.float64)
+    f32 = lambda x: float(np.float32(x))
+    oracle.adam(Xr, mr, vr, g["dX"].astype(np.float64), f32(1e-2), 1, f32(0.9), f32(0.999), f32(1e-8))
+    np.testing.assert_allclose(Xm.cpu().numpy(), Xr, rtol=1e-5, atol=1e-6)
+    assert torch.equal(out, Xm)
