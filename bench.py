@@ -384,7 +384,7 @@ def run_ours(args):
     # ---- Stage-3 glue after the last decode (not part of the timed step): conflict list + base
     # action + penalty list / active subgraphs, timed with CUDA events on the current stream
     stage3 = None
-    if graph.E_b > 0:
+    if graph.E_b > 0 and not args.no_extras:
         ca = graph.conflict_actions(viol, p)
         graph.apply_actions(ca["conflict_idx"], ca["action"], ca["count"])
         torch.cuda.synchronize()
@@ -439,7 +439,7 @@ def run_ours(args):
     # ---- the same step with the first layer's aggregated input kept across steps (X is a fixed
     # input, so this is legal; it is NOT the headline number, which recomputes it every step)
     cached = None
-    if w.L > 1:
+    if w.L > 1 and not args.no_extras:
         ax = torch.empty_like(X)
         graph.train_step(model, X, w.alpha, w.beta, w.lam, pen, opt, loss=loss, p=p, dX=dX,
                          flags=gnnco.WANT_DX | gnnco.AX_STORE | gnnco.WEIGHTS_UNTOUCHED, ax_cache=ax)
@@ -583,6 +583,8 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--no-extras", action="store_true",
+                    help="only the timed steps: no Stage-3 glue, fine-tuning or cached-aggregation legs (profiler captures)")
     args = ap.parse_args()
     if args.warmup < 3 and args.impl == "ours":
         args.warmup = 3
