@@ -44,7 +44,8 @@ struct Vec<float> {
     acc[2] += __uint_as_float(v.z) > 0.0f ? c : 0.0f; acc[3] += __uint_as_float(v.w) > 0.0f ? c : 0.0f;
   }
   __device__ static void store(float* p, const float (&f)[4]) {
-    *reinterpret_cast<float4*>(p) = make_float4(f[0], f[1], f[2], f[3]);
+    // streaming store: an output row is not read again by this kernel, the gathered rows are
+    __stcs(reinterpret_cast<float4*>(p), make_float4(f[0], f[1], f[2], f[3]));
   }
 };
 template <>
@@ -91,7 +92,7 @@ struct Vec<__nv_bfloat16> {
       __nv_bfloat162 b = __floats2bfloat162_rn(f[2 * k], f[2 * k + 1]);
       w[k] = *reinterpret_cast<uint32_t*>(&b);
     }
-    *reinterpret_cast<uint4*>(p) = make_uint4(w[0], w[1], w[2], w[3]);
+    __stcs(reinterpret_cast<uint4*>(p), make_uint4(w[0], w[1], w[2], w[3]));
   }
 };
 
