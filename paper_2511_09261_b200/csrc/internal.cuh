@@ -245,6 +245,9 @@ int32_t launch_transform_tc_pair(gnnco_handle* h, const void* A, const void* B, 
                                  int K, int N, bool relu, const float* row_scale, const uint8_t* mask_bits,
                                  uint8_t* bits_out, bool backward, const void* dot_w, int64_t dot_stride, float* dot_out,
                                  cudaStream_t st);
+bool tc_pair_weight_grad_supported(gnnco_handle* h, int dtype, int K, int N);
+int32_t launch_weight_grad_tc_pair(gnnco_handle* h, const void* A, const void* G, float* dW, float* scratch, int K, int N,
+                                   cudaStream_t st);
 bool tc_weight_grad_supported(int dtype, int K, int N);
 int32_t launch_weight_grad_tc(gnnco_handle* h, const void* A, const void* G, float* dW, float* scratch, int K, int N,
                               cudaStream_t st);

@@ -426,6 +426,182 @@ int32_t launch_pair(gnnco_handle* h, const void* A, const void* B, int64_t b_str
                                                     dot_stride, dot_out, clusters, per, st);
 }
 
+// ------------------------------------------------------------------------------------
+// Weight gradient by pairs of CTAs:  dW_s[256 x 256] = sum_{i in s} A[i, :]^T G[i, :]  (A = layer input, G = Q_l).
+//
+// The single-CTA kernel (tc_gemm.cu) needs all 512 TMEM columns for one 256 x 256 float32 accumulator, so a
+// subgraph's 256 KB result cannot leave while the next subgraph is being summed, and every subgraph pays an
+// unhidden pipeline fill and drain (about a tenth of its time at 2,400 rows).  With cta_group::2 the pair owns
+// one subgraph (or row chunk): each CTA stages, per 64 rows, only ITS 128 features of A (the M half) and ITS 128
+// features of G (the N half), the pair's MMAs (256 x 256 x 16, both operands MN-major) leave 128 x 256 of the result
+// in each CTA's TMEM -- 256 columns, so there are TWO accumulator buffers and a subgraph is written out while the
+// next one is summed.  Persistent over the chunk table; six stages of 32 KB per CTA, filled by TMA across chunk
+// boundaries.  A chunk's last, ragged stage lands on a private barrier; the producer warp zeroes the rows past the
+// chunk's end (they belong to the next subgraph) before it announces the stage.
+// Roles per CTA: warp 0 producer, warp 1 MMA issuer (even CTA), warps 2-9 write the result (TMEM lane quarter =
+// warp % 4, column half by which of the two warps of that quarter).
+constexpr int kWgpThreads = 320;
+constexpr int kWgpStages = 6;
+constexpr int kWgpRows = 64;                     // reduction rows per stage
+constexpr uint32_t kWgpHalf = 128 * 128;         // one operand's share of a stage: 64 rows x 128 features x 2 B
+constexpr uint32_t kWgpStage = 2 * kWgpHalf;     // A share + G share
+constexpr size_t kWgpSmem = 1024 + kWgpStages * kWgpStage + 256;
+
+__global__ void __launch_bounds__(kWgpThreads, 1)
+weight_grad_tc_pair(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_g,
+                    float* __restrict__ dW, float* __restrict__ scratch, const int32_t* __restrict__ wg_begin,
+                    const int32_t* __restrict__ wg_end, const int32_t* __restrict__ wg_slot, int n_chunks,
+                    int32_t* status) {
+  constexpr int KF = 256, NF = 256;
+  extern __shared__ uint8_t smem_raw[];
+  const uint32_t sbase = (tc::smem_u32(smem_raw) + 1023u) & ~1023u;
+  uint8_t* gen_base = smem_raw + (sbase - tc::smem_u32(smem_raw));
+  uint64_t* full = reinterpret_cast<uint64_t*>(gen_base + kWgpStages * kWgpStage);   // [6]  even CTA's copy is used
+  uint64_t* empty = full + kWgpStages;                                                // [6]  both CTAs
+  uint64_t* acc_full = empty + kWgpStages;                                            // [2]  both CTAs
+  uint64_t* acc_empty = acc_full + 2;                                                 // [2]  even CTA's copy is used
+  uint64_t* tail_bar = acc_empty + 2;                                                 // [1]  this CTA's ragged stages
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(tail_bar + 1);
+  volatile uint32_t* abort_flag = tmem_slot + 1;
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const uint32_t rank = tc::cluster_ctarank();
+  const int cluster_id = blockIdx.x >> 1, n_clusters = gridDim.x >> 1;
+  if (cluster_id >= n_chunks) return;                            // both CTAs of the cluster leave together
+
+  if (threadIdx.x == 0) {
+    for (int i = 0; i < kWgpStages; ++i) {
+      tc::mbar_init(full + i, 2);                                // one announcement per CTA
+      tc::mbar_init(empty + i, 1);
+    }
+    for (int i = 0; i < 2; ++i) {
+      tc::mbar_init(acc_full + i, 1);
+      tc::mbar_init(acc_empty + i, 2 * 8);                       // one arrival per result warp of both CTAs
+    }
+    tc::mbar_init(tail_bar, 1);
+    *abort_flag = 0;
+    tc::fence_mbar_init();
+  }
+  if (warp == 0) tc::tmem_alloc_pair(tmem_slot, 512);
+  tc::tc_fence_before_sync();
+  __syncthreads();
+  tc::cluster_sync_all();
+  tc::tc_fence_after_sync();
+  const uint32_t tmem = *tmem_slot;
+
+  if (warp == 0) {
+    // ------------------------------------------------------------------- producer
+    int g = 0;                                                   // stages issued so far (ring position)
+    int tails = 0;                                               // ragged stages so far (phase of tail_bar)
+    for (int c = cluster_id; c < n_chunks && !*abort_flag; c += n_clusters) {
+      const int32_t ra = wg_begin[c], rb = wg_end[c];
+      for (int32_t r0 = ra; r0 < rb && !*abort_flag; r0 += kWgpRows, ++g) {
+        const int slot = g % kWgpStages, use = g / kWgpStages;
+        const uint32_t sa = sbase + slot * kWgpStage, sg = sa + kWgpHalf;
+        const int valid = min(kWgpRows, rb - r0);
+        const uint32_t bar = tc::map_to_cta(tc::smem_u32(full + slot), 0);
+        if (use > 0 && !tc::mbar_wait_bounded(empty + slot, (use - 1) & 1)) *abort_flag = 1;
+        if (*abort_flag) break;
+        if (valid == kWgpRows) {
+          if (lane == 0) {
+            tc::mbar_arrive_expect_tx_cluster(bar, kWgpStage);
+            tc::tma_load_2d_pair(sa, &map_a, (int32_t)rank * 128, r0, bar);
+            tc::tma_load_2d_pair(sa + 8192, &map_a, (int32_t)rank * 128 + 64, r0, bar);
+            tc::tma_load_2d_pair(sg, &map_g, (int32_t)rank * 128, r0, bar);
+            tc::tma_load_2d_pair(sg + 8192, &map_g, (int32_t)rank * 128 + 64, r0, bar);
+          }
+        } else {
+          // ragged end of the chunk: land on this CTA's own barrier, zero the rows past the end, then announce
+          const uint32_t tb = tc::smem_u32(tail_bar);
+          if (lane == 0) {
+            tc::mbar_arrive_expect_tx_cluster(tb, kWgpStage);
+            tc::tma_load_2d_pair(sa, &map_a, (int32_t)rank * 128, r0, tb);
+            tc::tma_load_2d_pair(sa + 8192, &map_a, (int32_t)rank * 128 + 64, r0, tb);
+            tc::tma_load_2d_pair(sg, &map_g, (int32_t)rank * 128, r0, tb);
+            tc::tma_load_2d_pair(sg + 8192, &map_g, (int32_t)rank * 128 + 64, r0, tb);
+          }
+          if (!tc::mbar_wait_bounded(tail_bar, tails & 1)) *abort_flag = 1;
+          ++tails;
+          // row k of a 64-feature block is 128 bytes at (k/8)*1024 + (k%8)*128 whatever the swizzle does inside it
+          for (int q = lane; q < (kWgpRows - valid) * 4 * 8; q += 32) {
+            const int k = valid + q / 32, blk = (q / 8) & 3, piece = q & 7;
+            tc::st_shared_zero16(sa + blk * 8192 + (k >> 3) * 1024 + (k & 7) * 128 + piece * 16);
+          }
+          tc::fence_proxy_async_smem();
+          __syncwarp();
+          if (lane == 0) tc::mbar_arrive_expect_tx_cluster(bar, 0);
+        }
+        __syncwarp();
+      }
+    }
+  } else if (warp == 1) {
+    // -------------------------------------------------------------------- MMA issuer (even CTA)
+    if (rank == 0) {
+      constexpr uint32_t IDESC = tc::idesc_bf16_f32(256, NF, true, true);
+      int g = 0, j = 0;
+      for (int c = cluster_id; c < n_chunks && !*abort_flag; c += n_clusters, ++j) {
+        const int32_t ra = wg_begin[c], rb = wg_end[c];
+        const int iters = (rb - ra + kWgpRows - 1) / kWgpRows;
+        const int buf = j & 1;
+        if (j >= 2 && !tc::mbar_wait_bounded(acc_empty + buf, ((j >> 1) - 1) & 1)) *abort_flag = 1;
+        for (int it = 0; it < iters; ++it, ++g) {
+          const int slot = g % kWgpStages, use = g / kWgpStages;
+          if (!tc::mbar_wait_bounded(full + slot, use & 1)) *abort_flag = 1;
+          tc::tc_fence_after_sync();
+          if (lane == 0 && !*abort_flag) {
+            const uint32_t sa = sbase + slot * kWgpStage, sg = sa + kWgpHalf;
+#pragma unroll
+            for (int q = 0; q < kWgpRows / 16; ++q) {
+              const uint64_t ad = tc::smem_desc_sw128(sa + q * 2048, kWgpRows * 128, 1024);
+              const uint64_t gd = tc::smem_desc_sw128(sg + q * 2048, kWgpRows * 128, 1024);
+              tc::mma_bf16_pair(tmem + buf * NF, ad, gd, IDESC, (it | q) != 0);
+            }
+            tc::mma_commit_pair(empty + slot, 3);
+          }
+          __syncwarp();
+        }
+        if (lane == 0 && !*abort_flag) tc::mma_commit_pair(acc_full + buf, 3);
+        __syncwarp();
+      }
+    }
+  } else {
+    // ---------------------------------------------------------------------- result writers
+    const int quarter = warp & 3, half = (warp - 2) >> 2;        // warps 2..5 -> half 0, 6..9 -> half 1
+    const uint32_t acc_empty_even = tc::map_to_cta(tc::smem_u32(acc_empty), 0);
+    const int f = (int)rank * 128 + quarter * 32 + lane;          // this thread's row of dW
+    int j = 0;
+    for (int c = cluster_id; c < n_chunks && !*abort_flag; c += n_clusters, ++j) {
+      const int buf = j & 1;
+      const int32_t rows = wg_end[c] - wg_begin[c];
+      const int32_t slot = wg_slot[c];
+      float* out = slot < 0 ? dW + (int64_t)(-(slot + 1)) * KF * NF : scratch + (int64_t)slot * KF * NF;
+      if (!tc::mbar_wait_bounded(acc_full + buf, (j >> 1) & 1)) { *abort_flag = 1; break; }
+      tc::tc_fence_after_sync();
+#pragma unroll
+      for (int c0 = 0; c0 < NF / 2; c0 += 32) {
+        uint32_t r[32];
+        if (rows > 0) {
+          tc::tmem_ld_32x32(tmem + ((uint32_t)(quarter * 32) << 16) + buf * NF + half * (NF / 2) + c0, r);
+          tc::tmem_ld_wait();
+        } else {
+#pragma unroll
+          for (int q = 0; q < 32; ++q) r[q] = 0u;                 // a chunk without rows: no MMA ran
+        }
+        uint4* dst = reinterpret_cast<uint4*>(out + (int64_t)f * NF + half * (NF / 2) + c0);
+#pragma unroll
+        for (int q = 0; q < 8; ++q) dst[q] = make_uint4(r[4 * q], r[4 * q + 1], r[4 * q + 2], r[4 * q + 3]);
+      }
+      tc::tc_fence_before_sync();
+      __syncwarp();
+      if (lane == 0) tc::mbar_arrive_cluster(acc_empty_even + buf * 8);
+    }
+  }
+  if (*abort_flag && threadIdx.x == 0) atomicMin(status, (int32_t)GNNCO_INTERNAL);
+  tc::tc_fence_before_sync();
+  __syncthreads();
+  tc::cluster_sync_all();
+  if (warp == 0) tc::tmem_dealloc_pair(tmem, 512);
+}
+
 }  // namespace
 
 // The pair form is used for the widths where a single CTA cannot hold a second operand tile.
@@ -447,4 +623,36 @@ int32_t launch_transform_tc_pair(gnnco_handle* h, const void* A, const void* B, 
   if (((uintptr_t)mask_bits & 7) || ((uintptr_t)bits_out & 7)) return GNNCO_UNSUPPORTED;
   return launch_pair<256, 256>(h, A, B, b_stride, b_sets, Y, relu, row_scale, mask_bits, bits_out, dot_w, dot_stride, dot_out,
                                st);
+}
+
+bool tc_pair_weight_grad_supported(gnnco_handle* h, int dtype, int K, int N) {
+  return K == 256 && N == 256 && tc_pair_transform_supported(h, dtype, 256, 256) && h->n_wg_chunks > 0;
+}
+
+// dW[s] (256 x 256, float32) = sum_{i in s} A[i,:]^T G[i,:], A, G [n x 256] bf16; chunks of split subgraphs land in
+// `scratch` and are combined afterwards, as in the single-CTA kernel
+int32_t launch_weight_grad_tc_pair(gnnco_handle* h, const void* A, const void* G, float* dW, float* scratch, int K, int N,
+                                   cudaStream_t st) {
+  if (!tc_pair_weight_grad_supported(h, GNNCO_BF16, K, N)) return GNNCO_UNSUPPORTED;
+  if (((uintptr_t)A & 15) || ((uintptr_t)G & 15) || ((uintptr_t)dW & 15) || ((uintptr_t)scratch & 15)) return GNNCO_UNSUPPORTED;
+  ProfScope prof_(h, K_WEIGHT_GRAD, st);
+  CUtensorMap ma, mg;
+  if (!make_map(&ma, A, (uint64_t)h->n, 256, kWgpRows, 64, true)) return GNNCO_CUDA_ERROR;
+  if (!make_map(&mg, G, (uint64_t)h->n, 256, kWgpRows, 64, true)) return GNNCO_CUDA_ERROR;
+  GNNCO_CUDA_TRY(cudaFuncSetAttribute(weight_grad_tc_pair, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kWgpSmem));
+  const int clusters = h->pair_clusters < h->n_wg_chunks ? h->pair_clusters : h->n_wg_chunks;
+  cudaLaunchConfig_t cfg{};
+  cfg.gridDim = dim3(2 * clusters);
+  cfg.blockDim = dim3(kWgpThreads);
+  cfg.dynamicSmemBytes = kWgpSmem;
+  cfg.stream = st;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeClusterDimension;
+  attr[0].val.clusterDim.x = 2; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  GNNCO_CUDA_TRY(cudaLaunchKernelEx(&cfg, weight_grad_tc_pair, ma, mg, dW, scratch, (const int32_t*)h->wg_begin,
+                                    (const int32_t*)h->wg_end, (const int32_t*)h->wg_slot, (int)h->n_wg_chunks, h->status));
+  h->launches += 1;
+  return launch_wg_combine(h, scratch, dW, (int64_t)K * N, st);
 }

@@ -321,7 +321,10 @@ int32_t run_step_on(gnnco_handle* h, const gnnco_model_desc* m, const void* X, c
     }
     float* target = grad_target(l - 1);
     float* wg_out = sets == 1 ? T.dW_sets : target;
-    if (tc_weight_grad_supported(dt, K, N)) GNNCO_TRY(launch_weight_grad_tc(h, Hin, Q, wg_out, T.wg_scratch, K, N, st));
+    if (tc_pair_weight_grad_supported(h, dt, K, N))
+      GNNCO_TRY(launch_weight_grad_tc_pair(h, Hin, Q, wg_out, T.wg_scratch, K, N, st));
+    else if (tc_weight_grad_supported(dt, K, N))
+      GNNCO_TRY(launch_weight_grad_tc(h, Hin, Q, wg_out, T.wg_scratch, K, N, st));
     else if (dt == GNNCO_F32 && tc_f32_weight_grad_supported(K, N))
       GNNCO_TRY(launch_weight_grad_tc_f32(h, Hin, Q, wg_out, T.wg_scratch, K, N, st));
     else GNNCO_TRY(launch_weight_grad(h, dt, Hin, Q, wg_out, K, N, st));
