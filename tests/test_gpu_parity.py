@@ -352,6 +352,7 @@ def test_train_step_f32_tensor_core_widths(dims, n, S, sets):
 
 
 @pytest.mark.parametrize("dtype,dims,n,S", [("bf16", [256, 128, 1], 9000, 2), ("f32", [128, 64, 1], 7000, 1),
+                                            ("bf16", [256, 256, 256, 1], 7000, 3),
                                             ("bf16", [128, 128, 1], 6100, 3), ("f32", [64, 36, 1], 7000, 1),
                                             ("f32", [20, 24, 1], 5000, 2)])
 def test_train_step_few_very_long_subgraphs(dtype, dims, n, S):
