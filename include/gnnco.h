@@ -72,6 +72,14 @@ typedef enum { GNNCO_F32 = 0, GNNCO_BF16 = 1 } gnnco_dtype;
 #define GNNCO_WEIGHTS_UNTOUCHED 16u
 /* Fine-tuning on the active subgraphs only; see gnnco_active_plan. */
 #define GNNCO_ACTIVE_ONLY 32u
+/* bfloat16 features, hidden layers of width 256 -> 256 only (ignored elsewhere).  Such a layer of Eq. 3 then
+ * runs as ONE kernel: the aggregated rows are summed on chip straight into the operand of the matrix
+ * product and never reach device memory.  Rows are added in the same order as in the separate aggregation
+ * kernel, so the results are bit-identical to the plain step wherever no row has more than 256 neighbours.
+ * Off by default: on B200 the two separate kernels are faster (the fused kernel can keep about 60 KB of
+ * gathers in flight per SM beside its operands, the separate aggregation kernel more); the flag exists for
+ * devices and graphs where saving the write and the re-read of the aggregated features pays. */
+#define GNNCO_ONE_KERNEL_LAYERS 64u
 
 typedef struct gnnco_handle gnnco_handle;
 

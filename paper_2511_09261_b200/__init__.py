@@ -19,7 +19,7 @@ OK = 0
 INVALID_ARGUMENT, OUT_OF_RANGE, NOT_SIMPLE_GRAPH, UNSUPPORTED, WORKSPACE_TOO_SMALL, CUDA_ERROR, INTERNAL = (
     -1, -2, -3, -4, -5, -6, -7)
 F32, BF16 = 0, 1
-WANT_DX, FORWARD_ONLY, AX_STORE, AX_REUSE, WEIGHTS_UNTOUCHED, ACTIVE_ONLY = 1, 2, 4, 8, 16, 32
+WANT_DX, FORWARD_ONLY, AX_STORE, AX_REUSE, WEIGHTS_UNTOUCHED, ACTIVE_ONLY, ONE_KERNEL_LAYERS = 1, 2, 4, 8, 16, 32, 64
 
 EXPORTS = [
     "gnnco_status_string", "gnnco_partition_workspace_bytes", "gnnco_partition_load", "gnnco_graph_info",

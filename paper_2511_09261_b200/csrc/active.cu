@@ -14,6 +14,7 @@ namespace {
 struct PlanLayout {
   int32_t *tile_row0, *tile_rows, *pair_row0, *pair_rows, *item_row0, *item_row1, *part_item_ptr;
   int32_t *wg_begin, *wg_end, *wg_slot, *wg_mpart, *wg_mfirst, *wg_mcount, *chunk_row0, *chunk_rows;
+  FuseSet fuse;
   size_t bytes;
 };
 
@@ -40,6 +41,7 @@ PlanLayout carve_plan(void* base, int64_t n, int32_t S) {
   L.wg_mcount = c.take<int32_t>((size_t)S);
   L.chunk_row0 = c.take<int32_t>(rows256);
   L.chunk_rows = c.take<int32_t>(rows256);
+  L.fuse = carve_fuse_set(c, tiles);
   L.bytes = c.off;
   return L;
 }
@@ -93,6 +95,11 @@ extern "C" int32_t gnnco_active_plan(gnnco_handle* h, const uint8_t* active, voi
   w.n_tiles = (int32_t)tab.t0.size(); w.n_pairs = (int32_t)tab.p0.size(); w.n_items = (int32_t)tab.i0.size();
   w.n_wg_chunks = (int32_t)tab.wb.size(); w.n_wg_multi = (int32_t)tab.mp.size();
   w.row_chunks.row0 = P.chunk_row0; w.row_chunks.rows = P.chunk_rows; w.row_chunks.count = (int32_t)tab.c0.size();
+  w.fuse = P.fuse;
+  {
+    const int32_t rc = build_fuse_set(h, P.pair_row0, P.pair_rows, tab.p0, tab.pr, w.fuse, st);
+    if (rc != GNNCO_OK) return rc;
+  }
   int32_t count = 0;
   for (uint8_t f : flags) count += f ? 1 : 0;
   h->plan_active = active;

@@ -29,7 +29,8 @@ constexpr int kItemRows = 1024;      // rows of one objective work item (never s
 // Kernel families, for launch accounting and per-kernel timing.
 enum KernelKind {
   K_AGG_FWD, K_AGG_BWD, K_TRANSFORM_FWD, K_TRANSFORM_BWD, K_WEIGHT_GRAD, K_GEMV, K_WEIGHT_GRAD_VEC, K_RANK1,
-  K_SUM_SETS, K_CAST, K_ADAM, K_OUT_FWD, K_OBJECTIVE, K_OUT_BWD, K_DECODE, K_STAGE3, K_AGG_RANK1, K_EMBED, K_KIND_COUNT
+  K_SUM_SETS, K_CAST, K_ADAM, K_OUT_FWD, K_OBJECTIVE, K_OUT_BWD, K_DECODE, K_STAGE3, K_AGG_RANK1, K_EMBED,
+  K_AGG_TRANSFORM, K_KIND_COUNT
 };
 
 // Optional per-kernel timing: while `on`, every launcher brackets its launches with a pair
@@ -71,6 +72,21 @@ __device__ __forceinline__ bool chunk_row(const RowChunks& rc, int64_t linear, i
   return off < rc.rows[c];
 }
 
+// Work tables of the hidden layer that runs as one kernel (tc_gemm2.cu).  The double tiles are split into
+// LIGHT ones (short rows only: the kernel's adders give every row to one warp) with each CTA's extent in the
+// source list, cut into per-cluster ranges of about equal cost, and HEAVY ones (a long row or many entries),
+// which go through the separate aggregation and transform kernels -- their tables have the format of the
+// double-tile tables and of RowChunks.
+struct FuseSet {
+  int4* meta = nullptr;                 // [2 n_light] {tile's first row, this CTA's rows, list extent begin, end}
+  int32_t* cluster_begin = nullptr;     // [clusters + 1] light tiles of each CTA pair
+  int32_t *light_row0 = nullptr, *light_rows = nullptr, *heavy_row0 = nullptr, *heavy_rows = nullptr;
+  int2* weights = nullptr;              // [tiles] scratch of the build: {list entries, longest row}
+  int32_t n_light = 0, n_heavy = 0, clusters = 0;
+  bool built = false;
+};
+constexpr int kFuseMaxClusters = 256;
+
 // The per-graph work tables that the kernels of a step walk.  The handle holds the set for all
 // subgraphs; gnnco_active_plan builds a second set for the active subgraphs only, and a step with
 // GNNCO_ACTIVE_ONLY runs with that set swapped in.
@@ -81,6 +97,7 @@ struct WorkSet {
   int32_t *wg_mpart = nullptr, *wg_mfirst = nullptr, *wg_mcount = nullptr;
   int32_t n_tiles = 0, n_pairs = 0, n_items = 0, n_wg_chunks = 0, n_wg_multi = 0;
   RowChunks row_chunks;
+  FuseSet fuse;
 };
 
 struct gnnco_handle {
@@ -99,6 +116,8 @@ struct gnnco_handle {
   int32_t *item_row0 = nullptr, *item_row1 = nullptr;      // objective work items
   int32_t* part_item_ptr = nullptr;                        // [S+1] items of each subgraph
   int32_t* status = nullptr;                               // device status word + counters
+  FuseSet fuse;                                            // tables of the one-kernel layer for the running work set
+  int32_t* src_list = nullptr;                             // per row: its own index, then its neighbours' (n + 2 E_in entries)
   int4* row_head = nullptr;                                // {first CSR slot, degree, first two neighbours} per row
   int32_t* long_rows = nullptr;                            // ids of rows with degree > kLongRowDegree, ascending
   // the long rows' neighbour lists cut into segments: CSR slots [seg_begin, seg_end) of each segment, and
@@ -180,6 +199,19 @@ struct Carver {
   bool ok() const { return off <= cap; }
 };
 
+// the arrays of a FuseSet for at most `tiles` double tiles
+inline FuseSet carve_fuse_set(Carver& c, size_t tiles) {
+  FuseSet f;
+  f.meta = c.take<int4>(2 * tiles);
+  f.cluster_begin = c.take<int32_t>(kFuseMaxClusters + 1);
+  f.light_row0 = c.take<int32_t>(tiles);
+  f.light_rows = c.take<int32_t>(tiles);
+  f.heavy_row0 = c.take<int32_t>(tiles);
+  f.heavy_rows = c.take<int32_t>(tiles);
+  f.weights = c.take<int2>(tiles);
+  return f;
+}
+
 // ---- partition.cu : device primitives (stable LSD radix sort of 64-bit keys on bits [bit_lo, bit_hi) with an
 // optional 32-bit payload, exclusive scan of int32) and the sizes of their scratch arrays
 int32_t device_exclusive_scan(int32_t* data, int64_t N, int32_t* tile_sums, cudaStream_t st);
@@ -245,6 +277,15 @@ int32_t launch_transform_tc_pair(gnnco_handle* h, const void* A, const void* B, 
                                  int K, int N, bool relu, const float* row_scale, const uint8_t* mask_bits,
                                  uint8_t* bits_out, bool backward, const void* dot_w, int64_t dot_stride, float* dot_out,
                                  cudaStream_t st);
+bool aggregate_transform_pair_supported(gnnco_handle* h, int dtype, int K, int N);
+// Fills `fs` (whose arrays the caller has carved: meta 2 x tiles, cluster_begin kFuseMaxClusters + 1, the four
+// row tables and weights `tiles` each) for the double tiles p0 / pr (host copies of d_pair_row0 / d_pair_rows).
+// Synchronises `st`.  Leaves fs.built false where the one-kernel layer cannot run on this device or graph.
+int32_t build_fuse_set(gnnco_handle* h, const int32_t* d_pair_row0, const int32_t* d_pair_rows,
+                       const std::vector<int32_t>& p0, const std::vector<int32_t>& pr, FuseSet& fs, cudaStream_t st);
+int32_t launch_aggregate_transform_pair(gnnco_handle* h, const void* Hin, const void* B, int64_t b_stride, int32_t b_sets,
+                                        void* Y, int K, int N, const float* row_scale, uint8_t* bits_out, const void* dot_w,
+                                        int64_t dot_stride, float* dot_out, cudaStream_t st);
 bool tc_pair_weight_grad_supported(gnnco_handle* h, int dtype, int K, int N);
 int32_t launch_weight_grad_tc_pair(gnnco_handle* h, const void* A, const void* G, float* dW, float* scratch, int K, int N,
                                    cudaStream_t st);

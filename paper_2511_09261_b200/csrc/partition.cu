@@ -317,6 +317,19 @@ __global__ void gather_rows_kernel(const char* src, char* dst, const int32_t* in
   else reinterpret_cast<uint32_t*>(dst)[t] = reinterpret_cast<const uint32_t*>(src)[s];
 }
 
+// src[rowptr[i] + i] = i, then row i's neighbours: what the fused aggregation + transform gathers for row i, in
+// the order the aggregation kernels add.  Four threads per row.
+__global__ void build_source_list(const int32_t* rowptr, const int32_t* colidx, int64_t n, int32_t* src) {
+  const int64_t g = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+  const int64_t i = g >> 2;
+  const int sub = (int)(g & 3);
+  if (i >= n) return;
+  const int32_t a = rowptr[i], b = rowptr[i + 1];
+  int32_t* dst = src + a + i;
+  if (sub == 0) dst[0] = (int32_t)i;
+  for (int32_t k = a + sub; k < b; k += 4) dst[1 + k - a] = colidx[k];
+}
+
 inline int bits_for(int64_t count) {   // bits needed to hold ids 0..count-1
   int b = 0;
   while (b < 32 && ((int64_t)1 << b) < count) ++b;
@@ -332,6 +345,8 @@ struct PersistentLayout {
   int32_t *pair_row0, *pair_rows;
   int32_t *tile_row0, *tile_rows, *item_row0, *item_row1, *part_item_ptr, *status, *long_rows, *seg_begin, *seg_end, *long_first_seg;
   int4* row_head;
+  int32_t* src_list;
+  FuseSet fuse;
   int32_t *wg_begin, *wg_end, *wg_slot, *wg_mpart, *wg_mfirst, *wg_mcount;
   int64_t max_chunks;
   int64_t max_tiles, max_items, max_long, max_segs;
@@ -368,6 +383,8 @@ PersistentLayout carve_persistent(void* base, int64_t n, int64_t E, int32_t S) {
   L.seg_end = c.take<int32_t>(L.max_segs);
   L.long_first_seg = c.take<int32_t>(L.max_long + 1);
   L.row_head = c.take<int4>(n);
+  L.src_list = c.take<int32_t>((size_t)n + 2 * E + 8);
+  L.fuse = carve_fuse_set(c, (size_t)L.max_tiles);
   L.max_chunks = (int64_t)S + n / kWgChunkMinRows + 1;
   L.wg_begin = c.take<int32_t>(L.max_chunks);
   L.wg_end = c.take<int32_t>(L.max_chunks);
@@ -529,7 +546,7 @@ extern "C" int32_t gnnco_partition_load(const gnnco_graph_desc* g, void* persist
   h->pair_row0 = P.pair_row0; h->pair_rows = P.pair_rows;
   h->tile_row0 = P.tile_row0; h->tile_rows = P.tile_rows; h->item_row0 = P.item_row0; h->item_row1 = P.item_row1;
   h->part_item_ptr = P.part_item_ptr; h->status = P.status; h->long_rows = P.long_rows; h->seg_begin = P.seg_begin; h->seg_end = P.seg_end;
-  h->long_first_seg = P.long_first_seg; h->row_head = P.row_head;
+  h->long_first_seg = P.long_first_seg; h->row_head = P.row_head; h->src_list = P.src_list;
   h->wg_begin = P.wg_begin; h->wg_end = P.wg_end; h->wg_slot = P.wg_slot;
   h->wg_mpart = P.wg_mpart; h->wg_mfirst = P.wg_mfirst; h->wg_mcount = P.wg_mcount;
 
@@ -602,7 +619,8 @@ extern "C" int32_t gnnco_partition_load(const gnnco_graph_desc* g, void* persist
   degree_scale<<<grid_for(n, T), T, 0, st>>>(P.rowptr, n, P.inv_deg, P.status);
   collect_long_rows<<<grid_for(n, T), T, 0, st>>>(P.rowptr, n, P.long_rows, (int32_t)P.max_long, P.status);
   build_row_heads<<<grid_for(n, T), T, 0, st>>>(P.rowptr, P.colidx, n, P.row_head);
-  h->launches += 3;
+  build_source_list<<<grid_for(n * 4, T), T, 0, st>>>(P.rowptr, P.colidx, n, P.src_list);
+  h->launches += 4;
   GNNCO_LAUNCH_CHECK();
 
   // 5. host-built tables: dense-transform tiles, objective work items, weight-gradient chunks (from part_ptr)
@@ -675,6 +693,10 @@ extern "C" int32_t gnnco_partition_load(const gnnco_graph_desc* g, void* persist
     GNNCO_CUDA_TRY(up(P.long_first_seg, first));
     GNNCO_CUDA_TRY(cudaStreamSynchronize(st));      // the host vectors go out of scope
   }
+  // tables of the hidden layer that runs as one kernel (light / heavy double tiles, per-cluster ranges)
+  h->fuse = P.fuse;
+  rc = build_fuse_set(h, P.pair_row0, P.pair_rows, p0, pr, h->fuse, st);
+  if (rc != GNNCO_OK) return rc;
   guard.h = nullptr;
   *out = h;
   return GNNCO_OK;

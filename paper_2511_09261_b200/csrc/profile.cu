@@ -8,7 +8,7 @@ namespace {
 const char* kKindNames[K_KIND_COUNT] = {
     "aggregate_fwd", "aggregate_bwd", "transform_fwd", "transform_bwd", "weight_grad", "gemv", "weight_grad_vec",
     "rank1_masked", "sum_over_sets", "cast_bf16", "adam", "output_forward", "objective", "output_backward", "decode",
-    "stage3_glue", "aggregate_rank1", "embeddings"};
+    "stage3_glue", "aggregate_rank1", "embeddings", "aggregate_transform"};
 }
 
 extern "C" int32_t gnnco_profile_begin(gnnco_handle* h) {

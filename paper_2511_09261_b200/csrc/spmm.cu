@@ -759,7 +759,7 @@ void launch_vec(const T* in, T* out, gnnco_handle* h, const float* scale, const 
   // overlaps with the streaming of its neighbours); otherwise (small or hub-dominated graphs,
   // where one such walk would be the tail of the kernel) they get a block each, on a side
   // stream, beside the short rows.
-  const double stream_us = 2.0 * (double)h->n * F * sizeof(T) / 4.0e6;          // at ~4 TB/s
+  const double stream_us = 2.0 * (double)linear_rows(h) * F * sizeof(T) / 4.0e6;   // at ~4 TB/s
   const double walk_us = (double)h->max_row / 4.0;
   const bool inline_first = stream_us > 3.0 * walk_us;
   if (inline_first) {

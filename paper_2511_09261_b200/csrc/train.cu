@@ -128,6 +128,7 @@ WorkSet capture_work(const gnnco_handle* h) {
   w.n_tiles = h->n_tiles; w.n_pairs = h->n_pairs; w.n_items = h->n_items; w.n_wg_chunks = h->n_wg_chunks;
   w.n_wg_multi = h->n_wg_multi;
   w.row_chunks = h->row_chunks;
+  w.fuse = h->fuse;
   return w;
 }
 
@@ -139,6 +140,7 @@ void apply_work(gnnco_handle* h, const WorkSet& w) {
   h->n_tiles = w.n_tiles; h->n_pairs = w.n_pairs; h->n_items = w.n_items; h->n_wg_chunks = w.n_wg_chunks;
   h->n_wg_multi = w.n_wg_multi;
   h->row_chunks = w.row_chunks;
+  h->fuse = w.fuse;
 }
 
 // A step over all subgraphs, or (GNNCO_ACTIVE_ONLY) the same launch sequence with the plan's work tables
@@ -196,7 +198,40 @@ int32_t run_step_on(gnnco_handle* h, const gnnco_model_desc* m, const void* X, c
   for (int l = 1; l < L; ++l) {
     // aggregated input M_l; the first layer's can be kept across steps (X does not change)
     const void* Min = T.Ga;
-    if (l == 1 && (flags & (GNNCO_AX_STORE | GNNCO_AX_REUSE))) Min = out->ax_cache;
+    const bool cached_first = l == 1 && (flags & (GNNCO_AX_STORE | GNNCO_AX_REUSE));
+    if (cached_first) Min = out->ax_cache;
+    // on request, aggregation and transform in one kernel where there is one: M_l never reaches HBM (the
+    // backward pass does not need it: dW_l = H_{l-1}^T Q_l)
+    const bool one_kernel = (flags & GNNCO_ONE_KERNEL_LAYERS) && !cached_first && T.W_lp_t[l - 1] &&
+                            aggregate_transform_pair_supported(h, dt, m->dims[l - 1], m->dims[l]) &&
+                            !((uintptr_t)Hprev & 15);
+    if (one_kernel) {
+      const bool fuse = (l == L - 1);
+      uint8_t* bits = l < L - 1 ? T.Hbits[l] : nullptr;
+      if (h->fuse.n_light > 0)
+        GNNCO_TRY(launch_aggregate_transform_pair(h, Hprev, T.W_lp_t[l - 1], wstride[l - 1], sets, T.H[l], m->dims[l - 1],
+                                                  m->dims[l], h->inv_deg, bits, fuse ? Wc[L - 1] : nullptr, wstride[L - 1],
+                                                  fuse ? T.u : nullptr, st));
+      if (h->fuse.n_heavy > 0) {
+        // double tiles with a long row or very many entries: the two separate kernels, over those tiles only
+        // (their table has the format of the double-tile table and of the row chunks)
+        const WorkSet all = capture_work(h);
+        h->pair_row0 = h->fuse.heavy_row0; h->pair_rows = h->fuse.heavy_rows; h->n_pairs = h->fuse.n_heavy;
+        h->row_chunks.row0 = h->fuse.heavy_row0; h->row_chunks.rows = h->fuse.heavy_rows;
+        h->row_chunks.count = h->fuse.n_heavy;
+        rc = launch_aggregate(h, dt, Hprev, T.Ga, m->dims[l - 1], h->inv_deg, nullptr, st);
+        if (rc == GNNCO_OK)
+          rc = launch_transform_tc_pair(h, T.Ga, T.W_lp_t[l - 1], wstride[l - 1], sets, T.H[l], m->dims[l - 1], m->dims[l],
+                                        true, nullptr, nullptr, bits, false, fuse ? Wc[L - 1] : nullptr, wstride[L - 1],
+                                        fuse ? T.u : nullptr, st);
+        apply_work(h, all);
+        if (rc != GNNCO_OK) return rc;
+      }
+      bits_written[l] = bits != nullptr;
+      u_done = fuse;
+      Hprev = T.H[l];
+      continue;
+    }
     if (!(l == 1 && (flags & GNNCO_AX_REUSE)))
       GNNCO_TRY(launch_aggregate(h, dt, Hprev, const_cast<void*>(Min), m->dims[l - 1], h->inv_deg, nullptr, st));
     if (T.W_lp_t[l - 1]) {
@@ -341,7 +376,7 @@ int32_t check_step_args(const gnnco_handle* h, const gnnco_model_desc* m, const 
   int32_t rc = check_model(h, m, true);
   if (rc != GNNCO_OK) return rc;
   if (flags & ~(GNNCO_WANT_DX | GNNCO_FORWARD_ONLY | GNNCO_AX_STORE | GNNCO_AX_REUSE | GNNCO_WEIGHTS_UNTOUCHED |
-                GNNCO_ACTIVE_ONLY))
+                GNNCO_ACTIVE_ONLY | GNNCO_ONE_KERNEL_LAYERS))
     return GNNCO_INVALID_ARGUMENT;
   if (flags & GNNCO_ACTIVE_ONLY) {
     if (flags & (GNNCO_AX_STORE | GNNCO_AX_REUSE)) return GNNCO_INVALID_ARGUMENT;

@@ -150,6 +150,7 @@ class StepCase:
         self.sets = self.S if sets is None else sets
         self.alpha, self.beta, self.lam = alpha, beta, lam
         self.report = Report()
+        self.extra_flags = 0                      # ORed into the step's flags (e.g. ONE_KERNEL_LAYERS)
 
     def run(self, graph, X_new, W, pen_new=None, want_dx=True, adam=None, threads=4, parts=None, label=""):
         """X_new [n,F0] float32 numpy (bf16-representable when dtype is bf16), W list of
@@ -172,7 +173,7 @@ class StepCase:
         z = torch.full((self.n,), float("nan"), device=Xd.device)
         dX = torch.full_like(Xd, float("nan")) if want_dx else None
         pen_d = to_dev(pen_new.astype(np.float32)) if pen_new is not None else None
-        flags = gnnco.WANT_DX if want_dx else 0
+        flags = (gnnco.WANT_DX if want_dx else 0) | self.extra_flags
         loss, p = graph.train_step(model, Xd, self.alpha, self.beta, self.lam, pen_d, opt, z=z, dW=dW, dX=dX,
                                    flags=flags)
         torch.cuda.synchronize()

@@ -235,6 +235,54 @@ def test_cached_first_aggregation_is_bit_identical(cfg):
         assert e.value.status == gnnco.INVALID_ARGUMENT
 
 
+@pytest.mark.parametrize("dims,n,S", [([256, 256, 1], 3100, 5), ([256, 256, 256, 1], 3100, 5),
+                                      ([256, 256, 256, 1], 70000, 24)])
+def test_one_kernel_layers_equal_the_separate_kernels_bit_for_bit(dims, n, S):
+    """GNNCO_ONE_KERNEL_LAYERS, width 256 in bfloat16: a hidden layer runs as ONE kernel (the aggregated rows
+    are summed on chip into the MMA operand).  It adds a row's sources in the order of the stand-alone
+    aggregation kernel, so where no row is long enough for that kernel to sum it by segments the step must
+    give the bits of the plain step: loss, p, dX and the weights after two Adam steps.  The large case gives
+    every CTA pair several double tiles and several subgraphs (ring wrap-around, weight reloads)."""
+    import torch
+    import paper_2511_09261_b200 as gnnco
+    eu, ev, part = tiny_graph(n, float(S) / n, S, seed=131)     # about one neighbour inside the subgraph per row
+    graph = load_graph(n, eu, ev, part, S)
+    assert graph.max_row <= 256
+    X = to_dev(rand_features(n, dims[0], 137).astype(np.float32)).to(torch.bfloat16)
+    runs = []
+    for extra in (gnnco.ONE_KERNEL_LAYERS, 0):
+        W = [to_dev(si.round_to_bf16(w.astype(np.float32))) for w in rand_weights(dims, S, 139)]
+        model = gnnco.Model(dims, W, feat_dtype=gnnco.BF16)
+        opt = gnnco.Adam(model, lr=1e-2)
+        trace = []
+        before = graph.launch_count()
+        for step in range(2):
+            dX = torch.empty_like(X)
+            loss, p = graph.train_step(model, X, 2.0, 1.0, opt=opt, dX=dX, flags=gnnco.WANT_DX | extra)
+            trace += [loss.clone(), p.clone(), dX]
+        runs.append(trace + [t.clone() for t in W] + [graph.launch_count() - before])
+    assert runs[0][-1] < runs[1][-1]                 # the flag really replaced launches
+    for a, b in zip(runs[0][:-1], runs[1][:-1]):
+        assert torch.equal(a, b)
+
+
+@pytest.mark.parametrize("graph_name,dims", [("big_hub", [256, 256, 1]), ("big_hub", [256, 256, 256, 1]),
+                                             ("dense_small", [256, 256, 256, 1]), ("empty_parts", [256, 256, 1]), ("no_edges", [256, 256, 1])])
+def test_one_kernel_layers_against_the_oracle(graph_name, dims):
+    """The same flag on graphs with a hub row (its double tile goes through the separate kernels, the others
+    through the one-kernel layer) and on a small dense-ish graph, against the oracle."""
+    import paper_2511_09261_b200 as gnnco
+    eu, ev, part = GRAPHS[graph_name]()
+    n, S = _n_S(part)
+    book = oracle.bookkeeping(n, eu, ev, part, S)
+    graph = load_graph(n, eu, ev, part, S)
+    X = si.round_to_bf16(rand_features(n, dims[0], 31).astype(np.float32))
+    W = [si.round_to_bf16(w.astype(np.float32)) for w in rand_weights(dims, S, 37)]
+    case = StepCase(book, dims, "bf16", S)
+    case.extra_flags = gnnco.ONE_KERNEL_LAYERS
+    case.run(graph, X, W, None, want_dx=True, label="one-kernel")
+
+
 def test_weight_copies_left_by_adam_are_bit_identical_to_fresh_ones():
     """bfloat16 run: with GNNCO_WEIGHTS_UNTOUCHED the step reuses the bfloat16 weight copies that the
     previous step's Adam kernel wrote; four steps (the third with only some subgraphs active, then a
@@ -318,7 +366,7 @@ def test_train_step_bf16_long_subgraphs(dims, n, S):
     case.run(graph, X, W, None, want_dx=True, adam=adam, label="bf16-long")
 
 
-@pytest.mark.parametrize("dims", [[256, 64, 1], [64, 64, 1], [512, 64, 1]])
+@pytest.mark.parametrize("dims", [[256, 64, 1], [64, 64, 1], [512, 64, 1], [256, 256, 1]])
 def test_train_step_bf16_hub_row(dims):
     """A hub row longer than the block-per-row threshold, bf16 features."""
     eu, ev, part = GRAPHS["big_hub"]()
@@ -352,7 +400,7 @@ def test_train_step_f32_tensor_core_widths(dims, n, S, sets):
 
 
 @pytest.mark.parametrize("dtype,dims,n,S", [("bf16", [256, 128, 1], 9000, 2), ("f32", [128, 64, 1], 7000, 1),
-                                            ("bf16", [256, 256, 256, 1], 7000, 3),
+                                            ("bf16", [256, 256, 1], 7000, 3),
                                             ("bf16", [128, 128, 1], 6100, 3), ("f32", [64, 36, 1], 7000, 1),
                                             ("f32", [20, 24, 1], 5000, 2)])
 def test_train_step_few_very_long_subgraphs(dtype, dims, n, S):

@@ -120,9 +120,12 @@ def test_fine_tune_updates_active_subgraphs_only():
     assert e.value.status == gnnco.INVALID_ARGUMENT
 
 
-@pytest.mark.parametrize("dtype,dims,n,S", [("f32", [48, 24, 1], 900, 7), ("f32", [128, 128, 64, 1], 3000, 9),
-                                            ("bf16", [256, 256, 256, 1], 6000, 11), ("bf16", [64, 32, 1], 700, 5)])
-def test_active_only_step_equals_the_full_step_on_active_subgraphs(dtype, dims, n, S):
+@pytest.mark.parametrize("dtype,dims,n,S,one_kernel", [("f32", [48, 24, 1], 900, 7, False),
+                                                       ("f32", [128, 128, 64, 1], 3000, 9, False),
+                                                       ("bf16", [256, 256, 256, 1], 6000, 11, False),
+                                                       ("bf16", [256, 256, 256, 1], 6000, 11, True),
+                                                       ("bf16", [64, 32, 1], 700, 5, False)])
+def test_active_only_step_equals_the_full_step_on_active_subgraphs(dtype, dims, n, S, one_kernel):
     """A fine-tuning step restricted to the active subgraphs (gnnco_active_plan + GNNCO_ACTIVE_ONLY): loss, p, z,
     dW, dX and the updated weights and moments of every ACTIVE subgraph are bit-identical to those of a full
     step with the same Adam mask; everything that belongs to an inactive subgraph keeps the value it had
@@ -157,7 +160,7 @@ def test_active_only_step_equals_the_full_step_on_active_subgraphs(dtype, dims, 
             z = torch.full((n,), canary, device=X.device)
             dW = [torch.full_like(w, canary) for w in W]
             dX = torch.full_like(X, canary)
-            flags = gnnco.WANT_DX
+            flags = gnnco.WANT_DX | (gnnco.ONE_KERNEL_LAYERS if one_kernel else 0)   # the plan has its own tables for it
             if only:
                 assert graph.active_plan(active) == int(flags_np.sum())
                 flags |= gnnco.ACTIVE_ONLY
