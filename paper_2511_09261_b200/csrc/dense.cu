@@ -99,18 +99,21 @@ __global__ void __launch_bounds__(256) transform_fma(const TA* __restrict__ A, c
   }
 }
 
-// dW[s] tile (64 x 64) = sum over the rows of subgraph s of A[i, k]^T G[i, n]
+// One 64 x 64 tile of  sum over the rows of one chunk of A[i, k]^T G[i, n].  A chunk of the weight-gradient chunk
+// table is a whole subgraph, or a run of rows of a very long one whose partial result goes to a scratch slot and
+// is combined in chunk order afterwards (as in the tensor-core kernels): a partition into a few large
+// subgraphs still gives the whole GPU work.
 template <typename TA>
 __global__ void __launch_bounds__(256) weight_grad_fma(const TA* __restrict__ A, const TA* __restrict__ G,
-                                                       float* __restrict__ dW, int K, int N,
-                                                       const int32_t* __restrict__ part_ptr,
-                                                       const uint8_t* __restrict__ only) {
+                                                       float* __restrict__ dW, float* __restrict__ scratch, int K, int N,
+                                                       const int32_t* __restrict__ wg_begin,
+                                                       const int32_t* __restrict__ wg_end,
+                                                       const int32_t* __restrict__ wg_slot) {
   __shared__ __align__(16) float As[16][64 + 4];
   __shared__ __align__(16) float Gs[16][64 + 4];
   const int tid = threadIdx.x, tx = tid & 15, ty = tid >> 4;
-  const int s = blockIdx.x, k0 = blockIdx.y * 64, n0 = blockIdx.z * 64;
-  if (only && !only[s]) return;               // a step on the active subgraphs only (uniform across the block)
-  const int64_t ra = part_ptr[s], rb = part_ptr[s + 1];
+  const int c = blockIdx.x, k0 = blockIdx.y * 64, n0 = blockIdx.z * 64;
+  const int64_t ra = wg_begin[c], rb = wg_end[c];
   float acc[4][4];
 #pragma unroll
   for (int i = 0; i < 4; ++i)
@@ -138,7 +141,8 @@ __global__ void __launch_bounds__(256) weight_grad_fma(const TA* __restrict__ A,
     }
     __syncthreads();
   }
-  float* out = dW + (int64_t)s * K * N;
+  const int32_t slot = wg_slot[c];       // < 0: the whole subgraph -(slot + 1); >= 0: scratch slot of a split subgraph
+  float* out = slot < 0 ? dW + (int64_t)(-(slot + 1)) * K * N : scratch + (int64_t)slot * K * N;
 #pragma unroll
   for (int i = 0; i < 4; ++i)
 #pragma unroll
@@ -441,23 +445,23 @@ int32_t launch_gemv(gnnco_handle* h, int dtype, const void* H, const void* w, in
   return GNNCO_OK;
 }
 
-int32_t launch_weight_grad(gnnco_handle* h, int dtype, const void* A, const void* G, float* dW, int K, int N,
-                           cudaStream_t stream) {
+int32_t launch_weight_grad(gnnco_handle* h, int dtype, const void* A, const void* G, float* dW, float* scratch, int K,
+                           int N, cudaStream_t stream) {
   ProfScope prof_(h, K_WEIGHT_GRAD, stream);
-  dim3 grid(h->S, (K + 63) / 64, (N + 63) / 64);
+  if (h->n_wg_chunks <= 0) return GNNCO_OK;
+  dim3 grid(h->n_wg_chunks, (K + 63) / 64, (N + 63) / 64);
   if (grid.y > 65535 || grid.z > 65535) return GNNCO_UNSUPPORTED;
   if (dtype == GNNCO_F32)
-    weight_grad_fma<float><<<grid, 256, 0, stream>>>((const float*)A, (const float*)G, dW, K, N, h->part_ptr,
-                                                     h->row_chunks.row0 ? h->plan_active : nullptr);
+    weight_grad_fma<float><<<grid, 256, 0, stream>>>((const float*)A, (const float*)G, dW, scratch, K, N, h->wg_begin,
+                                                     h->wg_end, h->wg_slot);
   else if (dtype == GNNCO_BF16)
-    weight_grad_fma<__nv_bfloat16><<<grid, 256, 0, stream>>>((const __nv_bfloat16*)A, (const __nv_bfloat16*)G, dW, K,
-                                                             N, h->part_ptr,
-                                                             h->row_chunks.row0 ? h->plan_active : nullptr);
+    weight_grad_fma<__nv_bfloat16><<<grid, 256, 0, stream>>>((const __nv_bfloat16*)A, (const __nv_bfloat16*)G, dW, scratch,
+                                                             K, N, h->wg_begin, h->wg_end, h->wg_slot);
   else
     return GNNCO_UNSUPPORTED;
   h->launches += 1;
   GNNCO_LAUNCH_CHECK();
-  return GNNCO_OK;
+  return launch_wg_combine(h, scratch, dW, (int64_t)K * N, stream);
 }
 
 int32_t launch_weight_grad_vec(gnnco_handle* h, int dtype, const void* H, const float* g, float* dw, float* scratch,

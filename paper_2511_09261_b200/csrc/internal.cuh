@@ -243,8 +243,8 @@ int32_t launch_transform(gnnco_handle* h, int dtype, const void* A, const void* 
 int32_t launch_gemv(gnnco_handle* h, int dtype, const void* H, const void* w, int64_t w_stride, float* u, int F,
                     cudaStream_t st);
 // dW[s] (K x N) = sum_{i in s} A[i,:]^T G[i,:]
-int32_t launch_weight_grad(gnnco_handle* h, int dtype, const void* A, const void* G, float* dW, int K, int N,
-                           cudaStream_t st);
+int32_t launch_weight_grad(gnnco_handle* h, int dtype, const void* A, const void* G, float* dW, float* scratch, int K,
+                           int N, cudaStream_t st);
 // dw[s][f] = sum_{i in s} H[i,f] g[i]; scratch: F floats per slot of the weight-gradient chunk table.
 // bits_out (optional, n x F/8 bytes): receives [H > 0], one bit per element, when the kernel that runs
 // can produce it; *wrote_bits says whether it did.

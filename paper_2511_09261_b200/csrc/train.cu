@@ -362,7 +362,7 @@ int32_t run_step_on(gnnco_handle* h, const gnnco_model_desc* m, const void* X, c
       GNNCO_TRY(launch_weight_grad_tc(h, Hin, Q, wg_out, T.wg_scratch, K, N, st));
     else if (dt == GNNCO_F32 && tc_f32_weight_grad_supported(K, N))
       GNNCO_TRY(launch_weight_grad_tc_f32(h, Hin, Q, wg_out, T.wg_scratch, K, N, st));
-    else GNNCO_TRY(launch_weight_grad(h, dt, Hin, Q, wg_out, K, N, st));
+    else GNNCO_TRY(launch_weight_grad(h, dt, Hin, Q, wg_out, T.wg_scratch, K, N, st));
     if (sets == 1) GNNCO_TRY(launch_sum_over_sets(h, T.dW_sets, target, (int64_t)K * N, h->S, st));
     GNNCO_TRY(finish_layer(l - 1, target));
     if (l > 1) GNNCO_TRY(launch_aggregate(h, dt, other, Q, K, nullptr, nullptr, st));   // Q_{l-1} = (A+I) R
