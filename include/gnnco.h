@@ -262,9 +262,12 @@ int32_t gnnco_active_plan(gnnco_handle* h, const uint8_t* active, void* plan_ws,
 
 /* Same step with HOST buffers for the per-step data: X_host [n x dims[0]] (feat_dtype,
  * new order; pinned memory recommended), pen_host [n] or NULL, loss_host [S], p_host [n].
- * Weights, Adam moments and the work area stay on the device.  Copies run on `stream`,
- * which is synchronised before returning.  ws must hold
- * gnnco_train_host_workspace_bytes bytes. */
+ * Weights, Adam moments and the work area stay on the device.  `stream` is synchronised before
+ * returning.  Inputs of 64 MB and more (L >= 2, S >= 2, no GNNCO_ACTIVE_ONLY) are uploaded in eight
+ * ranges of subgraphs on a stream of the handle's own, ordered after whatever `stream` held at the call,
+ * and the first hidden layer (Eq. 3 needs only a subgraph's own rows of X) runs on each range as it
+ * arrives; smaller inputs are copied on `stream` itself.  Results are bit-identical to gnnco_train_step on
+ * the same data either way.  ws must hold gnnco_train_host_workspace_bytes bytes. */
 int32_t gnnco_train_host_workspace_bytes(const gnnco_handle* h, const gnnco_model_desc* m, uint32_t flags,
                                          size_t* bytes);
 int32_t gnnco_train_step_host(gnnco_handle* h, const gnnco_model_desc* m, const void* X_host, float alpha,

@@ -100,6 +100,16 @@ struct WorkSet {
   FuseSet fuse;
 };
 
+// The host-buffer step lets layer 1 start on a range of subgraphs as soon as that range of X has been uploaded:
+// per range the event its copy records and where its tiles and double tiles start in the tables.
+constexpr int kArrivalGroups = 8;
+struct ArrivalPlan {
+  int groups = 0;
+  cudaEvent_t ev[kArrivalGroups] = {};
+  cudaEvent_t ev_rest = nullptr;                             // everything else the step uploads (the penalty mask)
+  int32_t tile0[kArrivalGroups + 1] = {}, pair0[kArrivalGroups + 1] = {};
+};
+
 struct gnnco_handle {
   int64_t n = 0, E = 0, E_in = 0, E_b = 0;
   int32_t S = 0, max_row = 0;
@@ -147,6 +157,10 @@ struct gnnco_handle {
   bool shadow_fresh[GNNCO_MAX_LAYERS] = {false};
   // long rows are aggregated on a side stream, concurrently with the short rows
   cudaStream_t side_stream = nullptr;
+  // gnnco_train_step_host: the stream its uploads run on, their events, and (during such a step) the plan
+  cudaStream_t copy_stream = nullptr;
+  cudaEvent_t ev_arrive[kArrivalGroups] = {}, ev_rest = nullptr, ev_begin = nullptr;
+  const ArrivalPlan* arrival = nullptr;
   cudaEvent_t ev_fork = nullptr, ev_join = nullptr;
 };
 

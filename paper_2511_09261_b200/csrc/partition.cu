@@ -742,6 +742,11 @@ extern "C" int32_t gnnco_destroy(gnnco_handle* h) {
     if (h->ev_fork) cudaEventDestroy(h->ev_fork);
     if (h->ev_join) cudaEventDestroy(h->ev_join);
     if (h->side_stream) cudaStreamDestroy(h->side_stream);
+    if (h->copy_stream) cudaStreamDestroy(h->copy_stream);
+    for (cudaEvent_t e : h->ev_arrive)
+      if (e) cudaEventDestroy(e);
+    if (h->ev_rest) cudaEventDestroy(h->ev_rest);
+    if (h->ev_begin) cudaEventDestroy(h->ev_begin);
   }
   delete h;
   return GNNCO_OK;

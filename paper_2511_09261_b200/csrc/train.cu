@@ -195,14 +195,15 @@ int32_t run_step_on(gnnco_handle* h, const gnnco_model_desc* m, const void* X, c
   const void* Hprev = X;
   bool u_done = false;
   bool bits_written[GNNCO_MAX_LAYERS] = {false};
-  for (int l = 1; l < L; ++l) {
+  // hidden layer l of the forward pass over the work tables that the handle holds at the moment
+  auto forward_layer = [&](int l, const void* Hprev) -> int32_t {
     // aggregated input M_l; the first layer's can be kept across steps (X does not change)
     const void* Min = T.Ga;
     const bool cached_first = l == 1 && (flags & (GNNCO_AX_STORE | GNNCO_AX_REUSE));
     if (cached_first) Min = out->ax_cache;
     // on request, aggregation and transform in one kernel where there is one: M_l never reaches HBM (the
     // backward pass does not need it: dW_l = H_{l-1}^T Q_l)
-    const bool one_kernel = (flags & GNNCO_ONE_KERNEL_LAYERS) && !cached_first && T.W_lp_t[l - 1] &&
+    const bool one_kernel = (flags & GNNCO_ONE_KERNEL_LAYERS) && !cached_first && !(l == 1 && h->arrival) && T.W_lp_t[l - 1] &&
                             aggregate_transform_pair_supported(h, dt, m->dims[l - 1], m->dims[l]) &&
                             !((uintptr_t)Hprev & 15);
     if (one_kernel) {
@@ -229,8 +230,7 @@ int32_t run_step_on(gnnco_handle* h, const gnnco_model_desc* m, const void* X, c
       }
       bits_written[l] = bits != nullptr;
       u_done = fuse;
-      Hprev = T.H[l];
-      continue;
+      return GNNCO_OK;
     }
     if (!(l == 1 && (flags & GNNCO_AX_REUSE)))
       GNNCO_TRY(launch_aggregate(h, dt, Hprev, const_cast<void*>(Min), m->dims[l - 1], h->inv_deg, nullptr, st));
@@ -262,6 +262,30 @@ int32_t run_step_on(gnnco_handle* h, const gnnco_model_desc* m, const void* X, c
     } else
       GNNCO_TRY(launch_transform(h, dt, Min, Wc[l - 1], wstride[l - 1], T.H[l], m->dims[l - 1], m->dims[l], false,
                                  true, nullptr, nullptr, st));
+    return GNNCO_OK;
+  };
+  for (int l = 1; l < L; ++l) {
+    const ArrivalPlan* ap = l == 1 ? h->arrival : nullptr;
+    if (ap && ap->groups > 1) {
+      // the host variant: X arrives in ranges of subgraphs on another stream; layer 1 follows range by range
+      // (the tables are ordered by subgraph, so a range of subgraphs is a range of each table)
+      const WorkSet all = capture_work(h);
+      rc = GNNCO_OK;
+      for (int g = 0; g < ap->groups && rc == GNNCO_OK; ++g) {
+        if (cudaStreamWaitEvent(st, ap->ev[g], 0) != cudaSuccess) { rc = GNNCO_CUDA_ERROR; break; }
+        h->tile_row0 = all.tile_row0 + ap->tile0[g]; h->tile_rows = all.tile_rows + ap->tile0[g];
+        h->n_tiles = ap->tile0[g + 1] - ap->tile0[g];
+        h->pair_row0 = all.pair_row0 + ap->pair0[g]; h->pair_rows = all.pair_rows + ap->pair0[g];
+        h->n_pairs = ap->pair0[g + 1] - ap->pair0[g];
+        h->row_chunks.row0 = h->pair_row0; h->row_chunks.rows = h->pair_rows; h->row_chunks.count = h->n_pairs;
+        if (h->n_pairs > 0) rc = forward_layer(1, Hprev);
+      }
+      apply_work(h, all);
+      if (rc != GNNCO_OK) return rc;
+      if (cudaStreamWaitEvent(st, ap->ev_rest, 0) != cudaSuccess) return GNNCO_CUDA_ERROR;
+    } else {
+      GNNCO_TRY(forward_layer(l, Hprev));
+    }
     Hprev = T.H[l];
   }
   const int FL = m->dims[L - 1];
@@ -442,18 +466,70 @@ extern "C" int32_t gnnco_train_step_host(gnnco_handle* h, const gnnco_model_desc
   if (T.bytes > ws_bytes) return GNNCO_WORKSPACE_TOO_SMALL;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   const size_t n = (size_t)h->n;
-  GNNCO_CUDA_TRY(cudaMemcpyAsync(T.X_stage, X_host, n * m->dims[0] * elem_size(m->feat_dtype),
-                                 cudaMemcpyHostToDevice, st));
+  const size_t row_bytes = (size_t)m->dims[0] * elem_size(m->feat_dtype);
   gnnco_objective obj{alpha, beta, lambda, nullptr};
-  if (pen_host) {
-    GNNCO_CUDA_TRY(cudaMemcpyAsync(T.pen_stage, pen_host, n * sizeof(float), cudaMemcpyHostToDevice, st));
-    obj.pen = T.pen_stage;
-  }
+  if (pen_host) obj.pen = T.pen_stage;
   gnnco_train_out out{};
   out.loss = T.loss_stage;
   out.p = T.p_stage;
-  rc = run_step(h, m, T.X_stage, &obj, opt, &out, flags, T, st);
-  if (rc != GNNCO_OK) return rc;
+  // Large inputs arrive in ranges of subgraphs on a second stream, and the first hidden layer (which needs nothing
+  // but a subgraph's own rows of X) follows them range by range; the rest of the step starts when all are there.
+  // Results are those of the plain order bit for bit: every subgraph is cut into the same tiles.
+  ArrivalPlan plan;
+  const bool in_ranges = m->L >= 2 && h->S >= 2 && !(flags & GNNCO_ACTIVE_ONLY) && n * row_bytes >= ((size_t)64 << 20);
+  if (in_ranges) {
+    if (!h->copy_stream) {
+      GNNCO_CUDA_TRY(cudaStreamCreateWithFlags(&h->copy_stream, cudaStreamNonBlocking));
+      for (cudaEvent_t& e : h->ev_arrive) GNNCO_CUDA_TRY(cudaEventCreateWithFlags(&e, cudaEventDisableTiming));
+      GNNCO_CUDA_TRY(cudaEventCreateWithFlags(&h->ev_rest, cudaEventDisableTiming));
+      GNNCO_CUDA_TRY(cudaEventCreateWithFlags(&h->ev_begin, cudaEventDisableTiming));
+    }
+    // whatever the caller queued on `stream` before this call comes first
+    GNNCO_CUDA_TRY(cudaEventRecord(h->ev_begin, st));
+    GNNCO_CUDA_TRY(cudaStreamWaitEvent(h->copy_stream, h->ev_begin, 0));
+    const std::vector<int32_t>& pp = h->h_part_ptr;
+    int32_t tiles = 0, pairs = 0, s = 0;
+    for (int g = 0; g < kArrivalGroups; ++g) {
+      plan.tile0[g] = tiles;
+      plan.pair0[g] = pairs;
+      const int32_t s_begin = s;
+      const int64_t until = g + 1 == kArrivalGroups ? (int64_t)n : (int64_t)n * (g + 1) / kArrivalGroups;
+      while (s < h->S && (pp[s + 1] <= until || g + 1 == kArrivalGroups)) {
+        const int32_t rows = pp[s + 1] - pp[s];
+        tiles += (rows + kGemmTileRows - 1) / kGemmTileRows;
+        pairs += (rows + 2 * kGemmTileRows - 1) / (2 * kGemmTileRows);
+        ++s;
+      }
+      const size_t r0 = (size_t)pp[s_begin], r1 = (size_t)pp[s];
+      if (r1 > r0)
+        GNNCO_CUDA_TRY(cudaMemcpyAsync(static_cast<char*>(T.X_stage) + r0 * row_bytes,
+                                       static_cast<const char*>(X_host) + r0 * row_bytes, (r1 - r0) * row_bytes,
+                                       cudaMemcpyHostToDevice, h->copy_stream));
+      plan.ev[g] = h->ev_arrive[g];
+      GNNCO_CUDA_TRY(cudaEventRecord(plan.ev[g], h->copy_stream));
+    }
+    plan.tile0[kArrivalGroups] = tiles;
+    plan.pair0[kArrivalGroups] = pairs;
+    plan.groups = kArrivalGroups;
+    if (tiles != h->n_tiles || pairs != h->n_pairs) return GNNCO_INTERNAL;
+    if (pen_host)
+      GNNCO_CUDA_TRY(cudaMemcpyAsync(T.pen_stage, pen_host, n * sizeof(float), cudaMemcpyHostToDevice, h->copy_stream));
+    plan.ev_rest = h->ev_rest;
+    GNNCO_CUDA_TRY(cudaEventRecord(plan.ev_rest, h->copy_stream));
+    h->arrival = &plan;
+    rc = run_step(h, m, T.X_stage, &obj, opt, &out, flags, T, st);
+    h->arrival = nullptr;
+  } else {
+    GNNCO_CUDA_TRY(cudaMemcpyAsync(T.X_stage, X_host, n * row_bytes, cudaMemcpyHostToDevice, st));
+    if (pen_host)
+      GNNCO_CUDA_TRY(cudaMemcpyAsync(T.pen_stage, pen_host, n * sizeof(float), cudaMemcpyHostToDevice, st));
+    rc = run_step(h, m, T.X_stage, &obj, opt, &out, flags, T, st);
+  }
+  if (rc != GNNCO_OK) {
+    cudaStreamSynchronize(st);                      // nothing of this call is in flight when it returns an error
+    if (h->copy_stream) cudaStreamSynchronize(h->copy_stream);
+    return rc;
+  }
   GNNCO_CUDA_TRY(cudaMemcpyAsync(loss_host, T.loss_stage, (size_t)h->S * sizeof(float), cudaMemcpyDeviceToHost, st));
   GNNCO_CUDA_TRY(cudaMemcpyAsync(p_host, T.p_stage, n * sizeof(float), cudaMemcpyDeviceToHost, st));
   GNNCO_CUDA_TRY(cudaStreamSynchronize(st));

@@ -337,6 +337,50 @@ def test_host_variant_matches_device_variant():
         assert torch.equal(a, b)
 
 
+@pytest.mark.parametrize("dtype,dims,n,S,hub", [("bf16", [256, 256, 256, 1], 150000, 37, False),
+                                                ("f32", [128, 128, 1], 140000, 3, True)])
+def test_host_variant_with_inputs_arriving_in_ranges(dtype, dims, n, S, hub):
+    """Inputs of 64 MB and more reach the device in ranges of subgraphs while the first hidden layer already
+    runs on the ranges that are there; two steps give the bits of two device-buffer steps (loss, p, weights).
+    The second case has a row too long for the row-per-warp kernel (summed by segments on a side stream)."""
+    import torch
+    import paper_2511_09261_b200 as gnnco
+    eu, ev = si.random_regular(n, 3, 211)
+    part = si.contiguous_partition(n, S)
+    if hub:                                         # node 5 joined to 700 nodes of its own subgraph
+        extra = np.arange(100, 800, dtype=eu.dtype)
+        keep = ~(((eu == 5) & (ev >= 100) & (ev < 800)) | ((ev == 5) & (eu >= 100) & (eu < 800)))
+        eu, ev = np.concatenate([eu[keep], np.full(700, 5, eu.dtype)]), np.concatenate([ev[keep], extra])
+    graph = load_graph(n, eu, ev, part, S)
+    assert (graph.max_row > 256) == hub
+    bf16 = dtype == "bf16"
+    perm = graph.arrays()["perm"].cpu().numpy()
+    X = rand_features(n, dims[0], 223).astype(np.float32)[perm]
+    Xh = torch.from_numpy(X)
+    if bf16:
+        Xh = Xh.to(torch.bfloat16)
+    Xh = Xh.pin_memory()
+    assert Xh.numel() * Xh.element_size() >= 64 << 20
+    pen = torch.from_numpy((si.uniform01(227, 0, n) < 0.3).astype(np.float32)).pin_memory()
+    res = []
+    for host in (False, True):
+        W = [to_dev(si.round_to_bf16(w.astype(np.float32))) for w in rand_weights(dims, S, 229)]
+        model = gnnco.Model(dims, W, gnnco.BF16 if bf16 else gnnco.F32)
+        opt = gnnco.Adam(model, lr=1e-2)
+        out = []
+        for step in range(2):
+            if host:
+                loss, p = graph.train_step_host(model, Xh, 2.0, 1.0, 0.5, pen, opt)
+                out += [loss.clone(), p.clone()]
+            else:
+                loss, p = graph.train_step(model, Xh.cuda(), 2.0, 1.0, 0.5, pen.cuda(), opt)
+                out += [loss.cpu(), p.cpu()]
+        res.append(out + [t.cpu() for t in W])
+    assert graph.async_status() == 0
+    for a, b in zip(*res):
+        assert torch.equal(a, b)
+
+
 def test_gather_rows_roundtrip():
     import torch
     w = si.make_workload(1)
