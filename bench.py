@@ -573,6 +573,9 @@ def run_reference(args):
     rank = int(os.environ.get("RANK", "0"))
     if rank != 0:
         return
+    if args.partition != "config":
+        print(json.dumps({"impl": "reference", "unavailable": "the oracle arm times the configuration's own partition only"}))
+        return
     w = si.make_workload(args.config, args.scale)
     threads = _host_threads()
     book, parts, items, edges, t_book = _oracle_sample(w, ORACLE_SAMPLE_PARTS[args.config])
@@ -587,7 +590,13 @@ def run_reference(args):
     line = dict(metric=METRIC, value=value, unit="edges/s", n_gpus=int(os.environ.get("WORLD_SIZE", "1")),
                 steps=args.steps, warmup=args.warmup, ms_per_step=dt * 1e3, higher_is_better=True, scaling="weak",
                 vs_baseline=None, dtype="f64", data="synthetic", impl="reference",
-                config=dict(workload=w.name, index=args.config, n=w.n, E=w.E, S=w.S, dims=w.dims),
+                # the workload keys of the GPU arm's line, from the same generators; the timed sample is under
+                # cpu_baseline
+                config=dict(workload=w.name, index=args.config, n=w.n, E=w.E, E_in=int(book["rowptr"][-1]) // 2,
+                            E_b=w.E - int(book["rowptr"][-1]) // 2, S=w.S, dims=w.dims,
+                            max_intra_degree=int(np.diff(book["rowptr"]).max()) if w.n else 0, weight_sets=w.S,
+                            want_dx=True, l2="host caches", partition="config", louvain=None,
+                            parallelism="1 process, host cores", storage=w.dtype),
                 cpu_baseline=dict(value=value, unit="edges/s", kind="oracle", cores=min(threads, len(items)),
                                   sample=sample),
                 e2e=dict(value=value, unit="edges/s", h2d_bytes_per_step=0, d2h_bytes_per_step=0), gpu_launches=0)
