@@ -482,6 +482,43 @@ def run_ours(args):
                           note="hidden layers as one kernel each (light double tiles) plus the separate kernels on the "
                                "heavy tiles; profiling events inside the timed loop")
 
+    # ---- launch-bound workloads: the same step and decode recorded once in a CUDA graph (Adam's step counter on
+    # the device) and replayed, timed like the headline (per-replay events, L2 flushed between replays)
+    graph_replay = None
+    if ms_per_step < 5.0 and not args.no_extras:
+        opt_g = gnnco.Adam(model, lr=w.lr, device_step=True)
+        side = torch.cuda.Stream()
+        fl = gnnco.WANT_DX | gnnco.WEIGHTS_UNTOUCHED
+
+        def step_on(stream, o):
+            graph.train_step(model, X, w.alpha, w.beta, w.lam, pen, o, loss=loss, p=p, dX=dX, flags=fl, stream=stream)
+            graph.decode_boundary(p, 0.5, x=x, viol=viol, per_part=per_part, counts=counts, stream=stream)
+
+        with torch.cuda.stream(side):
+            step_on(side, opt_g)
+            torch.cuda.synchronize()
+            cg = torch.cuda.CUDAGraph()
+            cg.capture_begin()
+            step_on(side, opt_g)
+            cg.capture_end()
+        torch.cuda.synchronize()
+        for _ in range(args.warmup):
+            cg.replay()
+        gs = [torch.cuda.Event(enable_timing=True) for _ in range(args.steps)]
+        ge = [torch.cuda.Event(enable_timing=True) for _ in range(args.steps)]
+        for k in range(args.steps):
+            if flush is not None:
+                flush.fill_(k)
+            gs[k].record()
+            cg.replay()
+            ge[k].record()
+        torch.cuda.synchronize()
+        gms = max_over_ranks(dist, sum(a.elapsed_time(b) for a, b in zip(gs, ge)) / args.steps, dev)
+        graph_replay = dict(ms_per_step=round(gms, 4), value=whole_job_value(graph.E_in, world, gms), unit="edges/s",
+                            note="one step + decode captured once (gnnco_adam_state.step_dev), one graph launch per step; "
+                                 "reported beside the headline, which launches kernel by kernel")
+        del cg
+
     # ---- end to end through the host-buffer entry point (rank-local; copies inside the timed region)
     e2e = None
     if not args.no_e2e:
@@ -531,7 +568,7 @@ def run_ours(args):
                         partition_load_ms=round(load_ms, 3), edges_per_s_whole_graph=value * w.E / max(1, graph.E_in)),
             roofline=roofline, spmm_fwd_bwd=spmm, aggregate_kernels=agg, kernels=kern, cpu_baseline=cpu, clocks=clocks, e2e=e2e,
             gpu_launches=int(launches), stage3_glue=stage3, fine_tune_step=(stage3 or {}).get("fine_tune_step"),
-            cached_first_aggregation=cached, one_kernel_layers=one_kernel)
+            cached_first_aggregation=cached, one_kernel_layers=one_kernel, cuda_graph_replay=graph_replay)
         print(json.dumps(line))
     if dist is not None:
         dist.destroy_process_group()

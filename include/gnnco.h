@@ -145,13 +145,20 @@ typedef struct {
  * are being fine-tuned (Section 3.3: an action fine-tunes the model of ONE endpoint's
  * subgraph; Algorithm 1, Stage 3 groups the actions per subgraph): weights and moments of
  * a subgraph with active[s] == 0 are left bit-for-bit unchanged.  It needs per-subgraph
- * weights (weight_sets == S); the bias correction uses `step` for every active subgraph. */
+ * weights (weight_sets == S); the bias correction uses `step` for every active subgraph.
+ * `step_dev` (device, one int32, or NULL): when given, `step` is ignored; the step reads the number of
+ * updates done so far from *step_dev, adds one and uses that.  Nothing in such a step then depends on a host
+ * value that changes from step to step, so a run of steps recorded once in a CUDA graph (stream capture of
+ * gnnco_train_step / gnnco_decode_boundary on the capturing stream; same buffers at every replay) can be
+ * replayed any number of times -- for graphs of a few thousand nodes, where a step is tens of launches of a few
+ * microseconds, that removes most of its cost. */
 typedef struct {
   float lr, beta1, beta2, eps;
   int64_t step;
   float* m[GNNCO_MAX_LAYERS];
   float* v[GNNCO_MAX_LAYERS];
   const uint8_t* active;
+  int32_t* step_dev;
 } gnnco_adam_state;
 
 /* Outputs of a training step.  loss and p are required; the rest may be NULL. */

@@ -56,7 +56,7 @@ class Objective(ctypes.Structure):
 
 class AdamState(ctypes.Structure):
     _fields_ = [("lr", _f32), ("beta1", _f32), ("beta2", _f32), ("eps", _f32), ("step", _i64),
-                ("m", _vp * MAX_LAYERS), ("v", _vp * MAX_LAYERS), ("active", _vp)]
+                ("m", _vp * MAX_LAYERS), ("v", _vp * MAX_LAYERS), ("active", _vp), ("step_dev", _vp)]
 
 
 class TrainOut(ctypes.Structure):
@@ -194,11 +194,15 @@ class Adam:
     """Adam moments and hyper-parameters (``gnnco_adam_state``); ``step`` is advanced by
     ``PartitionedGraph.train_step`` after each update."""
 
-    def __init__(self, model: Model, lr: float = 1e-3, beta1: float = 0.9, beta2: float = 0.999, eps: float = 1e-8):
+    def __init__(self, model: Model, lr: float = 1e-3, beta1: float = 0.9, beta2: float = 0.999, eps: float = 1e-8,
+                 device_step: bool = False):
         import torch
         self.lr, self.beta1, self.beta2, self.eps = lr, beta1, beta2, eps
         self.step = 1
         self.active = None          # uint8 [S] device tensor: subgraphs being fine-tuned (None = all)
+        # ``gnnco_adam_state.step_dev``: number of updates done so far, kept on the device (steps that use it can be
+        # recorded in a CUDA graph and replayed)
+        self.step_dev = torch.zeros(1, dtype=torch.int32, device=model.W[0].device) if device_step else None
         self.m = [torch.zeros_like(w) for w in model.W]
         self.v = [torch.zeros_like(w) for w in model.W]
 
@@ -209,6 +213,7 @@ class Adam:
             a.m[l] = self.m[l].data_ptr()
             a.v[l] = self.v[l].data_ptr()
         a.active = _dptr(self.active)
+        a.step_dev = _dptr(self.step_dev)
         return a
 
 

@@ -359,9 +359,14 @@ __global__ void cast_bf16x8_kernel(const float4* __restrict__ in, uint4* __restr
 
 __global__ void adam_kernel(float* __restrict__ W, float* __restrict__ m, float* __restrict__ v,
                             const float* __restrict__ g, int64_t count, float lr, float b1, float b2, float eps,
-                            float inv_c1, float inv_c2, const uint8_t* __restrict__ active, int64_t per_set) {
+                            float inv_c1, float inv_c2, const uint8_t* __restrict__ active, int64_t per_set,
+                            const float2* __restrict__ bias) {
   const int64_t q = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
   if (q >= count) return;
+  if (bias) {            // bias corrections kept on the device (a step counter there: adam_tick)
+    inv_c1 = bias->x;
+    inv_c2 = bias->y;
+  }
   if (active && !active[q / per_set]) return;   // this subgraph is not being fine-tuned
   const float gq = g[q];
   const float mq = b1 * m[q] + (1.0f - b1) * gq;
@@ -376,9 +381,13 @@ __global__ void __launch_bounds__(256) adam_vec4_kernel(float4* __restrict__ W, 
                                                         float4* __restrict__ v, const float4* __restrict__ g,
                                                         int64_t quads, float lr, float b1, float b2, float eps,
                                                         float inv_c1, float inv_c2, const uint8_t* __restrict__ active,
-                                                        int64_t quads_per_set) {
+                                                        int64_t quads_per_set, const float2* __restrict__ bias) {
   const int64_t q = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
   if (q >= quads) return;
+  if (bias) {
+    inv_c1 = bias->x;
+    inv_c2 = bias->y;
+  }
   if (active && !active[q / quads_per_set]) return;
   const float4 gq = __ldg(g + q);
   float4 mq = m[q], vq = v[q], wq = W[q];
@@ -559,6 +568,24 @@ int32_t launch_cast_bf16(gnnco_handle* h, const float* in, __nv_bfloat16* out, i
   return GNNCO_OK;
 }
 
+// One thread: the device-side step counter advances and the bias corrections of THIS update,
+// 1 / (1 - beta^t), are left where the Adam kernels of the step read them.
+__global__ void adam_tick(int32_t* __restrict__ step_dev, float b1, float b2, float2* __restrict__ bias) {
+  const int32_t t = *step_dev + 1;
+  *step_dev = t;
+  const float c1 = (float)(1.0 - pow((double)b1, (double)t));
+  const float c2 = (float)(1.0 - pow((double)b2, (double)t));
+  *bias = make_float2(1.0f / c1, 1.0f / c2);
+}
+
+int32_t launch_adam_tick(gnnco_handle* h, int32_t* step_dev, float b1, float b2, float2* bias, cudaStream_t stream) {
+  ProfScope prof_(h, K_ADAM, stream);
+  adam_tick<<<1, 1, 0, stream>>>(step_dev, b1, b2, bias);
+  h->launches += 1;
+  GNNCO_LAUNCH_CHECK();
+  return GNNCO_OK;
+}
+
 int32_t launch_adam(gnnco_handle* h, float* W, float* m, float* v, const float* g, int64_t count, float lr, float b1,
                     float b2, float eps, float c1, float c2, const uint8_t* active, int64_t per_set,
                     cudaStream_t stream) {
@@ -568,10 +595,11 @@ int32_t launch_adam(gnnco_handle* h, float* W, float* m, float* v, const float* 
   if (vec)
     adam_vec4_kernel<<<blocks_for(count / 4, 256), 256, 0, stream>>>(
         reinterpret_cast<float4*>(W), reinterpret_cast<float4*>(m), reinterpret_cast<float4*>(v),
-        reinterpret_cast<const float4*>(g), count / 4, lr, b1, b2, eps, 1.0f / c1, 1.0f / c2, active, per_set / 4);
+        reinterpret_cast<const float4*>(g), count / 4, lr, b1, b2, eps, 1.0f / c1, 1.0f / c2, active, per_set / 4,
+        h->adam_bias);
   else
     adam_kernel<<<blocks_for(count, 256), 256, 0, stream>>>(W, m, v, g, count, lr, b1, b2, eps, 1.0f / c1, 1.0f / c2,
-                                                          active, per_set);
+                                                          active, per_set, h->adam_bias);
   h->launches += 1;
   GNNCO_LAUNCH_CHECK();
   return GNNCO_OK;

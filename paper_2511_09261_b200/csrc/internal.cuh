@@ -161,6 +161,8 @@ struct gnnco_handle {
   cudaStream_t copy_stream = nullptr;
   cudaEvent_t ev_arrive[kArrivalGroups] = {}, ev_rest = nullptr, ev_begin = nullptr;
   const ArrivalPlan* arrival = nullptr;
+  // during a step whose Adam state keeps its step counter on the device: where adam_tick left 1 / (1 - beta^t)
+  const float2* adam_bias = nullptr;
   cudaEvent_t ev_fork = nullptr, ev_join = nullptr;
 };
 
@@ -273,6 +275,7 @@ int32_t launch_wg_combine(gnnco_handle* h, const float* scratch, float* dW, int6
 int32_t launch_sum_over_sets(gnnco_handle* h, const float* in, float* out, int64_t count, int32_t sets, cudaStream_t st);
 int32_t launch_cast_bf16(gnnco_handle* h, const float* in, __nv_bfloat16* out, int64_t count, cudaStream_t st);
 // active (or nullptr): one byte per run of `per_set` consecutive elements; runs with a zero byte are skipped
+int32_t launch_adam_tick(gnnco_handle* h, int32_t* step_dev, float b1, float b2, float2* bias, cudaStream_t st);
 int32_t launch_adam(gnnco_handle* h, float* W, float* m, float* v, const float* g, int64_t count, float lr, float b1,
                     float b2, float eps, float c1, float c2, const uint8_t* active, int64_t per_set, cudaStream_t st);
 

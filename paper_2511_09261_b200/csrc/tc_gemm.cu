@@ -510,8 +510,13 @@ __global__ void __launch_bounds__(256) adam_cast_both_kernel(float* __restrict__
                                                              __nv_bfloat16* __restrict__ Wc, __nv_bfloat16* __restrict__ Wt,
                                                              int K, int N, float lr, float b1, float b2, float eps,
                                                              float inv_c1, float inv_c2,
-                                                             const uint8_t* __restrict__ active) {
+                                                             const uint8_t* __restrict__ active,
+                                                             const float2* __restrict__ bias) {
   __shared__ float tile[64][65];
+  if (bias) {            // bias corrections kept on the device (a step counter there: adam_tick)
+    inv_c1 = bias->x;
+    inv_c2 = bias->y;
+  }
   const int64_t base = (int64_t)blockIdx.x * K * N;          // the set index is on x (no 65,535 limit there)
   const int k0 = blockIdx.y * 64, n0 = blockIdx.z * 64;
   const int q = threadIdx.x & 15, r = threadIdx.x >> 4;   // 16 threads of four elements across, 16 rows per pass
@@ -631,7 +636,7 @@ int32_t launch_adam_cast_both(gnnco_handle* h, float* W, float* m, float* v, con
   if (!adam_cast_both_supported(W, m, v, g, Wc, Wt, K, N, sets)) return GNNCO_UNSUPPORTED;
   ProfScope prof_(h, K_ADAM, st);
   adam_cast_both_kernel<<<dim3(sets, K / 64, N / 64), 256, 0, st>>>(W, m, v, g, Wc, Wt, K, N, lr, b1, b2, eps, 1.0f / c1,
-                                                                     1.0f / c2, active);
+                                                                     1.0f / c2, active, h->adam_bias);
   h->launches += 1;
   GNNCO_LAUNCH_CHECK();
   return GNNCO_OK;

@@ -31,6 +31,7 @@ struct TrainLayout {
   float* dW_scratch;                  // one layer's gradient (all sets), when the caller wants none
   float* dW_sets;                     // per-subgraph partials when the model shares one weight set
   float* wg_scratch;                  // partial weight gradients of subgraphs that were split into row chunks
+  float2* adam_bias;                  // 1 / (1 - beta^t) of this update when the step counter lives on the device
   float* agg_partial;                 // partial sums of the segments of long rows (aggregation)
   uint8_t* Hbits[GNNCO_MAX_LAYERS];   // [H_l > 0], one bit per element (bfloat16; written by the transform that makes H_l,
                                       // or, for the last hidden layer, by the output layer's weight gradient)
@@ -91,6 +92,7 @@ TrainLayout carve_train(const gnnco_handle* h, const gnnco_model_desc* m, uint32
     T.dW_scratch = c.take<float>(max_wcount * m->weight_sets);
     if (m->weight_sets == 1) T.dW_sets = c.take<float>(max_wcount * (size_t)h->S);
     T.wg_scratch = c.take<float>(max_wcount * (size_t)h->n_wg_slots + 1);
+    T.adam_bias = c.take<float2>(1);
   }
   if (m->feat_dtype == GNNCO_BF16)
     for (int l = 0; l < L; ++l)
@@ -163,6 +165,7 @@ int32_t run_step_on(gnnco_handle* h, const gnnco_model_desc* m, const void* X, c
   const int L = m->L, dt = m->feat_dtype;
   const bool bf16 = dt == GNNCO_BF16;
   h->agg_partial = T.agg_partial;       // where this step's aggregations keep the segments of long rows
+  h->adam_bias = nullptr;
   const int32_t sets = m->weight_sets;
   int32_t rc;
 #define GNNCO_TRY(call) do { rc = (call); if (rc != GNNCO_OK) return rc; } while (0)
@@ -299,7 +302,13 @@ int32_t run_step_on(gnnco_handle* h, const gnnco_model_desc* m, const void* X, c
   // coef = D^-1 g takes the place of u, which the forward pass is done with
   GNNCO_TRY(launch_output_backward(h, T.t, T.g, L > 1 ? T.u : nullptr, st));
   float c1 = 1.0f, c2 = 1.0f;
-  if (opt) {
+  h->adam_bias = nullptr;
+  if (opt && opt->step_dev) {
+    // step counter on the device: one thread advances it and leaves this update's bias corrections for the Adam
+    // kernels (nothing below then depends on a host value that changes from step to step)
+    GNNCO_TRY(launch_adam_tick(h, opt->step_dev, opt->beta1, opt->beta2, T.adam_bias, st));
+    h->adam_bias = T.adam_bias;
+  } else if (opt) {
     c1 = (float)(1.0 - pow((double)opt->beta1, (double)opt->step));
     c2 = (float)(1.0 - pow((double)opt->beta2, (double)opt->step));
   }

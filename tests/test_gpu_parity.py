@@ -314,6 +314,64 @@ def test_weight_copies_left_by_adam_are_bit_identical_to_fresh_ones():
         assert torch.equal(a, b)
 
 
+@pytest.mark.parametrize("cfg", [1, 3])
+def test_steps_replayed_from_a_cuda_graph_equal_eager_steps(cfg):
+    """With the Adam step counter on the device (gnnco_adam_state.step_dev) a step depends on no host value that
+    changes between steps: ONE step plus its decode, recorded once by stream capture, replayed five times, gives
+    the bits of five eager steps (loss, p, weights, moments, decode counts), and the counter reads 5.  The same
+    five eager steps with the counter on the host give those bits too."""
+    import torch
+    import paper_2511_09261_b200 as gnnco
+    w = si.make_workload(cfg)
+    graph = load_graph(w.n, w.eu, w.ev, w.part, w.S)
+    perm = graph.arrays()["perm"].cpu().numpy()
+    X = to_dev(w.features_f32()[perm])
+    pen = to_dev(w.penalty()[perm])
+    loss, p = torch.empty(w.S, device=X.device), torch.empty(w.n, device=X.device)
+    counts = torch.zeros(3, dtype=torch.int64, device=X.device)
+    x = torch.empty(w.n, dtype=torch.uint8, device=X.device)
+    viol = torch.empty(graph.E_b, dtype=torch.uint8, device=X.device)
+    per_part = torch.empty(w.S, dtype=torch.int32, device=X.device)
+
+    def fresh(device_step):
+        W = [to_dev(w.weights(l)) for l in range(w.L)]
+        model = gnnco.Model(w.dims, W)
+        return W, model, gnnco.Adam(model, lr=w.lr, device_step=device_step)
+
+    def one(model, opt, stream=None):
+        graph.train_step(model, X, w.alpha, w.beta, w.lam, pen, opt, loss=loss, p=p, stream=stream)
+        graph.decode_boundary(p, 0.5, x=x, viol=viol, per_part=per_part, counts=counts, stream=stream)
+
+    results = []
+    for mode in ("host counter", "device counter", "graph"):
+        W, model, opt = fresh(mode != "host counter")
+        if mode == "graph":
+            side = torch.cuda.Stream()
+            with torch.cuda.stream(side):
+                W0, model0, opt0 = fresh(True)
+                one(model0, opt0, side)                  # everything lazy happens outside the capture
+                torch.cuda.synchronize()
+                g = torch.cuda.CUDAGraph()
+                g.capture_begin()
+                one(model, opt, side)
+                g.capture_end()
+            torch.cuda.synchronize()
+            for _ in range(5):
+                g.replay()
+        else:
+            for _ in range(5):
+                one(model, opt)
+        torch.cuda.synchronize()
+        assert graph.async_status() == 0
+        if opt.step_dev is not None:
+            assert int(opt.step_dev.item()) == 5
+        results.append([loss.clone(), p.clone(), counts.clone()] + [t.clone() for t in W] + [t.clone() for t in opt.m] +
+                       [t.clone() for t in opt.v])
+    for other in results[1:]:
+        for a, b in zip(results[0], other):
+            assert torch.equal(a, b)
+
+
 def test_host_variant_matches_device_variant():
     import torch
     import paper_2511_09261_b200 as gnnco
