@@ -580,14 +580,14 @@ def run_ours(args):
 # names the source file of its kernel and that file's SHA-1 when the counters were taken: when the file has
 # changed since, the entry no longer describes the kernel and the bench reports null.
 TRAFFIC_BYTES = {
-    "transform_fwd": (10.46e9, "tc_gemm2.cu", "69db3cca4022"),
-    "transform_bwd": (10.61e9, "tc_gemm2.cu", "69db3cca4022"),
-    "weight_grad": (12.15e9, "tc_gemm.cu", "834b9463b12c"),
-    "aggregate_fwd": (10.00e9, "spmm.cu", "621aa0f900a3"),
-    "aggregate_bwd": (10.00e9, "spmm.cu", "621aa0f900a3"),
-    "aggregate_rank1": (6.09e9, "spmm.cu", "621aa0f900a3"),
-    "weight_grad_vec": (5.46e9, "dense.cu", "6104b880bc2f"),
-    "adam": (8.12e9, "tc_gemm.cu", "834b9463b12c"),
+    "transform_fwd": (10.55e9, "tc_gemm2.cu", "588387481e83"),
+    "transform_bwd": (10.60e9, "tc_gemm2.cu", "588387481e83"),
+    "weight_grad": (12.46e9, "tc_gemm2.cu", "588387481e83"),
+    "aggregate_fwd": (9.97e9, "spmm.cu", "37036d305236"),
+    "aggregate_bwd": (9.97e9, "spmm.cu", "37036d305236"),
+    "aggregate_rank1": (5.59e9, "spmm.cu", "37036d305236"),
+    "weight_grad_vec": (5.47e9, "dense.cu", "02948ea8f38d"),
+    "adam": (8.12e9, "tc_gemm.cu", "f6e2323bd7ca"),
 }
 
 
