@@ -229,3 +229,43 @@ def test_config4_full_size_sampled_subgraphs():
 
 def test_config5_full_size_sampled_subgraphs():
     _full_size_sampled(5, steps=5, n_parts=64)
+
+
+def test_config5_full_size_one_kernel_layers_against_the_plain_step():
+    """GNNCO_ONE_KERNEL_LAYERS at the full size of configuration 5 (every CTA pair walks hundreds of double
+    tiles of dozens of subgraphs; the tiles around the hubs go through the separate kernels): two training steps
+    with the flag against two plain steps, whose parity with the oracle the test above establishes.  Subgraphs
+    without a row of more than 256 neighbours must agree bit for bit in loss and p; the others (the plain step
+    sums such rows inline at this size, the flagged step by segments) within the bfloat16 bound."""
+    import torch
+    import paper_2511_09261_b200 as gnnco
+    from gpu_common import BF16_RTOL, BF16_ATOL
+    w = si.make_workload(5)
+    graph = load_graph(w.n, w.eu, w.ev, w.part, w.S)
+    arr = graph.arrays()
+    X_orig = torch.from_numpy(w.features_bf16_bits().view(np.int16)).to("cuda:0").view(torch.bfloat16)
+    Xd = graph.gather_rows(X_orig, arr["perm"])
+    del X_orig
+    runs = []
+    for extra in (0, gnnco.ONE_KERNEL_LAYERS):
+        Wd = [to_dev(w.weights(l)) for l in range(w.L)]
+        model = gnnco.Model(w.dims, Wd, gnnco.BF16)
+        opt = gnnco.Adam(model, lr=w.lr)
+        for _ in range(2):
+            loss, p = graph.train_step(model, Xd, w.alpha, w.beta, flags=extra, opt=opt)
+        torch.cuda.synchronize()
+        assert graph.async_status() == 0
+        runs.append((loss.clone(), p.clone()))
+        del Wd, model, opt
+    (loss_a, p_a), (loss_b, p_b) = runs
+    rowptr, part_ptr = arr["rowptr"].long(), arr["part_ptr"].long()
+    deg = rowptr[1:] - rowptr[:-1]
+    node_part = arr["node_part"].long()
+    long_parts = torch.zeros(w.S, dtype=torch.bool, device=deg.device)
+    long_parts[node_part[deg > 256]] = True
+    assert 0 < int(long_parts.sum()) < w.S // 4
+    short = ~long_parts
+    assert torch.equal(loss_a[short], loss_b[short])
+    assert torch.equal(p_a[short[node_part]], p_b[short[node_part]])
+    assert torch.allclose(p_a, p_b, rtol=BF16_RTOL, atol=BF16_ATOL)
+    assert torch.allclose(loss_a, loss_b, rtol=BF16_RTOL, atol=BF16_ATOL * float(loss_a.abs().max()))
