@@ -181,7 +181,9 @@ const char* gnnco_status_string(int32_t status);
 
 /* Sizes (bytes) of the two work areas of gnnco_partition_load for a graph of n nodes,
  * E edges and S subgraphs: `persistent` must outlive the handle, `scratch` may be
- * released when gnnco_partition_load returns. */
+ * released when gnnco_partition_load returns.  `persistent` is about 41 n + 24 E bytes: the node
+ * order, the CSR of the intra edges, the boundary list, a 16-byte head record per row, the per-row source list
+ * of GNNCO_ONE_KERNEL_LAYERS (4 (n + 2 E) bytes) and the tile tables. */
 int32_t gnnco_partition_workspace_bytes(int64_t n, int64_t E, int32_t S, size_t* persistent, size_t* scratch);
 
 /* Build the block-diagonal batch (Section 3.3: split into subgraphs; cross edges set
