@@ -117,7 +117,7 @@ __device__ __forceinline__ void accumulate(float (&acc)[Vec<T>::N], const uint4&
 }
 
 // LPR lanes per row, VPL vectors per lane: row width F = LPR * VPL * Vec<T>::N elements.
-// Threads per block of the row-per-warp aggregation.  Measured on B200 (width 256, bfloat16, same-box A/B): 128
+// Threads per block of the row-per-warp aggregation.  Measured on B200 (width 256, bfloat16, alternating runs on one device): 128
 // threads 1.95-1.97 ms, 256 threads 1.99-2.01 ms, 64 threads 2.81-2.85 ms per launch of 10 M rows.
 constexpr int kAggThreads = 128;
 
