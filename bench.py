@@ -370,6 +370,11 @@ def run_ours(args):
                     traffic=measured_traffic(args, top),
                     peak_source="%s (MEASURED_PEAKS.json hbm_gbs)" % peak_src if peak_src == "measured" else "fallback",
                     algorithmic_bytes_per_launch=algorithmic_bytes(top, w, w.n, nnz, w.S))
+    if roofline["traffic"]:
+        # the same fraction on the DRAM bytes that ncu counted for this kernel (below the algorithmic figure where
+        # gathered rows were still in L2)
+        per_ms = prof[top][1] / prof[top][0]
+        roofline["frac_on_measured_traffic"] = round(roofline["traffic"] / (per_ms * 1e-3) / 1e9 / peak, 4)
     agg = {k: kern[k] for k in ("aggregate_fwd", "aggregate_bwd", "aggregate_rank1") if k in kern}
     # the neighbour aggregation forward + backward as one figure (all its launches of the timed steps)
     agg_bytes = sum(algorithmic_bytes(k, w, w.n, nnz, w.S) * prof[k][0] for k in agg)
