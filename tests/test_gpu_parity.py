@@ -32,6 +32,7 @@ GRAPHS = {
     "huge_hub": lambda: _star_plus_isolated(9000) + (np.zeros(9000, np.int32),),   # hub row of 4499 entries (block-summed)
     "no_edges": lambda: (np.zeros(0, np.int32), np.zeros(0, np.int32), si.contiguous_partition(50, 4)),
     "dense_small": lambda: tiny_graph(90, 0.5, 2, seed=8, contiguous=True),
+    "dense_medium": lambda: tiny_graph(400, 0.5, 2, seed=9, contiguous=True),    # every row has about 100 neighbours
 }
 
 
@@ -267,7 +268,8 @@ def test_one_kernel_layers_equal_the_separate_kernels_bit_for_bit(dims, n, S):
 
 
 @pytest.mark.parametrize("graph_name,dims", [("big_hub", [256, 256, 1]), ("big_hub", [256, 256, 256, 1]),
-                                             ("dense_small", [256, 256, 256, 1]), ("empty_parts", [256, 256, 1]), ("no_edges", [256, 256, 1])])
+                                             ("dense_small", [256, 256, 256, 1]), ("dense_medium", [256, 256, 1]), ("empty_parts", [256, 256, 1]),
+                                             ("no_edges", [256, 256, 1])])
 def test_one_kernel_layers_against_the_oracle(graph_name, dims):
     """The same flag on graphs with a hub row (its double tile goes through the separate kernels, the others
     through the one-kernel layer) and on a small dense-ish graph, against the oracle."""
