@@ -588,9 +588,9 @@ TRAFFIC_BYTES = {
     "transform_fwd": (10.55e9, "tc_gemm2.cu", "588387481e83"),
     "transform_bwd": (10.60e9, "tc_gemm2.cu", "588387481e83"),
     "weight_grad": (12.46e9, "tc_gemm2.cu", "588387481e83"),
-    "aggregate_fwd": (9.97e9, "spmm.cu", "c6164606526d"),
-    "aggregate_bwd": (9.97e9, "spmm.cu", "c6164606526d"),
-    "aggregate_rank1": (5.59e9, "spmm.cu", "c6164606526d"),
+    "aggregate_fwd": (9.98e9, "spmm.cu", "cb0acadd0a6d"),
+    "aggregate_bwd": (9.98e9, "spmm.cu", "cb0acadd0a6d"),
+    "aggregate_rank1": (5.59e9, "spmm.cu", "cb0acadd0a6d"),
     "weight_grad_vec": (5.47e9, "dense.cu", "02948ea8f38d"),
     "adam": (8.12e9, "tc_gemm.cu", "f6e2323bd7ca"),
 }
